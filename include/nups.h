@@ -1,0 +1,251 @@
+/*
+ * nups.h - C ABI of a single-GPU parameter store with non-uniform (skew-aware)
+ * parameter access, after NuPS (arXiv 2104.00501).
+ *
+ * The store keeps one fp32 value row per key in device memory (optionally a
+ * second "accumulator" row for AdaGrad), serves pull (row gather) and push
+ * (additive scatter) by key, manages hot keys by replication and the rest in
+ * place, and draws sampling accesses inside the store under the paper's four
+ * conformity levels.
+ *
+ * Conventions for every call below
+ *   - `nups_store*` is an opaque host object owned by the library.
+ *   - Arguments named d_* are DEVICE pointers owned by the caller; the library
+ *     reads or writes them only in stream order of the call and keeps no
+ *     reference afterwards.  Arguments named h_* are HOST pointers.  Everything
+ *     else is passed by value.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls enqueue work on it and return; results are ready when the stream
+ *     reaches that point.  Calls that return a value through an h_* pointer
+ *     synchronise the stream first and say so.
+ *   - Keys are uint32 in [0, num_keys).  A key outside the range is never
+ *     dereferenced: the access is skipped (a pulled row is zero-filled) and the
+ *     device status word is set to NUPS_EKEY; nups_status_check reports it.
+ *   - Rows hold `value_len` floats, contiguous; value_len must be a multiple of
+ *     4 so that every row starts on a 16-byte boundary.
+ *   - Item i of a call over n items belongs to logical worker
+ *     q(i) = floor(i * workers / n) (contiguous chunks).  Workers stand for the
+ *     paper's nodes: each has its own replica of every replicated key and its
+ *     own sample stream.
+ *   - Return value: NUPS_OK or a negative nups_status.  Host-detectable errors
+ *     are returned at once and enqueue nothing.
+ *   - The library's calls on one store are not thread-safe.
+ */
+#ifndef NUPS_H
+#define NUPS_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct nups_store nups_store;
+typedef int64_t nups_handle;
+typedef int32_t nups_status;
+
+enum {
+    NUPS_OK = 0,
+    NUPS_EINVAL = -1,  /* bad argument                                              */
+    NUPS_ENOMEM = -2,  /* device or host allocation failed, or a table is full       */
+    NUPS_ECUDA = -3,   /* a CUDA runtime call failed; see nups_last_cuda_error       */
+    NUPS_EKEY = -4,    /* a key >= num_keys was seen on the device (access skipped)  */
+    NUPS_ESTATE = -5,  /* over-pull of a handle, level needs ownership tracking, ... */
+    NUPS_ETIMEOUT = -6 /* a bounded device-side wait gave up                         */
+};
+enum { NUPS_SINGLE = 0, NUPS_REPLICATE = 1 };
+enum { NUPS_CONFORM = 1, NUPS_BOUNDED = 2, NUPS_LONGTERM = 3, NUPS_NONCONFORM = 4 };
+
+/* Creation-time settings.  Zero-initialise, then set what differs; a NULL config
+ * means all defaults.                                                           */
+typedef struct nups_config {
+    uint32_t workers;         /* R logical workers, 1..254; 0 = default 8                     */
+    uint32_t sync_interval;   /* nups_step_* merges replicas every this many steps;           */
+                              /* 0 = never automatically                                      */
+    uint32_t deterministic;   /* 1: pushes are applied in item order per destination row      */
+                              /*    (sort + ordered reduction; reproducible);                 */
+                              /* 0: atomic adds in any order (fast)                           */
+    uint32_t with_adagrad;    /* 1: allocate the accumulator table                            */
+    uint32_t count_accesses;  /* 1: every pulled, pushed or sampled key adds 1 to its count   */
+    uint32_t track_ownership; /* 1: keep the key -> owning worker map that LONG-TERM and      */
+                              /*    NON-CONFORM sampling need                                 */
+    uint32_t smem_hot_rows;   /* fast mode: hot slots below this number are accumulated in    */
+                              /*    shared memory inside a kernel before reaching the         */
+                              /*    worker's replica; 0 = library default                     */
+    uint32_t reserved[9];
+} nups_config;
+
+/* ---- store (Section 3.1: keys, pull, push) -------------------------------- */
+
+/* Allocate a store of num_keys rows of value_len floats, zero-filled, no key
+ * replicated.  *h_out receives the store.  NUPS_EINVAL: num_keys == 0 or
+ * > 2^32-1, value_len == 0 or not a multiple of 4, workers > 254.             */
+nups_status nups_create(uint64_t num_keys, uint32_t value_len, const nups_config* h_cfg, nups_store** h_out);
+
+/* Free everything the store owns.  Synchronises the device.                   */
+nups_status nups_destroy(nups_store* store);
+
+/* Device pointer of the value (which = 0) or accumulator (which = 1) table,
+ * row-major [num_keys][row_stride_floats].  The caller may read or write it in
+ * stream order (e.g. to load start values); rows of replicated keys do not
+ * include updates that are still pending in replicas.                         */
+nups_status nups_table_ptr(nups_store* store, int which, float** h_ptr, uint64_t* h_row_stride_floats);
+
+/* Fill a table with seeded start values: element e gets
+ * (int(bits 8..31 of word e mod 4 of Philox4x32-10(counter = (e/4, 0, which, 3),
+ *  key = seed)) - 2^23) * (scale * 2^-23), uniform in [-scale, scale).         */
+nups_status nups_init_uniform(nups_store* store, int which, uint64_t seed, float scale, void* stream);
+
+/* pull (Section 3.1): d_out[i][:] = current value of d_keys[i] as worker q(i)
+ * sees it: the stored row, plus the worker's own pending replica updates when
+ * the key is replicated (Section 3.2).  d_out is [n][value_len].
+ * nups_pull2 also returns the accumulator rows (either output may be NULL).   */
+nups_status nups_pull(nups_store* store, const uint32_t* d_keys, uint64_t n, float* d_out, void* stream);
+nups_status nups_pull2(nups_store* store, const uint32_t* d_keys, uint64_t n, float* d_out_val, float* d_out_acc,
+                       void* stream);
+
+/* push (Section 3.1; replica accumulation Section 3.1.2): add d_delta[i][:] to
+ * the row of d_keys[i], every duplicate applied.  Updates to a replicated key
+ * go to worker q(i)'s replica and reach the stored row at the next nups_sync.
+ * deterministic = 1: per destination row the deltas are added one by one in
+ * ascending i.  nups_push2 updates both tables from one call (AdaGrad state
+ * lives beside the value, Section 5.1 / Table 2); either delta may be NULL.   */
+nups_status nups_push(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta, void* stream);
+nups_status nups_push2(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta_val,
+                       const float* d_delta_acc, void* stream);
+
+/* ---- per-key management (Section 3.2, Section 5.1) ------------------------ */
+
+/* Set the technique of the listed keys.  Pending replica updates are merged
+ * first.  NUPS_REPLICATE appends every listed key that is not replicated yet as
+ * a new hot slot, in list order (first occurrence); NUPS_SINGLE removes the
+ * listed keys and renumbers the remaining slots in their old order.  May
+ * allocate; synchronises the stream.                                          */
+nups_status nups_set_management(nups_store* store, const uint32_t* d_keys, uint64_t n, int technique, void* stream);
+
+/* sync (Section 3.2: periodic sparse all-reduce of replica updates): for every
+ * hot slot touched since the last sync add the workers' pending updates, worker
+ * 0 first, to the stored row and clear them.  With no replicated key nothing is
+ * launched.                                                                   */
+nups_status nups_sync(nups_store* store, void* stream);
+
+/* Add 1 to the access count of every key of the stream (dataset frequency
+ * statistics, Section 5.1).                                                   */
+nups_status nups_count_accesses(nups_store* store, const uint32_t* d_keys, uint64_t n, void* stream);
+
+/* Copy the num_keys access counts to d_counts_out.                            */
+nups_status nups_get_counts(nups_store* store, uint64_t* d_counts_out, void* stream);
+
+/* Choose hot keys from the access counts (Section 5.1).  by_topk = 0: keys with
+ * count * num_keys > param * (sum of counts), i.e. more than `param` times the
+ * mean (the paper's heuristic uses 100).  by_topk = 1: the `param` most frequent
+ * keys.  Output order: count descending, smaller key first among equals.
+ * d_keys_out must hold min(param, num_keys) keys for by_topk = 1 and num_keys
+ * for the threshold rule; *h_n_out receives the number written.  Counts must be
+ * below 2^32 (NUPS_ESTATE otherwise).  Synchronises the stream.               */
+nups_status nups_select_hot(nups_store* store, int by_topk, uint64_t param, uint32_t* d_keys_out, uint64_t* h_n_out,
+                            void* stream);
+
+/* Number of replicated keys, and their keys in slot order (d_keys_out may be
+ * NULL).  Synchronises the stream when d_keys_out is given.                   */
+nups_status nups_get_hot(nups_store* store, uint64_t* h_n_out, uint32_t* d_keys_out, void* stream);
+
+/* Move the listed keys to the worker of their item (the paper's localize,
+ * Section 3.1.3); when a key is listed more than once the last item wins.
+ * Replicated keys are unaffected.  No-op unless track_ownership.              */
+nups_status nups_localize(nups_store* store, const uint32_t* d_keys, uint64_t n, void* stream);
+
+/* Owning worker of each listed key into d_owner_out (int32): the worker, or -2
+ * for a replicated key, -1 for a key out of range, -3 if ownership is not
+ * tracked.                                                                    */
+nups_status nups_get_owner(nups_store* store, const uint32_t* d_keys, uint64_t n, int32_t* d_owner_out, void* stream);
+
+/* ---- sampling access (Sections 4.3, 4.4) ---------------------------------- */
+
+/* register_distribution(pi, level): pi lives on keys [key_base, key_base + n);
+ * d_weights[j] is the integer weight of key_base + j, NULL = uniform.  level is
+ * one of NUPS_CONFORM .. NUPS_NONCONFORM; U (use frequency) and G (pool size)
+ * are used by NUPS_BOUNDED and NUPS_LONGTERM.  Builds the alias table on the
+ * device.  Requires n * sum(weights) < 2^64 and G <= 1024.  *h_dist_out receives
+ * the distribution id.  Synchronises the stream.                              */
+nups_status nups_register_distribution(nups_store* store, uint32_t key_base, const uint32_t* d_weights, uint64_t n,
+                                       int level, uint32_t U, uint32_t G, uint64_t seed, int32_t* h_dist_out,
+                                       void* stream);
+
+/* Copy a distribution's alias table (thresholds, aliases; n entries each) and
+ * return the total weight; for checking a build.                              */
+nups_status nups_get_alias_table(nups_store* store, int32_t dist, uint64_t* d_thr_out, uint32_t* d_alias_out,
+                                 uint64_t* h_total_weight_out, void* stream);
+
+/* handle = PrepareSample(dist, N): reserve the next N samples.  The N output
+ * positions are cut into `workers` contiguous sub-handles; sub-handle q takes
+ * the next stretch of worker q's sample stream and (except under NON-CONFORM)
+ * localizes its keys to worker q.  Returns without waiting for the device.    */
+nups_status nups_prepare_sample(nups_store* store, int32_t dist, uint64_t N, nups_handle* h_out, void* stream);
+
+/* keys, values = PullSample(handle, n): the next n keys of the handle into
+ * d_keys_out and, if d_vals_out is not NULL, their rows [n][value_len] as the
+ * sub-handle's worker pulls them.  Partial pulls may be of any sizes that add
+ * up to N; the handle is released by the pull that completes it.  NUPS_ESTATE
+ * when n exceeds what is left.
+ *   CONFORM     independent draws from pi.
+ *   BOUNDED     pools of G draws, each walked U times in a fresh random order.
+ *   LONG-TERM   as BOUNDED, but a sample whose key is not local to the worker
+ *               at the start of the call is re-localized and postponed to the
+ *               end of its sub-handle, at most once.
+ *   NON-CONFORM the first key local to the worker at or after an independent
+ *               candidate (64 probes, then the candidate itself).             */
+nups_status nups_pull_sample(nups_store* store, nups_handle handle, uint64_t n, uint32_t* d_keys_out,
+                             float* d_vals_out, void* stream);
+
+/* ---- workload steps (Section 5.1) ----------------------------------------- */
+/* One step over a batch of n items: draw the negatives (one handle of n*K
+ * samples from `dist`; item i uses samples i*K .. i*K+K-1), pull, compute, push,
+ * localize the item's direct keys to its worker, and merge replicas every
+ * sync_interval steps.  deterministic = 1: all pulls see the values from before
+ * the step, pushes are applied in item order.  Otherwise items race.
+ * d_loss_out (nullable) receives the mean loss over the batch as one float.   */
+
+/* Skip-gram with negative sampling: centre key c, context key o, negatives u_j:
+ * x_j = v.u_j, g_j = sigmoid(x_j) - [j = 0], u_j -= lr g_j v, v -= lr sum g_j u_j,
+ * loss = -log sigmoid(x_0) - sum_j log sigmoid(-x_j); scores clamped to +-30.  */
+nups_status nups_step_sgns(nups_store* store, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_pairs,
+                           int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream);
+
+/* ComplEx with AdaGrad: rows are [re | im]; phi = Re sum h r conj(t); negative j
+ * replaces the head when j is even, the tail when odd;
+ * loss = softplus(-phi_pos) + sum_j softplus(phi_j); per key role with summed
+ * gradient g: acc += g^2, val -= lr g / (sqrt(acc_pulled + g^2) + eps).
+ * Needs with_adagrad and an even value_len.                                   */
+nups_status nups_step_complex(nups_store* store, const uint32_t* d_h, const uint32_t* d_r, const uint32_t* d_t,
+                              uint64_t n, int32_t dist, uint32_t K, float lr, float eps, float* d_loss_out,
+                              void* stream);
+
+/* Matrix factorization by SGD: e = x - w.h, w += lr (e h - l2 w),
+ * h += lr (e w - l2 h), loss = mean e^2.                                      */
+nups_status nups_step_mf(nups_store* store, const uint32_t* d_row, const uint32_t* d_col, const float* d_x, uint64_t n,
+                         float lr, float l2, float* d_loss_out, void* stream);
+
+/* Keys drawn as negatives by the most recent step ([n * K], library-owned
+ * device memory, valid until the next step).                                  */
+nups_status nups_last_negatives(nups_store* store, const uint32_t** h_d_keys_out, uint64_t* h_n_out);
+
+/* ---- status and statistics ------------------------------------------------ */
+
+/* Read and clear the device status word (synchronises the stream): NUPS_OK,
+ * NUPS_EKEY or NUPS_ETIMEOUT.                                                 */
+nups_status nups_status_check(nups_store* store, void* stream);
+
+/* h_out[0..7]: steps, syncs launched, kernels launched by the library so far,
+ * accesses served from replicas, accesses served in place, hot slots, 0, 0.
+ * The two access counters are only kept when count_accesses is set.
+ * Synchronises the stream.                                                    */
+nups_status nups_get_stats(nups_store* store, uint64_t* h_out, void* stream);
+
+const char* nups_strerror(nups_status status);
+const char* nups_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NUPS_H */

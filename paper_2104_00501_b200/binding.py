@@ -1,0 +1,314 @@
+"""Thin ctypes binding of ``libnups.so``: argument marshalling only.
+
+Every method maps to the C-ABI call of the same name in ``include/nups.h``; tensors are
+torch CUDA tensors used purely as device memory, and the current torch stream is passed
+as the call's stream.  There is no CPU fallback: loading fails loudly when the library
+is missing or cannot be built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libnups.so")
+
+OK, EINVAL, ENOMEM, ECUDA, EKEY, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
+SINGLE, REPLICATE = 0, 1
+CONFORM, BOUNDED, LONGTERM, NONCONFORM = 1, 2, 3, 4
+
+EXPORTS = [
+    "nups_create", "nups_destroy", "nups_table_ptr", "nups_init_uniform", "nups_pull", "nups_pull2", "nups_push",
+    "nups_push2", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
+    "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
+    "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_step_complex", "nups_step_mf",
+    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_strerror", "nups_last_cuda_error",
+]
+
+
+class Config(C.Structure):
+    _fields_ = [("workers", C.c_uint32), ("sync_interval", C.c_uint32), ("deterministic", C.c_uint32),
+                ("with_adagrad", C.c_uint32), ("count_accesses", C.c_uint32), ("track_ownership", C.c_uint32),
+                ("smem_hot_rows", C.c_uint32), ("reserved", C.c_uint32 * 9)]
+
+
+class NupsError(RuntimeError):
+    def __init__(self, code, what, detail=""):
+        super().__init__(f"{what}: status {code} ({detail})")
+        self.code = code
+
+
+_lib = None
+
+
+def load(build_if_missing: bool = True):
+    """Load libnups.so (building it with nvcc first when it is absent or stale)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if build_if_missing:
+        from . import build as _build
+        try:
+            _build.build_library()
+        except Exception:
+            if not os.path.exists(LIB_PATH):
+                raise
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2104_00501_b200.build`")
+    L = C.CDLL(LIB_PATH)
+    vp, u64, u32, i32, f32 = C.c_void_p, C.c_uint64, C.c_uint32, C.c_int32, C.c_float
+    sig = {
+        "nups_create": [u64, u32, C.POINTER(Config), C.POINTER(vp)],
+        "nups_destroy": [vp],
+        "nups_table_ptr": [vp, C.c_int, C.POINTER(vp), C.POINTER(u64)],
+        "nups_init_uniform": [vp, C.c_int, u64, f32, vp],
+        "nups_pull": [vp, vp, u64, vp, vp],
+        "nups_pull2": [vp, vp, u64, vp, vp, vp],
+        "nups_push": [vp, vp, u64, vp, vp],
+        "nups_push2": [vp, vp, u64, vp, vp, vp],
+        "nups_set_management": [vp, vp, u64, C.c_int, vp],
+        "nups_sync": [vp, vp],
+        "nups_count_accesses": [vp, vp, u64, vp],
+        "nups_get_counts": [vp, vp, vp],
+        "nups_select_hot": [vp, C.c_int, u64, vp, C.POINTER(u64), vp],
+        "nups_get_hot": [vp, C.POINTER(u64), vp, vp],
+        "nups_localize": [vp, vp, u64, vp],
+        "nups_get_owner": [vp, vp, u64, vp, vp],
+        "nups_register_distribution": [vp, u32, vp, u64, C.c_int, u32, u32, u64, C.POINTER(i32), vp],
+        "nups_get_alias_table": [vp, i32, vp, vp, C.POINTER(u64), vp],
+        "nups_prepare_sample": [vp, i32, u64, C.POINTER(C.c_int64), vp],
+        "nups_pull_sample": [vp, C.c_int64, u64, vp, vp, vp],
+        "nups_step_sgns": [vp, vp, vp, u64, i32, u32, f32, vp, vp],
+        "nups_step_complex": [vp, vp, vp, vp, u64, i32, u32, f32, f32, vp, vp],
+        "nups_step_mf": [vp, vp, vp, vp, u64, f32, f32, vp, vp],
+        "nups_last_negatives": [vp, C.POINTER(vp), C.POINTER(u64)],
+        "nups_status_check": [vp, vp],
+        "nups_get_stats": [vp, C.POINTER(u64), vp],
+    }
+    for name, args in sig.items():
+        fn = getattr(L, name)
+        fn.restype, fn.argtypes = C.c_int32, args
+    L.nups_strerror.restype, L.nups_strerror.argtypes = C.c_char_p, [C.c_int32]
+    L.nups_last_cuda_error.restype, L.nups_last_cuda_error.argtypes = C.c_char_p, []
+    _lib = L
+    return L
+
+
+def _ptr(t, dtype=None):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "device tensors must be contiguous CUDA tensors"
+    if dtype is not None:
+        assert t.dtype == dtype, f"expected {dtype}, got {t.dtype}"
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def as_keys(t) -> torch.Tensor:
+    """Keys as the library wants them: contiguous CUDA int32 tensor holding uint32 bit patterns."""
+    if not torch.is_tensor(t):
+        t = torch.as_tensor(t)
+    if t.dtype != torch.int32:
+        t = t.to(torch.int64).cuda()
+        t = torch.where(t >= 2 ** 31, t - 2 ** 32, t).to(torch.int32)
+    return t.cuda().contiguous()
+
+
+class Store:
+    """One parameter store on the current CUDA device."""
+
+    def __init__(self, num_keys, value_len, workers=8, sync_interval=1, deterministic=False, with_adagrad=False,
+                 count_accesses=False, track_ownership=False, smem_hot_rows=0):
+        self._l = load()
+        cfg = Config(workers=workers, sync_interval=sync_interval, deterministic=int(deterministic),
+                     with_adagrad=int(with_adagrad), count_accesses=int(count_accesses),
+                     track_ownership=int(track_ownership), smem_hot_rows=smem_hot_rows)
+        h = C.c_void_p()
+        self._s = None
+        self._chk(self._l.nups_create(num_keys, value_len, C.byref(cfg), C.byref(h)), "nups_create")
+        self._s = h
+        self.num_keys, self.L, self.R = int(num_keys), int(value_len), int(workers)
+        self.with_adagrad = bool(with_adagrad)
+        self.device = torch.device("cuda", torch.cuda.current_device())
+
+    def _chk(self, code, what):
+        if code != OK:
+            detail = self._l.nups_strerror(code).decode()
+            if code == ECUDA:
+                detail += ": " + self._l.nups_last_cuda_error().decode()
+            raise NupsError(code, what, detail)
+
+    def close(self):
+        if self._s:
+            self._l.nups_destroy(self._s)
+            self._s = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- tables -------------------------------------------------------------------------
+    def table_ptr(self, which=0):
+        p, stride = C.c_void_p(), C.c_uint64()
+        self._chk(self._l.nups_table_ptr(self._s, which, C.byref(p), C.byref(stride)), "nups_table_ptr")
+        return p.value, stride.value
+
+    def write_table(self, which, values):
+        """Copy host (or device) values [num_keys, L] into a table."""
+        p, _ = self.table_ptr(which)
+        src = torch.as_tensor(values, dtype=torch.float32).contiguous()
+        assert src.shape == (self.num_keys, self.L)
+        src = src.cuda()
+        torch.cuda.current_stream().synchronize()
+        rc = torch.cuda.cudart().cudaMemcpy(p, src.data_ptr(), src.numel() * 4, 3)   # 3 = device to device
+        assert int(rc) == 0
+
+    def read_table(self, which=0, rows=None):
+        """Copy a table (or the given rows of it) out to a new CUDA tensor."""
+        p, _ = self.table_ptr(which)
+        out = torch.empty((self.num_keys, self.L), dtype=torch.float32, device=self.device)
+        torch.cuda.current_stream().synchronize()
+        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), p, out.numel() * 4, 3)
+        assert int(rc) == 0
+        return out if rows is None else out[rows]
+
+    def init_uniform(self, which, seed, scale):
+        self._chk(self._l.nups_init_uniform(self._s, which, seed, scale, _stream()), "nups_init_uniform")
+
+    # -- direct access ------------------------------------------------------------------
+    def pull(self, keys, out=None, with_acc=False, out_acc=None):
+        n = keys.numel()
+        if out is None:
+            out = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+        if with_acc:
+            if out_acc is None:
+                out_acc = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+            self._chk(self._l.nups_pull2(self._s, _ptr(keys, torch.int32), n, _ptr(out), _ptr(out_acc), _stream()),
+                      "nups_pull2")
+            return out, out_acc
+        self._chk(self._l.nups_pull(self._s, _ptr(keys, torch.int32), n, _ptr(out), _stream()), "nups_pull")
+        return out
+
+    def push(self, keys, delta, delta_acc=None):
+        n = keys.numel()
+        assert delta is None or (delta.dtype == torch.float32 and delta.numel() == n * self.L)
+        if delta_acc is None:
+            self._chk(self._l.nups_push(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _stream()), "nups_push")
+        else:
+            assert delta_acc.dtype == torch.float32 and delta_acc.numel() == n * self.L
+            self._chk(self._l.nups_push2(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _ptr(delta_acc), _stream()),
+                      "nups_push2")
+
+    def sync(self):
+        self._chk(self._l.nups_sync(self._s, _stream()), "nups_sync")
+
+    # -- management ---------------------------------------------------------------------
+    def set_management(self, keys, technique):
+        self._chk(self._l.nups_set_management(self._s, _ptr(keys, torch.int32), keys.numel(), technique, _stream()),
+                  "nups_set_management")
+
+    def count_accesses(self, keys):
+        self._chk(self._l.nups_count_accesses(self._s, _ptr(keys, torch.int32), keys.numel(), _stream()),
+                  "nups_count_accesses")
+
+    def counts(self):
+        out = torch.empty(self.num_keys, dtype=torch.int64, device=self.device)
+        self._chk(self._l.nups_get_counts(self._s, _ptr(out), _stream()), "nups_get_counts")
+        return out
+
+    def select_hot(self, by_topk, param):
+        cap = min(int(param), self.num_keys) if by_topk else self.num_keys
+        out = torch.empty(max(cap, 1), dtype=torch.int32, device=self.device)
+        m = C.c_uint64()
+        self._chk(self._l.nups_select_hot(self._s, int(by_topk), int(param), _ptr(out), C.byref(m), _stream()),
+                  "nups_select_hot")
+        return out[:m.value]
+
+    def hot_keys(self):
+        m = C.c_uint64()
+        self._chk(self._l.nups_get_hot(self._s, C.byref(m), None, _stream()), "nups_get_hot")
+        out = torch.empty(max(m.value, 1), dtype=torch.int32, device=self.device)
+        if m.value:
+            self._chk(self._l.nups_get_hot(self._s, C.byref(m), _ptr(out), _stream()), "nups_get_hot")
+        return out[:m.value]
+
+    def localize(self, keys):
+        self._chk(self._l.nups_localize(self._s, _ptr(keys, torch.int32), keys.numel(), _stream()), "nups_localize")
+
+    def owner_of(self, keys):
+        out = torch.empty(keys.numel(), dtype=torch.int32, device=self.device)
+        self._chk(self._l.nups_get_owner(self._s, _ptr(keys, torch.int32), keys.numel(), _ptr(out), _stream()),
+                  "nups_get_owner")
+        return out
+
+    # -- sampling -----------------------------------------------------------------------
+    def register_distribution(self, key_base, weights, n, level, U=16, G=250, seed=0):
+        d = C.c_int32()
+        if weights is not None:
+            assert weights.numel() == n
+        self._chk(self._l.nups_register_distribution(self._s, key_base, _ptr(weights, torch.int32), n, level, U, G,
+                                                     seed, C.byref(d), _stream()), "nups_register_distribution")
+        return d.value
+
+    def alias_table(self, dist, n):
+        thr = torch.empty(n, dtype=torch.int64, device=self.device)
+        alias = torch.empty(n, dtype=torch.int32, device=self.device)
+        W = C.c_uint64()
+        self._chk(self._l.nups_get_alias_table(self._s, dist, _ptr(thr), _ptr(alias), C.byref(W), _stream()),
+                  "nups_get_alias_table")
+        return W.value, thr, alias
+
+    def prepare_sample(self, dist, N):
+        h = C.c_int64()
+        self._chk(self._l.nups_prepare_sample(self._s, dist, N, C.byref(h), _stream()), "nups_prepare_sample")
+        return h.value
+
+    def pull_sample(self, handle, n, values=True, keys_out=None, vals_out=None):
+        if keys_out is None:
+            keys_out = torch.empty(n, dtype=torch.int32, device=self.device)
+        if values and vals_out is None:
+            vals_out = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+        self._chk(self._l.nups_pull_sample(self._s, handle, n, _ptr(keys_out), _ptr(vals_out) if values else None,
+                                           _stream()), "nups_pull_sample")
+        return (keys_out, vals_out) if values else keys_out
+
+    # -- workload steps -----------------------------------------------------------------
+    def step_sgns(self, center, context, dist, K, lr, loss_out=None):
+        self._chk(self._l.nups_step_sgns(self._s, _ptr(center, torch.int32), _ptr(context, torch.int32),
+                                         center.numel(), dist, K, lr, _ptr(loss_out), _stream()), "nups_step_sgns")
+
+    def step_complex(self, h, r, t, dist, K, lr, eps, loss_out=None):
+        self._chk(self._l.nups_step_complex(self._s, _ptr(h, torch.int32), _ptr(r, torch.int32), _ptr(t, torch.int32),
+                                            h.numel(), dist, K, lr, eps, _ptr(loss_out), _stream()),
+                  "nups_step_complex")
+
+    def step_mf(self, rows, cols, x, lr, l2, loss_out=None):
+        self._chk(self._l.nups_step_mf(self._s, _ptr(rows, torch.int32), _ptr(cols, torch.int32),
+                                       _ptr(x, torch.float32), rows.numel(), lr, l2, _ptr(loss_out), _stream()),
+                  "nups_step_mf")
+
+    def last_negatives(self):
+        p, n = C.c_void_p(), C.c_uint64()
+        self._chk(self._l.nups_last_negatives(self._s, C.byref(p), C.byref(n)), "nups_last_negatives")
+        out = torch.empty(max(n.value, 1), dtype=torch.int32, device=self.device)
+        if n.value:
+            torch.cuda.current_stream().synchronize()
+            rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), p.value, n.value * 4, 3)
+            assert int(rc) == 0
+        return out[:n.value]
+
+    # -- status -------------------------------------------------------------------------
+    def status_check(self):
+        return self._l.nups_status_check(self._s, _stream())
+
+    def stats(self):
+        out = (C.c_uint64 * 8)()
+        self._chk(self._l.nups_get_stats(self._s, out, _stream()), "nups_get_stats")
+        return dict(steps=out[0], syncs=out[1], launches=out[2], hot=out[3], cold=out[4], hot_slots=out[5])

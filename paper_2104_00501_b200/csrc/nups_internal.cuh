@@ -1,0 +1,252 @@
+// Internal declarations shared by the translation units of libnups.so.
+// Device helpers are inline; nothing here is exported.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/nups.h"
+
+#define NUPS_MAX_DISTS 64
+#define NUPS_MAX_HANDLES 256
+#define NUPS_LOCAL_PROBES 64
+#define NUPS_OWNER_DEFAULT 255
+#define NUPS_INVALID_KEY 0xFFFFFFFFu
+#define NUPS_MAX_POOL 1024
+
+// ---------------------------------------------------------------------------------------------
+// Device-resident status and statistics
+// ---------------------------------------------------------------------------------------------
+struct DevStat {
+    int status;                        // first device-detected error, 0 = none
+    int pad;
+    unsigned long long hot_hits;       // accesses served by a replica
+    unsigned long long cold_hits;      // accesses served in place
+    unsigned long long req_count;      // localize requests queued by the running call
+    unsigned long long tmp[4];
+};
+
+// What kernels need to know about a store; passed by value.
+struct View {
+    float* val;
+    float* acc;
+    float* dval;               // [R][Hcap][L] pending replica updates of the value table
+    float* dacc;               // same for the accumulator table
+    const uint32_t* hot_bits;  // one bit per key: replicated?
+    const int32_t* slot_of;    // key -> hot slot (>= 0) or negative
+    uint32_t* dirty;           // [Hcap] slot touched since last sync
+    unsigned long long* cnt;   // [num_keys] access counts
+    uint8_t* owner;            // [num_keys] owning worker or NUPS_OWNER_DEFAULT; NULL = not tracked
+    int* pending;              // [num_keys] localize requests of the running call (-1 = none)
+    DevStat* st;
+    uint64_t num_keys;
+    uint64_t Hcap;
+    uint32_t H;
+    uint32_t L4;               // floats per row / 4
+    uint32_t R;
+    uint32_t count;            // count accesses?
+};
+
+struct Dist {
+    int used, uniform, level;
+    uint32_t key_base, U, G;
+    uint64_t n, W, seed;
+    void* table;               // AliasEntry[n]
+    unsigned long long* off;   // device [R]: next unused position of each worker's stream
+};
+
+struct AliasEntry {
+    unsigned long long thr;
+    uint32_t alias;
+    uint32_t pad;
+};
+
+struct Handle {
+    int used, dist;
+    uint64_t N, cursor;
+    char* buf;                 // device buffer, kept for reuse after release
+    size_t cap;
+};
+
+struct nups_store {
+    uint64_t num_keys;
+    uint32_t L, R;
+    nups_config cfg;
+    float *val, *acc;
+    uint32_t* hot_bits;
+    int32_t* slot_of;
+    uint32_t* hot_keys;
+    uint64_t H, Hcap;
+    float *dval, *dacc;
+    uint32_t* dirty;
+    unsigned long long* cnt;
+    uint8_t* owner;
+    int* pending;
+    DevStat* st;
+    char* scratch;
+    size_t scratch_bytes;
+    uint32_t* req_keys;        // localize request list of the running call
+    size_t req_cap;
+    uint32_t* last_negs;
+    uint64_t last_negs_n, last_negs_cap;
+    uint64_t steps, syncs, launches;
+    int device, sm_count, max_smem;
+    Dist dist[NUPS_MAX_DISTS];
+    Handle handle[NUPS_MAX_HANDLES];
+};
+
+// ---------------------------------------------------------------------------------------------
+// Host helpers
+// ---------------------------------------------------------------------------------------------
+extern thread_local char g_nups_cuda_err[256];
+nups_status nups_cuda_fail(cudaError_t e, const char* what);
+
+#define CK(call)                                                   \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return nups_cuda_fail(e__, #call); \
+    } while (0)
+
+#define LAUNCH_CHECK(store)                                         \
+    do {                                                            \
+        (store)->launches++;                                        \
+        cudaError_t e__ = cudaGetLastError();                       \
+        if (e__ != cudaSuccess) return nups_cuda_fail(e__, "kernel launch"); \
+    } while (0)
+
+static inline unsigned grid_for(uint64_t work, unsigned per_block, unsigned cap = 0x7FFFFFFFu)
+{
+    uint64_t g = (work + per_block - 1) / per_block;
+    if (g < 1) g = 1;
+    if (g > cap) g = cap;
+    return (unsigned)g;
+}
+
+View nups_view(const nups_store* s);
+nups_status nups_scratch(nups_store* s, size_t bytes, char** out);     // grow-only scratch, 256-byte aligned
+nups_status nups_req_reserve(nups_store* s, size_t n);
+
+// primitives.cu
+size_t nups_scan_scratch_bytes(uint64_t n);
+size_t nups_sort_scratch_bytes(uint64_t n);
+// Exclusive prefix sum of n uint64 values (in place allowed); *d_total (device, nullable) receives the sum.
+nups_status nups_scan_u64(nups_store* s, const unsigned long long* d_in, unsigned long long* d_out, uint64_t n,
+                          unsigned long long* d_total, char* scratch, cudaStream_t st);
+// Stable LSD radix sort of (key, value) pairs on the low `bits` bits; result ends up in (k_out, v_out).
+nups_status nups_sort_pairs(nups_store* s, unsigned long long* k_in, uint32_t* v_in, unsigned long long* k_out,
+                            uint32_t* v_out, uint64_t n, int bits, char* scratch, cudaStream_t st);
+
+// store.cu internals used by steps.cu / sampling.cu
+nups_status nups_push_internal(nups_store* s, const uint32_t* d_keys, uint64_t n_rows, uint32_t rows_per_item,
+                               const float* d_dval, const float* d_dacc, cudaStream_t st);
+size_t nups_push_scratch_bytes(const nups_store* s, uint64_t n_rows);
+nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64_t n_rows, uint32_t rows_per_item,
+                                   const float* d_dval, const float* d_dacc, char* scratch, cudaStream_t st);
+nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
+                                 float* d_out_acc, int worker_map, uint64_t map_base, uint64_t map_total,
+                                 int do_count, cudaStream_t st);
+nups_status nups_localize_apply(nups_store* s, uint64_t max_requests, cudaStream_t st);
+nups_status nups_sync_internal(nups_store* s, cudaStream_t st);
+// sampling.cu internals used by steps.cu
+nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st);
+
+// ---------------------------------------------------------------------------------------------
+// Device helpers
+// ---------------------------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+__device__ __forceinline__ void philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3, uint32_t k0,
+                                              uint32_t k1, uint32_t out[4])
+{
+    // Philox4x32-10 (Salmon et al., SC'11): ten rounds, each two 32x32->64 multiplies with the
+    // halves crossed and xor-ed with the round key; the key advances by the Weyl constants.
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint32_t hi0 = __umulhi(0xD2511F53u, c0), lo0 = 0xD2511F53u * c0;
+        uint32_t hi1 = __umulhi(0xCD9E8D57u, c2), lo1 = 0xCD9E8D57u * c2;
+        uint32_t n0 = hi1 ^ c1 ^ k0, n2 = hi0 ^ c3 ^ k1;
+        c0 = n0; c1 = lo1; c2 = n2; c3 = lo0;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// Counter layout of every draw: (index lo, index hi, stream, purpose + 256 * block).
+__device__ __forceinline__ void philox_at(uint64_t seed, uint64_t index, uint32_t stream, uint32_t purpose,
+                                          uint32_t block, uint32_t out[4])
+{
+    philox4x32_10((uint32_t)index, (uint32_t)(index >> 32), stream, purpose + 256u * block, (uint32_t)seed,
+                  (uint32_t)(seed >> 32), out);
+}
+
+// Worker of item i of n: contiguous chunks, floor(i * R / n).
+__device__ __forceinline__ uint32_t worker_of_item(uint64_t i, uint64_t n, uint32_t R)
+{
+    if (R == 1) return 0;
+    return (uint32_t)((i * R) / n);          // calls take fewer than 2^32 items: i * R < 2^40
+}
+
+// Sub-handle boundaries of a handle of N samples: b_q = floor(q * N / R).
+__device__ __forceinline__ uint64_t chunk_begin(uint32_t q, uint64_t N, uint32_t R) { return ((uint64_t)q * N) / R; }
+__device__ __forceinline__ uint32_t chunk_of_pos(uint64_t pos, uint64_t N, uint32_t R)
+{
+    if (R == 1) return 0;
+    uint32_t q = (uint32_t)((pos * R) / N);
+    if (q >= R) q = R - 1;
+    while (q + 1 < R && chunk_begin(q + 1, N, R) <= pos) ++q;
+    while (q > 0 && chunk_begin(q, N, R) > pos) --q;
+    return q;
+}
+
+// worker_map: 0 = items of a call (floor(i*R/n), i = (base + idx) / rows_per_item handled by caller),
+//             1 = positions of a sample handle (sub-handle chunks)
+__device__ __forceinline__ uint32_t worker_by_map(int map, uint64_t idx, uint64_t total, uint32_t R)
+{
+    return map == 0 ? worker_of_item(idx, total, R) : chunk_of_pos(idx, total, R);
+}
+
+__device__ __forceinline__ bool key_is_hot(const View& v, uint32_t k)
+{
+    return v.H != 0 && ((__ldg(v.hot_bits + (k >> 5)) >> (k & 31)) & 1u);
+}
+
+__device__ __forceinline__ bool key_is_local(const View& v, uint32_t q, uint32_t k)
+{
+    if (key_is_hot(v, k)) return true;
+    if (!v.owner) return true;
+    uint32_t o = v.owner[k];
+    return (o == NUPS_OWNER_DEFAULT ? k % v.R : o) == q;
+}
+
+__device__ __forceinline__ void flag_bad_key(const View& v) { atomicCAS(&v.st->status, 0, NUPS_EKEY); }
+
+__device__ __forceinline__ void red_add_v4(float* addr, float4 x)
+{
+    // one 128-bit reduction to global memory, no return value
+    asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(addr), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ float4 ld_stream_v4(const float4* p)
+{
+    float4 r;
+    asm volatile("ld.global.cs.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(r.x), "=f"(r.y), "=f"(r.z), "=f"(r.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st_stream_v4(float4* p, float4 x)
+{
+    asm volatile("st.global.cs.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p), "f"(x.x), "f"(x.y), "f"(x.z), "f"(x.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
+__device__ __forceinline__ float warp_sum(float x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+    return x;
+}
+
+#endif  // __CUDACC__

@@ -1,0 +1,553 @@
+// Sampling access: register_distribution (alias table built on the device), PrepareSample and
+// PullSample under the four conformity levels.  NuPS Sections 4.3, 4.4.
+#include <string.h>
+
+#include "nups_internal.cuh"
+
+static inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// ---------------------------------------------------------------------------------------------
+// Alias table.  n buckets of capacity W = sum w; item j has mass n*w[j]; "lights" have mass < W.
+// Lights are topped up by the heavies in index order, and a heavy whose remainder drops below W
+// is itself topped up by the next heavy.  With D(a) the running sum of the lights' deficits and
+// S(h) the running sum of the heavies' surpluses (both in index order):
+//   light a is filled by the first heavy h with S(h) >= D(a-1);
+//   heavy h turns light right after the first light a with D(a) > S(h); it keeps
+//   W + S(h) - D(a) and is filled by heavy h+1; a heavy that never turns light keeps W.
+// ---------------------------------------------------------------------------------------------
+__global__ void weight_sum_kernel(const uint32_t* __restrict__ w, uint64_t n, DevStat* st)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    unsigned long long sum = 0;
+    for (; i < n; i += stride) sum += w[i];
+    for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+    if ((threadIdx.x & 31) == 0 && sum) atomicAdd(&st->tmp[0], sum);
+}
+
+__global__ void alias_classify_kernel(const uint32_t* __restrict__ w, uint64_t n, unsigned long long W,
+                                      unsigned long long* __restrict__ lflag, unsigned long long* __restrict__ dfl,
+                                      unsigned long long* __restrict__ sfl)
+{
+    uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    unsigned long long mass = n * (unsigned long long)w[j];
+    bool light = mass < W;
+    lflag[j] = light ? 1ull : 0ull;
+    dfl[j] = light ? W - mass : 0ull;
+    sfl[j] = light ? 0ull : mass - W;
+}
+
+__global__ void alias_rank_kernel(const uint32_t* __restrict__ w, uint64_t n, unsigned long long W,
+                                  const unsigned long long* __restrict__ lrank, const unsigned long long* __restrict__ dex,
+                                  const unsigned long long* __restrict__ sex, unsigned long long nL,
+                                  unsigned long long* __restrict__ inc /* D at [0,nL), S at [nL,n) */,
+                                  uint32_t* __restrict__ hidx)
+{
+    uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    unsigned long long mass = n * (unsigned long long)w[j];
+    unsigned long long a = lrank[j];
+    if (mass < W) inc[a] = dex[j] + (W - mass);
+    else {
+        unsigned long long h = j - a;
+        inc[nL + h] = sex[j] + (mass - W);
+        hidx[h] = (uint32_t)j;
+    }
+}
+
+__global__ void alias_fill_kernel(const uint32_t* __restrict__ w, uint64_t n, unsigned long long W,
+                                  const unsigned long long* __restrict__ lrank, const unsigned long long* __restrict__ dex,
+                                  unsigned long long nL, const unsigned long long* __restrict__ inc,
+                                  const uint32_t* __restrict__ hidx, AliasEntry* __restrict__ table)
+{
+    uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    const unsigned long long* D = inc;
+    const unsigned long long* S = inc + nL;
+    const unsigned long long nH = n - nL;
+    unsigned long long mass = n * (unsigned long long)w[j];
+    AliasEntry e;
+    e.pad = 0;
+    if (mass < W) {
+        unsigned long long target = dex[j];          // D(a-1)
+        unsigned long long lo = 0, hi = nH;          // first h with S[h] >= target
+        while (lo < hi) {
+            unsigned long long mid = (lo + hi) >> 1;
+            if (S[mid] >= target) hi = mid; else lo = mid + 1;
+        }
+        e.thr = mass;
+        e.alias = hidx[lo < nH ? lo : nH - 1];
+    } else {
+        unsigned long long h = j - lrank[j];
+        unsigned long long Sh = S[h];
+        unsigned long long lo = 0, hi = nL;          // first a with D[a] > Sh
+        while (lo < hi) {
+            unsigned long long mid = (lo + hi) >> 1;
+            if (D[mid] > Sh) hi = mid; else lo = mid + 1;
+        }
+        if (lo < nL && h + 1 < nH) {
+            e.thr = W + Sh - D[lo];
+            e.alias = hidx[h + 1];
+        } else {
+            e.thr = W;
+            e.alias = (uint32_t)j;
+        }
+    }
+    table[j] = e;
+}
+
+__global__ void alias_unpack_kernel(const AliasEntry* __restrict__ table, uint64_t n, unsigned long long* thr,
+                                    uint32_t* alias)
+{
+    uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n) return;
+    thr[j] = table[j].thr;
+    alias[j] = table[j].alias;
+}
+
+extern "C" nups_status nups_register_distribution(nups_store* s, uint32_t key_base, const uint32_t* d_weights,
+                                                  uint64_t n, int level, uint32_t U, uint32_t G, uint64_t seed,
+                                                  int32_t* h_dist_out, void* stream)
+{
+    if (!s || !h_dist_out) return NUPS_EINVAL;
+    if (n == 0 || (uint64_t)key_base + n > s->num_keys) return NUPS_EINVAL;
+    if (level < NUPS_CONFORM || level > NUPS_NONCONFORM) return NUPS_EINVAL;
+    bool reuse = level == NUPS_BOUNDED || level == NUPS_LONGTERM;
+    if (reuse && (U == 0 || G == 0 || G > NUPS_MAX_POOL)) return NUPS_EINVAL;
+    if ((level == NUPS_LONGTERM || level == NUPS_NONCONFORM) && !s->owner) return NUPS_ESTATE;
+    int id = -1;
+    for (int i = 0; i < NUPS_MAX_DISTS; ++i) if (!s->dist[i].used) { id = i; break; }
+    if (id < 0) return NUPS_ENOMEM;
+    cudaStream_t st = (cudaStream_t)stream;
+    Dist d;
+    memset(&d, 0, sizeof(d));
+    d.key_base = key_base; d.n = n; d.level = level; d.U = U; d.G = G; d.seed = seed;
+    if (!d_weights) d.uniform = 1;
+    else {
+        CK(cudaMemsetAsync(&s->st->tmp[0], 0, 8, st));
+        weight_sum_kernel<<<grid_for(n, 256, (unsigned)s->sm_count * 8), 256, 0, st>>>(d_weights, n, s->st);
+        LAUNCH_CHECK(s);
+        unsigned long long W = 0;
+        CK(cudaMemcpyAsync(&W, &s->st->tmp[0], 8, cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+        if (W == 0) return NUPS_EINVAL;
+        unsigned __int128 nW = (unsigned __int128)W * n;
+        if (nW >> 64) return NUPS_EINVAL;
+        d.W = W;
+        size_t need = 4 * align256(n * 8) + align256(n * 4) + nups_scan_scratch_bytes(n) + 256;
+        char* sc;
+        nups_status rc = nups_scratch(s, need, &sc);
+        if (rc != NUPS_OK) return rc;
+        unsigned long long* lrank = (unsigned long long*)sc; sc += align256(n * 8);
+        unsigned long long* dex = (unsigned long long*)sc; sc += align256(n * 8);
+        unsigned long long* sex = (unsigned long long*)sc; sc += align256(n * 8);
+        unsigned long long* inc = (unsigned long long*)sc; sc += align256(n * 8);
+        uint32_t* hidx = (uint32_t*)sc; sc += align256(n * 4);
+        unsigned long long* d_nL = (unsigned long long*)sc; sc += 256;
+        if (cudaMalloc(&d.table, n * sizeof(AliasEntry)) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        unsigned g = grid_for(n, 256);
+        alias_classify_kernel<<<g, 256, 0, st>>>(d_weights, n, W, lrank, dex, sex);
+        LAUNCH_CHECK(s);
+        rc = nups_scan_u64(s, lrank, lrank, n, d_nL, sc, st);
+        if (rc == NUPS_OK) rc = nups_scan_u64(s, dex, dex, n, nullptr, sc, st);
+        if (rc == NUPS_OK) rc = nups_scan_u64(s, sex, sex, n, nullptr, sc, st);
+        if (rc != NUPS_OK) { cudaFree(d.table); return rc; }
+        unsigned long long nL = 0;
+        CK(cudaMemcpyAsync(&nL, d_nL, 8, cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+        alias_rank_kernel<<<g, 256, 0, st>>>(d_weights, n, W, lrank, dex, sex, nL, inc, hidx);
+        LAUNCH_CHECK(s);
+        alias_fill_kernel<<<g, 256, 0, st>>>(d_weights, n, W, lrank, dex, nL, inc, hidx, (AliasEntry*)d.table);
+        LAUNCH_CHECK(s);
+        CK(cudaStreamSynchronize(st));
+    }
+    if (cudaMalloc(&d.off, s->R * 8) != cudaSuccess) { cudaGetLastError(); cudaFree(d.table); return NUPS_ENOMEM; }
+    CK(cudaMemsetAsync(d.off, 0, s->R * 8, st));
+    CK(cudaStreamSynchronize(st));
+    d.used = 1;
+    s->dist[id] = d;
+    *h_dist_out = id;
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_get_alias_table(nups_store* s, int32_t dist, uint64_t* d_thr_out, uint32_t* d_alias_out,
+                                            uint64_t* h_W_out, void* stream)
+{
+    if (!s || dist < 0 || dist >= NUPS_MAX_DISTS || !s->dist[dist].used) return NUPS_EINVAL;
+    Dist& d = s->dist[dist];
+    if (h_W_out) *h_W_out = d.W;
+    if (d.uniform) return d_thr_out || d_alias_out ? NUPS_EINVAL : NUPS_OK;
+    if (d_thr_out && d_alias_out) {
+        alias_unpack_kernel<<<grid_for(d.n, 256), 256, 0, (cudaStream_t)stream>>>((const AliasEntry*)d.table, d.n,
+                                                                              (unsigned long long*)d_thr_out, d_alias_out);
+        LAUNCH_CHECK(s);
+    }
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Draws
+// ---------------------------------------------------------------------------------------------
+struct DrawParams {
+    const AliasEntry* table;
+    unsigned long long n, W, seed;
+    uint32_t key_base, U, G;
+    int uniform;
+};
+
+static DrawParams draw_params(const Dist& d)
+{
+    DrawParams p;
+    p.table = (const AliasEntry*)d.table; p.n = d.n; p.W = d.W; p.seed = d.seed;
+    p.key_base = d.key_base; p.U = d.U; p.G = d.G; p.uniform = d.uniform;
+    return p;
+}
+
+// one iid draw from pi: position `pos` of worker q's stream; 64 bits pick the bucket, 64 bits the
+// point inside it
+__device__ __forceinline__ uint32_t draw_iid(const DrawParams& p, uint32_t q, unsigned long long pos)
+{
+    uint32_t x[4];
+    philox_at(p.seed, pos, q, 0, 0, x);
+    unsigned long long a = (unsigned long long)x[0] | ((unsigned long long)x[1] << 32);
+    unsigned long long b = (unsigned long long)x[2] | ((unsigned long long)x[3] << 32);
+    unsigned long long j = __umul64hi(a, p.n);
+    if (!p.uniform) {
+        AliasEntry e = p.table[j];
+        if (!(__umul64hi(b, p.W) < e.thr)) j = e.alias;
+    }
+    return p.key_base + (uint32_t)j;
+}
+
+// Handle buffer layout (device): start[R] (u64) | keys[N] (u32) | post[N] (u32) | state[R] (uint4)
+struct HandleView {
+    unsigned long long* start;
+    uint32_t* keys;
+    uint32_t* post;
+    uint4* state;      // LONG-TERM per sub-handle: x = walk position, y = postponed head, z = postponed tail
+};
+static size_t handle_bytes(uint64_t N, uint32_t R, int level)
+{
+    size_t b = align256((size_t)R * 8) + align256(N * 4);
+    if (level == NUPS_LONGTERM) b += align256(N * 4) + align256((size_t)R * 16);
+    return b;
+}
+static HandleView handle_view(char* buf, uint64_t N, uint32_t R)
+{
+    HandleView h;
+    h.start = (unsigned long long*)buf; buf += align256((size_t)R * 8);
+    h.keys = (uint32_t*)buf; buf += align256(N * 4);
+    h.post = (uint32_t*)buf; buf += align256(N * 4);
+    h.state = (uint4*)buf;
+    return h;
+}
+
+__global__ void handle_begin_kernel(unsigned long long* off, HandleView h, uint64_t N, uint32_t R, int longterm)
+{
+    uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q >= R) return;
+    unsigned long long size = chunk_begin(q + 1, N, R) - chunk_begin(q, N, R);
+    h.start[q] = off[q];
+    off[q] += size;
+    if (longterm) h.state[q] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+__global__ void draw_iid_kernel(DrawParams p, HandleView h, uint64_t N, uint32_t R)
+{
+    uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= N) return;
+    uint32_t q = chunk_of_pos(o, N, R);
+    h.keys[o] = draw_iid(p, q, h.start[q] + (o - chunk_begin(q, N, R)));
+}
+
+// Pooled reuse: pool `pl` of a worker holds G iid draws and is walked U times, each pass in a fresh
+// Fisher-Yates order.  Stream position s lies in pass number s / G overall (pool = pass / U).
+// One block produces one pass of one worker.
+__global__ void draw_reuse_kernel(DrawParams p, HandleView h, uint64_t N, uint32_t R)
+{
+    __shared__ uint32_t pool[NUPS_MAX_POOL];
+    __shared__ uint32_t perm[NUPS_MAX_POOL];
+    __shared__ uint32_t xs[NUPS_MAX_POOL];
+    const uint32_t q = blockIdx.y, G = p.G;
+    const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
+    if (size == 0) return;
+    const unsigned long long s0 = h.start[q], s1 = s0 + size;
+    const unsigned long long pass = s0 / G + blockIdx.x;
+    if (pass * G >= s1) return;
+    const unsigned long long pl = pass / p.U;
+    for (uint32_t m = threadIdx.x; m < G; m += blockDim.x) {
+        pool[m] = draw_iid(p, q, pl * G + m);
+        perm[m] = m;
+    }
+    // random words of the shuffle: word d of the pass's Philox stream (purpose 1), four per block
+    for (uint32_t blk = threadIdx.x; blk * 4 < G - 1; blk += blockDim.x) {
+        uint32_t x[4];
+        philox_at(p.seed, pass, q, 1, blk, x);
+        for (int k = 0; k < 4; ++k)
+            if (blk * 4 + k < G - 1) xs[blk * 4 + k] = x[k];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (uint32_t i = G - 1; i >= 1; --i) {
+            uint32_t r = __umulhi(xs[G - 1 - i], i + 1);
+            uint32_t t = perm[i]; perm[i] = perm[r]; perm[r] = t;
+        }
+    }
+    __syncthreads();
+    for (uint32_t j = threadIdx.x; j < G; j += blockDim.x) {
+        unsigned long long sp = pass * G + j;
+        if (sp >= s0 && sp < s1) h.keys[b0 + (sp - s0)] = pool[perm[j]];
+    }
+}
+
+// PrepareSample localizes the sampled keys to the sub-handle's worker
+__global__ void localize_handle_kernel(View v, const uint32_t* __restrict__ keys, uint64_t N, uint32_t* req,
+                                       uint64_t req_cap)
+{
+    uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (o >= N) return;
+    uint32_t k = keys[o];
+    uint32_t q = chunk_of_pos(o, N, v.R);
+    atomicMax(v.pending + k, (int)q);
+    unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
+    if (at < req_cap) req[at] = k;
+}
+
+static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int* slot_out, cudaStream_t st)
+{
+    if (dist < 0 || dist >= NUPS_MAX_DISTS || !s->dist[dist].used || N == 0 || N >= (1ull << 32)) return NUPS_EINVAL;
+    Dist& d = s->dist[dist];
+    size_t need = handle_bytes(N, s->R, d.level);
+    int id = -1;
+    for (int i = 0; i < NUPS_MAX_HANDLES && id < 0; ++i)
+        if (!s->handle[i].used && s->handle[i].cap >= need) id = i;      // reuse a released buffer
+    for (int i = 0; i < NUPS_MAX_HANDLES && id < 0; ++i)
+        if (!s->handle[i].used && s->handle[i].cap == 0) id = i;
+    for (int i = 0; i < NUPS_MAX_HANDLES && id < 0; ++i)
+        if (!s->handle[i].used) id = i;
+    if (id < 0) return NUPS_ENOMEM;
+    Handle& h = s->handle[id];
+    if (h.cap < need) {
+        if (h.buf) CK(cudaFree(h.buf));
+        h.buf = nullptr; h.cap = 0;
+        size_t want = need + need / 4;
+        if (cudaMalloc(&h.buf, want) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        h.cap = want;
+    }
+    bool reuse = d.level == NUPS_BOUNDED || d.level == NUPS_LONGTERM;
+    bool loc = s->owner && d.level != NUPS_NONCONFORM;
+    if (loc || d.level == NUPS_LONGTERM) {
+        nups_status rc = nups_req_reserve(s, N);
+        if (rc != NUPS_OK) return rc;
+    }
+    HandleView hv = handle_view(h.buf, N, s->R);
+    DrawParams p = draw_params(d);
+    handle_begin_kernel<<<grid_for(s->R, 64), 64, 0, st>>>(d.off, hv, N, s->R, d.level == NUPS_LONGTERM);
+    LAUNCH_CHECK(s);
+    if (reuse) {
+        uint64_t max_size = (N + s->R - 1) / s->R;
+        unsigned passes = (unsigned)(max_size / d.G + 2);
+        unsigned threads = ((d.G + 31) / 32) * 32;
+        if (threads > 256) threads = 256;
+        draw_reuse_kernel<<<dim3(passes, s->R), threads, 0, st>>>(p, hv, N, s->R);
+    } else {
+        draw_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(p, hv, N, s->R);
+    }
+    LAUNCH_CHECK(s);
+    if (loc) {
+        localize_handle_kernel<<<grid_for(N, 256), 256, 0, st>>>(nups_view(s), hv.keys, N, s->req_keys, s->req_cap);
+        LAUNCH_CHECK(s);
+        nups_status rc = nups_localize_apply(s, N, st);
+        if (rc != NUPS_OK) return rc;
+    }
+    h.used = 1; h.dist = dist; h.N = N; h.cursor = 0;
+    *slot_out = id;
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_prepare_sample(nups_store* s, int32_t dist, uint64_t N, nups_handle* h_out, void* stream)
+{
+    if (!s || !h_out) return NUPS_EINVAL;
+    int id = -1;
+    nups_status rc = prepare_internal(s, dist, N, &id, (cudaStream_t)stream);
+    if (rc == NUPS_OK) *h_out = id;
+    return rc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// PullSample
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void count_sample(const View& v, uint32_t key, bool emitted)
+{
+    if (!v.count) return;
+    const unsigned lane = threadIdx.x & 31;
+    bool hot = emitted && key_is_hot(v, key);
+    if (emitted) atomicAdd(v.cnt + key, 1ull);
+    unsigned hot_m = __ballot_sync(0xFFFFFFFFu, emitted && hot);
+    unsigned cold_m = __ballot_sync(0xFFFFFFFFu, emitted && !hot);
+    if (lane == 0) {
+        if (hot_m) atomicAdd(&v.st->hot_hits, (unsigned long long)__popc(hot_m));
+        if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
+    }
+}
+
+// independent draws / pooled reuse: the keys were fixed at PrepareSample.
+// local sampling: first key local to the worker at or after the candidate.
+__global__ void emit_kernel(View v, DrawParams p, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, int local_only,
+                            uint32_t* __restrict__ out)
+{
+    uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    bool in = o < n;
+    uint32_t k = 0;
+    if (in) {
+        uint64_t pos = cursor + o;
+        k = h.keys[pos];
+        if (local_only) {
+            uint32_t q = chunk_of_pos(pos, N, v.R);
+            uint32_t k0 = k;
+            for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
+                uint32_t cand = p.key_base + (uint32_t)(((unsigned long long)(k0 - p.key_base) + probe) % p.n);
+                if (key_is_local(v, q, cand)) { k = cand; break; }
+            }
+        }
+        out[o] = k;
+    }
+    count_sample(v, k, in);
+}
+
+// reuse with postponing: one block walks one sub-handle.  Entries not yet postponed are taken in
+// order; a local one is emitted, a non-local one is queued for re-localization and appended to the
+// sub-handle's postponed queue; when the fresh entries run out the postponed ones are emitted.
+__global__ void __launch_bounds__(256)
+longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
+                uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+{
+    __shared__ unsigned warp_tot[8];
+    __shared__ unsigned sh_consumed, sh_local;
+    const uint32_t q = q_first + blockIdx.x;
+    const unsigned tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint64_t b0 = chunk_begin(q, N, v.R), b1 = chunk_begin(q + 1, N, v.R);
+    const uint64_t lo = max(b0, cursor), hi = min(b1, cursor + n);
+    if (lo >= hi) return;
+    const uint64_t take = hi - lo, size = b1 - b0;
+    const uint64_t out_base = lo - cursor;
+    uint4 stt = h.state[q];
+    uint64_t oc = stt.x, ph = stt.y, pt = stt.z, emitted = 0;
+    while (emitted < take && oc < size) {
+        uint64_t i = oc + tid;
+        bool have = i < size;
+        uint32_t key = have ? h.keys[b0 + i] : 0u;
+        bool loc = have && key_is_local(v, q, key);
+        unsigned bal = __ballot_sync(0xFFFFFFFFu, loc);
+        unsigned excl = __popc(bal & ((1u << lane) - 1u));
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        for (unsigned w = 0; w < warp; ++w) excl += warp_tot[w];
+        uint64_t need = take - emitted;
+        bool consumed = have && excl < need;
+        if (consumed) {
+            if (loc) out[out_base + emitted + excl] = key;
+            else {
+                h.post[b0 + pt + (tid - excl)] = key;
+                atomicMax(v.pending + key, (int)q);
+                unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
+                if (at < req_cap) req[at] = key;
+            }
+        }
+        count_sample(v, key, consumed && loc);
+        unsigned cbal = __ballot_sync(0xFFFFFFFFu, consumed);
+        unsigned lbal = __ballot_sync(0xFFFFFFFFu, consumed && loc);
+        if (tid == 0) { sh_consumed = 0; sh_local = 0; }
+        __syncthreads();
+        if (lane == 0) { atomicAdd(&sh_consumed, __popc(cbal)); atomicAdd(&sh_local, __popc(lbal)); }
+        __syncthreads();
+        unsigned nc = sh_consumed, nl = sh_local;
+        emitted += nl; pt += nc - nl; oc += nc;
+        __syncthreads();
+    }
+    __syncthreads();
+    if (emitted < take) {
+        uint64_t cnt = take - emitted;
+        for (uint64_t i = tid; i < ((cnt + 255) / 256) * 256; i += 256) {
+            bool in = i < cnt;
+            uint32_t key = in ? h.post[b0 + ph + i] : 0u;
+            if (in) out[out_base + emitted + i] = key;
+            count_sample(v, key, in);
+        }
+        ph += cnt;
+    }
+    if (tid == 0) h.state[q] = make_uint4((unsigned)oc, (unsigned)ph, (unsigned)pt, 0u);
+}
+
+static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_keys_out, float* d_vals_out,
+                                 cudaStream_t st)
+{
+    Handle& h = s->handle[id];
+    Dist& d = s->dist[h.dist];
+    if (n > h.N - h.cursor) return NUPS_ESTATE;
+    if (n == 0) return NUPS_OK;
+    View v = nups_view(s);
+    HandleView hv = handle_view(h.buf, h.N, s->R);
+    DrawParams p = draw_params(d);
+    if (d.level == NUPS_LONGTERM) {
+        // sub-handles overlapped by [cursor, cursor + n)
+        uint32_t qf = 0, ql = 0;
+        for (uint32_t q = 0; q < s->R; ++q) {
+            uint64_t b0 = ((uint64_t)q * h.N) / s->R, b1 = ((uint64_t)(q + 1) * h.N) / s->R;
+            if (b0 <= h.cursor && h.cursor < b1) qf = q;
+            if (b0 <= h.cursor + n - 1 && h.cursor + n - 1 < b1) ql = q;
+        }
+        longterm_kernel<<<ql - qf + 1, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->req_keys, s->req_cap);
+        LAUNCH_CHECK(s);
+        nups_status rc = nups_localize_apply(s, h.N, st);
+        if (rc != NUPS_OK) return rc;
+    } else {
+        emit_kernel<<<grid_for(n, 256), 256, 0, st>>>(v, p, hv, h.N, h.cursor, n, d.level == NUPS_NONCONFORM, d_keys_out);
+        LAUNCH_CHECK(s);
+    }
+    if (d_vals_out) {
+        nups_status rc = nups_gather_internal(s, d_keys_out, n, d_vals_out, nullptr, 1, h.cursor, h.N, 0, st);
+        if (rc != NUPS_OK) return rc;
+    }
+    h.cursor += n;
+    if (h.cursor == h.N) h.used = 0;       // released; the buffer stays for the next handle
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_pull_sample(nups_store* s, nups_handle handle, uint64_t n, uint32_t* d_keys_out,
+                                        float* d_vals_out, void* stream)
+{
+    if (!s || handle < 0 || handle >= NUPS_MAX_HANDLES || !s->handle[handle].used) return NUPS_EINVAL;
+    if (n && !d_keys_out) return NUPS_EINVAL;
+    return pull_internal(s, (int)handle, n, d_keys_out, d_vals_out, (cudaStream_t)stream);
+}
+
+// negatives of a workload step: one handle of N samples, pulled at once into library memory
+nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st)
+{
+    s->last_negs_n = 0;
+    if (N == 0) return NUPS_OK;
+    if (N > s->last_negs_cap) {
+        if (s->last_negs) CK(cudaFree(s->last_negs));
+        s->last_negs = nullptr; s->last_negs_cap = 0;
+        uint64_t want = N + N / 4;
+        if (cudaMalloc(&s->last_negs, want * 4) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        s->last_negs_cap = want;
+    }
+    int id = -1;
+    nups_status rc = prepare_internal(s, dist, N, &id, st);
+    if (rc != NUPS_OK) return rc;
+    rc = pull_internal(s, id, N, s->last_negs, nullptr, st);
+    if (rc != NUPS_OK) return rc;
+    s->last_negs_n = N;
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_last_negatives(nups_store* s, const uint32_t** h_d_keys_out, uint64_t* h_n_out)
+{
+    if (!s || !h_d_keys_out || !h_n_out) return NUPS_EINVAL;
+    *h_d_keys_out = s->last_negs;
+    *h_n_out = s->last_negs_n;
+    return NUPS_OK;
+}

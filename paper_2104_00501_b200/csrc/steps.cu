@@ -1,0 +1,558 @@
+// Workload steps driving the store: skip-gram with negative sampling, ComplEx with AdaGrad and
+// matrix factorization (NuPS Section 5.1).  One warp per item: rows are pulled into registers,
+// dot products are reduced with warp shuffles, updates are pushed either straight to the store
+// (fast mode, 128-bit reductions) or into a row buffer that the ordered push applies afterwards
+// (deterministic mode, all pulls see the values from before the step).
+#include "nups_internal.cuh"
+
+static inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+namespace {
+
+__device__ __forceinline__ float clamp30(float x) { return fminf(30.f, fmaxf(-30.f, x)); }
+__device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
+__device__ __forceinline__ float softplusf_(float x) { return fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))); }
+
+// Where a key's row is read from and written to by worker q.
+struct RowRef {
+    const float* base;     // stored row
+    const float* pend;     // the worker's pending replica updates, or NULL
+    float* dst;            // where pushes go: the replica (hot) or the stored row
+    int slot;
+};
+
+template <bool HOT>
+__device__ __forceinline__ RowRef resolve(const View& v, uint32_t key, uint32_t q, int which)
+{
+    RowRef r;
+    float* table = which ? v.acc : v.val;
+    const uint64_t L = (uint64_t)v.L4 * 4;
+    r.base = table + (uint64_t)key * L;
+    r.pend = nullptr;
+    r.dst = table + (uint64_t)key * L;
+    r.slot = -1;
+    if (HOT && key_is_hot(v, key)) {
+        r.slot = __ldg(v.slot_of + key);
+        float* slab = which ? v.dacc : v.dval;
+        float* p = slab + ((uint64_t)q * v.Hcap + (uint64_t)r.slot) * L;
+        r.pend = p;
+        r.dst = p;
+    }
+    return r;
+}
+
+__device__ __forceinline__ void red_add_v2(float* addr, float2 x)
+{
+    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(x.x), "f"(x.y) : "memory");
+}
+
+// lane 0 of the item's warp: access count and replica/in-place statistics for one key
+__device__ __forceinline__ void note_access(const View& v, uint32_t key, int slot, unsigned times)
+{
+    atomicAdd(v.cnt + key, (unsigned long long)times);
+    atomicAdd(slot >= 0 ? &v.st->hot_hits : &v.st->cold_hits, (unsigned long long)times);
+}
+
+__device__ __forceinline__ void request_localize(const View& v, uint32_t key, uint32_t q, uint32_t* req, uint64_t cap)
+{
+    atomicMax(v.pending + key, (int)q);
+    unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
+    if (at < cap) req[at] = key;
+}
+
+// ---------------------------------------------------------------------------------------------
+// skip-gram with negative sampling
+// ---------------------------------------------------------------------------------------------
+template <bool HOT, bool DET, int CH>
+__global__ void __launch_bounds__(128)
+sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
+            const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float* __restrict__ upd,
+            uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, uint32_t* req, uint64_t req_cap)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = v.L4, per = K + 2;
+    for (uint64_t i = warp; i < n; i += nwarps) {
+        const uint32_t q = worker_of_item(i, n, v.R);
+        const uint32_t kc = center[i], ko = context[i];
+        bool ok = kc < v.num_keys && ko < v.num_keys;
+        for (uint32_t j = 0; j < K; ++j) ok = ok && negs[i * K + j] < v.num_keys;
+        if (DET && lane == 0) {
+            ukeys[i * per] = ok ? ko : NUPS_INVALID_KEY;
+            for (uint32_t j = 0; j < K; ++j) ukeys[i * per + 1 + j] = ok ? negs[i * K + j] : NUPS_INVALID_KEY;
+            ukeys[i * per + K + 1] = ok ? kc : NUPS_INVALID_KEY;
+        }
+        if (!ok) {
+            if (lane == 0) { flag_bad_key(v); loss_item[i] = 0.f; }
+            continue;
+        }
+        RowRef rc = resolve<HOT>(v, kc, q, 0);
+        float4 vr[CH], gv[CH];
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            uint32_t c = lane + 32 * m;
+            vr[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+            gv[m] = vr[m];
+            if (c < L4) {
+                vr[m] = ((const float4*)rc.base)[c];
+                if (rc.pend) vr[m] = add4(vr[m], ((const float4*)rc.pend)[c]);
+            }
+        }
+        float loss = 0.f;
+        for (uint32_t j = 0; j <= K; ++j) {
+            const uint32_t ku = j == 0 ? ko : negs[i * K + j - 1];
+            RowRef ru = resolve<HOT>(v, ku, q, 0);
+            float4 ur[CH];
+            float dot = 0.f;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                uint32_t c = lane + 32 * m;
+                ur[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+                if (c < L4) {
+                    ur[m] = ((const float4*)ru.base)[c];
+                    if (ru.pend) ur[m] = add4(ur[m], ((const float4*)ru.pend)[c]);
+                }
+                dot += vr[m].x * ur[m].x + vr[m].y * ur[m].y + vr[m].z * ur[m].z + vr[m].w * ur[m].w;
+            }
+            float x = clamp30(warp_sum(dot));
+            float g = sigmoidf_(x) - (j == 0 ? 1.f : 0.f);
+            loss += j == 0 ? softplusf_(-x) : softplusf_(x);
+            float sc = -lr * g;
+            float* out = DET ? upd + (i * per + j) * (uint64_t)L4 * 4 : ru.dst;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                uint32_t c = lane + 32 * m;
+                if (c < L4) {
+                    float4 du = make_float4(sc * vr[m].x, sc * vr[m].y, sc * vr[m].z, sc * vr[m].w);
+                    if (DET) ((float4*)out)[c] = du;
+                    else red_add_v4(out + 4 * c, du);
+                    gv[m].x += g * ur[m].x; gv[m].y += g * ur[m].y; gv[m].z += g * ur[m].z; gv[m].w += g * ur[m].w;
+                }
+            }
+            if (lane == 0) {
+                if (!DET && ru.slot >= 0) v.dirty[ru.slot] = 1u;
+                if (v.count) {
+                    if (j == 0) note_access(v, ku, ru.slot, DET ? 1u : 2u);      // pulled (+ pushed)
+                    else if (!DET) note_access(v, ku, ru.slot, 1u);              // pushed; the sample was counted at the draw
+                }
+            }
+        }
+        float* out = DET ? upd + (i * per + K + 1) * (uint64_t)L4 * 4 : rc.dst;
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            uint32_t c = lane + 32 * m;
+            if (c < L4) {
+                float4 dv = make_float4(-lr * gv[m].x, -lr * gv[m].y, -lr * gv[m].z, -lr * gv[m].w);
+                if (DET) ((float4*)out)[c] = dv;
+                else red_add_v4(out + 4 * c, dv);
+            }
+        }
+        if (lane == 0) {
+            if (!DET && rc.slot >= 0) v.dirty[rc.slot] = 1u;
+            if (v.count) note_access(v, kc, rc.slot, DET ? 1u : 2u);
+            if (v.owner) { request_localize(v, ko, q, req, req_cap); request_localize(v, kc, q, req, req_cap); }
+            loss_item[i] = loss;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// ComplEx with AdaGrad.  Rows are [re(0..d-1) | im(0..d-1)], d = L/2 (even); a lane owns pairs of
+// adjacent components: float2 of the real half and the matching float2 of the imaginary half.
+// ---------------------------------------------------------------------------------------------
+struct C2 { float2 re, im; };
+
+template <int CH>
+__device__ __forceinline__ void load_row(const RowRef& r, uint32_t d2, unsigned lane, C2 (&x)[CH])
+{
+    const float2* b = (const float2*)r.base;
+    const float2* p = (const float2*)r.pend;
+#pragma unroll
+    for (int m = 0; m < CH; ++m) {
+        uint32_t c = lane + 32 * m;
+        x[m].re = make_float2(0.f, 0.f);
+        x[m].im = x[m].re;
+        if (c < d2) {
+            x[m].re = b[c];
+            x[m].im = b[d2 + c];
+            if (p) {
+                float2 a = p[c], bb = p[d2 + c];
+                x[m].re.x += a.x; x[m].re.y += a.y; x[m].im.x += bb.x; x[m].im.y += bb.y;
+            }
+        }
+    }
+}
+
+template <int CH>
+__device__ __forceinline__ float score(const C2 (&h)[CH], const C2 (&r)[CH], const C2 (&t)[CH])
+{
+    float s = 0.f;
+#pragma unroll
+    for (int m = 0; m < CH; ++m) {
+        s += h[m].re.x * r[m].re.x * t[m].re.x + h[m].im.x * r[m].re.x * t[m].im.x + h[m].re.x * r[m].im.x * t[m].im.x -
+             h[m].im.x * r[m].im.x * t[m].re.x;
+        s += h[m].re.y * r[m].re.y * t[m].re.y + h[m].im.y * r[m].re.y * t[m].im.y + h[m].re.y * r[m].im.y * t[m].im.y -
+             h[m].im.y * r[m].im.y * t[m].re.y;
+    }
+    return warp_sum(s);
+}
+
+// g_h += coef * d(phi)/d(h), and likewise for r and t (any of the three may be skipped)
+template <int CH>
+__device__ __forceinline__ void grads(const C2 (&h)[CH], const C2 (&r)[CH], const C2 (&t)[CH], float coef, C2* gh,
+                                      C2* gr, C2* gt)
+{
+#pragma unroll
+    for (int m = 0; m < CH; ++m) {
+#define NUPS_C1(comp)                                                                                         \
+        {                                                                                                     \
+            float hr = h[m].re.comp, hi = h[m].im.comp, rr = r[m].re.comp, ri = r[m].im.comp;                 \
+            float tr = t[m].re.comp, ti = t[m].im.comp;                                                       \
+            if (gh) { gh[m].re.comp += coef * (rr * tr + ri * ti); gh[m].im.comp += coef * (rr * ti - ri * tr); } \
+            if (gt) { gt[m].re.comp += coef * (hr * rr - hi * ri); gt[m].im.comp += coef * (hi * rr + hr * ri); } \
+            if (gr) { gr[m].re.comp += coef * (hr * tr + hi * ti); gr[m].im.comp += coef * (hr * ti - hi * tr); } \
+        }
+        NUPS_C1(x)
+        NUPS_C1(y)
+#undef NUPS_C1
+    }
+}
+
+// AdaGrad update of one key role from its summed gradient: acc += g^2, val -= lr g / (sqrt(a + g^2) + eps)
+template <bool HOT, bool DET, int CH>
+__device__ __forceinline__ void adagrad_push(const View& v, uint32_t key, uint32_t q, const C2 (&g)[CH], uint32_t d2,
+                                             unsigned lane, float lr, float eps, float* uval_row, float* uacc_row,
+                                             bool pulled_too)
+{
+    RowRef rv = resolve<HOT>(v, key, q, 0);
+    RowRef ra = resolve<HOT>(v, key, q, 1);
+    const float2* ab = (const float2*)ra.base;
+    const float2* ap = (const float2*)ra.pend;
+    float2* ov = (float2*)(DET ? uval_row : rv.dst);
+    float2* oa = (float2*)(DET ? uacc_row : ra.dst);
+#pragma unroll
+    for (int m = 0; m < CH; ++m) {
+        uint32_t c = lane + 32 * m;
+        if (c < d2) {
+#pragma unroll
+            for (int half = 0; half < 2; ++half) {
+                uint32_t at = half ? d2 + c : c;
+                float2 gg = half ? g[m].im : g[m].re;
+                float2 a = ab[at];
+                if (ap) { float2 pa = ap[at]; a.x += pa.x; a.y += pa.y; }
+                float2 g2 = make_float2(gg.x * gg.x, gg.y * gg.y);
+                float2 dv = make_float2(-lr * gg.x / (sqrtf(a.x + g2.x) + eps), -lr * gg.y / (sqrtf(a.y + g2.y) + eps));
+                if (DET) { ov[at] = dv; oa[at] = g2; }
+                else { red_add_v2((float*)(ov + at), dv); red_add_v2((float*)(oa + at), g2); }
+            }
+        }
+    }
+    if (lane == 0) {
+        if (!DET && rv.slot >= 0) v.dirty[rv.slot] = 1u;
+        if (v.count) {
+            unsigned times = (pulled_too ? 1u : 0u) + (DET ? 0u : 1u);
+            if (times) note_access(v, key, rv.slot, times);
+        }
+    }
+}
+
+template <bool HOT, bool DET, int CH>
+__global__ void __launch_bounds__(128)
+complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restrict__ rk, const uint32_t* __restrict__ tk,
+               const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float eps, float* __restrict__ uval,
+               float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, uint32_t* req,
+               uint64_t req_cap)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t d2 = v.L4, per = K + 3;            // d/2 pairs = L/4
+    const uint64_t L = (uint64_t)v.L4 * 4;
+    for (uint64_t i = warp; i < n; i += nwarps) {
+        const uint32_t q = worker_of_item(i, n, v.R);
+        const uint32_t kh = hk[i], kr = rk[i], kt = tk[i];
+        bool ok = kh < v.num_keys && kr < v.num_keys && kt < v.num_keys;
+        for (uint32_t j = 0; j < K; ++j) ok = ok && negs[i * K + j] < v.num_keys;
+        if (DET && lane == 0) {
+            ukeys[i * per] = ok ? kh : NUPS_INVALID_KEY;
+            ukeys[i * per + 1] = ok ? kr : NUPS_INVALID_KEY;
+            ukeys[i * per + 2] = ok ? kt : NUPS_INVALID_KEY;
+            for (uint32_t j = 0; j < K; ++j) ukeys[i * per + 3 + j] = ok ? negs[i * K + j] : NUPS_INVALID_KEY;
+        }
+        if (!ok) {
+            if (lane == 0) { flag_bad_key(v); loss_item[i] = 0.f; }
+            continue;
+        }
+        C2 h[CH], r[CH], t[CH], gh[CH], gr[CH], gt[CH];
+        load_row<CH>(resolve<HOT>(v, kh, q, 0), d2, lane, h);
+        load_row<CH>(resolve<HOT>(v, kr, q, 0), d2, lane, r);
+        load_row<CH>(resolve<HOT>(v, kt, q, 0), d2, lane, t);
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            gh[m].re = make_float2(0.f, 0.f); gh[m].im = gh[m].re;
+            gr[m] = gh[m]; gt[m] = gh[m];
+        }
+        float phi = clamp30(score<CH>(h, r, t));
+        float loss = softplusf_(-phi);
+        grads<CH>(h, r, t, sigmoidf_(phi) - 1.f, gh, gr, gt);
+        for (uint32_t j = 0; j < K; ++j) {
+            const uint32_t ke = negs[i * K + j];
+            C2 e[CH], ge[CH];
+            load_row<CH>(resolve<HOT>(v, ke, q, 0), d2, lane, e);
+#pragma unroll
+            for (int m = 0; m < CH; ++m) { ge[m].re = make_float2(0.f, 0.f); ge[m].im = ge[m].re; }
+            if ((j & 1) == 0) {
+                float ph = clamp30(score<CH>(e, r, t));
+                loss += softplusf_(ph);
+                grads<CH>(e, r, t, sigmoidf_(ph), ge, gr, gt);
+            } else {
+                float ph = clamp30(score<CH>(h, r, e));
+                loss += softplusf_(ph);
+                grads<CH>(h, r, e, sigmoidf_(ph), gh, gr, ge);
+            }
+            adagrad_push<HOT, DET, CH>(v, ke, q, ge, d2, lane, lr, eps, DET ? uval + (i * per + 3 + j) * L : nullptr,
+                                       DET ? uacc + (i * per + 3 + j) * L : nullptr, false);
+        }
+        adagrad_push<HOT, DET, CH>(v, kh, q, gh, d2, lane, lr, eps, DET ? uval + (i * per) * L : nullptr,
+                                   DET ? uacc + (i * per) * L : nullptr, true);
+        adagrad_push<HOT, DET, CH>(v, kr, q, gr, d2, lane, lr, eps, DET ? uval + (i * per + 1) * L : nullptr,
+                                   DET ? uacc + (i * per + 1) * L : nullptr, true);
+        adagrad_push<HOT, DET, CH>(v, kt, q, gt, d2, lane, lr, eps, DET ? uval + (i * per + 2) * L : nullptr,
+                                   DET ? uacc + (i * per + 2) * L : nullptr, true);
+        if (lane == 0) {
+            if (v.owner) {
+                request_localize(v, kh, q, req, req_cap);
+                request_localize(v, kr, q, req, req_cap);
+                request_localize(v, kt, q, req, req_cap);
+            }
+            loss_item[i] = loss;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// matrix factorization
+// ---------------------------------------------------------------------------------------------
+template <bool HOT, bool DET, int CH>
+__global__ void __launch_bounds__(128)
+mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
+          uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
+          float* __restrict__ loss_item, uint32_t* req, uint64_t req_cap)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = v.L4;
+    for (uint64_t i = warp; i < n; i += nwarps) {
+        const uint32_t q = worker_of_item(i, n, v.R);
+        const uint32_t ki = rowk[i], kj = colk[i];
+        bool ok = ki < v.num_keys && kj < v.num_keys;
+        if (DET && lane == 0) {
+            ukeys[2 * i] = ok ? ki : NUPS_INVALID_KEY;
+            ukeys[2 * i + 1] = ok ? kj : NUPS_INVALID_KEY;
+        }
+        if (!ok) {
+            if (lane == 0) { flag_bad_key(v); loss_item[i] = 0.f; }
+            continue;
+        }
+        RowRef rw = resolve<HOT>(v, ki, q, 0), rh = resolve<HOT>(v, kj, q, 0);
+        float4 w[CH], h[CH];
+        float dot = 0.f;
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            uint32_t c = lane + 32 * m;
+            w[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+            h[m] = w[m];
+            if (c < L4) {
+                w[m] = ((const float4*)rw.base)[c];
+                h[m] = ((const float4*)rh.base)[c];
+                if (rw.pend) w[m] = add4(w[m], ((const float4*)rw.pend)[c]);
+                if (rh.pend) h[m] = add4(h[m], ((const float4*)rh.pend)[c]);
+            }
+            dot += w[m].x * h[m].x + w[m].y * h[m].y + w[m].z * h[m].z + w[m].w * h[m].w;
+        }
+        float err = x[i] - warp_sum(dot);
+        float* ow = DET ? upd + (2 * i) * (uint64_t)L4 * 4 : rw.dst;
+        float* oh = DET ? upd + (2 * i + 1) * (uint64_t)L4 * 4 : rh.dst;
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            uint32_t c = lane + 32 * m;
+            if (c < L4) {
+                float4 dw = make_float4(lr * (err * h[m].x - l2 * w[m].x), lr * (err * h[m].y - l2 * w[m].y),
+                                        lr * (err * h[m].z - l2 * w[m].z), lr * (err * h[m].w - l2 * w[m].w));
+                float4 dh = make_float4(lr * (err * w[m].x - l2 * h[m].x), lr * (err * w[m].y - l2 * h[m].y),
+                                        lr * (err * w[m].z - l2 * h[m].z), lr * (err * w[m].w - l2 * h[m].w));
+                if (DET) { ((float4*)ow)[c] = dw; ((float4*)oh)[c] = dh; }
+                else { red_add_v4(ow + 4 * c, dw); red_add_v4(oh + 4 * c, dh); }
+            }
+        }
+        if (lane == 0) {
+            if (!DET) {
+                if (rw.slot >= 0) v.dirty[rw.slot] = 1u;
+                if (rh.slot >= 0) v.dirty[rh.slot] = 1u;
+            }
+            if (v.count) {
+                note_access(v, ki, rw.slot, DET ? 1u : 2u);
+                note_access(v, kj, rh.slot, DET ? 1u : 2u);
+            }
+            if (v.owner) { request_localize(v, ki, q, req, req_cap); request_localize(v, kj, q, req, req_cap); }
+            loss_item[i] = err * err;
+        }
+    }
+}
+
+// mean of the per-item losses, summed in a fixed order
+__global__ void loss_mean_kernel(const float* __restrict__ loss_item, uint64_t n, float* __restrict__ out)
+{
+    __shared__ double sh[256];
+    double s = 0.0;
+    for (uint64_t i = threadIdx.x; i < n; i += 256) s += (double)loss_item[i];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *out = (float)(sh[0] / (double)(n ? n : 1));
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------------
+struct StepBuffers {
+    float* loss_item;
+    uint32_t* ukeys;
+    float* uval;
+    float* uacc;
+    char* push_scratch;
+};
+
+static nups_status step_buffers(nups_store* s, uint64_t n, uint64_t per, bool two_tables, StepBuffers* b)
+{
+    const bool det = s->cfg.deterministic;
+    uint64_t rows = n * per;
+    size_t row_bytes = (size_t)rows * s->L * sizeof(float);
+    size_t need = align256(n * 4);
+    if (det) need += align256(rows * 4) + align256(row_bytes) * (two_tables ? 2 : 1) + nups_push_scratch_bytes(s, rows);
+    char* sc;
+    nups_status rc = nups_scratch(s, need, &sc);
+    if (rc != NUPS_OK) return rc;
+    b->loss_item = (float*)sc; sc += align256(n * 4);
+    b->ukeys = nullptr; b->uval = nullptr; b->uacc = nullptr; b->push_scratch = nullptr;
+    if (det) {
+        b->ukeys = (uint32_t*)sc; sc += align256(rows * 4);
+        b->uval = (float*)sc; sc += align256(row_bytes);
+        if (two_tables) { b->uacc = (float*)sc; sc += align256(row_bytes); }
+        b->push_scratch = sc;
+    }
+    return NUPS_OK;
+}
+
+static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t direct_keys, const StepBuffers& b,
+                               float* d_loss_out, cudaStream_t st)
+{
+    nups_status rc;
+    if (s->cfg.deterministic) {
+        rc = nups_push_with_scratch(s, b.ukeys, n * per, (uint32_t)per, b.uval, b.uacc, b.push_scratch, st);
+        if (rc != NUPS_OK) return rc;
+    }
+    rc = nups_localize_apply(s, n * direct_keys, st);
+    if (rc != NUPS_OK) return rc;
+    if (d_loss_out) {
+        loss_mean_kernel<<<1, 256, 0, st>>>(b.loss_item, n, d_loss_out);
+        LAUNCH_CHECK(s);
+    }
+    s->steps++;
+    if (s->cfg.sync_interval && s->steps % s->cfg.sync_interval == 0) return nups_sync_internal(s, st);
+    return NUPS_OK;
+}
+
+static unsigned step_grid(const nups_store* s, uint64_t n)
+{
+    return grid_for(n, 4, (unsigned)s->sm_count * 16);     // 4 warps per block, one item per warp per pass
+}
+
+#define DISPATCH_CH(L4, ...)                                      \
+    do {                                                          \
+        if ((L4) <= 32) { constexpr int CH = 1; __VA_ARGS__; }    \
+        else if ((L4) <= 64) { constexpr int CH = 2; __VA_ARGS__; } \
+        else if ((L4) <= 96) { constexpr int CH = 3; __VA_ARGS__; } \
+        else { constexpr int CH = 4; __VA_ARGS__; }               \
+    } while (0)
+
+#define DISPATCH_MODE(s, ...)                                                                \
+    do {                                                                                     \
+        if ((s)->H) {                                                                        \
+            if ((s)->cfg.deterministic) { constexpr bool HOT = true, DET = true; __VA_ARGS__; } \
+            else { constexpr bool HOT = true, DET = false; __VA_ARGS__; }                    \
+        } else {                                                                             \
+            if ((s)->cfg.deterministic) { constexpr bool HOT = false, DET = true; __VA_ARGS__; } \
+            else { constexpr bool HOT = false, DET = false; __VA_ARGS__; }                   \
+        }                                                                                    \
+    } while (0)
+
+extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n,
+                                      int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream)
+{
+    if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
+    if (s->L / 4 > 128) return NUPS_EINVAL;                 // rows of up to 512 floats are held in registers
+    cudaStream_t st = (cudaStream_t)stream;
+    nups_status rc = nups_draw_negatives(s, dist, n * K, st);
+    if (rc != NUPS_OK) return rc;
+    rc = nups_req_reserve(s, n * 2);
+    if (rc != NUPS_OK) return rc;
+    StepBuffers b;
+    rc = step_buffers(s, n, K + 2, false, &b);
+    if (rc != NUPS_OK) return rc;
+    View v = nups_view(s);
+    unsigned grid = step_grid(s, n);
+    DISPATCH_MODE(s, DISPATCH_CH(v.L4, sgns_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
+        v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+    LAUNCH_CHECK(s);
+    return step_finish(s, n, K + 2, 2, b, d_loss_out, st);
+}
+
+extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, const uint32_t* d_r, const uint32_t* d_t,
+                                         uint64_t n, int32_t dist, uint32_t K, float lr, float eps, float* d_loss_out,
+                                         void* stream)
+{
+    if (!s || !d_h || !d_r || !d_t || n == 0 || n * (uint64_t)(K + 3) >= (1ull << 32)) return NUPS_EINVAL;
+    if (!s->acc || s->L / 4 > 128) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    nups_status rc = nups_draw_negatives(s, dist, n * K, st);
+    if (rc != NUPS_OK) return rc;
+    rc = nups_req_reserve(s, n * 3);
+    if (rc != NUPS_OK) return rc;
+    StepBuffers b;
+    rc = step_buffers(s, n, K + 3, true, &b);
+    if (rc != NUPS_OK) return rc;
+    View v = nups_view(s);
+    unsigned grid = step_grid(s, n);
+    DISPATCH_MODE(s, DISPATCH_CH(v.L4, complex_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
+        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+    LAUNCH_CHECK(s);
+    return step_finish(s, n, K + 3, 3, b, d_loss_out, st);
+}
+
+extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
+                                    uint64_t n, float lr, float l2, float* d_loss_out, void* stream)
+{
+    if (!s || !d_row || !d_col || !d_x || n == 0 || n * 2 >= (1ull << 32)) return NUPS_EINVAL;
+    if (s->L / 4 > 128) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    s->last_negs_n = 0;
+    nups_status rc = nups_req_reserve(s, n * 2);
+    if (rc != NUPS_OK) return rc;
+    StepBuffers b;
+    rc = step_buffers(s, n, 2, false, &b);
+    if (rc != NUPS_OK) return rc;
+    View v = nups_view(s);
+    unsigned grid = step_grid(s, n);
+    DISPATCH_MODE(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
+        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+    LAUNCH_CHECK(s);
+    return step_finish(s, n, 2, 2, b, d_loss_out, st);
+}

@@ -1,0 +1,1027 @@
+// Key store, direct access (pull / push), replica merge, access counting, hot-set selection and
+// per-key management.  NuPS Sections 3.1, 3.2, 5.1.
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include "nups_internal.cuh"
+
+thread_local char g_nups_cuda_err[256] = "";
+
+nups_status nups_cuda_fail(cudaError_t e, const char* what)
+{
+    snprintf(g_nups_cuda_err, sizeof(g_nups_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return NUPS_ECUDA;
+}
+
+extern "C" const char* nups_last_cuda_error(void) { return g_nups_cuda_err; }
+
+extern "C" const char* nups_strerror(nups_status st)
+{
+    switch (st) {
+        case NUPS_OK: return "ok";
+        case NUPS_EINVAL: return "invalid argument";
+        case NUPS_ENOMEM: return "out of memory or table full";
+        case NUPS_ECUDA: return "CUDA runtime error";
+        case NUPS_EKEY: return "key out of range seen on the device";
+        case NUPS_ESTATE: return "call not valid in the current state";
+        case NUPS_ETIMEOUT: return "bounded device-side wait gave up";
+        default: return "unknown status";
+    }
+}
+
+View nups_view(const nups_store* s)
+{
+    View v;
+    v.val = s->val; v.acc = s->acc; v.dval = s->dval; v.dacc = s->dacc;
+    v.hot_bits = s->hot_bits; v.slot_of = s->slot_of; v.dirty = s->dirty;
+    v.cnt = s->cnt; v.owner = s->owner; v.pending = s->pending; v.st = s->st;
+    v.num_keys = s->num_keys; v.Hcap = s->Hcap; v.H = (uint32_t)s->H; v.L4 = s->L / 4; v.R = s->R;
+    v.count = s->cfg.count_accesses;
+    return v;
+}
+
+nups_status nups_scratch(nups_store* s, size_t bytes, char** out)
+{
+    if (bytes > s->scratch_bytes) {
+        size_t want = bytes + bytes / 4 + (1u << 20);
+        if (s->scratch) CK(cudaFree(s->scratch));     // waits for work that may still use it
+        s->scratch = nullptr; s->scratch_bytes = 0;
+        cudaError_t e = cudaMalloc(&s->scratch, want);
+        if (e != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        s->scratch_bytes = want;
+    }
+    *out = s->scratch;
+    return NUPS_OK;
+}
+
+nups_status nups_req_reserve(nups_store* s, size_t n)
+{
+    if (!s->owner) return NUPS_OK;
+    if (n > s->req_cap) {
+        size_t want = n + n / 2 + 1024;
+        if (s->req_keys) CK(cudaFree(s->req_keys));
+        s->req_keys = nullptr; s->req_cap = 0;
+        if (cudaMalloc(&s->req_keys, want * sizeof(uint32_t)) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        s->req_cap = want;
+    }
+    return NUPS_OK;
+}
+
+static inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
+
+// ---------------------------------------------------------------------------------------------
+// create / destroy
+// ---------------------------------------------------------------------------------------------
+__global__ void fill_i32(int* p, uint64_t n, int value)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (; i < n; i += stride) p[i] = value;
+}
+
+extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const nups_config* cfg, nups_store** out)
+{
+    if (!out) return NUPS_EINVAL;
+    *out = nullptr;
+    if (num_keys == 0 || num_keys > 0xFFFFFFFFull || value_len == 0 || (value_len & 3)) return NUPS_EINVAL;
+    nups_config c;
+    memset(&c, 0, sizeof(c));
+    if (cfg) c = *cfg;
+    if (c.workers == 0) c.workers = 8;
+    if (c.workers > 254) return NUPS_EINVAL;
+    int dev = 0, count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) {
+        snprintf(g_nups_cuda_err, sizeof(g_nups_cuda_err), "no CUDA device");
+        cudaGetLastError();
+        return NUPS_ECUDA;
+    }
+    CK(cudaGetDevice(&dev));
+    nups_store* s = (nups_store*)calloc(1, sizeof(nups_store));
+    if (!s) return NUPS_ENOMEM;
+    s->num_keys = num_keys; s->L = value_len; s->R = c.workers; s->cfg = c; s->device = dev;
+    cudaDeviceGetAttribute(&s->sm_count, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&s->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    size_t table_bytes = (size_t)num_keys * value_len * sizeof(float);
+    bool ok = cudaMalloc(&s->val, table_bytes) == cudaSuccess;
+    if (ok && c.with_adagrad) ok = cudaMalloc(&s->acc, table_bytes) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->hot_bits, ((num_keys + 31) / 32) * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->slot_of, num_keys * 4) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->cnt, num_keys * 8) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->st, sizeof(DevStat)) == cudaSuccess;
+    if (ok && c.track_ownership) {
+        ok = cudaMalloc(&s->owner, num_keys) == cudaSuccess;
+        ok = ok && cudaMalloc(&s->pending, num_keys * 4) == cudaSuccess;
+    }
+    if (!ok) {
+        cudaGetLastError();
+        nups_destroy(s);
+        return NUPS_ENOMEM;
+    }
+    cudaMemset(s->val, 0, table_bytes);
+    if (s->acc) cudaMemset(s->acc, 0, table_bytes);
+    cudaMemset(s->hot_bits, 0, ((num_keys + 31) / 32) * 4);
+    cudaMemset(s->cnt, 0, num_keys * 8);
+    cudaMemset(s->st, 0, sizeof(DevStat));
+    fill_i32<<<grid_for(num_keys, 256, 4096), 256>>>(s->slot_of, num_keys, -1);
+    if (s->owner) {
+        cudaMemset(s->owner, NUPS_OWNER_DEFAULT, num_keys);
+        fill_i32<<<grid_for(num_keys, 256, 4096), 256>>>(s->pending, num_keys, -1);
+    }
+    cudaError_t e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        nups_destroy(s);
+        return nups_cuda_fail(e, "nups_create");
+    }
+    *out = s;
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_destroy(nups_store* s)
+{
+    if (!s) return NUPS_OK;
+    cudaDeviceSynchronize();
+    for (int i = 0; i < NUPS_MAX_HANDLES; ++i) cudaFree(s->handle[i].buf);
+    for (int i = 0; i < NUPS_MAX_DISTS; ++i) { cudaFree(s->dist[i].table); cudaFree(s->dist[i].off); }
+    cudaFree(s->val); cudaFree(s->acc); cudaFree(s->hot_bits); cudaFree(s->slot_of); cudaFree(s->hot_keys);
+    cudaFree(s->dval); cudaFree(s->dacc); cudaFree(s->dirty); cudaFree(s->cnt); cudaFree(s->owner);
+    cudaFree(s->pending); cudaFree(s->st); cudaFree(s->scratch); cudaFree(s->req_keys); cudaFree(s->last_negs);
+    cudaGetLastError();
+    free(s);
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_table_ptr(nups_store* s, int which, float** ptr, uint64_t* stride)
+{
+    if (!s || !ptr || (which != 0 && which != 1)) return NUPS_EINVAL;
+    if (which == 1 && !s->acc) return NUPS_EINVAL;
+    *ptr = which ? s->acc : s->val;
+    if (stride) *stride = s->L;
+    return NUPS_OK;
+}
+
+__global__ void init_uniform_kernel(float4* t, uint64_t total4, uint64_t seed, uint32_t which, float unit)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (; i < total4; i += stride) {
+        uint32_t x[4];
+        philox_at(seed, i, which, 3, 0, x);
+        float4 r;
+        r.x = __fmul_rn((float)((int)(x[0] >> 8) - 8388608), unit);
+        r.y = __fmul_rn((float)((int)(x[1] >> 8) - 8388608), unit);
+        r.z = __fmul_rn((float)((int)(x[2] >> 8) - 8388608), unit);
+        r.w = __fmul_rn((float)((int)(x[3] >> 8) - 8388608), unit);
+        t[i] = r;
+    }
+}
+
+extern "C" nups_status nups_init_uniform(nups_store* s, int which, uint64_t seed, float scale, void* stream)
+{
+    if (!s || (which != 0 && which != 1) || (which == 1 && !s->acc)) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint64_t total4 = s->num_keys * (s->L / 4);
+    float unit = scale * (1.0f / 8388608.0f);
+    init_uniform_kernel<<<grid_for(total4, 256, (unsigned)s->sm_count * 16), 256, 0, st>>>(
+        (float4*)(which ? s->acc : s->val), total4, seed, (uint32_t)which, unit);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// pull: row gather.  One warp walks windows of 32 keys; each lane fetches one key of the window,
+// the warp then copies the rows four at a time with 128-bit loads and streaming stores.
+// ---------------------------------------------------------------------------------------------
+constexpr int GATHER_UNROLL = 4;
+
+template <bool HOT>
+__global__ void __launch_bounds__(256)
+gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, float4* __restrict__ out_val,
+              float4* __restrict__ out_acc, int map, uint64_t map_base, uint64_t map_total, uint32_t rows_per_item,
+              int do_count)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = v.L4;
+    const float4* val4 = (const float4*)v.val;
+    const float4* acc4 = (const float4*)v.acc;
+    const float4* dval4 = (const float4*)v.dval;
+    const float4* dacc4 = (const float4*)v.dacc;
+    for (uint64_t base = warp * 32; base < n; base += nwarps * 32) {
+        uint64_t i = base + lane;
+        uint32_t key = i < n ? __ldg(keys + i) : 0u;
+        bool in = i < n;
+        bool valid = in && key < v.num_keys;
+        if (in && !valid) flag_bad_key(v);
+        int slot = -1;
+        uint32_t q = 0;
+        if (HOT && valid && key_is_hot(v, key)) {
+            slot = __ldg(v.slot_of + key);
+            uint64_t idx = map_base + i;
+            q = map == 0 ? worker_of_item(idx / rows_per_item, map_total, v.R) : chunk_of_pos(idx, map_total, v.R);
+        }
+        if (do_count && v.count) {
+            if (valid) atomicAdd(v.cnt + key, 1ull);
+            unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && slot >= 0);
+            unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && slot < 0);
+            if (lane == 0) {
+                if (hot_m) atomicAdd(&v.st->hot_hits, (unsigned long long)__popc(hot_m));
+                if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
+            }
+        }
+        const int rows = (int)min((uint64_t)32, n - base);
+        for (int r = 0; r < rows; r += GATHER_UNROLL) {
+            uint32_t k[GATHER_UNROLL];
+            int sl[GATHER_UNROLL];
+            uint32_t qq[GATHER_UNROLL];
+            bool ok[GATHER_UNROLL];
+#pragma unroll
+            for (int u = 0; u < GATHER_UNROLL; ++u) {
+                int src = min(r + u, 31);
+                k[u] = __shfl_sync(0xFFFFFFFFu, key, src);
+                sl[u] = __shfl_sync(0xFFFFFFFFu, slot, src);
+                qq[u] = __shfl_sync(0xFFFFFFFFu, q, src);
+                ok[u] = __shfl_sync(0xFFFFFFFFu, (int)valid, src) != 0;
+            }
+            for (uint32_t c = lane; c < L4; c += 32) {
+                float4 a[GATHER_UNROLL], b[GATHER_UNROLL];
+#pragma unroll
+                for (int u = 0; u < GATHER_UNROLL; ++u) {
+                    a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    b[u] = a[u];
+                    if (r + u < rows && ok[u]) {
+                        uint64_t ro = (uint64_t)k[u] * L4 + c;
+                        if (out_val) a[u] = __ldg(val4 + ro);
+                        if (out_acc) b[u] = __ldg(acc4 + ro);
+                        if (HOT && sl[u] >= 0) {
+                            uint64_t so = ((uint64_t)qq[u] * v.Hcap + (uint64_t)sl[u]) * L4 + c;
+                            if (out_val) a[u] = add4(a[u], dval4[so]);
+                            if (out_acc) b[u] = add4(b[u], dacc4[so]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < GATHER_UNROLL; ++u) {
+                    if (r + u < rows) {
+                        uint64_t oo = (base + r + u) * L4 + c;
+                        if (out_val) st_stream_v4(out_val + oo, a[u]);
+                        if (out_acc) st_stream_v4(out_acc + oo, b[u]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
+                                 float* d_out_acc, int worker_map, uint64_t map_base, uint64_t map_total,
+                                 int do_count, cudaStream_t st)
+{
+    if (n == 0 || (!d_out_val && !d_out_acc)) return NUPS_OK;
+    View v = nups_view(s);
+    unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 8);
+    if (s->H)
+        gather_kernel<true><<<grid, 256, 0, st>>>(v, d_keys, n, (float4*)d_out_val, (float4*)d_out_acc, worker_map,
+                                                  map_base, map_total, 1, do_count);
+    else
+        gather_kernel<false><<<grid, 256, 0, st>>>(v, d_keys, n, (float4*)d_out_val, (float4*)d_out_acc, worker_map,
+                                                   map_base, map_total, 1, do_count);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_pull2(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
+                                  float* d_out_acc, void* stream)
+{
+    if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
+    if (d_out_acc && !s->acc) return NUPS_EINVAL;
+    if (n && !d_out_val && !d_out_acc) return NUPS_EINVAL;
+    return nups_gather_internal(s, d_keys, n, d_out_val, d_out_acc, 0, 0, n, 1, (cudaStream_t)stream);
+}
+
+extern "C" nups_status nups_pull(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out, void* stream)
+{
+    if (n && !d_out) return NUPS_EINVAL;
+    return nups_pull2(s, d_keys, n, d_out, nullptr, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// push, fast mode: 128-bit reductions straight to the destination row.  Within a window of 32
+// rows, rows with the same destination are summed in registers first (__match_any_sync) so that
+// a hot destination receives one reduction per window instead of one per row.
+// ---------------------------------------------------------------------------------------------
+constexpr int PUSH_UNROLL = 4;
+
+template <bool HOT>
+__global__ void __launch_bounds__(256)
+push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const float4* __restrict__ dv,
+                   const float4* __restrict__ da, uint64_t n_items, uint32_t rows_per_item)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = v.L4;
+    for (uint64_t base = warp * 32; base < n; base += nwarps * 32) {
+        uint64_t i = base + lane;
+        bool in = i < n;
+        uint32_t key = in ? __ldg(keys + i) : 0u;
+        bool valid = in && key < v.num_keys;
+        if (in && !valid) flag_bad_key(v);
+        int slot = -1;
+        uint64_t row = 0;                 // destination row offset (in float4) inside its table or slab
+        if (valid) {
+            row = (uint64_t)key * L4;
+            if (HOT && key_is_hot(v, key)) {
+                slot = __ldg(v.slot_of + key);
+                uint32_t q = worker_of_item(i / rows_per_item, n_items, v.R);
+                row = ((uint64_t)q * v.Hcap + (uint64_t)slot) * L4;
+                v.dirty[slot] = 1u;
+            }
+        }
+        if (v.count) {
+            if (valid) atomicAdd(v.cnt + key, 1ull);
+            unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && slot >= 0);
+            unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && slot < 0);
+            if (lane == 0) {
+                if (hot_m) atomicAdd(&v.st->hot_hits, (unsigned long long)__popc(hot_m));
+                if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
+            }
+        }
+        // destination identity: (replica?, row offset); invalid rows get a value no one shares
+        unsigned long long dest = valid ? ((row << 1) | (slot >= 0 ? 1ull : 0ull)) : (~0ull - lane);
+        unsigned grp = __match_any_sync(0xFFFFFFFFu, dest);
+        bool leader = valid && (lane == (unsigned)(__ffs(grp) - 1));
+        unsigned singles = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) == 1);
+        unsigned multis = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) > 1);
+
+        // rows that are alone in their window: four at a time
+        while (singles) {
+            int src[PUSH_UNROLL];
+            uint64_t ro[PUSH_UNROLL];
+            int hs[PUSH_UNROLL];
+#pragma unroll
+            for (int u = 0; u < PUSH_UNROLL; ++u) {
+                if (singles) {
+                    src[u] = __ffs(singles) - 1;
+                    singles &= singles - 1;
+                } else src[u] = -1;
+                int from = src[u] < 0 ? 0 : src[u];
+                ro[u] = __shfl_sync(0xFFFFFFFFu, row, from);
+                hs[u] = __shfl_sync(0xFFFFFFFFu, slot, from);
+            }
+            for (uint32_t c = lane; c < L4; c += 32) {
+                float4 a[PUSH_UNROLL], b[PUSH_UNROLL];
+#pragma unroll
+                for (int u = 0; u < PUSH_UNROLL; ++u) {
+                    if (src[u] >= 0) {
+                        uint64_t in_off = (base + src[u]) * L4 + c;
+                        if (dv) a[u] = ld_stream_v4(dv + in_off);
+                        if (da) b[u] = ld_stream_v4(da + in_off);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < PUSH_UNROLL; ++u) {
+                    if (src[u] >= 0) {
+                        bool hot = HOT && hs[u] >= 0;
+                        if (dv) red_add_v4((hot ? v.dval : v.val) + (ro[u] + c) * 4, a[u]);
+                        if (da) red_add_v4((hot ? v.dacc : v.acc) + (ro[u] + c) * 4, b[u]);
+                    }
+                }
+            }
+        }
+        // destinations hit more than once in the window: sum the members, one reduction
+        while (multis) {
+            int ld = __ffs(multis) - 1;
+            multis &= multis - 1;
+            unsigned members = __shfl_sync(0xFFFFFFFFu, grp, ld);
+            uint64_t ro = __shfl_sync(0xFFFFFFFFu, row, ld);
+            int hs = __shfl_sync(0xFFFFFFFFu, slot, ld);
+            bool hot = HOT && hs >= 0;
+            for (uint32_t c = lane; c < L4; c += 32) {
+                float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+                unsigned mm = members;
+                while (mm) {
+                    int m = __ffs(mm) - 1;
+                    mm &= mm - 1;
+                    uint64_t in_off = (base + m) * L4 + c;
+                    if (dv) a = add4(a, ld_stream_v4(dv + in_off));
+                    if (da) b = add4(b, ld_stream_v4(da + in_off));
+                }
+                if (dv) red_add_v4((hot ? v.dval : v.val) + (ro + c) * 4, a);
+                if (da) red_add_v4((hot ? v.dacc : v.acc) + (ro + c) * 4, b);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// push, deterministic mode: rows are sorted (stably) by destination, then one warp per
+// destination adds its rows one by one in input order.
+// ---------------------------------------------------------------------------------------------
+template <bool HOT>
+__global__ void push_dest_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, uint64_t n_items,
+                                 uint32_t rows_per_item, unsigned long long invalid_dest,
+                                 unsigned long long* __restrict__ dest, uint32_t* __restrict__ idx)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned lane = threadIdx.x & 31;
+    bool in = i < n;
+    uint32_t key = in ? keys[i] : 0u;
+    bool valid = in && key < v.num_keys;
+    if (in && !valid) flag_bad_key(v);
+    bool hot = false;
+    unsigned long long d = invalid_dest;
+    if (valid) {
+        d = key;
+        if (HOT && key_is_hot(v, key)) {
+            hot = true;
+            uint32_t slot = (uint32_t)v.slot_of[key];
+            uint32_t q = worker_of_item(i / rows_per_item, n_items, v.R);
+            d = (1ull << 32) + (unsigned long long)q * v.H + slot;
+            v.dirty[slot] = 1u;
+        }
+    }
+    if (in) { dest[i] = d; idx[i] = (uint32_t)i; }
+    if (v.count) {
+        if (valid) atomicAdd(v.cnt + key, 1ull);
+        unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && hot);
+        unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && !hot);
+        if (lane == 0) {
+            if (hot_m) atomicAdd(&v.st->hot_hits, (unsigned long long)__popc(hot_m));
+            if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
+        }
+    }
+}
+
+__global__ void __launch_bounds__(256)
+push_ordered_kernel(View v, const unsigned long long* __restrict__ dest, const uint32_t* __restrict__ idx, uint64_t n,
+                    unsigned long long invalid_dest, const float4* __restrict__ dv, const float4* __restrict__ da)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t j = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    if (j >= n) return;
+    unsigned long long d = dest[j];
+    if (d == invalid_dest) return;
+    if (j > 0 && dest[j - 1] == d) return;           // not the first row of its destination
+    const uint32_t L4 = v.L4;
+    float4* tv;
+    float4* ta;
+    if (d >> 32) {
+        unsigned long long r = d - (1ull << 32);
+        uint64_t q = r / v.H, slot = r % v.H;
+        uint64_t off = (q * v.Hcap + slot) * L4;
+        tv = (float4*)v.dval + off;
+        ta = (float4*)v.dacc + off;
+    } else {
+        tv = (float4*)v.val + d * L4;
+        ta = (float4*)v.acc + d * L4;
+    }
+    uint64_t end = j + 1;
+    while (end < n && dest[end] == d) ++end;
+    for (uint32_t c = lane; c < L4; c += 32) {
+        float4 a = dv ? tv[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 b = da ? ta[c] : make_float4(0.f, 0.f, 0.f, 0.f);
+        uint64_t p = j;
+        for (; p + 4 <= end; p += 4) {               // loads issued together, adds kept in order
+            uint64_t o0 = (uint64_t)idx[p] * L4 + c, o1 = (uint64_t)idx[p + 1] * L4 + c;
+            uint64_t o2 = (uint64_t)idx[p + 2] * L4 + c, o3 = (uint64_t)idx[p + 3] * L4 + c;
+            if (dv) {
+                float4 x0 = dv[o0], x1 = dv[o1], x2 = dv[o2], x3 = dv[o3];
+                a = add4(add4(add4(add4(a, x0), x1), x2), x3);
+            }
+            if (da) {
+                float4 y0 = da[o0], y1 = da[o1], y2 = da[o2], y3 = da[o3];
+                b = add4(add4(add4(add4(b, y0), y1), y2), y3);
+            }
+        }
+        for (; p < end; ++p) {
+            uint64_t o = (uint64_t)idx[p] * L4 + c;
+            if (dv) a = add4(a, dv[o]);
+            if (da) b = add4(b, da[o]);
+        }
+        if (dv) tv[c] = a;
+        if (da) ta[c] = b;
+    }
+}
+
+static int bits_for(unsigned long long maxval)
+{
+    int b = 1;
+    while (b < 64 && (maxval >> b)) ++b;
+    return b;
+}
+
+size_t nups_push_scratch_bytes(const nups_store* s, uint64_t n)
+{
+    if (!s->cfg.deterministic) return 0;
+    return 2 * align256(n * 8) + 2 * align256(n * 4) + nups_sort_scratch_bytes(n);
+}
+
+nups_status nups_push_internal(nups_store* s, const uint32_t* d_keys, uint64_t n, uint32_t rows_per_item,
+                               const float* d_dval, const float* d_dacc, cudaStream_t st)
+{
+    char* sc = nullptr;
+    if (s->cfg.deterministic && n) {
+        nups_status rc = nups_scratch(s, nups_push_scratch_bytes(s, n), &sc);
+        if (rc != NUPS_OK) return rc;
+    }
+    return nups_push_with_scratch(s, d_keys, n, rows_per_item, d_dval, d_dacc, sc, st);
+}
+
+nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64_t n, uint32_t rows_per_item,
+                                   const float* d_dval, const float* d_dacc, char* sc, cudaStream_t st)
+{
+    if (n == 0 || (!d_dval && !d_dacc)) return NUPS_OK;
+    View v = nups_view(s);
+    uint64_t n_items = n / rows_per_item;
+    if (!s->cfg.deterministic) {
+        unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 8);
+        if (s->H)
+            push_atomic_kernel<true><<<grid, 256, 0, st>>>(v, d_keys, n, (const float4*)d_dval, (const float4*)d_dacc,
+                                                           n_items, rows_per_item);
+        else
+            push_atomic_kernel<false><<<grid, 256, 0, st>>>(v, d_keys, n, (const float4*)d_dval, (const float4*)d_dacc,
+                                                            n_items, rows_per_item);
+        LAUNCH_CHECK(s);
+        return NUPS_OK;
+    }
+    unsigned long long invalid_dest = s->H ? (1ull << 32) + (unsigned long long)s->R * s->H : s->num_keys;
+    int bits = bits_for(invalid_dest);
+    nups_status rc;
+    unsigned long long* k0 = (unsigned long long*)sc; sc += align256(n * 8);
+    unsigned long long* k1 = (unsigned long long*)sc; sc += align256(n * 8);
+    uint32_t* v0 = (uint32_t*)sc; sc += align256(n * 4);
+    uint32_t* v1 = (uint32_t*)sc; sc += align256(n * 4);
+    if (s->H)
+        push_dest_kernel<true><<<grid_for(n, 256), 256, 0, st>>>(v, d_keys, n, n_items, rows_per_item, invalid_dest, k0, v0);
+    else
+        push_dest_kernel<false><<<grid_for(n, 256), 256, 0, st>>>(v, d_keys, n, n_items, rows_per_item, invalid_dest, k0, v0);
+    LAUNCH_CHECK(s);
+    rc = nups_sort_pairs(s, k0, v0, k1, v1, n, bits, sc, st);
+    if (rc != NUPS_OK) return rc;
+    push_ordered_kernel<<<grid_for(n * 32, 256), 256, 0, st>>>(v, k1, v1, n, invalid_dest, (const float4*)d_dval,
+                                                               (const float4*)d_dacc);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_push2(nups_store* s, const uint32_t* d_keys, uint64_t n, const float* d_dval,
+                                  const float* d_dacc, void* stream)
+{
+    if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
+    if (d_dacc && !s->acc) return NUPS_EINVAL;
+    if (n && !d_dval && !d_dacc) return NUPS_EINVAL;
+    return nups_push_internal(s, d_keys, n, 1, d_dval, d_dacc, (cudaStream_t)stream);
+}
+
+extern "C" nups_status nups_push(nups_store* s, const uint32_t* d_keys, uint64_t n, const float* d_delta, void* stream)
+{
+    if (n && !d_delta) return NUPS_EINVAL;
+    return nups_push2(s, d_keys, n, d_delta, nullptr, stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// sync: merge the workers' pending updates of every touched hot slot into the stored row,
+// worker 0 first, and clear them.
+// ---------------------------------------------------------------------------------------------
+__global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
+{
+    const uint32_t L4 = v.L4;
+    uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint64_t total = (uint64_t)v.H * L4;
+    if (t >= total) return;
+    uint32_t slot = (uint32_t)(t / L4), c = (uint32_t)(t % L4);
+    if (!v.dirty[slot]) return;
+    uint32_t key = hot_keys[slot];
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int which = 0; which < 2; ++which) {
+        float4* table = (float4*)(which ? v.acc : v.val);
+        float4* slab = (float4*)(which ? v.dacc : v.dval);
+        if (!table || !slab) continue;
+        float4 sum = zero;
+        for (uint32_t r = 0; r < v.R; ++r) {
+            float4* p = slab + ((uint64_t)r * v.Hcap + slot) * L4 + c;
+            sum = add4(sum, *p);
+            *p = zero;
+        }
+        float4* row = table + (uint64_t)key * L4 + c;
+        *row = add4(*row, sum);
+    }
+}
+
+nups_status nups_sync_internal(nups_store* s, cudaStream_t st)
+{
+    if (s->H == 0) return NUPS_OK;        // nothing replicated: no work at all
+    View v = nups_view(s);
+    sync_kernel<<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
+    LAUNCH_CHECK(s);
+    CK(cudaMemsetAsync(s->dirty, 0, s->H * sizeof(uint32_t), st));
+    s->syncs++;
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_sync(nups_store* s, void* stream)
+{
+    if (!s) return NUPS_EINVAL;
+    return nups_sync_internal(s, (cudaStream_t)stream);
+}
+
+// ---------------------------------------------------------------------------------------------
+// access counting and hot-set selection
+// ---------------------------------------------------------------------------------------------
+__global__ void count_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const unsigned lane = threadIdx.x & 31;
+    bool in = i < n;
+    uint32_t key = in ? keys[i] : 0u;
+    bool valid = in && key < v.num_keys;
+    if (in && !valid) flag_bad_key(v);
+    unsigned long long tag = valid ? (unsigned long long)key : (~0ull - lane);
+    unsigned grp = __match_any_sync(0xFFFFFFFFu, tag);
+    if (valid && lane == (unsigned)(__ffs(grp) - 1)) atomicAdd(v.cnt + key, (unsigned long long)__popc(grp));
+}
+
+extern "C" nups_status nups_count_accesses(nups_store* s, const uint32_t* d_keys, uint64_t n, void* stream)
+{
+    if (!s || (n && !d_keys)) return NUPS_EINVAL;
+    if (n == 0) return NUPS_OK;
+    count_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(nups_view(s), d_keys, n);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_get_counts(nups_store* s, uint64_t* d_out, void* stream)
+{
+    if (!s || !d_out) return NUPS_EINVAL;
+    CK(cudaMemcpyAsync(d_out, s->cnt, s->num_keys * 8, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return NUPS_OK;
+}
+
+__global__ void count_sum_max_kernel(const unsigned long long* __restrict__ cnt, uint64_t n, DevStat* st)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    unsigned long long sum = 0, mx = 0;
+    for (; i < n; i += stride) {
+        unsigned long long c = cnt[i];
+        sum += c;
+        mx = c > mx ? c : mx;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        unsigned long long m2 = __shfl_xor_sync(0xFFFFFFFFu, mx, o);
+        mx = m2 > mx ? m2 : mx;
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicAdd(&st->tmp[0], sum);
+        atomicMax(&st->tmp[1], mx);
+    }
+}
+
+// flag[k] = 1 when key k is selected by the threshold rule cnt*num_keys > factor*total (exact)
+__global__ void threshold_flag_kernel(const unsigned long long* __restrict__ cnt, uint64_t n, unsigned long long factor,
+                                      unsigned long long total, unsigned long long* __restrict__ flag)
+{
+    uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    unsigned long long c = cnt[k];
+    unsigned long long lhi = __umul64hi(c, n), llo = c * n;
+    unsigned long long rhi = __umul64hi(factor, total), rlo = factor * total;
+    flag[k] = (lhi > rhi || (lhi == rhi && llo > rlo)) ? 1ull : 0ull;
+}
+
+// composite sort key: (max_cnt - cnt) in the high part, key in the low `key_bits` bits, so that an
+// ascending sort gives count descending, key ascending
+__global__ void composite_kernel(const unsigned long long* __restrict__ cnt, uint64_t n, unsigned long long max_cnt,
+                                 int key_bits, const unsigned long long* __restrict__ flag /* nullable */,
+                                 const unsigned long long* __restrict__ pos /* exclusive scan of flag */,
+                                 unsigned long long* __restrict__ comp, uint32_t* __restrict__ payload)
+{
+    uint64_t k = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (k >= n) return;
+    uint64_t o = k;
+    if (flag) {
+        if (!flag[k]) return;
+        o = pos[k];
+    }
+    comp[o] = ((max_cnt - cnt[k]) << key_bits) | k;
+    payload[o] = (uint32_t)k;
+}
+
+extern "C" nups_status nups_select_hot(nups_store* s, int by_topk, uint64_t param, uint32_t* d_keys_out,
+                                       uint64_t* h_n_out, void* stream)
+{
+    if (!s || !d_keys_out || !h_n_out) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint64_t n = s->num_keys;
+    *h_n_out = 0;
+    CK(cudaMemsetAsync(&s->st->tmp[0], 0, 16, st));
+    count_sum_max_kernel<<<grid_for(n, 256, (unsigned)s->sm_count * 8), 256, 0, st>>>(s->cnt, n, s->st);
+    LAUNCH_CHECK(s);
+    unsigned long long sm[2];
+    CK(cudaMemcpyAsync(sm, &s->st->tmp[0], 16, cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    unsigned long long total = sm[0], max_cnt = sm[1];
+    int key_bits = bits_for(n - 1), cnt_bits = bits_for(max_cnt);
+    if (key_bits + cnt_bits > 64) return NUPS_ESTATE;
+    size_t need = 4 * align256(n * 8) + 2 * align256(n * 4) + nups_sort_scratch_bytes(n) + nups_scan_scratch_bytes(n) + 256;
+    char* sc;
+    nups_status rc = nups_scratch(s, need, &sc);
+    if (rc != NUPS_OK) return rc;
+    unsigned long long* flag = (unsigned long long*)sc; sc += align256(n * 8);
+    unsigned long long* pos = (unsigned long long*)sc; sc += align256(n * 8);
+    unsigned long long* c0 = (unsigned long long*)sc; sc += align256(n * 8);
+    unsigned long long* c1 = (unsigned long long*)sc; sc += align256(n * 8);
+    uint32_t* p0 = (uint32_t*)sc; sc += align256(n * 4);
+    uint32_t* p1 = (uint32_t*)sc; sc += align256(n * 4);
+    unsigned long long* d_m = (unsigned long long*)sc; sc += 256;
+    uint64_t m = n;
+    if (!by_topk) {
+        threshold_flag_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->cnt, n, param, total, flag);
+        LAUNCH_CHECK(s);
+        rc = nups_scan_u64(s, flag, pos, n, d_m, sc, st);
+        if (rc != NUPS_OK) return rc;
+        unsigned long long hm = 0;
+        CK(cudaMemcpyAsync(&hm, d_m, 8, cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+        m = hm;
+        if (m == 0) return NUPS_OK;
+        composite_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->cnt, n, max_cnt, key_bits, flag, pos, c0, p0);
+    } else {
+        if (param == 0) return NUPS_OK;
+        composite_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->cnt, n, max_cnt, key_bits, nullptr, nullptr, c0, p0);
+    }
+    LAUNCH_CHECK(s);
+    char* sort_sc = sc + nups_scan_scratch_bytes(n);
+    rc = nups_sort_pairs(s, c0, p0, c1, p1, m, key_bits + cnt_bits, sort_sc, st);
+    if (rc != NUPS_OK) return rc;
+    uint64_t take = by_topk ? (param < m ? param : m) : m;
+    CK(cudaMemcpyAsync(d_keys_out, p1, take * 4, cudaMemcpyDeviceToDevice, st));
+    CK(cudaStreamSynchronize(st));
+    *h_n_out = take;
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-key management
+// ---------------------------------------------------------------------------------------------
+// REPLICATE, pass 1: every listed key that is not hot yet is claimed by its first list position.
+// slot_of holds: >= 0 hot slot; -1 single; <= -2 a claim by list position p encoded as -(p + 2).
+__global__ void claim_kernel(int* slot_of, uint64_t num_keys, const uint32_t* __restrict__ keys, uint64_t n, DevStat* st)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint32_t k = keys[i];
+    if (k >= num_keys) { atomicCAS(&st->status, 0, NUPS_EKEY); return; }
+    int mine = -(int)(i + 2);
+    int cur = slot_of[k];
+    while (cur < 0 && (cur == -1 || cur < mine)) {          // smaller position = larger (closer to -2) code
+        int prev = atomicCAS(&slot_of[k], cur, mine);
+        if (prev == cur) break;
+        cur = prev;
+    }
+}
+__global__ void winner_flag_kernel(const int* __restrict__ slot_of, uint64_t num_keys, const uint32_t* __restrict__ keys,
+                                   uint64_t n, unsigned long long* __restrict__ flag)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint32_t k = keys[i];
+    flag[i] = (k < num_keys && slot_of[k] == -(int)(i + 2)) ? 1ull : 0ull;
+}
+__global__ void assign_slots_kernel(int* slot_of, uint32_t* hot_bits, uint32_t* hot_keys, const uint32_t* __restrict__ keys,
+                                    uint64_t n, const unsigned long long* __restrict__ flag,
+                                    const unsigned long long* __restrict__ pos, uint64_t H_old)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n || !flag[i]) return;
+    uint32_t k = keys[i];
+    uint64_t slot = H_old + pos[i];
+    slot_of[k] = (int)slot;
+    hot_keys[slot] = k;
+    atomicOr(&hot_bits[k >> 5], 1u << (k & 31));
+}
+// SINGLE: drop the listed keys, then renumber the surviving slots in their old order.
+__global__ void demote_kernel(int* slot_of, uint32_t* hot_bits, uint64_t num_keys, const uint32_t* __restrict__ keys,
+                              uint64_t n, DevStat* st)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint32_t k = keys[i];
+    if (k >= num_keys) { atomicCAS(&st->status, 0, NUPS_EKEY); return; }
+    slot_of[k] = -1;
+    atomicAnd(&hot_bits[k >> 5], ~(1u << (k & 31)));
+}
+__global__ void alive_flag_kernel(const int* __restrict__ slot_of, const uint32_t* __restrict__ hot_keys, uint64_t H,
+                                  unsigned long long* __restrict__ flag)
+{
+    uint64_t sl = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sl >= H) return;
+    flag[sl] = slot_of[hot_keys[sl]] >= 0 ? 1ull : 0ull;
+}
+__global__ void renumber_kernel(int* slot_of, const uint32_t* __restrict__ hot_keys, uint32_t* __restrict__ hot_keys_new,
+                                uint64_t H, const unsigned long long* __restrict__ flag,
+                                const unsigned long long* __restrict__ pos)
+{
+    uint64_t sl = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (sl >= H || !flag[sl]) return;
+    uint32_t k = hot_keys[sl];
+    slot_of[k] = (int)pos[sl];
+    hot_keys_new[pos[sl]] = k;
+}
+
+static nups_status grow_hot(nups_store* s, uint64_t need)
+{
+    if (need <= s->Hcap) return NUPS_OK;
+    uint64_t cap = need + need / 4 + 16;
+    uint32_t* hk = nullptr;
+    uint32_t* dirty = nullptr;
+    float *dv = nullptr, *da = nullptr;
+    size_t slab = (size_t)s->R * cap * s->L * sizeof(float);
+    bool ok = cudaMalloc(&hk, cap * 4) == cudaSuccess && cudaMalloc(&dirty, cap * 4) == cudaSuccess &&
+              cudaMalloc(&dv, slab) == cudaSuccess && (!s->acc || cudaMalloc(&da, slab) == cudaSuccess);
+    if (!ok) {
+        cudaGetLastError();
+        cudaFree(hk); cudaFree(dirty); cudaFree(dv); cudaFree(da);
+        return NUPS_ENOMEM;
+    }
+    // pending updates are all zero here (the caller merged them), so fresh zeroed slabs are enough
+    if (s->H) CK(cudaMemcpy(hk, s->hot_keys, s->H * 4, cudaMemcpyDeviceToDevice));
+    CK(cudaMemset(dirty, 0, cap * 4));
+    CK(cudaMemset(dv, 0, slab));
+    if (da) CK(cudaMemset(da, 0, slab));
+    CK(cudaDeviceSynchronize());
+    cudaFree(s->hot_keys); cudaFree(s->dirty); cudaFree(s->dval); cudaFree(s->dacc);
+    s->hot_keys = hk; s->dirty = dirty; s->dval = dv; s->dacc = da; s->Hcap = cap;
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_set_management(nups_store* s, const uint32_t* d_keys, uint64_t n, int technique, void* stream)
+{
+    if (!s || (n && !d_keys) || (technique != NUPS_SINGLE && technique != NUPS_REPLICATE)) return NUPS_EINVAL;
+    if (n >= (1ull << 31) - 2) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    nups_status rc = nups_sync_internal(s, st);
+    if (rc != NUPS_OK) return rc;
+    CK(cudaStreamSynchronize(st));
+    if (n == 0) return NUPS_OK;
+    uint64_t m = technique == NUPS_REPLICATE ? n : (s->H > n ? s->H : n);
+    size_t need = 2 * align256(m * 8) + align256(m * 4) + nups_scan_scratch_bytes(m) + 256;
+    char* sc;
+    rc = nups_scratch(s, need, &sc);
+    if (rc != NUPS_OK) return rc;
+    unsigned long long* flag = (unsigned long long*)sc; sc += align256(m * 8);
+    unsigned long long* pos = (unsigned long long*)sc; sc += align256(m * 8);
+    uint32_t* hk_new = (uint32_t*)sc; sc += align256(m * 4);
+    unsigned long long* d_total = (unsigned long long*)sc; sc += 256;
+    unsigned long long total = 0;
+    if (technique == NUPS_REPLICATE) {
+        if (s->H + n >= (1ull << 31)) return NUPS_ENOMEM;
+        rc = grow_hot(s, s->H + n);
+        if (rc != NUPS_OK) return rc;
+        claim_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->slot_of, s->num_keys, d_keys, n, s->st);
+        LAUNCH_CHECK(s);
+        winner_flag_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->slot_of, s->num_keys, d_keys, n, flag);
+        LAUNCH_CHECK(s);
+        rc = nups_scan_u64(s, flag, pos, n, d_total, sc, st);
+        if (rc != NUPS_OK) return rc;
+        assign_slots_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->slot_of, s->hot_bits, s->hot_keys, d_keys, n, flag, pos, s->H);
+        LAUNCH_CHECK(s);
+        CK(cudaMemcpyAsync(&total, d_total, 8, cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+        s->H += total;
+    } else {
+        demote_kernel<<<grid_for(n, 256), 256, 0, st>>>(s->slot_of, s->hot_bits, s->num_keys, d_keys, n, s->st);
+        LAUNCH_CHECK(s);
+        if (s->H == 0) return NUPS_OK;
+        alive_flag_kernel<<<grid_for(s->H, 256), 256, 0, st>>>(s->slot_of, s->hot_keys, s->H, flag);
+        LAUNCH_CHECK(s);
+        rc = nups_scan_u64(s, flag, pos, s->H, d_total, sc, st);
+        if (rc != NUPS_OK) return rc;
+        renumber_kernel<<<grid_for(s->H, 256), 256, 0, st>>>(s->slot_of, s->hot_keys, hk_new, s->H, flag, pos);
+        LAUNCH_CHECK(s);
+        CK(cudaMemcpyAsync(&total, d_total, 8, cudaMemcpyDeviceToHost, st));
+        CK(cudaStreamSynchronize(st));
+        if (total) CK(cudaMemcpyAsync(s->hot_keys, hk_new, total * 4, cudaMemcpyDeviceToDevice, st));
+        CK(cudaStreamSynchronize(st));
+        s->H = total;
+    }
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_get_hot(nups_store* s, uint64_t* h_n_out, uint32_t* d_keys_out, void* stream)
+{
+    if (!s || !h_n_out) return NUPS_EINVAL;
+    *h_n_out = s->H;
+    if (d_keys_out && s->H) {
+        CK(cudaMemcpyAsync(d_keys_out, s->hot_keys, s->H * 4, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+        CK(cudaStreamSynchronize((cudaStream_t)stream));
+    }
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// ownership (the one-machine reading of "allocated at node q")
+// ---------------------------------------------------------------------------------------------
+__global__ void localize_request_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, uint32_t* req,
+                                        uint64_t req_cap)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint32_t k = keys[i];
+    if (k >= v.num_keys) { flag_bad_key(v); return; }
+    uint32_t q = worker_of_item(i, n, v.R);
+    atomicMax(v.pending + k, (int)q);
+    unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
+    if (at < req_cap) req[at] = k;
+}
+
+// requests of one call are applied in the order they were made, so the last one wins; workers are
+// visited in ascending order by every caller, hence the largest requesting worker gets the key
+__global__ void localize_apply_kernel(View v, const uint32_t* __restrict__ req, uint64_t max_requests)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= max_requests || i >= v.st->req_count) return;
+    uint32_t k = req[i];
+    int p = v.pending[k];
+    if (p >= 0) {
+        if (!key_is_hot(v, k)) v.owner[k] = (uint8_t)p;
+        v.pending[k] = -1;
+    }
+}
+__global__ void reset_req_kernel(DevStat* st) { st->req_count = 0; }
+
+nups_status nups_localize_apply(nups_store* s, uint64_t max_requests, cudaStream_t st)
+{
+    if (!s->owner || max_requests == 0) return NUPS_OK;
+    localize_apply_kernel<<<grid_for(max_requests, 256), 256, 0, st>>>(nups_view(s), s->req_keys, max_requests);
+    LAUNCH_CHECK(s);
+    reset_req_kernel<<<1, 1, 0, st>>>(s->st);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_localize(nups_store* s, const uint32_t* d_keys, uint64_t n, void* stream)
+{
+    if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
+    if (!s->owner || n == 0) return NUPS_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    nups_status rc = nups_req_reserve(s, n);
+    if (rc != NUPS_OK) return rc;
+    localize_request_kernel<<<grid_for(n, 256), 256, 0, st>>>(nups_view(s), d_keys, n, s->req_keys, s->req_cap);
+    LAUNCH_CHECK(s);
+    return nups_localize_apply(s, n, st);
+}
+
+__global__ void owner_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, int* __restrict__ out)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    uint32_t k = keys[i];
+    int r;
+    if (k >= v.num_keys) r = -1;
+    else if (key_is_hot(v, k)) r = -2;
+    else if (!v.owner) r = -3;
+    else r = v.owner[k] == NUPS_OWNER_DEFAULT ? (int)(k % v.R) : (int)v.owner[k];
+    out[i] = r;
+}
+
+extern "C" nups_status nups_get_owner(nups_store* s, const uint32_t* d_keys, uint64_t n, int32_t* d_out, void* stream)
+{
+    if (!s || (n && (!d_keys || !d_out))) return NUPS_EINVAL;
+    if (n == 0) return NUPS_OK;
+    owner_kernel<<<grid_for(n, 256), 256, 0, (cudaStream_t)stream>>>(nups_view(s), d_keys, n, d_out);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// status and statistics
+// ---------------------------------------------------------------------------------------------
+extern "C" nups_status nups_status_check(nups_store* s, void* stream)
+{
+    if (!s) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    int code = 0;
+    CK(cudaMemcpyAsync(&code, &s->st->status, sizeof(int), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    if (code != 0) {
+        CK(cudaMemsetAsync(&s->st->status, 0, sizeof(int), st));
+        CK(cudaStreamSynchronize(st));
+    }
+    return (nups_status)code;
+}
+
+extern "C" nups_status nups_get_stats(nups_store* s, uint64_t* h_out, void* stream)
+{
+    if (!s || !h_out) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    DevStat d;
+    CK(cudaMemcpyAsync(&d, s->st, sizeof(DevStat), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    h_out[0] = s->steps; h_out[1] = s->syncs; h_out[2] = s->launches;
+    h_out[3] = d.hot_hits; h_out[4] = d.cold_hits; h_out[5] = s->H; h_out[6] = 0; h_out[7] = 0;
+    return NUPS_OK;
+}

@@ -1,0 +1,185 @@
+"""CUDA path vs oracle: the three workload steps (deterministic mode: values within the stated
+tolerance, negatives and access counts bit-exact; fast mode: loss within 1 %)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import BOUNDED, CONFORM, LONGTERM, REPLICATE
+from paper_2104_00501_b200 import inputs
+from tests.common import ATOL, RTOL, dev_f32, dev_keys, host_keys, make_pair, tables_close
+
+pytestmark = pytest.mark.gpu
+
+
+def loss_buf():
+    return torch.zeros(1, dtype=torch.float32, device="cuda")
+
+
+def sgns_data(V, n_tokens, seed):
+    c, ctx, counts = inputs.sgns_batch_stream(V, n_tokens, 1.1, seed)
+    return inputs.u32(c), inputs.u32(ctx), inputs.integer_weights(counts).numpy().astype(np.uint32)
+
+
+@pytest.mark.parametrize("L,level,hot_n,interval", [(64, CONFORM, 0, 1), (64, CONFORM, 20, 1), (300, BOUNDED, 20, 3),
+                                                    (100, LONGTERM, 10, 2), (8, CONFORM, 5, 1)])
+def test_sgns_deterministic_parity(L, level, hot_n, interval):
+    V, K, R, batch = 300, 3, 4, 250
+    c, ctx, w = sgns_data(V, 400, 0)
+    init = inputs.normal_init(2 * V, L, 0.1, 0)
+    o, s = make_pair(2 * V, L, R=R, init=init, deterministic=True, sync_interval=interval, count_accesses=True,
+                     track_ownership=True)
+    if hot_n:
+        o.count_accesses(np.concatenate([c, ctx]))
+        s.count_accesses(dev_keys(np.concatenate([c, ctx])))
+        hot = o.select_hot(True, hot_n)
+        assert np.array_equal(host_keys(s.select_hot(True, hot_n)), hot)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(V, w, V, level, U=4, G=25, seed=3)
+    ds = s.register_distribution(V, dev_keys(w), V, level, U=4, G=25, seed=3)
+    lb = loss_buf()
+    for b in range(0, len(c) - batch, batch):
+        lo, negs = o.step_sgns(c[b:b + batch], ctx[b:b + batch], do, K, 0.05, return_negatives=True)
+        s.step_sgns(dev_keys(c[b:b + batch]), dev_keys(ctx[b:b + batch]), ds, K, 0.05, lb)
+        assert np.array_equal(host_keys(s.last_negatives()), negs)
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    o.sync()
+    s.sync()
+    tables_close(o, s)
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+    assert s.stats()["steps"] == o.stats()["steps"] and s.stats()["syncs"] == o.stats()["syncs"]
+    assert np.abs(o.table() - init).max() > 1e-3
+
+
+def test_sgns_ragged_and_single_item_batches():
+    V, L, K = 50, 12, 2
+    c, ctx, w = sgns_data(V, 80, 1)
+    init = inputs.normal_init(2 * V, L, 0.2, 1)
+    o, s = make_pair(2 * V, L, R=8, init=init, deterministic=True)
+    do = o.register_distribution(V, w, V, CONFORM, seed=1)
+    ds = s.register_distribution(V, dev_keys(w), V, CONFORM, seed=1)
+    lb = loss_buf()
+    at = 0
+    for n in (1, 3, 33, 129, 7):
+        lo = o.step_sgns(c[at:at + n], ctx[at:at + n], do, K, 0.1)
+        s.step_sgns(dev_keys(c[at:at + n]), dev_keys(ctx[at:at + n]), ds, K, 0.1, lb)
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+        at += n
+    tables_close(o, s)
+
+
+@pytest.mark.parametrize("L,hot_n,K", [(500, 0, 10), (500, 30, 10), (8, 4, 3), (64, 10, 0)])
+def test_complex_deterministic_parity(L, hot_n, K):
+    E, Rl, R, batch = 400, 12, 4, 100
+    h, r, t = [inputs.u32(x) for x in inputs.kge_triples(300, E, Rl, 0.9, 1.2, 0)]
+    rng = np.random.default_rng(0)
+    init = rng.normal(0, 0.1, size=(E + Rl, L)).astype(np.float32)
+    o, s = make_pair(E + Rl, L, R=R, init=init, deterministic=True, with_adagrad=True, count_accesses=True)
+    if hot_n:
+        hot = np.concatenate([np.arange(E, E + Rl), np.unique(h)[:hot_n]]).astype(np.uint32)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(0, None, E, CONFORM, seed=9)
+    ds = s.register_distribution(0, None, E, CONFORM, seed=9)
+    lb = loss_buf()
+    for b in range(0, 300, batch):
+        sl = slice(b, b + batch)
+        lo, negs = o.step_complex(h[sl], r[sl], t[sl], do, K, 0.1, 1e-10, return_negatives=True)
+        s.step_complex(dev_keys(h[sl]), dev_keys(r[sl]), dev_keys(t[sl]), ds, K, 0.1, 1e-10, lb)
+        assert np.array_equal(host_keys(s.last_negatives()), negs)
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    o.sync()
+    s.sync()
+    # the very first AdaGrad step divides by sqrt(g^2): |step| = lr whatever g, so a gradient of
+    # 1e-9 moves a value by 0.1 -- compare where the oracle's gradient is not vanishing
+    tables_close(o, s, 1, rtol=1e-4, atol=1e-9)
+    big = o.table(1) > 1e-8
+    got = s.read_table(0).cpu().numpy()
+    np.testing.assert_allclose(got[big], o.table(0)[big], rtol=1e-4, atol=1e-5)
+    assert big.mean() > 0.05
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+
+
+@pytest.mark.parametrize("L,hot_n", [(100, 0), (100, 25), (4, 3)])
+def test_mf_deterministic_parity(L, hot_n):
+    M, N, R, batch = 500, 200, 4, 512
+    i, j, x = inputs.mf_cells(2048, M, N, 0.8, max(L // 4, 2), 0.1, 0)
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    init = np.random.default_rng(0).normal(0, 0.3, size=(M + N, L)).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, init=init, deterministic=True, count_accesses=True)
+    if hot_n:
+        o.count_accesses(np.concatenate([i, j]))
+        s.count_accesses(dev_keys(np.concatenate([i, j])))
+        hot = o.select_hot(True, hot_n)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    lb = loss_buf()
+    for b in range(0, 2048, batch):
+        sl = slice(b, b + batch)
+        lo = o.step_mf(i[sl], j[sl], x[sl], 0.01, 0.01)
+        s.step_mf(dev_keys(i[sl]), dev_keys(j[sl]), dev_f32(x[sl]), 0.01, 0.01, lb)
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    o.sync()
+    s.sync()
+    tables_close(o, s)
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+
+
+def test_fast_mode_reaches_the_oracles_loss_within_one_percent():
+    # replicated + asynchronous mode: same number of epochs, final loss within 1 % of the oracle's
+    V, L, K, R, batch = 500, 32, 3, 8, 256
+    c, ctx, w = sgns_data(V, 4000, 2)
+    init = inputs.normal_init(2 * V, L, 0.1, 2)
+    o, s = make_pair(2 * V, L, R=R, init=init, deterministic=False, sync_interval=4)
+    o.count_accesses(np.concatenate([c, ctx]))
+    hot = o.select_hot(True, 20)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(V, w, V, BOUNDED, U=4, G=50, seed=3)
+    ds = s.register_distribution(V, dev_keys(w), V, BOUNDED, U=4, G=50, seed=3)
+    lb = loss_buf()
+    lo_hist, ls_hist = [], []
+    nb = (len(c) // batch)
+    for epoch in range(2):
+        for b in range(nb):
+            sl = slice(b * batch, (b + 1) * batch)
+            lo_hist.append(o.step_sgns(c[sl], ctx[sl], do, K, 0.025))
+            s.step_sgns(dev_keys(c[sl]), dev_keys(ctx[sl]), ds, K, 0.025, lb)
+            ls_hist.append(lb.item())
+    lo, ls = np.mean(lo_hist[-nb:]), np.mean(ls_hist[-nb:])
+    assert abs(ls - lo) <= 0.01 * lo
+    assert lo < 0.95 * np.mean(lo_hist[:20])
+    assert s.status_check() == 0
+
+
+def test_tiny_sgns_config_full_epoch():
+    # config 0: 10,000-word vocabulary (20,000 keys), dim 64, N(0, 0.01) start values, 256k pairs
+    # with Zipf(1.1) words, batch 256, 3 CONFORM negatives from unigram^0.75, lr 0.025, top-100 keys
+    # replicated, sync every step, one epoch, seed 0
+    V, L, K, R, batch = 10000, 64, 3, 8, 256
+    c, ctx, counts = inputs.sgns_batch_stream(V, 25700, 1.1, 0)
+    c, ctx = inputs.u32(c)[:256000], inputs.u32(ctx)[:256000]
+    w = inputs.integer_weights(counts).numpy().astype(np.uint32)
+    init = inputs.normal_init(2 * V, L, 0.01, 0)
+    o, s = make_pair(2 * V, L, R=R, init=init, deterministic=True, sync_interval=1, count_accesses=True)
+    both = np.concatenate([c, ctx])
+    o.count_accesses(both)
+    s.count_accesses(dev_keys(both))
+    hot = o.select_hot(True, 100)
+    assert np.array_equal(host_keys(s.select_hot(True, 100)), hot)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(V, w, V, CONFORM, seed=0)
+    ds = s.register_distribution(V, dev_keys(w), V, CONFORM, seed=0)
+    lb = torch.zeros(1000, dtype=torch.float32, device="cuda")
+    dc, dx = dev_keys(c), dev_keys(ctx)
+    lo = []
+    for b in range(1000):
+        sl = slice(b * batch, (b + 1) * batch)
+        lo.append(o.step_sgns(c[sl], ctx[sl], do, K, 0.025))
+        s.step_sgns(dc[sl], dx[sl], ds, K, 0.025, lb[b:b + 1])
+    ls = lb.cpu().numpy()
+    np.testing.assert_allclose(ls, np.array(lo, np.float32), rtol=1e-5)
+    tables_close(o, s)
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+    assert s.status_check() == 0

@@ -1,0 +1,44 @@
+"""The C-ABI library builds, loads and exports every symbol the public header declares (no GPU needed)."""
+import ctypes
+import os
+import re
+
+from paper_2104_00501_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "nups.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(nups_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_builds_and_exports_every_declared_symbol():
+    path = build.build_library()
+    lib = ctypes.CDLL(path)
+    names = declared_symbols()
+    assert len(names) >= 25
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in include/nups.h but not exported"
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_binding_fails_loudly_without_a_device():
+    import pytest
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a device is present")
+    with pytest.raises(binding.NupsError) as e:
+        binding.Store(10, 4)
+    assert e.value.code == binding.ECUDA
+
+
+def test_strerror_and_argument_checks_need_no_device():
+    lib = binding.load()
+    assert lib.nups_strerror(0) == b"ok"
+    assert b"invalid" in lib.nups_strerror(binding.EINVAL)
+    h = ctypes.c_void_p()
+    assert lib.nups_create(0, 4, None, ctypes.byref(h)) == binding.EINVAL
+    assert lib.nups_create(10, 3, None, ctypes.byref(h)) == binding.EINVAL      # rows must be 16-byte multiples
+    assert lib.nups_create(1 << 33, 4, None, ctypes.byref(h)) == binding.EINVAL
