@@ -91,6 +91,11 @@ nups_status nups_destroy(nups_store* store);
  * include updates that are still pending in replicas.                         */
 nups_status nups_table_ptr(nups_store* store, int which, float** h_ptr, uint64_t* h_row_stride_floats);
 
+/* Copy a whole table between the store and a caller buffer d_buf of
+ * num_keys * value_len floats, in stream order: to_store = 1 loads start values
+ * into the table, to_store = 0 takes a snapshot of it.                         */
+nups_status nups_table_copy(nups_store* store, int which, float* d_buf, int to_store, void* stream);
+
 /* Fill a table with seeded start values: element e gets
  * (int(bits 8..31 of word e mod 4 of Philox4x32-10(counter = (e/4, 0, which, 3),
  *  key = seed)) - 2^23) * (scale * 2^-23), uniform in [-scale, scale).         */
@@ -141,8 +146,9 @@ nups_status nups_get_counts(nups_store* store, uint64_t* d_counts_out, void* str
  * mean (the paper's heuristic uses 100).  by_topk = 1: the `param` most frequent
  * keys.  Output order: count descending, smaller key first among equals.
  * d_keys_out must hold min(param, num_keys) keys for by_topk = 1 and num_keys
- * for the threshold rule; *h_n_out receives the number written.  Counts must be
- * below 2^32 (NUPS_ESTATE otherwise).  Synchronises the stream.               */
+ * for the threshold rule; *h_n_out receives the number written.  The largest
+ * count and num_keys - 1 must fit 64 bits together (NUPS_ESTATE otherwise).
+ * Synchronises the stream.                                                    */
 nups_status nups_select_hot(nups_store* store, int by_topk, uint64_t param, uint32_t* d_keys_out, uint64_t* h_n_out,
                             void* stream);
 

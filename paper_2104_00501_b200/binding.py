@@ -20,7 +20,7 @@ SINGLE, REPLICATE = 0, 1
 CONFORM, BOUNDED, LONGTERM, NONCONFORM = 1, 2, 3, 4
 
 EXPORTS = [
-    "nups_create", "nups_destroy", "nups_table_ptr", "nups_init_uniform", "nups_pull", "nups_pull2", "nups_push",
+    "nups_create", "nups_destroy", "nups_table_ptr", "nups_table_copy", "nups_init_uniform", "nups_pull", "nups_pull2", "nups_push",
     "nups_push2", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_step_complex", "nups_step_mf",
@@ -63,6 +63,7 @@ def load(build_if_missing: bool = True):
         "nups_create": [u64, u32, C.POINTER(Config), C.POINTER(vp)],
         "nups_destroy": [vp],
         "nups_table_ptr": [vp, C.c_int, C.POINTER(vp), C.POINTER(u64)],
+        "nups_table_copy": [vp, C.c_int, vp, C.c_int, vp],
         "nups_init_uniform": [vp, C.c_int, u64, f32, vp],
         "nups_pull": [vp, vp, u64, vp, vp],
         "nups_pull2": [vp, vp, u64, vp, vp, vp],
@@ -162,21 +163,15 @@ class Store:
 
     def write_table(self, which, values):
         """Copy host (or device) values [num_keys, L] into a table."""
-        p, _ = self.table_ptr(which)
-        src = torch.as_tensor(values, dtype=torch.float32).contiguous()
+        src = torch.as_tensor(values, dtype=torch.float32).contiguous().cuda()
         assert src.shape == (self.num_keys, self.L)
-        src = src.cuda()
+        self._chk(self._l.nups_table_copy(self._s, which, _ptr(src), 1, _stream()), "nups_table_copy")
         torch.cuda.current_stream().synchronize()
-        rc = torch.cuda.cudart().cudaMemcpy(p, src.data_ptr(), src.numel() * 4, 3)   # 3 = device to device
-        assert int(rc) == 0
 
     def read_table(self, which=0, rows=None):
-        """Copy a table (or the given rows of it) out to a new CUDA tensor."""
-        p, _ = self.table_ptr(which)
+        """Snapshot of a table (or of the given rows of it) as a new CUDA tensor."""
         out = torch.empty((self.num_keys, self.L), dtype=torch.float32, device=self.device)
-        torch.cuda.current_stream().synchronize()
-        rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), p, out.numel() * 4, 3)
-        assert int(rc) == 0
+        self._chk(self._l.nups_table_copy(self._s, which, _ptr(out), 0, _stream()), "nups_table_copy")
         return out if rows is None else out[rows]
 
     def init_uniform(self, which, seed, scale):
@@ -297,12 +292,12 @@ class Store:
     def last_negatives(self):
         p, n = C.c_void_p(), C.c_uint64()
         self._chk(self._l.nups_last_negatives(self._s, C.byref(p), C.byref(n)), "nups_last_negatives")
-        out = torch.empty(max(n.value, 1), dtype=torch.int32, device=self.device)
-        if n.value:
-            torch.cuda.current_stream().synchronize()
-            rc = torch.cuda.cudart().cudaMemcpy(out.data_ptr(), p.value, n.value * 4, 3)
-            assert int(rc) == 0
-        return out[:n.value]
+        if not n.value:
+            return torch.empty(0, dtype=torch.int32, device=self.device)
+
+        class _Raw:        # the library's buffer seen through the CUDA array interface, then copied out
+            __cuda_array_interface__ = {"shape": (n.value,), "typestr": "<i4", "data": (p.value, False), "version": 2}
+        return torch.as_tensor(_Raw(), device=self.device).clone()
 
     # -- status -------------------------------------------------------------------------
     def status_check(self):

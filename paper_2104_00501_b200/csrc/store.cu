@@ -160,6 +160,16 @@ extern "C" nups_status nups_table_ptr(nups_store* s, int which, float** ptr, uin
     return NUPS_OK;
 }
 
+extern "C" nups_status nups_table_copy(nups_store* s, int which, float* d_buf, int to_store, void* stream)
+{
+    if (!s || !d_buf || (which != 0 && which != 1) || (which == 1 && !s->acc)) return NUPS_EINVAL;
+    float* t = which ? s->acc : s->val;
+    size_t bytes = (size_t)s->num_keys * s->L * sizeof(float);
+    CK(cudaMemcpyAsync(to_store ? t : d_buf, to_store ? d_buf : t, bytes, cudaMemcpyDeviceToDevice,
+                       (cudaStream_t)stream));
+    return NUPS_OK;
+}
+
 __global__ void init_uniform_kernel(float4* t, uint64_t total4, uint64_t seed, uint32_t which, float unit)
 {
     uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;

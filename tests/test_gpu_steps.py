@@ -143,8 +143,8 @@ def test_fast_mode_reaches_the_oracles_loss_within_one_percent():
     for epoch in range(2):
         for b in range(nb):
             sl = slice(b * batch, (b + 1) * batch)
-            lo_hist.append(o.step_sgns(c[sl], ctx[sl], do, K, 0.025))
-            s.step_sgns(dev_keys(c[sl]), dev_keys(ctx[sl]), ds, K, 0.025, lb)
+            lo_hist.append(o.step_sgns(c[sl], ctx[sl], do, K, 0.01))
+            s.step_sgns(dev_keys(c[sl]), dev_keys(ctx[sl]), ds, K, 0.01, lb)
             ls_hist.append(lb.item())
     lo, ls = np.mean(lo_hist[-nb:]), np.mean(ls_hist[-nb:])
     assert abs(ls - lo) <= 0.01 * lo
