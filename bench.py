@@ -1,0 +1,349 @@
+#!/usr/bin/env python
+"""Benchmark of the NuPS sparse access path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Workload: skip-gram with negative sampling on a 1M-word vocabulary, dimension 300
+(input and output vectors in one 2M-key store), token stream ~ Zipf(1.0), window 5, 3 negatives per
+pair from unigram^0.75 under pooled reuse (BOUNDED, U = 16, G = 250), batches of 4096 pairs, top 1 %
+of keys replicated, replicas merged every 16 batches, fast (atomic) mode.  One step = one batch through
+the whole path: PrepareSample, PullSample, pulls, dot products, pushes, localize bookkeeping, and the
+periodic merge.  Metric: key accesses per second (2 direct pulls + 3 sampled pulls + 5 pushes per pair).
+
+With N > 1 every rank runs an independent replica of the workload on its own GPU (the path has no
+exchange step on one node); the aggregate is total accesses over the slowest rank's time.
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2104_00501_b200 import inputs  # noqa: E402
+
+VOCAB, DIM, BATCH, NEG, WINDOW = 1_000_000, 300, 4096, 3, 5
+U_REUSE, G_POOL, SYNC_EVERY, WORKERS, LR = 16, 250, 16, 8, 0.025
+HOT_FRACTION = 0.01
+TOKENS = 100_000_000
+ACCESSES_PER_PAIR = 2 + NEG + (NEG + 2)          # direct pulls + sampled pulls + pushes
+UPDATES_PER_PAIR = NEG + 2
+MAX_DISTINCT_BATCHES = 4096
+
+# DRAM traffic of one launch of the fused step kernel, from an ncu capture (dram__bytes_read.sum +
+# dram__bytes_write.sum); valid only for the kernel source it was captured on.
+NCU_TRAFFIC = {"bytes_per_launch": None, "steps_cu_sha1": None}
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock and throttle-reason samples while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.t = threading.Thread(target=self._read, daemon=True)
+            self.t.start()
+        except Exception:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *a):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+                for n, v in zip(names, r[2:6]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            except Exception:
+                pass
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# --------------------------------------------------------------------------------------------
+# workload construction (seeded, synthetic; stands in for the One Billion Word Benchmark)
+# --------------------------------------------------------------------------------------------
+def make_sgns_data(device, n_batches, seed=0, store=None):
+    """Token stream in chunks: word counts, the pairs of the first batches, integer sampling weights.
+    With a store, every token is also counted as an access to its input key and to its output key."""
+    cdf = inputs.zipf_cdf(VOCAB, 1.0, device)
+    counts = torch.zeros(VOCAB, dtype=torch.int64, device=device)
+    chunk = 10_000_000
+    first = None
+    for i in range(TOKENS // chunk):
+        t = inputs.zipf_keys(chunk, VOCAB, 1.0, seed * 1000 + i, device, cdf=cdf)
+        counts += torch.bincount(t, minlength=VOCAB)
+        if store is not None:
+            t32 = t.to(torch.int32)
+            store.count_accesses(t32)
+            store.count_accesses(t32 + VOCAB)
+        if i == 0:
+            first = t
+    need = n_batches * BATCH
+    tok = first[: need // (2 * WINDOW) + 4 * WINDOW]
+    c, o = inputs.skipgram_pairs(tok, WINDOW)
+    assert c.numel() >= need, "token prefix too short for the requested number of batches"
+    c, o = c[:need].to(torch.int32).contiguous(), (o[:need] + VOCAB).to(torch.int32).contiguous()
+    weights = inputs.integer_weights(counts).to(torch.int32)
+    return c, o, counts, weights
+
+
+def build_store(binding, device, n_batches, seed, deterministic=False):
+    s = binding.Store(2 * VOCAB, DIM, workers=WORKERS, sync_interval=SYNC_EVERY, deterministic=deterministic,
+                      track_ownership=False)
+    s.init_uniform(0, 1, 0.5 / DIM)
+    c, o, counts, weights = make_sgns_data(device, n_batches, seed, store=s)
+    hot = s.select_hot(True, int(HOT_FRACTION * 2 * VOCAB))          # the most frequently accessed 1 % of keys
+    s.set_management(hot, binding.REPLICATE)
+    dist = s.register_distribution(VOCAB, weights.contiguous(), VOCAB, binding.BOUNDED, U=U_REUSE, G=G_POOL, seed=7)
+    return s, dist, hot.long(), c, o, weights
+
+
+def run_ours(args, rank, world, device):
+    from paper_2104_00501_b200 import binding
+    hbm_peak, peak_kind = peaks()
+    nb = min(args.steps + args.warmup, MAX_DISTINCT_BATCHES)
+    s, dist, hot, c, o, weights = build_store(binding, device, nb, seed=rank)
+    loss = torch.zeros(1, dtype=torch.float32, device=device)
+
+    def batch(i):
+        j = (i % nb) * BATCH
+        return c[j:j + BATCH], o[j:j + BATCH]
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        s.step_sgns(*batch(i), dist, NEG, LR, loss)
+    launches0 = s.stats()["launches"]
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    with ClockSampler(torch.cuda.current_device()) as clk:
+        ev0.record()
+        for i in range(args.steps):
+            s.step_sgns(*batch(args.warmup + i), dist, NEG, LR, loss)
+        ev1.record()
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    launches = s.stats()["launches"] - launches0
+    final_loss = float(loss.item())
+
+    # end to end: pairs start in pinned host memory, the loss is read back every step
+    hc, ho = c.cpu().pin_memory(), o.cpu().pin_memory()
+    dc = torch.empty(BATCH, dtype=torch.int32, device=device)
+    do = torch.empty(BATCH, dtype=torch.int32, device=device)
+    hl = torch.zeros(1, dtype=torch.float32).pin_memory()
+    e2e_steps = min(args.steps, 2048)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(e2e_steps):
+        j = (i % nb) * BATCH
+        dc.copy_(hc[j:j + BATCH], non_blocking=True)
+        do.copy_(ho[j:j + BATCH], non_blocking=True)
+        s.step_sgns(dc, do, dist, NEG, LR, loss)
+        hl.copy_(loss, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    # roofline of the dominant kernel (the fused step kernel), timed with event pairs on its stream
+    s.kernel_timing(True)
+    hot_mask = torch.zeros(2 * VOCAB, dtype=torch.bool, device=device)
+    hot_mask[hot] = True
+    cold_rows = []
+    for i in range(args.steps):
+        bc, bo = batch(i)
+        s.step_sgns(bc, bo, dist, NEG, LR, loss)
+        if i % max(1, args.steps // 16) == 0:
+            keys = torch.cat([bc.long(), bo.long(), s.last_negatives().long()])
+            uniq = torch.unique(keys)
+            cold_rows.append(int((~hot_mask[uniq]).sum()))
+    k_ms, k_launches = s.kernel_time()
+    s.kernel_timing(False)
+    row_bytes = DIM * 4
+    key_bytes = BATCH * 4 * (2 + NEG)
+    alg_bytes = key_bytes + 2 * row_bytes * float(np.mean(cold_rows))
+    logical_bytes = key_bytes + 2 * row_bytes * BATCH * (NEG + 2)
+    k_s = (k_ms / 1e3) / max(k_launches, 1)
+    sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2104_00501_b200", "csrc", "steps.cu"), "rb").read()).hexdigest()
+    traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["steps_cu_sha1"] == sha else None
+
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=device)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        ms, e2e_s = float(t[0]), float(t[1])
+    pairs = args.steps * BATCH * world
+    value = pairs * ACCESSES_PER_PAIR / (ms / 1e3)
+    out = {
+        "metric": "key accesses/s (pull+push+sample)", "value": value, "unit": "key accesses/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "SGNS word vectors: vocab 1M, dim 300, 100M-token Zipf(1.0) stream, window 5, "
+                               "3 negatives unigram^0.75 BOUNDED(U=16,G=250), batch 4096 pairs, top 1% keys replicated, "
+                               "sync every 16 batches, fast (atomic) mode",
+                   "workers": WORKERS, "l2": "tables (2.4 GB) larger than L2; no explicit flush",
+                   "distinct_batches": nb, "replicas": world},
+        "updates_per_s": pairs * UPDATES_PER_PAIR / (ms / 1e3),
+        "pairs_per_s": pairs / (ms / 1e3),
+        "final_loss": final_loss,
+        "clocks": clk.summary(),
+        "e2e": {"value": e2e_steps * BATCH * world * ACCESSES_PER_PAIR / e2e_s, "unit": "key accesses/s",
+                "h2d_bytes_per_step": 2 * BATCH * 4, "d2h_bytes_per_step": 4, "steps": e2e_steps},
+        "gpu_launches": int(launches),
+        "roofline": {"bound": "hbm", "kernel": "sgns_kernel (fused step)", "achieved": alg_bytes / k_s / 1e9,
+                     "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
+                     "frac": alg_bytes / k_s / 1e9 / hbm_peak, "traffic": traffic,
+                     "algorithmic_bytes_per_launch": alg_bytes, "logical_bytes_per_launch": logical_bytes,
+                     "logical_gbs": logical_bytes / k_s / 1e9, "kernel_us": k_s * 1e6,
+                     "kernel_share_of_step": (k_ms / max(k_launches, 1)) / (ms / args.steps),
+                     "distinct_cold_rows_per_batch": float(np.mean(cold_rows))},
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(c, o, weights, hot, budget_s=12.0)
+    return out
+
+
+# --------------------------------------------------------------------------------------------
+# the oracle as CPU baseline / reference arm
+# --------------------------------------------------------------------------------------------
+def oracle_setup(weights, hot):
+    import oracle
+    o = oracle.Oracle(2 * VOCAB, DIM, workers=WORKERS, sync_interval=SYNC_EVERY)
+    o.init_uniform(0, 1, 0.5 / DIM)
+    o.set_management(inputs.u32(hot), oracle.REPLICATE)
+    d = o.register_distribution(VOCAB, inputs.u32(weights), VOCAB, oracle.BOUNDED, U=U_REUSE, G=G_POOL, seed=7)
+    return o, d
+
+
+def cpu_baseline(c, o_keys, weights, hot, budget_s):
+    orc, d = oracle_setup(weights, hot)
+    hc, ho = inputs.u32(c), inputs.u32(o_keys)
+    nb = len(hc) // BATCH
+    t0 = time.perf_counter()
+    done = 0
+    while done < nb and time.perf_counter() - t0 < budget_s:
+        j = done * BATCH
+        orc.step_sgns(hc[j:j + BATCH], ho[j:j + BATCH], d, NEG, LR)
+        done += 1
+    dt = time.perf_counter() - t0
+    return {"value": done * BATCH * ACCESSES_PER_PAIR / dt, "unit": "key accesses/s", "cores": 1, "kind": "oracle",
+            "sample": f"first {done} batches of {BATCH} pairs of the same workload, full-size tables, "
+                      f"{dt:.1f} s on one host thread (of {os.cpu_count()} cores)"}
+
+
+def run_reference(args):
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    # bounded sample: the pairs of one step are a prefix of a batch, sized after a probe step so that the
+    # whole run stays within a few minutes
+    nb = min(args.steps + args.warmup, 512)
+    c, o, counts, weights = make_sgns_data(dev, nb, seed=0)
+    freq = torch.cat([counts, counts])
+    hot = torch.argsort(freq, descending=True, stable=True)[: int(HOT_FRACTION * 2 * VOCAB)]
+    orc, d = oracle_setup(weights.cpu(), hot.cpu())
+    hc, ho = inputs.u32(c), inputs.u32(o)
+    t0 = time.perf_counter()
+    orc.step_sgns(hc[:BATCH], ho[:BATCH], d, NEG, LR)
+    probe = time.perf_counter() - t0
+    per_step = BATCH
+    budget = 150.0
+    if probe * (args.steps + args.warmup) > budget:
+        per_step = max(64, int(BATCH * budget / (probe * (args.steps + args.warmup))) // 64 * 64)
+
+    def step(i):
+        j = (i % nb) * BATCH
+        orc.step_sgns(hc[j:j + per_step], ho[j:j + per_step], d, NEG, LR)
+
+    for i in range(args.warmup):
+        step(i)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        step(args.warmup + i)
+    dt = time.perf_counter() - t0
+    value = args.steps * per_step * ACCESSES_PER_PAIR / dt
+    sample = (f"{per_step} pairs per step (of the workload's {BATCH}), full-size tables, single host thread "
+              f"of {os.cpu_count()} cores")
+    return {
+        "impl": "reference", "metric": "key accesses/s (pull+push+sample)", "value": value, "unit": "key accesses/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "SGNS word vectors: vocab 1M, dim 300, Zipf(1.0) tokens, window 5, 3 negatives "
+                               "BOUNDED(U=16,G=250), batch 4096 pairs, top 1% keys replicated, sync every 16 batches",
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "key accesses/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "key accesses/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4096)
+    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        if rank == 0:
+            print(json.dumps(run_reference(args)), flush=True)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=device)
+    out = run_ours(args, rank, world, device)
+    if rank == 0:
+        print(json.dumps(out), flush=True)
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

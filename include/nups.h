@@ -248,6 +248,15 @@ nups_status nups_status_check(nups_store* store, void* stream);
  * Synchronises the stream.                                                    */
 nups_status nups_get_stats(nups_store* store, uint64_t* h_out, void* stream);
 
+/* Timing aid for benchmarks.  While enabled, the library records a pair of CUDA
+ * events on the call's stream around the main kernel of nups_pull*, nups_push*
+ * (fast mode) and nups_step_* (the row gather, the scatter-add, the fused step
+ * kernel).  nups_kernel_time synchronises the stream, adds up the elapsed
+ * times of all pairs recorded since the last query, returns the sum in
+ * milliseconds and the number of launches, and starts afresh.                 */
+nups_status nups_kernel_timing(nups_store* store, int enable);
+nups_status nups_kernel_time(nups_store* store, double* h_ms_out, uint64_t* h_launches_out, void* stream);
+
 const char* nups_strerror(nups_status status);
 const char* nups_last_cuda_error(void);
 

@@ -24,7 +24,7 @@ EXPORTS = [
     "nups_push2", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_step_complex", "nups_step_mf",
-    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_strerror", "nups_last_cuda_error",
+    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_strerror", "nups_last_cuda_error",
 ]
 
 
@@ -87,6 +87,8 @@ def load(build_if_missing: bool = True):
         "nups_last_negatives": [vp, C.POINTER(vp), C.POINTER(u64)],
         "nups_status_check": [vp, vp],
         "nups_get_stats": [vp, C.POINTER(u64), vp],
+        "nups_kernel_timing": [vp, C.c_int],
+        "nups_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -302,6 +304,15 @@ class Store:
     # -- status -------------------------------------------------------------------------
     def status_check(self):
         return self._l.nups_status_check(self._s, _stream())
+
+    def kernel_timing(self, enable):
+        self._chk(self._l.nups_kernel_timing(self._s, int(enable)), "nups_kernel_timing")
+
+    def kernel_time(self):
+        """(milliseconds, launches) of the main kernels since the last query."""
+        ms, n = C.c_double(), C.c_uint64()
+        self._chk(self._l.nups_kernel_time(self._s, C.byref(ms), C.byref(n), _stream()), "nups_kernel_time")
+        return ms.value, n.value
 
     def stats(self):
         out = (C.c_uint64 * 8)()

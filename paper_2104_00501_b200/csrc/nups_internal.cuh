@@ -13,6 +13,7 @@
 #define NUPS_OWNER_DEFAULT 255
 #define NUPS_INVALID_KEY 0xFFFFFFFFu
 #define NUPS_MAX_POOL 1024
+#define NUPS_MAX_TIMED 4096
 
 // ---------------------------------------------------------------------------------------------
 // Device-resident status and statistics
@@ -91,6 +92,11 @@ struct nups_store {
     uint64_t last_negs_n, last_negs_cap;
     uint64_t steps, syncs, launches;
     int device, sm_count, max_smem;
+    int timing;                // record events around the main kernels?
+    cudaEvent_t* ev;           // [2 * NUPS_MAX_TIMED] begin/end pairs
+    uint32_t ev_n;             // pairs recorded since the last query
+    double ev_ms;              // time of pairs folded in when the ring filled up
+    uint64_t ev_launches;
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };
@@ -123,6 +129,8 @@ static inline unsigned grid_for(uint64_t work, unsigned per_block, unsigned cap 
 }
 
 View nups_view(const nups_store* s);
+void nups_time_begin(nups_store* s, cudaStream_t st);
+void nups_time_end(nups_store* s, cudaStream_t st);
 nups_status nups_scratch(nups_store* s, size_t bytes, char** out);     // grow-only scratch, 256-byte aligned
 nups_status nups_req_reserve(nups_store* s, size_t n);
 

@@ -209,9 +209,14 @@ __device__ __forceinline__ void grads(const C2 (&h)[CH], const C2 (&r)[CH], cons
         {                                                                                                     \
             float hr = h[m].re.comp, hi = h[m].im.comp, rr = r[m].re.comp, ri = r[m].im.comp;                 \
             float tr = t[m].re.comp, ti = t[m].im.comp;                                                       \
-            if (gh) { gh[m].re.comp += coef * (rr * tr + ri * ti); gh[m].im.comp += coef * (rr * ti - ri * tr); } \
-            if (gt) { gt[m].re.comp += coef * (hr * rr - hi * ri); gt[m].im.comp += coef * (hi * rr + hr * ri); } \
-            if (gr) { gr[m].re.comp += coef * (hr * tr + hi * ti); gr[m].im.comp += coef * (hr * ti - hi * tr); } \
+            /* differences of products are formed without fused multiply-add, so that a gradient  */ \
+            /* that cancels exactly (head == tail) is exactly zero here too                       */ \
+            if (gh) { gh[m].re.comp += coef * (rr * tr + ri * ti);                                    \
+                      gh[m].im.comp += coef * __fsub_rn(__fmul_rn(rr, ti), __fmul_rn(ri, tr)); }      \
+            if (gt) { gt[m].re.comp += coef * __fsub_rn(__fmul_rn(hr, rr), __fmul_rn(hi, ri));        \
+                      gt[m].im.comp += coef * (hi * rr + hr * ri); }                                  \
+            if (gr) { gr[m].re.comp += coef * (hr * tr + hi * ti);                                    \
+                      gr[m].im.comp += coef * __fsub_rn(__fmul_rn(hr, ti), __fmul_rn(hi, tr)); }      \
         }
         NUPS_C1(x)
         NUPS_C1(y)
@@ -509,8 +514,10 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
     unsigned grid = step_grid(s, n);
+    nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, sgns_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
         v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+    nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return step_finish(s, n, K + 2, 2, b, d_loss_out, st);
 }
@@ -531,8 +538,10 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
     unsigned grid = step_grid(s, n);
+    nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, complex_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
         v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+    nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return step_finish(s, n, K + 3, 3, b, d_loss_out, st);
 }
@@ -551,8 +560,10 @@ extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const 
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
     unsigned grid = step_grid(s, n);
+    nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
         v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+    nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return step_finish(s, n, 2, 2, b, d_loss_out, st);
 }

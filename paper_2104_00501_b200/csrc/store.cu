@@ -71,6 +71,56 @@ nups_status nups_req_reserve(nups_store* s, size_t n)
 static inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
 
 // ---------------------------------------------------------------------------------------------
+// optional event pairs around the main kernels (benchmark aid)
+// ---------------------------------------------------------------------------------------------
+static void timing_fold(nups_store* s)
+{
+    for (uint32_t i = 0; i < s->ev_n; ++i) {
+        float ms = 0.f;
+        if (cudaEventSynchronize(s->ev[2 * i + 1]) == cudaSuccess &&
+            cudaEventElapsedTime(&ms, s->ev[2 * i], s->ev[2 * i + 1]) == cudaSuccess)
+            s->ev_ms += ms;
+    }
+    s->ev_launches += s->ev_n;
+    s->ev_n = 0;
+    cudaGetLastError();
+}
+void nups_time_begin(nups_store* s, cudaStream_t st)
+{
+    if (!s->timing) return;
+    if (s->ev_n == NUPS_MAX_TIMED) timing_fold(s);
+    cudaEventRecord(s->ev[2 * s->ev_n], st);
+}
+void nups_time_end(nups_store* s, cudaStream_t st)
+{
+    if (!s->timing) return;
+    cudaEventRecord(s->ev[2 * s->ev_n + 1], st);
+    s->ev_n++;
+}
+extern "C" nups_status nups_kernel_timing(nups_store* s, int enable)
+{
+    if (!s) return NUPS_EINVAL;
+    if (enable && !s->ev) {
+        s->ev = (cudaEvent_t*)calloc(2 * NUPS_MAX_TIMED, sizeof(cudaEvent_t));
+        if (!s->ev) return NUPS_ENOMEM;
+        for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) CK(cudaEventCreate(&s->ev[i]));
+    }
+    if (s->ev) timing_fold(s);
+    s->ev_ms = 0; s->ev_launches = 0;
+    s->timing = enable ? 1 : 0;
+    return NUPS_OK;
+}
+extern "C" nups_status nups_kernel_time(nups_store* s, double* h_ms_out, uint64_t* h_launches_out, void* stream)
+{
+    if (!s || !h_ms_out || !h_launches_out) return NUPS_EINVAL;
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    if (s->ev) timing_fold(s);
+    *h_ms_out = s->ev_ms; *h_launches_out = s->ev_launches;
+    s->ev_ms = 0; s->ev_launches = 0;
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // create / destroy
 // ---------------------------------------------------------------------------------------------
 __global__ void fill_i32(int* p, uint64_t n, int value)
@@ -146,6 +196,10 @@ extern "C" nups_status nups_destroy(nups_store* s)
     cudaFree(s->val); cudaFree(s->acc); cudaFree(s->hot_bits); cudaFree(s->slot_of); cudaFree(s->hot_keys);
     cudaFree(s->dval); cudaFree(s->dacc); cudaFree(s->dirty); cudaFree(s->cnt); cudaFree(s->owner);
     cudaFree(s->pending); cudaFree(s->st); cudaFree(s->scratch); cudaFree(s->req_keys); cudaFree(s->last_negs);
+    if (s->ev) {
+        for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) cudaEventDestroy(s->ev[i]);
+        free(s->ev);
+    }
     cudaGetLastError();
     free(s);
     return NUPS_OK;
@@ -291,12 +345,14 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
     if (n == 0 || (!d_out_val && !d_out_acc)) return NUPS_OK;
     View v = nups_view(s);
     unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 8);
+    nups_time_begin(s, st);
     if (s->H)
         gather_kernel<true><<<grid, 256, 0, st>>>(v, d_keys, n, (float4*)d_out_val, (float4*)d_out_acc, worker_map,
                                                   map_base, map_total, 1, do_count);
     else
         gather_kernel<false><<<grid, 256, 0, st>>>(v, d_keys, n, (float4*)d_out_val, (float4*)d_out_acc, worker_map,
                                                    map_base, map_total, 1, do_count);
+    nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return NUPS_OK;
 }
@@ -547,12 +603,14 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
     uint64_t n_items = n / rows_per_item;
     if (!s->cfg.deterministic) {
         unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 8);
+        nups_time_begin(s, st);
         if (s->H)
             push_atomic_kernel<true><<<grid, 256, 0, st>>>(v, d_keys, n, (const float4*)d_dval, (const float4*)d_dacc,
                                                            n_items, rows_per_item);
         else
             push_atomic_kernel<false><<<grid, 256, 0, st>>>(v, d_keys, n, (const float4*)d_dval, (const float4*)d_dacc,
                                                             n_items, rows_per_item);
+        nups_time_end(s, st);
         LAUNCH_CHECK(s);
         return NUPS_OK;
     }
