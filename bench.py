@@ -33,7 +33,7 @@ sys.path.insert(0, ROOT)
 from paper_2104_00501_b200 import inputs  # noqa: E402
 
 VOCAB, DIM, BATCH, NEG, WINDOW = 1_000_000, 300, 4096, 3, 5
-U_REUSE, G_POOL, SYNC_EVERY, WORKERS, LR = 16, 250, 16, 8, 0.025
+U_REUSE, G_POOL, SYNC_EVERY, WORKERS, LR = 16, 250, 16, 8, 0.005
 HOT_FRACTION = 0.01
 TOKENS = 100_000_000
 ACCESSES_PER_PAIR = 2 + NEG + (NEG + 2)          # direct pulls + sampled pulls + pushes
@@ -316,6 +316,64 @@ def run_reference(args):
     }
 
 
+# --------------------------------------------------------------------------------------------
+# pull / push / PullSample microbenchmark (not the default line): 100M keys x 128 floats, batches of
+# 1M keys ~ Zipf(s), top-k replicated; one JSON line per sweep point
+# --------------------------------------------------------------------------------------------
+def run_ps_sweep(args, device):
+    from paper_2104_00501_b200 import binding
+    hbm_peak, peak_kind = peaks()
+    NK, L, N = args.ps_keys, 128, 1 << 20
+    row = L * 4
+    reps = max(args.steps, 5)
+    delta = torch.randn(N, L, device=device)
+    out = torch.empty(N, L, device=device)
+    lines = []
+    for skew in [float(x) for x in args.ps_skews.split(",")]:
+        cdf = inputs.zipf_cdf(NK, skew, device) if skew > 0 else None
+        batches = [inputs.zipf_keys(N, NK, skew, 100 + i, device, cdf=cdf).to(torch.int32) for i in range(4)]
+        key_of_rank = None
+        for topk in [int(x) for x in args.ps_topk.split(",")]:
+            s = binding.Store(NK, L, workers=WORKERS, deterministic=False)
+            s.init_uniform(0, 3, 0.1)
+            if topk:
+                if key_of_rank is None:
+                    key_of_rank = inputs.zipf_key_of_rank(NK, device)
+                s.set_management(key_of_rank[:topk].to(torch.int32).contiguous(), binding.REPLICATE)
+            hot_mask = None
+            if topk:
+                hot_mask = torch.zeros(NK, dtype=torch.bool, device=device)
+                hot_mask[key_of_rank[:topk]] = True
+            ucold = []
+            for b in batches:
+                u = torch.unique(b.long())
+                ucold.append(int(u.numel() if hot_mask is None else (~hot_mask[u]).sum()))
+            ucold = float(np.mean(ucold))
+            s.kernel_timing(True)
+            res = {}
+            for op in ("pull", "push"):
+                for i in range(3):
+                    (s.pull(batches[i % 4], out) if op == "pull" else s.push(batches[i % 4], delta))
+                s.kernel_time()
+                for i in range(reps):
+                    (s.pull(batches[i % 4], out) if op == "pull" else s.push(batches[i % 4], delta))
+                    if op == "push" and topk and (i + 1) % 16 == 0:
+                        s.sync()
+                ms, n = s.kernel_time()
+                t = ms / 1e3 / n
+                alg = 4 * N + row * N + (1 if op == "pull" else 2) * row * ucold
+                res[op] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
+                           "frac": alg / t / 1e9 / hbm_peak, "logical_gbs": (4 * N + (2 if op == "pull" else 3) * row * N) / t / 1e9}
+            line = {"workload": "ps microbenchmark", "keys": NK, "value_len": L, "batch": N, "zipf_s": skew, "topk": topk,
+                    "distinct_cold_rows": ucold, "peak": hbm_peak, "peak_kind": peak_kind, **res}
+            print(json.dumps(line), flush=True)
+            lines.append(line)
+            s.close()
+            del s
+            torch.cuda.empty_cache()
+    return lines
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -323,6 +381,10 @@ def main():
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="sgns", choices=["sgns", "ps"])
+    ap.add_argument("--ps-keys", type=int, default=100_000_000)
+    ap.add_argument("--ps-skews", default="0,0.6,1.0,1.4")
+    ap.add_argument("--ps-topk", default="0,1000,100000")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     rank = int(os.environ.get("RANK", "0"))
@@ -336,6 +398,9 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local)
     device = torch.device("cuda", local)
+    if args.workload == "ps":
+        run_ps_sweep(args, device)
+        return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)
     out = run_ours(args, rank, world, device)
