@@ -119,6 +119,30 @@ nups_status nups_push(nups_store* store, const uint32_t* d_keys, uint64_t n, con
 nups_status nups_push2(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta_val,
                        const float* d_delta_acc, void* stream);
 
+/* Ordered push for callers that must not allocate device memory while they run:
+ * code between the start and end of a latency-critical serving loop, a process
+ * whose memory pool was handed out in full at start-up, or a host thread that
+ * may not take the allocator's device-wide synchronisation.  (The paper has no
+ * counterpart; nups_push in deterministic mode sorts the rows by destination and
+ * may grow the store's scratch buffer with cudaMalloc/cudaFree when a call is
+ * larger than any before it.)  This variant does the same work with its sort
+ * buffers in a fixed 2 MiB array inside the library image, so it calls no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *   - Same result as nups_push on a store created with deterministic = 1;
+ *     NUPS_ESTATE on any other store, or when the store's device is not current.
+ *   - n may be at most NUPS_NOALLOC_MAX_ROWS; larger calls return NUPS_EINVAL
+ *     (nups_last_cuda_error names the limit) and enqueue nothing.
+ *   - The first call on a device looks up the array's device address; make that
+ *     first call before any stream capture begins.
+ *   - All calls, on all stores of the process, share the one array per device.
+ *     It keeps whatever the last call left; every buffer in it is rewritten in
+ *     full before it is read, so nothing needs clearing.  Two calls whose work
+ *     overlaps on the GPU (different streams, no ordering between them) race on
+ *     it: order them, or use nups_push for one of them.                        */
+#define NUPS_NOALLOC_MAX_ROWS 65536
+nups_status nups_push_noalloc(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta,
+                              void* stream);
+
 /* ---- per-key management (Section 3.2, Section 5.1) ------------------------ */
 
 /* Set the technique of the listed keys.  Pending replica updates are merged

@@ -18,10 +18,11 @@ LIB_PATH = os.path.join(_HERE, "libnups.so")
 OK, EINVAL, ENOMEM, ECUDA, EKEY, ESTATE, ETIMEOUT = 0, -1, -2, -3, -4, -5, -6
 SINGLE, REPLICATE = 0, 1
 CONFORM, BOUNDED, LONGTERM, NONCONFORM = 1, 2, 3, 4
+NOALLOC_MAX_ROWS = 65536
 
 EXPORTS = [
     "nups_create", "nups_destroy", "nups_table_ptr", "nups_table_copy", "nups_init_uniform", "nups_pull", "nups_pull2", "nups_push",
-    "nups_push2", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
+    "nups_push2", "nups_push_noalloc", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_step_complex", "nups_step_mf",
     "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_strerror", "nups_last_cuda_error",
@@ -69,6 +70,7 @@ def load(build_if_missing: bool = True):
         "nups_pull2": [vp, vp, u64, vp, vp, vp],
         "nups_push": [vp, vp, u64, vp, vp],
         "nups_push2": [vp, vp, u64, vp, vp, vp],
+        "nups_push_noalloc": [vp, vp, u64, vp, vp],
         "nups_set_management": [vp, vp, u64, C.c_int, vp],
         "nups_sync": [vp, vp],
         "nups_count_accesses": [vp, vp, u64, vp],
@@ -144,6 +146,8 @@ class Store:
             detail = self._l.nups_strerror(code).decode()
             if code == ECUDA:
                 detail += ": " + self._l.nups_last_cuda_error().decode()
+            elif code == EINVAL and what == "nups_push_noalloc":
+                detail += ": " + self._l.nups_last_cuda_error().decode()
             raise NupsError(code, what, detail)
 
     def close(self):
@@ -202,6 +206,14 @@ class Store:
             assert delta_acc.dtype == torch.float32 and delta_acc.numel() == n * self.L
             self._chk(self._l.nups_push2(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _ptr(delta_acc), _stream()),
                       "nups_push2")
+
+    def push_noalloc(self, keys, delta):
+        """Ordered push with its sort buffers in the library's fixed device array: for callers that
+        may not allocate device memory while they run.  At most NOALLOC_MAX_ROWS rows per call."""
+        n = keys.numel()
+        assert delta.dtype == torch.float32 and delta.numel() == n * self.L
+        self._chk(self._l.nups_push_noalloc(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _stream()),
+                  "nups_push_noalloc")
 
     def sync(self):
         self._chk(self._l.nups_sync(self._s, _stream()), "nups_sync")
