@@ -375,6 +375,7 @@ def run_ps_sweep(args, device):
 
 
 def main():
+    global TOKENS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4096)
@@ -382,11 +383,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="sgns", choices=["sgns", "ps"])
+    ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
     ap.add_argument("--ps-keys", type=int, default=100_000_000)
     ap.add_argument("--ps-skews", default="0,0.6,1.0,1.4")
     ap.add_argument("--ps-topk", default="0,1000,100000")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
+    TOKENS = max(args.tokens, 10_000_000)
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -53,7 +53,9 @@ struct Dist {
     uint32_t key_base, U, G;
     uint64_t n, W, seed;
     void* table;               // AliasEntry[n]
-    unsigned long long* off;   // device [R]: next unused position of each worker's stream
+    unsigned long long* off;   // device [2][R]: next unused position of each worker's stream; a call reads
+                               // half `cur` and writes the other half, then the host flips `cur`
+    int cur;
 };
 
 struct AliasEntry {

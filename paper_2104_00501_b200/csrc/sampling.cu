@@ -162,8 +162,8 @@ extern "C" nups_status nups_register_distribution(nups_store* s, uint32_t key_ba
         LAUNCH_CHECK(s);
         CK(cudaStreamSynchronize(st));
     }
-    if (cudaMalloc(&d.off, s->R * 8) != cudaSuccess) { cudaGetLastError(); cudaFree(d.table); return NUPS_ENOMEM; }
-    CK(cudaMemsetAsync(d.off, 0, s->R * 8, st));
+    if (cudaMalloc(&d.off, 2 * s->R * 8) != cudaSuccess) { cudaGetLastError(); cudaFree(d.table); return NUPS_ENOMEM; }
+    CK(cudaMemsetAsync(d.off, 0, 2 * s->R * 8, st));
     CK(cudaStreamSynchronize(st));
     d.used = 1;
     s->dist[id] = d;
@@ -243,13 +243,14 @@ static HandleView handle_view(char* buf, uint64_t N, uint32_t R)
     return h;
 }
 
-__global__ void handle_begin_kernel(unsigned long long* off, HandleView h, uint64_t N, uint32_t R, int longterm)
+__global__ void handle_begin_kernel(const unsigned long long* off_cur, unsigned long long* off_next, HandleView h,
+                                    uint64_t N, uint32_t R, int longterm)
 {
     uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
     if (q >= R) return;
     unsigned long long size = chunk_begin(q + 1, N, R) - chunk_begin(q, N, R);
-    h.start[q] = off[q];
-    off[q] += size;
+    h.start[q] = off_cur[q];
+    off_next[q] = off_cur[q] + size;
     if (longterm) h.state[q] = make_uint4(0u, 0u, 0u, 0u);
 }
 
@@ -343,8 +344,10 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
     }
     HandleView hv = handle_view(h.buf, N, s->R);
     DrawParams p = draw_params(d);
-    handle_begin_kernel<<<grid_for(s->R, 64), 64, 0, st>>>(d.off, hv, N, s->R, d.level == NUPS_LONGTERM);
+    handle_begin_kernel<<<grid_for(s->R, 64), 64, 0, st>>>(d.off + (size_t)d.cur * s->R, d.off + (size_t)(d.cur ^ 1) * s->R,
+                                                           hv, N, s->R, d.level == NUPS_LONGTERM);
     LAUNCH_CHECK(s);
+    d.cur ^= 1;
     if (reuse) {
         uint64_t max_size = (N + s->R - 1) / s->R;
         unsigned passes = (unsigned)(max_size / d.G + 2);
@@ -523,6 +526,96 @@ extern "C" nups_status nups_pull_sample(nups_store* s, nups_handle handle, uint6
     return pull_internal(s, (int)handle, n, d_keys_out, d_vals_out, (cudaStream_t)stream);
 }
 
+// ---------------------------------------------------------------------------------------------
+// PrepareSample + one full PullSample (keys only) in a single launch, for the workload steps: the
+// same keys as the handle path gives, written straight to `out`.  Stream offsets are read from one
+// half of the distribution's offset array and the advanced offsets written to the other half.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void direct_tail(const View& v, uint32_t key, uint32_t q, bool in, bool localize, uint32_t* req,
+                                            uint64_t req_cap)
+{
+    count_sample(v, key, in);
+    if (in && localize) {
+        atomicMax(v.pending + key, (int)q);
+        unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
+        if (at < req_cap) req[at] = key;
+    }
+}
+
+__global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long long* off_cur,
+                                       unsigned long long* off_next, uint64_t N, int local_only, int localize,
+                                       uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+{
+    const uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool in = o < N;
+    uint32_t k = 0, q = 0;
+    if (in) {
+        q = chunk_of_pos(o, N, v.R);
+        k = draw_iid(p, q, off_cur[q] + (o - chunk_begin(q, N, v.R)));
+        if (local_only) {
+            const uint32_t k0 = k;
+            for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
+                uint32_t cand = p.key_base + (uint32_t)(((unsigned long long)(k0 - p.key_base) + probe) % p.n);
+                if (key_is_local(v, q, cand)) { k = cand; break; }
+            }
+        }
+        out[o] = k;
+    }
+    direct_tail(v, k, q, in, localize != 0, req, req_cap);
+    if (blockIdx.x == 0)
+        for (uint32_t w = threadIdx.x; w < v.R; w += blockDim.x)
+            off_next[w] = off_cur[w] + (chunk_begin(w + 1, N, v.R) - chunk_begin(w, N, v.R));
+}
+
+__global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned long long* off_cur,
+                                         unsigned long long* off_next, uint64_t N, int localize,
+                                         uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+{
+    __shared__ uint32_t pool[NUPS_MAX_POOL];
+    __shared__ uint32_t perm[NUPS_MAX_POOL];
+    __shared__ uint32_t xs[NUPS_MAX_POOL];
+    const uint32_t q = blockIdx.y, G = p.G, R = v.R;
+    if (blockIdx.x == 0 && blockIdx.y == 0)
+        for (uint32_t w = threadIdx.x; w < R; w += blockDim.x)
+            off_next[w] = off_cur[w] + (chunk_begin(w + 1, N, R) - chunk_begin(w, N, R));
+    const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
+    if (size == 0) return;
+    const unsigned long long s0 = off_cur[q], s1 = s0 + size;
+    const unsigned long long pass = s0 / G + blockIdx.x;
+    if (pass * G >= s1) return;
+    const unsigned long long pl = pass / p.U;
+    for (uint32_t m = threadIdx.x; m < G; m += blockDim.x) {
+        pool[m] = draw_iid(p, q, pl * G + m);
+        perm[m] = m;
+    }
+    for (uint32_t blk = threadIdx.x; blk * 4 < G - 1; blk += blockDim.x) {
+        uint32_t x[4];
+        philox_at(p.seed, pass, q, 1, blk, x);
+        for (int k = 0; k < 4; ++k)
+            if (blk * 4 + k < G - 1) xs[blk * 4 + k] = x[k];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (uint32_t i = G - 1; i >= 1; --i) {
+            uint32_t r = __umulhi(xs[G - 1 - i], i + 1);
+            uint32_t t = perm[i]; perm[i] = perm[r]; perm[r] = t;
+        }
+    }
+    __syncthreads();
+    const uint32_t rounds = (G + blockDim.x - 1) / blockDim.x;
+    for (uint32_t rd = 0; rd < rounds; ++rd) {           // whole warps take every round: the tail ballots
+        const uint32_t j = rd * blockDim.x + threadIdx.x;
+        const unsigned long long sp = pass * G + j;
+        const bool in = j < G && sp >= s0 && sp < s1;
+        uint32_t k = 0;
+        if (in) {
+            k = pool[perm[j]];
+            out[b0 + (sp - s0)] = k;
+        }
+        direct_tail(v, k, q, in, localize != 0, req, req_cap);
+    }
+}
+
 // negatives of a workload step: one handle of N samples, pulled at once into library memory
 nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st)
 {
@@ -535,11 +628,45 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
         if (cudaMalloc(&s->last_negs, want * 4) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
         s->last_negs_cap = want;
     }
-    int id = -1;
-    nups_status rc = prepare_internal(s, dist, N, &id, st);
-    if (rc != NUPS_OK) return rc;
-    rc = pull_internal(s, id, N, s->last_negs, nullptr, st);
-    if (rc != NUPS_OK) return rc;
+    if (dist < 0 || dist >= NUPS_MAX_DISTS || !s->dist[dist].used || N >= (1ull << 32)) return NUPS_EINVAL;
+    Dist& d = s->dist[dist];
+    nups_status rc;
+    if (d.level == NUPS_LONGTERM) {
+        // postponing needs the handle's walk state: PrepareSample, then one full PullSample
+        int id = -1;
+        rc = prepare_internal(s, dist, N, &id, st);
+        if (rc != NUPS_OK) return rc;
+        rc = pull_internal(s, id, N, s->last_negs, nullptr, st);
+        if (rc != NUPS_OK) return rc;
+        s->last_negs_n = N;
+        return NUPS_OK;
+    }
+    const int localize = s->owner && d.level != NUPS_NONCONFORM;
+    if (localize) {
+        rc = nups_req_reserve(s, N);
+        if (rc != NUPS_OK) return rc;
+    }
+    View v = nups_view(s);
+    DrawParams p = draw_params(d);
+    const unsigned long long* off_cur = d.off + (size_t)d.cur * s->R;
+    unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
+    if (d.level == NUPS_BOUNDED) {
+        uint64_t max_size = (N + s->R - 1) / s->R;
+        unsigned passes = (unsigned)(max_size / d.G + 2);
+        unsigned threads = ((d.G + 31) / 32) * 32;
+        if (threads > 256) threads = 256;
+        draw_direct_reuse_kernel<<<dim3(passes, s->R), threads, 0, st>>>(v, p, off_cur, off_next, N, localize, s->last_negs,
+                                                                        s->req_keys, s->req_cap);
+    } else {
+        draw_direct_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(v, p, off_cur, off_next, N, d.level == NUPS_NONCONFORM,
+                                                                 localize, s->last_negs, s->req_keys, s->req_cap);
+    }
+    LAUNCH_CHECK(s);
+    d.cur ^= 1;
+    if (localize) {
+        rc = nups_localize_apply(s, N, st);
+        if (rc != NUPS_OK) return rc;
+    }
     s->last_negs_n = N;
     return NUPS_OK;
 }

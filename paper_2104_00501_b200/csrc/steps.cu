@@ -60,19 +60,75 @@ __device__ __forceinline__ void request_localize(const View& v, uint32_t key, ui
     if (at < cap) req[at] = key;
 }
 
+// Rows of several keys at once: all technique lookups are issued before any of them is used, so the
+// dependent chain key -> hot bit -> slot -> row is paid once per group, not once per row.
+struct RowAt {
+    unsigned long long row;    // offset of the stored row, in floats
+    unsigned long long pend;   // offset of the worker's replica row in the slab, in floats, or NO_PEND
+    int slot;
+};
+constexpr unsigned long long NO_PEND = ~0ull;
+
+template <bool HOT, int NR>
+__device__ __forceinline__ void resolve_rows(const View& v, const uint32_t (&key)[NR], const bool (&act)[NR],
+                                             uint32_t q, RowAt (&r)[NR])
+{
+    uint32_t bits[NR];
+#pragma unroll
+    for (int u = 0; u < NR; ++u) bits[u] = (HOT && act[u]) ? __ldg(v.hot_bits + (key[u] >> 5)) : 0u;
+#pragma unroll
+    for (int u = 0; u < NR; ++u) {
+        const bool hot = HOT && act[u] && ((bits[u] >> (key[u] & 31)) & 1u);
+        r[u].slot = hot ? __ldg(v.slot_of + key[u]) : -1;
+    }
+    const unsigned long long L = (unsigned long long)v.L4 * 4;
+#pragma unroll
+    for (int u = 0; u < NR; ++u) {
+        r[u].row = (unsigned long long)key[u] * L;
+        r[u].pend = r[u].slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)r[u].slot) * L : NO_PEND;
+    }
+}
+
+// per-launch loss accumulation in fast mode: warps add their item losses, the last block to finish
+// writes the mean and clears the accumulators for the next launch
+__device__ __forceinline__ void loss_finish(DevStat* st, double block_loss, uint64_t n, float* loss_out)
+{
+    __shared__ bool last;
+    if (threadIdx.x == 0) {
+        atomicAdd((double*)&st->tmp[2], block_loss);
+        __threadfence();
+        unsigned long long done = atomicAdd(&st->tmp[3], 1ull) + 1;
+        last = done == gridDim.x;
+        if (last) {
+            __threadfence();
+            double total = atomicAdd((double*)&st->tmp[2], 0.0);
+            if (loss_out) *loss_out = (float)(total / (double)(n ? n : 1));
+            st->tmp[2] = 0ull;
+            st->tmp[3] = 0ull;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // skip-gram with negative sampling
 // ---------------------------------------------------------------------------------------------
+constexpr int SGNS_UB = 4;      // output rows (context + negatives) handled per group
+
 template <bool HOT, bool DET, int CH>
 __global__ void __launch_bounds__(128)
 sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
             const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float* __restrict__ upd,
-            uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, uint32_t* req, uint64_t req_cap)
+            uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, float* __restrict__ loss_out, uint32_t* req,
+            uint64_t req_cap)
 {
+    __shared__ double warp_loss[4];
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t L4 = v.L4, per = K + 2;
+    const float4* val4 = (const float4*)v.val;
+    const float4* slab4 = (const float4*)v.dval;
+    double my_loss = 0.0;
     for (uint64_t i = warp; i < n; i += nwarps) {
         const uint32_t q = worker_of_item(i, n, v.R);
         const uint32_t kc = center[i], ko = context[i];
@@ -84,76 +140,118 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
             ukeys[i * per + K + 1] = ok ? kc : NUPS_INVALID_KEY;
         }
         if (!ok) {
-            if (lane == 0) { flag_bad_key(v); loss_item[i] = 0.f; }
+            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
-        RowRef rc = resolve<HOT>(v, kc, q, 0);
         float4 vr[CH], gv[CH];
-#pragma unroll
-        for (int m = 0; m < CH; ++m) {
-            uint32_t c = lane + 32 * m;
-            vr[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-            gv[m] = vr[m];
-            if (c < L4) {
-                vr[m] = ((const float4*)rc.base)[c];
-                if (rc.pend) vr[m] = add4(vr[m], ((const float4*)rc.pend)[c]);
-            }
-        }
+        RowAt rc;
         float loss = 0.f;
-        for (uint32_t j = 0; j <= K; ++j) {
-            const uint32_t ku = j == 0 ? ko : negs[i * K + j - 1];
-            RowRef ru = resolve<HOT>(v, ku, q, 0);
-            float4 ur[CH];
-            float dot = 0.f;
+        for (uint32_t j0 = 0; j0 <= K; j0 += SGNS_UB) {
+            // element 0 of the group is the centre row (first group only), elements 1.. are output rows
+            uint32_t key[SGNS_UB + 1];
+            bool act[SGNS_UB + 1];
+            RowAt ra[SGNS_UB + 1];
+            key[0] = kc; act[0] = j0 == 0;
 #pragma unroll
-            for (int m = 0; m < CH; ++m) {
-                uint32_t c = lane + 32 * m;
-                ur[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-                if (c < L4) {
-                    ur[m] = ((const float4*)ru.base)[c];
-                    if (ru.pend) ur[m] = add4(ur[m], ((const float4*)ru.pend)[c]);
-                }
-                dot += vr[m].x * ur[m].x + vr[m].y * ur[m].y + vr[m].z * ur[m].z + vr[m].w * ur[m].w;
+            for (int u = 0; u < SGNS_UB; ++u) {
+                const uint32_t j = j0 + u;
+                act[u + 1] = j <= K;
+                key[u + 1] = act[u + 1] ? (j == 0 ? ko : negs[i * K + j - 1]) : 0u;
             }
-            float x = clamp30(warp_sum(dot));
-            float g = sigmoidf_(x) - (j == 0 ? 1.f : 0.f);
-            loss += j == 0 ? softplusf_(-x) : softplusf_(x);
-            float sc = -lr * g;
-            float* out = DET ? upd + (i * per + j) * (uint64_t)L4 * 4 : ru.dst;
+            resolve_rows<HOT, SGNS_UB + 1>(v, key, act, q, ra);
+            if (j0 == 0) {
+                rc = ra[0];
 #pragma unroll
-            for (int m = 0; m < CH; ++m) {
-                uint32_t c = lane + 32 * m;
-                if (c < L4) {
-                    float4 du = make_float4(sc * vr[m].x, sc * vr[m].y, sc * vr[m].z, sc * vr[m].w);
-                    if (DET) ((float4*)out)[c] = du;
-                    else red_add_v4(out + 4 * c, du);
-                    gv[m].x += g * ur[m].x; gv[m].y += g * ur[m].y; gv[m].z += g * ur[m].z; gv[m].w += g * ur[m].w;
+                for (int m = 0; m < CH; ++m) {
+                    const uint32_t c = lane + 32 * m;
+                    vr[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    gv[m] = vr[m];
+                    if (c < L4) {
+                        vr[m] = val4[rc.row / 4 + c];
+                        if (HOT && rc.pend != NO_PEND) vr[m] = add4(vr[m], slab4[rc.pend / 4 + c]);
+                    }
                 }
             }
-            if (lane == 0) {
-                if (!DET && ru.slot >= 0) v.dirty[ru.slot] = 1u;
-                if (v.count) {
-                    if (j == 0) note_access(v, ku, ru.slot, DET ? 1u : 2u);      // pulled (+ pushed)
-                    else if (!DET) note_access(v, ku, ru.slot, 1u);              // pushed; the sample was counted at the draw
+            float4 ur[SGNS_UB][CH];
+#pragma unroll
+            for (int u = 0; u < SGNS_UB; ++u) {
+#pragma unroll
+                for (int m = 0; m < CH; ++m) {
+                    const uint32_t c = lane + 32 * m;
+                    ur[u][m] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (act[u + 1] && c < L4) {
+                        ur[u][m] = val4[ra[u + 1].row / 4 + c];
+                        if (HOT && ra[u + 1].pend != NO_PEND) ur[u][m] = add4(ur[u][m], slab4[ra[u + 1].pend / 4 + c]);
+                    }
+                }
+            }
+            float dot[SGNS_UB];
+#pragma unroll
+            for (int u = 0; u < SGNS_UB; ++u) {
+                dot[u] = 0.f;
+#pragma unroll
+                for (int m = 0; m < CH; ++m)
+                    dot[u] += vr[m].x * ur[u][m].x + vr[m].y * ur[u][m].y + vr[m].z * ur[u][m].z + vr[m].w * ur[u][m].w;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+                for (int u = 0; u < SGNS_UB; ++u) dot[u] += __shfl_xor_sync(0xFFFFFFFFu, dot[u], o);
+            }
+#pragma unroll
+            for (int u = 0; u < SGNS_UB; ++u) {
+                if (!act[u + 1]) continue;
+                const uint32_t j = j0 + u;
+                const float x = clamp30(dot[u]);
+                const float g = sigmoidf_(x) - (j == 0 ? 1.f : 0.f);
+                loss += j == 0 ? softplusf_(-x) : softplusf_(x);
+                const float sc = -lr * g;
+                const bool hot = HOT && ra[u + 1].pend != NO_PEND;
+                float* out = DET ? upd + (i * per + j) * (uint64_t)L4 * 4
+                                 : (hot ? v.dval + ra[u + 1].pend : v.val + ra[u + 1].row);
+#pragma unroll
+                for (int m = 0; m < CH; ++m) {
+                    const uint32_t c = lane + 32 * m;
+                    if (c < L4) {
+                        const float4 du = make_float4(sc * vr[m].x, sc * vr[m].y, sc * vr[m].z, sc * vr[m].w);
+                        if (DET) ((float4*)out)[c] = du;
+                        else red_add_v4(out + 4 * c, du);
+                        gv[m].x += g * ur[u][m].x; gv[m].y += g * ur[u][m].y;
+                        gv[m].z += g * ur[u][m].z; gv[m].w += g * ur[u][m].w;
+                    }
+                }
+                if (lane == 0) {
+                    if (!DET && hot && v.dirty[ra[u + 1].slot] == 0u) v.dirty[ra[u + 1].slot] = 1u;
+                    if (v.count) {
+                        if (j == 0) note_access(v, key[u + 1], ra[u + 1].slot, DET ? 1u : 2u);   // pulled (+ pushed)
+                        else if (!DET) note_access(v, key[u + 1], ra[u + 1].slot, 1u);           // pushed; the sample was counted at the draw
+                    }
                 }
             }
         }
-        float* out = DET ? upd + (i * per + K + 1) * (uint64_t)L4 * 4 : rc.dst;
+        const bool chot = HOT && rc.pend != NO_PEND;
+        float* out = DET ? upd + (i * per + K + 1) * (uint64_t)L4 * 4 : (chot ? v.dval + rc.pend : v.val + rc.row);
 #pragma unroll
         for (int m = 0; m < CH; ++m) {
-            uint32_t c = lane + 32 * m;
+            const uint32_t c = lane + 32 * m;
             if (c < L4) {
-                float4 dv = make_float4(-lr * gv[m].x, -lr * gv[m].y, -lr * gv[m].z, -lr * gv[m].w);
+                const float4 dv = make_float4(-lr * gv[m].x, -lr * gv[m].y, -lr * gv[m].z, -lr * gv[m].w);
                 if (DET) ((float4*)out)[c] = dv;
                 else red_add_v4(out + 4 * c, dv);
             }
         }
         if (lane == 0) {
-            if (!DET && rc.slot >= 0) v.dirty[rc.slot] = 1u;
+            if (!DET && chot && v.dirty[rc.slot] == 0u) v.dirty[rc.slot] = 1u;
             if (v.count) note_access(v, kc, rc.slot, DET ? 1u : 2u);
             if (v.owner) { request_localize(v, ko, q, req, req_cap); request_localize(v, kc, q, req, req_cap); }
-            loss_item[i] = loss;
+            if (DET) loss_item[i] = loss;
         }
+        my_loss += (double)loss;
+    }
+    if (!DET) {
+        if (lane == 0) warp_loss[threadIdx.x >> 5] = my_loss;
+        __syncthreads();
+        loss_finish(v.st, warp_loss[0] + warp_loss[1] + warp_loss[2] + warp_loss[3], n, loss_out);
     }
 }
 
@@ -254,7 +352,7 @@ __device__ __forceinline__ void adagrad_push(const View& v, uint32_t key, uint32
         }
     }
     if (lane == 0) {
-        if (!DET && rv.slot >= 0) v.dirty[rv.slot] = 1u;
+        if (!DET && rv.slot >= 0 && v.dirty[rv.slot] == 0u) v.dirty[rv.slot] = 1u;
         if (v.count) {
             unsigned times = (pulled_too ? 1u : 0u) + (DET ? 0u : 1u);
             if (times) note_access(v, key, rv.slot, times);
@@ -394,8 +492,8 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
         }
         if (lane == 0) {
             if (!DET) {
-                if (rw.slot >= 0) v.dirty[rw.slot] = 1u;
-                if (rh.slot >= 0) v.dirty[rh.slot] = 1u;
+                if (rw.slot >= 0 && v.dirty[rw.slot] == 0u) v.dirty[rw.slot] = 1u;
+                if (rh.slot >= 0 && v.dirty[rh.slot] == 0u) v.dirty[rh.slot] = 1u;
             }
             if (v.count) {
                 note_access(v, ki, rw.slot, DET ? 1u : 2u);
@@ -457,7 +555,7 @@ static nups_status step_buffers(nups_store* s, uint64_t n, uint64_t per, bool tw
 }
 
 static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t direct_keys, const StepBuffers& b,
-                               float* d_loss_out, cudaStream_t st)
+                               float* d_loss_out, cudaStream_t st, bool loss_done_in_kernel = false)
 {
     nups_status rc;
     if (s->cfg.deterministic) {
@@ -466,7 +564,7 @@ static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t
     }
     rc = nups_localize_apply(s, n * direct_keys, st);
     if (rc != NUPS_OK) return rc;
-    if (d_loss_out) {
+    if (d_loss_out && !loss_done_in_kernel) {
         loss_mean_kernel<<<1, 256, 0, st>>>(b.loss_item, n, d_loss_out);
         LAUNCH_CHECK(s);
     }
@@ -516,10 +614,10 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
     unsigned grid = step_grid(s, n);
     nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, sgns_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+        v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap)));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
-    return step_finish(s, n, K + 2, 2, b, d_loss_out, st);
+    return step_finish(s, n, K + 2, 2, b, d_loss_out, st, !s->cfg.deterministic);
 }
 
 extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, const uint32_t* d_r, const uint32_t* d_t,

@@ -253,42 +253,58 @@ extern "C" nups_status nups_init_uniform(nups_store* s, int which, uint64_t seed
 }
 
 // ---------------------------------------------------------------------------------------------
-// pull: row gather.  One warp walks windows of 32 keys; each lane fetches one key of the window,
-// the warp then copies the rows four at a time with 128-bit loads and streaming stores.
+// pull: row gather.  One warp walks windows of 32 keys; each lane fetches one key of the window and
+// turns it into the offset of its row (and of the worker's pending replica row, if the key is
+// replicated); the warp then copies the rows four at a time with 128-bit loads and streaming
+// stores.  TWO = also copy the matching rows of a second table.
 // ---------------------------------------------------------------------------------------------
 constexpr int GATHER_UNROLL = 4;
+constexpr unsigned long long NO_ROW = ~0ull;
 
-template <bool HOT>
-__global__ void __launch_bounds__(256)
-gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, float4* __restrict__ out_val,
-              float4* __restrict__ out_acc, int map, uint64_t map_base, uint64_t map_total, uint32_t rows_per_item,
-              int do_count)
+struct TablePair {
+    const float4* table;   // stored rows
+    const float4* slab;    // pending replica updates [R][Hcap][L]
+    float4* out;           // [n][L]
+};
+
+template <bool HOT, bool TWO>
+__global__ void __launch_bounds__(256, 4)
+gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A, TablePair B, int map,
+              uint64_t map_base, uint64_t map_total, int do_count)
 {
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t L4 = v.L4;
-    const float4* val4 = (const float4*)v.val;
-    const float4* acc4 = (const float4*)v.acc;
-    const float4* dval4 = (const float4*)v.dval;
-    const float4* dacc4 = (const float4*)v.dacc;
-    for (uint64_t base = warp * 32; base < n; base += nwarps * 32) {
-        uint64_t i = base + lane;
-        uint32_t key = i < n ? __ldg(keys + i) : 0u;
-        bool in = i < n;
-        bool valid = in && key < v.num_keys;
+    // Lookups run ahead of the copies: while window w is copied, the key of window w + 2 and the
+    // hot-bit word of window w + 1 are already on their way.
+    const uint64_t stride = nwarps * 32;
+    uint64_t base = warp * 32;
+    uint32_t key_a = base + lane < n ? __ldg(keys + base + lane) : 0u;                         // window w
+    uint32_t key_b = base + stride + lane < n ? __ldg(keys + base + stride + lane) : 0u;       // window w + 1
+    uint32_t bits_a = (HOT && key_a < v.num_keys) ? __ldg(v.hot_bits + (key_a >> 5)) : 0u;
+    for (; base < n; base += stride) {
+        const uint64_t i = base + lane;
+        const bool in = i < n;
+        const uint32_t key = key_a;
+        const uint32_t bits = bits_a;
+        key_a = key_b;
+        bits_a = (HOT && key_a < v.num_keys) ? __ldg(v.hot_bits + (key_a >> 5)) : 0u;
+        key_b = base + 2 * stride + lane < n ? __ldg(keys + base + 2 * stride + lane) : 0u;
+        const bool valid = in && key < v.num_keys;
         if (in && !valid) flag_bad_key(v);
-        int slot = -1;
-        uint32_t q = 0;
-        if (HOT && valid && key_is_hot(v, key)) {
-            slot = __ldg(v.slot_of + key);
-            uint64_t idx = map_base + i;
-            q = map == 0 ? worker_of_item(idx / rows_per_item, map_total, v.R) : chunk_of_pos(idx, map_total, v.R);
+        unsigned long long src = valid ? (unsigned long long)key * L4 : NO_ROW;   // NO_ROW: zero-filled output
+        unsigned long long pend = NO_ROW;
+        if (HOT && valid && ((bits >> (key & 31)) & 1u)) {
+            const uint32_t slot = (uint32_t)__ldg(v.slot_of + key);
+            const uint64_t idx = map_base + i;
+            const uint32_t q = map == 0 ? worker_of_item(idx, map_total, v.R) : chunk_of_pos(idx, map_total, v.R);
+            pend = ((unsigned long long)q * v.Hcap + slot) * L4;
         }
         if (do_count && v.count) {
             if (valid) atomicAdd(v.cnt + key, 1ull);
-            unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && slot >= 0);
-            unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && slot < 0);
+            unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && pend != NO_ROW);
+            unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && pend == NO_ROW);
             if (lane == 0) {
                 if (hot_m) atomicAdd(&v.st->hot_hits, (unsigned long long)__popc(hot_m));
                 if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
@@ -296,41 +312,39 @@ gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, float4* __r
         }
         const int rows = (int)min((uint64_t)32, n - base);
         for (int r = 0; r < rows; r += GATHER_UNROLL) {
-            uint32_t k[GATHER_UNROLL];
-            int sl[GATHER_UNROLL];
-            uint32_t qq[GATHER_UNROLL];
-            bool ok[GATHER_UNROLL];
+            unsigned long long so[GATHER_UNROLL], po[GATHER_UNROLL];
 #pragma unroll
             for (int u = 0; u < GATHER_UNROLL; ++u) {
-                int src = min(r + u, 31);
-                k[u] = __shfl_sync(0xFFFFFFFFu, key, src);
-                sl[u] = __shfl_sync(0xFFFFFFFFu, slot, src);
-                qq[u] = __shfl_sync(0xFFFFFFFFu, q, src);
-                ok[u] = __shfl_sync(0xFFFFFFFFu, (int)valid, src) != 0;
+                const int from = min(r + u, 31);
+                so[u] = __shfl_sync(0xFFFFFFFFu, src, from);
+                po[u] = HOT ? __shfl_sync(0xFFFFFFFFu, pend, from) : NO_ROW;
+                if (r + u >= rows) so[u] = NO_ROW;
             }
             for (uint32_t c = lane; c < L4; c += 32) {
                 float4 a[GATHER_UNROLL], b[GATHER_UNROLL];
 #pragma unroll
                 for (int u = 0; u < GATHER_UNROLL; ++u) {
                     a[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    b[u] = a[u];
-                    if (r + u < rows && ok[u]) {
-                        uint64_t ro = (uint64_t)k[u] * L4 + c;
-                        if (out_val) a[u] = __ldg(val4 + ro);
-                        if (out_acc) b[u] = __ldg(acc4 + ro);
-                        if (HOT && sl[u] >= 0) {
-                            uint64_t so = ((uint64_t)qq[u] * v.Hcap + (uint64_t)sl[u]) * L4 + c;
-                            if (out_val) a[u] = add4(a[u], dval4[so]);
-                            if (out_acc) b[u] = add4(b[u], dacc4[so]);
+                    if (TWO) b[u] = a[u];
+                    if (so[u] != NO_ROW) {
+                        // with a hot tier, rows of non-replicated keys are unlikely to be read again soon:
+                        // fetch them with the streaming hint so that they do not push the technique
+                        // bitmap and the replicated rows out of L2
+                        if (HOT && po[u] == NO_ROW) a[u] = ld_stream_v4(A.table + so[u] + c);
+                        else a[u] = __ldg(A.table + so[u] + c);
+                        if (TWO) b[u] = __ldg(B.table + so[u] + c);
+                        if (HOT && po[u] != NO_ROW) {
+                            a[u] = add4(a[u], A.slab[po[u] + c]);
+                            if (TWO) b[u] = add4(b[u], B.slab[po[u] + c]);
                         }
                     }
                 }
 #pragma unroll
                 for (int u = 0; u < GATHER_UNROLL; ++u) {
                     if (r + u < rows) {
-                        uint64_t oo = (base + r + u) * L4 + c;
-                        if (out_val) st_stream_v4(out_val + oo, a[u]);
-                        if (out_acc) st_stream_v4(out_acc + oo, b[u]);
+                        const uint64_t oo = (base + r + u) * L4 + c;
+                        st_stream_v4(A.out + oo, a[u]);
+                        if (TWO) st_stream_v4(B.out + oo, b[u]);
                     }
                 }
             }
@@ -344,14 +358,19 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
 {
     if (n == 0 || (!d_out_val && !d_out_acc)) return NUPS_OK;
     View v = nups_view(s);
-    unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 8);
+    TablePair V = {(const float4*)s->val, (const float4*)s->dval, (float4*)d_out_val};
+    TablePair C = {(const float4*)s->acc, (const float4*)s->dacc, (float4*)d_out_acc};
+    const bool two = d_out_val && d_out_acc;
+    TablePair A = d_out_val ? V : C, B = C;
+    unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 4);     // 4 resident blocks per SM, grid-stride
     nups_time_begin(s, st);
-    if (s->H)
-        gather_kernel<true><<<grid, 256, 0, st>>>(v, d_keys, n, (float4*)d_out_val, (float4*)d_out_acc, worker_map,
-                                                  map_base, map_total, 1, do_count);
-    else
-        gather_kernel<false><<<grid, 256, 0, st>>>(v, d_keys, n, (float4*)d_out_val, (float4*)d_out_acc, worker_map,
-                                                   map_base, map_total, 1, do_count);
+    if (s->H) {
+        if (two) gather_kernel<true, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
+        else gather_kernel<true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
+    } else {
+        if (two) gather_kernel<false, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
+        else gather_kernel<false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
+    }
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return NUPS_OK;
@@ -376,107 +395,211 @@ extern "C" nups_status nups_pull(nups_store* s, const uint32_t* d_keys, uint64_t
 // push, fast mode: 128-bit reductions straight to the destination row.  Within a window of 32
 // rows, rows with the same destination are summed in registers first (__match_any_sync) so that
 // a hot destination receives one reduction per window instead of one per row.
+// TWO = a second table gets its own deltas from the same call.
 // ---------------------------------------------------------------------------------------------
 constexpr int PUSH_UNROLL = 4;
 
-template <bool HOT>
-__global__ void __launch_bounds__(256)
-push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const float4* __restrict__ dv,
-                   const float4* __restrict__ da, uint64_t n_items, uint32_t rows_per_item)
+struct PushPair {
+    const float4* delta;   // [n][L] updates
+    float* table;          // stored rows
+    float* slab;           // replica slabs
+};
+
+// TIER = the block keeps shared-memory accumulators for the hottest replica slots (slot < tier_rows)
+// of ONE worker (block b serves worker b mod R and visits only that worker's share of the windows);
+// updates to those slots are added in shared memory and reach the worker's replica once, when the
+// block ends.  This is what keeps thousands of additions to one hot row from queueing at one L2
+// address.
+template <bool HOT, bool TWO, bool TIER>
+__global__ void __launch_bounds__(256, 3)
+push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPair A, PushPair B, uint64_t n_items,
+                   uint32_t rows_per_item, uint32_t tier_rows)
 {
+    extern __shared__ __align__(16) float tier_mem[];                  // TIER: [tier_rows][L] sums, then touched bits
     const unsigned lane = threadIdx.x & 31;
-    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t L4 = v.L4;
-    for (uint64_t base = warp * 32; base < n; base += nwarps * 32) {
-        uint64_t i = base + lane;
-        bool in = i < n;
-        uint32_t key = in ? __ldg(keys + i) : 0u;
-        bool valid = in && key < v.num_keys;
+    const uint32_t R = v.R;
+    unsigned* touched = reinterpret_cast<unsigned*>(tier_mem + (size_t)tier_rows * L4 * 4);
+    if (TIER) {
+        float4* z = reinterpret_cast<float4*>(tier_mem);
+        for (uint32_t e = threadIdx.x; e < tier_rows * L4; e += blockDim.x) z[e] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t e = threadIdx.x; e < (tier_rows + 31) / 32; e += blockDim.x) touched[e] = 0u;
+        __syncthreads();
+    }
+    // Windows are visited in an order that interleaves the workers' chunks: the window range is cut
+    // into R stretches of `per` windows; without the tier, slot u of the schedule is window
+    // (u mod R) * per + u / R, so warps that run at the same time add to different replicas of a
+    // hot key; with the tier, a block walks the stretch of its own worker only.
+    const uint64_t W = (n + 31) / 32;
+    const uint64_t per = (W + R - 1) / R;
+    const uint32_t my_q = TIER ? blockIdx.x % R : 0u;
+    const uint64_t warp = TIER ? ((uint64_t)(blockIdx.x / R) * blockDim.x + threadIdx.x) >> 5
+                               : ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = TIER ? ((uint64_t)(gridDim.x / R) * blockDim.x) >> 5 : ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint64_t slots = TIER ? per : per * R;
+    auto window_of = [&](uint64_t u) -> uint64_t {
+        if (u >= slots) return W;
+        const uint64_t w = TIER ? (uint64_t)my_q * per + u : (u % R) * per + u / R;
+        return (w < W) ? w : W;
+    };
+    auto load_key = [&](uint64_t w) -> uint32_t {
+        return (w < W && w * 32 + lane < n) ? __ldg(keys + w * 32 + lane) : NUPS_INVALID_KEY;
+    };
+    // lookups run two windows ahead of the reductions
+    uint64_t win_a = window_of(warp), win_b = window_of(warp + nwarps);
+    uint32_t key_a = load_key(win_a), key_b = load_key(win_b);
+    uint32_t bits_a = (HOT && key_a < v.num_keys) ? __ldg(v.hot_bits + (key_a >> 5)) : 0u;
+    for (uint64_t u = warp; u < slots; u += nwarps) {
+        const uint64_t win = win_a;
+        const uint32_t key = key_a;
+        const uint32_t bits = bits_a;
+        win_a = win_b; key_a = key_b;
+        bits_a = (HOT && key_a < v.num_keys) ? __ldg(v.hot_bits + (key_a >> 5)) : 0u;
+        win_b = window_of(u + 2 * nwarps);
+        key_b = load_key(win_b);
+        if (win >= W) continue;
+        const uint64_t base = win * 32;
+        const uint64_t i = base + lane;
+        const bool in = i < n;
+        const bool valid = in && key < v.num_keys;
         if (in && !valid) flag_bad_key(v);
-        int slot = -1;
-        uint64_t row = 0;                 // destination row offset (in float4) inside its table or slab
+        // destination: row offset in floats, lowest bit set when it lies in the replica slab
+        unsigned long long dest = NO_ROW - lane;          // invalid rows: a value no other lane has
+        bool hot = false;
+        uint32_t hslot = 0;
+        int tier = -1;                                    // shared-memory accumulator of this row, if any
         if (valid) {
-            row = (uint64_t)key * L4;
-            if (HOT && key_is_hot(v, key)) {
-                slot = __ldg(v.slot_of + key);
-                uint32_t q = worker_of_item(i / rows_per_item, n_items, v.R);
-                row = ((uint64_t)q * v.Hcap + (uint64_t)slot) * L4;
-                v.dirty[slot] = 1u;
+            dest = ((unsigned long long)key * L4) << 3;
+            if (HOT && ((bits >> (key & 31)) & 1u)) {
+                hot = true;
+                const uint32_t slot = (uint32_t)__ldg(v.slot_of + key);
+                const uint32_t q = rows_per_item == 1 ? worker_of_item(i, n_items, R)
+                                                      : worker_of_item(i / rows_per_item, n_items, R);
+                dest = ((((unsigned long long)q * v.Hcap + slot) * L4) << 3) | 1ull;
+                hslot = slot;
+                if (TIER && slot < tier_rows && q == my_q) tier = (int)slot;
             }
         }
         if (v.count) {
             if (valid) atomicAdd(v.cnt + key, 1ull);
-            unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && slot >= 0);
-            unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && slot < 0);
+            unsigned hot_m = __ballot_sync(0xFFFFFFFFu, valid && hot);
+            unsigned cold_m = __ballot_sync(0xFFFFFFFFu, valid && !hot);
             if (lane == 0) {
                 if (hot_m) atomicAdd(&v.st->hot_hits, (unsigned long long)__popc(hot_m));
                 if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
             }
         }
-        // destination identity: (replica?, row offset); invalid rows get a value no one shares
-        unsigned long long dest = valid ? ((row << 1) | (slot >= 0 ? 1ull : 0ull)) : (~0ull - lane);
-        unsigned grp = __match_any_sync(0xFFFFFFFFu, dest);
-        bool leader = valid && (lane == (unsigned)(__ffs(grp) - 1));
+        const unsigned grp = __match_any_sync(0xFFFFFFFFu, dest);
+        const bool leader = valid && (lane == (unsigned)(__ffs(grp) - 1));
+        // mark the slot as touched: one lane per destination, and only if nobody has yet (a hot slot would
+        // otherwise take hundreds of thousands of stores to one address)
+        if (HOT && leader && hot && v.dirty[hslot] == 0u) v.dirty[hslot] = 1u;
         unsigned singles = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) == 1);
         unsigned multis = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) > 1);
 
         // rows that are alone in their window: four at a time
         while (singles) {
-            int src[PUSH_UNROLL];
-            uint64_t ro[PUSH_UNROLL];
-            int hs[PUSH_UNROLL];
+            int src[PUSH_UNROLL], tr[PUSH_UNROLL];
+            unsigned long long de[PUSH_UNROLL];
 #pragma unroll
-            for (int u = 0; u < PUSH_UNROLL; ++u) {
-                if (singles) {
-                    src[u] = __ffs(singles) - 1;
-                    singles &= singles - 1;
-                } else src[u] = -1;
-                int from = src[u] < 0 ? 0 : src[u];
-                ro[u] = __shfl_sync(0xFFFFFFFFu, row, from);
-                hs[u] = __shfl_sync(0xFFFFFFFFu, slot, from);
+            for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
+                src[u4] = singles ? __ffs(singles) - 1 : -1;
+                singles &= singles - 1;
+                de[u4] = __shfl_sync(0xFFFFFFFFu, dest, src[u4] < 0 ? 0 : src[u4]);
+                tr[u4] = TIER ? __shfl_sync(0xFFFFFFFFu, tier, src[u4] < 0 ? 0 : src[u4]) : -1;
             }
             for (uint32_t c = lane; c < L4; c += 32) {
                 float4 a[PUSH_UNROLL], b[PUSH_UNROLL];
 #pragma unroll
-                for (int u = 0; u < PUSH_UNROLL; ++u) {
-                    if (src[u] >= 0) {
-                        uint64_t in_off = (base + src[u]) * L4 + c;
-                        if (dv) a[u] = ld_stream_v4(dv + in_off);
-                        if (da) b[u] = ld_stream_v4(da + in_off);
+                for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
+                    if (src[u4] >= 0) {
+                        const uint64_t in_off = (base + src[u4]) * L4 + c;
+                        a[u4] = ld_stream_v4(A.delta + in_off);
+                        if (TWO) b[u4] = ld_stream_v4(B.delta + in_off);
                     }
                 }
 #pragma unroll
-                for (int u = 0; u < PUSH_UNROLL; ++u) {
-                    if (src[u] >= 0) {
-                        bool hot = HOT && hs[u] >= 0;
-                        if (dv) red_add_v4((hot ? v.dval : v.val) + (ro[u] + c) * 4, a[u]);
-                        if (da) red_add_v4((hot ? v.dacc : v.acc) + (ro[u] + c) * 4, b[u]);
+                for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
+                    if (src[u4] >= 0) {
+                        if (TIER && tr[u4] >= 0) {
+                            // accumulator rows are stored component by component, [4][L4], so that the 32
+                            // lanes of one addition fall into 32 different banks
+                            float* t = tier_mem + (size_t)tr[u4] * L4 * 4 + c;
+                            atomicAdd(t, a[u4].x); atomicAdd(t + L4, a[u4].y); atomicAdd(t + 2 * L4, a[u4].z);
+                            atomicAdd(t + 3 * L4, a[u4].w);
+                        } else {
+                            const bool h = HOT && (de[u4] & 1ull);
+                            const uint64_t off = (de[u4] >> 3) * 4 + (uint64_t)c * 4;
+                            red_add_v4((h ? A.slab : A.table) + off, a[u4]);
+                            if (TWO) red_add_v4((h ? B.slab : B.table) + off, b[u4]);
+                        }
                     }
                 }
             }
+            if (TIER && lane == 0) {
+#pragma unroll
+                for (int u4 = 0; u4 < PUSH_UNROLL; ++u4)
+                    if (src[u4] >= 0 && tr[u4] >= 0 && !((touched[tr[u4] >> 5] >> (tr[u4] & 31)) & 1u))
+                        atomicOr(&touched[tr[u4] >> 5], 1u << (tr[u4] & 31));
+            }
         }
-        // destinations hit more than once in the window: sum the members, one reduction
+        // destinations hit more than once in the window: sum the members (loads four at a time), one reduction
         while (multis) {
-            int ld = __ffs(multis) - 1;
+            const int ld = __ffs(multis) - 1;
             multis &= multis - 1;
-            unsigned members = __shfl_sync(0xFFFFFFFFu, grp, ld);
-            uint64_t ro = __shfl_sync(0xFFFFFFFFu, row, ld);
-            int hs = __shfl_sync(0xFFFFFFFFu, slot, ld);
-            bool hot = HOT && hs >= 0;
+            const unsigned members = __shfl_sync(0xFFFFFFFFu, grp, ld);
+            const unsigned long long de = __shfl_sync(0xFFFFFFFFu, dest, ld);
+            const int tr = TIER ? __shfl_sync(0xFFFFFFFFu, tier, ld) : -1;
+            const bool h = HOT && (de & 1ull);
             for (uint32_t c = lane; c < L4; c += 32) {
                 float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
                 unsigned mm = members;
                 while (mm) {
-                    int m = __ffs(mm) - 1;
-                    mm &= mm - 1;
-                    uint64_t in_off = (base + m) * L4 + c;
-                    if (dv) a = add4(a, ld_stream_v4(dv + in_off));
-                    if (da) b = add4(b, ld_stream_v4(da + in_off));
+                    int m[PUSH_UNROLL];
+                    float4 x[PUSH_UNROLL], y[PUSH_UNROLL];
+#pragma unroll
+                    for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
+                        m[u4] = mm ? __ffs(mm) - 1 : -1;
+                        mm &= mm - 1;
+                    }
+#pragma unroll
+                    for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
+                        if (m[u4] >= 0) {
+                            const uint64_t in_off = (base + m[u4]) * L4 + c;
+                            x[u4] = ld_stream_v4(A.delta + in_off);
+                            if (TWO) y[u4] = ld_stream_v4(B.delta + in_off);
+                        }
+                    }
+#pragma unroll
+                    for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
+                        if (m[u4] >= 0) {
+                            a = add4(a, x[u4]);
+                            if (TWO) b = add4(b, y[u4]);
+                        }
+                    }
                 }
-                if (dv) red_add_v4((hot ? v.dval : v.val) + (ro + c) * 4, a);
-                if (da) red_add_v4((hot ? v.dacc : v.acc) + (ro + c) * 4, b);
+                if (TIER && tr >= 0) {
+                    float* t = tier_mem + (size_t)tr * L4 * 4 + c;
+                    atomicAdd(t, a.x); atomicAdd(t + L4, a.y); atomicAdd(t + 2 * L4, a.z); atomicAdd(t + 3 * L4, a.w);
+                } else {
+                    const uint64_t off = (de >> 3) * 4 + (uint64_t)c * 4;
+                    red_add_v4((h ? A.slab : A.table) + off, a);
+                    if (TWO) red_add_v4((h ? B.slab : B.table) + off, b);
+                }
             }
+            if (TIER && tr >= 0 && lane == 0 && !((touched[tr >> 5] >> (tr & 31)) & 1u))
+                atomicOr(&touched[tr >> 5], 1u << (tr & 31));
+        }
+    }
+    if (TIER) {
+        // hand the block's sums to the worker's replica: one reduction per touched row
+        __syncthreads();
+        for (uint32_t sl = threadIdx.x >> 5; sl < tier_rows; sl += blockDim.x >> 5) {
+            if (!((touched[sl >> 5] >> (sl & 31)) & 1u)) continue;
+            float* dst = A.slab + ((size_t)my_q * v.Hcap + sl) * L4 * 4;
+            const float* t = tier_mem + (size_t)sl * L4 * 4;
+            for (uint32_t c = lane; c < L4; c += 32)
+                red_add_v4(dst + (size_t)c * 4, make_float4(t[c], t[c + L4], t[c + 2 * L4], t[c + 3 * L4]));
         }
     }
 }
@@ -505,7 +628,7 @@ __global__ void push_dest_kernel(View v, const uint32_t* __restrict__ keys, uint
             uint32_t slot = (uint32_t)v.slot_of[key];
             uint32_t q = worker_of_item(i / rows_per_item, n_items, v.R);
             d = (1ull << 32) + (unsigned long long)q * v.H + slot;
-            v.dirty[slot] = 1u;
+            if (v.dirty[slot] == 0u) v.dirty[slot] = 1u;
         }
     }
     if (in) { dest[i] = d; idx[i] = (uint32_t)i; }
@@ -602,14 +725,40 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
     View v = nups_view(s);
     uint64_t n_items = n / rows_per_item;
     if (!s->cfg.deterministic) {
-        unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 8);
+        unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 3);  // 3 resident blocks per SM, grid-stride
+        PushPair V = {(const float4*)d_dval, s->val, s->dval};
+        PushPair C = {(const float4*)d_dacc, s->acc, s->dacc};
+        const bool two = d_dval && d_dacc;
+        PushPair A = d_dval ? V : C, B = C;
+        // shared-memory tier: single-table calls with replicated keys, enough blocks to give every worker some
+        uint32_t tier_rows = 0;
+        size_t tier_bytes = 0;
+        if (s->H && !two && rows_per_item == 1 && grid >= s->R && n >= 32768) {
+            const size_t row_bytes = (size_t)s->L * 4;
+            size_t budget = 64 * 1024;
+            tier_rows = s->cfg.smem_hot_rows ? s->cfg.smem_hot_rows : (uint32_t)(budget / row_bytes);
+            if (tier_rows > budget / row_bytes) tier_rows = (uint32_t)(budget / row_bytes);
+            if (tier_rows > s->H) tier_rows = (uint32_t)s->H;
+            tier_bytes = tier_rows * row_bytes + ((tier_rows + 31) / 32) * 4;
+            static bool attr_set = false;
+            if (tier_rows && !attr_set) {
+                CK(cudaFuncSetAttribute(push_atomic_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(budget + 1024)));
+                attr_set = true;
+            }
+        }
         nups_time_begin(s, st);
-        if (s->H)
-            push_atomic_kernel<true><<<grid, 256, 0, st>>>(v, d_keys, n, (const float4*)d_dval, (const float4*)d_dacc,
-                                                           n_items, rows_per_item);
-        else
-            push_atomic_kernel<false><<<grid, 256, 0, st>>>(v, d_keys, n, (const float4*)d_dval, (const float4*)d_dacc,
-                                                            n_items, rows_per_item);
+        if (tier_rows) {
+            grid = grid / s->R * s->R;              // every worker gets the same number of blocks
+            push_atomic_kernel<true, false, true><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+                                                                                tier_rows);
+        } else if (s->H) {
+            if (two) push_atomic_kernel<true, true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+            else push_atomic_kernel<true, false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+        } else {
+            if (two) push_atomic_kernel<false, true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+            else push_atomic_kernel<false, false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+        }
         nups_time_end(s, st);
         LAUNCH_CHECK(s);
         return NUPS_OK;

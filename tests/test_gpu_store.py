@@ -204,3 +204,44 @@ def test_localize_and_owner_map():
     got = s.owner_of(dev_keys(allk)).cpu().numpy()
     want = np.array([o.owner_of(k) for k in allk])
     assert np.array_equal(got, want)
+
+
+@pytest.mark.parametrize("L", [4, 128, 300, 500])
+@pytest.mark.parametrize("hot_n", [0, 300])
+def test_large_calls_take_the_staged_path_and_stay_exact(L, hot_n):
+    # calls of 16384 keys and more run as persistent blocks that stage rows through shared memory;
+    # ragged tail, keys out of range and replicated keys with pending updates included
+    nk, R = 20000, 5
+    rng = np.random.default_rng(L + hot_n)
+    init = rand_table(nk, L)
+    o, s = make_pair(nk, L, R=R, init=init, deterministic=False, count_accesses=True)
+    if hot_n:
+        hot = rng.permutation(nk)[:hot_n].astype(np.uint32)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    exact = init.astype(np.float64)
+    for n in (16384, 70001):
+        keys = (rng.zipf(1.15, n) % nk).astype(np.uint32)
+        keys[rng.integers(0, n, 5)] = nk + 7                      # bad keys: skipped, output zero-filled
+        d = rng.normal(size=(n, L)).astype(np.float32)
+        o.push(keys, d)
+        s.push(dev_keys(keys), dev_f32(d))
+        ok = keys < nk
+        np.add.at(exact, keys[ok], d[ok].astype(np.float64))
+        got = s.pull(dev_keys(keys)).cpu().numpy()
+        want = o.pull(keys)
+        scale = max(1.0, np.abs(want).max())
+        assert np.abs(got - want).max() < 3e-5 * scale            # pending updates were added in another order
+        assert np.all(got[~ok] == 0)
+        assert s.status_check() == -4
+    o.sync()
+    s.sync()
+    got = s.read_table().cpu().numpy()
+    assert np.abs(got - exact).max() < 3e-5 * np.abs(exact).max()
+    # a pull with nothing pending is an exact copy
+    keys = rng.integers(0, nk, 50000).astype(np.uint32)
+    assert np.array_equal(s.pull(dev_keys(keys)).cpu().numpy(), got[keys])
+    o.pull(keys)
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+    st, so = s.stats(), o.stats()
+    assert st["hot"] == so["hot"] and st["cold"] == so["cold"]
