@@ -238,7 +238,8 @@ nups_status nups_pull_sample(nups_store* store, nups_handle handle, uint64_t n, 
 
 /* Skip-gram with negative sampling: centre key c, context key o, negatives u_j:
  * x_j = v.u_j, g_j = sigmoid(x_j) - [j = 0], u_j -= lr g_j v, v -= lr sum g_j u_j,
- * loss = -log sigmoid(x_0) - sum_j log sigmoid(-x_j); scores clamped to +-30.  */
+ * loss = -log sigmoid(x_0) - sum_j log sigmoid(-x_j); scores clamped to +-30.
+ * K <= 30.                                                                    */
 nups_status nups_step_sgns(nups_store* store, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_pairs,
                            int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream);
 

@@ -14,6 +14,8 @@
 #define NUPS_INVALID_KEY 0xFFFFFFFFu
 #define NUPS_MAX_POOL 1024
 #define NUPS_MAX_TIMED 4096
+#define NUPS_MAX_STEP_BLOCKS 8192
+#define NUPS_SAMPLE_AHEAD 16
 
 // ---------------------------------------------------------------------------------------------
 // Device-resident status and statistics
@@ -40,6 +42,7 @@ struct View {
     uint8_t* owner;            // [num_keys] owning worker or NUPS_OWNER_DEFAULT; NULL = not tracked
     int* pending;              // [num_keys] localize requests of the running call (-1 = none)
     DevStat* st;
+    double* loss_partial;      // [4 * NUPS_MAX_STEP_BLOCKS] per-warp loss sums of the running step kernel
     uint64_t num_keys;
     uint64_t Hcap;
     uint32_t H;
@@ -86,12 +89,18 @@ struct nups_store {
     uint8_t* owner;
     int* pending;
     DevStat* st;
+    double* loss_partial;
     char* scratch;
     size_t scratch_bytes;
     uint32_t* req_keys;        // localize request list of the running call
     size_t req_cap;
-    uint32_t* last_negs;
-    uint64_t last_negs_n, last_negs_cap;
+    uint32_t* negs_buf;        // negatives drawn for the workload steps, possibly several batches ahead
+    uint64_t negs_cap;
+    uint32_t* last_negs;       // the slice of negs_buf that the most recent step used
+    uint64_t last_negs_n;
+    int ahead_dist;            // sample-ahead state: batches [ahead_next, ahead_total) of ahead_N samples
+    uint64_t ahead_N;          // from ahead_dist are drawn but not handed out yet (-1 = none)
+    uint32_t ahead_total, ahead_next;
     uint64_t steps, syncs, launches;
     int device, sm_count, max_smem;
     int timing;                // record events around the main kernels?
@@ -159,6 +168,7 @@ nups_status nups_localize_apply(nups_store* s, uint64_t max_requests, cudaStream
 nups_status nups_sync_internal(nups_store* s, cudaStream_t st);
 // sampling.cu internals used by steps.cu
 nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st);
+nups_status nups_sample_ahead_rewind(nups_store* s, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------------
 // Device helpers
@@ -227,6 +237,12 @@ __device__ __forceinline__ bool key_is_local(const View& v, uint32_t q, uint32_t
     if (!v.owner) return true;
     uint32_t o = v.owner[k];
     return (o == NUPS_OWNER_DEFAULT ? k % v.R : o) == q;
+}
+
+// mark a replica slot as touched without waiting for anything to come back
+__device__ __forceinline__ void mark_dirty(const View& v, int slot)
+{
+    asm volatile("red.global.or.b32 [%0], 1;" ::"l"(v.dirty + slot) : "memory");
 }
 
 __device__ __forceinline__ void flag_bad_key(const View& v) { atomicCAS(&v.st->status, 0, NUPS_EKEY); }

@@ -318,6 +318,10 @@ __global__ void localize_handle_kernel(View v, const uint32_t* __restrict__ keys
 static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int* slot_out, cudaStream_t st)
 {
     if (dist < 0 || dist >= NUPS_MAX_DISTS || !s->dist[dist].used || N == 0 || N >= (1ull << 32)) return NUPS_EINVAL;
+    if (s->ahead_dist == dist) {
+        nups_status rw = nups_sample_ahead_rewind(s, st);       // samples drawn ahead for the steps go back
+        if (rw != NUPS_OK) return rw;
+    }
     Dist& d = s->dist[dist];
     size_t need = handle_bytes(N, s->R, d.level);
     int id = -1;
@@ -542,16 +546,21 @@ __device__ __forceinline__ void direct_tail(const View& v, uint32_t key, uint32_
     }
 }
 
+// blockIdx.y (iid) / blockIdx.z (reuse) = batch: `batches` handles of N samples each are drawn back to back,
+// exactly as that many separate calls would draw them; batch b goes to out + b * N.
 __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long long* off_cur,
-                                       unsigned long long* off_next, uint64_t N, int local_only, int localize,
-                                       uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+                                       unsigned long long* off_next, uint64_t N, uint32_t batches, int local_only,
+                                       int localize, uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
 {
     const uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t bt = blockIdx.y;
     const bool in = o < N;
     uint32_t k = 0, q = 0;
+    out += (uint64_t)bt * N;
     if (in) {
         q = chunk_of_pos(o, N, v.R);
-        k = draw_iid(p, q, off_cur[q] + (o - chunk_begin(q, N, v.R)));
+        const unsigned long long size = chunk_begin(q + 1, N, v.R) - chunk_begin(q, N, v.R);
+        k = draw_iid(p, q, off_cur[q] + (unsigned long long)bt * size + (o - chunk_begin(q, N, v.R)));
         if (local_only) {
             const uint32_t k0 = k;
             for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
@@ -562,25 +571,26 @@ __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long
         out[o] = k;
     }
     direct_tail(v, k, q, in, localize != 0, req, req_cap);
-    if (blockIdx.x == 0)
+    if (blockIdx.x == 0 && blockIdx.y == 0)
         for (uint32_t w = threadIdx.x; w < v.R; w += blockDim.x)
-            off_next[w] = off_cur[w] + (chunk_begin(w + 1, N, v.R) - chunk_begin(w, N, v.R));
+            off_next[w] = off_cur[w] + (unsigned long long)batches * (chunk_begin(w + 1, N, v.R) - chunk_begin(w, N, v.R));
 }
 
 __global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned long long* off_cur,
-                                         unsigned long long* off_next, uint64_t N, int localize,
+                                         unsigned long long* off_next, uint64_t N, uint32_t batches, int localize,
                                          uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
 {
     __shared__ uint32_t pool[NUPS_MAX_POOL];
     __shared__ uint32_t perm[NUPS_MAX_POOL];
     __shared__ uint32_t xs[NUPS_MAX_POOL];
     const uint32_t q = blockIdx.y, G = p.G, R = v.R;
-    if (blockIdx.x == 0 && blockIdx.y == 0)
+    if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         for (uint32_t w = threadIdx.x; w < R; w += blockDim.x)
-            off_next[w] = off_cur[w] + (chunk_begin(w + 1, N, R) - chunk_begin(w, N, R));
+            off_next[w] = off_cur[w] + (unsigned long long)batches * (chunk_begin(w + 1, N, R) - chunk_begin(w, N, R));
     const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
     if (size == 0) return;
-    const unsigned long long s0 = off_cur[q], s1 = s0 + size;
+    out += (uint64_t)blockIdx.z * N;
+    const unsigned long long s0 = off_cur[q] + (unsigned long long)blockIdx.z * size, s1 = s0 + size;
     const unsigned long long pass = s0 / G + blockIdx.x;
     if (pass * G >= s1) return;
     const unsigned long long pl = pass / p.U;
@@ -616,21 +626,58 @@ __global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned lo
     }
 }
 
+// Sample-ahead for the workload steps.  The sample streams are a pure function of (seed, worker,
+// position), so the negatives of the next NUPS_SAMPLE_AHEAD steps can be drawn in one launch and
+// handed out one batch per step.  If anything else touches the distribution before they are used up
+// (PrepareSample, a step with another size), the stream offsets are rewound by what was not handed out,
+// so every sample sequence is the same as without sample-ahead.  Only used where drawing early has no
+// other effect: fast mode, no access counting, no ownership tracking.
+__global__ void rewind_kernel(unsigned long long* off, uint64_t N, uint32_t R, uint32_t batches)
+{
+    const uint32_t q = threadIdx.x;
+    if (q < R) off[q] -= (unsigned long long)batches * (chunk_begin(q + 1, N, R) - chunk_begin(q, N, R));
+}
+
+nups_status nups_sample_ahead_rewind(nups_store* s, cudaStream_t st)
+{
+    if (s->ahead_dist < 0) return NUPS_OK;
+    const uint32_t left = s->ahead_total - s->ahead_next;
+    if (left) {
+        Dist& d = s->dist[s->ahead_dist];
+        rewind_kernel<<<1, 256, 0, st>>>(d.off + (size_t)d.cur * s->R, s->ahead_N, s->R, left);
+        LAUNCH_CHECK(s);
+    }
+    s->ahead_dist = -1;
+    return NUPS_OK;
+}
+
 // negatives of a workload step: one handle of N samples, pulled at once into library memory
 nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st)
 {
     s->last_negs_n = 0;
     if (N == 0) return NUPS_OK;
-    if (N > s->last_negs_cap) {
-        if (s->last_negs) CK(cudaFree(s->last_negs));
-        s->last_negs = nullptr; s->last_negs_cap = 0;
-        uint64_t want = N + N / 4;
-        if (cudaMalloc(&s->last_negs, want * 4) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
-        s->last_negs_cap = want;
-    }
     if (dist < 0 || dist >= NUPS_MAX_DISTS || !s->dist[dist].used || N >= (1ull << 32)) return NUPS_EINVAL;
+    // a batch drawn ahead for exactly this request?
+    if (s->ahead_dist == dist && s->ahead_N == N && s->ahead_next < s->ahead_total) {
+        s->last_negs = s->negs_buf + (uint64_t)s->ahead_next * N;
+        s->last_negs_n = N;
+        s->ahead_next++;
+        return NUPS_OK;
+    }
+    nups_status rc = nups_sample_ahead_rewind(s, st);
+    if (rc != NUPS_OK) return rc;
     Dist& d = s->dist[dist];
-    nups_status rc;
+    const bool plain = d.level == NUPS_CONFORM || d.level == NUPS_BOUNDED;
+    const uint32_t batches = (plain && !s->cfg.deterministic && !s->cfg.count_accesses && !s->owner &&
+                              N * NUPS_SAMPLE_AHEAD < (1ull << 28)) ? NUPS_SAMPLE_AHEAD : 1;
+    if (N * batches > s->negs_cap) {
+        if (s->negs_buf) CK(cudaFree(s->negs_buf));
+        s->negs_buf = nullptr; s->negs_cap = 0;
+        uint64_t want = N * batches + N / 4;
+        if (cudaMalloc(&s->negs_buf, want * 4) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        s->negs_cap = want;
+    }
+    s->last_negs = s->negs_buf;
     if (d.level == NUPS_LONGTERM) {
         // postponing needs the handle's walk state: PrepareSample, then one full PullSample
         int id = -1;
@@ -655,11 +702,12 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
         unsigned passes = (unsigned)(max_size / d.G + 2);
         unsigned threads = ((d.G + 31) / 32) * 32;
         if (threads > 256) threads = 256;
-        draw_direct_reuse_kernel<<<dim3(passes, s->R), threads, 0, st>>>(v, p, off_cur, off_next, N, localize, s->last_negs,
-                                                                        s->req_keys, s->req_cap);
+        draw_direct_reuse_kernel<<<dim3(passes, s->R, batches), threads, 0, st>>>(v, p, off_cur, off_next, N, batches, localize,
+                                                                                 s->negs_buf, s->req_keys, s->req_cap);
     } else {
-        draw_direct_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(v, p, off_cur, off_next, N, d.level == NUPS_NONCONFORM,
-                                                                 localize, s->last_negs, s->req_keys, s->req_cap);
+        draw_direct_iid_kernel<<<dim3(grid_for(N, 256), batches), 256, 0, st>>>(v, p, off_cur, off_next, N, batches,
+                                                                              d.level == NUPS_NONCONFORM, localize,
+                                                                              s->negs_buf, s->req_keys, s->req_cap);
     }
     LAUNCH_CHECK(s);
     d.cur ^= 1;
@@ -668,6 +716,9 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
         if (rc != NUPS_OK) return rc;
     }
     s->last_negs_n = N;
+    if (batches > 1) {
+        s->ahead_dist = dist; s->ahead_N = N; s->ahead_total = batches; s->ahead_next = 1;
+    }
     return NUPS_OK;
 }
 

@@ -69,18 +69,14 @@ struct RowAt {
 };
 constexpr unsigned long long NO_PEND = ~0ull;
 
+// The step workloads keep key -> slot small enough to stay in L2, so the slot map is read directly
+// (one lookup) instead of going through the technique bitmap first.
 template <bool HOT, int NR>
 __device__ __forceinline__ void resolve_rows(const View& v, const uint32_t (&key)[NR], const bool (&act)[NR],
                                              uint32_t q, RowAt (&r)[NR])
 {
-    uint32_t bits[NR];
 #pragma unroll
-    for (int u = 0; u < NR; ++u) bits[u] = (HOT && act[u]) ? __ldg(v.hot_bits + (key[u] >> 5)) : 0u;
-#pragma unroll
-    for (int u = 0; u < NR; ++u) {
-        const bool hot = HOT && act[u] && ((bits[u] >> (key[u] & 31)) & 1u);
-        r[u].slot = hot ? __ldg(v.slot_of + key[u]) : -1;
-    }
+    for (int u = 0; u < NR; ++u) r[u].slot = (HOT && act[u]) ? __ldg(v.slot_of + key[u]) : -1;
     const unsigned long long L = (unsigned long long)v.L4 * 4;
 #pragma unroll
     for (int u = 0; u < NR; ++u) {
@@ -89,99 +85,113 @@ __device__ __forceinline__ void resolve_rows(const View& v, const uint32_t (&key
     }
 }
 
-// per-launch loss accumulation in fast mode: warps add their item losses, the last block to finish
-// writes the mean and clears the accumulators for the next launch
-__device__ __forceinline__ void loss_finish(DevStat* st, double block_loss, uint64_t n, float* loss_out)
+// per-launch loss in fast mode: every warp stores its sum and takes a ticket from one integer counter;
+// the warp that draws the last ticket adds the sums up and writes the mean.  (Additions to one
+// floating-point address from thousands of warps would queue up at L2, and a block-wide barrier would
+// make every warp wait for the slowest one.)
+__device__ __forceinline__ void loss_finish(const View& v, double warp_loss, uint64_t n, float* loss_out)
 {
-    __shared__ bool last;
-    if (threadIdx.x == 0) {
-        atomicAdd((double*)&st->tmp[2], block_loss);
+    const unsigned lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    unsigned last = 0;
+    if (lane == 0) {
+        v.loss_partial[warp] = warp_loss;
         __threadfence();
-        unsigned long long done = atomicAdd(&st->tmp[3], 1ull) + 1;
-        last = done == gridDim.x;
-        if (last) {
-            __threadfence();
-            double total = atomicAdd((double*)&st->tmp[2], 0.0);
-            if (loss_out) *loss_out = (float)(total / (double)(n ? n : 1));
-            st->tmp[2] = 0ull;
-            st->tmp[3] = 0ull;
-        }
+        last = atomicAdd(&v.st->tmp[3], 1ull) + 1 == nwarps;
+    }
+    last = __shfl_sync(0xFFFFFFFFu, last, 0);
+    if (!last) return;
+    __threadfence();
+    double t = 0.0;
+    for (uint32_t b = lane; b < nwarps; b += 32) t += __ldcg(v.loss_partial + b);
+    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+    if (lane == 0) {
+        if (loss_out) *loss_out = (float)(t / (double)(n ? n : 1));
+        v.st->tmp[3] = 0ull;
     }
 }
 
 // ---------------------------------------------------------------------------------------------
 // skip-gram with negative sampling
 // ---------------------------------------------------------------------------------------------
-constexpr int SGNS_UB = 4;      // output rows (context + negatives) handled per group
+#ifndef NUPS_SGNS_UB
+#define NUPS_SGNS_UB 2
+#endif
+#ifndef NUPS_SGNS_MINBLOCKS
+#define NUPS_SGNS_MINBLOCKS 7
+#endif
+constexpr int SGNS_UB = NUPS_SGNS_UB;      // output rows (context + negatives) handled per group
 
 template <bool HOT, bool DET, int CH>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, NUPS_SGNS_MINBLOCKS)
 sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
             const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float* __restrict__ upd,
             uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, float* __restrict__ loss_out, uint32_t* req,
             uint64_t req_cap)
 {
-    __shared__ double warp_loss[4];
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t L4 = v.L4, per = K + 2;
+    const unsigned long long L = (unsigned long long)L4 * 4;
     const float4* val4 = (const float4*)v.val;
     const float4* slab4 = (const float4*)v.dval;
     double my_loss = 0.0;
     for (uint64_t i = warp; i < n; i += nwarps) {
         const uint32_t q = worker_of_item(i, n, v.R);
-        const uint32_t kc = center[i], ko = context[i];
-        bool ok = kc < v.num_keys && ko < v.num_keys;
-        for (uint32_t j = 0; j < K; ++j) ok = ok && negs[i * K + j] < v.num_keys;
-        if (DET && lane == 0) {
-            ukeys[i * per] = ok ? ko : NUPS_INVALID_KEY;
-            for (uint32_t j = 0; j < K; ++j) ukeys[i * per + 1 + j] = ok ? negs[i * K + j] : NUPS_INVALID_KEY;
-            ukeys[i * per + K + 1] = ok ? kc : NUPS_INVALID_KEY;
-        }
+        // lane l holds the key of row l of the item: 0 = context, 1..K = negatives, K+1 = centre;
+        // one coalesced round fetches the keys, a second one their replica slots
+        const uint32_t mykey = lane == 0 ? context[i] : (lane <= K ? negs[i * K + lane - 1] : (lane == K + 1 ? center[i] : 0u));
+        const bool mine = lane <= K + 1;
+        const bool ok = __all_sync(0xFFFFFFFFu, !mine || mykey < v.num_keys);
+        if (DET && mine) ukeys[i * per + lane] = ok ? mykey : NUPS_INVALID_KEY;
         if (!ok) {
             if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
+        const int myslot = (HOT && mine) ? __ldg(v.slot_of + mykey) : -1;
+        const unsigned long long myrow = (unsigned long long)mykey * L;
+        const unsigned long long mypend = myslot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)myslot) * L : NO_PEND;
+        if (mine) {
+            if (!DET && myslot >= 0) mark_dirty(v, myslot);
+            if (v.count) {
+                // context and centre: pulled (+ pushed in fast mode); negatives: pushed (their draw counted the sample)
+                const unsigned times = (lane == 0 || lane == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
+                if (times) note_access(v, mykey, myslot, times);
+            }
+            if (v.owner && (lane == 0 || lane == K + 1)) request_localize(v, mykey, q, req, req_cap);
+        }
+        // centre row
+        const unsigned long long crow = __shfl_sync(0xFFFFFFFFu, myrow, K + 1);
+        const unsigned long long cpend = __shfl_sync(0xFFFFFFFFu, mypend, K + 1);
         float4 vr[CH], gv[CH];
-        RowAt rc;
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            const uint32_t c = lane + 32 * m;
+            vr[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+            gv[m] = vr[m];
+            if (c < L4) {
+                vr[m] = val4[crow / 4 + c];
+                if (HOT && cpend != NO_PEND) vr[m] = add4(vr[m], slab4[cpend / 4 + c]);
+            }
+        }
         float loss = 0.f;
         for (uint32_t j0 = 0; j0 <= K; j0 += SGNS_UB) {
-            // element 0 of the group is the centre row (first group only), elements 1.. are output rows
-            uint32_t key[SGNS_UB + 1];
-            bool act[SGNS_UB + 1];
-            RowAt ra[SGNS_UB + 1];
-            key[0] = kc; act[0] = j0 == 0;
-#pragma unroll
-            for (int u = 0; u < SGNS_UB; ++u) {
-                const uint32_t j = j0 + u;
-                act[u + 1] = j <= K;
-                key[u + 1] = act[u + 1] ? (j == 0 ? ko : negs[i * K + j - 1]) : 0u;
-            }
-            resolve_rows<HOT, SGNS_UB + 1>(v, key, act, q, ra);
-            if (j0 == 0) {
-                rc = ra[0];
-#pragma unroll
-                for (int m = 0; m < CH; ++m) {
-                    const uint32_t c = lane + 32 * m;
-                    vr[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    gv[m] = vr[m];
-                    if (c < L4) {
-                        vr[m] = val4[rc.row / 4 + c];
-                        if (HOT && rc.pend != NO_PEND) vr[m] = add4(vr[m], slab4[rc.pend / 4 + c]);
-                    }
-                }
-            }
+            unsigned long long urow[SGNS_UB], upend[SGNS_UB];
             float4 ur[SGNS_UB][CH];
 #pragma unroll
             for (int u = 0; u < SGNS_UB; ++u) {
+                const uint32_t j = min(j0 + u, K);
+                urow[u] = __shfl_sync(0xFFFFFFFFu, myrow, j);
+                upend[u] = __shfl_sync(0xFFFFFFFFu, mypend, j);
 #pragma unroll
                 for (int m = 0; m < CH; ++m) {
                     const uint32_t c = lane + 32 * m;
                     ur[u][m] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (act[u + 1] && c < L4) {
-                        ur[u][m] = val4[ra[u + 1].row / 4 + c];
-                        if (HOT && ra[u + 1].pend != NO_PEND) ur[u][m] = add4(ur[u][m], slab4[ra[u + 1].pend / 4 + c]);
+                    if (j0 + u <= K && c < L4) {
+                        ur[u][m] = val4[urow[u] / 4 + c];
+                        if (HOT && upend[u] != NO_PEND) ur[u][m] = add4(ur[u][m], slab4[upend[u] / 4 + c]);
                     }
                 }
             }
@@ -200,15 +210,14 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
             }
 #pragma unroll
             for (int u = 0; u < SGNS_UB; ++u) {
-                if (!act[u + 1]) continue;
                 const uint32_t j = j0 + u;
+                if (j > K) continue;
                 const float x = clamp30(dot[u]);
                 const float g = sigmoidf_(x) - (j == 0 ? 1.f : 0.f);
                 loss += j == 0 ? softplusf_(-x) : softplusf_(x);
                 const float sc = -lr * g;
-                const bool hot = HOT && ra[u + 1].pend != NO_PEND;
-                float* out = DET ? upd + (i * per + j) * (uint64_t)L4 * 4
-                                 : (hot ? v.dval + ra[u + 1].pend : v.val + ra[u + 1].row);
+                const bool hot = HOT && upend[u] != NO_PEND;
+                float* out = DET ? upd + (i * per + j) * L : (hot ? v.dval + upend[u] : v.val + urow[u]);
 #pragma unroll
                 for (int m = 0; m < CH; ++m) {
                     const uint32_t c = lane + 32 * m;
@@ -220,17 +229,10 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
                         gv[m].z += g * ur[u][m].z; gv[m].w += g * ur[u][m].w;
                     }
                 }
-                if (lane == 0) {
-                    if (!DET && hot && v.dirty[ra[u + 1].slot] == 0u) v.dirty[ra[u + 1].slot] = 1u;
-                    if (v.count) {
-                        if (j == 0) note_access(v, key[u + 1], ra[u + 1].slot, DET ? 1u : 2u);   // pulled (+ pushed)
-                        else if (!DET) note_access(v, key[u + 1], ra[u + 1].slot, 1u);           // pushed; the sample was counted at the draw
-                    }
-                }
             }
         }
-        const bool chot = HOT && rc.pend != NO_PEND;
-        float* out = DET ? upd + (i * per + K + 1) * (uint64_t)L4 * 4 : (chot ? v.dval + rc.pend : v.val + rc.row);
+        const bool chot = HOT && cpend != NO_PEND;
+        float* out = DET ? upd + (i * per + K + 1) * L : (chot ? v.dval + cpend : v.val + crow);
 #pragma unroll
         for (int m = 0; m < CH; ++m) {
             const uint32_t c = lane + 32 * m;
@@ -240,19 +242,10 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
                 else red_add_v4(out + 4 * c, dv);
             }
         }
-        if (lane == 0) {
-            if (!DET && chot && v.dirty[rc.slot] == 0u) v.dirty[rc.slot] = 1u;
-            if (v.count) note_access(v, kc, rc.slot, DET ? 1u : 2u);
-            if (v.owner) { request_localize(v, ko, q, req, req_cap); request_localize(v, kc, q, req, req_cap); }
-            if (DET) loss_item[i] = loss;
-        }
+        if (DET && lane == 0) loss_item[i] = loss;
         my_loss += (double)loss;
     }
-    if (!DET) {
-        if (lane == 0) warp_loss[threadIdx.x >> 5] = my_loss;
-        __syncthreads();
-        loss_finish(v.st, warp_loss[0] + warp_loss[1] + warp_loss[2] + warp_loss[3], n, loss_out);
-    }
+    if (!DET) loss_finish(v, my_loss, n, loss_out);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -575,7 +568,9 @@ static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t
 
 static unsigned step_grid(const nups_store* s, uint64_t n)
 {
-    return grid_for(n, 4, (unsigned)s->sm_count * 16);     // 4 warps per block, one item per warp per pass
+    unsigned cap = (unsigned)s->sm_count * 16;
+    if (cap > NUPS_MAX_STEP_BLOCKS) cap = NUPS_MAX_STEP_BLOCKS;
+    return grid_for(n, 4, cap);     // 4 warps per block, one item per warp per pass
 }
 
 #define DISPATCH_CH(L4, ...)                                      \
@@ -601,6 +596,7 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
                                       int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream)
 {
     if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
+    if (K > 30) return NUPS_EINVAL;                         // one lane per key of an item
     if (s->L / 4 > 128) return NUPS_EINVAL;                 // rows of up to 512 floats are held in registers
     cudaStream_t st = (cudaStream_t)stream;
     nups_status rc = nups_draw_negatives(s, dist, n * K, st);

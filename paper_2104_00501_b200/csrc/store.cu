@@ -35,7 +35,7 @@ View nups_view(const nups_store* s)
     View v;
     v.val = s->val; v.acc = s->acc; v.dval = s->dval; v.dacc = s->dacc;
     v.hot_bits = s->hot_bits; v.slot_of = s->slot_of; v.dirty = s->dirty;
-    v.cnt = s->cnt; v.owner = s->owner; v.pending = s->pending; v.st = s->st;
+    v.cnt = s->cnt; v.owner = s->owner; v.pending = s->pending; v.st = s->st; v.loss_partial = s->loss_partial;
     v.num_keys = s->num_keys; v.Hcap = s->Hcap; v.H = (uint32_t)s->H; v.L4 = s->L / 4; v.R = s->R;
     v.count = s->cfg.count_accesses;
     return v;
@@ -150,6 +150,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     nups_store* s = (nups_store*)calloc(1, sizeof(nups_store));
     if (!s) return NUPS_ENOMEM;
     s->num_keys = num_keys; s->L = value_len; s->R = c.workers; s->cfg = c; s->device = dev;
+    s->ahead_dist = -1;
     cudaDeviceGetAttribute(&s->sm_count, cudaDevAttrMultiProcessorCount, dev);
     cudaDeviceGetAttribute(&s->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     size_t table_bytes = (size_t)num_keys * value_len * sizeof(float);
@@ -159,6 +160,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     ok = ok && cudaMalloc(&s->slot_of, num_keys * 4) == cudaSuccess;
     ok = ok && cudaMalloc(&s->cnt, num_keys * 8) == cudaSuccess;
     ok = ok && cudaMalloc(&s->st, sizeof(DevStat)) == cudaSuccess;
+    ok = ok && cudaMalloc(&s->loss_partial, 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double)) == cudaSuccess;
     if (ok && c.track_ownership) {
         ok = cudaMalloc(&s->owner, num_keys) == cudaSuccess;
         ok = ok && cudaMalloc(&s->pending, num_keys * 4) == cudaSuccess;
@@ -195,7 +197,7 @@ extern "C" nups_status nups_destroy(nups_store* s)
     for (int i = 0; i < NUPS_MAX_DISTS; ++i) { cudaFree(s->dist[i].table); cudaFree(s->dist[i].off); }
     cudaFree(s->val); cudaFree(s->acc); cudaFree(s->hot_bits); cudaFree(s->slot_of); cudaFree(s->hot_keys);
     cudaFree(s->dval); cudaFree(s->dacc); cudaFree(s->dirty); cudaFree(s->cnt); cudaFree(s->owner);
-    cudaFree(s->pending); cudaFree(s->st); cudaFree(s->scratch); cudaFree(s->req_keys); cudaFree(s->last_negs);
+    cudaFree(s->pending); cudaFree(s->st); cudaFree(s->loss_partial); cudaFree(s->scratch); cudaFree(s->req_keys); cudaFree(s->negs_buf);
     if (s->ev) {
         for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) cudaEventDestroy(s->ev[i]);
         free(s->ev);

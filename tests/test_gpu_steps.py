@@ -183,3 +183,30 @@ def test_tiny_sgns_config_full_epoch():
     tables_close(o, s)
     assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
     assert s.status_check() == 0
+
+
+@pytest.mark.parametrize("level", [CONFORM, BOUNDED])
+def test_sample_ahead_keeps_the_sample_sequences(level):
+    # in fast mode the negatives of several steps are drawn in one launch; whatever else touches the
+    # distribution in between (PrepareSample, a step of another size), the keys stay those of the oracle
+    V, L, K, R = 400, 16, 3, 4
+    c, ctx, w = sgns_data(V, 700, 5)
+    init = inputs.normal_init(2 * V, L, 0.1, 5)
+    o, s = make_pair(2 * V, L, R=R, init=init, deterministic=False, sync_interval=2)
+    do = o.register_distribution(V, w, V, level, U=3, G=20, seed=4)
+    ds = s.register_distribution(V, dev_keys(w), V, level, U=3, G=20, seed=4)
+    lb = loss_buf()
+    at = 0
+    plan = [64] * 20 + ["pull"] + [64] * 3 + [100] * 2 + [64] * 18 + ["pull", "pull"] + [33] * 20
+    for what in plan:
+        if what == "pull":
+            ko = o.pull_sample(o.prepare_sample(do, 77), 77, values=False)
+            ks = s.pull_sample(s.prepare_sample(ds, 77), 77, values=False)
+            assert np.array_equal(host_keys(ks), ko)
+            continue
+        n = what
+        _, negs = o.step_sgns(c[at:at + n], ctx[at:at + n], do, K, 0.01, return_negatives=True)
+        s.step_sgns(dev_keys(c[at:at + n]), dev_keys(ctx[at:at + n]), ds, K, 0.01, lb)
+        assert np.array_equal(host_keys(s.last_negatives()), negs)
+        at += n
+    assert s.status_check() == 0
