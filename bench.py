@@ -134,7 +134,8 @@ def build_store(binding, device, n_batches, seed, deterministic=False):
     s.init_uniform(0, 1, 0.5 / DIM)
     c, o, counts, weights = make_sgns_data(device, n_batches, seed, store=s)
     hot = s.select_hot(True, int(HOT_FRACTION * 2 * VOCAB))          # the most frequently accessed 1 % of keys
-    s.set_management(hot, binding.REPLICATE)
+    if hot.numel():
+        s.set_management(hot, binding.REPLICATE)
     dist = s.register_distribution(VOCAB, weights.contiguous(), VOCAB, binding.BOUNDED, U=U_REUSE, G=G_POOL, seed=7)
     return s, dist, hot.long(), c, o, weights
 
@@ -375,7 +376,7 @@ def run_ps_sweep(args, device):
 
 
 def main():
-    global TOKENS
+    global TOKENS, HOT_FRACTION, WORKERS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=4096)
@@ -383,6 +384,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--workload", default="sgns", choices=["sgns", "ps"])
+    ap.add_argument("--hot-fraction", type=float, default=HOT_FRACTION, help="share of keys to replicate (default 0.01)")
+    ap.add_argument("--workers", type=int, default=WORKERS)
     ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
     ap.add_argument("--ps-keys", type=int, default=100_000_000)
     ap.add_argument("--ps-skews", default="0,0.6,1.0,1.4")
@@ -390,6 +393,7 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     TOKENS = max(args.tokens, 10_000_000)
+    HOT_FRACTION, WORKERS = args.hot_fraction, args.workers
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))

@@ -37,7 +37,7 @@ struct View {
     float* dacc;               // same for the accumulator table
     const uint32_t* hot_bits;  // one bit per key: replicated?
     const int32_t* slot_of;    // key -> hot slot (>= 0) or negative
-    uint32_t* dirty;           // [Hcap] slot touched since last sync
+    uint32_t* dirty;           // [R][Hcap] worker's replica of the slot touched since last sync
     unsigned long long* cnt;   // [num_keys] access counts
     uint8_t* owner;            // [num_keys] owning worker or NUPS_OWNER_DEFAULT; NULL = not tracked
     int* pending;              // [num_keys] localize requests of the running call (-1 = none)
@@ -240,10 +240,11 @@ __device__ __forceinline__ bool key_is_local(const View& v, uint32_t q, uint32_t
 }
 
 // mark a replica slot as touched without waiting for anything to come back
-__device__ __forceinline__ void mark_dirty(const View& v, int slot)
+__device__ __forceinline__ void mark_dirty(const View& v, uint32_t q, int slot)
 {
-    asm volatile("red.global.or.b32 [%0], 1;" ::"l"(v.dirty + slot) : "memory");
+    asm volatile("red.global.or.b32 [%0], 1;" ::"l"(v.dirty + (size_t)q * v.Hcap + slot) : "memory");
 }
+__device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
 __device__ __forceinline__ void flag_bad_key(const View& v) { atomicCAS(&v.st->status, 0, NUPS_EKEY); }
 

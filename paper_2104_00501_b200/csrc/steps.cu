@@ -85,30 +85,23 @@ __device__ __forceinline__ void resolve_rows(const View& v, const uint32_t (&key
     }
 }
 
-// per-launch loss in fast mode: every warp stores its sum and takes a ticket from one integer counter;
-// the warp that draws the last ticket adds the sums up and writes the mean.  (Additions to one
-// floating-point address from thousands of warps would queue up at L2, and a block-wide barrier would
-// make every warp wait for the slowest one.)
+// per-launch loss in fast mode: one 64-bit integer addition per warp carries both the warp's loss (fixed
+// point, 2^-16 units, low 48 bits) and a ticket (high 16 bits); integer additions to one address do not
+// queue up the way floating-point ones do, need no fence and give a sum that does not depend on the
+// order.  The warp that draws the last ticket sees the total, writes the mean and clears the word.
+// Grids of the step kernels have fewer than 2^16 warps; the sum may reach 2^32.
 __device__ __forceinline__ void loss_finish(const View& v, double warp_loss, uint64_t n, float* loss_out)
 {
     const unsigned lane = threadIdx.x & 31;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
-    unsigned last = 0;
-    if (lane == 0) {
-        v.loss_partial[warp] = warp_loss;
-        __threadfence();
-        last = atomicAdd(&v.st->tmp[3], 1ull) + 1 == nwarps;
-    }
-    last = __shfl_sync(0xFFFFFFFFu, last, 0);
-    if (!last) return;
-    __threadfence();
-    double t = 0.0;
-    for (uint32_t b = lane; b < nwarps; b += 32) t += __ldcg(v.loss_partial + b);
-    for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
-    if (lane == 0) {
-        if (loss_out) *loss_out = (float)(t / (double)(n ? n : 1));
-        v.st->tmp[3] = 0ull;
+    if (lane != 0) return;
+    const unsigned long long nwarps = ((unsigned long long)gridDim.x * blockDim.x) >> 5;
+    const unsigned long long fixed = (unsigned long long)llrint(fmin(fmax(warp_loss, 0.0), 4.0e9) * 65536.0);
+    const unsigned long long mine = (fixed & 0xFFFFFFFFFFFFull) + (1ull << 48);
+    const unsigned long long old = atomicAdd(&v.st->tmp[3], mine);
+    const unsigned long long now = old + mine;
+    if ((now >> 48) == nwarps) {
+        if (loss_out) *loss_out = (float)((double)(now & 0xFFFFFFFFFFFFull) / 65536.0 / (double)(n ? n : 1));
+        atomicExch(&v.st->tmp[3], 0ull);
     }
 }
 
@@ -150,11 +143,16 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
             if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
-        const int myslot = (HOT && mine) ? __ldg(v.slot_of + mykey) : -1;
         const unsigned long long myrow = (unsigned long long)mykey * L;
+        const int myslot = (HOT && mine) ? __ldg(v.slot_of + mykey) : -1;
+        if (mine) {
+            // pull the lane's row towards L2 while the slots are looked up and the first rows are used
+            const char* rp = (const char*)(v.val + myrow);
+            for (uint32_t b = 0; b < L4 * 16; b += 128) prefetch_l2(rp + b);
+        }
         const unsigned long long mypend = myslot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)myslot) * L : NO_PEND;
         if (mine) {
-            if (!DET && myslot >= 0) mark_dirty(v, myslot);
+            if (!DET && myslot >= 0) mark_dirty(v, q, myslot);
             if (v.count) {
                 // context and centre: pulled (+ pushed in fast mode); negatives: pushed (their draw counted the sample)
                 const unsigned times = (lane == 0 || lane == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
@@ -345,7 +343,7 @@ __device__ __forceinline__ void adagrad_push(const View& v, uint32_t key, uint32
         }
     }
     if (lane == 0) {
-        if (!DET && rv.slot >= 0 && v.dirty[rv.slot] == 0u) v.dirty[rv.slot] = 1u;
+        if (!DET && rv.slot >= 0) mark_dirty(v, q, rv.slot);
         if (v.count) {
             unsigned times = (pulled_too ? 1u : 0u) + (DET ? 0u : 1u);
             if (times) note_access(v, key, rv.slot, times);
@@ -485,8 +483,8 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
         }
         if (lane == 0) {
             if (!DET) {
-                if (rw.slot >= 0 && v.dirty[rw.slot] == 0u) v.dirty[rw.slot] = 1u;
-                if (rh.slot >= 0 && v.dirty[rh.slot] == 0u) v.dirty[rh.slot] = 1u;
+                if (rw.slot >= 0) mark_dirty(v, q, rw.slot);
+                if (rh.slot >= 0) mark_dirty(v, q, rh.slot);
             }
             if (v.count) {
                 note_access(v, ki, rw.slot, DET ? 1u : 2u);

@@ -468,7 +468,7 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
         // destination: row offset in floats, lowest bit set when it lies in the replica slab
         unsigned long long dest = NO_ROW - lane;          // invalid rows: a value no other lane has
         bool hot = false;
-        uint32_t hslot = 0;
+        size_t hrow = 0;
         int tier = -1;                                    // shared-memory accumulator of this row, if any
         if (valid) {
             dest = ((unsigned long long)key * L4) << 3;
@@ -478,7 +478,7 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
                 const uint32_t q = rows_per_item == 1 ? worker_of_item(i, n_items, R)
                                                       : worker_of_item(i / rows_per_item, n_items, R);
                 dest = ((((unsigned long long)q * v.Hcap + slot) * L4) << 3) | 1ull;
-                hslot = slot;
+                hrow = (size_t)q * v.Hcap + slot;
                 if (TIER && slot < tier_rows && q == my_q) tier = (int)slot;
             }
         }
@@ -495,7 +495,10 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
         const bool leader = valid && (lane == (unsigned)(__ffs(grp) - 1));
         // mark the slot as touched: one lane per destination, and only if nobody has yet (a hot slot would
         // otherwise take hundreds of thousands of stores to one address)
-        if (HOT && leader && hot && v.dirty[hslot] == 0u) v.dirty[hslot] = 1u;
+        if (HOT && leader && hot) {
+            uint32_t* flag = v.dirty + hrow;          // replica row index = q * Hcap + slot
+            if (*flag == 0u) *flag = 1u;
+        }
         unsigned singles = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) == 1);
         unsigned multis = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) > 1);
 
@@ -630,7 +633,7 @@ __global__ void push_dest_kernel(View v, const uint32_t* __restrict__ keys, uint
             uint32_t slot = (uint32_t)v.slot_of[key];
             uint32_t q = worker_of_item(i / rows_per_item, n_items, v.R);
             d = (1ull << 32) + (unsigned long long)q * v.H + slot;
-            if (v.dirty[slot] == 0u) v.dirty[slot] = 1u;
+            if (v.dirty[(size_t)q * v.Hcap + slot] == 0u) v.dirty[(size_t)q * v.Hcap + slot] = 1u;
         }
     }
     if (in) { dest[i] = d; idx[i] = (uint32_t)i; }
@@ -811,7 +814,10 @@ __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
     uint64_t total = (uint64_t)v.H * L4;
     if (t >= total) return;
     uint32_t slot = (uint32_t)(t / L4), c = (uint32_t)(t % L4);
-    if (!v.dirty[slot]) return;
+    // only replicas that were written since the last sync are read, added (worker 0 first) and cleared
+    bool any = false;
+    for (uint32_t r = 0; r < v.R; ++r) any = any || v.dirty[(size_t)r * v.Hcap + slot] != 0u;
+    if (!any) return;
     uint32_t key = hot_keys[slot];
     const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int which = 0; which < 2; ++which) {
@@ -819,10 +825,21 @@ __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
         float4* slab = (float4*)(which ? v.dacc : v.dval);
         if (!table || !slab) continue;
         float4 sum = zero;
-        for (uint32_t r = 0; r < v.R; ++r) {
-            float4* p = slab + ((uint64_t)r * v.Hcap + slot) * L4 + c;
-            sum = add4(sum, *p);
-            *p = zero;
+        for (uint32_t r0 = 0; r0 < v.R; r0 += 4) {
+            float4 x[4];
+            bool d[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                d[u] = r0 + u < v.R && v.dirty[(size_t)(r0 + u) * v.Hcap + slot] != 0u;
+                if (d[u]) x[u] = slab[((uint64_t)(r0 + u) * v.Hcap + slot) * L4 + c];
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (d[u]) {
+                    sum = add4(sum, x[u]);
+                    slab[((uint64_t)(r0 + u) * v.Hcap + slot) * L4 + c] = zero;
+                }
+            }
         }
         float4* row = table + (uint64_t)key * L4 + c;
         *row = add4(*row, sum);
@@ -835,7 +852,7 @@ nups_status nups_sync_internal(nups_store* s, cudaStream_t st)
     View v = nups_view(s);
     sync_kernel<<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
     LAUNCH_CHECK(s);
-    CK(cudaMemsetAsync(s->dirty, 0, s->H * sizeof(uint32_t), st));
+    CK(cudaMemsetAsync(s->dirty, 0, (size_t)s->R * s->Hcap * sizeof(uint32_t), st));
     s->syncs++;
     return NUPS_OK;
 }
@@ -1059,7 +1076,7 @@ static nups_status grow_hot(nups_store* s, uint64_t need)
     uint32_t* dirty = nullptr;
     float *dv = nullptr, *da = nullptr;
     size_t slab = (size_t)s->R * cap * s->L * sizeof(float);
-    bool ok = cudaMalloc(&hk, cap * 4) == cudaSuccess && cudaMalloc(&dirty, cap * 4) == cudaSuccess &&
+    bool ok = cudaMalloc(&hk, cap * 4) == cudaSuccess && cudaMalloc(&dirty, (size_t)s->R * cap * 4) == cudaSuccess &&
               cudaMalloc(&dv, slab) == cudaSuccess && (!s->acc || cudaMalloc(&da, slab) == cudaSuccess);
     if (!ok) {
         cudaGetLastError();
@@ -1068,7 +1085,7 @@ static nups_status grow_hot(nups_store* s, uint64_t need)
     }
     // pending updates are all zero here (the caller merged them), so fresh zeroed slabs are enough
     if (s->H) CK(cudaMemcpy(hk, s->hot_keys, s->H * 4, cudaMemcpyDeviceToDevice));
-    CK(cudaMemset(dirty, 0, cap * 4));
+    CK(cudaMemset(dirty, 0, (size_t)s->R * cap * 4));
     CK(cudaMemset(dv, 0, slab));
     if (da) CK(cudaMemset(da, 0, slab));
     CK(cudaDeviceSynchronize());
