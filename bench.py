@@ -140,6 +140,20 @@ def build_store(binding, device, n_batches, seed, deterministic=False):
     return s, dist, hot.long(), c, o, weights
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank's time counts)."""
+    if world <= 1:
+        return [float(x) for x in values]
+    t = torch.tensor(values, dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_throughput(units_per_rank, seconds, world):
+    """Whole-job throughput of `world` independent replicas: all units over the slowest rank's time."""
+    return units_per_rank * world / seconds
+
+
 def run_ours(args, rank, world, device):
     from paper_2104_00501_b200 import binding
     hbm_peak, peak_kind = peaks()
@@ -211,12 +225,9 @@ def run_ours(args, rank, world, device):
     sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2104_00501_b200", "csrc", "steps.cu"), "rb").read()).hexdigest()
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["steps_cu_sha1"] == sha else None
 
-    if world > 1:
-        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=device)
-        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
-        ms, e2e_s = float(t[0]), float(t[1])
+    ms, e2e_s = max_over_ranks([ms, e2e_s], world, device)
     pairs = args.steps * BATCH * world
-    value = pairs * ACCESSES_PER_PAIR / (ms / 1e3)
+    value = aggregate_throughput(args.steps * BATCH * ACCESSES_PER_PAIR, ms / 1e3, world)
     out = {
         "metric": "key accesses/s (pull+push+sample)", "value": value, "unit": "key accesses/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,

@@ -1,0 +1,69 @@
+"""Parity at the benchmark's full size and launch configuration (2M keys x 300 floats, batches of 4096
+pairs, 3 pooled-reuse negatives, top 1 % of keys replicated, 8 workers, merge every 16 batches)."""
+import numpy as np
+import pytest
+import torch
+
+import bench
+from oracle import Oracle, BOUNDED, REPLICATE
+from paper_2104_00501_b200 import binding, inputs
+from tests.common import host_keys
+
+pytestmark = pytest.mark.gpu
+
+V, L, B, K = bench.VOCAB, bench.DIM, bench.BATCH, bench.NEG
+
+
+def _setup(deterministic, n_batches, tokens=10_000_000):
+    bench.TOKENS = tokens
+    s, dist, hot, c, o, weights = bench.build_store(binding, torch.device("cuda"), n_batches, seed=0,
+                                                    deterministic=deterministic)
+    orc = Oracle(2 * V, L, workers=bench.WORKERS, sync_interval=bench.SYNC_EVERY)
+    orc.init_uniform(0, 1, 0.5 / L)
+    orc.set_management(inputs.u32(hot), REPLICATE)
+    d = orc.register_distribution(V, inputs.u32(weights), V, BOUNDED, U=bench.U_REUSE, G=bench.G_POOL, seed=7)
+    return s, dist, orc, d, c, o
+
+
+def test_full_size_deterministic_steps_match_the_oracle():
+    s, dist, orc, d, c, o = _setup(True, 3)
+    hc, ho = inputs.u32(c), inputs.u32(o)
+    lb = torch.zeros(1, device="cuda")
+    touched = []
+    for b in range(3):
+        sl = slice(b * B, (b + 1) * B)
+        lo, negs = orc.step_sgns(hc[sl], ho[sl], d, K, bench.LR, return_negatives=True)
+        s.step_sgns(c[sl], o[sl], dist, K, bench.LR, lb)
+        assert np.array_equal(host_keys(s.last_negatives()), negs)          # bit-exact keys
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+        touched.append(np.concatenate([hc[sl], ho[sl], negs]))
+    orc.sync()
+    s.sync()
+    # every touched row plus a random sample of untouched ones, element by element
+    rng = np.random.default_rng(0)
+    rows = np.unique(np.concatenate(touched + [rng.integers(0, 2 * V, 5000).astype(np.uint32)]))
+    got = s.read_table()[torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy()
+    np.testing.assert_allclose(got, orc.table()[rows], rtol=1e-5, atol=1e-6)
+    assert np.abs(got - np.asarray(orc.table()[rows])).max() < 1e-6
+    assert s.status_check() == 0
+
+
+def test_full_size_fast_mode_tracks_the_oracle_loss():
+    # replicated + asynchronous mode as the benchmark runs it: the loss after the same number of
+    # batches stays within 1 % of the oracle's, and the sampled keys are still the oracle's
+    steps = 48
+    s, dist, orc, d, c, o = _setup(False, steps)
+    hc, ho = inputs.u32(c), inputs.u32(o)
+    lb = torch.zeros(steps, device="cuda")
+    lo = []
+    for b in range(steps):
+        sl = slice(b * B, (b + 1) * B)
+        l, negs = orc.step_sgns(hc[sl], ho[sl], d, K, bench.LR, return_negatives=True)
+        lo.append(l)
+        s.step_sgns(c[sl], o[sl], dist, K, bench.LR, lb[b:b + 1])
+        if b % 7 == 0:
+            assert np.array_equal(host_keys(s.last_negatives()), negs)
+    ls = lb.cpu().numpy()
+    assert abs(ls[-16:].mean() - np.mean(lo[-16:])) <= 0.01 * np.mean(lo[-16:])
+    assert np.all(np.isfinite(ls))
+    assert s.status_check() == 0
