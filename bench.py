@@ -33,7 +33,7 @@ sys.path.insert(0, ROOT)
 from paper_2104_00501_b200 import inputs  # noqa: E402
 
 VOCAB, DIM, BATCH, NEG, WINDOW = 1_000_000, 300, 4096, 3, 5
-U_REUSE, G_POOL, SYNC_EVERY, WORKERS, LR = 16, 250, 16, 8, 0.005
+U_REUSE, G_POOL, SYNC_EVERY, WORKERS, LR = 16, 250, 16, 8, 0.001
 HOT_FRACTION = 0.01
 TOKENS = 100_000_000
 ACCESSES_PER_PAIR = 2 + NEG + (NEG + 2)          # direct pulls + sampled pulls + pushes
@@ -42,7 +42,7 @@ MAX_DISTINCT_BATCHES = 4096
 
 # DRAM traffic of one launch of the fused step kernel, from an ncu capture (dram__bytes_read.sum +
 # dram__bytes_write.sum); valid only for the kernel source it was captured on.
-NCU_TRAFFIC = {"bytes_per_launch": None, "steps_cu_sha1": None}
+NCU_TRAFFIC = {"bytes_per_launch": 5092352, "steps_cu_sha1": "64fd33d13e74d963f4f34ede2b6a202b86de2eb3"}
 
 
 def peaks():
@@ -390,7 +390,7 @@ def main():
     global TOKENS, HOT_FRACTION, WORKERS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=4096)
+    ap.add_argument("--steps", type=int, default=16384)
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
