@@ -386,6 +386,112 @@ def run_ps_sweep(args, device):
     return lines
 
 
+def _time_calls(fn, reps, warm=3):
+    """Mean device time of fn() in seconds: CUDA events on the current stream around `reps` calls."""
+    for _ in range(warm):
+        fn()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / 1e3 / reps
+
+
+def run_sample_sweep(args, device):
+    """PullSample of 1M keys (keys + values) from a Zipf(1.0) target over the whole store, four levels."""
+    from paper_2104_00501_b200 import binding
+    hbm_peak, peak_kind = peaks()
+    NK, L, N = args.ps_keys, 128, 1 << 20
+    s = binding.Store(NK, L, workers=WORKERS, deterministic=False, track_ownership=True)
+    s.init_uniform(0, 3, 0.1)
+    key_of_rank = inputs.zipf_key_of_rank(NK, device)
+    s.set_management(key_of_rank[:1000].to(torch.int32).contiguous(), binding.REPLICATE)
+    w = inputs.zipf_integer_weights(NK, 1.0, device).to(torch.int32).contiguous()
+    t0 = time.perf_counter()
+    dists = {name: s.register_distribution(0, w, NK, lvl, U=U_REUSE, G=G_POOL, seed=11 + lvl)
+             for name, lvl in (("CONFORM", binding.CONFORM), ("BOUNDED", binding.BOUNDED),
+                               ("LONG-TERM", binding.LONGTERM), ("NON-CONFORM", binding.NONCONFORM))}
+    torch.cuda.synchronize()
+    build_s = (time.perf_counter() - t0) / 4
+    keys = torch.empty(N, dtype=torch.int32, device=device)
+    vals = torch.empty(N, L, device=device)
+    for name, d in dists.items():
+        def once():
+            h = s.prepare_sample(d, N)
+            s.pull_sample(h, N, True, keys, vals)
+        t = _time_calls(once, max(args.steps, 5))
+        uniq = int(torch.unique(keys).numel())
+        alg = 4 * N + L * 4 * N + L * 4 * uniq + 16 * N
+        print(json.dumps({"workload": "PullSample", "level": name, "keys": NK, "value_len": L, "samples": N,
+                          "us": t * 1e6, "keys_per_s": N / t, "distinct_keys": uniq, "algorithmic_gbs": alg / t / 1e9,
+                          "frac": alg / t / 1e9 / hbm_peak, "peak_kind": peak_kind,
+                          "alias_build_s": build_s}), flush=True)
+    s.close()
+
+
+def run_step_workload(args, device, which):
+    """ComplEx + AdaGrad (config 3) or matrix factorization (config 4) steps in fast mode."""
+    from paper_2104_00501_b200 import binding
+    hbm_peak, peak_kind = peaks()
+    loss = torch.zeros(1, device=device)
+    reps = max(args.steps, 20)
+    if which == "kge":
+        E, Rl, L, B, K = 5_000_000, 1000, 500, 8192, 10
+        s = binding.Store(E + Rl, L, workers=WORKERS, sync_interval=SYNC_EVERY, deterministic=False, with_adagrad=True)
+        s.init_uniform(0, 5, 0.05)
+        nb = 64
+        h, r, t = inputs.kge_triples(nb * B, E, Rl, 0.9, 1.2, 0, device)
+        h, r, t = (x.to(torch.int32).contiguous() for x in (h, r, t))
+        s.count_accesses(torch.cat([h, t]))
+        hot = s.select_hot(False, 100)                               # the 100 x mean rule on the entities ...
+        rel = torch.arange(E, E + Rl, device=device, dtype=torch.int32)
+        s.set_management(torch.cat([rel, hot]).contiguous(), binding.REPLICATE)   # ... and every relation
+        dist = s.register_distribution(0, None, E, binding.CONFORM, seed=3)
+        state = {"i": 0}
+
+        def step():
+            j = (state["i"] % nb) * B
+            state["i"] += 1
+            s.step_complex(h[j:j + B], r[j:j + B], t[j:j + B], dist, K, 0.1, 1e-10, loss)
+        per_item, upd, rows_per_item = 3 + K + (K + 3), K + 3, 2 * (K + 3)
+        name, cfg = "complex_kernel", f"ComplEx+AdaGrad: 5M entities, 1000 relations, 500 fp32/row + accumulator, batch {B}, {K} negatives"
+    else:
+        M, N, L, B = 10_000_000, 1_000_000, 100, 65536
+        s = binding.Store(M + N, L, workers=WORKERS, sync_interval=SYNC_EVERY, deterministic=False)
+        s.init_uniform(0, 5, 0.3)
+        nb = 32
+        i, j, x = inputs.mf_cells(nb * B, M, N, 0.8, 100, 0.1, 0, device)
+        i, j, x = i.to(torch.int32).contiguous(), j.to(torch.int32).contiguous(), x.contiguous()
+        s.count_accesses(torch.cat([i, j]))
+        hot = s.select_hot(False, 100)
+        if hot.numel():
+            s.set_management(hot, binding.REPLICATE)
+        state = {"i": 0}
+
+        def step():
+            a = (state["i"] % nb) * B
+            state["i"] += 1
+            s.step_mf(i[a:a + B], j[a:a + B], x[a:a + B], 1e-4, 0.01, loss)
+        per_item, upd, rows_per_item = 4, 2, 2
+        name, cfg = "mf_kernel", f"MF: 10M x 1M, rank 100, batch {B}, L2 0.01"
+    t = _time_calls(step, reps)
+    s.kernel_timing(True)
+    _time_calls(step, reps, warm=0)
+    k_ms, k_n = s.kernel_time()
+    s.kernel_timing(False)
+    k_s = k_ms / 1e3 / max(k_n, 1)
+    tables = 2 if which == "kge" else 1
+    logical = B * rows_per_item * L * 4 * 2 * (1 if which == "mf" else 1)      # every touched row read and written once
+    print(json.dumps({"workload": cfg, "kernel": name, "hot_slots": s.stats()["hot_slots"], "us_per_step": t * 1e6,
+                      "kernel_us": k_s * 1e6, "key_accesses_per_s": B * per_item / t, "updates_per_s": B * upd / t,
+                      "logical_gbs": logical / k_s / 1e9, "logical_frac_of_hbm_peak": logical / k_s / 1e9 / hbm_peak,
+                      "peak_kind": peak_kind, "final_loss": float(loss.item()), "tables": tables}), flush=True)
+    s.close()
+
+
 def main():
     global TOKENS, HOT_FRACTION, WORKERS
     ap = argparse.ArgumentParser()
@@ -394,7 +500,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="sgns", choices=["sgns", "ps"])
+    ap.add_argument("--workload", default="sgns", choices=["sgns", "ps", "sample", "kge", "mf"])
     ap.add_argument("--hot-fraction", type=float, default=HOT_FRACTION, help="share of keys to replicate (default 0.01)")
     ap.add_argument("--workers", type=int, default=WORKERS)
     ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
@@ -418,6 +524,12 @@ def main():
     device = torch.device("cuda", local)
     if args.workload == "ps":
         run_ps_sweep(args, device)
+        return
+    if args.workload == "sample":
+        run_sample_sweep(args, device)
+        return
+    if args.workload in ("kge", "mf"):
+        run_step_workload(args, device, args.workload)
         return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)

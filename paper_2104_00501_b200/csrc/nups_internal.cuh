@@ -204,6 +204,7 @@ __device__ __forceinline__ void philox_at(uint64_t seed, uint64_t index, uint32_
 __device__ __forceinline__ uint32_t worker_of_item(uint64_t i, uint64_t n, uint32_t R)
 {
     if (R == 1) return 0;
+    if (((n * R) >> 32) == 0) return ((uint32_t)i * R) / (uint32_t)n;   // the usual case: a 32-bit division
     return (uint32_t)((i * R) / n);          // calls take fewer than 2^32 items: i * R < 2^40
 }
 

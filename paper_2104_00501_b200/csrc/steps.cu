@@ -21,6 +21,8 @@ struct RowRef {
     int slot;
 };
 
+// (the step workloads keep key -> slot small enough to stay in L2, so the slot map is read directly
+// instead of going through the technique bitmap first)
 template <bool HOT>
 __device__ __forceinline__ RowRef resolve(const View& v, uint32_t key, uint32_t q, int which)
 {
@@ -30,15 +32,28 @@ __device__ __forceinline__ RowRef resolve(const View& v, uint32_t key, uint32_t 
     r.base = table + (uint64_t)key * L;
     r.pend = nullptr;
     r.dst = table + (uint64_t)key * L;
-    r.slot = -1;
-    if (HOT && key_is_hot(v, key)) {
-        r.slot = __ldg(v.slot_of + key);
+    r.slot = HOT ? __ldg(v.slot_of + key) : -1;
+    if (r.slot >= 0) {
         float* slab = which ? v.dacc : v.dval;
         float* p = slab + ((uint64_t)q * v.Hcap + (uint64_t)r.slot) * L;
         r.pend = p;
         r.dst = p;
-    }
+    } else r.slot = -1;
     return r;
+}
+
+// Warp-cooperative L2 prefetch of the row of `key` in the value table (and the accumulator table):
+// issued for the warp's NEXT item while the current one is being worked on.
+__device__ __forceinline__ void prefetch_row(const View& v, uint32_t key, bool with_acc, unsigned lane)
+{
+    const uint32_t row_bytes = v.L4 * 16;
+    const uint32_t lines = (row_bytes + 127) / 128;
+    const char* a = (const char*)(v.val + (uint64_t)key * v.L4 * 4);
+    const char* b = (const char*)(v.acc + (uint64_t)key * v.L4 * 4);
+    for (uint32_t idx = lane; idx < lines * (with_acc ? 2u : 1u); idx += 32) {
+        const uint32_t line = idx < lines ? idx : idx - lines;
+        prefetch_l2((idx < lines ? a : b) + (size_t)line * 128);
+    }
 }
 
 __device__ __forceinline__ void red_add_v2(float* addr, float2 x)
@@ -355,15 +370,25 @@ template <bool HOT, bool DET, int CH>
 __global__ void __launch_bounds__(128)
 complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restrict__ rk, const uint32_t* __restrict__ tk,
                const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float eps, float* __restrict__ uval,
-               float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, uint32_t* req,
-               uint64_t req_cap)
+               float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
+               float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
 {
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t d2 = v.L4, per = K + 3;            // d/2 pairs = L/4
     const uint64_t L = (uint64_t)v.L4 * 4;
+    double my_loss = 0.0;
     for (uint64_t i = warp; i < n; i += nwarps) {
+        // start moving the rows of the warp's next item towards L2 (values and accumulators of its 3 + K keys)
+        if (i + nwarps < n) {
+            const uint64_t nx = i + nwarps;
+            uint32_t nk = lane == 0 ? hk[nx] : lane == 1 ? rk[nx] : lane == 2 ? tk[nx] : (lane < 3 + K ? negs[nx * K + lane - 3] : 0u);
+            for (uint32_t r = 0; r < 3 + K && r < 32; ++r) {
+                const uint32_t key = __shfl_sync(0xFFFFFFFFu, nk, r);
+                if (key < v.num_keys) prefetch_row(v, key, true, lane);
+            }
+        }
         const uint32_t q = worker_of_item(i, n, v.R);
         const uint32_t kh = hk[i], kr = rk[i], kt = tk[i];
         bool ok = kh < v.num_keys && kr < v.num_keys && kt < v.num_keys;
@@ -375,7 +400,7 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             for (uint32_t j = 0; j < K; ++j) ukeys[i * per + 3 + j] = ok ? negs[i * K + j] : NUPS_INVALID_KEY;
         }
         if (!ok) {
-            if (lane == 0) { flag_bad_key(v); loss_item[i] = 0.f; }
+            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
         C2 h[CH], r[CH], t[CH], gh[CH], gr[CH], gt[CH];
@@ -420,80 +445,140 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
                 request_localize(v, kr, q, req, req_cap);
                 request_localize(v, kt, q, req, req_cap);
             }
-            loss_item[i] = loss;
+            if (DET) loss_item[i] = loss;
         }
+        my_loss += (double)loss;
     }
+    if (!DET) loss_finish(v, my_loss, n, loss_out);
 }
 
 // ---------------------------------------------------------------------------------------------
 // matrix factorization
 // ---------------------------------------------------------------------------------------------
+// A warp keeps MF_DEPTH items in flight: the stored rows of the next MF_DEPTH items are already on their
+// way (and the keys of the MF_DEPTH after those) while it does the dot product and the updates of the
+// current one.  The workload is bound by DRAM: what counts is how many row fetches are outstanding.
+#ifndef NUPS_MF_DEPTH
+#define NUPS_MF_DEPTH 2
+#endif
+constexpr int MF_DEPTH = NUPS_MF_DEPTH;
+
 template <bool HOT, bool DET, int CH>
 __global__ void __launch_bounds__(128)
 mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
           uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
-          float* __restrict__ loss_item, uint32_t* req, uint64_t req_cap)
+          float* __restrict__ loss_item, float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
 {
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
     const uint32_t L4 = v.L4;
-    for (uint64_t i = warp; i < n; i += nwarps) {
-        const uint32_t q = worker_of_item(i, n, v.R);
-        const uint32_t ki = rowk[i], kj = colk[i];
-        bool ok = ki < v.num_keys && kj < v.num_keys;
-        if (DET && lane == 0) {
-            ukeys[2 * i] = ok ? ki : NUPS_INVALID_KEY;
-            ukeys[2 * i + 1] = ok ? kj : NUPS_INVALID_KEY;
-        }
-        if (!ok) {
-            if (lane == 0) { flag_bad_key(v); loss_item[i] = 0.f; }
-            continue;
-        }
-        RowRef rw = resolve<HOT>(v, ki, q, 0), rh = resolve<HOT>(v, kj, q, 0);
-        float4 w[CH], h[CH];
-        float dot = 0.f;
+    const float4* val4 = (const float4*)v.val;
+    const float4* slab4 = (const float4*)v.dval;
+    double my_loss = 0.0;
+
+    // ring A: keys and cell values of the items 2*MF_DEPTH .. MF_DEPTH+1 steps ahead
+    // ring B: keys, slots and stored rows of the items MF_DEPTH .. 1 steps ahead
+    uint32_t kiA[MF_DEPTH], kjA[MF_DEPTH], kiB[MF_DEPTH], kjB[MF_DEPTH];
+    float xA[MF_DEPTH], xB[MF_DEPTH];
+    int siB[MF_DEPTH], sjB[MF_DEPTH];
+    float4 wB[MF_DEPTH][CH], hB[MF_DEPTH][CH];
+    auto load_keys = [&](int u, uint64_t i) {
+        if (i < n) { kiA[u] = rowk[i]; kjA[u] = colk[i]; xA[u] = x[i]; }
+        else { kiA[u] = NUPS_INVALID_KEY; kjA[u] = NUPS_INVALID_KEY; xA[u] = 0.f; }
+    };
+    auto fetch_rows = [&](int u) {
+        kiB[u] = kiA[u]; kjB[u] = kjA[u]; xB[u] = xA[u];
+        const bool ok = kiB[u] < v.num_keys && kjB[u] < v.num_keys;
+        siB[u] = (HOT && ok) ? __ldg(v.slot_of + kiB[u]) : -1;
+        sjB[u] = (HOT && ok) ? __ldg(v.slot_of + kjB[u]) : -1;
 #pragma unroll
         for (int m = 0; m < CH; ++m) {
-            uint32_t c = lane + 32 * m;
-            w[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-            h[m] = w[m];
-            if (c < L4) {
-                w[m] = ((const float4*)rw.base)[c];
-                h[m] = ((const float4*)rh.base)[c];
-                if (rw.pend) w[m] = add4(w[m], ((const float4*)rw.pend)[c]);
-                if (rh.pend) h[m] = add4(h[m], ((const float4*)rh.pend)[c]);
+            const uint32_t c = lane + 32 * m;
+            wB[u][m] = make_float4(0.f, 0.f, 0.f, 0.f);
+            hB[u][m] = wB[u][m];
+            if (ok && c < L4) {
+                wB[u][m] = val4[(uint64_t)kiB[u] * L4 + c];
+                hB[u][m] = val4[(uint64_t)kjB[u] * L4 + c];
             }
-            dot += w[m].x * h[m].x + w[m].y * h[m].y + w[m].z * h[m].z + w[m].w * h[m].w;
         }
-        float err = x[i] - warp_sum(dot);
-        float* ow = DET ? upd + (2 * i) * (uint64_t)L4 * 4 : rw.dst;
-        float* oh = DET ? upd + (2 * i + 1) * (uint64_t)L4 * 4 : rh.dst;
+    };
 #pragma unroll
-        for (int m = 0; m < CH; ++m) {
-            uint32_t c = lane + 32 * m;
-            if (c < L4) {
-                float4 dw = make_float4(lr * (err * h[m].x - l2 * w[m].x), lr * (err * h[m].y - l2 * w[m].y),
-                                        lr * (err * h[m].z - l2 * w[m].z), lr * (err * h[m].w - l2 * w[m].w));
-                float4 dh = make_float4(lr * (err * w[m].x - l2 * h[m].x), lr * (err * w[m].y - l2 * h[m].y),
-                                        lr * (err * w[m].z - l2 * h[m].z), lr * (err * w[m].w - l2 * h[m].w));
-                if (DET) { ((float4*)ow)[c] = dw; ((float4*)oh)[c] = dh; }
-                else { red_add_v4(ow + 4 * c, dw); red_add_v4(oh + 4 * c, dh); }
+    for (int u = 0; u < MF_DEPTH; ++u) load_keys(u, warp + (uint64_t)u * nwarps);
+#pragma unroll
+    for (int u = 0; u < MF_DEPTH; ++u) fetch_rows(u);
+#pragma unroll
+    for (int u = 0; u < MF_DEPTH; ++u) load_keys(u, warp + (uint64_t)(MF_DEPTH + u) * nwarps);
+
+    for (uint64_t i0 = warp; i0 < n; i0 += (uint64_t)MF_DEPTH * nwarps) {
+#pragma unroll
+        for (int u = 0; u < MF_DEPTH; ++u) {
+            const uint64_t i = i0 + (uint64_t)u * nwarps;
+            if (i >= n) break;
+            // take over what ring B fetched for this item, then refill both rings before computing
+            const uint32_t ki = kiB[u], kj = kjB[u];
+            const float xv = xB[u];
+            const int si = siB[u], sj = sjB[u];
+            float4 w[CH], h[CH];
+#pragma unroll
+            for (int m = 0; m < CH; ++m) { w[m] = wB[u][m]; h[m] = hB[u][m]; }
+            fetch_rows(u);
+            load_keys(u, i + 2ull * MF_DEPTH * nwarps);
+
+            const uint32_t q = worker_of_item(i, n, v.R);
+            const bool ok = ki < v.num_keys && kj < v.num_keys;
+            if (DET && lane == 0) {
+                ukeys[2 * i] = ok ? ki : NUPS_INVALID_KEY;
+                ukeys[2 * i + 1] = ok ? kj : NUPS_INVALID_KEY;
             }
-        }
-        if (lane == 0) {
-            if (!DET) {
-                if (rw.slot >= 0) mark_dirty(v, q, rw.slot);
-                if (rh.slot >= 0) mark_dirty(v, q, rh.slot);
+            if (!ok) {
+                if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+                continue;
             }
-            if (v.count) {
-                note_access(v, ki, rw.slot, DET ? 1u : 2u);
-                note_access(v, kj, rh.slot, DET ? 1u : 2u);
+            const uint64_t pw = si >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)si) * L4 : 0;
+            const uint64_t ph = sj >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)sj) * L4 : 0;
+            float dot = 0.f;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                const uint32_t c = lane + 32 * m;
+                if (c < L4) {
+                    if (HOT && si >= 0) w[m] = add4(w[m], slab4[pw + c]);       // the worker's pending replica updates
+                    if (HOT && sj >= 0) h[m] = add4(h[m], slab4[ph + c]);
+                }
+                dot += w[m].x * h[m].x + w[m].y * h[m].y + w[m].z * h[m].z + w[m].w * h[m].w;
             }
-            if (v.owner) { request_localize(v, ki, q, req, req_cap); request_localize(v, kj, q, req, req_cap); }
-            loss_item[i] = err * err;
+            const float err = xv - warp_sum(dot);
+            float* ow = DET ? upd + (2 * i) * (uint64_t)L4 * 4 : (si >= 0 ? v.dval + pw * 4 : v.val + (uint64_t)ki * L4 * 4);
+            float* oh = DET ? upd + (2 * i + 1) * (uint64_t)L4 * 4
+                            : (sj >= 0 ? v.dval + ph * 4 : v.val + (uint64_t)kj * L4 * 4);
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                const uint32_t c = lane + 32 * m;
+                if (c < L4) {
+                    const float4 dw = make_float4(lr * (err * h[m].x - l2 * w[m].x), lr * (err * h[m].y - l2 * w[m].y),
+                                                  lr * (err * h[m].z - l2 * w[m].z), lr * (err * h[m].w - l2 * w[m].w));
+                    const float4 dh = make_float4(lr * (err * w[m].x - l2 * h[m].x), lr * (err * w[m].y - l2 * h[m].y),
+                                                  lr * (err * w[m].z - l2 * h[m].z), lr * (err * w[m].w - l2 * h[m].w));
+                    if (DET) { ((float4*)ow)[c] = dw; ((float4*)oh)[c] = dh; }
+                    else { red_add_v4(ow + 4 * c, dw); red_add_v4(oh + 4 * c, dh); }
+                }
+            }
+            if (lane == 0) {
+                if (!DET) {
+                    if (si >= 0) mark_dirty(v, q, si);
+                    if (sj >= 0) mark_dirty(v, q, sj);
+                }
+                if (v.count) {
+                    note_access(v, ki, si, DET ? 1u : 2u);
+                    note_access(v, kj, sj, DET ? 1u : 2u);
+                }
+                if (v.owner) { request_localize(v, ki, q, req, req_cap); request_localize(v, kj, q, req, req_cap); }
+                if (DET) loss_item[i] = err * err;
+            }
+            my_loss += (double)(err * err);
         }
     }
+    if (!DET) loss_finish(v, my_loss, n, loss_out);
 }
 
 // mean of the per-item losses, summed in a fixed order
@@ -564,11 +649,13 @@ static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t
     return NUPS_OK;
 }
 
-static unsigned step_grid(const nups_store* s, uint64_t n)
+// 4 warps per block, one item per warp per pass; at most `blocks_per_sm` blocks per SM, so that the grid is
+// resident at once and a warp with several items can prefetch for its next one
+static unsigned step_grid(const nups_store* s, uint64_t n, unsigned blocks_per_sm = 16)
 {
-    unsigned cap = (unsigned)s->sm_count * 16;
+    unsigned cap = (unsigned)s->sm_count * blocks_per_sm;
     if (cap > NUPS_MAX_STEP_BLOCKS) cap = NUPS_MAX_STEP_BLOCKS;
-    return grid_for(n, 4, cap);     // 4 warps per block, one item per warp per pass
+    return grid_for(n, 4, cap);
 }
 
 #define DISPATCH_CH(L4, ...)                                      \
@@ -629,13 +716,13 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     rc = step_buffers(s, n, K + 3, true, &b);
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
-    unsigned grid = step_grid(s, n);
+    unsigned grid = step_grid(s, n, 2);      // register-heavy kernel: two resident blocks per SM
     nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, complex_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap)));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
-    return step_finish(s, n, K + 3, 3, b, d_loss_out, st);
+    return step_finish(s, n, K + 3, 3, b, d_loss_out, st, !s->cfg.deterministic);
 }
 
 extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
@@ -651,11 +738,11 @@ extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const 
     rc = step_buffers(s, n, 2, false, &b);
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
-    unsigned grid = step_grid(s, n);
+    unsigned grid = step_grid(s, n, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2));   // resident blocks at that depth's register use
     nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, s->req_keys, s->req_cap)));
+        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap)));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
-    return step_finish(s, n, 2, 2, b, d_loss_out, st);
+    return step_finish(s, n, 2, 2, b, d_loss_out, st, !s->cfg.deterministic);
 }
