@@ -439,7 +439,7 @@ def run_step_workload(args, device, which):
     loss = torch.zeros(1, device=device)
     reps = max(args.steps, 20)
     if which == "kge":
-        E, Rl, L, B, K = 5_000_000, 1000, 500, 8192, 10
+        E, Rl, L, B, K = args.kge_entities, 1000, 500, 8192, 10
         s = binding.Store(E + Rl, L, workers=WORKERS, sync_interval=SYNC_EVERY, deterministic=False, with_adagrad=True)
         s.init_uniform(0, 5, 0.05)
         nb = 64
@@ -459,7 +459,7 @@ def run_step_workload(args, device, which):
         per_item, upd, rows_per_item = 3 + K + (K + 3), K + 3, 2 * (K + 3)
         name, cfg = "complex_kernel", f"ComplEx+AdaGrad: 5M entities, 1000 relations, 500 fp32/row + accumulator, batch {B}, {K} negatives"
     else:
-        M, N, L, B = 10_000_000, 1_000_000, 100, 65536
+        M, N, L, B = args.mf_rows, args.mf_rows // 10, 100, 65536
         s = binding.Store(M + N, L, workers=WORKERS, sync_interval=SYNC_EVERY, deterministic=False)
         s.init_uniform(0, 5, 0.3)
         nb = 32
@@ -477,7 +477,7 @@ def run_step_workload(args, device, which):
             s.step_mf(i[a:a + B], j[a:a + B], x[a:a + B], 1e-4, 0.01, loss)
         per_item, upd, rows_per_item = 4, 2, 2
         name, cfg = "mf_kernel", f"MF: 10M x 1M, rank 100, batch {B}, L2 0.01"
-    t = _time_calls(step, reps)
+    dt = _time_calls(step, reps)
     s.kernel_timing(True)
     _time_calls(step, reps, warm=0)
     k_ms, k_n = s.kernel_time()
@@ -485,8 +485,8 @@ def run_step_workload(args, device, which):
     k_s = k_ms / 1e3 / max(k_n, 1)
     tables = 2 if which == "kge" else 1
     logical = B * rows_per_item * L * 4 * 2 * (1 if which == "mf" else 1)      # every touched row read and written once
-    print(json.dumps({"workload": cfg, "kernel": name, "hot_slots": s.stats()["hot_slots"], "us_per_step": t * 1e6,
-                      "kernel_us": k_s * 1e6, "key_accesses_per_s": B * per_item / t, "updates_per_s": B * upd / t,
+    print(json.dumps({"workload": cfg, "kernel": name, "hot_slots": s.stats()["hot_slots"], "us_per_step": dt * 1e6,
+                      "kernel_us": k_s * 1e6, "key_accesses_per_s": B * per_item / dt, "updates_per_s": B * upd / dt,
                       "logical_gbs": logical / k_s / 1e9, "logical_frac_of_hbm_peak": logical / k_s / 1e9 / hbm_peak,
                       "peak_kind": peak_kind, "final_loss": float(loss.item()), "tables": tables}), flush=True)
     s.close()
@@ -505,6 +505,8 @@ def main():
     ap.add_argument("--workers", type=int, default=WORKERS)
     ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
     ap.add_argument("--ps-keys", type=int, default=100_000_000)
+    ap.add_argument("--kge-entities", type=int, default=5_000_000, help="smaller for profiling runs")
+    ap.add_argument("--mf-rows", type=int, default=10_000_000, help="smaller for profiling runs")
     ap.add_argument("--ps-skews", default="0,0.6,1.0,1.4")
     ap.add_argument("--ps-topk", default="0,1000,100000")
     args = ap.parse_args()

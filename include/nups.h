@@ -247,7 +247,7 @@ nups_status nups_step_sgns(nups_store* store, const uint32_t* d_center, const ui
  * replaces the head when j is even, the tail when odd;
  * loss = softplus(-phi_pos) + sum_j softplus(phi_j); per key role with summed
  * gradient g: acc += g^2, val -= lr g / (sqrt(acc_pulled + g^2) + eps).
- * Needs with_adagrad and an even value_len.                                   */
+ * Needs with_adagrad, value_len <= 512 and K <= 30.                           */
 nups_status nups_step_complex(nups_store* store, const uint32_t* d_h, const uint32_t* d_r, const uint32_t* d_t,
                               uint64_t n, int32_t dist, uint32_t K, float lr, float eps, float* d_loss_out,
                               void* stream);

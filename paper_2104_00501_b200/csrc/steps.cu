@@ -262,192 +262,217 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
 }
 
 // ---------------------------------------------------------------------------------------------
-// ComplEx with AdaGrad.  Rows are [re(0..d-1) | im(0..d-1)], d = L/2 (even); a lane owns pairs of
-// adjacent components: float2 of the real half and the matching float2 of the imaginary half.
+// ComplEx with AdaGrad.  Rows are [re(0..d-1) | im(0..d-1)], d = L/2 (even).  One block of 128 threads
+// works on one triple at a time; thread c owns the two adjacent complex components 2c, 2c+1 (a float2
+// of the real half and the matching float2 of the imaginary half), so d <= 256.  All 2 * (3 + K) rows of
+// the triple (values and accumulators) are brought into shared memory by asynchronous copies at once,
+// each thread its own column; then two passes around one block-wide reduction: pass 1 forms the 1 + K
+// partial scores, the block adds them up, pass 2 forms the gradients and pushes the AdaGrad updates.
 // ---------------------------------------------------------------------------------------------
 struct C2 { float2 re, im; };
+constexpr int CPX_THREADS = 128;
+constexpr int CPX_MAX_KEYS = 34;          // 3 + K with K <= 30, rounded up
 
-template <int CH>
-__device__ __forceinline__ void load_row(const RowRef& r, uint32_t d2, unsigned lane, C2 (&x)[CH])
+__device__ __forceinline__ C2 c2_zero() { C2 z; z.re = make_float2(0.f, 0.f); z.im = z.re; return z; }
+
+__device__ __forceinline__ float c2_score(const C2& h, const C2& r, const C2& t)
 {
-    const float2* b = (const float2*)r.base;
-    const float2* p = (const float2*)r.pend;
-#pragma unroll
-    for (int m = 0; m < CH; ++m) {
-        uint32_t c = lane + 32 * m;
-        x[m].re = make_float2(0.f, 0.f);
-        x[m].im = x[m].re;
-        if (c < d2) {
-            x[m].re = b[c];
-            x[m].im = b[d2 + c];
-            if (p) {
-                float2 a = p[c], bb = p[d2 + c];
-                x[m].re.x += a.x; x[m].re.y += a.y; x[m].im.x += bb.x; x[m].im.y += bb.y;
-            }
-        }
-    }
+    return h.re.x * r.re.x * t.re.x + h.im.x * r.re.x * t.im.x + h.re.x * r.im.x * t.im.x - h.im.x * r.im.x * t.re.x +
+           h.re.y * r.re.y * t.re.y + h.im.y * r.re.y * t.im.y + h.re.y * r.im.y * t.im.y - h.im.y * r.im.y * t.re.y;
 }
 
-template <int CH>
-__device__ __forceinline__ float score(const C2 (&h)[CH], const C2 (&r)[CH], const C2 (&t)[CH])
+// g_h += coef * d(phi)/d(h), likewise for r and t (any of the three may be skipped).  Differences of
+// products are formed without fused multiply-add, so that a gradient that cancels exactly
+// (head == tail) is exactly zero here too.
+__device__ __forceinline__ void c2_grads(const C2& h, const C2& r, const C2& t, float coef, C2* gh, C2* gr, C2* gt)
 {
-    float s = 0.f;
-#pragma unroll
-    for (int m = 0; m < CH; ++m) {
-        s += h[m].re.x * r[m].re.x * t[m].re.x + h[m].im.x * r[m].re.x * t[m].im.x + h[m].re.x * r[m].im.x * t[m].im.x -
-             h[m].im.x * r[m].im.x * t[m].re.x;
-        s += h[m].re.y * r[m].re.y * t[m].re.y + h[m].im.y * r[m].re.y * t[m].im.y + h[m].re.y * r[m].im.y * t[m].im.y -
-             h[m].im.y * r[m].im.y * t[m].re.y;
+#define NUPS_C1(comp)                                                                                     \
+    {                                                                                                     \
+        const float hr = h.re.comp, hi = h.im.comp, rr = r.re.comp, ri = r.im.comp;                       \
+        const float tr = t.re.comp, ti = t.im.comp;                                                       \
+        if (gh) { gh->re.comp += coef * (rr * tr + ri * ti);                                              \
+                  gh->im.comp += coef * __fsub_rn(__fmul_rn(rr, ti), __fmul_rn(ri, tr)); }                \
+        if (gt) { gt->re.comp += coef * __fsub_rn(__fmul_rn(hr, rr), __fmul_rn(hi, ri));                  \
+                  gt->im.comp += coef * (hi * rr + hr * ri); }                                            \
+        if (gr) { gr->re.comp += coef * (hr * tr + hi * ti);                                              \
+                  gr->im.comp += coef * __fsub_rn(__fmul_rn(hr, ti), __fmul_rn(hi, tr)); }                \
     }
-    return warp_sum(s);
-}
-
-// g_h += coef * d(phi)/d(h), and likewise for r and t (any of the three may be skipped)
-template <int CH>
-__device__ __forceinline__ void grads(const C2 (&h)[CH], const C2 (&r)[CH], const C2 (&t)[CH], float coef, C2* gh,
-                                      C2* gr, C2* gt)
-{
-#pragma unroll
-    for (int m = 0; m < CH; ++m) {
-#define NUPS_C1(comp)                                                                                         \
-        {                                                                                                     \
-            float hr = h[m].re.comp, hi = h[m].im.comp, rr = r[m].re.comp, ri = r[m].im.comp;                 \
-            float tr = t[m].re.comp, ti = t[m].im.comp;                                                       \
-            /* differences of products are formed without fused multiply-add, so that a gradient  */ \
-            /* that cancels exactly (head == tail) is exactly zero here too                       */ \
-            if (gh) { gh[m].re.comp += coef * (rr * tr + ri * ti);                                    \
-                      gh[m].im.comp += coef * __fsub_rn(__fmul_rn(rr, ti), __fmul_rn(ri, tr)); }      \
-            if (gt) { gt[m].re.comp += coef * __fsub_rn(__fmul_rn(hr, rr), __fmul_rn(hi, ri));        \
-                      gt[m].im.comp += coef * (hi * rr + hr * ri); }                                  \
-            if (gr) { gr[m].re.comp += coef * (hr * tr + hi * ti);                                    \
-                      gr[m].im.comp += coef * __fsub_rn(__fmul_rn(hr, ti), __fmul_rn(hi, tr)); }      \
-        }
-        NUPS_C1(x)
-        NUPS_C1(y)
+    NUPS_C1(x)
+    NUPS_C1(y)
 #undef NUPS_C1
-    }
 }
 
-// AdaGrad update of one key role from its summed gradient: acc += g^2, val -= lr g / (sqrt(a + g^2) + eps)
-template <bool HOT, bool DET, int CH>
-__device__ __forceinline__ void adagrad_push(const View& v, uint32_t key, uint32_t q, const C2 (&g)[CH], uint32_t d2,
-                                             unsigned lane, float lr, float eps, float* uval_row, float* uacc_row,
-                                             bool pulled_too)
+// step = -lr * g / (sqrt(a + g^2) + eps) with the hardware's reciprocal square root (2 ulp)
+__device__ __forceinline__ float adagrad_step(float g, float g2, float a, float lr, float eps)
 {
-    RowRef rv = resolve<HOT>(v, key, q, 0);
-    RowRef ra = resolve<HOT>(v, key, q, 1);
-    const float2* ab = (const float2*)ra.base;
-    const float2* ap = (const float2*)ra.pend;
-    float2* ov = (float2*)(DET ? uval_row : rv.dst);
-    float2* oa = (float2*)(DET ? uacc_row : ra.dst);
-#pragma unroll
-    for (int m = 0; m < CH; ++m) {
-        uint32_t c = lane + 32 * m;
-        if (c < d2) {
-#pragma unroll
-            for (int half = 0; half < 2; ++half) {
-                uint32_t at = half ? d2 + c : c;
-                float2 gg = half ? g[m].im : g[m].re;
-                float2 a = ab[at];
-                if (ap) { float2 pa = ap[at]; a.x += pa.x; a.y += pa.y; }
-                float2 g2 = make_float2(gg.x * gg.x, gg.y * gg.y);
-                float2 dv = make_float2(-lr * gg.x / (sqrtf(a.x + g2.x) + eps), -lr * gg.y / (sqrtf(a.y + g2.y) + eps));
-                if (DET) { ov[at] = dv; oa[at] = g2; }
-                else { red_add_v2((float*)(ov + at), dv); red_add_v2((float*)(oa + at), g2); }
-            }
-        }
-    }
-    if (lane == 0) {
-        if (!DET && rv.slot >= 0) mark_dirty(v, q, rv.slot);
-        if (v.count) {
-            unsigned times = (pulled_too ? 1u : 0u) + (DET ? 0u : 1u);
-            if (times) note_access(v, key, rv.slot, times);
-        }
+    const float y = a + g2;
+    const float root = y > 0.f ? y * rsqrtf(y) : 0.f;
+    return __fdividef(-lr * g, root + eps);
+}
+
+// AdaGrad update of one key role from the thread's part of its summed gradient:
+// acc += g^2, val -= lr g / (sqrt(acc_pulled + g^2) + eps)
+template <bool DET>
+__device__ __forceinline__ void c2_adagrad_push(const View& v, const C2& g, const C2& a, unsigned long long row,
+                                                unsigned long long pend, uint32_t d2, uint32_t c, float lr, float eps,
+                                                float* uval_row, float* uacc_row)
+{
+    const float2 g2r = make_float2(g.re.x * g.re.x, g.re.y * g.re.y);
+    const float2 g2i = make_float2(g.im.x * g.im.x, g.im.y * g.im.y);
+    const float2 dvr = make_float2(adagrad_step(g.re.x, g2r.x, a.re.x, lr, eps), adagrad_step(g.re.y, g2r.y, a.re.y, lr, eps));
+    const float2 dvi = make_float2(adagrad_step(g.im.x, g2i.x, a.im.x, lr, eps), adagrad_step(g.im.y, g2i.y, a.im.y, lr, eps));
+    if (DET) {
+        float2* ov = (float2*)uval_row;
+        float2* oa = (float2*)uacc_row;
+        ov[c] = dvr; ov[d2 + c] = dvi; oa[c] = g2r; oa[d2 + c] = g2i;
+    } else {
+        float* ov = pend != NO_PEND ? v.dval + pend : v.val + row;
+        float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + row;
+        red_add_v2(ov + 2 * c, dvr); red_add_v2(ov + 2 * (d2 + c), dvi);
+        red_add_v2(oa + 2 * c, g2r); red_add_v2(oa + 2 * (d2 + c), g2i);
     }
 }
 
-template <bool HOT, bool DET, int CH>
-__global__ void __launch_bounds__(128)
+// the thread's part (re.x, re.y, im.x, im.y) of a parked row, plus the worker's pending replica updates
+__device__ __forceinline__ C2 c2_parked(const float4* park, uint32_t slot_idx, uint32_t tid, const float* slab,
+                                        unsigned long long pend, uint32_t d2)
+{
+    const float4 p = park[slot_idx * CPX_THREADS + tid];
+    C2 x;
+    x.re = make_float2(p.x, p.y);
+    x.im = make_float2(p.z, p.w);
+    if (pend != NO_PEND) {
+        const float2* s = (const float2*)(slab + pend);
+        const float2 a = s[tid], b = s[d2 + tid];
+        x.re.x += a.x; x.re.y += a.y; x.im.x += b.x; x.im.y += b.y;
+    }
+    return x;
+}
+
+__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gmem_src)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+
+template <bool HOT, bool DET>
+__global__ void __launch_bounds__(CPX_THREADS, 4)
 complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restrict__ rk, const uint32_t* __restrict__ tk,
                const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float eps, float* __restrict__ uval,
                float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
                float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
 {
-    const unsigned lane = threadIdx.x & 31;
-    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-    const uint32_t d2 = v.L4, per = K + 3;            // d/2 pairs = L/4
+    // park[2 * role][tid] = the thread's part of the role's value row, park[2 * role + 1][tid] = of its
+    // accumulator row; filled by asynchronous copies, all 2 * (3 + K) rows of a triple in flight at once
+    extern __shared__ __align__(16) float4 park[];
+    __shared__ unsigned long long s_row[CPX_MAX_KEYS], s_pend[CPX_MAX_KEYS];
+    __shared__ float s_part[CPX_THREADS / 32][32];                 // per-warp partial scores
+    __shared__ int s_ok;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t d2 = v.L4, per = K + 3;                         // d/2 component pairs = L/4
+    const bool mine = tid < d2;                                    // threads beyond the row width only help reduce
     const uint64_t L = (uint64_t)v.L4 * 4;
     double my_loss = 0.0;
-    for (uint64_t i = warp; i < n; i += nwarps) {
-        // start moving the rows of the warp's next item towards L2 (values and accumulators of its 3 + K keys)
-        if (i + nwarps < n) {
-            const uint64_t nx = i + nwarps;
-            uint32_t nk = lane == 0 ? hk[nx] : lane == 1 ? rk[nx] : lane == 2 ? tk[nx] : (lane < 3 + K ? negs[nx * K + lane - 3] : 0u);
-            for (uint32_t r = 0; r < 3 + K && r < 32; ++r) {
-                const uint32_t key = __shfl_sync(0xFFFFFFFFu, nk, r);
-                if (key < v.num_keys) prefetch_row(v, key, true, lane);
-            }
-        }
+    for (uint64_t i = blockIdx.x; i < n; i += gridDim.x) {
         const uint32_t q = worker_of_item(i, n, v.R);
-        const uint32_t kh = hk[i], kr = rk[i], kt = tk[i];
-        bool ok = kh < v.num_keys && kr < v.num_keys && kt < v.num_keys;
-        for (uint32_t j = 0; j < K; ++j) ok = ok && negs[i * K + j] < v.num_keys;
-        if (DET && lane == 0) {
-            ukeys[i * per] = ok ? kh : NUPS_INVALID_KEY;
-            ukeys[i * per + 1] = ok ? kr : NUPS_INVALID_KEY;
-            ukeys[i * per + 2] = ok ? kt : NUPS_INVALID_KEY;
-            for (uint32_t j = 0; j < K; ++j) ukeys[i * per + 3 + j] = ok ? negs[i * K + j] : NUPS_INVALID_KEY;
+        // thread j < 3 + K looks up role j: head, relation, tail, negatives
+        if (tid == 0) s_ok = 1;
+        __syncthreads();
+        uint32_t key = 0;
+        int slot = -1;
+        if (tid < per) {
+            key = tid == 0 ? hk[i] : tid == 1 ? rk[i] : tid == 2 ? tk[i] : negs[i * K + tid - 3];
+            const bool ok = key < v.num_keys;
+            if (!ok) s_ok = 0;
+            slot = (HOT && ok) ? __ldg(v.slot_of + key) : -1;
+            if (slot < 0) slot = -1;
+            s_row[tid] = (unsigned long long)key * L;
+            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : NO_PEND;
         }
-        if (!ok) {
-            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+        __syncthreads();
+        if (!s_ok) {                                               // a key out of range: the whole item is skipped
+            if (DET && tid < per) ukeys[i * per + tid] = NUPS_INVALID_KEY;
+            if (tid == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
-        C2 h[CH], r[CH], t[CH], gh[CH], gr[CH], gt[CH];
-        load_row<CH>(resolve<HOT>(v, kh, q, 0), d2, lane, h);
-        load_row<CH>(resolve<HOT>(v, kr, q, 0), d2, lane, r);
-        load_row<CH>(resolve<HOT>(v, kt, q, 0), d2, lane, t);
-#pragma unroll
-        for (int m = 0; m < CH; ++m) {
-            gh[m].re = make_float2(0.f, 0.f); gh[m].im = gh[m].re;
-            gr[m] = gh[m]; gt[m] = gh[m];
+        if (tid < per) {
+            if (DET) ukeys[i * per + tid] = key;
+            if (!DET && slot >= 0) mark_dirty(v, q, slot);
+            if (v.count) {
+                const unsigned times = (tid < 3 ? 1u : 0u) + (DET ? 0u : 1u);       // pulled (+ pushed in fast mode)
+                if (times) note_access(v, key, slot, times);
+            }
+            if (v.owner && tid < 3) request_localize(v, key, q, req, req_cap);
         }
-        float phi = clamp30(score<CH>(h, r, t));
-        float loss = softplusf_(-phi);
-        grads<CH>(h, r, t, sigmoidf_(phi) - 1.f, gh, gr, gt);
+        if (mine) {
+            for (uint32_t role = 0; role < per; ++role) {
+                const float2* a = (const float2*)(v.val + s_row[role]);
+                const float2* b = (const float2*)(v.acc + s_row[role]);
+                float4* pv = park + (2 * role) * CPX_THREADS + tid;
+                float4* pa = park + (2 * role + 1) * CPX_THREADS + tid;
+                cp_async_8(pv, a + tid); cp_async_8((float2*)pv + 1, a + d2 + tid);
+                cp_async_8(pa, b + tid); cp_async_8((float2*)pa + 1, b + d2 + tid);
+            }
+            asm volatile("cp.async.commit_group;\n cp.async.wait_group 0;" ::: "memory");
+        }
+        C2 h = c2_zero(), r = c2_zero(), t = c2_zero();
+        if (mine) {
+            h = c2_parked(park, 0, tid, v.dval, s_pend[0], d2);
+            r = c2_parked(park, 2, tid, v.dval, s_pend[1], d2);
+            t = c2_parked(park, 4, tid, v.dval, s_pend[2], d2);
+        }
+        // pass 1: partial scores; lane j of each warp ends up holding the warp's sum of score j
+        float part = 0.f;
+        {
+            const float sc = warp_sum(mine ? c2_score(h, r, t) : 0.f);
+            if (lane == 0) part = sc;
+        }
         for (uint32_t j = 0; j < K; ++j) {
-            const uint32_t ke = negs[i * K + j];
-            C2 e[CH], ge[CH];
-            load_row<CH>(resolve<HOT>(v, ke, q, 0), d2, lane, e);
+            float sc = 0.f;
+            if (mine) {
+                const C2 e = c2_parked(park, 2 * (3 + j), tid, v.dval, s_pend[3 + j], d2);
+                sc = (j & 1) == 0 ? c2_score(e, r, t) : c2_score(h, r, e);
+            }
+            sc = warp_sum(sc);
+            if (lane == j + 1) part = sc;
+        }
+        s_part[warp][lane] = part;
+        __syncthreads();
+        // every thread needs every score: lane j adds the warps' sums of score j, then they are passed around
+        float phi_l = 0.f;
 #pragma unroll
-            for (int m = 0; m < CH; ++m) { ge[m].re = make_float2(0.f, 0.f); ge[m].im = ge[m].re; }
-            if ((j & 1) == 0) {
-                float ph = clamp30(score<CH>(e, r, t));
-                loss += softplusf_(ph);
-                grads<CH>(e, r, t, sigmoidf_(ph), ge, gr, gt);
-            } else {
-                float ph = clamp30(score<CH>(h, r, e));
-                loss += softplusf_(ph);
-                grads<CH>(h, r, e, sigmoidf_(ph), gh, gr, ge);
-            }
-            adagrad_push<HOT, DET, CH>(v, ke, q, ge, d2, lane, lr, eps, DET ? uval + (i * per + 3 + j) * L : nullptr,
-                                       DET ? uacc + (i * per + 3 + j) * L : nullptr, false);
+        for (int w = 0; w < CPX_THREADS / 32; ++w) phi_l += s_part[w][lane];
+        phi_l = clamp30(phi_l);
+        const float coef_l = lane == 0 ? sigmoidf_(phi_l) - 1.f : sigmoidf_(phi_l);
+        float loss_l = lane == 0 ? softplusf_(-phi_l) : (lane <= K ? softplusf_(phi_l) : 0.f);
+        loss_l = warp_sum(loss_l);
+        // pass 2: gradients and updates
+        C2 gh = c2_zero(), gr = c2_zero(), gt = c2_zero();
+        c2_grads(h, r, t, __shfl_sync(0xFFFFFFFFu, coef_l, 0), &gh, &gr, &gt);
+        for (uint32_t j = 0; j < K; ++j) {
+            const float coef = __shfl_sync(0xFFFFFFFFu, coef_l, j + 1);
+            if (!mine) continue;
+            const C2 e = c2_parked(park, 2 * (3 + j), tid, v.dval, s_pend[3 + j], d2);
+            C2 ge = c2_zero();
+            if ((j & 1) == 0) c2_grads(e, r, t, coef, &ge, &gr, &gt);
+            else c2_grads(h, r, e, coef, &gh, &gr, &ge);
+            const C2 a = c2_parked(park, 2 * (3 + j) + 1, tid, v.dacc, s_pend[3 + j], d2);
+            c2_adagrad_push<DET>(v, ge, a, s_row[3 + j], s_pend[3 + j], d2, tid, lr, eps,
+                                 DET ? uval + (i * per + 3 + j) * L : nullptr, DET ? uacc + (i * per + 3 + j) * L : nullptr);
         }
-        adagrad_push<HOT, DET, CH>(v, kh, q, gh, d2, lane, lr, eps, DET ? uval + (i * per) * L : nullptr,
-                                   DET ? uacc + (i * per) * L : nullptr, true);
-        adagrad_push<HOT, DET, CH>(v, kr, q, gr, d2, lane, lr, eps, DET ? uval + (i * per + 1) * L : nullptr,
-                                   DET ? uacc + (i * per + 1) * L : nullptr, true);
-        adagrad_push<HOT, DET, CH>(v, kt, q, gt, d2, lane, lr, eps, DET ? uval + (i * per + 2) * L : nullptr,
-                                   DET ? uacc + (i * per + 2) * L : nullptr, true);
-        if (lane == 0) {
-            if (v.owner) {
-                request_localize(v, kh, q, req, req_cap);
-                request_localize(v, kr, q, req, req_cap);
-                request_localize(v, kt, q, req, req_cap);
+        if (mine) {
+            const C2* g3[3] = {&gh, &gr, &gt};
+#pragma unroll
+            for (int role = 0; role < 3; ++role) {
+                const C2 a = c2_parked(park, 2 * role + 1, tid, v.dacc, s_pend[role], d2);
+                c2_adagrad_push<DET>(v, *g3[role], a, s_row[role], s_pend[role], d2, tid, lr, eps,
+                                     DET ? uval + (i * per + role) * L : nullptr, DET ? uacc + (i * per + role) * L : nullptr);
             }
-            if (DET) loss_item[i] = loss;
         }
-        my_loss += (double)loss;
+        if (tid == 0) {
+            if (DET) loss_item[i] = loss_l;
+            my_loss += (double)loss_l;
+        }
     }
     if (!DET) loss_finish(v, my_loss, n, loss_out);
 }
@@ -706,7 +731,7 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
                                          void* stream)
 {
     if (!s || !d_h || !d_r || !d_t || n == 0 || n * (uint64_t)(K + 3) >= (1ull << 32)) return NUPS_EINVAL;
-    if (!s->acc || s->L / 4 > 128) return NUPS_EINVAL;
+    if (!s->acc || s->L / 4 > CPX_THREADS || K > 30) return NUPS_EINVAL;    // one thread per component pair, one lane per score
     cudaStream_t st = (cudaStream_t)stream;
     nups_status rc = nups_draw_negatives(s, dist, n * K, st);
     if (rc != NUPS_OK) return rc;
@@ -716,10 +741,28 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     rc = step_buffers(s, n, K + 3, true, &b);
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
-    unsigned grid = step_grid(s, n, 2);      // register-heavy kernel: two resident blocks per SM
+    // shared memory: one 16-byte column entry per thread for the value and the accumulator row of every role
+    const size_t smem = (size_t)2 * (K + 3) * CPX_THREADS * sizeof(float4);
+    if (smem > (size_t)s->max_smem - 4096) return NUPS_EINVAL;
+    unsigned per_sm = (unsigned)(((size_t)s->max_smem - 1024) / (smem + 2048));
+    if (per_sm > 4) per_sm = 4;
+    if (per_sm < 1) per_sm = 1;
+    uint64_t want = n < (uint64_t)s->sm_count * per_sm ? n : (uint64_t)s->sm_count * per_sm;
+    unsigned grid = (unsigned)want;
+    static bool attr_set[2][2] = {{false, false}, {false, false}};
+    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0;
+    if (!attr_set[hi][di]) {
+        cudaError_t e;
+        if (hi && di) e = cudaFuncSetAttribute(complex_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else if (hi) e = cudaFuncSetAttribute(complex_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else if (di) e = cudaFuncSetAttribute(complex_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else e = cudaFuncSetAttribute(complex_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
+        attr_set[hi][di] = true;
+    }
     nups_time_begin(s, st);
-    DISPATCH_MODE(s, DISPATCH_CH(v.L4, complex_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap)));
+    DISPATCH_MODE(s, complex_kernel<HOT, DET><<<grid, CPX_THREADS, smem, st>>>(
+        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return step_finish(s, n, K + 3, 3, b, d_loss_out, st, !s->cfg.deterministic);
