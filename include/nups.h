@@ -282,6 +282,14 @@ nups_status nups_get_stats(nups_store* store, uint64_t* h_out, void* stream);
 nups_status nups_kernel_timing(nups_store* store, int enable);
 nups_status nups_kernel_time(nups_store* store, double* h_ms_out, uint64_t* h_launches_out, void* stream);
 
+/* Measurement aid: the rate at which this GPU applies 128-bit floating-point
+ * reductions (red.global.add.v4.f32, the instruction every fast-mode update
+ * uses) to distinct, streaming addresses.  Adds zeros to the first `bytes` bytes
+ * of the value table `reps` times (the table is unchanged) and returns the
+ * payload rate in GB/s.  This is the ceiling of push and of the workload steps
+ * in fast mode.  Synchronises the stream.                                      */
+nups_status nups_probe_reduction_rate(nups_store* store, uint64_t bytes, uint32_t reps, double* h_gbs_out, void* stream);
+
 const char* nups_strerror(nups_status status);
 const char* nups_last_cuda_error(void);
 

@@ -25,7 +25,7 @@ EXPORTS = [
     "nups_push2", "nups_push_noalloc", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_step_complex", "nups_step_mf",
-    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_strerror", "nups_last_cuda_error",
+    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_probe_reduction_rate", "nups_strerror", "nups_last_cuda_error",
 ]
 
 
@@ -91,6 +91,7 @@ def load(build_if_missing: bool = True):
         "nups_get_stats": [vp, C.POINTER(u64), vp],
         "nups_kernel_timing": [vp, C.c_int],
         "nups_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
+        "nups_probe_reduction_rate": [vp, u64, u32, C.POINTER(C.c_double), vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -325,6 +326,13 @@ class Store:
         ms, n = C.c_double(), C.c_uint64()
         self._chk(self._l.nups_kernel_time(self._s, C.byref(ms), C.byref(n), _stream()), "nups_kernel_time")
         return ms.value, n.value
+
+    def probe_reduction_rate(self, nbytes, reps=10):
+        """GB/s of 128-bit floating-point reductions to streaming addresses (the ceiling of fast-mode updates)."""
+        g = C.c_double()
+        self._chk(self._l.nups_probe_reduction_rate(self._s, nbytes, reps, C.byref(g), _stream()),
+                  "nups_probe_reduction_rate")
+        return g.value
 
     def stats(self):
         out = (C.c_uint64 * 8)()

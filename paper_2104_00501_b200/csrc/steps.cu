@@ -1,8 +1,9 @@
 // Workload steps driving the store: skip-gram with negative sampling, ComplEx with AdaGrad and
-// matrix factorization (NuPS Section 5.1).  One warp per item: rows are pulled into registers,
-// dot products are reduced with warp shuffles, updates are pushed either straight to the store
-// (fast mode, 128-bit reductions) or into a row buffer that the ordered push applies afterwards
-// (deterministic mode, all pulls see the values from before the step).
+// matrix factorization (NuPS Section 5.1).  SGNS and ComplEx: one block per item, rows staged in shared
+// memory by asynchronous copies, one thread per chunk of a row; MF: one warp per item with a ring of
+// items in flight.  Updates are pushed either straight to the store (fast mode, vector reductions) or
+// into a row buffer that the ordered push applies afterwards (deterministic mode, all pulls see the
+// values from before the step).
 #include "nups_internal.cuh"
 
 static inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
@@ -12,49 +13,6 @@ namespace {
 __device__ __forceinline__ float clamp30(float x) { return fminf(30.f, fmaxf(-30.f, x)); }
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 __device__ __forceinline__ float softplusf_(float x) { return fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))); }
-
-// Where a key's row is read from and written to by worker q.
-struct RowRef {
-    const float* base;     // stored row
-    const float* pend;     // the worker's pending replica updates, or NULL
-    float* dst;            // where pushes go: the replica (hot) or the stored row
-    int slot;
-};
-
-// (the step workloads keep key -> slot small enough to stay in L2, so the slot map is read directly
-// instead of going through the technique bitmap first)
-template <bool HOT>
-__device__ __forceinline__ RowRef resolve(const View& v, uint32_t key, uint32_t q, int which)
-{
-    RowRef r;
-    float* table = which ? v.acc : v.val;
-    const uint64_t L = (uint64_t)v.L4 * 4;
-    r.base = table + (uint64_t)key * L;
-    r.pend = nullptr;
-    r.dst = table + (uint64_t)key * L;
-    r.slot = HOT ? __ldg(v.slot_of + key) : -1;
-    if (r.slot >= 0) {
-        float* slab = which ? v.dacc : v.dval;
-        float* p = slab + ((uint64_t)q * v.Hcap + (uint64_t)r.slot) * L;
-        r.pend = p;
-        r.dst = p;
-    } else r.slot = -1;
-    return r;
-}
-
-// Warp-cooperative L2 prefetch of the row of `key` in the value table (and the accumulator table):
-// issued for the warp's NEXT item while the current one is being worked on.
-__device__ __forceinline__ void prefetch_row(const View& v, uint32_t key, bool with_acc, unsigned lane)
-{
-    const uint32_t row_bytes = v.L4 * 16;
-    const uint32_t lines = (row_bytes + 127) / 128;
-    const char* a = (const char*)(v.val + (uint64_t)key * v.L4 * 4);
-    const char* b = (const char*)(v.acc + (uint64_t)key * v.L4 * 4);
-    for (uint32_t idx = lane; idx < lines * (with_acc ? 2u : 1u); idx += 32) {
-        const uint32_t line = idx < lines ? idx : idx - lines;
-        prefetch_l2((idx < lines ? a : b) + (size_t)line * 128);
-    }
-}
 
 __device__ __forceinline__ void red_add_v2(float* addr, float2 x)
 {
@@ -75,30 +33,8 @@ __device__ __forceinline__ void request_localize(const View& v, uint32_t key, ui
     if (at < cap) req[at] = key;
 }
 
-// Rows of several keys at once: all technique lookups are issued before any of them is used, so the
-// dependent chain key -> hot bit -> slot -> row is paid once per group, not once per row.
-struct RowAt {
-    unsigned long long row;    // offset of the stored row, in floats
-    unsigned long long pend;   // offset of the worker's replica row in the slab, in floats, or NO_PEND
-    int slot;
-};
+// offset value meaning "this key has no replica row"
 constexpr unsigned long long NO_PEND = ~0ull;
-
-// The step workloads keep key -> slot small enough to stay in L2, so the slot map is read directly
-// (one lookup) instead of going through the technique bitmap first.
-template <bool HOT, int NR>
-__device__ __forceinline__ void resolve_rows(const View& v, const uint32_t (&key)[NR], const bool (&act)[NR],
-                                             uint32_t q, RowAt (&r)[NR])
-{
-#pragma unroll
-    for (int u = 0; u < NR; ++u) r[u].slot = (HOT && act[u]) ? __ldg(v.slot_of + key[u]) : -1;
-    const unsigned long long L = (unsigned long long)v.L4 * 4;
-#pragma unroll
-    for (int u = 0; u < NR; ++u) {
-        r[u].row = (unsigned long long)key[u] * L;
-        r[u].pend = r[u].slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)r[u].slot) * L : NO_PEND;
-    }
-}
 
 // per-launch loss in fast mode: one 64-bit integer addition per warp carries both the warp's loss (fixed
 // point, 2^-16 units, low 48 bits) and a ticket (high 16 bits); integer additions to one address do not
@@ -121,142 +57,125 @@ __device__ __forceinline__ void loss_finish(const View& v, double warp_loss, uin
 }
 
 // ---------------------------------------------------------------------------------------------
-// skip-gram with negative sampling
+// skip-gram with negative sampling.  One block works on one pair at a time; thread c owns float4 chunk c
+// of every row (blockDim = row width in float4 rounded up to whole warps, at most 128).  The 2 + K rows
+// of the pair - and the worker's pending replica rows of the replicated ones - are brought into shared
+// memory by asynchronous 16-byte copies, all in flight at once, each thread its own column; the 1 + K
+// dot products are reduced across the block once; then every thread forms and pushes its chunk of the
+// updates.
 // ---------------------------------------------------------------------------------------------
-#ifndef NUPS_SGNS_UB
-#define NUPS_SGNS_UB 2
-#endif
-#ifndef NUPS_SGNS_MINBLOCKS
-#define NUPS_SGNS_MINBLOCKS 7
-#endif
-constexpr int SGNS_UB = NUPS_SGNS_UB;      // output rows (context + negatives) handled per group
+constexpr int SGNS_MAX_THREADS = 128;
 
-template <bool HOT, bool DET, int CH>
-__global__ void __launch_bounds__(128, NUPS_SGNS_MINBLOCKS)
-sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
-            const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float* __restrict__ upd,
-            uint32_t* __restrict__ ukeys, float* __restrict__ loss_item, float* __restrict__ loss_out, uint32_t* req,
-            uint64_t req_cap)
+__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src)
 {
-    const unsigned lane = threadIdx.x & 31;
-    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+
+template <bool HOT, bool DET>
+__global__ void __launch_bounds__(SGNS_MAX_THREADS, 8)
+sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
+            const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr,
+            float* __restrict__ upd, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
+            float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
+{
+    // park[2 * role][tid] = the thread's chunk of the role's stored row, park[2 * role + 1][tid] = of the
+    // worker's pending replica row (only filled for replicated keys).  Roles: 0 context, 1..K negatives,
+    // K + 1 centre.
+    extern __shared__ __align__(16) float4 park[];
+    __shared__ unsigned long long s_row[32], s_pend[32];
+    __shared__ float s_part[SGNS_MAX_THREADS / 32][32];
+    __shared__ int s_ok;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
     const uint32_t L4 = v.L4, per = K + 2;
-    const unsigned long long L = (unsigned long long)L4 * 4;
-    const float4* val4 = (const float4*)v.val;
-    const float4* slab4 = (const float4*)v.dval;
+    const bool mine = tid < L4;
+    const uint64_t L = (uint64_t)L4 * 4;
     double my_loss = 0.0;
-    for (uint64_t i = warp; i < n; i += nwarps) {
+    for (uint64_t i = blockIdx.x; i < n; i += gridDim.x) {
         const uint32_t q = worker_of_item(i, n, v.R);
-        // lane l holds the key of row l of the item: 0 = context, 1..K = negatives, K+1 = centre;
-        // one coalesced round fetches the keys, a second one their replica slots
-        const uint32_t mykey = lane == 0 ? context[i] : (lane <= K ? negs[i * K + lane - 1] : (lane == K + 1 ? center[i] : 0u));
-        const bool mine = lane <= K + 1;
-        const bool ok = __all_sync(0xFFFFFFFFu, !mine || mykey < v.num_keys);
-        if (DET && mine) ukeys[i * per + lane] = ok ? mykey : NUPS_INVALID_KEY;
-        if (!ok) {
-            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+        if (tid == 0) s_ok = 1;
+        __syncthreads();
+        uint32_t key = 0;
+        int slot = -1;
+        if (tid < per) {
+            key = tid == 0 ? context[i] : (tid <= K ? negs[i * K + tid - 1] : center[i]);
+            const bool ok = key < v.num_keys;
+            if (!ok) s_ok = 0;
+            slot = (HOT && ok) ? __ldg(v.slot_of + key) : -1;
+            if (slot < 0) slot = -1;
+            s_row[tid] = (unsigned long long)key * L;
+            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : NO_PEND;
+        }
+        __syncthreads();
+        if (!s_ok) {                                               // a key out of range: the whole item is skipped
+            if (DET && tid < per) ukeys[i * per + tid] = NUPS_INVALID_KEY;
+            if (tid == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
-        const unsigned long long myrow = (unsigned long long)mykey * L;
-        const int myslot = (HOT && mine) ? __ldg(v.slot_of + mykey) : -1;
-        if (mine) {
-            // pull the lane's row towards L2 while the slots are looked up and the first rows are used
-            const char* rp = (const char*)(v.val + myrow);
-            for (uint32_t b = 0; b < L4 * 16; b += 128) prefetch_l2(rp + b);
-        }
-        const unsigned long long mypend = myslot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)myslot) * L : NO_PEND;
-        if (mine) {
-            if (!DET && myslot >= 0) mark_dirty(v, q, myslot);
+        if (tid < per) {
+            if (DET) ukeys[i * per + tid] = key;
+            if (!DET && slot >= 0) mark_dirty(v, q, slot);
             if (v.count) {
                 // context and centre: pulled (+ pushed in fast mode); negatives: pushed (their draw counted the sample)
-                const unsigned times = (lane == 0 || lane == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
-                if (times) note_access(v, mykey, myslot, times);
+                const unsigned times = (tid == 0 || tid == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
+                if (times) note_access(v, key, slot, times);
             }
-            if (v.owner && (lane == 0 || lane == K + 1)) request_localize(v, mykey, q, req, req_cap);
+            if (v.owner && (tid == 0 || tid == K + 1)) request_localize(v, key, q, req, req_cap);
         }
-        // centre row
-        const unsigned long long crow = __shfl_sync(0xFFFFFFFFu, myrow, K + 1);
-        const unsigned long long cpend = __shfl_sync(0xFFFFFFFFu, mypend, K + 1);
-        float4 vr[CH], gv[CH];
-#pragma unroll
-        for (int m = 0; m < CH; ++m) {
-            const uint32_t c = lane + 32 * m;
-            vr[m] = make_float4(0.f, 0.f, 0.f, 0.f);
-            gv[m] = vr[m];
-            if (c < L4) {
-                vr[m] = val4[crow / 4 + c];
-                if (HOT && cpend != NO_PEND) vr[m] = add4(vr[m], slab4[cpend / 4 + c]);
+        if (mine) {
+            for (uint32_t role = 0; role < per; ++role) {
+                cp_async_16(park + (2 * role) * nthr + tid, (const float4*)(v.val + s_row[role]) + tid);
+                if (HOT && s_pend[role] != NO_PEND)
+                    cp_async_16(park + (2 * role + 1) * nthr + tid, (const float4*)(v.dval + s_pend[role]) + tid);
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        float loss = 0.f;
-        for (uint32_t j0 = 0; j0 <= K; j0 += SGNS_UB) {
-            unsigned long long urow[SGNS_UB], upend[SGNS_UB];
-            float4 ur[SGNS_UB][CH];
-#pragma unroll
-            for (int u = 0; u < SGNS_UB; ++u) {
-                const uint32_t j = min(j0 + u, K);
-                urow[u] = __shfl_sync(0xFFFFFFFFu, myrow, j);
-                upend[u] = __shfl_sync(0xFFFFFFFFu, mypend, j);
-#pragma unroll
-                for (int m = 0; m < CH; ++m) {
-                    const uint32_t c = lane + 32 * m;
-                    ur[u][m] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (j0 + u <= K && c < L4) {
-                        ur[u][m] = val4[urow[u] / 4 + c];
-                        if (HOT && upend[u] != NO_PEND) ur[u][m] = add4(ur[u][m], slab4[upend[u] / 4 + c]);
-                    }
-                }
+        if (mine) asm volatile("cp.async.wait_group 0;" ::: "memory");
+        auto parked = [&](uint32_t role) -> float4 {
+            float4 x = park[(2 * role) * nthr + tid];
+            if (HOT && s_pend[role] != NO_PEND) x = add4(x, park[(2 * role + 1) * nthr + tid]);
+            return x;
+        };
+        const float4 vr = mine ? parked(K + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
+        // partial dot products; lane j of each warp ends up holding the warp's part of x_j
+        float part = 0.f;
+        for (uint32_t j = 0; j <= K; ++j) {
+            float d = 0.f;
+            if (mine) {
+                const float4 u = parked(j);
+                d = vr.x * u.x + vr.y * u.y + vr.z * u.z + vr.w * u.w;
             }
-            float dot[SGNS_UB];
-#pragma unroll
-            for (int u = 0; u < SGNS_UB; ++u) {
-                dot[u] = 0.f;
-#pragma unroll
-                for (int m = 0; m < CH; ++m)
-                    dot[u] += vr[m].x * ur[u][m].x + vr[m].y * ur[u][m].y + vr[m].z * ur[u][m].z + vr[m].w * ur[u][m].w;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-#pragma unroll
-                for (int u = 0; u < SGNS_UB; ++u) dot[u] += __shfl_xor_sync(0xFFFFFFFFu, dot[u], o);
-            }
-#pragma unroll
-            for (int u = 0; u < SGNS_UB; ++u) {
-                const uint32_t j = j0 + u;
-                if (j > K) continue;
-                const float x = clamp30(dot[u]);
-                const float g = sigmoidf_(x) - (j == 0 ? 1.f : 0.f);
-                loss += j == 0 ? softplusf_(-x) : softplusf_(x);
-                const float sc = -lr * g;
-                const bool hot = HOT && upend[u] != NO_PEND;
-                float* out = DET ? upd + (i * per + j) * L : (hot ? v.dval + upend[u] : v.val + urow[u]);
-#pragma unroll
-                for (int m = 0; m < CH; ++m) {
-                    const uint32_t c = lane + 32 * m;
-                    if (c < L4) {
-                        const float4 du = make_float4(sc * vr[m].x, sc * vr[m].y, sc * vr[m].z, sc * vr[m].w);
-                        if (DET) ((float4*)out)[c] = du;
-                        else red_add_v4(out + 4 * c, du);
-                        gv[m].x += g * ur[u][m].x; gv[m].y += g * ur[u][m].y;
-                        gv[m].z += g * ur[u][m].z; gv[m].w += g * ur[u][m].w;
-                    }
-                }
-            }
+            d = warp_sum(d);
+            if (lane == j) part = d;
         }
-        const bool chot = HOT && cpend != NO_PEND;
-        float* out = DET ? upd + (i * per + K + 1) * L : (chot ? v.dval + cpend : v.val + crow);
-#pragma unroll
-        for (int m = 0; m < CH; ++m) {
-            const uint32_t c = lane + 32 * m;
-            if (c < L4) {
-                const float4 dv = make_float4(-lr * gv[m].x, -lr * gv[m].y, -lr * gv[m].z, -lr * gv[m].w);
-                if (DET) ((float4*)out)[c] = dv;
-                else red_add_v4(out + 4 * c, dv);
-            }
+        s_part[warp][lane] = part;
+        __syncthreads();
+        float x_l = 0.f;
+        for (uint32_t w = 0; w < (nthr >> 5); ++w) x_l += s_part[w][lane];
+        x_l = clamp30(x_l);
+        const float g_l = sigmoidf_(x_l) - (lane == 0 ? 1.f : 0.f);
+        float loss_l = lane == 0 ? softplusf_(-x_l) : (lane <= K ? softplusf_(x_l) : 0.f);
+        loss_l = warp_sum(loss_l);
+        float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (uint32_t j = 0; j <= K; ++j) {
+            const float g = __shfl_sync(0xFFFFFFFFu, g_l, j);
+            if (!mine) continue;
+            const float4 u = parked(j);
+            const float sc = -lr * g;
+            const float4 du = make_float4(sc * vr.x, sc * vr.y, sc * vr.z, sc * vr.w);
+            if (DET) ((float4*)(upd + (i * per + j) * L))[tid] = du;
+            else red_add_v4((s_pend[j] != NO_PEND ? v.dval + s_pend[j] : v.val + s_row[j]) + 4 * tid, du);
+            gv.x += g * u.x; gv.y += g * u.y; gv.z += g * u.z; gv.w += g * u.w;
         }
-        if (DET && lane == 0) loss_item[i] = loss;
-        my_loss += (double)loss;
+        if (mine) {
+            const float4 dv = make_float4(-lr * gv.x, -lr * gv.y, -lr * gv.z, -lr * gv.w);
+            if (DET) ((float4*)(upd + (i * per + K + 1) * L))[tid] = dv;
+            else red_add_v4((s_pend[K + 1] != NO_PEND ? v.dval + s_pend[K + 1] : v.val + s_row[K + 1]) + 4 * tid, dv);
+        }
+        if (tid == 0) {
+            if (DET) loss_item[i] = loss_l;
+            my_loss += (double)loss_l;
+        }
     }
     if (!DET) loss_finish(v, my_loss, n, loss_out);
 }
@@ -707,7 +626,7 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
 {
     if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
     if (K > 30) return NUPS_EINVAL;                         // one lane per key of an item
-    if (s->L / 4 > 128) return NUPS_EINVAL;                 // rows of up to 512 floats are held in registers
+    if (s->L / 4 > SGNS_MAX_THREADS) return NUPS_EINVAL;    // one thread per float4 chunk of a row: at most 512 floats
     cudaStream_t st = (cudaStream_t)stream;
     nups_status rc = nups_draw_negatives(s, dist, n * K, st);
     if (rc != NUPS_OK) return rc;
@@ -717,10 +636,32 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
     rc = step_buffers(s, n, K + 2, false, &b);
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
-    unsigned grid = step_grid(s, n);
+    const unsigned threads = ((v.L4 + 31) / 32) * 32;           // one thread per float4 chunk of a row
+    const size_t smem = (size_t)2 * (K + 2) * threads * sizeof(float4);
+    unsigned per_sm = (unsigned)(((size_t)s->max_smem - 1024) / (smem + 2048));
+#ifndef NUPS_SGNS_PER_SM
+#define NUPS_SGNS_PER_SM 12
+#endif
+    if (per_sm > NUPS_SGNS_PER_SM) per_sm = NUPS_SGNS_PER_SM;
+    if (per_sm > 2048 / threads) per_sm = 2048 / threads;
+    if (per_sm < 1) return NUPS_EINVAL;
+    const uint64_t want = n < (uint64_t)s->sm_count * per_sm ? n : (uint64_t)s->sm_count * per_sm;
+    const unsigned grid = (unsigned)want;
+    static bool attr_set[2][2] = {{false, false}, {false, false}};
+    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0;
+    if (smem > 48 * 1024 && !attr_set[hi][di]) {
+        cudaError_t e;
+        if (hi && di) e = cudaFuncSetAttribute(sgns_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else if (hi) e = cudaFuncSetAttribute(sgns_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else if (di) e = cudaFuncSetAttribute(sgns_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else e = cudaFuncSetAttribute(sgns_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
+        attr_set[hi][di] = true;
+    }
     nups_time_begin(s, st);
-    DISPATCH_MODE(s, DISPATCH_CH(v.L4, sgns_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap)));
+    DISPATCH_MODE(s, sgns_kernel<HOT, DET><<<grid, threads, smem, st>>>(
+        v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys,
+        s->req_cap));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return step_finish(s, n, K + 2, 2, b, d_loss_out, st, !s->cfg.deterministic);

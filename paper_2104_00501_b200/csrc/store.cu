@@ -1234,6 +1234,44 @@ extern "C" nups_status nups_get_owner(nups_store* s, const uint32_t* d_keys, uin
 }
 
 // ---------------------------------------------------------------------------------------------
+// reduction-rate probe
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+red_probe_kernel(float* base, uint64_t n4)
+{
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (; i < n4; i += stride) red_add_v4(base + 4 * i, zero);
+}
+
+extern "C" nups_status nups_probe_reduction_rate(nups_store* s, uint64_t bytes, uint32_t reps, double* h_gbs_out, void* stream)
+{
+    if (!s || !h_gbs_out || reps == 0) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint64_t table_bytes = (uint64_t)s->num_keys * s->L * sizeof(float);
+    if (bytes > table_bytes) bytes = table_bytes;
+    const uint64_t n4 = bytes / 16;
+    if (n4 == 0) return NUPS_EINVAL;
+    cudaEvent_t a, b;
+    CK(cudaEventCreate(&a));
+    CK(cudaEventCreate(&b));
+    const unsigned grid = grid_for(n4, 256, (unsigned)s->sm_count * 8);
+    red_probe_kernel<<<grid, 256, 0, st>>>(s->val, n4);          // warm-up
+    CK(cudaEventRecord(a, st));
+    for (uint32_t r = 0; r < reps; ++r) red_probe_kernel<<<grid, 256, 0, st>>>(s->val, n4);
+    CK(cudaEventRecord(b, st));
+    s->launches += reps + 1;
+    CK(cudaEventSynchronize(b));
+    float ms = 0.f;
+    CK(cudaEventElapsedTime(&ms, a, b));
+    cudaEventDestroy(a);
+    cudaEventDestroy(b);
+    *h_gbs_out = (double)n4 * 16.0 * reps / (ms * 1e-3) / 1e9;
+    return NUPS_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
 // status and statistics
 // ---------------------------------------------------------------------------------------------
 extern "C" nups_status nups_status_check(nups_store* s, void* stream)
