@@ -186,18 +186,16 @@ def run_ours(args, rank, world, device):
     final_loss = float(loss.item())
 
     # end to end: pairs start in pinned host memory, the loss is read back every step
-    hc, ho = c.cpu().pin_memory(), o.cpu().pin_memory()
-    dc = torch.empty(BATCH, dtype=torch.int32, device=device)
-    do = torch.empty(BATCH, dtype=torch.int32, device=device)
+    # (centre and context keys of a batch sit side by side in one pinned buffer: one copy per step)
+    hpairs = torch.stack([c.view(nb, BATCH), o.view(nb, BATCH)], dim=1).cpu().pin_memory()      # [nb, 2, BATCH]
+    dpairs = torch.empty(2, BATCH, dtype=torch.int32, device=device)
     hl = torch.zeros(1, dtype=torch.float32).pin_memory()
     e2e_steps = min(args.steps, 2048)
     barrier()
     t0 = time.perf_counter()
     for i in range(e2e_steps):
-        j = (i % nb) * BATCH
-        dc.copy_(hc[j:j + BATCH], non_blocking=True)
-        do.copy_(ho[j:j + BATCH], non_blocking=True)
-        s.step_sgns(dc, do, dist, NEG, LR, loss)
+        dpairs.copy_(hpairs[i % nb], non_blocking=True)
+        s.step_sgns(dpairs[0], dpairs[1], dist, NEG, LR, loss)
         hl.copy_(loss, non_blocking=True)
         torch.cuda.current_stream().synchronize()
     barrier()

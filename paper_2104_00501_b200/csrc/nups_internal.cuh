@@ -247,6 +247,24 @@ __device__ __forceinline__ void mark_dirty(const View& v, uint32_t q, int slot)
 }
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
+// Queue a localize request (key -> worker q) of the running call.  Called by whole warps: the lanes that
+// have a request share one addition to the list's counter instead of queueing up at it one by one.
+__device__ __forceinline__ void queue_localize(const View& v, bool active, uint32_t key, uint32_t q, uint32_t* req,
+                                               uint64_t req_cap)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const unsigned m = __ballot_sync(0xFFFFFFFFu, active);
+    if (m == 0) return;
+    unsigned long long base = 0;
+    if (lane == (unsigned)(__ffs(m) - 1)) base = atomicAdd(&v.st->req_count, (unsigned long long)__popc(m));
+    base = __shfl_sync(0xFFFFFFFFu, base, __ffs(m) - 1);
+    if (active) {
+        atomicMax(v.pending + key, (int)q);
+        const unsigned long long at = base + __popc(m & ((1u << lane) - 1u));
+        if (at < req_cap) req[at] = key;
+    }
+}
+
 __device__ __forceinline__ void flag_bad_key(const View& v) { atomicCAS(&v.st->status, 0, NUPS_EKEY); }
 
 __device__ __forceinline__ void red_add_v4(float* addr, float4 x)

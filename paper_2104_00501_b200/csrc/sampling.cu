@@ -307,12 +307,8 @@ __global__ void localize_handle_kernel(View v, const uint32_t* __restrict__ keys
                                        uint64_t req_cap)
 {
     uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (o >= N) return;
-    uint32_t k = keys[o];
-    uint32_t q = chunk_of_pos(o, N, v.R);
-    atomicMax(v.pending + k, (int)q);
-    unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
-    if (at < req_cap) req[at] = k;
+    const bool in = o < N;
+    queue_localize(v, in, in ? keys[o] : 0u, in ? chunk_of_pos(o, N, v.R) : 0u, req, req_cap);
 }
 
 static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int* slot_out, cudaStream_t st)
@@ -426,11 +422,14 @@ __global__ void emit_kernel(View v, DrawParams p, HandleView h, uint64_t N, uint
 // reuse with postponing: one block walks one sub-handle.  Entries not yet postponed are taken in
 // order; a local one is emitted, a non-local one is queued for re-localization and appended to the
 // sub-handle's postponed queue; when the fresh entries run out the postponed ones are emitted.
-__global__ void __launch_bounds__(256)
+constexpr int LT_THREADS = 1024;
+constexpr int LT_ITEMS = 4;                 // consecutive list entries per thread and round
+
+__global__ void __launch_bounds__(LT_THREADS)
 longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
                 uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
 {
-    __shared__ unsigned warp_tot[8];
+    __shared__ unsigned warp_tot[LT_THREADS / 32];
     __shared__ unsigned sh_consumed, sh_local;
     const uint32_t q = q_first + blockIdx.x;
     const unsigned tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -442,43 +441,68 @@ longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, u
     uint4 stt = h.state[q];
     uint64_t oc = stt.x, ph = stt.y, pt = stt.z, emitted = 0;
     while (emitted < take && oc < size) {
-        uint64_t i = oc + tid;
-        bool have = i < size;
-        uint32_t key = have ? h.keys[b0 + i] : 0u;
-        bool loc = have && key_is_local(v, q, key);
-        unsigned bal = __ballot_sync(0xFFFFFFFFu, loc);
-        unsigned excl = __popc(bal & ((1u << lane) - 1u));
-        if (lane == 0) warp_tot[warp] = __popc(bal);
-        __syncthreads();
-        for (unsigned w = 0; w < warp; ++w) excl += warp_tot[w];
-        uint64_t need = take - emitted;
-        bool consumed = have && excl < need;
-        if (consumed) {
-            if (loc) out[out_base + emitted + excl] = key;
-            else {
-                h.post[b0 + pt + (tid - excl)] = key;
-                atomicMax(v.pending + key, (int)q);
-                unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
-                if (at < req_cap) req[at] = key;
-            }
+        // a round looks at LT_THREADS * LT_ITEMS fresh entries in list order: thread t owns entries
+        // t * LT_ITEMS .. t * LT_ITEMS + LT_ITEMS - 1 of the round
+        uint32_t key[LT_ITEMS];
+        bool have[LT_ITEMS], loc[LT_ITEMS];
+        unsigned mine = 0;
+#pragma unroll
+        for (int k = 0; k < LT_ITEMS; ++k) {
+            const uint64_t i = oc + (uint64_t)tid * LT_ITEMS + k;
+            have[k] = i < size;
+            key[k] = have[k] ? h.keys[b0 + i] : 0u;
+            loc[k] = have[k] && key_is_local(v, q, key[k]);
+            mine += loc[k] ? 1u : 0u;
         }
-        count_sample(v, key, consumed && loc);
-        unsigned cbal = __ballot_sync(0xFFFFFFFFu, consumed);
-        unsigned lbal = __ballot_sync(0xFFFFFFFFu, consumed && loc);
+        // exclusive count of local entries before this thread's first entry
+        unsigned inc = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned y = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= (unsigned)o) inc += y;
+        }
+        if (lane == 31) warp_tot[warp] = inc;
         if (tid == 0) { sh_consumed = 0; sh_local = 0; }
         __syncthreads();
-        if (lane == 0) { atomicAdd(&sh_consumed, __popc(cbal)); atomicAdd(&sh_local, __popc(lbal)); }
+        unsigned excl = inc - mine;
+        for (unsigned w = 0; w < warp; ++w) excl += warp_tot[w];
+        const uint64_t need = take - emitted;
+        unsigned nc = 0, nl = 0;
+#pragma unroll
+        for (int k = 0; k < LT_ITEMS; ++k) {
+            // the walk stops right after the need-th local entry: an entry is reached iff fewer than
+            // `need` local entries lie before it
+            const bool consumed = have[k] && excl < need;
+            if (consumed) {
+                if (loc[k]) out[out_base + emitted + excl] = key[k];
+                else {
+                    h.post[b0 + pt + ((uint64_t)tid * LT_ITEMS + k - excl)] = key[k];     // non-local entries before it
+                    atomicMax(v.pending + key[k], (int)q);
+                    const unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
+                    if (at < req_cap) req[at] = key[k];
+                }
+                nc++;
+                nl += loc[k] ? 1u : 0u;
+            }
+            count_sample(v, key[k], consumed && loc[k]);
+            excl += loc[k] ? 1u : 0u;
+        }
+        for (int o = 16; o > 0; o >>= 1) {
+            nc += __shfl_xor_sync(0xFFFFFFFFu, nc, o);
+            nl += __shfl_xor_sync(0xFFFFFFFFu, nl, o);
+        }
+        if (lane == 0) { atomicAdd(&sh_consumed, nc); atomicAdd(&sh_local, nl); }
         __syncthreads();
-        unsigned nc = sh_consumed, nl = sh_local;
-        emitted += nl; pt += nc - nl; oc += nc;
+        const unsigned tc = sh_consumed, tl = sh_local;
+        emitted += tl; pt += tc - tl; oc += tc;
         __syncthreads();
     }
     __syncthreads();
     if (emitted < take) {
-        uint64_t cnt = take - emitted;
-        for (uint64_t i = tid; i < ((cnt + 255) / 256) * 256; i += 256) {
-            bool in = i < cnt;
-            uint32_t key = in ? h.post[b0 + ph + i] : 0u;
+        const uint64_t cnt = take - emitted;
+        for (uint64_t i = tid; i < ((cnt + LT_THREADS - 1) / LT_THREADS) * LT_THREADS; i += LT_THREADS) {
+            const bool in = i < cnt;
+            const uint32_t key = in ? h.post[b0 + ph + i] : 0u;
             if (in) out[out_base + emitted + i] = key;
             count_sample(v, key, in);
         }
@@ -505,7 +529,7 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
             if (b0 <= h.cursor && h.cursor < b1) qf = q;
             if (b0 <= h.cursor + n - 1 && h.cursor + n - 1 < b1) ql = q;
         }
-        longterm_kernel<<<ql - qf + 1, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->req_keys, s->req_cap);
+        longterm_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->req_keys, s->req_cap);
         LAUNCH_CHECK(s);
         nups_status rc = nups_localize_apply(s, h.N, st);
         if (rc != NUPS_OK) return rc;
@@ -539,11 +563,7 @@ __device__ __forceinline__ void direct_tail(const View& v, uint32_t key, uint32_
                                             uint64_t req_cap)
 {
     count_sample(v, key, in);
-    if (in && localize) {
-        atomicMax(v.pending + key, (int)q);
-        unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
-        if (at < req_cap) req[at] = key;
-    }
+    if (localize) queue_localize(v, in, key, q, req, req_cap);
 }
 
 // blockIdx.y (iid) / blockIdx.z (reuse) = batch: `batches` handles of N samples each are drawn back to back,

@@ -1165,13 +1165,11 @@ __global__ void localize_request_kernel(View v, const uint32_t* __restrict__ key
                                         uint64_t req_cap)
 {
     uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= n) return;
-    uint32_t k = keys[i];
-    if (k >= v.num_keys) { flag_bad_key(v); return; }
-    uint32_t q = worker_of_item(i, n, v.R);
-    atomicMax(v.pending + k, (int)q);
-    unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
-    if (at < req_cap) req[at] = k;
+    const bool in = i < n;
+    const uint32_t k = in ? keys[i] : 0u;
+    const bool ok = in && k < v.num_keys;
+    if (in && !ok) flag_bad_key(v);
+    queue_localize(v, ok, k, ok ? worker_of_item(i, n, v.R) : 0u, req, req_cap);
 }
 
 // requests of one call are applied in the order they were made, so the last one wins; workers are
