@@ -157,7 +157,7 @@ def aggregate_throughput(units_per_rank, seconds, world):
 def run_ours(args, rank, world, device):
     from paper_2104_00501_b200 import binding
     hbm_peak, peak_kind = peaks()
-    nb = min(args.steps + args.warmup, MAX_DISTINCT_BATCHES)
+    nb = min(-(-(args.steps + args.warmup) // 64) * 64, MAX_DISTINCT_BATCHES)
     s, dist, hot, c, o, weights = build_store(binding, device, nb, seed=rank)
     loss = torch.zeros(1, dtype=torch.float32, device=device)
 
@@ -170,17 +170,31 @@ def run_ours(args, rank, world, device):
             torch.distributed.barrier()
         torch.cuda.synchronize()
 
-    for i in range(args.warmup):
-        s.step_sgns(*batch(i), dist, NEG, LR, loss)
+    # the timed loop hands the library CHUNK consecutive batches per call (nups_run_sgns): every batch is still one
+    # step of the path, but the steps between two replica merges share a kernel launch
+    CHUNK = 4 * SYNC_EVERY
+    assert nb % CHUNK == 0 or nb < CHUNK
+    losses = torch.zeros(CHUNK, dtype=torch.float32, device=device)
+
+    def run(first, count):
+        done = 0
+        while done < count:
+            j = (first + done) % nb
+            m = min(CHUNK, count - done, nb - j)
+            s.run_sgns(c[j * BATCH:(j + m) * BATCH], o[j * BATCH:(j + m) * BATCH], BATCH, dist, NEG, LR, losses[:m])
+            done += m
+        return m
+
+    run(0, args.warmup)
     launches0 = s.stats()["launches"]
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
     with ClockSampler(torch.cuda.current_device()) as clk:
         ev0.record()
-        for i in range(args.steps):
-            s.step_sgns(*batch(args.warmup + i), dist, NEG, LR, loss)
+        last = run(args.warmup, args.steps)
         ev1.record()
         barrier()
+    loss.copy_(losses[last - 1:last])
     ms = ev0.elapsed_time(ev1)
     launches = s.stats()["launches"] - launches0
     final_loss = float(loss.item())
@@ -201,25 +215,30 @@ def run_ours(args, rank, world, device):
     barrier()
     e2e_s = time.perf_counter() - t0
 
-    # roofline of the dominant kernel (the fused step kernel), timed with event pairs on its stream
-    s.kernel_timing(True)
+    # roofline of the dominant kernel (the fused step kernel) in the launch configuration that was timed above:
+    # event pairs on its stream around every launch (one launch = the steps between two replica merges)
     hot_mask = torch.zeros(2 * VOCAB, dtype=torch.bool, device=device)
-    hot_mask[hot] = True
+    if hot.numel():
+        hot_mask[hot] = True
     cold_rows = []
-    for i in range(args.steps):
+    for i in range(0, nb, max(1, nb // 16)):              # data property: distinct non-replicated rows of a batch
         bc, bo = batch(i)
         s.step_sgns(bc, bo, dist, NEG, LR, loss)
-        if i % max(1, args.steps // 16) == 0:
-            keys = torch.cat([bc.long(), bo.long(), s.last_negatives().long()])
-            uniq = torch.unique(keys)
-            cold_rows.append(int((~hot_mask[uniq]).sum()))
+        keys = torch.cat([bc.long(), bo.long(), s.last_negatives().long()])
+        cold_rows.append(int((~hot_mask[torch.unique(keys)]).sum()))
+    s.kernel_timing(True)
+    run(0, args.steps)
     k_ms, k_launches = s.kernel_time()
     s.kernel_timing(False)
+    steps_per_launch = args.steps / max(k_launches, 1)
     row_bytes = DIM * 4
     key_bytes = BATCH * 4 * (2 + NEG)
-    alg_bytes = key_bytes + 2 * row_bytes * float(np.mean(cold_rows))
-    logical_bytes = key_bytes + 2 * row_bytes * BATCH * (NEG + 2)
+    alg_bytes = (key_bytes + 2 * row_bytes * float(np.mean(cold_rows))) * steps_per_launch
+    logical_bytes = (key_bytes + 2 * row_bytes * BATCH * (NEG + 2)) * steps_per_launch
+    update_bytes = row_bytes * BATCH * (NEG + 2) * steps_per_launch
     k_s = (k_ms / 1e3) / max(k_launches, 1)
+    red_l2 = s.probe_reduction_rate(64 << 20, 20)          # update payload rate with L2-resident targets
+    red_dram = s.probe_reduction_rate(2 << 30, 5)          # ... with targets streaming from DRAM
     sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2104_00501_b200", "csrc", "steps.cu"), "rb").read()).hexdigest()
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["steps_cu_sha1"] == sha else None
 
@@ -247,8 +266,11 @@ def run_ours(args, rank, world, device):
                      "frac": alg_bytes / k_s / 1e9 / hbm_peak, "traffic": traffic,
                      "algorithmic_bytes_per_launch": alg_bytes, "logical_bytes_per_launch": logical_bytes,
                      "logical_gbs": logical_bytes / k_s / 1e9, "kernel_us": k_s * 1e6,
-                     "kernel_share_of_step": (k_ms / max(k_launches, 1)) / (ms / args.steps),
-                     "distinct_cold_rows_per_batch": float(np.mean(cold_rows))},
+                     "steps_per_launch": steps_per_launch,
+                     "kernel_share_of_step": (k_ms / args.steps) / (ms / args.steps),
+                     "distinct_cold_rows_per_batch": float(np.mean(cold_rows)),
+                     "update_payload_gbs": update_bytes / k_s / 1e9,
+                     "reduction_rate_l2_resident_gbs": red_l2, "reduction_rate_dram_gbs": red_dram},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(c, o, weights, hot, budget_s=12.0)

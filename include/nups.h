@@ -243,6 +243,17 @@ nups_status nups_pull_sample(nups_store* store, nups_handle handle, uint64_t n, 
 nups_status nups_step_sgns(nups_store* store, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_pairs,
                            int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream);
 
+/* Many skip-gram steps from one call: n_total pairs are taken as n_total / batch
+ * consecutive steps of `batch` pairs, each exactly like one nups_step_sgns
+ * (own handle of batch * K negatives, replicas merged every sync_interval
+ * steps).  d_loss_out (nullable) receives one mean loss per step.  In fast mode
+ * (and without access counting or ownership tracking) the steps between two
+ * merges share one kernel launch, so pairs of different steps of that stretch
+ * race like pairs of one step do; otherwise the steps run one after the other.
+ * n_total must be a multiple of batch.                                        */
+nups_status nups_run_sgns(nups_store* store, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_total,
+                          uint64_t batch, int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream);
+
 /* ComplEx with AdaGrad: rows are [re | im]; phi = Re sum h r conj(t); negative j
  * replaces the head when j is even, the tail when odd;
  * loss = softplus(-phi_pos) + sum_j softplus(phi_j); per key role with summed

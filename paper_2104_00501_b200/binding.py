@@ -24,7 +24,7 @@ EXPORTS = [
     "nups_create", "nups_destroy", "nups_table_ptr", "nups_table_copy", "nups_init_uniform", "nups_pull", "nups_pull2", "nups_push",
     "nups_push2", "nups_push_noalloc", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
-    "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_step_complex", "nups_step_mf",
+    "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_run_sgns", "nups_step_complex", "nups_step_mf",
     "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_probe_reduction_rate", "nups_strerror", "nups_last_cuda_error",
 ]
 
@@ -84,6 +84,7 @@ def load(build_if_missing: bool = True):
         "nups_prepare_sample": [vp, i32, u64, C.POINTER(C.c_int64), vp],
         "nups_pull_sample": [vp, C.c_int64, u64, vp, vp, vp],
         "nups_step_sgns": [vp, vp, vp, u64, i32, u32, f32, vp, vp],
+        "nups_run_sgns": [vp, vp, vp, u64, u64, i32, u32, f32, vp, vp],
         "nups_step_complex": [vp, vp, vp, vp, u64, i32, u32, f32, f32, vp, vp],
         "nups_step_mf": [vp, vp, vp, vp, u64, f32, f32, vp, vp],
         "nups_last_negatives": [vp, C.POINTER(vp), C.POINTER(u64)],
@@ -293,6 +294,11 @@ class Store:
     def step_sgns(self, center, context, dist, K, lr, loss_out=None):
         self._chk(self._l.nups_step_sgns(self._s, _ptr(center, torch.int32), _ptr(context, torch.int32),
                                          center.numel(), dist, K, lr, _ptr(loss_out), _stream()), "nups_step_sgns")
+
+    def run_sgns(self, center, context, batch, dist, K, lr, loss_out=None):
+        """center.numel() / batch consecutive steps of `batch` pairs; loss_out: one float per step."""
+        self._chk(self._l.nups_run_sgns(self._s, _ptr(center, torch.int32), _ptr(context, torch.int32), center.numel(),
+                                        batch, dist, K, lr, _ptr(loss_out), _stream()), "nups_run_sgns")
 
     def step_complex(self, h, r, t, dist, K, lr, eps, loss_out=None):
         self._chk(self._l.nups_step_complex(self._s, _ptr(h, torch.int32), _ptr(r, torch.int32), _ptr(t, torch.int32),

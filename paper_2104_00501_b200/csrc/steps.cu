@@ -72,12 +72,14 @@ __device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src
                  : "memory");
 }
 
-template <bool HOT, bool DET>
+// KT = number of negatives when it is known at compile time (loops unroll), 0 = take it from K
+template <bool HOT, bool DET, int KT>
 __global__ void __launch_bounds__(SGNS_MAX_THREADS, 8)
 sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
-            const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr,
+            const uint32_t* __restrict__ negs, uint64_t n, uint32_t K_arg, float lr,
             float* __restrict__ upd, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
-            float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
+            float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap, uint32_t group,
+            unsigned long long* __restrict__ loss_acc)
 {
     // park[2 * role][tid] = the thread's chunk of the role's stored row, park[2 * role + 1][tid] = of the
     // worker's pending replica row (only filled for replicated keys).  Roles: 0 context, 1..K negatives,
@@ -86,19 +88,24 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
     __shared__ unsigned long long s_row[32], s_pend[32];
     __shared__ float s_part[SGNS_MAX_THREADS / 32][32];
     __shared__ int s_ok;
+    const uint32_t K = KT > 0 ? (uint32_t)KT : K_arg;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
     const uint32_t L4 = v.L4, per = K + 2;
     const bool mine = tid < L4;
     const uint64_t L = (uint64_t)L4 * 4;
     double my_loss = 0.0;
-    for (uint64_t i = blockIdx.x; i < n; i += gridDim.x) {
+    // `group` consecutive steps of n pairs each may share one launch (fast mode): pair e belongs to step
+    // e / n; keys, negatives and the per-step loss sums are laid out step after step
+    for (uint64_t e = blockIdx.x; e < n * group; e += gridDim.x) {
+        const uint32_t step = group > 1 ? (uint32_t)(e / n) : 0u;
+        const uint64_t i = e - (uint64_t)step * n;
         const uint32_t q = worker_of_item(i, n, v.R);
         if (tid == 0) s_ok = 1;
         __syncthreads();
         uint32_t key = 0;
         int slot = -1;
         if (tid < per) {
-            key = tid == 0 ? context[i] : (tid <= K ? negs[i * K + tid - 1] : center[i]);
+            key = tid == 0 ? context[e] : (tid <= K ? negs[e * K + tid - 1] : center[e]);
             const bool ok = key < v.num_keys;
             if (!ok) s_ok = 0;
             slot = (HOT && ok) ? __ldg(v.slot_of + key) : -1;
@@ -123,6 +130,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
             if (v.owner && (tid == 0 || tid == K + 1)) request_localize(v, key, q, req, req_cap);
         }
         if (mine) {
+#pragma unroll
             for (uint32_t role = 0; role < per; ++role) {
                 cp_async_16(park + (2 * role) * nthr + tid, (const float4*)(v.val + s_row[role]) + tid);
                 if (HOT && s_pend[role] != NO_PEND)
@@ -139,6 +147,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         const float4 vr = mine ? parked(K + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
         // partial dot products; lane j of each warp ends up holding the warp's part of x_j
         float part = 0.f;
+#pragma unroll
         for (uint32_t j = 0; j <= K; ++j) {
             float d = 0.f;
             if (mine) {
@@ -157,6 +166,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         float loss_l = lane == 0 ? softplusf_(-x_l) : (lane <= K ? softplusf_(x_l) : 0.f);
         loss_l = warp_sum(loss_l);
         float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
         for (uint32_t j = 0; j <= K; ++j) {
             const float g = __shfl_sync(0xFFFFFFFFu, g_l, j);
             if (!mine) continue;
@@ -174,10 +184,11 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         }
         if (tid == 0) {
             if (DET) loss_item[i] = loss_l;
-            my_loss += (double)loss_l;
+            if (loss_acc) atomicAdd(loss_acc + step, (unsigned long long)llrintf(fminf(loss_l, 60000.f) * 65536.f));
+            else my_loss += (double)loss_l;
         }
     }
-    if (!DET) loss_finish(v, my_loss, n, loss_out);
+    if (!DET && !loss_acc) loss_finish(v, my_loss, n, loss_out);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -621,20 +632,12 @@ static unsigned step_grid(const nups_store* s, uint64_t n, unsigned blocks_per_s
         }                                                                                    \
     } while (0)
 
-extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n,
-                                      int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream)
+// launch of the fused skip-gram kernel over `group` consecutive steps of n pairs (group > 1: fast mode only;
+// the negatives of all those steps lie back to back at s->last_negs, per-step losses go to loss_acc)
+static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n, uint32_t K,
+                               float lr, const StepBuffers& b, float* d_loss_out, uint32_t group,
+                               unsigned long long* loss_acc, cudaStream_t st)
 {
-    if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
-    if (K > 30) return NUPS_EINVAL;                         // one lane per key of an item
-    if (s->L / 4 > SGNS_MAX_THREADS) return NUPS_EINVAL;    // one thread per float4 chunk of a row: at most 512 floats
-    cudaStream_t st = (cudaStream_t)stream;
-    nups_status rc = nups_draw_negatives(s, dist, n * K, st);
-    if (rc != NUPS_OK) return rc;
-    rc = nups_req_reserve(s, n * 2);
-    if (rc != NUPS_OK) return rc;
-    StepBuffers b;
-    rc = step_buffers(s, n, K + 2, false, &b);
-    if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
     const unsigned threads = ((v.L4 + 31) / 32) * 32;           // one thread per float4 chunk of a row
     const size_t smem = (size_t)2 * (K + 2) * threads * sizeof(float4);
@@ -645,26 +648,117 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
     if (per_sm > NUPS_SGNS_PER_SM) per_sm = NUPS_SGNS_PER_SM;
     if (per_sm > 2048 / threads) per_sm = 2048 / threads;
     if (per_sm < 1) return NUPS_EINVAL;
-    const uint64_t want = n < (uint64_t)s->sm_count * per_sm ? n : (uint64_t)s->sm_count * per_sm;
+    const uint64_t items = n * group;
+    const uint64_t want = items < (uint64_t)s->sm_count * per_sm ? items : (uint64_t)s->sm_count * per_sm;
     const unsigned grid = (unsigned)want;
     static bool attr_set[2][2] = {{false, false}, {false, false}};
     const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0;
     if (smem > 48 * 1024 && !attr_set[hi][di]) {
         cudaError_t e;
-        if (hi && di) e = cudaFuncSetAttribute(sgns_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else if (hi) e = cudaFuncSetAttribute(sgns_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else if (di) e = cudaFuncSetAttribute(sgns_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else e = cudaFuncSetAttribute(sgns_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        if (hi && di) e = cudaFuncSetAttribute(sgns_kernel<true, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else if (hi) e = cudaFuncSetAttribute(sgns_kernel<true, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else if (di) e = cudaFuncSetAttribute(sgns_kernel<false, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
+        else e = cudaFuncSetAttribute(sgns_kernel<false, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
         if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
         attr_set[hi][di] = true;
     }
     nups_time_begin(s, st);
-    DISPATCH_MODE(s, sgns_kernel<HOT, DET><<<grid, threads, smem, st>>>(
-        v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys,
-        s->req_cap));
+    if (K == 3) {
+        DISPATCH_MODE(s, sgns_kernel<HOT, DET, 3><<<grid, threads, smem, st>>>(
+            v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap,
+            group, loss_acc));
+    } else {
+        DISPATCH_MODE(s, sgns_kernel<HOT, DET, 0><<<grid, threads, smem, st>>>(
+            v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap,
+            group, loss_acc));
+    }
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+static nups_status sgns_check(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n, uint32_t K)
+{
+    if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
+    if (K > 30) return NUPS_EINVAL;                         // one lane per key of an item
+    if (s->L / 4 > SGNS_MAX_THREADS) return NUPS_EINVAL;    // one thread per float4 chunk of a row: at most 512 floats
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n,
+                                      int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream)
+{
+    nups_status rc = sgns_check(s, d_center, d_context, n, K);
+    if (rc != NUPS_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    rc = nups_draw_negatives(s, dist, n * K, st);
+    if (rc != NUPS_OK) return rc;
+    rc = nups_req_reserve(s, n * 2);
+    if (rc != NUPS_OK) return rc;
+    StepBuffers b;
+    rc = step_buffers(s, n, K + 2, false, &b);
+    if (rc != NUPS_OK) return rc;
+    rc = sgns_launch(s, d_center, d_context, n, K, lr, b, d_loss_out, 1, nullptr, st);
+    if (rc != NUPS_OK) return rc;
     return step_finish(s, n, K + 2, 2, b, d_loss_out, st, !s->cfg.deterministic);
+}
+
+// per-step losses of a grouped launch: fixed-point sums -> means, and the sums are cleared for the next group
+__global__ void loss_group_kernel(unsigned long long* acc, uint32_t group, uint64_t n, float* loss_out)
+{
+    const uint32_t g = threadIdx.x;
+    if (g >= group) return;
+    if (loss_out) loss_out[g] = (float)((double)acc[g] / 65536.0 / (double)n);
+    acc[g] = 0ull;
+}
+
+extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_total,
+                                     uint64_t batch, int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream)
+{
+    if (batch == 0 || n_total == 0 || n_total % batch) return NUPS_EINVAL;
+    nups_status rc = sgns_check(s, d_center, d_context, batch, K);
+    if (rc != NUPS_OK) return rc;
+    const uint64_t steps = n_total / batch;
+    // where a step has side effects that must happen in step order (ordered pushes, access counts,
+    // ownership changes), the steps are simply taken one by one
+    if (s->cfg.deterministic || s->cfg.count_accesses || s->owner) {
+        for (uint64_t t = 0; t < steps; ++t) {
+            rc = nups_step_sgns(s, d_center + t * batch, d_context + t * batch, batch, dist, K, lr,
+                                d_loss_out ? d_loss_out + t : nullptr, stream);
+            if (rc != NUPS_OK) return rc;
+        }
+        return NUPS_OK;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long* acc = (unsigned long long*)s->loss_partial;      // zero between launches
+    StepBuffers b;
+    b.loss_item = nullptr; b.ukeys = nullptr; b.uval = nullptr; b.uacc = nullptr; b.push_scratch = nullptr;
+    uint64_t t = 0;
+    while (t < steps) {
+        // one launch covers the steps up to the next replica merge, as far as their negatives are drawn already
+        rc = nups_draw_negatives(s, dist, batch * K, st);                 // this step's negatives (may draw ahead)
+        if (rc != NUPS_OK) return rc;
+        uint64_t group = 1;
+        if (s->ahead_dist == dist && s->ahead_N == batch * K) group += s->ahead_total - s->ahead_next;
+        if (group > steps - t) group = steps - t;
+        if (s->cfg.sync_interval) {
+            const uint64_t to_sync = s->cfg.sync_interval - s->steps % s->cfg.sync_interval;
+            if (group > to_sync) group = to_sync;
+        }
+        if (group > 1024) group = 1024;
+        if (group > 1) s->ahead_next += (uint32_t)(group - 1);            // those batches are handed out now
+        rc = sgns_launch(s, d_center + t * batch, d_context + t * batch, batch, K, lr, b, nullptr, (uint32_t)group, acc, st);
+        if (rc != NUPS_OK) return rc;
+        loss_group_kernel<<<1, 1024, 0, st>>>(acc, (uint32_t)group, batch, d_loss_out ? d_loss_out + t : nullptr);
+        LAUNCH_CHECK(s);
+        s->steps += group;
+        t += group;
+        if (s->cfg.sync_interval && s->steps % s->cfg.sync_interval == 0) {
+            rc = nups_sync_internal(s, st);
+            if (rc != NUPS_OK) return rc;
+        }
+    }
+    return NUPS_OK;
 }
 
 extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, const uint32_t* d_r, const uint32_t* d_t,

@@ -175,6 +175,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     cudaMemset(s->hot_bits, 0, ((num_keys + 31) / 32) * 4);
     cudaMemset(s->cnt, 0, num_keys * 8);
     cudaMemset(s->st, 0, sizeof(DevStat));
+    cudaMemset(s->loss_partial, 0, 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double));
     fill_i32<<<grid_for(num_keys, 256, 4096), 256>>>(s->slot_of, num_keys, -1);
     if (s->owner) {
         cudaMemset(s->owner, NUPS_OWNER_DEFAULT, num_keys);

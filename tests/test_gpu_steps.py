@@ -210,3 +210,40 @@ def test_sample_ahead_keeps_the_sample_sequences(level):
         assert np.array_equal(host_keys(s.last_negatives()), negs)
         at += n
     assert s.status_check() == 0
+
+
+def test_run_sgns_matches_step_by_step():
+    # deterministic mode: nups_run_sgns is the step loop, exactly; fast mode: steps between two merges share a
+    # launch, negatives and merge cadence stay the same and the loss tracks the oracle's within 1 %
+    V, L, K, R, B = 600, 32, 3, 4, 128
+    c, ctx, w = sgns_data(V, 2000, 7)
+    steps = 40
+    c, ctx = c[:steps * B], ctx[:steps * B]
+    init = inputs.normal_init(2 * V, L, 0.1, 7)
+    o, s = make_pair(2 * V, L, R=R, init=init, deterministic=True, sync_interval=3)
+    do = o.register_distribution(V, w, V, BOUNDED, U=4, G=30, seed=2)
+    ds = s.register_distribution(V, dev_keys(w), V, BOUNDED, U=4, G=30, seed=2)
+    lo = [o.step_sgns(c[t * B:(t + 1) * B], ctx[t * B:(t + 1) * B], do, K, 0.02) for t in range(steps)]
+    lb = torch.zeros(steps, device="cuda")
+    s.run_sgns(dev_keys(c), dev_keys(ctx), B, ds, K, 0.02, lb)
+    np.testing.assert_allclose(lb.cpu().numpy(), np.array(lo, np.float32), rtol=1e-5)
+    o.sync()
+    s.sync()
+    tables_close(o, s)
+    assert s.stats()["steps"] == steps and s.stats()["syncs"] == o.stats()["syncs"]
+
+    _, f = make_pair(2 * V, L, R=R, init=init, deterministic=False, sync_interval=3)
+    hot = np.unique(c)[:30].astype(np.uint32)
+    f.set_management(dev_keys(hot), REPLICATE)
+    df = f.register_distribution(V, dev_keys(w), V, BOUNDED, U=4, G=30, seed=2)
+    lf = torch.zeros(steps, device="cuda")
+    f.run_sgns(dev_keys(c[:17 * B]), dev_keys(ctx[:17 * B]), B, df, K, 0.02, lf[:17])      # ragged split of the run
+    f.run_sgns(dev_keys(c[17 * B:]), dev_keys(ctx[17 * B:]), B, df, K, 0.02, lf[17:])
+    lf = lf.cpu().numpy()
+    assert np.all(np.isfinite(lf)) and abs(lf[-10:].mean() - np.mean(lo[-10:])) <= 0.01 * np.mean(lo[-10:])
+    assert f.stats()["steps"] == steps and f.stats()["syncs"] == steps // 3
+    # the negatives handed to the last step of the run are the oracle's
+    ko = o.pull_sample(o.prepare_sample(do, 50), 50, values=False)
+    kf = f.pull_sample(f.prepare_sample(df, 50), 50, values=False)
+    assert np.array_equal(host_keys(kf), ko)
+    assert f.status_check() == 0
