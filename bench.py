@@ -207,11 +207,24 @@ def run_ours(args, rank, world, device):
     e2e_steps = min(args.steps, 2048)
     barrier()
     t0 = time.perf_counter()
+    # two buffers in flight: the host waits for step k-1's loss to have landed before it issues step k+1
+    dpairs2 = [dpairs, torch.empty_like(dpairs)]
+    hl2 = [hl, torch.zeros(1, dtype=torch.float32).pin_memory()]
+    dl2 = [torch.zeros(1, device=device), torch.zeros(1, device=device)]
+    done = [torch.cuda.Event(), torch.cuda.Event()]
+    seen = 0.0
     for i in range(e2e_steps):
-        dpairs.copy_(hpairs[i % nb], non_blocking=True)
-        s.step_sgns(dpairs[0], dpairs[1], dist, NEG, LR, loss)
-        hl.copy_(loss, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        k = i & 1
+        if i >= 2:
+            done[k].synchronize()
+            seen += float(hl2[k][0])                      # the host really reads every step's loss
+        dpairs2[k].copy_(hpairs[i % nb], non_blocking=True)
+        s.step_sgns(dpairs2[k][0], dpairs2[k][1], dist, NEG, LR, dl2[k])
+        hl2[k].copy_(dl2[k], non_blocking=True)
+        done[k].record()
+    for k in range(2):
+        done[k].synchronize()
+        seen += float(hl2[k][0])
     barrier()
     e2e_s = time.perf_counter() - t0
 
@@ -396,8 +409,24 @@ def run_ps_sweep(args, device):
                 alg = 4 * N + row * N + (1 if op == "pull" else 2) * row * ucold
                 res[op] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
                            "frac": alg / t / 1e9 / hbm_peak, "logical_gbs": (4 * N + (2 if op == "pull" else 3) * row * N) / t / 1e9}
+            # replica merge cost: pushes with a merge every `interval` pushes, time per push including its share
+            sync_sweep = {}
+            if topk:
+                s.kernel_timing(False)
+                for interval in (1, 16, 256):
+                    n_push = max(interval, 32)
+                    state = {"i": 0}
+
+                    def push_and_merge():
+                        for _ in range(n_push):
+                            s.push(batches[state["i"] % 4], delta)
+                            state["i"] += 1
+                            if state["i"] % interval == 0:
+                                s.sync()
+                    sync_sweep[str(interval)] = _time_calls(push_and_merge, 2, warm=1) / n_push * 1e6
             line = {"workload": "ps microbenchmark", "keys": NK, "value_len": L, "batch": N, "zipf_s": skew, "topk": topk,
-                    "distinct_cold_rows": ucold, "peak": hbm_peak, "peak_kind": peak_kind, **res}
+                    "distinct_cold_rows": ucold, "peak": hbm_peak, "peak_kind": peak_kind,
+                    "push_us_incl_merge_every": sync_sweep, **res}
             print(json.dumps(line), flush=True)
             lines.append(line)
             s.close()
