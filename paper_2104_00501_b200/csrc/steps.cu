@@ -57,134 +57,171 @@ __device__ __forceinline__ void loss_finish(const View& v, double warp_loss, uin
 }
 
 // ---------------------------------------------------------------------------------------------
-// skip-gram with negative sampling.  One block works on one pair at a time; thread c owns float4 chunk c
-// of every row (blockDim = row width in float4 rounded up to whole warps, at most 128).  The 2 + K rows
-// of the pair - and the worker's pending replica rows of the replicated ones - are brought into shared
-// memory by asynchronous 16-byte copies, all in flight at once, each thread its own column; the 1 + K
-// dot products are reduced across the block once; then every thread forms and pushes its chunk of the
-// updates.
+// skip-gram with negative sampling.  One warp works on one pair at a time: lane l owns the float4 chunks
+// l, l + 32, ... of every row (CH of them, a compile-time count, so that every shared-memory and row offset
+// is an immediate).  The 2 + K stored rows of the pair are brought into shared memory by asynchronous
+// 16-byte copies, all in flight at once, each lane its own column; the worker's pending replica rows of
+// the replicated roles are then folded into the staged rows, so that both passes read each chunk with one
+// load; the 1 + K dot products take one warp reduction each; then every lane forms and pushes its chunks
+// of the updates.  Nothing is shared between the warps of a block.
 // ---------------------------------------------------------------------------------------------
-constexpr int SGNS_MAX_THREADS = 128;
+constexpr int SGNS_MAX_CHUNKS = 128;                               // float4 chunks of a row: at most 512 floats
+// A launch over several steps adds each pair's loss (fixed point) to one of LOSS_SLOTS words of its step:
+// additions to one word would queue up behind one another.
+constexpr uint32_t LOSS_SLOTS = 32;
+constexpr uint32_t LOSS_STEPS = 1024;                             // most steps one launch may cover; word = [slot][step]
+static_assert(LOSS_SLOTS * LOSS_STEPS <= 4 * NUPS_MAX_STEP_BLOCKS, "the per-step loss words live in the loss_partial buffer");
 
-__device__ __forceinline__ void cp_async_16(void* smem_dst, const void* gmem_src)
+constexpr int SGNS_WARPS = 2;                                      // warps (= pairs in flight) per block
+
+// asynchronous 16-byte copy to the shared-memory address (32-bit, shared window) smem_dst
+__device__ __forceinline__ void cp_async_16s(uint32_t smem_dst, const void* gmem_src)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
-                 : "memory");
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 
-// KT = number of negatives when it is known at compile time (loops unroll), 0 = take it from K
-template <bool HOT, bool DET, int KT>
-__global__ void __launch_bounds__(SGNS_MAX_THREADS, 8)
+template <bool HOT, bool DET, int KT, int CH>
+__global__ void __launch_bounds__(32 * SGNS_WARPS)
 sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
             const uint32_t* __restrict__ negs, uint64_t n, uint32_t K_arg, float lr,
             float* __restrict__ upd, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
             float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap, uint32_t group,
             unsigned long long* __restrict__ loss_acc)
 {
-    // park[2 * role][tid] = the thread's chunk of the role's stored row, park[2 * role + 1][tid] = of the
-    // worker's pending replica row (only filled for replicated keys).  Roles: 0 context, 1..K negatives,
-    // K + 1 centre.
-    extern __shared__ __align__(16) float4 park[];
-    __shared__ unsigned long long s_row[32], s_pend[32];
-    __shared__ float s_part[SGNS_MAX_THREADS / 32][32];
-    __shared__ int s_ok;
+    extern __shared__ __align__(16) float4 park_all[];
+    __shared__ const float4* s_src[SGNS_WARPS][32];                // the role's stored row
+    __shared__ float* s_dst[SGNS_WARPS][32];                       // where its update goes: replica row or stored row
+    __shared__ float s_g[SGNS_WARPS][32];                          // d(loss)/d(score) of the role
+    constexpr uint32_t cols = 32 * CH;
+    constexpr uint32_t NR = KT > 0 ? KT + 2 : 1;                   // roles kept in registers when K is fixed
     const uint32_t K = KT > 0 ? (uint32_t)KT : K_arg;
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nthr = blockDim.x;
-    const uint32_t L4 = v.L4, per = K + 2;
-    const bool mine = tid < L4;
+    const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5, per = K + 2;
+    const uint32_t L4 = v.L4;
     const uint64_t L = (uint64_t)L4 * 4;
+    float4* park = park_all + (size_t)wib * per * cols + lane;          // the lane's column
+    const uint32_t park_s = (uint32_t)__cvta_generic_to_shared(park);
+    const uint64_t nwarps = (uint64_t)gridDim.x * SGNS_WARPS, total = n * group;
+    const uint64_t w0 = (uint64_t)blockIdx.x * SGNS_WARPS + wib;
     double my_loss = 0.0;
-    // `group` consecutive steps of n pairs each may share one launch (fast mode): pair e belongs to step
-    // e / n; keys, negatives and the per-step loss sums are laid out step after step
-    for (uint64_t e = blockIdx.x; e < n * group; e += gridDim.x) {
-        const uint32_t step = group > 1 ? (uint32_t)(e / n) : 0u;
-        const uint64_t i = e - (uint64_t)step * n;
+    auto key_of = [&](uint64_t e) -> uint32_t {
+        if (lane >= per || e >= total) return 0u;
+        return lane == 0 ? context[e] : (lane <= K ? negs[e * K + lane - 1] : center[e]);
+    };
+    auto slot_of = [&](uint32_t key) -> int {
+        return (HOT && lane < per && key < v.num_keys) ? __ldg(v.slot_of + key) : -1;
+    };
+    // the lookups run two pairs ahead of the work, so that neither the key nor the slot load is waited for
+    uint32_t key1 = key_of(w0), key2 = key_of(w0 + nwarps);
+    int slot1 = slot_of(key1);
+    uint32_t step = (uint32_t)(w0 / n);
+    uint64_t i = w0 - (uint64_t)step * n;
+    for (uint64_t e = w0; e < total; e += nwarps, i += nwarps) {
+        while (i >= n) { i -= n; ++step; }
         const uint32_t q = worker_of_item(i, n, v.R);
-        if (tid == 0) s_ok = 1;
-        __syncthreads();
-        uint32_t key = 0;
-        int slot = -1;
-        if (tid < per) {
-            key = tid == 0 ? context[e] : (tid <= K ? negs[e * K + tid - 1] : center[e]);
-            const bool ok = key < v.num_keys;
-            if (!ok) s_ok = 0;
-            slot = (HOT && ok) ? __ldg(v.slot_of + key) : -1;
-            if (slot < 0) slot = -1;
-            s_row[tid] = (unsigned long long)key * L;
-            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : NO_PEND;
-        }
-        __syncthreads();
-        if (!s_ok) {                                               // a key out of range: the whole item is skipped
-            if (DET && tid < per) ukeys[i * per + tid] = NUPS_INVALID_KEY;
-            if (tid == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+        const uint32_t key = key1;
+        const int slot = slot1;
+        key1 = key2;
+        slot1 = slot_of(key2);
+        key2 = key_of(e + 2 * nwarps);
+        const bool ok = lane >= per || key < v.num_keys;
+        if (!__all_sync(0xFFFFFFFFu, ok)) {                        // a key out of range: the whole item is skipped
+            if (DET && lane < per) ukeys[i * per + lane] = NUPS_INVALID_KEY;
+            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
-        if (tid < per) {
-            if (DET) ukeys[i * per + tid] = key;
+        const uint32_t mask = HOT ? __ballot_sync(0xFFFFFFFFu, slot >= 0) : 0u;
+        __syncwarp();                                              // the previous pair's readers are done
+        if (lane < per) {
+            float* row = v.val + (unsigned long long)key * L;
+            s_src[wib][lane] = (const float4*)row;
+            s_dst[wib][lane] = slot >= 0 ? v.dval + ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : row;
+        }
+        __syncwarp();
+        float* dstp[NR];                                           // the lane's first chunk of each destination row
+#pragma unroll
+        for (uint32_t role = 0; role < per; ++role) {
+            const float4* src = s_src[wib][role] + lane;
+            float* dst = s_dst[wib][role] + 4 * lane;
+            if (KT > 0) dstp[KT > 0 ? role : 0] = dst;
+#pragma unroll
+            for (int m = 0; m < CH; ++m)
+                if (lane + 32 * m < L4) cp_async_16s(park_s + (role * cols + 32 * m) * 16, src + 32 * m);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        if (lane < per) {
+            if (DET) ukeys[i * per + lane] = key;
             if (!DET && slot >= 0) mark_dirty(v, q, slot);
             if (v.count) {
                 // context and centre: pulled (+ pushed in fast mode); negatives: pushed (their draw counted the sample)
-                const unsigned times = (tid == 0 || tid == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
+                const unsigned times = (lane == 0 || lane == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
                 if (times) note_access(v, key, slot, times);
             }
-            if (v.owner && (tid == 0 || tid == K + 1)) request_localize(v, key, q, req, req_cap);
+            if (v.owner && (lane == 0 || lane == K + 1)) request_localize(v, key, q, req, req_cap);
         }
-        if (mine) {
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        // fold the worker's pending replica rows (read straight from the slab) into the staged rows
+        if (HOT && mask) {
 #pragma unroll
             for (uint32_t role = 0; role < per; ++role) {
-                cp_async_16(park + (2 * role) * nthr + tid, (const float4*)(v.val + s_row[role]) + tid);
-                if (HOT && s_pend[role] != NO_PEND)
-                    cp_async_16(park + (2 * role + 1) * nthr + tid, (const float4*)(v.dval + s_pend[role]) + tid);
+                if (!(mask >> role & 1u)) continue;
+                const float4* pnd = (const float4*)(KT > 0 ? dstp[KT > 0 ? role : 0] : s_dst[wib][role] + 4 * lane);
+#pragma unroll
+                for (int m = 0; m < CH; ++m)
+                    if (lane + 32 * m < L4) park[role * cols + 32 * m] = add4(park[role * cols + 32 * m], __ldg(pnd + 32 * m));
             }
-            asm volatile("cp.async.commit_group;" ::: "memory");
         }
-        if (mine) asm volatile("cp.async.wait_group 0;" ::: "memory");
-        auto parked = [&](uint32_t role) -> float4 {
-            float4 x = park[(2 * role) * nthr + tid];
-            if (HOT && s_pend[role] != NO_PEND) x = add4(x, park[(2 * role + 1) * nthr + tid]);
-            return x;
-        };
-        const float4 vr = mine ? parked(K + 1) : make_float4(0.f, 0.f, 0.f, 0.f);
-        // partial dot products; lane j of each warp ends up holding the warp's part of x_j
-        float part = 0.f;
+        // lane j ends up holding the score x_j of role j <= K
+        float4 a[CH];
+#pragma unroll
+        for (int m = 0; m < CH; ++m)
+            a[m] = lane + 32 * m < L4 ? park[(K + 1) * cols + 32 * m] : make_float4(0.f, 0.f, 0.f, 0.f);
+        float x_l = 0.f;
 #pragma unroll
         for (uint32_t j = 0; j <= K; ++j) {
             float d = 0.f;
-            if (mine) {
-                const float4 u = parked(j);
-                d = vr.x * u.x + vr.y * u.y + vr.z * u.z + vr.w * u.w;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                if (lane + 32 * m < L4) {
+                    const float4 u = park[j * cols + 32 * m];
+                    d += a[m].x * u.x + a[m].y * u.y + a[m].z * u.z + a[m].w * u.w;
+                }
             }
             d = warp_sum(d);
-            if (lane == j) part = d;
+            if (lane == j) x_l = d;
         }
-        s_part[warp][lane] = part;
-        __syncthreads();
-        float x_l = 0.f;
-        for (uint32_t w = 0; w < (nthr >> 5); ++w) x_l += s_part[w][lane];
         x_l = clamp30(x_l);
         const float g_l = sigmoidf_(x_l) - (lane == 0 ? 1.f : 0.f);
+        float gk[NR];
+        if (KT > 0) {
+#pragma unroll
+            for (int j = 0; j <= KT; ++j) gk[j] = __shfl_sync(0xFFFFFFFFu, g_l, j);
+        } else {
+            s_g[wib][lane] = g_l;
+        }
         float loss_l = lane == 0 ? softplusf_(-x_l) : (lane <= K ? softplusf_(x_l) : 0.f);
         loss_l = warp_sum(loss_l);
-        float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncwarp();
 #pragma unroll
-        for (uint32_t j = 0; j <= K; ++j) {
-            const float g = __shfl_sync(0xFFFFFFFFu, g_l, j);
-            if (!mine) continue;
-            const float4 u = parked(j);
-            const float sc = -lr * g;
-            const float4 du = make_float4(sc * vr.x, sc * vr.y, sc * vr.z, sc * vr.w);
-            if (DET) ((float4*)(upd + (i * per + j) * L))[tid] = du;
-            else red_add_v4((s_pend[j] != NO_PEND ? v.dval + s_pend[j] : v.val + s_row[j]) + 4 * tid, du);
-            gv.x += g * u.x; gv.y += g * u.y; gv.z += g * u.z; gv.w += g * u.w;
-        }
-        if (mine) {
+        for (int m = 0; m < CH; ++m) {
+            if (lane + 32 * m >= L4) continue;
+            float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (uint32_t j = 0; j <= K; ++j) {
+                const float g = KT > 0 ? gk[KT > 0 ? j : 0] : s_g[wib][j];
+                const float4 u = park[j * cols + 32 * m];
+                const float sc = -lr * g;
+                const float4 du = make_float4(sc * a[m].x, sc * a[m].y, sc * a[m].z, sc * a[m].w);
+                if (DET) ((float4*)(upd + (i * per + j) * L))[lane + 32 * m] = du;
+                else red_add_v4((KT > 0 ? dstp[KT > 0 ? j : 0] : s_dst[wib][j] + 4 * lane) + 128 * m, du);
+                gv.x += g * u.x; gv.y += g * u.y; gv.z += g * u.z; gv.w += g * u.w;
+            }
             const float4 dv = make_float4(-lr * gv.x, -lr * gv.y, -lr * gv.z, -lr * gv.w);
-            if (DET) ((float4*)(upd + (i * per + K + 1) * L))[tid] = dv;
-            else red_add_v4((s_pend[K + 1] != NO_PEND ? v.dval + s_pend[K + 1] : v.val + s_row[K + 1]) + 4 * tid, dv);
+            if (DET) ((float4*)(upd + (i * per + K + 1) * L))[lane + 32 * m] = dv;
+            else red_add_v4((KT > 0 ? dstp[KT > 0 ? KT + 1 : 0] : s_dst[wib][K + 1] + 4 * lane) + 128 * m, dv);
         }
-        if (tid == 0) {
+        if (lane == 0) {
             if (DET) loss_item[i] = loss_l;
-            if (loss_acc) atomicAdd(loss_acc + step, (unsigned long long)llrintf(fminf(loss_l, 60000.f) * 65536.f));
+            if (loss_acc) atomicAdd(loss_acc + (uint32_t)(w0 % LOSS_SLOTS) * LOSS_STEPS + step, (unsigned long long)llrintf(fminf(loss_l, 60000.f) * 65536.f));
             else my_loss += (double)loss_l;
         }
     }
@@ -639,40 +676,35 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
                                unsigned long long* loss_acc, cudaStream_t st)
 {
     View v = nups_view(s);
-    const unsigned threads = ((v.L4 + 31) / 32) * 32;           // one thread per float4 chunk of a row
-    const size_t smem = (size_t)2 * (K + 2) * threads * sizeof(float4);
-    unsigned per_sm = (unsigned)(((size_t)s->max_smem - 1024) / (smem + 2048));
-#ifndef NUPS_SGNS_PER_SM
-#define NUPS_SGNS_PER_SM 12
-#endif
-    if (per_sm > NUPS_SGNS_PER_SM) per_sm = NUPS_SGNS_PER_SM;
-    if (per_sm > 2048 / threads) per_sm = 2048 / threads;
-    if (per_sm < 1) return NUPS_EINVAL;
+    const uint32_t cols = ((v.L4 + 31) / 32) * 32, per = K + 2;    // a warp's staging area: per rows of cols chunks
+    const size_t smem = (size_t)per * cols * sizeof(float4) * SGNS_WARPS;
+    if (smem > (size_t)s->max_smem - 4096) return NUPS_EINVAL;
+    // as many blocks as fit a multiprocessor's shared memory (each also holds about 2.5 KB besides its rows)
+    unsigned per_sm = (unsigned)(((size_t)228 * 1024) / (smem + 2560));
+    if (per_sm > 32) per_sm = 32;
+    if (per_sm < 1) per_sm = 1;
     const uint64_t items = n * group;
-    const uint64_t want = items < (uint64_t)s->sm_count * per_sm ? items : (uint64_t)s->sm_count * per_sm;
-    const unsigned grid = (unsigned)want;
-    static bool attr_set[2][2] = {{false, false}, {false, false}};
-    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0;
-    if (smem > 48 * 1024 && !attr_set[hi][di]) {
-        cudaError_t e;
-        if (hi && di) e = cudaFuncSetAttribute(sgns_kernel<true, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else if (hi) e = cudaFuncSetAttribute(sgns_kernel<true, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else if (di) e = cudaFuncSetAttribute(sgns_kernel<false, true, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else e = cudaFuncSetAttribute(sgns_kernel<false, false, 0>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
-        attr_set[hi][di] = true;
-    }
-    nups_time_begin(s, st);
-    if (K == 3) {
-        DISPATCH_MODE(s, sgns_kernel<HOT, DET, 3><<<grid, threads, smem, st>>>(
-            v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap,
-            group, loss_acc));
-    } else {
-        DISPATCH_MODE(s, sgns_kernel<HOT, DET, 0><<<grid, threads, smem, st>>>(
-            v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap,
-            group, loss_acc));
-    }
-    nups_time_end(s, st);
+    const uint64_t blocks_needed = (items + SGNS_WARPS - 1) / SGNS_WARPS;
+    const uint64_t cap = (uint64_t)s->sm_count * per_sm;
+    const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
+    cudaError_t e = cudaSuccess;
+#define NUPS_SGNS_GO(KT_)                                                                                              \
+    DISPATCH_CH(v.L4, DISPATCH_MODE(s, {                                                                               \
+        auto kern = sgns_kernel<HOT, DET, KT_, CH>;                                                               \
+        if (smem > 48 * 1024)                                                                                          \
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);           \
+        if (e == cudaSuccess) {                                                                                        \
+            nups_time_begin(s, st);                                                                                    \
+            kern<<<grid, 32 * SGNS_WARPS, smem, st>>>(v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
+                                                      b.loss_item, d_loss_out, s->req_keys, s->req_cap, group,        \
+                                                      loss_acc);                                                       \
+            nups_time_end(s, st);                                                                                      \
+        }                                                                                                              \
+    }))
+    if (K == 3) NUPS_SGNS_GO(3);
+    else NUPS_SGNS_GO(0);
+#undef NUPS_SGNS_GO
+    if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
     LAUNCH_CHECK(s);
     return NUPS_OK;
 }
@@ -681,7 +713,7 @@ static nups_status sgns_check(nups_store* s, const uint32_t* d_center, const uin
 {
     if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
     if (K > 30) return NUPS_EINVAL;                         // one lane per key of an item
-    if (s->L / 4 > SGNS_MAX_THREADS) return NUPS_EINVAL;    // one thread per float4 chunk of a row: at most 512 floats
+    if (s->L / 4 > SGNS_MAX_CHUNKS) return NUPS_EINVAL;     // four float4 chunks of a row per lane: at most 512 floats
     return NUPS_OK;
 }
 
@@ -708,8 +740,9 @@ __global__ void loss_group_kernel(unsigned long long* acc, uint32_t group, uint6
 {
     const uint32_t g = threadIdx.x;
     if (g >= group) return;
-    if (loss_out) loss_out[g] = (float)((double)acc[g] / 65536.0 / (double)n);
-    acc[g] = 0ull;
+    unsigned long long sum = 0;
+    for (uint32_t k = 0; k < LOSS_SLOTS; ++k) { sum += acc[k * LOSS_STEPS + g]; acc[k * LOSS_STEPS + g] = 0ull; }
+    if (loss_out) loss_out[g] = (float)((double)sum / 65536.0 / (double)n);
 }
 
 extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_total,
@@ -745,11 +778,11 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
             const uint64_t to_sync = s->cfg.sync_interval - s->steps % s->cfg.sync_interval;
             if (group > to_sync) group = to_sync;
         }
-        if (group > 1024) group = 1024;
+        if (group > LOSS_STEPS) group = LOSS_STEPS;
         if (group > 1) s->ahead_next += (uint32_t)(group - 1);            // those batches are handed out now
         rc = sgns_launch(s, d_center + t * batch, d_context + t * batch, batch, K, lr, b, nullptr, (uint32_t)group, acc, st);
         if (rc != NUPS_OK) return rc;
-        loss_group_kernel<<<1, 1024, 0, st>>>(acc, (uint32_t)group, batch, d_loss_out ? d_loss_out + t : nullptr);
+        loss_group_kernel<<<1, LOSS_STEPS, 0, st>>>(acc, (uint32_t)group, batch, d_loss_out ? d_loss_out + t : nullptr);
         LAUNCH_CHECK(s);
         s->steps += group;
         t += group;
