@@ -25,7 +25,7 @@ struct DevStat {
     int pad;
     unsigned long long hot_hits;       // accesses served by a replica
     unsigned long long cold_hits;      // accesses served in place
-    unsigned long long req_count;      // localize requests queued by the running call
+    unsigned long long unused0;
     unsigned long long tmp[4];
 };
 
@@ -39,8 +39,7 @@ struct View {
     const int32_t* slot_of;    // key -> hot slot (>= 0) or negative
     uint32_t* dirty;           // [R][Hcap] worker's replica of the slot touched since last sync
     unsigned long long* cnt;   // [num_keys] access counts
-    uint8_t* owner;            // [num_keys] owning worker or NUPS_OWNER_DEFAULT; NULL = not tracked
-    int* pending;              // [num_keys] localize requests of the running call (-1 = none)
+    uint32_t* own;             // [num_keys] ownership words (see mark_localize); NULL = not tracked
     DevStat* st;
     double* loss_partial;      // [4 * NUPS_MAX_STEP_BLOCKS] per-warp loss sums of the running step kernel
     uint64_t num_keys;
@@ -49,6 +48,7 @@ struct View {
     uint32_t L4;               // floats per row / 4
     uint32_t R;
     uint32_t count;            // count accesses?
+    uint32_t epoch_tag;        // number of the running call, shifted into the upper 24 bits of an ownership word
 };
 
 struct Dist {
@@ -86,14 +86,12 @@ struct nups_store {
     float *dval, *dacc;
     uint32_t* dirty;
     unsigned long long* cnt;
-    uint8_t* owner;
-    int* pending;
+    uint32_t* own;
+    uint32_t epoch;            // calls that moved keys so far (24 bits, see nups_new_epoch)
     DevStat* st;
     double* loss_partial;
     char* scratch;
     size_t scratch_bytes;
-    uint32_t* req_keys;        // localize request list of the running call
-    size_t req_cap;
     uint32_t* negs_buf;        // negatives drawn for the workload steps, possibly several batches ahead
     uint64_t negs_cap;
     uint32_t* last_negs;       // the slice of negs_buf that the most recent step used
@@ -143,7 +141,7 @@ View nups_view(const nups_store* s);
 void nups_time_begin(nups_store* s, cudaStream_t st);
 void nups_time_end(nups_store* s, cudaStream_t st);
 nups_status nups_scratch(nups_store* s, size_t bytes, char** out);     // grow-only scratch, 256-byte aligned
-nups_status nups_req_reserve(nups_store* s, size_t n);
+nups_status nups_new_epoch(nups_store* s, cudaStream_t st);          // call before taking the view of a call that moves keys
 
 // primitives.cu
 size_t nups_scan_scratch_bytes(uint64_t n);
@@ -164,7 +162,6 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
 nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
                                  float* d_out_acc, int worker_map, uint64_t map_base, uint64_t map_total,
                                  int do_count, cudaStream_t st);
-nups_status nups_localize_apply(nups_store* s, uint64_t max_requests, cudaStream_t st);
 nups_status nups_sync_internal(nups_store* s, cudaStream_t st);
 // sampling.cu internals used by steps.cu
 nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st);
@@ -232,12 +229,19 @@ __device__ __forceinline__ bool key_is_hot(const View& v, uint32_t k)
     return v.H != 0 && ((__ldg(v.hot_bits + (k >> 5)) >> (k & 31)) & 1u);
 }
 
+// Ownership word of a key: low byte = owning worker (NUPS_OWNER_DEFAULT = never moved: key mod R),
+// upper 24 bits = number of the call that wrote it.
+__device__ __forceinline__ bool word_is_local(uint32_t word, uint32_t q, uint32_t k, uint32_t R)
+{
+    const uint32_t o = word & 0xFFu;
+    return (o == NUPS_OWNER_DEFAULT ? k % R : o) == q;
+}
+
 __device__ __forceinline__ bool key_is_local(const View& v, uint32_t q, uint32_t k)
 {
     if (key_is_hot(v, k)) return true;
-    if (!v.owner) return true;
-    uint32_t o = v.owner[k];
-    return (o == NUPS_OWNER_DEFAULT ? k % v.R : o) == q;
+    if (!v.own) return true;
+    return word_is_local(v.own[k], q, k, v.R);
 }
 
 // mark a replica slot as touched without waiting for anything to come back
@@ -247,22 +251,19 @@ __device__ __forceinline__ void mark_dirty(const View& v, uint32_t q, int slot)
 }
 __device__ __forceinline__ void prefetch_l2(const void* p) { asm volatile("prefetch.global.L2 [%0];" ::"l"(p)); }
 
-// Queue a localize request (key -> worker q) of the running call.  Called by whole warps: the lanes that
-// have a request share one addition to the list's counter instead of queueing up at it one by one.
-__device__ __forceinline__ void queue_localize(const View& v, bool active, uint32_t key, uint32_t q, uint32_t* req,
-                                               uint64_t req_cap)
+// Move key -> worker q (the paper's localize).  Requests of one call take effect when the call ends
+// and the last one wins; callers visit workers in ascending order, so the largest requesting worker
+// gets the key.  Nothing reads ownership while a call that moves keys runs, so the word can be
+// written at once: the call's number sits above the worker, hence one atomic maximum both replaces
+// whatever an earlier call left and keeps the largest worker of this call.  Replicated keys are
+// local to every worker and never move, which also keeps the hottest keys from queueing at one
+// address; a word that already shows this call and a worker >= q needs no atomic.
+__device__ __forceinline__ void mark_localize(const View& v, uint32_t key, uint32_t q)
 {
-    const unsigned lane = threadIdx.x & 31;
-    const unsigned m = __ballot_sync(0xFFFFFFFFu, active);
-    if (m == 0) return;
-    unsigned long long base = 0;
-    if (lane == (unsigned)(__ffs(m) - 1)) base = atomicAdd(&v.st->req_count, (unsigned long long)__popc(m));
-    base = __shfl_sync(0xFFFFFFFFu, base, __ffs(m) - 1);
-    if (active) {
-        atomicMax(v.pending + key, (int)q);
-        const unsigned long long at = base + __popc(m & ((1u << lane) - 1u));
-        if (at < req_cap) req[at] = key;
-    }
+    if (key_is_hot(v, key)) return;
+    const uint32_t want = v.epoch_tag | q;
+    if (__ldcg(v.own + key) >= want) return;
+    atomicMax(v.own + key, want);
 }
 
 __device__ __forceinline__ void flag_bad_key(const View& v) { atomicCAS(&v.st->status, 0, NUPS_EKEY); }

@@ -115,7 +115,7 @@ extern "C" nups_status nups_register_distribution(nups_store* s, uint32_t key_ba
     if (level < NUPS_CONFORM || level > NUPS_NONCONFORM) return NUPS_EINVAL;
     bool reuse = level == NUPS_BOUNDED || level == NUPS_LONGTERM;
     if (reuse && (U == 0 || G == 0 || G > NUPS_MAX_POOL)) return NUPS_EINVAL;
-    if ((level == NUPS_LONGTERM || level == NUPS_NONCONFORM) && !s->owner) return NUPS_ESTATE;
+    if ((level == NUPS_LONGTERM || level == NUPS_NONCONFORM) && !s->own) return NUPS_ESTATE;
     int id = -1;
     for (int i = 0; i < NUPS_MAX_DISTS; ++i) if (!s->dist[i].used) { id = i; break; }
     if (id < 0) return NUPS_ENOMEM;
@@ -220,95 +220,186 @@ __device__ __forceinline__ uint32_t draw_iid(const DrawParams& p, uint32_t q, un
     return p.key_base + (uint32_t)j;
 }
 
-// Handle buffer layout (device): start[R] (u64) | keys[N] (u32) | post[N] (u32) | state[R] (uint4)
+// Handle buffer layout (device): keys[N] (u32) | post[N] (u32) | state[R] (uint4) | flags (one bit per entry)
 struct HandleView {
-    unsigned long long* start;
     uint32_t* keys;
     uint32_t* post;
-    uint4* state;      // LONG-TERM per sub-handle: x = walk position, y = postponed head, z = postponed tail
+    uint4* state;      // LONG-TERM per sub-handle: x = walk position, y = postponed head, z = postponed tail,
+                       // w = postponed tail before the most recent call
+    uint32_t* flags;   // LONG-TERM: "is local" bit of the fresh entries that the running call may reach;
+                       // sub-handle q owns the words from (b_q / 32) + q on, so no two share a word
 };
 static size_t handle_bytes(uint64_t N, uint32_t R, int level)
 {
-    size_t b = align256((size_t)R * 8) + align256(N * 4);
-    if (level == NUPS_LONGTERM) b += align256(N * 4) + align256((size_t)R * 16);
+    size_t b = align256(N * 4);
+    if (level == NUPS_LONGTERM) b += align256(N * 4) + align256((size_t)R * 16) + align256((N / 32 + R + 2) * 4);
     return b;
 }
 static HandleView handle_view(char* buf, uint64_t N, uint32_t R)
 {
     HandleView h;
-    h.start = (unsigned long long*)buf; buf += align256((size_t)R * 8);
     h.keys = (uint32_t*)buf; buf += align256(N * 4);
     h.post = (uint32_t*)buf; buf += align256(N * 4);
-    h.state = (uint4*)buf;
+    h.state = (uint4*)buf; buf += align256((size_t)R * 16);
+    h.flags = (uint32_t*)buf;
     return h;
 }
 
-__global__ void handle_begin_kernel(const unsigned long long* off_cur, unsigned long long* off_next, HandleView h,
-                                    uint64_t N, uint32_t R, int longterm)
+// Local sampling: the first key local to worker q among the candidate k0 and the 63 keys after it
+// (wrapping inside the distribution's key range), else k0.  The candidates are consecutive keys, so
+// their ownership words are consecutive too: they are read sixteen at a time with 128-bit loads (most
+// walks end within the first sixteen), and their technique bits lie in at most three words.
+__device__ __forceinline__ uint32_t first_local(const View& v, const DrawParams& p, uint32_t q, uint32_t k0)
 {
-    uint32_t q = blockIdx.x * blockDim.x + threadIdx.x;
-    if (q >= R) return;
-    unsigned long long size = chunk_begin(q + 1, N, R) - chunk_begin(q, N, R);
-    h.start[q] = off_cur[q];
-    off_next[q] = off_cur[q] + size;
-    if (longterm) h.state[q] = make_uint4(0u, 0u, 0u, 0u);
+    if (!v.own) return k0;
+    const unsigned long long rel = k0 - p.key_base;
+    const uint32_t R = v.R;
+    const uint64_t a0 = (uint64_t)k0 & ~3ull;                // 16-byte aligned start
+    if (rel + NUPS_LOCAL_PROBES <= p.n && a0 + NUPS_LOCAL_PROBES + 16 <= v.num_keys) {
+        // bit j of `hot` belongs to key 32 * (k0 / 32) + j
+        uint32_t h0 = 0, h1 = 0, h2 = 0;
+        if (v.H) {
+            const uint64_t w0 = (uint64_t)k0 >> 5, wlast = ((uint64_t)k0 + NUPS_LOCAL_PROBES - 1) >> 5;
+            h0 = __ldg(v.hot_bits + w0);
+            if (w0 + 1 <= wlast) h1 = __ldg(v.hot_bits + w0 + 1);
+            if (w0 + 2 <= wlast) h2 = __ldg(v.hot_bits + w0 + 2);
+        }
+        const uint4* op = reinterpret_cast<const uint4*>(v.own + a0);
+        uint32_t res = (uint32_t)(a0 % R);                   // key mod R of the key looked at, kept by counting
+        const uint32_t hbase = k0 & ~31u;
+        for (int g = 0; g < 5; ++g) {                        // keys a0 + 16 g ... a0 + 16 g + 15
+            uint4 o4[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) o4[u] = __ldg(op + g * 4 + u);
+            uint32_t found = 0;                              // bit t: key a0 + 16 g + t is a candidate and local
+#pragma unroll
+            for (int t = 0; t < 16; ++t) {
+                const uint4 o = o4[t >> 2];
+                const uint32_t w = (t & 3) == 0 ? o.x : (t & 3) == 1 ? o.y : (t & 3) == 2 ? o.z : o.w;
+                const uint32_t key = (uint32_t)a0 + g * 16 + t;
+                const uint32_t ob = w & 0xFFu;
+                bool loc = (ob == NUPS_OWNER_DEFAULT ? res : ob) == q;
+                const uint32_t hb = key - hbase;             // 0 .. 95 for candidates
+                const uint32_t hw = hb < 32 ? h0 : hb < 64 ? h1 : h2;
+                loc = loc || ((hw >> (hb & 31)) & 1u);
+                if (loc && key >= k0 && key < k0 + NUPS_LOCAL_PROBES) found |= 1u << t;
+                res = res + 1 == R ? 0 : res + 1;
+            }
+            if (found) return (uint32_t)a0 + g * 16 + (__ffs(found) - 1);
+        }
+        return k0;
+    }
+    for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
+        const uint32_t cand = p.key_base + (uint32_t)((rel + probe) % p.n);
+        if (key_is_local(v, q, cand)) return cand;
+    }
+    return k0;
 }
 
-__global__ void draw_iid_kernel(DrawParams p, HandleView h, uint64_t N, uint32_t R)
+// independent draws: one thread per sample.  The advanced stream offsets go to the other half of the
+// distribution's offset array.
+__global__ void draw_iid_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
+                                unsigned long long* __restrict__ off_next, HandleView h, uint64_t N, int localize)
 {
+    const uint32_t R = v.R;
+    if (blockIdx.x == 0)
+        for (uint32_t w = threadIdx.x; w < R; w += blockDim.x)
+            off_next[w] = off_cur[w] + (chunk_begin(w + 1, N, R) - chunk_begin(w, N, R));
     uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (o >= N) return;
-    uint32_t q = chunk_of_pos(o, N, R);
-    h.keys[o] = draw_iid(p, q, h.start[q] + (o - chunk_begin(q, N, R)));
+    const uint32_t q = chunk_of_pos(o, N, R);
+    const uint32_t k = draw_iid(p, q, off_cur[q] + (o - chunk_begin(q, N, R)));
+    h.keys[o] = k;
+    if (localize) mark_localize(v, k, q);          // PrepareSample localizes what it sampled
 }
 
 // Pooled reuse: pool `pl` of a worker holds G iid draws and is walked U times, each pass in a fresh
 // Fisher-Yates order.  Stream position s lies in pass number s / G overall (pool = pass / U).
-// One block produces one pass of one worker.
-__global__ void draw_reuse_kernel(DrawParams p, HandleView h, uint64_t N, uint32_t R)
+// One block visits one pool: it draws the pool once, then each warp produces whole passes: the
+// shuffle itself is sequential (one lane), the random words and the output are warp-wide.
+// Shared memory: pool[G] | per warp xs[G] | per warp perm[G] (16-bit).
+struct ReuseShape {
+    unsigned warps;
+    size_t smem;
+};
+static ReuseShape reuse_shape(uint32_t U, uint32_t G)
 {
-    __shared__ uint32_t pool[NUPS_MAX_POOL];
-    __shared__ uint32_t perm[NUPS_MAX_POOL];
-    __shared__ uint32_t xs[NUPS_MAX_POOL];
-    const uint32_t q = blockIdx.y, G = p.G;
-    const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
-    if (size == 0) return;
-    const unsigned long long s0 = h.start[q], s1 = s0 + size;
-    const unsigned long long pass = s0 / G + blockIdx.x;
-    if (pass * G >= s1) return;
-    const unsigned long long pl = pass / p.U;
-    for (uint32_t m = threadIdx.x; m < G; m += blockDim.x) {
-        pool[m] = draw_iid(p, q, pl * G + m);
-        perm[m] = m;
-    }
-    // random words of the shuffle: word d of the pass's Philox stream (purpose 1), four per block
-    for (uint32_t blk = threadIdx.x; blk * 4 < G - 1; blk += blockDim.x) {
-        uint32_t x[4];
-        philox_at(p.seed, pass, q, 1, blk, x);
-        for (int k = 0; k < 4; ++k)
-            if (blk * 4 + k < G - 1) xs[blk * 4 + k] = x[k];
-    }
+    ReuseShape r;
+    r.warps = G > 512 ? 4 : 8;
+    if (r.warps > U) r.warps = U;
+    if (r.warps < 1) r.warps = 1;
+    r.smem = (size_t)G * 4 + (size_t)r.warps * G * 4 + (((size_t)r.warps * G * 2 + 15) / 16) * 16;
+    return r;
+}
+static unsigned reuse_pools(uint64_t max_size, uint32_t U, uint32_t G)
+{
+    return (unsigned)(max_size / ((uint64_t)U * G) + 2);      // a stretch may begin and end inside a pool
+}
+
+template <class Emit>
+__device__ __forceinline__ void reuse_pool_visit(const DrawParams& p, uint32_t q, unsigned long long s0,
+                                                 unsigned long long s1, Emit emit)
+{
+    extern __shared__ __align__(16) uint32_t reuse_mem[];
+    const uint32_t G = p.G, U = p.U;
+    const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const unsigned long long span = (unsigned long long)U * G;
+    const unsigned long long pl = s0 / span + blockIdx.x;
+    if (pl * span >= s1) return;
+    uint32_t* pool = reuse_mem;
+    uint32_t* xs = reuse_mem + G + (size_t)warp * G;
+    uint16_t* perm = reinterpret_cast<uint16_t*>(reuse_mem + G + (size_t)nwarps * G) + (size_t)warp * G;
+    for (uint32_t m = threadIdx.x; m < G; m += blockDim.x) pool[m] = draw_iid(p, q, pl * G + m);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        for (uint32_t i = G - 1; i >= 1; --i) {
-            uint32_t r = __umulhi(xs[G - 1 - i], i + 1);
-            uint32_t t = perm[i]; perm[i] = perm[r]; perm[r] = t;
+    for (uint32_t t = warp; t < U; t += nwarps) {
+        const unsigned long long pass = pl * U + t, lo = pass * G;
+        if (lo + G <= s0 || lo >= s1) continue;
+        // random words of the shuffle: word d of the pass's Philox stream (purpose 1), four per block
+        for (uint32_t blk = lane; blk * 4 + 1 < G; blk += 32) {
+            uint32_t x[4];
+            philox_at(p.seed, pass, q, 1, blk, x);
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+                if (blk * 4 + k + 1 < G) xs[blk * 4 + k] = x[k];
         }
-    }
-    __syncthreads();
-    for (uint32_t j = threadIdx.x; j < G; j += blockDim.x) {
-        unsigned long long sp = pass * G + j;
-        if (sp >= s0 && sp < s1) h.keys[b0 + (sp - s0)] = pool[perm[j]];
+        for (uint32_t m = lane; m < G; m += 32) perm[m] = (uint16_t)m;
+        __syncwarp();
+        if (lane == 0) {
+            for (uint32_t i = G - 1; i >= 1; --i) {
+                const uint32_t r = __umulhi(xs[G - 1 - i], i + 1);
+                const uint16_t tmp = perm[i]; perm[i] = perm[r]; perm[r] = tmp;
+            }
+        }
+        __syncwarp();
+        for (uint32_t j0 = 0; j0 < G; j0 += 32) {             // whole warps: emit may ballot
+            const uint32_t j = j0 + lane;
+            const unsigned long long sp = lo + j;
+            const bool in = j < G && sp >= s0 && sp < s1;
+            const uint32_t k = in ? pool[perm[j]] : 0u;
+            emit(in, k, sp - s0);
+        }
+        __syncwarp();
     }
 }
 
-// PrepareSample localizes the sampled keys to the sub-handle's worker
-__global__ void localize_handle_kernel(View v, const uint32_t* __restrict__ keys, uint64_t N, uint32_t* req,
-                                       uint64_t req_cap)
+__global__ void draw_reuse_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
+                                  unsigned long long* __restrict__ off_next, HandleView h, uint64_t N, int localize,
+                                  int longterm)
 {
-    uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool in = o < N;
-    queue_localize(v, in, in ? keys[o] : 0u, in ? chunk_of_pos(o, N, v.R) : 0u, req, req_cap);
+    const uint32_t q = blockIdx.y, R = v.R;
+    const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
+    const unsigned long long s0 = off_cur[q];
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        off_next[q] = s0 + size;
+        if (longterm) h.state[q] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    if (size == 0) return;
+    reuse_pool_visit(p, q, s0, s0 + size, [&](bool in, uint32_t k, unsigned long long rel) {
+        if (in) {
+            h.keys[b0 + rel] = k;
+            if (localize) mark_localize(v, k, q);
+        }
+    });
 }
 
 static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int* slot_out, cudaStream_t st)
@@ -336,34 +427,26 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
         if (cudaMalloc(&h.buf, want) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
         h.cap = want;
     }
-    bool reuse = d.level == NUPS_BOUNDED || d.level == NUPS_LONGTERM;
-    bool loc = s->owner && d.level != NUPS_NONCONFORM;
-    if (loc || d.level == NUPS_LONGTERM) {
-        nups_status rc = nups_req_reserve(s, N);
+    const bool reuse = d.level == NUPS_BOUNDED || d.level == NUPS_LONGTERM;
+    const bool loc = s->own && d.level != NUPS_NONCONFORM;
+    if (loc) {
+        nups_status rc = nups_new_epoch(s, st);
         if (rc != NUPS_OK) return rc;
     }
     HandleView hv = handle_view(h.buf, N, s->R);
     DrawParams p = draw_params(d);
-    handle_begin_kernel<<<grid_for(s->R, 64), 64, 0, st>>>(d.off + (size_t)d.cur * s->R, d.off + (size_t)(d.cur ^ 1) * s->R,
-                                                           hv, N, s->R, d.level == NUPS_LONGTERM);
+    View v = nups_view(s);
+    const unsigned long long* off_cur = d.off + (size_t)d.cur * s->R;
+    unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
+    if (reuse) {
+        const ReuseShape sh = reuse_shape(d.U, d.G);
+        draw_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R), sh.warps * 32, sh.smem, st>>>(
+            v, p, off_cur, off_next, hv, N, loc, d.level == NUPS_LONGTERM);
+    } else {
+        draw_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(v, p, off_cur, off_next, hv, N, loc);
+    }
     LAUNCH_CHECK(s);
     d.cur ^= 1;
-    if (reuse) {
-        uint64_t max_size = (N + s->R - 1) / s->R;
-        unsigned passes = (unsigned)(max_size / d.G + 2);
-        unsigned threads = ((d.G + 31) / 32) * 32;
-        if (threads > 256) threads = 256;
-        draw_reuse_kernel<<<dim3(passes, s->R), threads, 0, st>>>(p, hv, N, s->R);
-    } else {
-        draw_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(p, hv, N, s->R);
-    }
-    LAUNCH_CHECK(s);
-    if (loc) {
-        localize_handle_kernel<<<grid_for(N, 256), 256, 0, st>>>(nups_view(s), hv.keys, N, s->req_keys, s->req_cap);
-        LAUNCH_CHECK(s);
-        nups_status rc = nups_localize_apply(s, N, st);
-        if (rc != NUPS_OK) return rc;
-    }
     h.used = 1; h.dist = dist; h.N = N; h.cursor = 0;
     *slot_out = id;
     return NUPS_OK;
@@ -406,28 +489,50 @@ __global__ void emit_kernel(View v, DrawParams p, HandleView h, uint64_t N, uint
     if (in) {
         uint64_t pos = cursor + o;
         k = h.keys[pos];
-        if (local_only) {
-            uint32_t q = chunk_of_pos(pos, N, v.R);
-            uint32_t k0 = k;
-            for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
-                uint32_t cand = p.key_base + (uint32_t)(((unsigned long long)(k0 - p.key_base) + probe) % p.n);
-                if (key_is_local(v, q, cand)) { k = cand; break; }
-            }
-        }
+        if (local_only) k = first_local(v, p, chunk_of_pos(pos, N, v.R), k);
         out[o] = k;
     }
     count_sample(v, k, in);
 }
 
-// reuse with postponing: one block walks one sub-handle.  Entries not yet postponed are taken in
-// order; a local one is emitted, a non-local one is queued for re-localization and appended to the
-// sub-handle's postponed queue; when the fresh entries run out the postponed ones are emitted.
+// Reuse with postponing.  Entries of a sub-handle not yet postponed are taken in list order: a local
+// one is emitted, a non-local one is re-localized and appended to the sub-handle's postponed queue;
+// when the fresh entries run out the postponed ones are emitted.  Locality is judged by the
+// ownership at the start of the call.
+// The ownership lookups are scattered reads, so they are done ahead of the walk by a kernel that
+// spreads them over the whole GPU (one bit per entry); the walk itself, one block per sub-handle,
+// then only streams keys and bits.  The lookup covers the fresh entries that the call is likely to
+// reach (twice what it must emit, plus a margin); should the walk go further, it looks up the rest itself.
 constexpr int LT_THREADS = 1024;
-constexpr int LT_ITEMS = 4;                 // consecutive list entries per thread and round
+constexpr uint64_t LT_MARGIN = 4096;
+
+__device__ __forceinline__ uint64_t lt_window(uint64_t oc, uint64_t size, uint64_t take)
+{
+    const uint64_t w = 2 * take + LT_MARGIN;
+    return w < size - oc ? w : size - oc;
+}
+
+__global__ void lt_flags_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
+{
+    const uint32_t q = q_first + blockIdx.y;
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t b0 = chunk_begin(q, N, v.R), b1 = chunk_begin(q + 1, N, v.R);
+    const uint64_t lo = max(b0, cursor), hi = min(b1, cursor + n);
+    if (lo >= hi) return;
+    const uint64_t size = b1 - b0, oc = h.state[q].x;
+    if (oc >= size) return;
+    const uint64_t w_end = (oc + lt_window(oc, size, hi - lo) + 31) >> 5;
+    const uint64_t word = (oc >> 5) + (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    if (word >= w_end) return;
+    const uint64_t i = word * 32 + lane;
+    const bool loc = i < size && key_is_local(v, q, h.keys[b0 + i]);
+    const unsigned bits = __ballot_sync(0xFFFFFFFFu, loc);
+    if (lane == 0) h.flags[(b0 >> 5) + q + word] = bits;
+}
 
 __global__ void __launch_bounds__(LT_THREADS)
 longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
-                uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+                uint32_t* __restrict__ out)
 {
     __shared__ unsigned warp_tot[LT_THREADS / 32];
     __shared__ unsigned sh_consumed, sh_local;
@@ -438,23 +543,35 @@ longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, u
     if (lo >= hi) return;
     const uint64_t take = hi - lo, size = b1 - b0;
     const uint64_t out_base = lo - cursor;
-    uint4 stt = h.state[q];
+    const uint4 stt = h.state[q];
     uint64_t oc = stt.x, ph = stt.y, pt = stt.z, emitted = 0;
+    const uint64_t pt0 = pt;
+    const uint64_t w_known = oc < size ? (oc + lt_window(oc, size, take) + 31) >> 5 : 0;   // bits below were looked up
+    const uint32_t* flags = h.flags + (b0 >> 5) + q;
     while (emitted < take && oc < size) {
-        // a round looks at LT_THREADS * LT_ITEMS fresh entries in list order: thread t owns entries
-        // t * LT_ITEMS .. t * LT_ITEMS + LT_ITEMS - 1 of the round
-        uint32_t key[LT_ITEMS];
-        bool have[LT_ITEMS], loc[LT_ITEMS];
-        unsigned mine = 0;
-#pragma unroll
-        for (int k = 0; k < LT_ITEMS; ++k) {
-            const uint64_t i = oc + (uint64_t)tid * LT_ITEMS + k;
-            have[k] = i < size;
-            key[k] = have[k] ? h.keys[b0 + i] : 0u;
-            loc[k] = have[k] && key_is_local(v, q, key[k]);
-            mine += loc[k] ? 1u : 0u;
+        // a round looks at the 32 * LT_THREADS entries from the word of `oc` on, in list order: lane l of
+        // warp w holds the bits of word 32 w + l of the round
+        const uint64_t word0 = (oc >> 5) + (uint64_t)warp * 32;
+        const uint64_t myword = word0 + lane, e0 = myword * 32;
+        uint32_t valid = 0;                       // entries of my word inside [oc, size)
+        if (e0 + 32 > oc && e0 < size) {
+            valid = 0xFFFFFFFFu;
+            if (e0 < oc) valid &= 0xFFFFFFFFu << (unsigned)(oc - e0);
+            if (e0 + 32 > size) valid &= 0xFFFFFFFFu >> (unsigned)(e0 + 32 - size);
         }
-        // exclusive count of local entries before this thread's first entry
+        uint32_t bits = (valid && myword < w_known) ? flags[myword] : 0u;
+        unsigned missing = __ballot_sync(0xFFFFFFFFu, valid != 0 && myword >= w_known);
+        while (missing) {
+            const int w = __ffs(missing) - 1;
+            missing &= missing - 1;
+            const uint64_t i = (word0 + w) * 32 + lane;
+            const bool loc = i < size && key_is_local(v, q, h.keys[b0 + i]);
+            const unsigned b = __ballot_sync(0xFFFFFFFFu, loc);
+            if ((int)lane == w) bits = b;
+        }
+        bits &= valid;
+        // exclusive count of local entries before this lane's word
+        const unsigned mine = __popc(bits);
         unsigned inc = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -464,34 +581,35 @@ longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, u
         if (lane == 31) warp_tot[warp] = inc;
         if (tid == 0) { sh_consumed = 0; sh_local = 0; }
         __syncthreads();
-        unsigned excl = inc - mine;
-        for (unsigned w = 0; w < warp; ++w) excl += warp_tot[w];
+        unsigned long long wexcl = 0;
+        for (unsigned w = 0; w < warp; ++w) wexcl += warp_tot[w];
+        const unsigned wpre = inc - mine;
         const uint64_t need = take - emitted;
         unsigned nc = 0, nl = 0;
-#pragma unroll
-        for (int k = 0; k < LT_ITEMS; ++k) {
+        for (int w = 0; w < 32; ++w) {
+            const uint32_t vb = __shfl_sync(0xFFFFFFFFu, valid, w);
+            if (vb == 0) continue;
+            const uint32_t wb = __shfl_sync(0xFFFFFFFFu, bits, w);
+            const unsigned pre = __shfl_sync(0xFFFFFFFFu, wpre, w);
+            const uint64_t i = (word0 + w) * 32 + lane;
+            const bool have = (vb >> lane) & 1u, loc = (wb >> lane) & 1u;
             // the walk stops right after the need-th local entry: an entry is reached iff fewer than
             // `need` local entries lie before it
-            const bool consumed = have[k] && excl < need;
+            const unsigned long long before = wexcl + pre + __popc(wb & ((1u << lane) - 1u));
+            const bool consumed = have && before < need;
+            uint32_t key = 0;
             if (consumed) {
-                if (loc[k]) out[out_base + emitted + excl] = key[k];
+                key = h.keys[b0 + i];
+                if (loc) out[out_base + emitted + before] = key;
                 else {
-                    h.post[b0 + pt + ((uint64_t)tid * LT_ITEMS + k - excl)] = key[k];     // non-local entries before it
-                    atomicMax(v.pending + key[k], (int)q);
-                    const unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
-                    if (at < req_cap) req[at] = key[k];
+                    h.post[b0 + pt + ((i - oc) - before)] = key;              // non-local entries before it
                 }
-                nc++;
-                nl += loc[k] ? 1u : 0u;
             }
-            count_sample(v, key[k], consumed && loc[k]);
-            excl += loc[k] ? 1u : 0u;
+            nc += __popc(__ballot_sync(0xFFFFFFFFu, consumed));
+            nl += __popc(__ballot_sync(0xFFFFFFFFu, consumed && loc));
+            count_sample(v, key, consumed && loc);
         }
-        for (int o = 16; o > 0; o >>= 1) {
-            nc += __shfl_xor_sync(0xFFFFFFFFu, nc, o);
-            nl += __shfl_xor_sync(0xFFFFFFFFu, nl, o);
-        }
-        if (lane == 0) { atomicAdd(&sh_consumed, nc); atomicAdd(&sh_local, nl); }
+        if (lane == 0 && nc) { atomicAdd(&sh_consumed, nc); atomicAdd(&sh_local, nl); }
         __syncthreads();
         const unsigned tc = sh_consumed, tl = sh_local;
         emitted += tl; pt += tc - tl; oc += tc;
@@ -508,7 +626,20 @@ longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, u
         }
         ph += cnt;
     }
-    if (tid == 0) h.state[q] = make_uint4((unsigned)oc, (unsigned)ph, (unsigned)pt, 0u);
+    if (tid == 0) h.state[q] = make_uint4((unsigned)oc, (unsigned)ph, (unsigned)pt, (unsigned)pt0);
+}
+
+// the entries that the walk just postponed move to their worker (when the call ends: the walk itself
+// judged locality by the ownership from before the call)
+__global__ void lt_localize_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
+{
+    const uint32_t q = q_first + blockIdx.y;
+    const uint64_t b0 = chunk_begin(q, N, v.R), b1 = chunk_begin(q + 1, N, v.R);
+    if (max(b0, cursor) >= min(b1, cursor + n)) return;
+    const uint4 stt = h.state[q];
+    const uint64_t rel = (uint64_t)stt.w + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (rel >= stt.z) return;
+    mark_localize(v, h.post[b0 + rel], q);
 }
 
 static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_keys_out, float* d_vals_out,
@@ -518,21 +649,33 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
     Dist& d = s->dist[h.dist];
     if (n > h.N - h.cursor) return NUPS_ESTATE;
     if (n == 0) return NUPS_OK;
+    if (d.level == NUPS_LONGTERM) {
+        nups_status rc = nups_new_epoch(s, st);
+        if (rc != NUPS_OK) return rc;
+    }
     View v = nups_view(s);
     HandleView hv = handle_view(h.buf, h.N, s->R);
     DrawParams p = draw_params(d);
     if (d.level == NUPS_LONGTERM) {
-        // sub-handles overlapped by [cursor, cursor + n)
+        // sub-handles overlapped by [cursor, cursor + n), and the most that one of them must emit
         uint32_t qf = 0, ql = 0;
+        uint64_t max_take = 0;
         for (uint32_t q = 0; q < s->R; ++q) {
             uint64_t b0 = ((uint64_t)q * h.N) / s->R, b1 = ((uint64_t)(q + 1) * h.N) / s->R;
             if (b0 <= h.cursor && h.cursor < b1) qf = q;
             if (b0 <= h.cursor + n - 1 && h.cursor + n - 1 < b1) ql = q;
+            uint64_t lo = b0 > h.cursor ? b0 : h.cursor, hi = b1 < h.cursor + n ? b1 : h.cursor + n;
+            if (hi > lo && hi - lo > max_take) max_take = hi - lo;
         }
-        longterm_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->req_keys, s->req_cap);
+        const uint64_t max_size = (h.N + s->R - 1) / s->R;
+        uint64_t window = 2 * max_take + LT_MARGIN;
+        if (window > max_size) window = max_size;
+        lt_flags_kernel<<<dim3(grid_for(window / 32 + 2, 8), ql - qf + 1), 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
         LAUNCH_CHECK(s);
-        nups_status rc = nups_localize_apply(s, h.N, st);
-        if (rc != NUPS_OK) return rc;
+        longterm_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
+        LAUNCH_CHECK(s);
+        lt_localize_kernel<<<dim3(grid_for(max_size, 256), ql - qf + 1), 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
+        LAUNCH_CHECK(s);
     } else {
         emit_kernel<<<grid_for(n, 256), 256, 0, st>>>(v, p, hv, h.N, h.cursor, n, d.level == NUPS_NONCONFORM, d_keys_out);
         LAUNCH_CHECK(s);
@@ -559,18 +702,11 @@ extern "C" nups_status nups_pull_sample(nups_store* s, nups_handle handle, uint6
 // same keys as the handle path gives, written straight to `out`.  Stream offsets are read from one
 // half of the distribution's offset array and the advanced offsets written to the other half.
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void direct_tail(const View& v, uint32_t key, uint32_t q, bool in, bool localize, uint32_t* req,
-                                            uint64_t req_cap)
-{
-    count_sample(v, key, in);
-    if (localize) queue_localize(v, in, key, q, req, req_cap);
-}
-
 // blockIdx.y (iid) / blockIdx.z (reuse) = batch: `batches` handles of N samples each are drawn back to back,
 // exactly as that many separate calls would draw them; batch b goes to out + b * N.
-__global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long long* off_cur,
-                                       unsigned long long* off_next, uint64_t N, uint32_t batches, int local_only,
-                                       int localize, uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+__global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
+                                       unsigned long long* __restrict__ off_next, uint64_t N, uint32_t batches,
+                                       int local_only, int localize, uint32_t* __restrict__ out)
 {
     const uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t bt = blockIdx.y;
@@ -581,69 +717,35 @@ __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long
         q = chunk_of_pos(o, N, v.R);
         const unsigned long long size = chunk_begin(q + 1, N, v.R) - chunk_begin(q, N, v.R);
         k = draw_iid(p, q, off_cur[q] + (unsigned long long)bt * size + (o - chunk_begin(q, N, v.R)));
-        if (local_only) {
-            const uint32_t k0 = k;
-            for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
-                uint32_t cand = p.key_base + (uint32_t)(((unsigned long long)(k0 - p.key_base) + probe) % p.n);
-                if (key_is_local(v, q, cand)) { k = cand; break; }
-            }
-        }
+        if (local_only) k = first_local(v, p, q, k);
         out[o] = k;
+        if (localize) mark_localize(v, k, q);
     }
-    direct_tail(v, k, q, in, localize != 0, req, req_cap);
+    count_sample(v, k, in);
     if (blockIdx.x == 0 && blockIdx.y == 0)
         for (uint32_t w = threadIdx.x; w < v.R; w += blockDim.x)
             off_next[w] = off_cur[w] + (unsigned long long)batches * (chunk_begin(w + 1, N, v.R) - chunk_begin(w, N, v.R));
 }
 
-__global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned long long* off_cur,
-                                         unsigned long long* off_next, uint64_t N, uint32_t batches, int localize,
-                                         uint32_t* __restrict__ out, uint32_t* req, uint64_t req_cap)
+__global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
+                                         unsigned long long* __restrict__ off_next, uint64_t N, uint32_t batches,
+                                         int localize, uint32_t* __restrict__ out)
 {
-    __shared__ uint32_t pool[NUPS_MAX_POOL];
-    __shared__ uint32_t perm[NUPS_MAX_POOL];
-    __shared__ uint32_t xs[NUPS_MAX_POOL];
-    const uint32_t q = blockIdx.y, G = p.G, R = v.R;
+    const uint32_t q = blockIdx.y, R = v.R;
     if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         for (uint32_t w = threadIdx.x; w < R; w += blockDim.x)
             off_next[w] = off_cur[w] + (unsigned long long)batches * (chunk_begin(w + 1, N, R) - chunk_begin(w, N, R));
     const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
     if (size == 0) return;
     out += (uint64_t)blockIdx.z * N;
-    const unsigned long long s0 = off_cur[q] + (unsigned long long)blockIdx.z * size, s1 = s0 + size;
-    const unsigned long long pass = s0 / G + blockIdx.x;
-    if (pass * G >= s1) return;
-    const unsigned long long pl = pass / p.U;
-    for (uint32_t m = threadIdx.x; m < G; m += blockDim.x) {
-        pool[m] = draw_iid(p, q, pl * G + m);
-        perm[m] = m;
-    }
-    for (uint32_t blk = threadIdx.x; blk * 4 < G - 1; blk += blockDim.x) {
-        uint32_t x[4];
-        philox_at(p.seed, pass, q, 1, blk, x);
-        for (int k = 0; k < 4; ++k)
-            if (blk * 4 + k < G - 1) xs[blk * 4 + k] = x[k];
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        for (uint32_t i = G - 1; i >= 1; --i) {
-            uint32_t r = __umulhi(xs[G - 1 - i], i + 1);
-            uint32_t t = perm[i]; perm[i] = perm[r]; perm[r] = t;
-        }
-    }
-    __syncthreads();
-    const uint32_t rounds = (G + blockDim.x - 1) / blockDim.x;
-    for (uint32_t rd = 0; rd < rounds; ++rd) {           // whole warps take every round: the tail ballots
-        const uint32_t j = rd * blockDim.x + threadIdx.x;
-        const unsigned long long sp = pass * G + j;
-        const bool in = j < G && sp >= s0 && sp < s1;
-        uint32_t k = 0;
+    const unsigned long long s0 = off_cur[q] + (unsigned long long)blockIdx.z * size;
+    reuse_pool_visit(p, q, s0, s0 + size, [&](bool in, uint32_t k, unsigned long long rel) {
         if (in) {
-            k = pool[perm[j]];
-            out[b0 + (sp - s0)] = k;
+            out[b0 + rel] = k;
+            if (localize) mark_localize(v, k, q);
         }
-        direct_tail(v, k, q, in, localize != 0, req, req_cap);
-    }
+        count_sample(v, k, in);
+    });
 }
 
 // Sample-ahead for the workload steps.  The sample streams are a pure function of (seed, worker,
@@ -688,7 +790,7 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
     if (rc != NUPS_OK) return rc;
     Dist& d = s->dist[dist];
     const bool plain = d.level == NUPS_CONFORM || d.level == NUPS_BOUNDED;
-    const uint32_t batches = (plain && !s->cfg.deterministic && !s->cfg.count_accesses && !s->owner &&
+    const uint32_t batches = (plain && !s->cfg.deterministic && !s->cfg.count_accesses && !s->own &&
                               N * NUPS_SAMPLE_AHEAD < (1ull << 28)) ? NUPS_SAMPLE_AHEAD : 1;
     if (N * batches > s->negs_cap) {
         if (s->negs_buf) CK(cudaFree(s->negs_buf));
@@ -708,9 +810,9 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
         s->last_negs_n = N;
         return NUPS_OK;
     }
-    const int localize = s->owner && d.level != NUPS_NONCONFORM;
+    const int localize = s->own && d.level != NUPS_NONCONFORM;
     if (localize) {
-        rc = nups_req_reserve(s, N);
+        rc = nups_new_epoch(s, st);
         if (rc != NUPS_OK) return rc;
     }
     View v = nups_view(s);
@@ -718,23 +820,16 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
     const unsigned long long* off_cur = d.off + (size_t)d.cur * s->R;
     unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
     if (d.level == NUPS_BOUNDED) {
-        uint64_t max_size = (N + s->R - 1) / s->R;
-        unsigned passes = (unsigned)(max_size / d.G + 2);
-        unsigned threads = ((d.G + 31) / 32) * 32;
-        if (threads > 256) threads = 256;
-        draw_direct_reuse_kernel<<<dim3(passes, s->R, batches), threads, 0, st>>>(v, p, off_cur, off_next, N, batches, localize,
-                                                                                 s->negs_buf, s->req_keys, s->req_cap);
+        const ReuseShape sh = reuse_shape(d.U, d.G);
+        draw_direct_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R, batches), sh.warps * 32, sh.smem,
+                                   st>>>(v, p, off_cur, off_next, N, batches, localize, s->negs_buf);
     } else {
         draw_direct_iid_kernel<<<dim3(grid_for(N, 256), batches), 256, 0, st>>>(v, p, off_cur, off_next, N, batches,
                                                                               d.level == NUPS_NONCONFORM, localize,
-                                                                              s->negs_buf, s->req_keys, s->req_cap);
+                                                                              s->negs_buf);
     }
     LAUNCH_CHECK(s);
     d.cur ^= 1;
-    if (localize) {
-        rc = nups_localize_apply(s, N, st);
-        if (rc != NUPS_OK) return rc;
-    }
     s->last_negs_n = N;
     if (batches > 1) {
         s->ahead_dist = dist; s->ahead_N = N; s->ahead_total = batches; s->ahead_next = 1;

@@ -26,13 +26,6 @@ __device__ __forceinline__ void note_access(const View& v, uint32_t key, int slo
     atomicAdd(slot >= 0 ? &v.st->hot_hits : &v.st->cold_hits, (unsigned long long)times);
 }
 
-__device__ __forceinline__ void request_localize(const View& v, uint32_t key, uint32_t q, uint32_t* req, uint64_t cap)
-{
-    atomicMax(v.pending + key, (int)q);
-    unsigned long long at = atomicAdd(&v.st->req_count, 1ull);
-    if (at < cap) req[at] = key;
-}
-
 // offset value meaning "this key has no replica row"
 constexpr unsigned long long NO_PEND = ~0ull;
 
@@ -85,7 +78,7 @@ __global__ void __launch_bounds__(32 * SGNS_WARPS)
 sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
             const uint32_t* __restrict__ negs, uint64_t n, uint32_t K_arg, float lr,
             float* __restrict__ upd, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
-            float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap, uint32_t group,
+            float* __restrict__ loss_out, uint32_t group,
             unsigned long long* __restrict__ loss_acc)
 {
     extern __shared__ __align__(16) float4 park_all[];
@@ -156,7 +149,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
                 const unsigned times = (lane == 0 || lane == K + 1) ? (DET ? 1u : 2u) : (DET ? 0u : 1u);
                 if (times) note_access(v, key, slot, times);
             }
-            if (v.owner && (lane == 0 || lane == K + 1)) request_localize(v, key, q, req, req_cap);
+            if (v.own && (lane == 0 || lane == K + 1)) mark_localize(v, key, q);
         }
         asm volatile("cp.async.wait_group 0;" ::: "memory");
         // fold the worker's pending replica rows (read straight from the slab) into the staged rows
@@ -327,7 +320,7 @@ __global__ void __launch_bounds__(CPX_THREADS, 4)
 complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restrict__ rk, const uint32_t* __restrict__ tk,
                const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float eps, float* __restrict__ uval,
                float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
-               float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
+               float* __restrict__ loss_out)
 {
     // park[2 * role][tid] = the thread's part of the role's value row, park[2 * role + 1][tid] = of its
     // accumulator row; filled by asynchronous copies, all 2 * (3 + K) rows of a triple in flight at once
@@ -369,7 +362,7 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
                 const unsigned times = (tid < 3 ? 1u : 0u) + (DET ? 0u : 1u);       // pulled (+ pushed in fast mode)
                 if (times) note_access(v, key, slot, times);
             }
-            if (v.owner && tid < 3) request_localize(v, key, q, req, req_cap);
+            if (v.own && tid < 3) mark_localize(v, key, q);
         }
         if (mine) {
             for (uint32_t role = 0; role < per; ++role) {
@@ -459,7 +452,7 @@ template <bool HOT, bool DET, int CH>
 __global__ void __launch_bounds__(128)
 mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
           uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
-          float* __restrict__ loss_item, float* __restrict__ loss_out, uint32_t* req, uint64_t req_cap)
+          float* __restrict__ loss_item, float* __restrict__ loss_out)
 {
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -564,7 +557,7 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
                     note_access(v, ki, si, DET ? 1u : 2u);
                     note_access(v, kj, sj, DET ? 1u : 2u);
                 }
-                if (v.owner) { request_localize(v, ki, q, req, req_cap); request_localize(v, kj, q, req, req_cap); }
+                if (v.own) { mark_localize(v, ki, q); mark_localize(v, kj, q); }
                 if (DET) loss_item[i] = err * err;
             }
             my_loss += (double)(err * err);
@@ -622,7 +615,7 @@ static nups_status step_buffers(nups_store* s, uint64_t n, uint64_t per, bool tw
     return NUPS_OK;
 }
 
-static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t direct_keys, const StepBuffers& b,
+static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, const StepBuffers& b,
                                float* d_loss_out, cudaStream_t st, bool loss_done_in_kernel = false)
 {
     nups_status rc;
@@ -630,8 +623,6 @@ static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, uint64_t
         rc = nups_push_with_scratch(s, b.ukeys, n * per, (uint32_t)per, b.uval, b.uacc, b.push_scratch, st);
         if (rc != NUPS_OK) return rc;
     }
-    rc = nups_localize_apply(s, n * direct_keys, st);
-    if (rc != NUPS_OK) return rc;
     if (d_loss_out && !loss_done_in_kernel) {
         loss_mean_kernel<<<1, 256, 0, st>>>(b.loss_item, n, d_loss_out);
         LAUNCH_CHECK(s);
@@ -696,7 +687,7 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
         if (e == cudaSuccess) {                                                                                        \
             nups_time_begin(s, st);                                                                                    \
             kern<<<grid, 32 * SGNS_WARPS, smem, st>>>(v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
-                                                      b.loss_item, d_loss_out, s->req_keys, s->req_cap, group,        \
+                                                      b.loss_item, d_loss_out, group,                                  \
                                                       loss_acc);                                                       \
             nups_time_end(s, st);                                                                                      \
         }                                                                                                              \
@@ -725,14 +716,14 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
     cudaStream_t st = (cudaStream_t)stream;
     rc = nups_draw_negatives(s, dist, n * K, st);
     if (rc != NUPS_OK) return rc;
-    rc = nups_req_reserve(s, n * 2);
+    rc = nups_new_epoch(s, st);
     if (rc != NUPS_OK) return rc;
     StepBuffers b;
     rc = step_buffers(s, n, K + 2, false, &b);
     if (rc != NUPS_OK) return rc;
     rc = sgns_launch(s, d_center, d_context, n, K, lr, b, d_loss_out, 1, nullptr, st);
     if (rc != NUPS_OK) return rc;
-    return step_finish(s, n, K + 2, 2, b, d_loss_out, st, !s->cfg.deterministic);
+    return step_finish(s, n, K + 2, b, d_loss_out, st, !s->cfg.deterministic);
 }
 
 // per-step losses of a grouped launch: fixed-point sums -> means, and the sums are cleared for the next group
@@ -754,7 +745,7 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
     const uint64_t steps = n_total / batch;
     // where a step has side effects that must happen in step order (ordered pushes, access counts,
     // ownership changes), the steps are simply taken one by one
-    if (s->cfg.deterministic || s->cfg.count_accesses || s->owner) {
+    if (s->cfg.deterministic || s->cfg.count_accesses || s->own) {
         for (uint64_t t = 0; t < steps; ++t) {
             rc = nups_step_sgns(s, d_center + t * batch, d_context + t * batch, batch, dist, K, lr,
                                 d_loss_out ? d_loss_out + t : nullptr, stream);
@@ -803,7 +794,7 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     cudaStream_t st = (cudaStream_t)stream;
     nups_status rc = nups_draw_negatives(s, dist, n * K, st);
     if (rc != NUPS_OK) return rc;
-    rc = nups_req_reserve(s, n * 3);
+    rc = nups_new_epoch(s, st);
     if (rc != NUPS_OK) return rc;
     StepBuffers b;
     rc = step_buffers(s, n, K + 3, true, &b);
@@ -830,10 +821,10 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     }
     nups_time_begin(s, st);
     DISPATCH_MODE(s, complex_kernel<HOT, DET><<<grid, CPX_THREADS, smem, st>>>(
-        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap));
+        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, d_loss_out));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
-    return step_finish(s, n, K + 3, 3, b, d_loss_out, st, !s->cfg.deterministic);
+    return step_finish(s, n, K + 3, b, d_loss_out, st, !s->cfg.deterministic);
 }
 
 extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
@@ -843,7 +834,7 @@ extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const 
     if (s->L / 4 > 128) return NUPS_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     s->last_negs_n = 0;
-    nups_status rc = nups_req_reserve(s, n * 2);
+    nups_status rc = nups_new_epoch(s, st);
     if (rc != NUPS_OK) return rc;
     StepBuffers b;
     rc = step_buffers(s, n, 2, false, &b);
@@ -852,8 +843,8 @@ extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const 
     unsigned grid = step_grid(s, n, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2));   // resident blocks at that depth's register use
     nups_time_begin(s, st);
     DISPATCH_MODE(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out, s->req_keys, s->req_cap)));
+        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out)));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
-    return step_finish(s, n, 2, 2, b, d_loss_out, st, !s->cfg.deterministic);
+    return step_finish(s, n, 2, b, d_loss_out, st, !s->cfg.deterministic);
 }

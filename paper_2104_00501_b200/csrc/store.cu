@@ -35,7 +35,7 @@ View nups_view(const nups_store* s)
     View v;
     v.val = s->val; v.acc = s->acc; v.dval = s->dval; v.dacc = s->dacc;
     v.hot_bits = s->hot_bits; v.slot_of = s->slot_of; v.dirty = s->dirty;
-    v.cnt = s->cnt; v.owner = s->owner; v.pending = s->pending; v.st = s->st; v.loss_partial = s->loss_partial;
+    v.cnt = s->cnt; v.own = s->own; v.epoch_tag = s->epoch << 8; v.st = s->st; v.loss_partial = s->loss_partial;
     v.num_keys = s->num_keys; v.Hcap = s->Hcap; v.H = (uint32_t)s->H; v.L4 = s->L / 4; v.R = s->R;
     v.count = s->cfg.count_accesses;
     return v;
@@ -55,16 +55,24 @@ nups_status nups_scratch(nups_store* s, size_t bytes, char** out)
     return NUPS_OK;
 }
 
-nups_status nups_req_reserve(nups_store* s, size_t n)
+// Calls that move keys are numbered; the number is stored above the owner in every word such a call
+// writes.  When the 24 bits run out, the numbers in the table are cleared and counting restarts.
+__global__ void own_clear_epoch_kernel(uint32_t* own, uint64_t n)
 {
-    if (!s->owner) return NUPS_OK;
-    if (n > s->req_cap) {
-        size_t want = n + n / 2 + 1024;
-        if (s->req_keys) CK(cudaFree(s->req_keys));
-        s->req_keys = nullptr; s->req_cap = 0;
-        if (cudaMalloc(&s->req_keys, want * sizeof(uint32_t)) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
-        s->req_cap = want;
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (; i < n; i += stride) own[i] &= 0xFFu;
+}
+
+nups_status nups_new_epoch(nups_store* s, cudaStream_t st)
+{
+    if (!s->own) return NUPS_OK;
+    if (s->epoch >= 0xFFFFFFu) {
+        own_clear_epoch_kernel<<<grid_for(s->num_keys, 256, 8192), 256, 0, st>>>(s->own, s->num_keys);
+        LAUNCH_CHECK(s);
+        s->epoch = 0;
     }
+    s->epoch++;
     return NUPS_OK;
 }
 
@@ -162,8 +170,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     ok = ok && cudaMalloc(&s->st, sizeof(DevStat)) == cudaSuccess;
     ok = ok && cudaMalloc(&s->loss_partial, 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double)) == cudaSuccess;
     if (ok && c.track_ownership) {
-        ok = cudaMalloc(&s->owner, num_keys) == cudaSuccess;
-        ok = ok && cudaMalloc(&s->pending, num_keys * 4) == cudaSuccess;
+        ok = cudaMalloc(&s->own, num_keys * 4) == cudaSuccess;
     }
     if (!ok) {
         cudaGetLastError();
@@ -177,9 +184,8 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     cudaMemset(s->st, 0, sizeof(DevStat));
     cudaMemset(s->loss_partial, 0, 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double));
     fill_i32<<<grid_for(num_keys, 256, 4096), 256>>>(s->slot_of, num_keys, -1);
-    if (s->owner) {
-        cudaMemset(s->owner, NUPS_OWNER_DEFAULT, num_keys);
-        fill_i32<<<grid_for(num_keys, 256, 4096), 256>>>(s->pending, num_keys, -1);
+    if (s->own) {
+        fill_i32<<<grid_for(num_keys, 256, 4096), 256>>>((int*)s->own, num_keys, NUPS_OWNER_DEFAULT);
     }
     cudaError_t e = cudaDeviceSynchronize();
     if (e != cudaSuccess) {
@@ -197,8 +203,8 @@ extern "C" nups_status nups_destroy(nups_store* s)
     for (int i = 0; i < NUPS_MAX_HANDLES; ++i) cudaFree(s->handle[i].buf);
     for (int i = 0; i < NUPS_MAX_DISTS; ++i) { cudaFree(s->dist[i].table); cudaFree(s->dist[i].off); }
     cudaFree(s->val); cudaFree(s->acc); cudaFree(s->hot_bits); cudaFree(s->slot_of); cudaFree(s->hot_keys);
-    cudaFree(s->dval); cudaFree(s->dacc); cudaFree(s->dirty); cudaFree(s->cnt); cudaFree(s->owner);
-    cudaFree(s->pending); cudaFree(s->st); cudaFree(s->loss_partial); cudaFree(s->scratch); cudaFree(s->req_keys); cudaFree(s->negs_buf);
+    cudaFree(s->dval); cudaFree(s->dacc); cudaFree(s->dirty); cudaFree(s->cnt); cudaFree(s->own);
+    cudaFree(s->st); cudaFree(s->loss_partial); cudaFree(s->scratch); cudaFree(s->negs_buf);
     if (s->ev) {
         for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) cudaEventDestroy(s->ev[i]);
         free(s->ev);
@@ -1162,52 +1168,25 @@ extern "C" nups_status nups_get_hot(nups_store* s, uint64_t* h_n_out, uint32_t* 
 // ---------------------------------------------------------------------------------------------
 // ownership (the one-machine reading of "allocated at node q")
 // ---------------------------------------------------------------------------------------------
-__global__ void localize_request_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, uint32_t* req,
-                                        uint64_t req_cap)
+__global__ void localize_request_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n)
 {
     uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool in = i < n;
-    const uint32_t k = in ? keys[i] : 0u;
-    const bool ok = in && k < v.num_keys;
-    if (in && !ok) flag_bad_key(v);
-    queue_localize(v, ok, k, ok ? worker_of_item(i, n, v.R) : 0u, req, req_cap);
-}
-
-// requests of one call are applied in the order they were made, so the last one wins; workers are
-// visited in ascending order by every caller, hence the largest requesting worker gets the key
-__global__ void localize_apply_kernel(View v, const uint32_t* __restrict__ req, uint64_t max_requests)
-{
-    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= max_requests || i >= v.st->req_count) return;
-    uint32_t k = req[i];
-    int p = v.pending[k];
-    if (p >= 0) {
-        if (!key_is_hot(v, k)) v.owner[k] = (uint8_t)p;
-        v.pending[k] = -1;
-    }
-}
-__global__ void reset_req_kernel(DevStat* st) { st->req_count = 0; }
-
-nups_status nups_localize_apply(nups_store* s, uint64_t max_requests, cudaStream_t st)
-{
-    if (!s->owner || max_requests == 0) return NUPS_OK;
-    localize_apply_kernel<<<grid_for(max_requests, 256), 256, 0, st>>>(nups_view(s), s->req_keys, max_requests);
-    LAUNCH_CHECK(s);
-    reset_req_kernel<<<1, 1, 0, st>>>(s->st);
-    LAUNCH_CHECK(s);
-    return NUPS_OK;
+    if (i >= n) return;
+    const uint32_t k = keys[i];
+    if (k >= v.num_keys) { flag_bad_key(v); return; }
+    mark_localize(v, k, worker_of_item(i, n, v.R));
 }
 
 extern "C" nups_status nups_localize(nups_store* s, const uint32_t* d_keys, uint64_t n, void* stream)
 {
     if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
-    if (!s->owner || n == 0) return NUPS_OK;
+    if (!s->own || n == 0) return NUPS_OK;
     cudaStream_t st = (cudaStream_t)stream;
-    nups_status rc = nups_req_reserve(s, n);
+    nups_status rc = nups_new_epoch(s, st);
     if (rc != NUPS_OK) return rc;
-    localize_request_kernel<<<grid_for(n, 256), 256, 0, st>>>(nups_view(s), d_keys, n, s->req_keys, s->req_cap);
+    localize_request_kernel<<<grid_for(n, 256), 256, 0, st>>>(nups_view(s), d_keys, n);
     LAUNCH_CHECK(s);
-    return nups_localize_apply(s, n, st);
+    return NUPS_OK;
 }
 
 __global__ void owner_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, int* __restrict__ out)
@@ -1218,8 +1197,8 @@ __global__ void owner_kernel(View v, const uint32_t* __restrict__ keys, uint64_t
     int r;
     if (k >= v.num_keys) r = -1;
     else if (key_is_hot(v, k)) r = -2;
-    else if (!v.owner) r = -3;
-    else r = v.owner[k] == NUPS_OWNER_DEFAULT ? (int)(k % v.R) : (int)v.owner[k];
+    else if (!v.own) r = -3;
+    else r = (v.own[k] & 0xFFu) == NUPS_OWNER_DEFAULT ? (int)(k % v.R) : (int)(v.own[k] & 0xFFu);
     out[i] = r;
 }
 

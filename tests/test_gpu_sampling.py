@@ -113,3 +113,30 @@ def test_large_sample_frequencies_match_target():
     for q in (0, 3, 7):
         for i in (0, 1, 12345, N // 8 - 1):
             assert ks[q * (N // 8) + i] == o.draw_iid(do, q, i)
+
+
+@pytest.mark.parametrize("level", [LONGTERM, NONCONFORM, BOUNDED])
+def test_large_handles_with_most_keys_taken_by_other_workers(level):
+    # sub-handles longer than one round of the postponing walk; between the partial pulls nearly every key
+    # is moved away, so a small pull has to walk far past the stretch whose locality was looked up ahead
+    nk, L, R = 150_000, 4, 4
+    rng = np.random.default_rng(3)
+    w = inputs.zipf_integer_weights(120_000, 0.7).numpy().astype(np.uint32)
+    o, s = make_pair(nk, L, R=R, track_ownership=True)
+    hot = rng.choice(nk, 50, replace=False).astype(np.uint32)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(1000, w, 120_000, level, U=4, G=250, seed=21)
+    ds = s.register_distribution(1000, dev_keys(w), 120_000, level, U=4, G=250, seed=21)
+    N = 400_000
+    ho, hs = o.prepare_sample(do, N), s.prepare_sample(ds, N)
+    for c in (100, 5_000, 150_000, 1, 244_899):
+        moved = rng.permutation(nk).astype(np.uint32)[: nk - 2000]
+        o.localize(moved)
+        s.localize(dev_keys(moved))
+        ko = o.pull_sample(ho, c, values=False)
+        ks = s.pull_sample(hs, c, values=False)
+        assert np.array_equal(host_keys(ks), ko)
+    allk = np.arange(nk, dtype=np.uint32)
+    assert np.array_equal(s.owner_of(dev_keys(allk)).cpu().numpy(), np.array([o.owner_of(k) for k in allk]))
+    assert s.status_check() == 0
