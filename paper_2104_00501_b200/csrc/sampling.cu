@@ -220,19 +220,21 @@ __device__ __forceinline__ uint32_t draw_iid(const DrawParams& p, uint32_t q, un
     return p.key_base + (uint32_t)j;
 }
 
-// Handle buffer layout (device): keys[N] (u32) | post[N] (u32) | state[R] (uint4) | flags (one bit per entry)
+// Handle buffer layout (device): keys[N] (u32) | post[N] (u32) | state[3][R] (uint4) | flags | prefix
 struct HandleView {
     uint32_t* keys;
-    uint32_t* post;
-    uint4* state;      // LONG-TERM per sub-handle: x = walk position, y = postponed head, z = postponed tail,
-                       // w = postponed tail before the most recent call
-    uint32_t* flags;   // LONG-TERM: "is local" bit of the fresh entries that the running call may reach;
-                       // sub-handle q owns the words from (b_q / 32) + q on, so no two share a word
+    uint32_t* post;    // LONG-TERM: postponed entries of each sub-handle, in the order they were postponed
+    uint4* state;      // LONG-TERM per sub-handle: x = walk position, y = postponed head, z = postponed tail
+    uint4* prev;       //   the state before the running call
+    uint4* walk;       //   what the running call does: x = fresh entries walked, y = of those local,
+                       //   z = postponed entries emitted
+    uint32_t* flags;   // LONG-TERM: "is local" bit of every fresh entry, and the number of local entries before
+    uint32_t* prefix;  //   each 32-entry word; sub-handle q owns the words from (b_q / 32) + q on
 };
 static size_t handle_bytes(uint64_t N, uint32_t R, int level)
 {
     size_t b = align256(N * 4);
-    if (level == NUPS_LONGTERM) b += align256(N * 4) + align256((size_t)R * 16) + align256((N / 32 + R + 2) * 4);
+    if (level == NUPS_LONGTERM) b += align256(N * 4) + 3 * align256((size_t)R * 16) + 2 * align256((N / 32 + R + 2) * 4);
     return b;
 }
 static HandleView handle_view(char* buf, uint64_t N, uint32_t R)
@@ -241,59 +243,84 @@ static HandleView handle_view(char* buf, uint64_t N, uint32_t R)
     h.keys = (uint32_t*)buf; buf += align256(N * 4);
     h.post = (uint32_t*)buf; buf += align256(N * 4);
     h.state = (uint4*)buf; buf += align256((size_t)R * 16);
-    h.flags = (uint32_t*)buf;
+    h.prev = (uint4*)buf; buf += align256((size_t)R * 16);
+    h.walk = (uint4*)buf; buf += align256((size_t)R * 16);
+    h.flags = (uint32_t*)buf; buf += align256((N / 32 + R + 2) * 4);
+    h.prefix = (uint32_t*)buf;
     return h;
 }
 
 // Local sampling: the first key local to worker q among the candidate k0 and the 63 keys after it
 // (wrapping inside the distribution's key range), else k0.  The candidates are consecutive keys, so
-// their ownership words are consecutive too: they are read sixteen at a time with 128-bit loads (most
-// walks end within the first sixteen), and their technique bits lie in at most three words.
-__device__ __forceinline__ uint32_t first_local(const View& v, const DrawParams& p, uint32_t q, uint32_t k0)
+// their ownership words are consecutive too.  Four lanes serve one candidate: each reads the four words
+// of its part of a 16-key group with one 128-bit load (the four loads of a candidate fall into one cache
+// line, so a warp instruction touches 8 lines instead of 32), and the walk goes group by group until
+// a local key shows up (most walks end within the first group).
+// Called by all four lanes of a quad with the same arguments; whole warps must call.
+__device__ __forceinline__ uint32_t first_local_quad(const View& v, const DrawParams& p, uint32_t q, uint32_t k0,
+                                                     bool active)
 {
-    if (!v.own) return k0;
-    const unsigned long long rel = k0 - p.key_base;
+    const unsigned sub = threadIdx.x & 3;
     const uint32_t R = v.R;
-    const uint64_t a0 = (uint64_t)k0 & ~3ull;                // 16-byte aligned start
-    if (rel + NUPS_LOCAL_PROBES <= p.n && a0 + NUPS_LOCAL_PROBES + 16 <= v.num_keys) {
-        // bit j of `hot` belongs to key 32 * (k0 / 32) + j
-        uint32_t h0 = 0, h1 = 0, h2 = 0;
-        if (v.H) {
-            const uint64_t w0 = (uint64_t)k0 >> 5, wlast = ((uint64_t)k0 + NUPS_LOCAL_PROBES - 1) >> 5;
-            h0 = __ldg(v.hot_bits + w0);
-            if (w0 + 1 <= wlast) h1 = __ldg(v.hot_bits + w0 + 1);
-            if (w0 + 2 <= wlast) h2 = __ldg(v.hot_bits + w0 + 2);
+    uint32_t result = k0;
+    bool searching = active && v.own != nullptr;
+    const unsigned long long rel = k0 - p.key_base;
+    const uint32_t a0 = k0 & ~3u;                            // 16-byte aligned start
+    if (searching && !(rel + NUPS_LOCAL_PROBES <= p.n && (uint64_t)a0 + NUPS_LOCAL_PROBES + 16 <= v.num_keys)) {
+        // near the end of the key range: probe one key at a time
+        for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
+            const uint32_t cand = p.key_base + (uint32_t)((rel + probe) % p.n);
+            if (key_is_local(v, q, cand)) { result = cand; break; }
         }
-        const uint4* op = reinterpret_cast<const uint4*>(v.own + a0);
-        uint32_t res = (uint32_t)(a0 % R);                   // key mod R of the key looked at, kept by counting
-        const uint32_t hbase = k0 & ~31u;
-        for (int g = 0; g < 5; ++g) {                        // keys a0 + 16 g ... a0 + 16 g + 15
-            uint4 o4[4];
+        searching = false;
+    }
+    const uint32_t res0 = searching ? a0 % R : 0u;           // key mod R of key a0
+    for (uint32_t g = 0; g < NUPS_LOCAL_PROBES / 16 + 1; ++g) {
+        if (!__any_sync(0xFFFFFFFFu, searching)) break;
+        uint32_t m = 0;                                      // bit t: my key t is a candidate and local
+        const uint32_t kb = a0 + 16 * g + 4 * sub;           // my four keys: kb ... kb + 3
+        if (searching) {
+            const uint4 o = __ldg(reinterpret_cast<const uint4*>(v.own + kb));
+            const uint32_t hw = v.H ? __ldg(v.hot_bits + (kb >> 5)) >> (kb & 31) : 0u;     // replicated: local to all
+            uint32_t r = (res0 + 16 * g + 4 * sub) % R;
 #pragma unroll
-            for (int u = 0; u < 4; ++u) o4[u] = __ldg(op + g * 4 + u);
-            uint32_t found = 0;                              // bit t: key a0 + 16 g + t is a candidate and local
-#pragma unroll
-            for (int t = 0; t < 16; ++t) {
-                const uint4 o = o4[t >> 2];
-                const uint32_t w = (t & 3) == 0 ? o.x : (t & 3) == 1 ? o.y : (t & 3) == 2 ? o.z : o.w;
-                const uint32_t key = (uint32_t)a0 + g * 16 + t;
+            for (int t = 0; t < 4; ++t) {
+                const uint32_t w = t == 0 ? o.x : t == 1 ? o.y : t == 2 ? o.z : o.w;
                 const uint32_t ob = w & 0xFFu;
-                bool loc = (ob == NUPS_OWNER_DEFAULT ? res : ob) == q;
-                const uint32_t hb = key - hbase;             // 0 .. 95 for candidates
-                const uint32_t hw = hb < 32 ? h0 : hb < 64 ? h1 : h2;
-                loc = loc || ((hw >> (hb & 31)) & 1u);
-                if (loc && key >= k0 && key < k0 + NUPS_LOCAL_PROBES) found |= 1u << t;
-                res = res + 1 == R ? 0 : res + 1;
+                const bool loc = (ob == NUPS_OWNER_DEFAULT ? r : ob) == q || ((hw >> t) & 1u);
+                const uint32_t key = kb + t;
+                if (loc && key >= k0 && key - k0 < NUPS_LOCAL_PROBES) m |= 1u << t;
+                r = r + 1 == R ? 0u : r + 1;
             }
-            if (found) return (uint32_t)a0 + g * 16 + (__ffs(found) - 1);
+            m <<= 4 * sub;
         }
-        return k0;
+        m |= __shfl_xor_sync(0xFFFFFFFFu, m, 1);
+        m |= __shfl_xor_sync(0xFFFFFFFFu, m, 2);
+        if (searching && m) {
+            result = a0 + 16 * g + (uint32_t)(__ffs(m) - 1);
+            searching = false;
+        }
     }
-    for (uint32_t probe = 0; probe < NUPS_LOCAL_PROBES; ++probe) {
-        const uint32_t cand = p.key_base + (uint32_t)((rel + probe) % p.n);
-        if (key_is_local(v, q, cand)) return cand;
+    return result;
+}
+
+// one candidate per lane: the quads take the warp's candidates eight at a time
+__device__ __forceinline__ uint32_t first_local_warp(const View& v, const DrawParams& p, uint32_t q, uint32_t k0,
+                                                     bool active)
+{
+    const unsigned lane = threadIdx.x & 31;
+    uint32_t mine = k0;
+#pragma unroll
+    for (int r = 0; r < 4; ++r) {
+        const int src = 8 * r + (int)(lane >> 2);
+        const uint32_t kk = __shfl_sync(0xFFFFFFFFu, k0, src);
+        const uint32_t qq = __shfl_sync(0xFFFFFFFFu, q, src);
+        const bool act = __shfl_sync(0xFFFFFFFFu, (int)active, src) != 0;
+        const uint32_t res = first_local_quad(v, p, qq, kk, act);
+        const uint32_t back = __shfl_sync(0xFFFFFFFFu, res, 4 * (int)(lane & 7));
+        if ((int)(lane >> 3) == r) mine = back;
     }
-    return k0;
+    return mine;
 }
 
 // independent draws: one thread per sample.  The advanced stream offsets go to the other half of the
@@ -315,20 +342,22 @@ __global__ void draw_iid_kernel(View v, DrawParams p, const unsigned long long* 
 
 // Pooled reuse: pool `pl` of a worker holds G iid draws and is walked U times, each pass in a fresh
 // Fisher-Yates order.  Stream position s lies in pass number s / G overall (pool = pass / U).
-// One block visits one pool: it draws the pool once, then each warp produces whole passes: the
-// shuffle itself is sequential (one lane), the random words and the output are warp-wide.
-// Shared memory: pool[G] | per warp xs[G] | per warp perm[G] (16-bit).
+// One block visits one pool: it draws the pool once, then shuffles up to T passes at a time.  A shuffle
+// is a chain of dependent swaps, so each of the T passes gets one thread, and the passes' arrays are
+// interleaved ([element][pass]) so that the threads of a warp work side by side in shared memory;
+// drawing the swap partners and writing the output are block-wide.
+// Shared memory: pool[G] (u32) | partner[G][T] (u16) | perm[G][T] (u16).
+constexpr unsigned REUSE_THREADS = 256;
 struct ReuseShape {
-    unsigned warps;
+    unsigned T;
     size_t smem;
 };
 static ReuseShape reuse_shape(uint32_t U, uint32_t G)
 {
     ReuseShape r;
-    r.warps = G > 512 ? 4 : 8;
-    if (r.warps > U) r.warps = U;
-    if (r.warps < 1) r.warps = 1;
-    r.smem = (size_t)G * 4 + (size_t)r.warps * G * 4 + (((size_t)r.warps * G * 2 + 15) / 16) * 16;
+    r.T = U < 32 ? U : 32;
+    while (r.T > 1 && (size_t)r.T * G * 4 > 40 * 1024) r.T--;
+    r.smem = (size_t)G * 4 + (size_t)r.T * G * 4;
     return r;
 }
 static unsigned reuse_pools(uint64_t max_size, uint32_t U, uint32_t G)
@@ -338,53 +367,75 @@ static unsigned reuse_pools(uint64_t max_size, uint32_t U, uint32_t G)
 
 template <class Emit>
 __device__ __forceinline__ void reuse_pool_visit(const DrawParams& p, uint32_t q, unsigned long long s0,
-                                                 unsigned long long s1, Emit emit)
+                                                 unsigned long long s1, uint32_t T, Emit emit)
 {
     extern __shared__ __align__(16) uint32_t reuse_mem[];
     const uint32_t G = p.G, U = p.U;
-    const unsigned lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    const unsigned tid = threadIdx.x;
     const unsigned long long span = (unsigned long long)U * G;
     const unsigned long long pl = s0 / span + blockIdx.x;
     if (pl * span >= s1) return;
     uint32_t* pool = reuse_mem;
-    uint32_t* xs = reuse_mem + G + (size_t)warp * G;
-    uint16_t* perm = reinterpret_cast<uint16_t*>(reuse_mem + G + (size_t)nwarps * G) + (size_t)warp * G;
-    for (uint32_t m = threadIdx.x; m < G; m += blockDim.x) pool[m] = draw_iid(p, q, pl * G + m);
-    __syncthreads();
-    for (uint32_t t = warp; t < U; t += nwarps) {
-        const unsigned long long pass = pl * U + t, lo = pass * G;
-        if (lo + G <= s0 || lo >= s1) continue;
-        // random words of the shuffle: word d of the pass's Philox stream (purpose 1), four per block
-        for (uint32_t blk = lane; blk * 4 + 1 < G; blk += 32) {
+    uint16_t* partner = reinterpret_cast<uint16_t*>(reuse_mem + G);
+    uint16_t* perm = partner + (size_t)T * G;
+    for (uint32_t m = tid; m < G; m += blockDim.x) pool[m] = draw_iid(p, q, pl * G + m);
+    const uint32_t blocks_per_pass = (G + 2) / 4;            // Philox blocks that hold the G - 1 shuffle words
+    for (uint32_t t0 = 0; t0 < U; t0 += T) {
+        const uint32_t nt = U - t0 < T ? U - t0 : T;
+        const unsigned long long pass0 = pl * U + t0;
+        if ((pass0 + nt) * G <= s0 || pass0 * G >= s1) continue;          // none of these passes is asked for
+        __syncthreads();
+        // swap partners: step i = G-1 ... 1 of a pass swaps i with mulhi(x, i + 1), x = word G-1-i of the
+        // pass's Philox stream (purpose 1, four words per block)
+        for (uint32_t e = tid; e < nt * blocks_per_pass; e += blockDim.x) {
+            const uint32_t t = e / blocks_per_pass, blk = e % blocks_per_pass;
             uint32_t x[4];
-            philox_at(p.seed, pass, q, 1, blk, x);
+            philox_at(p.seed, pass0 + t, q, 1, blk, x);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (blk * 4 + k + 1 < G) xs[blk * 4 + k] = x[k];
-        }
-        for (uint32_t m = lane; m < G; m += 32) perm[m] = (uint16_t)m;
-        __syncwarp();
-        if (lane == 0) {
-            for (uint32_t i = G - 1; i >= 1; --i) {
-                const uint32_t r = __umulhi(xs[G - 1 - i], i + 1);
-                const uint16_t tmp = perm[i]; perm[i] = perm[r]; perm[r] = tmp;
+            for (int k = 0; k < 4; ++k) {
+                const uint32_t d = blk * 4 + k;
+                if (d + 1 < G) partner[(size_t)(G - 1 - d) * T + t] = (uint16_t)__umulhi(x[k], G - d);
             }
         }
-        __syncwarp();
-        for (uint32_t j0 = 0; j0 < G; j0 += 32) {             // whole warps: emit may ballot
-            const uint32_t j = j0 + lane;
-            const unsigned long long sp = lo + j;
-            const bool in = j < G && sp >= s0 && sp < s1;
-            const uint32_t k = in ? pool[perm[j]] : 0u;
+        for (uint32_t e = tid; e < nt * G; e += blockDim.x) perm[(size_t)(e / nt) * T + e % nt] = (uint16_t)(e / nt);
+        __syncthreads();
+        if (tid < nt) {
+            // the swaps depend on one another; their partners do not and are fetched eight at a time
+            uint16_t* pm = perm + tid;
+            const uint16_t* pa = partner + tid;
+            uint32_t i = G - 1;
+            for (; i >= 8; i -= 8) {
+                uint32_t r[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) r[k] = pa[(size_t)(i - k) * T];
+#pragma unroll
+                for (int k = 0; k < 8; ++k) {
+                    const uint16_t tmp = pm[(size_t)(i - k) * T];
+                    pm[(size_t)(i - k) * T] = pm[(size_t)r[k] * T];
+                    pm[(size_t)r[k] * T] = tmp;
+                }
+            }
+            for (; i >= 1; --i) {
+                const uint32_t r = pa[(size_t)i * T];
+                const uint16_t tmp = pm[(size_t)i * T]; pm[(size_t)i * T] = pm[(size_t)r * T]; pm[(size_t)r * T] = tmp;
+            }
+        }
+        __syncthreads();
+        const uint32_t total = nt * G;
+        for (uint32_t e0 = 0; e0 < total; e0 += blockDim.x) {          // whole warps: emit may ballot
+            const uint32_t e = e0 + tid;
+            const uint32_t t = e / G, j = e % G;
+            const unsigned long long sp = (pass0 + t) * G + j;
+            const bool in = e < total && sp >= s0 && sp < s1;
+            const uint32_t k = in ? pool[perm[(size_t)j * T + t]] : 0u;
             emit(in, k, sp - s0);
         }
-        __syncwarp();
     }
 }
 
 __global__ void draw_reuse_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
                                   unsigned long long* __restrict__ off_next, HandleView h, uint64_t N, int localize,
-                                  int longterm)
+                                  int longterm, uint32_t T)
 {
     const uint32_t q = blockIdx.y, R = v.R;
     const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
@@ -394,7 +445,7 @@ __global__ void draw_reuse_kernel(View v, DrawParams p, const unsigned long long
         if (longterm) h.state[q] = make_uint4(0u, 0u, 0u, 0u);
     }
     if (size == 0) return;
-    reuse_pool_visit(p, q, s0, s0 + size, [&](bool in, uint32_t k, unsigned long long rel) {
+    reuse_pool_visit(p, q, s0, s0 + size, T, [&](bool in, uint32_t k, unsigned long long rel) {
         if (in) {
             h.keys[b0 + rel] = k;
             if (localize) mark_localize(v, k, q);
@@ -440,8 +491,8 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
     unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
     if (reuse) {
         const ReuseShape sh = reuse_shape(d.U, d.G);
-        draw_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R), sh.warps * 32, sh.smem, st>>>(
-            v, p, off_cur, off_next, hv, N, loc, d.level == NUPS_LONGTERM);
+        draw_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R), REUSE_THREADS, sh.smem, st>>>(
+            v, p, off_cur, off_next, hv, N, loc, d.level == NUPS_LONGTERM, sh.T);
     } else {
         draw_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(v, p, off_cur, off_next, hv, N, loc);
     }
@@ -486,92 +537,84 @@ __global__ void emit_kernel(View v, DrawParams p, HandleView h, uint64_t N, uint
     uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     bool in = o < n;
     uint32_t k = 0;
+    uint32_t q = 0;
     if (in) {
-        uint64_t pos = cursor + o;
-        k = h.keys[pos];
-        if (local_only) k = first_local(v, p, chunk_of_pos(pos, N, v.R), k);
-        out[o] = k;
+        k = h.keys[cursor + o];
+        if (local_only) q = chunk_of_pos(cursor + o, N, v.R);
     }
+    if (local_only) k = first_local_warp(v, p, q, k, in);
+    if (in) out[o] = k;
     count_sample(v, k, in);
 }
 
 // Reuse with postponing.  Entries of a sub-handle not yet postponed are taken in list order: a local
 // one is emitted, a non-local one is re-localized and appended to the sub-handle's postponed queue;
-// when the fresh entries run out the postponed ones are emitted.  Locality is judged by the
-// ownership at the start of the call.
-// The ownership lookups are scattered reads, so they are done ahead of the walk by a kernel that
-// spreads them over the whole GPU (one bit per entry); the walk itself, one block per sub-handle,
-// then only streams keys and bits.  The lookup covers the fresh entries that the call is likely to
-// reach (twice what it must emit, plus a margin); should the walk go further, it looks up the rest itself.
-constexpr int LT_THREADS = 1024;
-constexpr uint64_t LT_MARGIN = 4096;
-
-__device__ __forceinline__ uint64_t lt_window(uint64_t oc, uint64_t size, uint64_t take)
+// the walk stops right after the last entry it must emit, and when the fresh entries run out the
+// postponed ones are emitted.  Locality is judged by the ownership at the start of the call.
+// Where an entry goes depends only on how many local entries lie before it, so the walk is a
+// prefix sum, not a loop: (1) one bit per fresh entry, looked up by the whole GPU; (2) per sub-handle,
+// a scan of the bit counts that also finds where the walk stops; (3) every entry is placed on its
+// own; (4) postponed entries are emitted where needed and what was postponed moves to its worker.
+struct LtChunk {
+    uint32_t q;
+    uint64_t b0, size, take, out_base;
+    bool active;
+};
+__device__ __forceinline__ LtChunk lt_chunk(uint32_t q, uint64_t N, uint32_t R, uint64_t cursor, uint64_t n)
 {
-    const uint64_t w = 2 * take + LT_MARGIN;
-    return w < size - oc ? w : size - oc;
+    LtChunk c;
+    c.q = q;
+    c.b0 = chunk_begin(q, N, R);
+    const uint64_t b1 = chunk_begin(q + 1, N, R);
+    const uint64_t lo = max(c.b0, cursor), hi = min(b1, cursor + n);
+    c.active = lo < hi;
+    c.size = b1 - c.b0;
+    c.take = c.active ? hi - lo : 0;
+    c.out_base = c.active ? lo - cursor : 0;
+    return c;
 }
 
 __global__ void lt_flags_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
 {
-    const uint32_t q = q_first + blockIdx.y;
+    const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
+    if (!c.active) return;
     const unsigned lane = threadIdx.x & 31;
-    const uint64_t b0 = chunk_begin(q, N, v.R), b1 = chunk_begin(q + 1, N, v.R);
-    const uint64_t lo = max(b0, cursor), hi = min(b1, cursor + n);
-    if (lo >= hi) return;
-    const uint64_t size = b1 - b0, oc = h.state[q].x;
-    if (oc >= size) return;
-    const uint64_t w_end = (oc + lt_window(oc, size, hi - lo) + 31) >> 5;
+    const uint64_t oc = h.state[c.q].x;
     const uint64_t word = (oc >> 5) + (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
-    if (word >= w_end) return;
+    if (word * 32 >= c.size) return;
     const uint64_t i = word * 32 + lane;
-    const bool loc = i < size && key_is_local(v, q, h.keys[b0 + i]);
+    const bool loc = i >= oc && i < c.size && key_is_local(v, c.q, h.keys[c.b0 + i]);
     const unsigned bits = __ballot_sync(0xFFFFFFFFu, loc);
-    if (lane == 0) h.flags[(b0 >> 5) + q + word] = bits;
+    if (lane == 0) h.flags[(c.b0 >> 5) + c.q + word] = bits;
 }
 
+constexpr int LT_THREADS = 1024;
+constexpr int LT_WORDS = 4;                  // flag words per thread and round of the scan
+
 __global__ void __launch_bounds__(LT_THREADS)
-longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
-                uint32_t* __restrict__ out)
+lt_scan_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
 {
     __shared__ unsigned warp_tot[LT_THREADS / 32];
-    __shared__ unsigned sh_consumed, sh_local;
-    const uint32_t q = q_first + blockIdx.x;
+    __shared__ unsigned long long sh_stop;       // walk position right after the last entry that must be emitted
+    const LtChunk c = lt_chunk(q_first + blockIdx.x, N, v.R, cursor, n);
+    if (!c.active) return;
     const unsigned tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint64_t b0 = chunk_begin(q, N, v.R), b1 = chunk_begin(q + 1, N, v.R);
-    const uint64_t lo = max(b0, cursor), hi = min(b1, cursor + n);
-    if (lo >= hi) return;
-    const uint64_t take = hi - lo, size = b1 - b0;
-    const uint64_t out_base = lo - cursor;
-    const uint4 stt = h.state[q];
-    uint64_t oc = stt.x, ph = stt.y, pt = stt.z, emitted = 0;
-    const uint64_t pt0 = pt;
-    const uint64_t w_known = oc < size ? (oc + lt_window(oc, size, take) + 31) >> 5 : 0;   // bits below were looked up
-    const uint32_t* flags = h.flags + (b0 >> 5) + q;
-    while (emitted < take && oc < size) {
-        // a round looks at the 32 * LT_THREADS entries from the word of `oc` on, in list order: lane l of
-        // warp w holds the bits of word 32 w + l of the round
-        const uint64_t word0 = (oc >> 5) + (uint64_t)warp * 32;
-        const uint64_t myword = word0 + lane, e0 = myword * 32;
-        uint32_t valid = 0;                       // entries of my word inside [oc, size)
-        if (e0 + 32 > oc && e0 < size) {
-            valid = 0xFFFFFFFFu;
-            if (e0 < oc) valid &= 0xFFFFFFFFu << (unsigned)(oc - e0);
-            if (e0 + 32 > size) valid &= 0xFFFFFFFFu >> (unsigned)(e0 + 32 - size);
+    const uint4 stt = h.state[c.q];
+    const uint64_t oc = stt.x, ph = stt.y, pt = stt.z;
+    const uint64_t w0 = oc >> 5, w1 = oc < c.size ? (c.size + 31) >> 5 : w0;
+    const uint32_t* flags = h.flags + (c.b0 >> 5) + c.q;
+    uint32_t* prefix = h.prefix + (c.b0 >> 5) + c.q;
+    if (tid == 0) sh_stop = ~0ull;
+    unsigned long long carry = 0;                // local entries before the round
+    for (uint64_t base = w0; base < w1 && carry < c.take; base += (uint64_t)LT_THREADS * LT_WORDS) {
+        uint32_t bits[LT_WORDS];
+        unsigned mine = 0;
+#pragma unroll
+        for (int k = 0; k < LT_WORDS; ++k) {
+            const uint64_t w = base + (uint64_t)tid * LT_WORDS + k;
+            bits[k] = w < w1 ? flags[w] : 0u;
+            mine += __popc(bits[k]);
         }
-        uint32_t bits = (valid && myword < w_known) ? flags[myword] : 0u;
-        unsigned missing = __ballot_sync(0xFFFFFFFFu, valid != 0 && myword >= w_known);
-        while (missing) {
-            const int w = __ffs(missing) - 1;
-            missing &= missing - 1;
-            const uint64_t i = (word0 + w) * 32 + lane;
-            const bool loc = i < size && key_is_local(v, q, h.keys[b0 + i]);
-            const unsigned b = __ballot_sync(0xFFFFFFFFu, loc);
-            if ((int)lane == w) bits = b;
-        }
-        bits &= valid;
-        // exclusive count of local entries before this lane's word
-        const unsigned mine = __popc(bits);
         unsigned inc = mine;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -579,67 +622,81 @@ longterm_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, u
             if (lane >= (unsigned)o) inc += y;
         }
         if (lane == 31) warp_tot[warp] = inc;
-        if (tid == 0) { sh_consumed = 0; sh_local = 0; }
         __syncthreads();
-        unsigned long long wexcl = 0;
-        for (unsigned w = 0; w < warp; ++w) wexcl += warp_tot[w];
-        const unsigned wpre = inc - mine;
-        const uint64_t need = take - emitted;
-        unsigned nc = 0, nl = 0;
-        for (int w = 0; w < 32; ++w) {
-            const uint32_t vb = __shfl_sync(0xFFFFFFFFu, valid, w);
-            if (vb == 0) continue;
-            const uint32_t wb = __shfl_sync(0xFFFFFFFFu, bits, w);
-            const unsigned pre = __shfl_sync(0xFFFFFFFFu, wpre, w);
-            const uint64_t i = (word0 + w) * 32 + lane;
-            const bool have = (vb >> lane) & 1u, loc = (wb >> lane) & 1u;
-            // the walk stops right after the need-th local entry: an entry is reached iff fewer than
-            // `need` local entries lie before it
-            const unsigned long long before = wexcl + pre + __popc(wb & ((1u << lane) - 1u));
-            const bool consumed = have && before < need;
-            uint32_t key = 0;
-            if (consumed) {
-                key = h.keys[b0 + i];
-                if (loc) out[out_base + emitted + before] = key;
-                else {
-                    h.post[b0 + pt + ((i - oc) - before)] = key;              // non-local entries before it
-                }
-            }
-            nc += __popc(__ballot_sync(0xFFFFFFFFu, consumed));
-            nl += __popc(__ballot_sync(0xFFFFFFFFu, consumed && loc));
-            count_sample(v, key, consumed && loc);
+        unsigned long long before = carry + (inc - mine);
+        unsigned total = 0;
+        for (unsigned w = 0; w < LT_THREADS / 32; ++w) {
+            if (w < warp) before += warp_tot[w];
+            total += warp_tot[w];
         }
-        if (lane == 0 && nc) { atomicAdd(&sh_consumed, nc); atomicAdd(&sh_local, nl); }
-        __syncthreads();
-        const unsigned tc = sh_consumed, tl = sh_local;
-        emitted += tl; pt += tc - tl; oc += tc;
+#pragma unroll
+        for (int k = 0; k < LT_WORDS; ++k) {
+            const uint64_t w = base + (uint64_t)tid * LT_WORDS + k;
+            if (w < w1) prefix[w] = (uint32_t)before;
+            const unsigned cnt = __popc(bits[k]);
+            if (before < c.take && c.take <= before + cnt) {
+                // the take-th local entry is the (take - before)-th set bit of this word
+                uint32_t b = bits[k];
+                for (unsigned long long skip = c.take - before - 1; skip; --skip) b &= b - 1;
+                sh_stop = w * 32 + (unsigned)(__ffs(b) - 1) + 1;
+            }
+            before += cnt;
+        }
+        carry += total;
         __syncthreads();
     }
     __syncthreads();
-    if (emitted < take) {
-        const uint64_t cnt = take - emitted;
-        for (uint64_t i = tid; i < ((cnt + LT_THREADS - 1) / LT_THREADS) * LT_THREADS; i += LT_THREADS) {
-            const bool in = i < cnt;
-            const uint32_t key = in ? h.post[b0 + ph + i] : 0u;
-            if (in) out[out_base + emitted + i] = key;
-            count_sample(v, key, in);
-        }
-        ph += cnt;
+    if (tid == 0) {
+        const uint64_t fresh = oc < c.size ? c.size - oc : 0;
+        const uint64_t tc = carry >= c.take ? (uint64_t)sh_stop - oc : fresh;      // fresh entries walked
+        const uint64_t tl = carry >= c.take ? c.take : (uint64_t)carry;             // of those local = emitted
+        const uint64_t cnt = c.take - tl;                                           // postponed entries emitted
+        h.prev[c.q] = stt;
+        h.walk[c.q] = make_uint4((unsigned)tc, (unsigned)tl, (unsigned)cnt, 0u);
+        h.state[c.q] = make_uint4((unsigned)(oc + tc), (unsigned)(ph + cnt), (unsigned)(pt + tc - tl), 0u);
     }
-    if (tid == 0) h.state[q] = make_uint4((unsigned)oc, (unsigned)ph, (unsigned)pt, (unsigned)pt0);
 }
 
-// the entries that the walk just postponed move to their worker (when the call ends: the walk itself
-// judged locality by the ownership from before the call)
-__global__ void lt_localize_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
+__global__ void lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
+                                uint32_t* __restrict__ out)
 {
-    const uint32_t q = q_first + blockIdx.y;
-    const uint64_t b0 = chunk_begin(q, N, v.R), b1 = chunk_begin(q + 1, N, v.R);
-    if (max(b0, cursor) >= min(b1, cursor + n)) return;
-    const uint4 stt = h.state[q];
-    const uint64_t rel = (uint64_t)stt.w + (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (rel >= stt.z) return;
-    mark_localize(v, h.post[b0 + rel], q);
+    const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
+    if (!c.active) return;
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t oc = h.prev[c.q].x, pt = h.prev[c.q].z, end = oc + h.walk[c.q].x;
+    const uint64_t word = (oc >> 5) + (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
+    if (word * 32 >= end) return;
+    const uint64_t i = word * 32 + lane;
+    const bool walked = i >= oc && i < end;
+    const uint32_t bits = h.flags[(c.b0 >> 5) + c.q + word];
+    const uint64_t before = (uint64_t)h.prefix[(c.b0 >> 5) + c.q + word] + __popc(bits & ((1u << lane) - 1u));
+    const bool loc = (bits >> lane) & 1u;
+    uint32_t key = 0;
+    if (walked) {
+        key = h.keys[c.b0 + i];
+        if (loc) out[c.out_base + before] = key;
+        else h.post[c.b0 + pt + ((i - oc) - before)] = key;          // non-local entries before it
+    }
+    count_sample(v, key, walked && loc);
+}
+
+__global__ void lt_finish_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
+                                 uint32_t* __restrict__ out)
+{
+    const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
+    if (!c.active) return;
+    const uint4 pv = h.prev[c.q], wk = h.walk[c.q];
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const bool in = t < wk.z;                                       // a postponed entry to emit
+    uint32_t key = 0;
+    if (in) {
+        key = h.post[c.b0 + pv.y + t];
+        out[c.out_base + wk.y + t] = key;
+    }
+    count_sample(v, key, in);
+    // what this call postponed moves to the worker (when the call ends: the walk judged locality by
+    // the ownership from before the call)
+    if (t < (uint64_t)wk.x - wk.y) mark_localize(v, h.post[c.b0 + pv.z + t], c.q);
 }
 
 static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_keys_out, float* d_vals_out,
@@ -657,24 +714,22 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
     HandleView hv = handle_view(h.buf, h.N, s->R);
     DrawParams p = draw_params(d);
     if (d.level == NUPS_LONGTERM) {
-        // sub-handles overlapped by [cursor, cursor + n), and the most that one of them must emit
+        // sub-handles overlapped by [cursor, cursor + n)
         uint32_t qf = 0, ql = 0;
-        uint64_t max_take = 0;
         for (uint32_t q = 0; q < s->R; ++q) {
             uint64_t b0 = ((uint64_t)q * h.N) / s->R, b1 = ((uint64_t)(q + 1) * h.N) / s->R;
             if (b0 <= h.cursor && h.cursor < b1) qf = q;
             if (b0 <= h.cursor + n - 1 && h.cursor + n - 1 < b1) ql = q;
-            uint64_t lo = b0 > h.cursor ? b0 : h.cursor, hi = b1 < h.cursor + n ? b1 : h.cursor + n;
-            if (hi > lo && hi - lo > max_take) max_take = hi - lo;
         }
         const uint64_t max_size = (h.N + s->R - 1) / s->R;
-        uint64_t window = 2 * max_take + LT_MARGIN;
-        if (window > max_size) window = max_size;
-        lt_flags_kernel<<<dim3(grid_for(window / 32 + 2, 8), ql - qf + 1), 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
+        const dim3 by_word(grid_for(max_size / 32 + 2, 8), ql - qf + 1), by_entry(grid_for(max_size, 256), ql - qf + 1);
+        lt_flags_kernel<<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
         LAUNCH_CHECK(s);
-        longterm_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
+        lt_scan_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
         LAUNCH_CHECK(s);
-        lt_localize_kernel<<<dim3(grid_for(max_size, 256), ql - qf + 1), 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
+        lt_place_kernel<<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
+        LAUNCH_CHECK(s);
+        lt_finish_kernel<<<by_entry, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
         LAUNCH_CHECK(s);
     } else {
         emit_kernel<<<grid_for(n, 256), 256, 0, st>>>(v, p, hv, h.N, h.cursor, n, d.level == NUPS_NONCONFORM, d_keys_out);
@@ -717,7 +772,9 @@ __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long
         q = chunk_of_pos(o, N, v.R);
         const unsigned long long size = chunk_begin(q + 1, N, v.R) - chunk_begin(q, N, v.R);
         k = draw_iid(p, q, off_cur[q] + (unsigned long long)bt * size + (o - chunk_begin(q, N, v.R)));
-        if (local_only) k = first_local(v, p, q, k);
+    }
+    if (local_only) k = first_local_warp(v, p, q, k, in);
+    if (in) {
         out[o] = k;
         if (localize) mark_localize(v, k, q);
     }
@@ -729,7 +786,7 @@ __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long
 
 __global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
                                          unsigned long long* __restrict__ off_next, uint64_t N, uint32_t batches,
-                                         int localize, uint32_t* __restrict__ out)
+                                         int localize, uint32_t* __restrict__ out, uint32_t T)
 {
     const uint32_t q = blockIdx.y, R = v.R;
     if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
@@ -739,7 +796,7 @@ __global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned lo
     if (size == 0) return;
     out += (uint64_t)blockIdx.z * N;
     const unsigned long long s0 = off_cur[q] + (unsigned long long)blockIdx.z * size;
-    reuse_pool_visit(p, q, s0, s0 + size, [&](bool in, uint32_t k, unsigned long long rel) {
+    reuse_pool_visit(p, q, s0, s0 + size, T, [&](bool in, uint32_t k, unsigned long long rel) {
         if (in) {
             out[b0 + rel] = k;
             if (localize) mark_localize(v, k, q);
@@ -821,8 +878,8 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
     unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
     if (d.level == NUPS_BOUNDED) {
         const ReuseShape sh = reuse_shape(d.U, d.G);
-        draw_direct_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R, batches), sh.warps * 32, sh.smem,
-                                   st>>>(v, p, off_cur, off_next, N, batches, localize, s->negs_buf);
+        draw_direct_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R, batches), REUSE_THREADS, sh.smem,
+                                   st>>>(v, p, off_cur, off_next, N, batches, localize, s->negs_buf, sh.T);
     } else {
         draw_direct_iid_kernel<<<dim3(grid_for(N, 256), batches), 256, 0, st>>>(v, p, off_cur, off_next, N, batches,
                                                                               d.level == NUPS_NONCONFORM, localize,
