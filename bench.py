@@ -128,8 +128,8 @@ def make_sgns_data(device, n_batches, seed=0, store=None):
     return c, o, counts, weights
 
 
-def build_store(binding, device, n_batches, seed, deterministic=False):
-    s = binding.Store(2 * VOCAB, DIM, workers=WORKERS, sync_interval=SYNC_EVERY, deterministic=deterministic,
+def build_store(binding, device, n_batches, seed, deterministic=False, sync_interval=SYNC_EVERY):
+    s = binding.Store(2 * VOCAB, DIM, workers=WORKERS, sync_interval=sync_interval, deterministic=deterministic,
                       track_ownership=False)
     s.init_uniform(0, 1, 0.5 / DIM)
     c, o, counts, weights = make_sgns_data(device, n_batches, seed, store=s)
@@ -481,6 +481,55 @@ def run_sample_sweep(args, device):
     s.close()
 
 
+def run_staleness_sweep(args, device):
+    """The SGNS workload with replicas merged by step count (every 16 batches) or by time: throughput and loss after
+    the same number of steps from the same start values.  The periods span the paper's staleness experiment (125, 25
+    and 5 merges per second, never) and, because a step takes about 10 us here, much shorter ones: what matters for
+    the model is how many updates a replica absorbs between two merges."""
+    from paper_2104_00501_b200 import binding
+    steps = max(args.steps, 32768)
+    nb = MAX_DISTINCT_BATCHES
+    CHUNK = 64
+    losses = torch.zeros(CHUNK, dtype=torch.float32, device=device)
+    settings = [("every 16 steps", SYNC_EVERY, 0)] + [(f"every {us / 1000:g} ms", 0, us)
+                                                      for us in (150, 500, 2_000, 8_000, 40_000, 200_000)] + [("never", 0, 0)]
+    store, prev_interval = None, None
+    for name, interval, period_us in settings:
+        if store is None or interval != prev_interval:
+            if store is not None:
+                store.close()
+            store, dist, hot, c, o, weights = build_store(binding, device, nb, seed=0, sync_interval=interval)
+            prev_interval = interval
+        else:
+            store.sync()
+            store.init_uniform(0, 1, 0.5 / DIM)
+        store.set_sync_period(period_us)
+
+        def run(count):
+            done = 0
+            while done < count:
+                j = done % nb
+                m = min(CHUNK, count - done, nb - j)
+                store.run_sgns(c[j * BATCH:(j + m) * BATCH], o[j * BATCH:(j + m) * BATCH], BATCH, dist, NEG, LR, losses[:m])
+                done += m
+        run(args.warmup)
+        m0 = store.stats()["background_merges"]
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        run(steps)
+        e1.record()
+        torch.cuda.synchronize()
+        t = e0.elapsed_time(e1) / 1e3
+        st = store.stats()
+        store.set_sync_period(0)
+        print(json.dumps({"workload": "SGNS, replica staleness", "merge": name, "steps": steps, "seconds": t,
+                          "key_accesses_per_s": steps * BATCH * ACCESSES_PER_PAIR / t, "us_per_step": t / steps * 1e6,
+                          "background_merges": st["background_merges"] - m0, "loss_last_64_steps": float(losses.mean())}),
+              flush=True)
+    store.close()
+
+
 def run_step_workload(args, device, which):
     """ComplEx + AdaGrad (config 3) or matrix factorization (config 4) steps in fast mode."""
     from paper_2104_00501_b200 import binding
@@ -549,7 +598,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=64)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="sgns", choices=["sgns", "ps", "sample", "kge", "mf"])
+    ap.add_argument("--workload", default="sgns", choices=["sgns", "ps", "sample", "kge", "mf", "staleness"])
     ap.add_argument("--hot-fraction", type=float, default=HOT_FRACTION, help="share of keys to replicate (default 0.01)")
     ap.add_argument("--workers", type=int, default=WORKERS)
     ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
@@ -581,6 +630,9 @@ def main():
         return
     if args.workload in ("kge", "mf"):
         run_step_workload(args, device, args.workload)
+        return
+    if args.workload == "staleness":
+        run_staleness_sweep(args, device)
         return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)

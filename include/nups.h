@@ -72,7 +72,9 @@ typedef struct nups_config {
     uint32_t smem_hot_rows;   /* fast mode: hot slots below this number are accumulated in    */
                               /*    shared memory inside a kernel before reaching the         */
                               /*    worker's replica; 0 = library default                     */
-    uint32_t reserved[9];
+    uint32_t sync_period_us;  /* > 0: a background thread merges the replicas every this many  */
+                              /*    microseconds, see nups_set_sync_period; fast mode only    */
+    uint32_t reserved[8];
 } nups_config;
 
 /* ---- store (Section 3.1: keys, pull, push) -------------------------------- */
@@ -272,6 +274,26 @@ nups_status nups_step_mf(nups_store* store, const uint32_t* d_row, const uint32_
  * device memory, valid until the next step).                                  */
 nups_status nups_last_negatives(nups_store* store, const uint32_t** h_d_keys_out, uint64_t* h_n_out);
 
+/* Time-based replica synchronisation (Section 3.2: replicas are synchronised
+ * periodically by a background thread and staleness is bounded by time, not by
+ * a logical clock; Section 5.6 varies the period from 8 ms to 5 s).  With
+ * period_us > 0 a host thread owned by the store enqueues a merge of all
+ * replicas every period_us microseconds on a stream of its own, so merging
+ * overlaps the caller's work and never blocks it; a tick is skipped while the
+ * previous merge is still running.  period_us = 0 stops the ticks and returns
+ * once merges already enqueued have finished.  Independent of sync_interval
+ * and nups_sync, which keep working (a caller that wants only time-based
+ * merging creates the store with sync_interval = 0).
+ * Such a merge runs concurrently with pulls, pushes and steps: no update is
+ * lost or applied twice, but a pull that overlaps it may miss, for that one
+ * read, updates that are just moving from a replica to the stored row.  After
+ * nups_set_sync_period(store, 0) and nups_sync every update is in the stored
+ * rows.  NUPS_ESTATE on a deterministic store (merges at arbitrary times are not
+ * reproducible); nups_create rejects that combination with NUPS_EINVAL.
+ * The merge reads every replicated slot of every worker each period: meant for
+ * periods of a millisecond and more.                                          */
+nups_status nups_set_sync_period(nups_store* store, uint32_t period_us);
+
 /* ---- status and statistics ------------------------------------------------ */
 
 /* Read and clear the device status word (synchronises the stream): NUPS_OK,
@@ -279,7 +301,8 @@ nups_status nups_last_negatives(nups_store* store, const uint32_t** h_d_keys_out
 nups_status nups_status_check(nups_store* store, void* stream);
 
 /* h_out[0..7]: steps, syncs launched, kernels launched by the library so far,
- * accesses served from replicas, accesses served in place, hot slots, 0, 0.
+ * accesses served from replicas, accesses served in place, hot slots,
+ * background merges enqueued, 0.
  * The two access counters are only kept when count_accesses is set.
  * Synchronises the stream.                                                    */
 nups_status nups_get_stats(nups_store* store, uint64_t* h_out, void* stream);

@@ -106,6 +106,7 @@ struct nups_store {
     uint32_t ev_n;             // pairs recorded since the last query
     double ev_ms;              // time of pairs folded in when the ring filled up
     uint64_t ev_launches;
+    struct nups_background* bg; // time-based replica synchronisation (background.cu); NULL = never started
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };
@@ -142,6 +143,13 @@ void nups_time_begin(nups_store* s, cudaStream_t st);
 void nups_time_end(nups_store* s, cudaStream_t st);
 nups_status nups_scratch(nups_store* s, size_t bytes, char** out);     // grow-only scratch, 256-byte aligned
 nups_status nups_new_epoch(nups_store* s, cudaStream_t st);          // call before taking the view of a call that moves keys
+
+// background.cu
+nups_status nups_background_start(nups_store* s, uint32_t period_us);
+void nups_background_stop(nups_store* s);
+void nups_background_begin(nups_store* s, cudaStream_t st);
+void nups_background_end(nups_store* s, cudaStream_t st);
+uint64_t nups_background_merges(nups_store* s);
 
 // primitives.cu
 size_t nups_scan_scratch_bytes(uint64_t n);

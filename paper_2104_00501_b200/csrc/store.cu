@@ -148,6 +148,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     if (cfg) c = *cfg;
     if (c.workers == 0) c.workers = 8;
     if (c.workers > 254) return NUPS_EINVAL;
+    if (c.sync_period_us && c.deterministic) return NUPS_EINVAL;
     int dev = 0, count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) {
         snprintf(g_nups_cuda_err, sizeof(g_nups_cuda_err), "no CUDA device");
@@ -192,6 +193,13 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
         nups_destroy(s);
         return nups_cuda_fail(e, "nups_create");
     }
+    if (c.sync_period_us) {
+        nups_status rc = nups_background_start(s, c.sync_period_us);
+        if (rc != NUPS_OK) {
+            nups_destroy(s);
+            return rc;
+        }
+    }
     *out = s;
     return NUPS_OK;
 }
@@ -199,6 +207,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
 extern "C" nups_status nups_destroy(nups_store* s)
 {
     if (!s) return NUPS_OK;
+    nups_background_stop(s);
     cudaDeviceSynchronize();
     for (int i = 0; i < NUPS_MAX_HANDLES; ++i) cudaFree(s->handle[i].buf);
     for (int i = 0; i < NUPS_MAX_DISTS; ++i) { cudaFree(s->dist[i].table); cudaFree(s->dist[i].off); }
@@ -857,9 +866,13 @@ nups_status nups_sync_internal(nups_store* s, cudaStream_t st)
 {
     if (s->H == 0) return NUPS_OK;        // nothing replicated: no work at all
     View v = nups_view(s);
+    nups_background_begin(s, st);
     sync_kernel<<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
-    LAUNCH_CHECK(s);
-    CK(cudaMemsetAsync(s->dirty, 0, (size_t)s->R * s->Hcap * sizeof(uint32_t), st));
+    cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaMemsetAsync(s->dirty, 0, (size_t)s->R * s->Hcap * sizeof(uint32_t), st);
+    nups_background_end(s, st);
+    if (e != cudaSuccess) return nups_cuda_fail(e, "replica merge");
+    s->launches++;
     s->syncs++;
     return NUPS_OK;
 }
@@ -1110,6 +1123,13 @@ extern "C" nups_status nups_set_management(nups_store* s, const uint32_t* d_keys
     if (rc != NUPS_OK) return rc;
     CK(cudaStreamSynchronize(st));
     if (n == 0) return NUPS_OK;
+    // no background merge may be enqueued or running while slots and replicas are rebuilt
+    struct Bracket {
+        nups_store* s;
+        cudaStream_t st;
+        Bracket(nups_store* s_, cudaStream_t st_) : s(s_), st(st_) { nups_background_begin(s, st); }
+        ~Bracket() { nups_background_end(s, st); }
+    } bracket(s, st);
     uint64_t m = technique == NUPS_REPLICATE ? n : (s->H > n ? s->H : n);
     size_t need = 2 * align256(m * 8) + align256(m * 4) + nups_scan_scratch_bytes(m) + 256;
     char* sc;
@@ -1274,6 +1294,6 @@ extern "C" nups_status nups_get_stats(nups_store* s, uint64_t* h_out, void* stre
     CK(cudaMemcpyAsync(&d, s->st, sizeof(DevStat), cudaMemcpyDeviceToHost, st));
     CK(cudaStreamSynchronize(st));
     h_out[0] = s->steps; h_out[1] = s->syncs; h_out[2] = s->launches;
-    h_out[3] = d.hot_hits; h_out[4] = d.cold_hits; h_out[5] = s->H; h_out[6] = 0; h_out[7] = 0;
+    h_out[3] = d.hot_hits; h_out[4] = d.cold_hits; h_out[5] = s->H; h_out[6] = nups_background_merges(s); h_out[7] = 0;
     return NUPS_OK;
 }
