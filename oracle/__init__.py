@@ -58,6 +58,8 @@ def lib():
             "orc_pull2": (C.c_int, [C.c_void_p, _u32p, C.c_uint64, _f32p, _f32p]),
             "orc_push2": (C.c_int, [C.c_void_p, _u32p, C.c_uint64, _f32p, _f32p]),
             "orc_sync": (C.c_int, [C.c_void_p]),
+            "orc_set_clipping": (None, [C.c_void_p, C.c_double]),
+            "orc_clip_stats": (None, [C.c_void_p, C.POINTER(C.c_double), _u64p]),
             "orc_count_accesses": (C.c_int, [C.c_void_p, _u32p, C.c_uint64]),
             "orc_select_hot": (C.c_uint64, [C.c_void_p, C.c_int, C.c_uint64, _u32p]),
             "orc_set_management": (C.c_int, [C.c_void_p, _u32p, C.c_uint64, C.c_int]),
@@ -243,6 +245,15 @@ class Oracle:
         return (keys, vals) if values else keys
 
     # -- workload steps ---------------------------------------------------
+    def set_clipping(self, factor):
+        """Clip updates to replicated keys at `factor` times the mean norm of earlier such updates (0 = off)."""
+        self._l.orc_set_clipping(self._s, float(factor))
+
+    def clip_stats(self):
+        s, c = C.c_double(0), C.c_uint64(0)
+        self._l.orc_clip_stats(self._s, C.byref(s), C.byref(c))
+        return s.value, c.value
+
     def step_sgns(self, center, context, dist, K, lr, return_negatives=False):
         c, cp = _u32(center)
         o, op = _u32(context)

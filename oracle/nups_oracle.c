@@ -180,6 +180,9 @@ typedef struct {
     uint64_t* cnt;
     uint8_t* owner;         /* ORC_OWNER_DEFAULT = never moved: owner is key mod R   */
     uint64_t steps, syncs, hot_hits, cold_hits;
+    double clip_factor;     /* 0 = updates are never clipped                         */
+    double clip_sum;        /* sum of the norms of the replicated-key updates that    */
+    uint64_t clip_cnt;      /*   earlier steps applied, and how many there were       */
     int status;
     orc_dist dist[ORC_MAX_DISTS];
     orc_handle handle[ORC_MAX_HANDLES];
@@ -696,6 +699,52 @@ static double clamp30(double x) { return x > 30.0 ? 30.0 : (x < -30.0 ? -30.0 : 
 static double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 static double softplus(double x) { return (x > 0 ? x : 0) + log1p(exp(-fabs(x))); }
 
+/* Gradient-norm clipping for replicated keys (Section 5.1, "Implementation and
+ * cluster": updates to replicated parameters that exceed the average norm by
+ * more than 2x are clipped, in the word-vector and matrix-factorization tasks).
+ * Reading: the average is the mean Euclidean norm of all updates to replicated
+ * keys that EARLIER steps applied (after their own clipping), so the bound is
+ * fixed while a step runs and no update of a batch depends on another one of
+ * the same batch; an update row d with |d| > factor * mean becomes
+ * d * (factor * mean / |d|); before any such update has been applied nothing
+ * is clipped.  The step's own norms join the statistics when the step ends.   */
+typedef struct { double sum; uint64_t cnt; } clip_step;
+
+void orc_set_clipping(void* p, double factor)
+{
+    orc_store* s = (orc_store*)p;
+    s->clip_factor = factor > 0 ? factor : 0;
+}
+
+void orc_clip_stats(void* p, double* sum, uint64_t* cnt)
+{
+    orc_store* s = (orc_store*)p;
+    *sum = s->clip_sum; *cnt = s->clip_cnt;
+}
+
+/* d[0..L): the update about to be pushed to key k (in double, not yet rounded) */
+static void clip_update(const orc_store* s, uint32_t k, double* d, clip_step* st)
+{
+    if (s->clip_factor == 0 || s->slot[k] < 0) return;
+    double n2 = 0;
+    for (uint32_t e = 0; e < s->L; ++e) n2 += d[e] * d[e];
+    double n = sqrt(n2);
+    if (s->clip_cnt > 0) {
+        double bound = s->clip_factor * (s->clip_sum / (double)s->clip_cnt);
+        if (n > bound) {
+            double f = bound / n;
+            for (uint32_t e = 0; e < s->L; ++e) d[e] *= f;
+            n = bound;
+        }
+    }
+    st->sum += n; st->cnt++;
+}
+
+static void clip_end_of_step(orc_store* s, const clip_step* st)
+{
+    s->clip_sum += st->sum; s->clip_cnt += st->cnt;
+}
+
 static void end_of_step(orc_store* s)
 {
     s->steps++;
@@ -726,6 +775,8 @@ int orc_step_sgns(void* p, const uint32_t* center, const uint32_t* context, uint
     float* v = (float*)malloc(L * sizeof(float));
     float* u = (float*)malloc(L * sizeof(float));
     double* gv = (double*)malloc(L * sizeof(double));
+    double* dd = (double*)malloc(L * sizeof(double));
+    clip_step clip = {0, 0};
     double loss = 0;
     for (uint64_t i = 0; i < n; ++i) {
         uint32_t q = worker_of(s, i, n);
@@ -750,13 +801,18 @@ int orc_step_sgns(void* p, const uint32_t* center, const uint32_t* context, uint
             loss += (j == 0) ? softplus(-x) : softplus(x);
             float* du = upd + (i * per + j) * L;
             for (uint32_t e = 0; e < L; ++e) {
-                du[e] = (float)(-(double)lr * g * (double)v[e]);
+                dd[e] = -(double)lr * g * (double)v[e];
                 gv[e] += g * (double)u[e];
             }
+            clip_update(s, kk[j], dd, &clip);
+            for (uint32_t e = 0; e < L; ++e) du[e] = (float)dd[e];
         }
         float* dv = upd + (i * per + K + 1) * L;
-        for (uint32_t e = 0; e < L; ++e) dv[e] = (float)(-(double)lr * gv[e]);
+        for (uint32_t e = 0; e < L; ++e) dd[e] = -(double)lr * gv[e];
+        clip_update(s, center[i], dd, &clip);
+        for (uint32_t e = 0; e < L; ++e) dv[e] = (float)dd[e];
     }
+    clip_end_of_step(s, &clip);
     loc_queue lq = {0};
     for (uint64_t i = 0; i < n; ++i) {
         if (!okv[i]) continue;
@@ -771,7 +827,7 @@ int orc_step_sgns(void* p, const uint32_t* center, const uint32_t* context, uint
     }
     loc_apply(s, &lq);
     if (loss_out) *loss_out = (float)(loss / (double)(n ? n : 1));
-    free(nk); free(upd); free(uk); free(okv); free(v); free(u); free(gv);
+    free(nk); free(upd); free(uk); free(okv); free(v); free(u); free(gv); free(dd);
     end_of_step(s);
     return ORC_OK;
 }
@@ -898,6 +954,8 @@ int orc_step_mf(void* p, const uint32_t* rowk, const uint32_t* colk, const float
     uint8_t* okv = (uint8_t*)calloc(n, 1);
     float* w = (float*)malloc(L * sizeof(float));
     float* h = (float*)malloc(L * sizeof(float));
+    double* dd = (double*)malloc(L * sizeof(double));
+    clip_step clip = {0, 0};
     double loss = 0;
     for (uint64_t i = 0; i < n; ++i) {
         uint32_t q = worker_of(s, i, n);
@@ -914,11 +972,14 @@ int orc_step_mf(void* p, const uint32_t* rowk, const uint32_t* colk, const float
         loss += err * err;
         float* dw = upd + (i * 2) * L;
         float* dh = upd + (i * 2 + 1) * L;
-        for (uint32_t e = 0; e < L; ++e) {
-            dw[e] = (float)((double)lr * (err * (double)h[e] - (double)l2 * (double)w[e]));
-            dh[e] = (float)((double)lr * (err * (double)w[e] - (double)l2 * (double)h[e]));
-        }
+        for (uint32_t e = 0; e < L; ++e) dd[e] = (double)lr * (err * (double)h[e] - (double)l2 * (double)w[e]);
+        clip_update(s, rowk[i], dd, &clip);
+        for (uint32_t e = 0; e < L; ++e) dw[e] = (float)dd[e];
+        for (uint32_t e = 0; e < L; ++e) dd[e] = (double)lr * (err * (double)w[e] - (double)l2 * (double)h[e]);
+        clip_update(s, colk[i], dd, &clip);
+        for (uint32_t e = 0; e < L; ++e) dh[e] = (float)dd[e];
     }
+    clip_end_of_step(s, &clip);
     loc_queue lq = {0};
     for (uint64_t i = 0; i < n; ++i) {
         if (!okv[i]) continue;
@@ -932,7 +993,7 @@ int orc_step_mf(void* p, const uint32_t* rowk, const uint32_t* colk, const float
     }
     loc_apply(s, &lq);
     if (loss_out) *loss_out = (float)(loss / (double)(n ? n : 1));
-    free(upd); free(okv); free(w); free(h);
+    free(upd); free(okv); free(w); free(h); free(dd);
     end_of_step(s);
     return ORC_OK;
 }

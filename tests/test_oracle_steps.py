@@ -233,3 +233,74 @@ def test_tiny_sgns_loss_decreases():
     c, ctx = inputs.u32(c), inputs.u32(ctx)
     losses = [o.step_sgns(c[i:i + 64], ctx[i:i + 64], d, K, 0.025) for i in range(0, 64 * 400, 64)]
     assert np.mean(losses[-50:]) < 0.9 * np.mean(losses[:50])
+
+
+# ---------------------------------------------------------------------------------------------------------
+# gradient-norm clipping for replicated keys (Section 5.1): pinned by a worked case with a closed form
+# ---------------------------------------------------------------------------------------------------------
+def _mf_clip_store(L=4):
+    # rows 0..9 start at zero and are replicated; column key 10 holds h and is not replicated.  With w = 0 and
+    # l2 = 0 a cell (i, 10, x) gives dw = lr * x * h (norm lr * |x| * |h|) and dh = lr * x * w = 0: h never moves.
+    o = Oracle(11, L, workers=2)
+    h = np.array([3.0, 0.0, 4.0, 0.0], np.float32)[:L]
+    o.table()[10] = h
+    o.set_management(np.arange(10, dtype=np.uint32), REPLICATE)
+    return o, h
+
+
+def test_clipping_closed_form_on_matrix_factorization_cells():
+    lr = 0.5
+    o, h = _mf_clip_store()
+    o.set_clipping(2.0)
+    hn = float(np.linalg.norm(h))                           # 5
+    # step 1: nothing to compare with yet -> applied as it is; the mean norm becomes lr * 1 * 5 = 2.5
+    o.step_mf([0], [10], [1.0], lr, 0.0)
+    assert o.clip_stats() == (pytest.approx(lr * hn), 1)
+    # step 2: two cells of one batch with x = 10 and x = -40: norms 25 and 100, both above 2 * 2.5 = 5 and both
+    # judged against the same bound (the batch does not see itself): each becomes 5 long, direction kept
+    o.step_mf([1, 2], [10, 10], [10.0, -40.0], lr, 0.0)
+    s, c = o.clip_stats()
+    assert c == 3 and s == pytest.approx(2.5 + 5.0 + 5.0)
+    # step 3: mean is 12.5 / 3, bound 8.33: x = 3 (norm 7.5) passes, x = 4 (norm 10) is cut to 8.33
+    o.step_mf([3, 4], [10, 10], [3.0, 4.0], lr, 0.0)
+    o.sync()
+    t = o.table()
+    np.testing.assert_allclose(t[0], lr * 1.0 * h, rtol=1e-6)
+    np.testing.assert_allclose(t[1], 5.0 * h / hn, rtol=1e-6)
+    np.testing.assert_allclose(t[2], -5.0 * h / hn, rtol=1e-6)
+    np.testing.assert_allclose(t[3], lr * 3.0 * h, rtol=1e-6)
+    np.testing.assert_allclose(t[4], (2.0 * 12.5 / 3.0) * h / hn, rtol=1e-6)
+    np.testing.assert_array_equal(t[10], h)                  # the column row never moved (w was zero)
+    s, c = o.clip_stats()
+    assert c == 5 and s == pytest.approx(12.5 + 7.5 + 2.0 * 12.5 / 3.0)
+
+
+def test_clipping_leaves_non_replicated_keys_and_unclipped_runs_alone():
+    rng = np.random.default_rng(5)
+    V, L, K, n = 60, 8, 2, 64
+    init = rng.normal(0, 0.5, (2 * V, L)).astype(np.float32)
+    c, ctx = rng.integers(0, V, n).astype(np.uint32), (V + rng.integers(0, V, n)).astype(np.uint32)
+    w = rng.integers(1, 50, V).astype(np.uint32)
+
+    def run(hot, factor):
+        o = Oracle(2 * V, L, workers=3)
+        o.table()[:] = init
+        if len(hot):
+            o.set_management(np.asarray(hot, np.uint32), REPLICATE)
+        o.set_clipping(factor)
+        d = o.register_distribution(V, w, V, CONFORM, seed=4)
+        for _ in range(4):
+            o.step_sgns(c, ctx, d, K, 0.5)
+        return o.table().copy(), o.clip_stats()
+
+    plain, st0 = run([], 0.0)
+    same, st1 = run([], 2.0)                                 # nothing replicated: nothing to clip, nothing counted
+    assert np.array_equal(plain, same) and st0 == (0.0, 0) and st1 == (0.0, 0)
+    hot = np.arange(0, 2 * V, 3)
+    base, _ = run(hot, 0.0)
+    huge, st = run(hot, 1e9)                                 # a bound nobody reaches: same values, norms still counted
+    assert np.array_equal(base, huge) and st[1] > 0
+    tight, _ = run(hot, 0.5)                                 # a tight bound changes replicated rows only through
+    assert not np.array_equal(base, tight)                   # what was pushed to them; every update got shorter:
+    d_base, d_tight = np.abs(base - init).sum(), np.abs(tight - init).sum()
+    assert d_tight < d_base
