@@ -74,7 +74,10 @@ typedef struct nups_config {
                               /*    worker's replica; 0 = library default                     */
     uint32_t sync_period_us;  /* > 0: a background thread merges the replicas every this many  */
                               /*    microseconds, see nups_set_sync_period; fast mode only    */
-    uint32_t reserved[8];
+    float    clip_factor;     /* > 0: nups_step_sgns and nups_step_mf clip every update to a   */
+                              /*    replicated key at clip_factor times the mean norm of such  */
+                              /*    updates so far, see nups_get_clip_stats; 0 = no clipping   */
+    uint32_t reserved[7];
 } nups_config;
 
 /* ---- store (Section 3.1: keys, pull, push) -------------------------------- */
@@ -293,6 +296,20 @@ nups_status nups_last_negatives(nups_store* store, const uint32_t** h_d_keys_out
  * The merge reads every replicated slot of every worker each period: meant for
  * periods of a millisecond and more.                                          */
 nups_status nups_set_sync_period(nups_store* store, uint32_t period_us);
+
+/* Gradient-norm clipping for replicated keys (Section 5.1, implementation
+ * notes: updates to replicated parameters that exceed the average norm by more
+ * than 2x are clipped in the word-vector and matrix-factorization tasks).  With
+ * clip_factor > 0 the skip-gram and matrix-factorization steps compare the
+ * Euclidean norm of every update row bound for a replicated key with
+ * clip_factor times the mean norm of all such updates that earlier steps
+ * applied, and scale a longer row down to that bound (direction kept).  The
+ * bound is fixed while a step runs (in fast mode: while one launch of
+ * nups_run_sgns runs, which may cover several steps); nothing is clipped before
+ * the first such update has been applied.  This call returns the statistics:
+ * *h_sum = sum of the norms as applied, *h_count = number of updates; it
+ * synchronises the stream.                                                    */
+nups_status nups_get_clip_stats(nups_store* store, double* h_sum, uint64_t* h_count, void* stream);
 
 /* ---- status and statistics ------------------------------------------------ */
 

@@ -25,14 +25,14 @@ EXPORTS = [
     "nups_push2", "nups_push_noalloc", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_run_sgns", "nups_step_complex", "nups_step_mf",
-    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_strerror", "nups_last_cuda_error",
+    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_get_clip_stats", "nups_strerror", "nups_last_cuda_error",
 ]
 
 
 class Config(C.Structure):
     _fields_ = [("workers", C.c_uint32), ("sync_interval", C.c_uint32), ("deterministic", C.c_uint32),
                 ("with_adagrad", C.c_uint32), ("count_accesses", C.c_uint32), ("track_ownership", C.c_uint32),
-                ("smem_hot_rows", C.c_uint32), ("sync_period_us", C.c_uint32), ("reserved", C.c_uint32 * 8)]
+                ("smem_hot_rows", C.c_uint32), ("sync_period_us", C.c_uint32), ("clip_factor", C.c_float), ("reserved", C.c_uint32 * 7)]
 
 
 class NupsError(RuntimeError):
@@ -94,6 +94,7 @@ def load(build_if_missing: bool = True):
         "nups_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
         "nups_probe_reduction_rate": [vp, u64, u32, C.POINTER(C.c_double), vp],
         "nups_set_sync_period": [vp, u32],
+        "nups_get_clip_stats": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -131,11 +132,11 @@ class Store:
     """One parameter store on the current CUDA device."""
 
     def __init__(self, num_keys, value_len, workers=8, sync_interval=1, deterministic=False, with_adagrad=False,
-                 count_accesses=False, track_ownership=False, smem_hot_rows=0, sync_period_us=0):
+                 count_accesses=False, track_ownership=False, smem_hot_rows=0, sync_period_us=0, clip_factor=0.0):
         self._l = load()
         cfg = Config(workers=workers, sync_interval=sync_interval, deterministic=int(deterministic),
                      with_adagrad=int(with_adagrad), count_accesses=int(count_accesses),
-                     track_ownership=int(track_ownership), smem_hot_rows=smem_hot_rows, sync_period_us=sync_period_us)
+                     track_ownership=int(track_ownership), smem_hot_rows=smem_hot_rows, sync_period_us=sync_period_us, clip_factor=clip_factor)
         h = C.c_void_p()
         self._s = None
         self._chk(self._l.nups_create(num_keys, value_len, C.byref(cfg), C.byref(h)), "nups_create")
@@ -346,6 +347,12 @@ class Store:
         self._chk(self._l.nups_get_stats(self._s, out, _stream()), "nups_get_stats")
         return dict(steps=out[0], syncs=out[1], launches=out[2], hot=out[3], cold=out[4], hot_slots=out[5],
                     background_merges=out[6])
+
+    def clip_stats(self):
+        """(sum of the norms of the replicated-key updates applied so far, their number)."""
+        sm, cnt = C.c_double(0), C.c_uint64(0)
+        self._chk(self._l.nups_get_clip_stats(self._s, C.byref(sm), C.byref(cnt), _stream()), "nups_get_clip_stats")
+        return sm.value, cnt.value
 
     def set_sync_period(self, period_us):
         """Background merging of the replicas every `period_us` microseconds; 0 stops it."""

@@ -27,6 +27,11 @@ struct DevStat {
     unsigned long long cold_hits;      // accesses served in place
     unsigned long long unused0;
     unsigned long long tmp[4];
+    // gradient-norm clipping of replicated-key updates: norms applied by finished steps, and by the running one
+    double clip_sum;
+    unsigned long long clip_cnt;
+    double clip_step_sum;
+    unsigned long long clip_step_cnt;
 };
 
 // What kernels need to know about a store; passed by value.
@@ -49,6 +54,7 @@ struct View {
     uint32_t R;
     uint32_t count;            // count accesses?
     uint32_t epoch_tag;        // number of the running call, shifted into the upper 24 bits of an ownership word
+    float clip_factor;         // > 0: updates to replicated keys are clipped at this multiple of their mean norm
 };
 
 struct Dist {

@@ -67,24 +67,47 @@ static_assert(LOSS_SLOTS * LOSS_STEPS <= 4 * NUPS_MAX_STEP_BLOCKS, "the per-step
 
 constexpr int SGNS_WARPS = 2;                                      // warps (= pairs in flight) per block
 
+// Gradient-norm clipping of updates to replicated keys: the bound that holds for the whole launch
+// (factor x mean norm of the updates applied by finished steps; infinite before there was any).
+__device__ __forceinline__ float clip_bound(const View& v)
+{
+    const unsigned long long cnt = v.st->clip_cnt;
+    return cnt ? v.clip_factor * (float)(v.st->clip_sum / (double)cnt) : __int_as_float(0x7f800000);
+}
+// norm of an update as applied: cut to the bound; *scale receives the factor for the row
+__device__ __forceinline__ float clip_norm(float norm, float bound, float* scale)
+{
+    *scale = norm > bound ? bound / norm : 1.f;
+    return norm > bound ? bound : norm;
+}
+// fast mode: a warp's share of the running step's statistics, once per warp and launch
+__device__ __forceinline__ void clip_finish(const View& v, double sum, unsigned cnt)
+{
+    if ((threadIdx.x & 31) == 0 && cnt) {
+        atomicAdd(&v.st->clip_step_sum, sum);
+        atomicAdd(&v.st->clip_step_cnt, (unsigned long long)cnt);
+    }
+}
+
 // asynchronous 16-byte copy to the shared-memory address (32-bit, shared window) smem_dst
 __device__ __forceinline__ void cp_async_16s(uint32_t smem_dst, const void* gmem_src)
 {
     asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(gmem_src) : "memory");
 }
 
-template <bool HOT, bool DET, int KT, int CH>
+template <bool HOT, bool DET, int KT, int CH, bool CLIP>
 __global__ void __launch_bounds__(32 * SGNS_WARPS)
 sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
             const uint32_t* __restrict__ negs, uint64_t n, uint32_t K_arg, float lr,
             float* __restrict__ upd, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
             float* __restrict__ loss_out, uint32_t group,
-            unsigned long long* __restrict__ loss_acc)
+            unsigned long long* __restrict__ loss_acc, float2* __restrict__ clip_item)
 {
     extern __shared__ __align__(16) float4 park_all[];
     __shared__ const float4* s_src[SGNS_WARPS][32];                // the role's stored row
     __shared__ float* s_dst[SGNS_WARPS][32];                       // where its update goes: replica row or stored row
     __shared__ float s_g[SGNS_WARPS][32];                          // d(loss)/d(score) of the role
+    __shared__ float s_f[SGNS_WARPS][32];                          // clipping factor of the role's update
     constexpr uint32_t cols = 32 * CH;
     constexpr uint32_t NR = KT > 0 ? KT + 2 : 1;                   // roles kept in registers when K is fixed
     const uint32_t K = KT > 0 ? (uint32_t)KT : K_arg;
@@ -96,6 +119,9 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
     const uint64_t nwarps = (uint64_t)gridDim.x * SGNS_WARPS, total = n * group;
     const uint64_t w0 = (uint64_t)blockIdx.x * SGNS_WARPS + wib;
     double my_loss = 0.0;
+    const float bound = CLIP ? clip_bound(v) : 0.f;
+    double my_clip = 0.0;                                          // fast mode: norms applied by this warp
+    unsigned my_clipped = 0;
     auto key_of = [&](uint64_t e) -> uint32_t {
         if (lane >= per || e >= total) return 0u;
         return lane == 0 ? context[e] : (lane <= K ? negs[e * K + lane - 1] : center[e]);
@@ -119,7 +145,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         const bool ok = lane >= per || key < v.num_keys;
         if (!__all_sync(0xFFFFFFFFu, ok)) {                        // a key out of range: the whole item is skipped
             if (DET && lane < per) ukeys[i * per + lane] = NUPS_INVALID_KEY;
-            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; if (DET && CLIP) clip_item[i] = make_float2(0.f, 0.f); }
             continue;
         }
         const uint32_t mask = HOT ? __ballot_sync(0xFFFFFFFFu, slot >= 0) : 0u;
@@ -193,24 +219,69 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         }
         float loss_l = lane == 0 ? softplusf_(-x_l) : (lane <= K ? softplusf_(x_l) : 0.f);
         loss_l = warp_sum(loss_l);
+        // clipping: the update of role j <= K is -lr g_j a, of norm lr |g_j| |a|; lane j holds its factor
+        float f_l = 1.f, clip_sum_item = 0.f;
+        const bool clip_here = CLIP && mask != 0u;                 // some role of the pair is replicated
+        if (clip_here) {
+            float a2 = 0.f;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) a2 += a[m].x * a[m].x + a[m].y * a[m].y + a[m].z * a[m].z + a[m].w * a[m].w;
+            const float an = sqrtf(warp_sum(a2));
+            float applied = 0.f;
+            if (lane <= K && (mask >> lane & 1u)) applied = clip_norm(lr * fabsf(g_l) * an, bound, &f_l);
+            clip_sum_item = warp_sum(applied);
+        }
+        float fk[NR];
+        if (CLIP && KT > 0) {
+#pragma unroll
+            for (int j = 0; j <= KT; ++j) fk[j] = __shfl_sync(0xFFFFFFFFu, f_l, j);
+        } else if (CLIP) {
+            s_f[wib][lane] = f_l;
+        }
         __syncwarp();
+        float4 gvv[CLIP ? CH : 1];
 #pragma unroll
         for (int m = 0; m < CH; ++m) {
-            if (lane + 32 * m >= L4) continue;
+            if (lane + 32 * m >= L4) { if (CLIP) gvv[CLIP ? m : 0] = make_float4(0.f, 0.f, 0.f, 0.f); continue; }
             float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
             for (uint32_t j = 0; j <= K; ++j) {
                 const float g = KT > 0 ? gk[KT > 0 ? j : 0] : s_g[wib][j];
                 const float4 u = park[j * cols + 32 * m];
-                const float sc = -lr * g;
+                float sc = -lr * g;
+                if (CLIP) sc *= KT > 0 ? fk[KT > 0 ? j : 0] : s_f[wib][j];
                 const float4 du = make_float4(sc * a[m].x, sc * a[m].y, sc * a[m].z, sc * a[m].w);
                 if (DET) ((float4*)(upd + (i * per + j) * L))[lane + 32 * m] = du;
                 else red_add_v4((KT > 0 ? dstp[KT > 0 ? j : 0] : s_dst[wib][j] + 4 * lane) + 128 * m, du);
                 gv.x += g * u.x; gv.y += g * u.y; gv.z += g * u.z; gv.w += g * u.w;
             }
+            if (CLIP) { gvv[CLIP ? m : 0] = gv; continue; }          // the centre's update waits for its norm
             const float4 dv = make_float4(-lr * gv.x, -lr * gv.y, -lr * gv.z, -lr * gv.w);
             if (DET) ((float4*)(upd + (i * per + K + 1) * L))[lane + 32 * m] = dv;
             else red_add_v4((KT > 0 ? dstp[KT > 0 ? KT + 1 : 0] : s_dst[wib][K + 1] + 4 * lane) + 128 * m, dv);
+        }
+        if (CLIP) {
+            float fc = 1.f;
+            if (mask >> (K + 1) & 1u) {                            // the centre word is replicated
+                float g2 = 0.f;
+#pragma unroll
+                for (int m = 0; m < CH; ++m) {
+                    const float4 gv = gvv[CLIP ? m : 0];
+                    g2 += gv.x * gv.x + gv.y * gv.y + gv.z * gv.z + gv.w * gv.w;
+                }
+                clip_sum_item += clip_norm(lr * sqrtf(warp_sum(g2)), bound, &fc);
+            }
+            const float sc = -lr * fc;
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                if (lane + 32 * m >= L4) continue;
+                const float4 gv = gvv[CLIP ? m : 0];
+                const float4 dv = make_float4(sc * gv.x, sc * gv.y, sc * gv.z, sc * gv.w);
+                if (DET) ((float4*)(upd + (i * per + K + 1) * L))[lane + 32 * m] = dv;
+                else red_add_v4((KT > 0 ? dstp[KT > 0 ? KT + 1 : 0] : s_dst[wib][K + 1] + 4 * lane) + 128 * m, dv);
+            }
+            if (DET) { if (lane == 0) clip_item[i] = make_float2(clip_sum_item, (float)__popc(mask)); }
+            else { my_clip += (double)clip_sum_item; my_clipped += __popc(mask); }
         }
         if (lane == 0) {
             if (DET) loss_item[i] = loss_l;
@@ -219,6 +290,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         }
     }
     if (!DET && !loss_acc) loss_finish(v, my_loss, n, loss_out);
+    if (CLIP && !DET) clip_finish(v, my_clip, my_clipped);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -448,11 +520,11 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
 #endif
 constexpr int MF_DEPTH = NUPS_MF_DEPTH;
 
-template <bool HOT, bool DET, int CH>
+template <bool HOT, bool DET, int CH, bool CLIP>
 __global__ void __launch_bounds__(128)
 mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
           uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
-          float* __restrict__ loss_item, float* __restrict__ loss_out)
+          float* __restrict__ loss_item, float* __restrict__ loss_out, float2* __restrict__ clip_item)
 {
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -461,6 +533,9 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
     const float4* val4 = (const float4*)v.val;
     const float4* slab4 = (const float4*)v.dval;
     double my_loss = 0.0;
+    const float bound = CLIP ? clip_bound(v) : 0.f;
+    double my_clip = 0.0;
+    unsigned my_clipped = 0;
 
     // ring A: keys and cell values of the items 2*MF_DEPTH .. MF_DEPTH+1 steps ahead
     // ring B: keys, slots and stored rows of the items MF_DEPTH .. 1 steps ahead
@@ -517,7 +592,7 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
                 ukeys[2 * i + 1] = ok ? kj : NUPS_INVALID_KEY;
             }
             if (!ok) {
-                if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+                if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; if (DET && CLIP) clip_item[i] = make_float2(0.f, 0.f); }
                 continue;
             }
             const uint64_t pw = si >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)si) * L4 : 0;
@@ -533,6 +608,29 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
                 dot += w[m].x * h[m].x + w[m].y * h[m].y + w[m].z * h[m].z + w[m].w * h[m].w;
             }
             const float err = xv - warp_sum(dot);
+            float fw = lr, fh = lr;                                 // learning rate times the clipping factor
+            if (CLIP && (si >= 0 || sj >= 0)) {
+                float nw2 = 0.f, nh2 = 0.f;
+#pragma unroll
+                for (int m = 0; m < CH; ++m) {
+                    if (lane + 32 * m < L4) {
+                        const float4 a = make_float4(err * h[m].x - l2 * w[m].x, err * h[m].y - l2 * w[m].y,
+                                                     err * h[m].z - l2 * w[m].z, err * h[m].w - l2 * w[m].w);
+                        const float4 b = make_float4(err * w[m].x - l2 * h[m].x, err * w[m].y - l2 * h[m].y,
+                                                     err * w[m].z - l2 * h[m].z, err * w[m].w - l2 * h[m].w);
+                        nw2 += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+                        nh2 += b.x * b.x + b.y * b.y + b.z * b.z + b.w * b.w;
+                    }
+                }
+                float applied = 0.f, f;
+                if (si >= 0) { applied += clip_norm(lr * sqrtf(warp_sum(nw2)), bound, &f); fw = lr * f; }
+                if (sj >= 0) { applied += clip_norm(lr * sqrtf(warp_sum(nh2)), bound, &f); fh = lr * f; }
+                const unsigned hot_roles = (si >= 0 ? 1u : 0u) + (sj >= 0 ? 1u : 0u);
+                if (DET) { if (lane == 0) clip_item[i] = make_float2(applied, (float)hot_roles); }
+                else { my_clip += (double)applied; my_clipped += hot_roles; }
+            } else if (CLIP && DET && lane == 0) {
+                clip_item[i] = make_float2(0.f, 0.f);
+            }
             float* ow = DET ? upd + (2 * i) * (uint64_t)L4 * 4 : (si >= 0 ? v.dval + pw * 4 : v.val + (uint64_t)ki * L4 * 4);
             float* oh = DET ? upd + (2 * i + 1) * (uint64_t)L4 * 4
                             : (sj >= 0 ? v.dval + ph * 4 : v.val + (uint64_t)kj * L4 * 4);
@@ -540,10 +638,10 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
             for (int m = 0; m < CH; ++m) {
                 const uint32_t c = lane + 32 * m;
                 if (c < L4) {
-                    const float4 dw = make_float4(lr * (err * h[m].x - l2 * w[m].x), lr * (err * h[m].y - l2 * w[m].y),
-                                                  lr * (err * h[m].z - l2 * w[m].z), lr * (err * h[m].w - l2 * w[m].w));
-                    const float4 dh = make_float4(lr * (err * w[m].x - l2 * h[m].x), lr * (err * w[m].y - l2 * h[m].y),
-                                                  lr * (err * w[m].z - l2 * h[m].z), lr * (err * w[m].w - l2 * h[m].w));
+                    const float4 dw = make_float4(fw * (err * h[m].x - l2 * w[m].x), fw * (err * h[m].y - l2 * w[m].y),
+                                                  fw * (err * h[m].z - l2 * w[m].z), fw * (err * h[m].w - l2 * w[m].w));
+                    const float4 dh = make_float4(fh * (err * w[m].x - l2 * h[m].x), fh * (err * w[m].y - l2 * h[m].y),
+                                                  fh * (err * w[m].z - l2 * h[m].z), fh * (err * w[m].w - l2 * h[m].w));
                     if (DET) { ((float4*)ow)[c] = dw; ((float4*)oh)[c] = dh; }
                     else { red_add_v4(ow + 4 * c, dw); red_add_v4(oh + 4 * c, dh); }
                 }
@@ -564,6 +662,32 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
         }
     }
     if (!DET) loss_finish(v, my_loss, n, loss_out);
+    if (CLIP && !DET) clip_finish(v, my_clip, my_clipped);
+}
+
+// the finished step's clipping statistics join those of the earlier steps.  Deterministic mode: the
+// per-item values (x = norms applied, y = how many) are summed in a fixed order first.
+__global__ void clip_fold_kernel(DevStat* st, const float2* __restrict__ clip_item, uint64_t n)
+{
+    __shared__ double sh_s[256];
+    __shared__ unsigned long long sh_c[256];
+    double sm = 0.0;
+    unsigned long long cn = 0;
+    if (clip_item) {
+        for (uint64_t i = threadIdx.x; i < n; i += 256) { sm += (double)clip_item[i].x; cn += (unsigned long long)clip_item[i].y; }
+    }
+    sh_s[threadIdx.x] = sm; sh_c[threadIdx.x] = cn;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if ((int)threadIdx.x < o) { sh_s[threadIdx.x] += sh_s[threadIdx.x + o]; sh_c[threadIdx.x] += sh_c[threadIdx.x + o]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        st->clip_sum += sh_s[0] + st->clip_step_sum;
+        st->clip_cnt += sh_c[0] + st->clip_step_cnt;
+        st->clip_step_sum = 0.0;
+        st->clip_step_cnt = 0;
+    }
 }
 
 // mean of the per-item losses, summed in a fixed order
@@ -587,6 +711,7 @@ __global__ void loss_mean_kernel(const float* __restrict__ loss_item, uint64_t n
 // host side
 // ---------------------------------------------------------------------------------------------
 struct StepBuffers {
+    float2* clip_item;      // deterministic mode with clipping: per item (norms applied, how many)
     float* loss_item;
     uint32_t* ukeys;
     float* uval;
@@ -599,12 +724,15 @@ static nups_status step_buffers(nups_store* s, uint64_t n, uint64_t per, bool tw
     const bool det = s->cfg.deterministic;
     uint64_t rows = n * per;
     size_t row_bytes = (size_t)rows * s->L * sizeof(float);
-    size_t need = align256(n * 4);
+    const bool clip = det && s->cfg.clip_factor > 0.f && s->H;
+    size_t need = align256(n * 4) + (clip ? align256(n * 8) : 0);
     if (det) need += align256(rows * 4) + align256(row_bytes) * (two_tables ? 2 : 1) + nups_push_scratch_bytes(s, rows);
     char* sc;
     nups_status rc = nups_scratch(s, need, &sc);
     if (rc != NUPS_OK) return rc;
     b->loss_item = (float*)sc; sc += align256(n * 4);
+    b->clip_item = nullptr;
+    if (clip) { b->clip_item = (float2*)sc; sc += align256(n * 8); }
     b->ukeys = nullptr; b->uval = nullptr; b->uacc = nullptr; b->push_scratch = nullptr;
     if (det) {
         b->ukeys = (uint32_t*)sc; sc += align256(rows * 4);
@@ -616,7 +744,7 @@ static nups_status step_buffers(nups_store* s, uint64_t n, uint64_t per, bool tw
 }
 
 static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, const StepBuffers& b,
-                               float* d_loss_out, cudaStream_t st, bool loss_done_in_kernel = false)
+                               float* d_loss_out, cudaStream_t st, bool loss_done_in_kernel = false, bool clips = false)
 {
     nups_status rc;
     if (s->cfg.deterministic) {
@@ -625,6 +753,10 @@ static nups_status step_finish(nups_store* s, uint64_t n, uint64_t per, const St
     }
     if (d_loss_out && !loss_done_in_kernel) {
         loss_mean_kernel<<<1, 256, 0, st>>>(b.loss_item, n, d_loss_out);
+        LAUNCH_CHECK(s);
+    }
+    if (clips && s->cfg.clip_factor > 0.f && s->H) {
+        clip_fold_kernel<<<1, 256, 0, st>>>(s->st, b.clip_item, n);
         LAUNCH_CHECK(s);
     }
     s->steps++;
@@ -647,6 +779,12 @@ static unsigned step_grid(const nups_store* s, uint64_t n, unsigned blocks_per_s
         else if ((L4) <= 64) { constexpr int CH = 2; __VA_ARGS__; } \
         else if ((L4) <= 96) { constexpr int CH = 3; __VA_ARGS__; } \
         else { constexpr int CH = 4; __VA_ARGS__; }               \
+    } while (0)
+
+#define DISPATCH_CLIP(s, ...)                                                                  \
+    do {                                                                                     \
+        if ((s)->cfg.clip_factor > 0.f && (s)->H) { constexpr bool CLIP = true; __VA_ARGS__; } \
+        else { constexpr bool CLIP = false; __VA_ARGS__; }                                   \
     } while (0)
 
 #define DISPATCH_MODE(s, ...)                                                                \
@@ -680,18 +818,18 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
     const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
     cudaError_t e = cudaSuccess;
 #define NUPS_SGNS_GO(KT_)                                                                                              \
-    DISPATCH_CH(v.L4, DISPATCH_MODE(s, {                                                                               \
-        auto kern = sgns_kernel<HOT, DET, KT_, CH>;                                                               \
+    DISPATCH_CH(v.L4, DISPATCH_MODE(s, DISPATCH_CLIP(s, {                                                              \
+        auto kern = sgns_kernel<HOT, DET, KT_, CH, (HOT && CLIP)>;                                                     \
         if (smem > 48 * 1024)                                                                                          \
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);           \
         if (e == cudaSuccess) {                                                                                        \
             nups_time_begin(s, st);                                                                                    \
             kern<<<grid, 32 * SGNS_WARPS, smem, st>>>(v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
                                                       b.loss_item, d_loss_out, group,                                  \
-                                                      loss_acc);                                                       \
+                                                      loss_acc, b.clip_item);                                          \
             nups_time_end(s, st);                                                                                      \
         }                                                                                                              \
-    }))
+    })))
     if (K == 3) NUPS_SGNS_GO(3);
     else NUPS_SGNS_GO(0);
 #undef NUPS_SGNS_GO
@@ -723,7 +861,7 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
     if (rc != NUPS_OK) return rc;
     rc = sgns_launch(s, d_center, d_context, n, K, lr, b, d_loss_out, 1, nullptr, st);
     if (rc != NUPS_OK) return rc;
-    return step_finish(s, n, K + 2, b, d_loss_out, st, !s->cfg.deterministic);
+    return step_finish(s, n, K + 2, b, d_loss_out, st, !s->cfg.deterministic, true);
 }
 
 // per-step losses of a grouped launch: fixed-point sums -> means, and the sums are cleared for the next group
@@ -756,7 +894,8 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
     cudaStream_t st = (cudaStream_t)stream;
     unsigned long long* acc = (unsigned long long*)s->loss_partial;      // zero between launches
     StepBuffers b;
-    b.loss_item = nullptr; b.ukeys = nullptr; b.uval = nullptr; b.uacc = nullptr; b.push_scratch = nullptr;
+    b.loss_item = nullptr; b.clip_item = nullptr; b.ukeys = nullptr; b.uval = nullptr; b.uacc = nullptr;
+    b.push_scratch = nullptr;
     uint64_t t = 0;
     while (t < steps) {
         // one launch covers the steps up to the next replica merge, as far as their negatives are drawn already
@@ -775,6 +914,10 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
         if (rc != NUPS_OK) return rc;
         loss_group_kernel<<<1, LOSS_STEPS, 0, st>>>(acc, (uint32_t)group, batch, d_loss_out ? d_loss_out + t : nullptr);
         LAUNCH_CHECK(s);
+        if (s->cfg.clip_factor > 0.f && s->H) {
+            clip_fold_kernel<<<1, 256, 0, st>>>(s->st, nullptr, 0);      // the launch's clipping statistics join the rest
+            LAUNCH_CHECK(s);
+        }
         s->steps += group;
         t += group;
         if (s->cfg.sync_interval && s->steps % s->cfg.sync_interval == 0) {
@@ -842,9 +985,21 @@ extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const 
     View v = nups_view(s);
     unsigned grid = step_grid(s, n, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2));   // resident blocks at that depth's register use
     nups_time_begin(s, st);
-    DISPATCH_MODE(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH><<<grid, 128, 0, st>>>(
-        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out)));
+    DISPATCH_MODE(s, DISPATCH_CLIP(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH, (HOT && CLIP)><<<grid, 128, 0, st>>>(
+        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out, b.clip_item))));
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
-    return step_finish(s, n, 2, b, d_loss_out, st, !s->cfg.deterministic);
+    return step_finish(s, n, 2, b, d_loss_out, st, !s->cfg.deterministic, true);
+}
+
+extern "C" nups_status nups_get_clip_stats(nups_store* s, double* h_sum, uint64_t* h_count, void* stream)
+{
+    if (!s || !h_sum || !h_count) return NUPS_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    DevStat d;
+    CK(cudaMemcpyAsync(&d, s->st, sizeof(DevStat), cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    *h_sum = d.clip_sum;
+    *h_count = d.clip_cnt;
+    return NUPS_OK;
 }

@@ -38,6 +38,7 @@ View nups_view(const nups_store* s)
     v.cnt = s->cnt; v.own = s->own; v.epoch_tag = s->epoch << 8; v.st = s->st; v.loss_partial = s->loss_partial;
     v.num_keys = s->num_keys; v.Hcap = s->Hcap; v.H = (uint32_t)s->H; v.L4 = s->L / 4; v.R = s->R;
     v.count = s->cfg.count_accesses;
+    v.clip_factor = s->cfg.clip_factor;
     return v;
 }
 
@@ -149,6 +150,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     if (c.workers == 0) c.workers = 8;
     if (c.workers > 254) return NUPS_EINVAL;
     if (c.sync_period_us && c.deterministic) return NUPS_EINVAL;
+    if (!(c.clip_factor >= 0.f)) return NUPS_EINVAL;
     int dev = 0, count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) {
         snprintf(g_nups_cuda_err, sizeof(g_nups_cuda_err), "no CUDA device");

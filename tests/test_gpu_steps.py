@@ -247,3 +247,83 @@ def test_run_sgns_matches_step_by_step():
     kf = f.pull_sample(f.prepare_sample(df, 50), 50, values=False)
     assert np.array_equal(host_keys(kf), ko)
     assert f.status_check() == 0
+
+
+@pytest.mark.parametrize("K", [3, 5])
+def test_sgns_clipping_of_replicated_key_updates_matches_the_oracle(K):
+    # a learning rate at which the unclipped run blows up (its loss grows step by step): the clipped run stays
+    # put, and the CUDA path follows the oracle through it
+    from paper_2104_00501_b200 import binding
+    V, L, R, batch = 300, 64, 4, 250
+    c, ctx, w = sgns_data(V, 400, 7)
+    init = inputs.normal_init(2 * V, L, 0.3, 7)
+    tables, losses = {}, {}
+    for factor in (0.0, 0.7):
+        o, s = make_pair(2 * V, L, R=R, init=init, deterministic=True, sync_interval=2)
+        s.close()
+        s = binding.Store(2 * V, L, workers=R, sync_interval=2, deterministic=True, clip_factor=factor)
+        s.write_table(0, init)
+        o.set_clipping(factor)
+        o.count_accesses(np.concatenate([c, ctx]))
+        hot = o.select_hot(True, 25)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+        do = o.register_distribution(V, w, V, BOUNDED, U=4, G=50, seed=3)
+        ds = s.register_distribution(V, dev_keys(w), V, BOUNDED, U=4, G=50, seed=3)
+        lb = loss_buf()
+        for b in range(6):
+            sl = slice(b * batch, (b + 1) * batch)
+            lo = o.step_sgns(c[sl], ctx[sl], do, K, 0.2)
+            if factor:
+                s.step_sgns(dev_keys(c[sl]), dev_keys(ctx[sl]), ds, K, 0.2, lb)
+                assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+            losses.setdefault(factor, []).append(lo)
+        o.sync()
+        tables[factor] = o.table().copy()
+        if factor:
+            s.sync()
+            tables_close(o, s)
+            (so, co), (ss, cs) = o.clip_stats(), s.clip_stats()
+            assert co == cs and co > 0 and ss == pytest.approx(so, rel=1e-5)
+            assert s.status_check() == 0
+        else:
+            assert o.clip_stats() == (0.0, 0)
+        s.close()
+    assert not np.array_equal(tables[0.0], tables[0.7])               # the bound was tight enough to bite
+    assert losses[0.7][-1] < losses[0.0][-1]
+
+
+def test_mf_clipping_matches_the_oracle_and_fast_mode_counts_the_same_updates():
+    from paper_2104_00501_b200 import binding
+    M, N, L, R, n = 200, 60, 100, 4, 1500
+    rng = np.random.default_rng(8)
+    rows = inputs.u32(inputs.zipf_keys(n, M, 0.8, 1, "cpu"))
+    cols = (M + inputs.u32(inputs.zipf_keys(n, N, 0.8, 2, "cpu"))).astype(np.uint32)
+    x = rng.normal(0, 1, n).astype(np.float32)
+    init = rng.normal(0, 0.3, (M + N, L)).astype(np.float32)
+    hot = np.unique(np.concatenate([rows[:40], cols[:40]])).astype(np.uint32)
+    o, s0 = make_pair(M + N, L, R=R, init=init, deterministic=True)
+    s0.close()
+    o.set_clipping(0.8)
+    o.set_management(hot, REPLICATE)
+    stores = {}
+    for det in (True, False):
+        s = binding.Store(M + N, L, workers=R, sync_interval=1, deterministic=det, clip_factor=0.8)
+        s.write_table(0, init)
+        s.set_management(dev_keys(hot), REPLICATE)
+        stores[det] = s
+    lb = loss_buf()
+    for b in range(3):
+        sl = slice(b * 500, (b + 1) * 500)
+        lo = o.step_mf(rows[sl], cols[sl], x[sl], 0.05, 0.01)
+        for det, s in stores.items():
+            s.step_mf(dev_keys(rows[sl]), dev_keys(cols[sl]), dev_f32(x[sl]), 0.05, 0.01, lb)
+            if det:
+                assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    tables_close(o, stores[True])
+    so, co = o.clip_stats()
+    for det, s in stores.items():
+        ss, cs = s.clip_stats()
+        assert cs == co
+        assert ss == pytest.approx(so, rel=1e-5 if det else 0.25)
+        s.close()
