@@ -42,7 +42,7 @@ MAX_DISTINCT_BATCHES = 4096
 
 # DRAM traffic of one launch of the fused step kernel (16 steps per launch), from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum); valid only for the kernel source it was captured on.
-NCU_TRAFFIC = {"bytes_per_launch": 41198976, "steps_cu_sha1": "9cde156838943f07d607102e7b1a23cf34e3cf1f"}
+NCU_TRAFFIC = {"bytes_per_launch": 41699200, "steps_cu_sha1": "11ce7c4f854f4e4a5d7ec7ee6f5506810715641f"}
 
 
 def peaks():
@@ -128,9 +128,9 @@ def make_sgns_data(device, n_batches, seed=0, store=None):
     return c, o, counts, weights
 
 
-def build_store(binding, device, n_batches, seed, deterministic=False, sync_interval=SYNC_EVERY):
+def build_store(binding, device, n_batches, seed, deterministic=False, sync_interval=SYNC_EVERY, clip_factor=0.0):
     s = binding.Store(2 * VOCAB, DIM, workers=WORKERS, sync_interval=sync_interval, deterministic=deterministic,
-                      track_ownership=False)
+                      track_ownership=False, clip_factor=clip_factor)
     s.init_uniform(0, 1, 0.5 / DIM)
     c, o, counts, weights = make_sgns_data(device, n_batches, seed, store=s)
     hot = s.select_hot(True, int(HOT_FRACTION * 2 * VOCAB))          # the most frequently accessed 1 % of keys
@@ -471,7 +471,7 @@ def run_sample_sweep(args, device):
         def once():
             h = s.prepare_sample(d, N)
             s.pull_sample(h, N, True, keys, vals)
-        t = _time_calls(once, max(args.steps, 5))
+        t = _time_calls(once, max(args.steps, 1), warm=min(3, args.warmup))
         uniq = int(torch.unique(keys).numel())
         alg = 4 * N + L * 4 * N + L * 4 * uniq + 16 * N
         print(json.dumps({"workload": "PullSample", "level": name, "keys": NK, "value_len": L, "samples": N,
@@ -498,7 +498,8 @@ def run_staleness_sweep(args, device):
         if store is None or interval != prev_interval:
             if store is not None:
                 store.close()
-            store, dist, hot, c, o, weights = build_store(binding, device, nb, seed=0, sync_interval=interval)
+            store, dist, hot, c, o, weights = build_store(binding, device, nb, seed=0, sync_interval=interval,
+                                                          clip_factor=args.clip_factor)
             prev_interval = interval
         else:
             store.sync()
@@ -523,7 +524,8 @@ def run_staleness_sweep(args, device):
         t = e0.elapsed_time(e1) / 1e3
         st = store.stats()
         store.set_sync_period(0)
-        print(json.dumps({"workload": "SGNS, replica staleness", "merge": name, "steps": steps, "seconds": t,
+        print(json.dumps({"workload": "SGNS, replica staleness", "merge": name, "clip_factor": args.clip_factor,
+                          "steps": steps, "seconds": t,
                           "key_accesses_per_s": steps * BATCH * ACCESSES_PER_PAIR / t, "us_per_step": t / steps * 1e6,
                           "background_merges": st["background_merges"] - m0, "loss_last_64_steps": float(losses.mean())}),
               flush=True)
@@ -601,6 +603,8 @@ def main():
     ap.add_argument("--workload", default="sgns", choices=["sgns", "ps", "sample", "kge", "mf", "staleness"])
     ap.add_argument("--hot-fraction", type=float, default=HOT_FRACTION, help="share of keys to replicate (default 0.01)")
     ap.add_argument("--workers", type=int, default=WORKERS)
+    ap.add_argument("--clip-factor", type=float, default=0.0,
+                    help="staleness workload: clip replicated-key updates at this multiple of their mean norm")
     ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
     ap.add_argument("--ps-keys", type=int, default=100_000_000)
     ap.add_argument("--kge-entities", type=int, default=5_000_000, help="smaller for profiling runs")
