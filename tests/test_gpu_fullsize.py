@@ -67,3 +67,39 @@ def test_full_size_fast_mode_tracks_the_oracle_loss():
     assert abs(ls[-16:].mean() - np.mean(lo[-16:])) <= 0.01 * np.mean(lo[-16:])
     assert np.all(np.isfinite(ls))
     assert s.status_check() == 0
+
+
+@pytest.mark.parametrize("level_name", ["CONFORM", "BOUNDED", "LONGTERM", "NONCONFORM"])
+def test_full_size_pull_sample_keys_match_the_oracle(level_name):
+    # the PS sweep's sampling case: 1,048,576 samples per handle from a Zipf(1.0) target over 100M keys, 8 workers,
+    # top-1000 keys replicated, pools of 250 used 16 times; keys bit for bit, with ownership moving between
+    # and inside the calls (rows are 4 floats wide here: the width plays no part in which keys are drawn)
+    import oracle as orc_mod
+    NK, N, R = 100_000_000, 1 << 20, bench.WORKERS
+    level = {"CONFORM": orc_mod.CONFORM, "BOUNDED": orc_mod.BOUNDED, "LONGTERM": orc_mod.LONGTERM,
+             "NONCONFORM": orc_mod.NONCONFORM}[level_name]
+    dev = torch.device("cuda")
+    w_dev = inputs.zipf_integer_weights(NK, 1.0, dev).to(torch.int32).contiguous()
+    w = w_dev.cpu().numpy().view(np.uint32)
+    hot = inputs.u32(inputs.zipf_key_of_rank(NK, dev)[:1000])
+    s = binding.Store(NK, 4, workers=R, deterministic=False, track_ownership=True)
+    o = Oracle(NK, 4, workers=R, track_ownership=True)
+    s.set_management(torch.from_numpy(hot.view(np.int32)).cuda(), binding.REPLICATE)
+    o.set_management(hot, REPLICATE)
+    ds = s.register_distribution(0, w_dev, NK, level, U=bench.U_REUSE, G=bench.G_POOL, seed=23)
+    do = o.register_distribution(0, w, NK, level, U=bench.U_REUSE, G=bench.G_POOL, seed=23)
+    rng = np.random.default_rng(9)
+    for cuts in ([N], [1000, N - 1000]):
+        moved = rng.integers(0, NK, 200_000).astype(np.uint32)
+        o.localize(moved)
+        s.localize(torch.from_numpy(moved.view(np.int32)).cuda())
+        hs, ho = s.prepare_sample(ds, N), o.prepare_sample(do, N)
+        for c in cuts:
+            ks = s.pull_sample(hs, c, values=False)
+            ko = o.pull_sample(ho, c, values=False)
+            assert np.array_equal(host_keys(ks), ko)
+    probe = np.concatenate([moved[:2000], ko[:2000]]).astype(np.uint32)
+    got = s.owner_of(torch.from_numpy(probe.view(np.int32)).cuda()).cpu().numpy()
+    assert np.array_equal(got, np.array([o.owner_of(int(k)) for k in probe]))
+    assert s.status_check() == 0
+    s.close()
