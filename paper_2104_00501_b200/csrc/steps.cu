@@ -120,7 +120,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
     const uint64_t w0 = (uint64_t)blockIdx.x * SGNS_WARPS + wib;
     double my_loss = 0.0;
     const float bound = CLIP ? clip_bound(v) : 0.f;
-    double my_clip = 0.0;                                          // fast mode: norms applied by this warp
+    float my_clip = 0.f;                                           // fast mode: norms applied, this lane's share
     unsigned my_clipped = 0;
     auto key_of = [&](uint64_t e) -> uint32_t {
         if (lane >= per || e >= total) return 0u;
@@ -229,7 +229,8 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
             const float an = sqrtf(warp_sum(a2));
             float applied = 0.f;
             if (lane <= K && (mask >> lane & 1u)) applied = clip_norm(lr * fabsf(g_l) * an, bound, &f_l);
-            clip_sum_item = warp_sum(applied);
+            if (DET) clip_sum_item = warp_sum(applied);            // per item, in a fixed order
+            else my_clip += applied;                               // summed over the lanes when the kernel ends
         }
         float fk[NR];
         if (CLIP && KT > 0) {
@@ -269,7 +270,9 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
                     const float4 gv = gvv[CLIP ? m : 0];
                     g2 += gv.x * gv.x + gv.y * gv.y + gv.z * gv.z + gv.w * gv.w;
                 }
-                clip_sum_item += clip_norm(lr * sqrtf(warp_sum(g2)), bound, &fc);
+                const float applied = clip_norm(lr * sqrtf(warp_sum(g2)), bound, &fc);
+                if (DET) clip_sum_item += applied;
+                else if (lane == 0) my_clip += applied;
             }
             const float sc = -lr * fc;
 #pragma unroll
@@ -281,7 +284,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
                 else red_add_v4((KT > 0 ? dstp[KT > 0 ? KT + 1 : 0] : s_dst[wib][K + 1] + 4 * lane) + 128 * m, dv);
             }
             if (DET) { if (lane == 0) clip_item[i] = make_float2(clip_sum_item, (float)__popc(mask)); }
-            else { my_clip += (double)clip_sum_item; my_clipped += __popc(mask); }
+            else my_clipped += __popc(mask);
         }
         if (lane == 0) {
             if (DET) loss_item[i] = loss_l;
@@ -290,7 +293,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
         }
     }
     if (!DET && !loss_acc) loss_finish(v, my_loss, n, loss_out);
-    if (CLIP && !DET) clip_finish(v, my_clip, my_clipped);
+    if (CLIP && !DET) clip_finish(v, (double)warp_sum(my_clip), my_clipped);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -534,7 +537,7 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
     const float4* slab4 = (const float4*)v.dval;
     double my_loss = 0.0;
     const float bound = CLIP ? clip_bound(v) : 0.f;
-    double my_clip = 0.0;
+    float my_clip = 0.f;
     unsigned my_clipped = 0;
 
     // ring A: keys and cell values of the items 2*MF_DEPTH .. MF_DEPTH+1 steps ahead
@@ -627,7 +630,7 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
                 if (sj >= 0) { applied += clip_norm(lr * sqrtf(warp_sum(nh2)), bound, &f); fh = lr * f; }
                 const unsigned hot_roles = (si >= 0 ? 1u : 0u) + (sj >= 0 ? 1u : 0u);
                 if (DET) { if (lane == 0) clip_item[i] = make_float2(applied, (float)hot_roles); }
-                else { my_clip += (double)applied; my_clipped += hot_roles; }
+                else { my_clip += applied; my_clipped += hot_roles; }
             } else if (CLIP && DET && lane == 0) {
                 clip_item[i] = make_float2(0.f, 0.f);
             }
@@ -662,7 +665,7 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
         }
     }
     if (!DET) loss_finish(v, my_loss, n, loss_out);
-    if (CLIP && !DET) clip_finish(v, my_clip, my_clipped);
+    if (CLIP && !DET) clip_finish(v, (double)my_clip, my_clipped);
 }
 
 // the finished step's clipping statistics join those of the earlier steps.  Deterministic mode: the
