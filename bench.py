@@ -42,7 +42,7 @@ MAX_DISTINCT_BATCHES = 4096
 
 # DRAM traffic of one launch of the fused step kernel (16 steps per launch), from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum); valid only for the kernel source it was captured on.
-NCU_TRAFFIC = {"bytes_per_launch": 41699200, "steps_cu_sha1": "11ce7c4f854f4e4a5d7ec7ee6f5506810715641f"}
+NCU_TRAFFIC = {"bytes_per_launch": 41385472, "steps_cu_sha1": "658662f0c0d79163ca262348586c4cafc65d2e00"}
 
 
 def peaks():
@@ -199,25 +199,54 @@ def run_ours(args, rank, world, device):
     launches = s.stats()["launches"] - launches0
     final_loss = float(loss.item())
 
-    # end to end: pairs start in pinned host memory, the loss is read back every step
-    # (centre and context keys of a batch sit side by side in one pinned buffer: one copy per step)
+    # end to end through the public API (`Store.run_sgns`, CHUNK steps per call, as in the device-timed loop): every
+    # step's pairs start in pinned host memory and are copied to the device inside the timed region, every step's
+    # loss is copied back and read by the host.  Two buffers in flight: the host waits for call k-1's losses to
+    # have landed before it issues call k+1.
+    n_chunks = nb // CHUNK if nb >= CHUNK else 0
+    e2e_steps = min(args.steps, nb) // CHUNK * CHUNK if n_chunks else 0
+    e2e_s = float("nan")
+    if e2e_steps:
+        hchunks = torch.stack([c.view(n_chunks, CHUNK * BATCH), o.view(n_chunks, CHUNK * BATCH)], dim=1).cpu().pin_memory()
+        dbuf = [torch.empty(2, CHUNK * BATCH, dtype=torch.int32, device=device) for _ in range(2)]
+        dls = [torch.zeros(CHUNK, device=device) for _ in range(2)]
+        hls = [torch.zeros(CHUNK, dtype=torch.float32).pin_memory() for _ in range(2)]
+        done = [torch.cuda.Event(), torch.cuda.Event()]
+        seen = 0.0
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(e2e_steps // CHUNK):
+            k = i & 1
+            if i >= 2:
+                done[k].synchronize()
+                seen += float(hls[k].sum())                   # the host really reads every step's loss
+            dbuf[k].copy_(hchunks[i % n_chunks], non_blocking=True)
+            s.run_sgns(dbuf[k][0], dbuf[k][1], BATCH, dist, NEG, LR, dls[k])
+            hls[k].copy_(dls[k], non_blocking=True)
+            done[k].record()
+        for k in range(2):
+            done[k].synchronize()
+            seen += float(hls[k].sum())
+        barrier()
+        e2e_s = time.perf_counter() - t0
+        assert np.isfinite(seen)
+
+    # the same with one library call per step (`Store.step_sgns`): what a caller pays who needs every step's loss
+    # before it decides on the next step
     hpairs = torch.stack([c.view(nb, BATCH), o.view(nb, BATCH)], dim=1).cpu().pin_memory()      # [nb, 2, BATCH]
-    dpairs = torch.empty(2, BATCH, dtype=torch.int32, device=device)
-    hl = torch.zeros(1, dtype=torch.float32).pin_memory()
-    e2e_steps = min(args.steps, 2048)
-    barrier()
-    t0 = time.perf_counter()
-    # two buffers in flight: the host waits for step k-1's loss to have landed before it issues step k+1
-    dpairs2 = [dpairs, torch.empty_like(dpairs)]
-    hl2 = [hl, torch.zeros(1, dtype=torch.float32).pin_memory()]
+    step_calls = min(args.steps, 2048)
+    dpairs2 = [torch.empty(2, BATCH, dtype=torch.int32, device=device) for _ in range(2)]
+    hl2 = [torch.zeros(1, dtype=torch.float32).pin_memory() for _ in range(2)]
     dl2 = [torch.zeros(1, device=device), torch.zeros(1, device=device)]
     done = [torch.cuda.Event(), torch.cuda.Event()]
     seen = 0.0
-    for i in range(e2e_steps):
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(step_calls):
         k = i & 1
         if i >= 2:
             done[k].synchronize()
-            seen += float(hl2[k][0])                      # the host really reads every step's loss
+            seen += float(hl2[k][0])
         dpairs2[k].copy_(hpairs[i % nb], non_blocking=True)
         s.step_sgns(dpairs2[k][0], dpairs2[k][1], dist, NEG, LR, dl2[k])
         hl2[k].copy_(dl2[k], non_blocking=True)
@@ -226,7 +255,10 @@ def run_ours(args, rank, world, device):
         done[k].synchronize()
         seen += float(hl2[k][0])
     barrier()
-    e2e_s = time.perf_counter() - t0
+    per_step_s = time.perf_counter() - t0
+    e2e_steps_per_call = CHUNK
+    if not e2e_steps:                                         # runs too short for one chunked call
+        e2e_steps, e2e_s, e2e_steps_per_call = step_calls, per_step_s, 1
 
     # roofline of the dominant kernel (the fused step kernel) in the launch configuration that was timed above:
     # event pairs on its stream around every launch (one launch = the steps between two replica merges)
@@ -255,7 +287,7 @@ def run_ours(args, rank, world, device):
     sha = hashlib.sha1(open(os.path.join(ROOT, "paper_2104_00501_b200", "csrc", "steps.cu"), "rb").read()).hexdigest()
     traffic = NCU_TRAFFIC["bytes_per_launch"] if NCU_TRAFFIC["steps_cu_sha1"] == sha else None
 
-    ms, e2e_s = max_over_ranks([ms, e2e_s], world, device)
+    ms, e2e_s, per_step_s = max_over_ranks([ms, e2e_s, per_step_s], world, device)
     pairs = args.steps * BATCH * world
     value = aggregate_throughput(args.steps * BATCH * ACCESSES_PER_PAIR, ms / 1e3, world)
     out = {
@@ -272,7 +304,10 @@ def run_ours(args, rank, world, device):
         "final_loss": final_loss,
         "clocks": clk.summary(),
         "e2e": {"value": e2e_steps * BATCH * world * ACCESSES_PER_PAIR / e2e_s, "unit": "key accesses/s",
-                "h2d_bytes_per_step": 2 * BATCH * 4, "d2h_bytes_per_step": 4, "steps": e2e_steps},
+                "h2d_bytes_per_step": 2 * BATCH * 4, "d2h_bytes_per_step": 4, "steps": e2e_steps,
+                "steps_per_call": e2e_steps_per_call,
+                "one_call_per_step": {"value": step_calls * BATCH * world * ACCESSES_PER_PAIR / per_step_s,
+                                      "unit": "key accesses/s", "steps": step_calls}},
         "gpu_launches": int(launches),
         "roofline": {"bound": "hbm", "kernel": "sgns_kernel (fused step)", "achieved": alg_bytes / k_s / 1e9,
                      "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
