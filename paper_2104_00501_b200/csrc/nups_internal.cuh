@@ -113,6 +113,8 @@ struct nups_store {
     double ev_ms;              // time of pairs folded in when the ring filled up
     uint64_t ev_launches;
     struct nups_background* bg; // time-based replica synchronisation (background.cu); NULL = never started
+    cudaStream_t side;          // nups_run_sgns: a due replica merge runs here, beside the next steps' sample draw
+    cudaEvent_t side_fork, side_join;
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };

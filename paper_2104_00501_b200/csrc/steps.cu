@@ -899,11 +899,23 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
     StepBuffers b;
     b.loss_item = nullptr; b.clip_item = nullptr; b.ukeys = nullptr; b.uval = nullptr; b.uacc = nullptr;
     b.push_scratch = nullptr;
+    // A replica merge that falls due while more steps of this call follow runs on a stream of its own, beside the
+    // draw of the next steps' negatives (the draw touches neither replicas nor rows); the next step kernel waits for it.
+    if (!s->side) {
+        CK(cudaStreamCreateWithFlags(&s->side, cudaStreamNonBlocking));
+        CK(cudaEventCreateWithFlags(&s->side_fork, cudaEventDisableTiming));
+        CK(cudaEventCreateWithFlags(&s->side_join, cudaEventDisableTiming));
+    }
+    bool merge_in_flight = false;
     uint64_t t = 0;
     while (t < steps) {
         // one launch covers the steps up to the next replica merge, as far as their negatives are drawn already
         rc = nups_draw_negatives(s, dist, batch * K, st);                 // this step's negatives (may draw ahead)
         if (rc != NUPS_OK) return rc;
+        if (merge_in_flight) {
+            CK(cudaStreamWaitEvent(st, s->side_join, 0));
+            merge_in_flight = false;
+        }
         uint64_t group = 1;
         if (s->ahead_dist == dist && s->ahead_N == batch * K) group += s->ahead_total - s->ahead_next;
         if (group > steps - t) group = steps - t;
@@ -924,8 +936,17 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
         s->steps += group;
         t += group;
         if (s->cfg.sync_interval && s->steps % s->cfg.sync_interval == 0) {
-            rc = nups_sync_internal(s, st);
-            if (rc != NUPS_OK) return rc;
+            if (t < steps) {
+                CK(cudaEventRecord(s->side_fork, st));
+                CK(cudaStreamWaitEvent(s->side, s->side_fork, 0));
+                rc = nups_sync_internal(s, s->side);
+                if (rc != NUPS_OK) return rc;
+                CK(cudaEventRecord(s->side_join, s->side));
+                merge_in_flight = true;
+            } else {
+                rc = nups_sync_internal(s, st);
+                if (rc != NUPS_OK) return rc;
+            }
         }
     }
     return NUPS_OK;

@@ -211,6 +211,7 @@ extern "C" nups_status nups_destroy(nups_store* s)
     if (!s) return NUPS_OK;
     nups_background_stop(s);
     cudaDeviceSynchronize();
+    if (s->side) { cudaStreamDestroy(s->side); cudaEventDestroy(s->side_fork); cudaEventDestroy(s->side_join); }
     for (int i = 0; i < NUPS_MAX_HANDLES; ++i) cudaFree(s->handle[i].buf);
     for (int i = 0; i < NUPS_MAX_DISTS; ++i) { cudaFree(s->dist[i].table); cudaFree(s->dist[i].off); }
     cudaFree(s->val); cudaFree(s->acc); cudaFree(s->hot_bits); cudaFree(s->slot_of); cudaFree(s->hot_keys);
