@@ -134,13 +134,19 @@ def mf_cells(num: int, rows: int, cols: int, s: float, rank: int, noise: float, 
     g = _gen(seed + 77, device)
     sigma = float(rank) ** -0.25
 
+    def mix(z):
+        # 64-bit finaliser (multiply / xor-shift rounds, wrapping int64 arithmetic): neighbouring inputs give
+        # unrelated outputs, so the components of a factor row are independent
+        for mul in (-4658895280553007687, -7723592293110705685):     # 0xBF58476D1CE4E5B9, 0x94D049BB133111EB as int64
+            z = (z ^ ((z >> 30) & 0x3FFFFFFFF)) * mul
+        return z ^ ((z >> 31) & 0x1FFFFFFFF)
+
     def factor(idx, salt):
         comp = torch.arange(rank, device=device, dtype=torch.int64).unsqueeze(0)
-        h = (idx.unsqueeze(1) * 1000003 + comp * 7919 + salt + factor_seed) % 2147483647
-        h = (h * 48271) % 2147483647
-        h2 = (h * 69621) % 2147483647
-        u1 = (h.to(torch.float64) + 1.0) / 2147483648.0
-        u2 = h2.to(torch.float64) / 2147483647.0
+        z = mix(idx.unsqueeze(1) * 1000003 + comp * 7919 + (salt * 104729 + factor_seed))
+        z2 = mix(z + 0x632BE5AB)
+        u1 = ((z >> 11) & ((1 << 52) - 1)).to(torch.float64) / float(1 << 52) + 2.0 ** -53
+        u2 = ((z2 >> 11) & ((1 << 52) - 1)).to(torch.float64) / float(1 << 52)
         return torch.sqrt(-2.0 * torch.log(u1)) * torch.cos(2.0 * math.pi * u2) * sigma
 
     x = torch.empty(num, device=device, dtype=torch.float64)
