@@ -444,6 +444,19 @@ def run_ps_sweep(args, device):
                 alg = 4 * N + row * N + (1 if op == "pull" else 2) * row * ucold
                 res[op] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
                            "frac": alg / t / 1e9 / hbm_peak, "logical_gbs": (4 * N + (2 if op == "pull" else 3) * row * N) / t / 1e9}
+            if topk:
+                # pull again while the replicas hold unmerged updates (the pulls above saw freshly merged replicas,
+                # whose rows need not be read)
+                for i in range(4):
+                    s.push(batches[i % 4], delta)
+                s.kernel_time()
+                for i in range(reps):
+                    s.pull(batches[i % 4], out)
+                ms, n = s.kernel_time()
+                t = ms / 1e3 / n
+                alg = 4 * N + row * N + row * ucold
+                res["pull_with_pending_updates"] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
+                                                    "frac": alg / t / 1e9 / hbm_peak}
             # replica merge cost: pushes with a merge every `interval` pushes, time per push including its share
             sync_sweep = {}
             if topk:
