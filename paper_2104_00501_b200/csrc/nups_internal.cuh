@@ -177,7 +177,8 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
                                    const float* d_dval, const float* d_dacc, char* scratch, cudaStream_t st);
 nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
                                  float* d_out_acc, int worker_map, uint64_t map_base, uint64_t map_total,
-                                 int do_count, cudaStream_t st);
+                                 int do_count, cudaStream_t st,
+                                 uint32_t* d_keys_copy /* nullable: also write the keys here */);
 nups_status nups_sync_internal(nups_store* s, cudaStream_t st);
 // sampling.cu internals used by steps.cu
 nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStream_t st);

@@ -347,7 +347,7 @@ __global__ void draw_iid_kernel(View v, DrawParams p, const unsigned long long* 
 // interleaved ([element][pass]) so that the threads of a warp work side by side in shared memory;
 // drawing the swap partners and writing the output are block-wide.
 // Shared memory: pool[G] (u32) | partner[G][T] (u16) | perm[G][T] (u16).
-constexpr unsigned REUSE_THREADS = 256;
+constexpr unsigned REUSE_THREADS = 512;
 struct ReuseShape {
     unsigned T;
     size_t smem;
@@ -553,8 +553,8 @@ __global__ void emit_kernel(View v, DrawParams p, HandleView h, uint64_t N, uint
 // postponed ones are emitted.  Locality is judged by the ownership at the start of the call.
 // Where an entry goes depends only on how many local entries lie before it, so the walk is a
 // prefix sum, not a loop: (1) one bit per fresh entry, looked up by the whole GPU; (2) per sub-handle,
-// a scan of the bit counts that also finds where the walk stops; (3) every entry is placed on its
-// own; (4) postponed entries are emitted where needed and what was postponed moves to its worker.
+// a scan of the bit counts that also finds where the walk stops (and emits entries that earlier calls
+// postponed); (3) every entry is placed on its own, and what is postponed moves to its worker.
 struct LtChunk {
     uint32_t q;
     uint64_t b0, size, take, out_base;
@@ -592,8 +592,10 @@ constexpr int LT_THREADS = 1024;
 constexpr int LT_WORDS = 4;                  // flag words per thread and round of the scan
 
 __global__ void __launch_bounds__(LT_THREADS)
-lt_scan_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
+lt_scan_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
+               uint32_t* __restrict__ out)
 {
+    __shared__ unsigned sh_tl, sh_old;
     __shared__ unsigned warp_tot[LT_THREADS / 32];
     __shared__ unsigned long long sh_stop;       // walk position right after the last entry that must be emitted
     const LtChunk c = lt_chunk(q_first + blockIdx.x, N, v.R, cursor, n);
@@ -654,6 +656,22 @@ lt_scan_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, ui
         h.prev[c.q] = stt;
         h.walk[c.q] = make_uint4((unsigned)tc, (unsigned)tl, (unsigned)cnt, 0u);
         h.state[c.q] = make_uint4((unsigned)(oc + tc), (unsigned)(ph + cnt), (unsigned)(pt + tc - tl), 0u);
+        sh_tl = (unsigned)tl;
+        sh_old = (unsigned)(cnt < pt - ph ? cnt : pt - ph);         // postponed by earlier calls, emitted by this one
+    }
+    __syncthreads();
+    // postponed entries come after the local ones; those that earlier calls postponed are already in place
+    // (what this call postpones and emits is handled where it is placed)
+    const unsigned tl = sh_tl, old = sh_old;
+    for (unsigned j0 = 0; j0 < old; j0 += LT_THREADS) {
+        const unsigned j = j0 + tid;
+        const bool in = j < old;
+        uint32_t key = 0;
+        if (in) {
+            key = h.post[c.b0 + ph + j];
+            out[c.out_base + tl + j] = key;
+        }
+        count_sample(v, key, in);
     }
 }
 
@@ -663,7 +681,8 @@ __global__ void lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t curso
     const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
     if (!c.active) return;
     const unsigned lane = threadIdx.x & 31;
-    const uint64_t oc = h.prev[c.q].x, pt = h.prev[c.q].z, end = oc + h.walk[c.q].x;
+    const uint4 pv = h.prev[c.q], wk = h.walk[c.q];
+    const uint64_t oc = pv.x, ph = pv.y, pt = pv.z, end = oc + wk.x, tl = wk.y, cnt = wk.z;
     const uint64_t word = (oc >> 5) + (((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5);
     if (word * 32 >= end) return;
     const uint64_t i = word * 32 + lane;
@@ -672,31 +691,26 @@ __global__ void lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t curso
     const uint64_t before = (uint64_t)h.prefix[(c.b0 >> 5) + c.q + word] + __popc(bits & ((1u << lane) - 1u));
     const bool loc = (bits >> lane) & 1u;
     uint32_t key = 0;
+    bool emitted = false;
     if (walked) {
         key = h.keys[c.b0 + i];
-        if (loc) out[c.out_base + before] = key;
-        else h.post[c.b0 + pt + ((i - oc) - before)] = key;          // non-local entries before it
+        if (loc) {
+            out[c.out_base + before] = key;
+            emitted = true;
+        } else {
+            // postponed: queued behind the non-local entries before it, emitted by this very call if the queue's
+            // head gets that far, and moved to the worker.  (Locality was judged before any key moved: the bits
+            // were all looked up by the kernel before this one.)
+            const uint64_t at = pt + ((i - oc) - before);
+            h.post[c.b0 + at] = key;
+            if (at >= ph && at < ph + cnt) {
+                out[c.out_base + tl + (at - ph)] = key;
+                emitted = true;
+            }
+            mark_localize(v, key, c.q);
+        }
     }
-    count_sample(v, key, walked && loc);
-}
-
-__global__ void lt_finish_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
-                                 uint32_t* __restrict__ out)
-{
-    const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
-    if (!c.active) return;
-    const uint4 pv = h.prev[c.q], wk = h.walk[c.q];
-    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const bool in = t < wk.z;                                       // a postponed entry to emit
-    uint32_t key = 0;
-    if (in) {
-        key = h.post[c.b0 + pv.y + t];
-        out[c.out_base + wk.y + t] = key;
-    }
-    count_sample(v, key, in);
-    // what this call postponed moves to the worker (when the call ends: the walk judged locality by
-    // the ownership from before the call)
-    if (t < (uint64_t)wk.x - wk.y) mark_localize(v, h.post[c.b0 + pv.z + t], c.q);
+    count_sample(v, key, emitted);
 }
 
 static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_keys_out, float* d_vals_out,
@@ -722,21 +736,25 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
             if (b0 <= h.cursor + n - 1 && h.cursor + n - 1 < b1) ql = q;
         }
         const uint64_t max_size = (h.N + s->R - 1) / s->R;
-        const dim3 by_word(grid_for(max_size / 32 + 2, 8), ql - qf + 1), by_entry(grid_for(max_size, 256), ql - qf + 1);
+        const dim3 by_word(grid_for(max_size / 32 + 2, 8), ql - qf + 1);
         lt_flags_kernel<<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
         LAUNCH_CHECK(s);
-        lt_scan_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
+        lt_scan_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
         LAUNCH_CHECK(s);
         lt_place_kernel<<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
         LAUNCH_CHECK(s);
-        lt_finish_kernel<<<by_entry, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
-        LAUNCH_CHECK(s);
+    } else if (d_vals_out && d.level != NUPS_NONCONFORM && !s->cfg.count_accesses) {
+        // keys fixed at PrepareSample and nothing to count: the row gather reads them from the handle and hands them out
+        // on its way, which saves a launch
+        h.cursor += n;
+        if (h.cursor == h.N) h.used = 0;
+        return nups_gather_internal(s, hv.keys + (h.cursor - n), n, d_vals_out, nullptr, 1, h.cursor - n, h.N, 0, st, d_keys_out);
     } else {
         emit_kernel<<<grid_for(n, 256), 256, 0, st>>>(v, p, hv, h.N, h.cursor, n, d.level == NUPS_NONCONFORM, d_keys_out);
         LAUNCH_CHECK(s);
     }
     if (d_vals_out) {
-        nups_status rc = nups_gather_internal(s, d_keys_out, n, d_vals_out, nullptr, 1, h.cursor, h.N, 0, st);
+        nups_status rc = nups_gather_internal(s, d_keys_out, n, d_vals_out, nullptr, 1, h.cursor, h.N, 0, st, nullptr);
         if (rc != NUPS_OK) return rc;
     }
     h.cursor += n;

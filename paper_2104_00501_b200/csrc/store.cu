@@ -291,7 +291,7 @@ struct TablePair {
 template <bool HOT, bool TWO>
 __global__ void __launch_bounds__(256, 4)
 gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A, TablePair B, int map,
-              uint64_t map_base, uint64_t map_total, int do_count)
+              uint64_t map_base, uint64_t map_total, int do_count, uint32_t* __restrict__ keys_copy)
 {
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -314,6 +314,7 @@ gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A
         key_b = base + 2 * stride + lane < n ? __ldg(keys + base + 2 * stride + lane) : 0u;
         const bool valid = in && key < v.num_keys;
         if (in && !valid) flag_bad_key(v);
+        if (keys_copy && in) keys_copy[i] = key;                   // PullSample hands the keys out as well
         unsigned long long src = valid ? (unsigned long long)key * L4 : NO_ROW;   // NO_ROW: zero-filled output
         unsigned long long pend = NO_ROW;
         if (HOT && valid && ((bits >> (key & 31)) & 1u)) {
@@ -409,7 +410,8 @@ __device__ __forceinline__ void st8_stream(float* p, const F8& r)
 template <bool HOT, int C8>
 __global__ void __launch_bounds__(256, 4)
 gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const float* __restrict__ table,
-               const float* slab, float* __restrict__ out, int map, uint64_t map_base, uint64_t map_total, int do_count)
+               const float* slab, float* __restrict__ out, int map, uint64_t map_base, uint64_t map_total, int do_count,
+               uint32_t* __restrict__ keys_copy)
 {
     constexpr int RPI = 32 / C8;                       // rows per warp instruction
     constexpr int UNR = 2;                             // instructions in flight
@@ -433,6 +435,7 @@ gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const floa
         key_b = base + 2 * stride + lane < n ? __ldg(keys + base + 2 * stride + lane) : 0u;
         const bool valid = in && key < v.num_keys;
         if (in && !valid) flag_bad_key(v);
+        if (keys_copy && in) keys_copy[i] = key;                   // PullSample hands the keys out as well
         // row numbers instead of offsets: one 32-bit shuffle each; 0xFFFFFFFF = no such row
         uint32_t src = valid ? key : 0xFFFFFFFFu;
         uint32_t pend = 0xFFFFFFFFu;                    // replica row (worker * Hcap + slot) of a replicated key
@@ -488,7 +491,7 @@ gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const floa
 
 nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
                                  float* d_out_acc, int worker_map, uint64_t map_base, uint64_t map_total,
-                                 int do_count, cudaStream_t st)
+                                 int do_count, cudaStream_t st, uint32_t* d_keys_copy)
 {
     if (n == 0 || (!d_out_val && !d_out_acc)) return NUPS_OK;
     View v = nups_view(s);
@@ -510,7 +513,7 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
         nups_time_begin(s, st);
 #define NUPS_G8(C8_)                                                                                                     \
         gather8_kernel<true, C8_><<<grid, 256, 0, st>>>(v, d_keys, n, table, slab, out1, worker_map, map_base, map_total, \
-                                                        do_count)
+                                                        do_count, d_keys_copy)
         if (c8 == 8) NUPS_G8(8);
         else if (c8 == 16) NUPS_G8(16);
         else NUPS_G8(32);
@@ -521,11 +524,11 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
     }
     nups_time_begin(s, st);
     if (s->H) {
-        if (two) gather_kernel<true, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
-        else gather_kernel<true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
+        if (two) gather_kernel<true, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
+        else gather_kernel<true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
     } else {
-        if (two) gather_kernel<false, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
-        else gather_kernel<false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count);
+        if (two) gather_kernel<false, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
+        else gather_kernel<false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
     }
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
@@ -538,7 +541,7 @@ extern "C" nups_status nups_pull2(nups_store* s, const uint32_t* d_keys, uint64_
     if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
     if (d_out_acc && !s->acc) return NUPS_EINVAL;
     if (n && !d_out_val && !d_out_acc) return NUPS_EINVAL;
-    return nups_gather_internal(s, d_keys, n, d_out_val, d_out_acc, 0, 0, n, 1, (cudaStream_t)stream);
+    return nups_gather_internal(s, d_keys, n, d_out_val, d_out_acc, 0, 0, n, 1, (cudaStream_t)stream, nullptr);
 }
 
 extern "C" nups_status nups_pull(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out, void* stream)
