@@ -365,9 +365,13 @@ static unsigned reuse_pools(uint64_t max_size, uint32_t U, uint32_t G)
     return (unsigned)(max_size / ((uint64_t)U * G) + 2);      // a stretch may begin and end inside a pool
 }
 
-template <class Emit>
+// emit(in, key, position in the stretch, mark): called by whole warps for every output position; `mark` says
+// whether the key still has to be localized there.  When a whole pass of the pool lies inside the stretch, every
+// key of the pool is sampled by this call, so the pool's keys are localized once each (mark_key) instead of once
+// per output position (U times as often).
+template <class Emit, class Mark>
 __device__ __forceinline__ void reuse_pool_visit(const DrawParams& p, uint32_t q, unsigned long long s0,
-                                                 unsigned long long s1, uint32_t T, Emit emit)
+                                                 unsigned long long s1, uint32_t T, Emit emit, Mark mark_key)
 {
     extern __shared__ __align__(16) uint32_t reuse_mem[];
     const uint32_t G = p.G, U = p.U;
@@ -378,7 +382,18 @@ __device__ __forceinline__ void reuse_pool_visit(const DrawParams& p, uint32_t q
     uint32_t* pool = reuse_mem;
     uint16_t* partner = reinterpret_cast<uint16_t*>(reuse_mem + G);
     uint16_t* perm = partner + (size_t)T * G;
-    for (uint32_t m = tid; m < G; m += blockDim.x) pool[m] = draw_iid(p, q, pl * G + m);
+    bool whole_pass;                                         // does a pass of this pool lie fully inside [s0, s1)?
+    {
+        const unsigned long long first = (s0 + G - 1) / G, last_plus_1 = s1 / G;           // passes fully inside
+        const unsigned long long lo = first > pl * U ? first : pl * U;
+        const unsigned long long hi = last_plus_1 < (pl + 1) * U ? last_plus_1 : (pl + 1) * U;
+        whole_pass = lo < hi;
+    }
+    for (uint32_t m = tid; m < G; m += blockDim.x) {
+        const uint32_t k = draw_iid(p, q, pl * G + m);
+        pool[m] = k;
+        if (whole_pass) mark_key(k);
+    }
     const uint32_t blocks_per_pass = (G + 2) / 4;            // Philox blocks that hold the G - 1 shuffle words
     for (uint32_t t0 = 0; t0 < U; t0 += T) {
         const uint32_t nt = U - t0 < T ? U - t0 : T;
@@ -428,7 +443,7 @@ __device__ __forceinline__ void reuse_pool_visit(const DrawParams& p, uint32_t q
             const unsigned long long sp = (pass0 + t) * G + j;
             const bool in = e < total && sp >= s0 && sp < s1;
             const uint32_t k = in ? pool[perm[(size_t)j * T + t]] : 0u;
-            emit(in, k, sp - s0);
+            emit(in, k, sp - s0, !whole_pass);
         }
     }
 }
@@ -445,12 +460,12 @@ __global__ void draw_reuse_kernel(View v, DrawParams p, const unsigned long long
         if (longterm) h.state[q] = make_uint4(0u, 0u, 0u, 0u);
     }
     if (size == 0) return;
-    reuse_pool_visit(p, q, s0, s0 + size, T, [&](bool in, uint32_t k, unsigned long long rel) {
+    reuse_pool_visit(p, q, s0, s0 + size, T, [&](bool in, uint32_t k, unsigned long long rel, bool mark) {
         if (in) {
             h.keys[b0 + rel] = k;
-            if (localize) mark_localize(v, k, q);
+            if (localize && mark) mark_localize(v, k, q);
         }
-    });
+    }, [&](uint32_t k) { if (localize) mark_localize(v, k, q); });
 }
 
 static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int* slot_out, cudaStream_t st)
@@ -814,13 +829,13 @@ __global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned lo
     if (size == 0) return;
     out += (uint64_t)blockIdx.z * N;
     const unsigned long long s0 = off_cur[q] + (unsigned long long)blockIdx.z * size;
-    reuse_pool_visit(p, q, s0, s0 + size, T, [&](bool in, uint32_t k, unsigned long long rel) {
+    reuse_pool_visit(p, q, s0, s0 + size, T, [&](bool in, uint32_t k, unsigned long long rel, bool mark) {
         if (in) {
             out[b0 + rel] = k;
-            if (localize) mark_localize(v, k, q);
+            if (localize && mark) mark_localize(v, k, q);
         }
         count_sample(v, k, in);
-    });
+    }, [&](uint32_t k) { if (localize) mark_localize(v, k, q); });
 }
 
 // Sample-ahead for the workload steps.  The sample streams are a pure function of (seed, worker,
