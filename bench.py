@@ -633,9 +633,17 @@ def run_step_workload(args, device, which):
     k_s = k_ms / 1e3 / max(k_n, 1)
     tables = 2 if which == "kge" else 1
     logical = B * rows_per_item * L * 4 * 2 * (1 if which == "mf" else 1)      # every touched row read and written once
+    # What the atomic update path allows: nearly all rows of these steps are cold, so every row is read once (at best
+    # at the copy peak) and every update is a floating-point reduction to a DRAM-resident row, whose rate the library
+    # measures by itself.  floor = both in full overlap, read_then_reduce = one after the other.
+    red_dram = s.probe_reduction_rate(2 << 30, 5)
+    t_read, t_red = (logical / 2) / (hbm_peak * 1e9), (logical / 2) / (red_dram * 1e9)
     print(json.dumps({"workload": cfg, "kernel": name, "hot_slots": s.stats()["hot_slots"], "us_per_step": dt * 1e6,
                       "kernel_us": k_s * 1e6, "key_accesses_per_s": B * per_item / dt, "updates_per_s": B * upd / dt,
                       "logical_gbs": logical / k_s / 1e9, "logical_frac_of_hbm_peak": logical / k_s / 1e9 / hbm_peak,
+                      "reduction_rate_dram_gbs": red_dram, "floor_us_reads_and_reductions_overlapped": max(t_read, t_red) * 1e6,
+                      "us_read_then_reduce": (t_read + t_red) * 1e6,
+                      "frac_of_overlapped_floor": max(t_read, t_red) / k_s,
                       "peak_kind": peak_kind, "final_loss": float(loss.item()), "tables": tables}), flush=True)
     s.close()
 

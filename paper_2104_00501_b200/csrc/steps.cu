@@ -524,7 +524,7 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
 constexpr int MF_DEPTH = NUPS_MF_DEPTH;
 
 template <bool HOT, bool DET, int CH, bool CLIP>
-__global__ void __launch_bounds__(128)
+__global__ void __launch_bounds__(128, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2))      // the grid is sized for this many blocks per SM
 mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
           uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
           float* __restrict__ loss_item, float* __restrict__ loss_out, float2* __restrict__ clip_item)
