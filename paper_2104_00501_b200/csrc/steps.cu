@@ -817,15 +817,18 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
     if (per_sm < 1) per_sm = 1;
     const uint64_t items = n * group;
     const uint64_t blocks_needed = (items + SGNS_WARPS - 1) / SGNS_WARPS;
-    const uint64_t cap = (uint64_t)s->sm_count * per_sm;
-    const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
     cudaError_t e = cudaSuccess;
 #define NUPS_SGNS_GO(KT_)                                                                                              \
     DISPATCH_CH(v.L4, DISPATCH_MODE(s, DISPATCH_CLIP(s, {                                                              \
         auto kern = sgns_kernel<HOT, DET, KT_, CH, (HOT && CLIP)>;                                                     \
         if (smem > 48 * 1024)                                                                                          \
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);           \
+        int fit = 0;       /* registers may allow fewer resident blocks than shared memory does: no second wave */ \
+        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kern, 32 * SGNS_WARPS, smem);    \
         if (e == cudaSuccess) {                                                                                        \
+            if (fit >= 1 && (unsigned)fit < per_sm) per_sm = (unsigned)fit;                                            \
+            const uint64_t cap = (uint64_t)s->sm_count * per_sm;                                                       \
+            const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);                               \
             nups_time_begin(s, st);                                                                                    \
             kern<<<grid, 32 * SGNS_WARPS, smem, st>>>(v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
                                                       b.loss_item, d_loss_out, group,                                  \
@@ -836,7 +839,7 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
     if (K == 3) NUPS_SGNS_GO(3);
     else NUPS_SGNS_GO(0);
 #undef NUPS_SGNS_GO
-    if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
+    if (e != cudaSuccess) return nups_cuda_fail(e, "skip-gram kernel set-up");
     LAUNCH_CHECK(s);
     return NUPS_OK;
 }
