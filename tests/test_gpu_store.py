@@ -23,6 +23,31 @@ def test_pull_bit_exact(L, n):
     assert np.array_equal(got, o.pull(keys))
 
 
+@pytest.mark.parametrize("L", [8, 64, 128, 256, 300])
+@pytest.mark.parametrize("n", [1, 33, 4097])
+def test_pull_with_replicated_keys_and_unmerged_updates_is_bit_exact(L, n):
+    # rows of 64, 128 and 256 floats take the 256-bit copy kernel once keys are replicated; a replicated key reads as
+    # stored row + the pulling worker's own unmerged updates
+    nk, R = 977, 3
+    rng = np.random.default_rng(L + n)
+    o, s = make_pair(nk, L, R=R, init=rand_table(nk, L))
+    hot = rng.choice(nk, 60, replace=False).astype(np.uint32)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    pk = np.where(rng.random(500) < 0.5, rng.choice(hot, 500), rng.integers(0, nk, 500)).astype(np.uint32)
+    d = rng.normal(size=(500, L)).astype(np.float32)
+    o.push(pk, d)
+    s.push(dev_keys(pk), dev_f32(d))
+    keys = np.where(rng.random(n) < 0.5, rng.choice(hot, n), rng.integers(0, nk, n)).astype(np.uint32)
+    got = s.pull(dev_keys(keys)).cpu().numpy()
+    assert np.array_equal(got, o.pull(keys))
+    # an output buffer that starts 16 bytes into an allocation (not 32-byte aligned) takes the 128-bit kernel
+    buf = torch.empty(n * L + 4, device="cuda")
+    out = buf[4:].view(n, L)
+    s.pull(dev_keys(keys), out)
+    assert np.array_equal(out.cpu().numpy(), o.pull(keys))
+
+
 def test_init_uniform_bit_exact():
     o, s = make_pair(1003, 12, with_adagrad=True)
     for which, seed, scale in ((0, 5, 0.25), (1, 6, 1e-3)):
