@@ -255,7 +255,10 @@ nups_status nups_step_sgns(nups_store* store, const uint32_t* d_center, const ui
  * (and without access counting or ownership tracking) the steps between two
  * merges share one kernel launch, so pairs of different steps of that stretch
  * race like pairs of one step do; otherwise the steps run one after the other.
- * n_total must be a multiple of batch.                                        */
+ * A merge that falls due before the call's last step runs on a stream that the
+ * library owns, beside the drawing of the next steps' negatives; the next step
+ * kernel waits for it, and when the call returns all of its work is ordered on
+ * `stream` as usual.  n_total must be a multiple of batch.                     */
 nups_status nups_run_sgns(nups_store* store, const uint32_t* d_center, const uint32_t* d_context, uint64_t n_total,
                           uint64_t batch, int32_t dist, uint32_t K, float lr, float* d_loss_out, void* stream);
 
