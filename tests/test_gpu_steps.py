@@ -327,3 +327,33 @@ def test_mf_clipping_matches_the_oracle_and_fast_mode_counts_the_same_updates():
         assert cs == co
         assert ss == pytest.approx(so, rel=1e-5 if det else 0.25)
         s.close()
+
+
+def test_fast_mode_with_clipping_tracks_the_clipped_oracle():
+    # replicated + asynchronous mode with clipping on, steps taken 16 at a time (the bound is then fixed per launch):
+    # the loss stays within 2 % of the oracle's clipped run and exactly the same updates are counted
+    from paper_2104_00501_b200 import binding
+    V, L, K, R, batch = 500, 32, 3, 8, 256
+    c, ctx, w = sgns_data(V, 4000, 2)
+    init = inputs.normal_init(2 * V, L, 0.1, 2)
+    o, s0 = make_pair(2 * V, L, R=R, init=init, deterministic=False, sync_interval=4)
+    s0.close()
+    s = binding.Store(2 * V, L, workers=R, sync_interval=4, deterministic=False, clip_factor=1.5)
+    s.write_table(0, init)
+    o.set_clipping(1.5)
+    o.count_accesses(np.concatenate([c, ctx]))
+    hot = o.select_hot(True, 20)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(V, w, V, BOUNDED, U=4, G=50, seed=3)
+    ds = s.register_distribution(V, dev_keys(w), V, BOUNDED, U=4, G=50, seed=3)
+    nb = len(c) // batch
+    lo = [o.step_sgns(c[b * batch:(b + 1) * batch], ctx[b * batch:(b + 1) * batch], do, K, 0.02) for b in range(nb)]
+    ls = torch.zeros(nb, device="cuda")
+    s.run_sgns(dev_keys(c[:nb * batch]), dev_keys(ctx[:nb * batch]), batch, ds, K, 0.02, ls)
+    ls = ls.cpu().numpy()
+    assert abs(ls[-20:].mean() - np.mean(lo[-20:])) <= 0.02 * np.mean(lo[-20:])
+    (so, co), (ss, cs) = o.clip_stats(), s.clip_stats()
+    assert cs == co and ss == pytest.approx(so, rel=0.1)
+    assert s.status_check() == 0
+    s.close()
