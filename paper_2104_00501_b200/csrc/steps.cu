@@ -1,9 +1,12 @@
 // Workload steps driving the store: skip-gram with negative sampling, ComplEx with AdaGrad and
-// matrix factorization (NuPS Section 5.1).  SGNS and ComplEx: one block per item, rows staged in shared
-// memory by asynchronous copies, one thread per chunk of a row; MF: one warp per item with a ring of
-// items in flight.  Updates are pushed either straight to the store (fast mode, vector reductions) or
+// matrix factorization (NuPS Section 5.1).  SGNS: one warp per pair, ComplEx: one block per triple, rows
+// staged in shared memory by asynchronous copies, one thread per chunk of a row; MF: one warp per cell
+// with a ring of cells in flight.  Updates are pushed either straight to the store (fast mode, vector reductions) or
 // into a row buffer that the ordered push applies afterwards (deterministic mode, all pulls see the
 // values from before the step).
+#include <mutex>
+#include <vector>
+
 #include "nups_internal.cuh"
 
 static inline size_t align256(size_t x) { return (x + 255) / 256 * 256; }
@@ -801,6 +804,21 @@ static unsigned step_grid(const nups_store* s, uint64_t n, unsigned blocks_per_s
         }                                                                                    \
     } while (0)
 
+// resident blocks per multiprocessor of a kernel variant at a shared-memory size, asked of the runtime once and kept
+template <class Query>
+static cudaError_t resident_blocks(const void* fn, size_t smem, int* out, Query query)
+{
+    struct Entry { const void* fn; size_t smem; int fit; };
+    static std::mutex mu;
+    static std::vector<Entry> seen;
+    std::lock_guard<std::mutex> g(mu);
+    for (const Entry& e : seen)
+        if (e.fn == fn && e.smem == smem) { *out = e.fit; return cudaSuccess; }
+    cudaError_t rc = query(out);
+    if (rc == cudaSuccess) seen.push_back({fn, smem, *out});
+    return rc;
+}
+
 // launch of the fused skip-gram kernel over `group` consecutive steps of n pairs (group > 1: fast mode only;
 // the negatives of all those steps lie back to back at s->last_negs, per-step losses go to loss_acc)
 static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const uint32_t* d_context, uint64_t n, uint32_t K,
@@ -824,7 +842,8 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
         if (smem > 48 * 1024)                                                                                          \
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);           \
         int fit = 0;       /* registers may allow fewer resident blocks than shared memory does: no second wave */ \
-        if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&fit, kern, 32 * SGNS_WARPS, smem);    \
+        if (e == cudaSuccess) e = resident_blocks((const void*)kern, smem, &fit, [&](int* out) {                       \
+            return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, kern, 32 * SGNS_WARPS, smem); });                \
         if (e == cudaSuccess) {                                                                                        \
             if (fit >= 1 && (unsigned)fit < per_sm) per_sm = (unsigned)fit;                                            \
             const uint64_t cap = (uint64_t)s->sm_count * per_sm;                                                       \
