@@ -453,6 +453,22 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             }
             asm volatile("cp.async.commit_group;\n cp.async.wait_group 0;" ::: "memory");
         }
+        // while this triple is worked on, the rows of the block's next triple start moving towards L2
+        {
+            const uint64_t nx = i + gridDim.x;
+            if (nx < n) {
+                const uint32_t lines_per_row = (uint32_t)((L * 4 + 127) / 128);
+                for (uint32_t e = tid; e < per * lines_per_row; e += CPX_THREADS) {
+                    const uint32_t role = e / lines_per_row, line = e % lines_per_row;
+                    const uint32_t k = role == 0 ? hk[nx] : role == 1 ? rk[nx] : role == 2 ? tk[nx] : negs[nx * K + role - 3];
+                    const size_t off = (size_t)k * L + (size_t)line * 32;
+                    if (k < v.num_keys && off + 32 <= (size_t)v.num_keys * L) {       // a whole line inside the table
+                        prefetch_l2(v.val + off);
+                        prefetch_l2(v.acc + off);
+                    }
+                }
+            }
+        }
         C2 h = c2_zero(), r = c2_zero(), t = c2_zero();
         if (mine) {
             h = c2_parked(park, 0, tid, v.dval, s_pend[0], d2);
