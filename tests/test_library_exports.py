@@ -42,3 +42,30 @@ def test_strerror_and_argument_checks_need_no_device():
     assert lib.nups_create(0, 4, None, ctypes.byref(h)) == binding.EINVAL
     assert lib.nups_create(10, 3, None, ctypes.byref(h)) == binding.EINVAL      # rows must be 16-byte multiples
     assert lib.nups_create(1 << 33, 4, None, ctypes.byref(h)) == binding.EINVAL
+
+
+def test_binding_config_mirrors_the_header_struct():
+    # field for field, in order and width: a drifted mirror would silently hand the library other settings
+    text = open(os.path.join(ROOT, "include", "nups.h")).read()
+    body = re.search(r"typedef struct nups_config \{(.*?)\} nups_config;", text, flags=re.S).group(1)
+    body = re.sub(r"/\*.*?\*/", "", body, flags=re.S)
+    header = []
+    for ctype, name, dim in re.findall(r"\b(uint32_t|float)\s+([a-z_0-9]+)(?:\[(\d+)\])?;", body):
+        header.append((name, ctype, int(dim) if dim else 1))
+    mirror = []
+    for name, ct in binding.Config._fields_:
+        if hasattr(ct, "_length_"):
+            mirror.append((name, "uint32_t" if ct._type_ is ctypes.c_uint32 else "float", ct._length_))
+        else:
+            mirror.append((name, "uint32_t" if ct is ctypes.c_uint32 else "float", 1))
+    assert mirror == header
+    assert ctypes.sizeof(binding.Config) == 64
+    # creation rejects settings that cannot go together, before it looks for a device
+    lib = binding.load()
+    h = ctypes.c_void_p()
+    cfg = binding.Config(deterministic=1, sync_period_us=100)
+    assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL
+    cfg = binding.Config(clip_factor=-1.0)
+    assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL
+    cfg = binding.Config(workers=255)
+    assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL
