@@ -103,3 +103,50 @@ def test_full_size_pull_sample_keys_match_the_oracle(level_name):
     assert np.array_equal(got, np.array([o.owner_of(int(k)) for k in probe]))
     assert s.status_check() == 0
     s.close()
+
+
+def test_full_size_ps_pull_is_an_exact_copy_and_push_conserves_every_update():
+    # the PS sweep's store: 100M keys x 128 floats (51 GB), 1M-key batches ~ Zipf(1.0), top-1000 keys replicated over
+    # 8 workers, fast (atomic) mode.  Properties that hold at any size, checked on every key of a batch with torch's
+    # own index routines as the textbook definition: a pull returns the stored rows bit for bit, and after the merge
+    # every row is the sum of everything pushed to it (updates are multiples of 2^-6, so their sums are exact in fp32
+    # whatever the order of the additions).
+    NK, L, N = 100_000_000, 128, 1 << 20
+    dev = torch.device("cuda")
+    s = binding.Store(NK, L, workers=bench.WORKERS, deterministic=False)
+    hot = inputs.zipf_key_of_rank(NK, dev)[:1000]
+    s.set_management(hot.to(torch.int32).contiguous(), binding.REPLICATE)
+    cdf = inputs.zipf_cdf(NK, 1.0, dev)
+    g = torch.Generator(device=dev)
+    g.manual_seed(5)
+    total = None
+    for b in range(3):
+        keys = inputs.zipf_keys(N, NK, 1.0, 200 + b, dev, cdf=cdf)
+        delta = torch.randint(-8, 9, (N, L), generator=g, device=dev, dtype=torch.int32).to(torch.float32) / 64.0
+        s.push(keys.to(torch.int32).contiguous(), delta)
+        u, inv = torch.unique(keys, return_inverse=True)
+        part = torch.zeros(u.numel(), L, device=dev).index_add_(0, inv, delta)
+        if total is None:
+            total_keys, total = u, part
+        else:
+            allk = torch.cat([total_keys, u])
+            uu, ii = torch.unique(allk, return_inverse=True)
+            total = torch.zeros(uu.numel(), L, device=dev).index_add_(0, ii, torch.cat([total, part]))
+            total_keys = uu
+        del delta, part
+    s.sync()
+    got = s.pull(total_keys.to(torch.int32).contiguous())
+    assert torch.equal(got, total)
+    del got, total
+    untouched = torch.randint(0, NK, (100_000,), generator=g, device=dev)
+    untouched = untouched[~torch.isin(untouched, total_keys)]
+    assert not s.pull(untouched.to(torch.int32).contiguous()).any()
+    # pull against the table itself, after start values that are not round numbers
+    s.init_uniform(0, 3, 0.1)
+    table = s.read_table()
+    keys = inputs.zipf_keys(N, NK, 1.0, 300, dev, cdf=cdf)
+    assert torch.equal(s.pull(keys.to(torch.int32).contiguous()), table[keys])
+    assert s.status_check() == 0
+    s.close()
+    del table
+    torch.cuda.empty_cache()                 # hand the 51 GB copy back before the next test allocates
