@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import bench
-from oracle import Oracle, BOUNDED, REPLICATE
+from oracle import Oracle, BOUNDED, CONFORM, REPLICATE
 from paper_2104_00501_b200 import binding, inputs
 from tests.common import host_keys
 
@@ -150,3 +150,76 @@ def test_full_size_ps_pull_is_an_exact_copy_and_push_conserves_every_update():
     s.close()
     del table
     torch.cuda.empty_cache()                 # hand the 51 GB copy back before the next test allocates
+
+
+def test_benchmark_sized_complex_batches_match_the_oracle():
+    # the knowledge-graph workload's launch configuration (batches of 8192 triples, 10 negatives, rows of 500 floats
+    # plus accumulator, relations and frequent entities replicated) on a key space the oracle holds in memory: every
+    # block works on many triples one after the other, as in the benchmark
+    E, Rl, L, B, K, R = 200_000, 1000, 500, 8192, 10, bench.WORKERS
+    # (one batch: AdaGrad's first step of a component is lr long whatever the gradient's size, so a second batch would
+    # start from values that differ wherever a first gradient was within rounding of zero)
+    h, r, t = [inputs.u32(x) for x in inputs.kge_triples(B, E, Rl, 0.9, 1.2, 0)]
+    o = Oracle(E + Rl, L, workers=R, with_adagrad=True, sync_interval=1)
+    s = binding.Store(E + Rl, L, workers=R, sync_interval=1, deterministic=True, with_adagrad=True)
+    o.init_uniform(0, 5, 0.05)
+    s.init_uniform(0, 5, 0.05)
+    o.count_accesses(np.concatenate([h, t]))
+    hot = np.concatenate([np.arange(E, E + Rl, dtype=np.uint32), o.select_hot(False, 100)])
+    o.set_management(hot, REPLICATE)
+    s.set_management(torch.from_numpy(hot.view(np.int32)).cuda(), binding.REPLICATE)
+    do = o.register_distribution(0, None, E, CONFORM, seed=3)
+    ds = s.register_distribution(0, None, E, binding.CONFORM, seed=3)
+    lb = torch.zeros(1, device="cuda")
+    dk = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).cuda()
+    touched = []
+    for b in range(1):
+        sl = slice(b * B, (b + 1) * B)
+        lo, negs = o.step_complex(h[sl], r[sl], t[sl], do, K, 0.1, 1e-10, return_negatives=True)
+        s.step_complex(dk(h[sl]), dk(r[sl]), dk(t[sl]), ds, K, 0.1, 1e-10, lb)
+        assert np.array_equal(host_keys(s.last_negatives()), negs)
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+        touched.append(np.concatenate([h[sl], r[sl], t[sl], negs]))
+    rows = np.unique(np.concatenate(touched))
+    idx = torch.from_numpy(rows.astype(np.int64)).cuda()
+    acc = s.read_table(1)[idx].cpu().numpy()
+    np.testing.assert_allclose(acc, o.table(1)[rows], rtol=1e-4, atol=1e-9)
+    # the first AdaGrad step of a component moves it by lr whatever the gradient's size: compare values where
+    # the oracle's squared gradients are not vanishing
+    big = o.table(1)[rows] > 1e-8
+    val, ref = s.read_table(0)[idx].cpu().numpy()[big], o.table(0)[rows][big]
+    # ... and a key pushed to by many triples of the batch takes one such step per triple: a handful of components
+    # whose gradient in one of them is within rounding of zero (while others make the sum large) may differ by a
+    # small part of lr; anything else is within tolerance
+    off = ~np.isclose(val, ref, rtol=1e-4, atol=1e-5)
+    assert off.mean() < 1e-5 and (not off.any() or np.abs(val - ref)[off].max() < 0.02)
+    assert big.mean() > 0.05 and s.status_check() == 0
+    s.close()
+
+
+def test_benchmark_sized_mf_batches_match_the_oracle():
+    # the matrix-factorization workload's launch configuration (batches of 65,536 cells, rank 100, frequent rows and
+    # columns replicated): every warp works through many cells, its ring of prefetched rows refilled all the way
+    M, N, L, B, R = 1_000_000, 100_000, 100, 65_536, bench.WORKERS
+    i, j, x = inputs.mf_cells(2 * B, M, N, 0.8, 100, 0.1, 0)
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    o = Oracle(M + N, L, workers=R, sync_interval=2)
+    s = binding.Store(M + N, L, workers=R, sync_interval=2, deterministic=True)
+    o.init_uniform(0, 5, 0.3)
+    s.init_uniform(0, 5, 0.3)
+    o.count_accesses(np.concatenate([i, j]))
+    hot = o.select_hot(False, 100)
+    o.set_management(hot, REPLICATE)
+    s.set_management(torch.from_numpy(hot.view(np.int32)).cuda(), binding.REPLICATE)
+    lb = torch.zeros(1, device="cuda")
+    dk = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).cuda()
+    for b in range(2):
+        sl = slice(b * B, (b + 1) * B)
+        lo = o.step_mf(i[sl], j[sl], x[sl], 0.01, 0.01)
+        s.step_mf(dk(i[sl]), dk(j[sl]), torch.from_numpy(x[sl].copy()).cuda(), 0.01, 0.01, lb)
+        assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    rows = np.unique(np.concatenate([i, j]))
+    got = s.read_table(0)[torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy()
+    np.testing.assert_allclose(got, o.table(0)[rows], rtol=1e-5, atol=1e-6)
+    assert len(hot) > 0 and s.status_check() == 0
+    s.close()
