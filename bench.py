@@ -326,6 +326,7 @@ def run_ours(args, rank, world, device):
                      "kernel_share_of_step": (k_ms / args.steps) / (ms / args.steps),
                      "distinct_cold_rows_per_batch": float(np.mean(cold_rows)),
                      "update_payload_gbs": update_bytes / k_s / 1e9,
+                     "frac_of_l2_reduction_ceiling": update_bytes / k_s / 1e9 / red_l2,
                      "reduction_rate_l2_resident_gbs": red_l2, "reduction_rate_dram_gbs": red_dram},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
