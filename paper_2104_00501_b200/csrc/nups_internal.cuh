@@ -283,6 +283,18 @@ __device__ __forceinline__ void mark_localize(const View& v, uint32_t key, uint3
     atomicMax(v.own + key, want);
 }
 
+// The same for the keys of independent draws, which rarely repeat: reading the word first would add one more
+// scattered memory access per sample (these kernels are bound by the rate of such accesses).  `repeats` = the key
+// shows up more than once among the warp's samples, the sign of a very frequent key: those still look first, so that
+// a frequent key that is not replicated does not queue thousands of atomics at one address.
+__device__ __forceinline__ void mark_localize_rare(const View& v, uint32_t key, uint32_t q, bool repeats)
+{
+    if (key_is_hot(v, key)) return;
+    const uint32_t want = v.epoch_tag | q;
+    if (repeats && __ldcg(v.own + key) >= want) return;
+    atomicMax(v.own + key, want);
+}
+
 __device__ __forceinline__ void flag_bad_key(const View& v) { atomicCAS(&v.st->status, 0, NUPS_EKEY); }
 
 __device__ __forceinline__ void red_add_v4(float* addr, float4 x)

@@ -337,7 +337,8 @@ __global__ void draw_iid_kernel(View v, DrawParams p, const unsigned long long* 
     const uint32_t q = chunk_of_pos(o, N, R);
     const uint32_t k = draw_iid(p, q, off_cur[q] + (o - chunk_begin(q, N, R)));
     h.keys[o] = k;
-    if (localize) mark_localize(v, k, q);          // PrepareSample localizes what it sampled
+    if (localize)                                  // PrepareSample localizes what it sampled
+        mark_localize_rare(v, k, q, __popc(__match_any_sync(__activemask(), k)) > 1);
 }
 
 // Pooled reuse: pool `pl` of a worker holds G iid draws and is walked U times, each pass in a fresh
@@ -807,9 +808,10 @@ __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long
         k = draw_iid(p, q, off_cur[q] + (unsigned long long)bt * size + (o - chunk_begin(q, N, v.R)));
     }
     if (local_only) k = first_local_warp(v, p, q, k, in);
+    const bool repeats = localize && __popc(__match_any_sync(0xFFFFFFFFu, in ? k : 0xFFFFFFFFu - (threadIdx.x & 31))) > 1;
     if (in) {
         out[o] = k;
-        if (localize) mark_localize(v, k, q);
+        if (localize) mark_localize_rare(v, k, q, repeats);
     }
     count_sample(v, k, in);
     if (blockIdx.x == 0 && blockIdx.y == 0)
