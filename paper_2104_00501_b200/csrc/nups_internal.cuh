@@ -316,6 +316,35 @@ __device__ __forceinline__ void st_stream_v4(float4* p, float4 x)
                  : "memory");
 }
 
+// 256-bit global loads and stores (sm_100): 32-byte aligned addresses
+struct F8 { float4 a, b; };
+__device__ __forceinline__ F8 ld8_cached(const float* p)
+{
+    F8 r;
+    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.a.x), "=f"(r.a.y), "=f"(r.a.z), "=f"(r.a.w), "=f"(r.b.x), "=f"(r.b.y), "=f"(r.b.z), "=f"(r.b.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ F8 ld8_stream(const float* p)
+{
+    F8 r;
+    asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.a.x), "=f"(r.a.y), "=f"(r.a.z), "=f"(r.a.w), "=f"(r.b.x), "=f"(r.b.y), "=f"(r.b.z), "=f"(r.b.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ F8 ld8_plain(const float* p)
+{
+    F8 r;
+    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=f"(r.a.x), "=f"(r.a.y), "=f"(r.a.z), "=f"(r.a.w), "=f"(r.b.x), "=f"(r.b.y), "=f"(r.b.z), "=f"(r.b.w) : "l"(p));
+    return r;
+}
+__device__ __forceinline__ void st8_stream(float* p, const F8& r)
+{
+    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(r.a.x), "f"(r.a.y), "f"(r.a.z),
+                 "f"(r.a.w), "f"(r.b.x), "f"(r.b.y), "f"(r.b.z), "f"(r.b.w) : "memory");
+}
+
 __device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
 
 __device__ __forceinline__ float warp_sum(float x)

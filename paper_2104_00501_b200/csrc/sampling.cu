@@ -691,8 +691,13 @@ lt_scan_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, ui
     }
 }
 
-__global__ void lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
-                                uint32_t* __restrict__ out)
+// C8 > 0: the kernel also copies the rows of the keys it emits (rows of C8 chunks of 32 bytes, 32 / C8 rows per warp
+// instruction, as gather8_kernel does), which saves the separate gather launch of a full PullSample with values.
+template <int C8>
+__global__ void __launch_bounds__(256)
+lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
+                uint32_t* __restrict__ out, const float* __restrict__ table, const float* slab,
+                float* __restrict__ out_vals)
 {
     const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
     if (!c.active) return;
@@ -708,10 +713,12 @@ __global__ void lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t curso
     const bool loc = (bits >> lane) & 1u;
     uint32_t key = 0;
     bool emitted = false;
+    uint32_t opos = 0;                                               // where the emitted key went
     if (walked) {
         key = h.keys[c.b0 + i];
         if (loc) {
-            out[c.out_base + before] = key;
+            opos = (uint32_t)(c.out_base + before);
+            out[opos] = key;
             emitted = true;
         } else {
             // postponed: queued behind the non-local entries before it, emitted by this very call if the queue's
@@ -720,13 +727,47 @@ __global__ void lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t curso
             const uint64_t at = pt + ((i - oc) - before);
             h.post[c.b0 + at] = key;
             if (at >= ph && at < ph + cnt) {
-                out[c.out_base + tl + (at - ph)] = key;
+                opos = (uint32_t)(c.out_base + tl + (at - ph));
+                out[opos] = key;
                 emitted = true;
             }
             mark_localize(v, key, c.q);
         }
     }
     count_sample(v, key, emitted);
+    if (C8 > 0) {
+        constexpr int RPI = C8 > 0 ? 32 / C8 : 1, UNR = 2;
+        const unsigned sub = lane / (C8 > 0 ? C8 : 1), ch = lane % (C8 > 0 ? C8 : 1);
+        const uint64_t L = (uint64_t)v.L4 * 4;
+        const uint32_t src = emitted ? key : 0xFFFFFFFFu;
+        uint32_t pend = 0xFFFFFFFFu;                                 // replica row of a replicated key
+        if (emitted && key_is_hot(v, key)) pend = c.q * (uint32_t)v.Hcap + (uint32_t)__ldg(v.slot_of + key);
+        for (int r0 = 0; r0 < 32; r0 += UNR * RPI) {
+            uint32_t so[UNR], po[UNR], oo[UNR];
+            F8 a[UNR];
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                const int row = r0 + u * RPI + (int)sub;
+                so[u] = __shfl_sync(0xFFFFFFFFu, src, row);
+                po[u] = __shfl_sync(0xFFFFFFFFu, pend, row);
+                oo[u] = __shfl_sync(0xFFFFFFFFu, opos, row);
+            }
+#pragma unroll
+            for (int u = 0; u < UNR; ++u) {
+                if (so[u] == 0xFFFFFFFFu) continue;
+                const float* p = table + (uint64_t)so[u] * L + 8 * ch;
+                a[u] = po[u] == 0xFFFFFFFFu ? ld8_stream(p) : ld8_cached(p);
+                if (po[u] != 0xFFFFFFFFu) {
+                    const F8 d = ld8_plain(slab + (uint64_t)po[u] * L + 8 * ch);
+                    a[u].a = add4(a[u].a, d.a);
+                    a[u].b = add4(a[u].b, d.b);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < UNR; ++u)
+                if (so[u] != 0xFFFFFFFFu) st8_stream(out_vals + (uint64_t)oo[u] * L + 8 * ch, a[u]);
+        }
+    }
 }
 
 static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_keys_out, float* d_vals_out,
@@ -757,8 +798,21 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         LAUNCH_CHECK(s);
         lt_scan_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
         LAUNCH_CHECK(s);
-        lt_place_kernel<<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
+        // a full pull of a fresh handle has no entries postponed by earlier calls to emit: the placement pass can copy
+        // the rows itself (one table of 64, 128 or 256 floats per row, 32-byte aligned output)
+        const uint32_t c8 = s->L / 8;
+        const bool fused = d_vals_out && h.cursor == 0 && n == h.N && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) &&
+                           ((uintptr_t)d_vals_out & 31) == 0 && (uint64_t)s->R * s->Hcap < 0xFFFFFFFFull;
+        if (fused && c8 == 8) lt_place_kernel<8><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
+        else if (fused && c8 == 16) lt_place_kernel<16><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
+        else if (fused) lt_place_kernel<32><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
+        else lt_place_kernel<0><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, nullptr, nullptr, nullptr);
         LAUNCH_CHECK(s);
+        if (fused) {
+            h.cursor += n;
+            h.used = 0;
+            return NUPS_OK;
+        }
     } else if (d_vals_out && d.level != NUPS_NONCONFORM && !s->cfg.count_accesses) {
         // keys fixed at PrepareSample and nothing to count: the row gather reads them from the handle and hands them out
         // on its way, which saves a launch

@@ -379,34 +379,6 @@ gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A
 // 32 / C8 whole rows, which halves the load/store instructions per byte.  Used when some keys are replicated: once
 // many rows come from L2 (hot or repeated keys) the copy is bound by the instructions its rows take in the
 // load/store pipe, not by DRAM.
-struct F8 { float4 a, b; };
-__device__ __forceinline__ F8 ld8_cached(const float* p)
-{
-    F8 r;
-    asm volatile("ld.global.nc.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(r.a.x), "=f"(r.a.y), "=f"(r.a.z), "=f"(r.a.w), "=f"(r.b.x), "=f"(r.b.y), "=f"(r.b.z), "=f"(r.b.w) : "l"(p));
-    return r;
-}
-__device__ __forceinline__ F8 ld8_stream(const float* p)
-{
-    F8 r;
-    asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(r.a.x), "=f"(r.a.y), "=f"(r.a.z), "=f"(r.a.w), "=f"(r.b.x), "=f"(r.b.y), "=f"(r.b.z), "=f"(r.b.w) : "l"(p));
-    return r;
-}
-__device__ __forceinline__ F8 ld8_plain(const float* p)
-{
-    F8 r;
-    asm volatile("ld.global.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-                 : "=f"(r.a.x), "=f"(r.a.y), "=f"(r.a.z), "=f"(r.a.w), "=f"(r.b.x), "=f"(r.b.y), "=f"(r.b.z), "=f"(r.b.w) : "l"(p));
-    return r;
-}
-__device__ __forceinline__ void st8_stream(float* p, const F8& r)
-{
-    asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "f"(r.a.x), "f"(r.a.y), "f"(r.a.z),
-                 "f"(r.a.w), "f"(r.b.x), "f"(r.b.y), "f"(r.b.z), "f"(r.b.w) : "memory");
-}
-
 template <bool HOT, int C8>
 __global__ void __launch_bounds__(256, 4)
 gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const float* __restrict__ table,

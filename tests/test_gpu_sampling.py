@@ -140,3 +140,36 @@ def test_large_handles_with_most_keys_taken_by_other_workers(level):
     allk = np.arange(nk, dtype=np.uint32)
     assert np.array_equal(s.owner_of(dev_keys(allk)).cpu().numpy(), np.array([o.owner_of(k) for k in allk]))
     assert s.status_check() == 0
+
+
+@pytest.mark.parametrize("L", [64, 128, 256])
+def test_full_pull_with_values_under_postponing_copies_the_rows_itself(L):
+    # rows of 64 / 128 / 256 floats: a full PullSample of a fresh LONG-TERM handle places keys and copies rows in one
+    # pass; replicated keys carry unmerged updates, ownership has been stirred, and a second handle is pulled in parts
+    # (the separate gather) for comparison with the same oracle
+    nk, R, N = 5000, 4, 20_000
+    rng = np.random.default_rng(L)
+    init = rng.normal(size=(nk, L)).astype(np.float32)
+    w = inputs.zipf_integer_weights(4000, 0.9).numpy().astype(np.uint32)
+    o, s = make_pair(nk, L, R=R, init=init, track_ownership=True)
+    hot = rng.choice(nk, 40, replace=False).astype(np.uint32)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    pk = np.where(rng.random(300) < 0.6, rng.choice(hot, 300), rng.integers(0, nk, 300)).astype(np.uint32)
+    d = rng.normal(size=(300, L)).astype(np.float32)
+    o.push(pk, d)
+    s.push(dev_keys(pk), torch.from_numpy(d).cuda())
+    do = o.register_distribution(500, w, 4000, LONGTERM, U=4, G=50, seed=5)
+    ds = s.register_distribution(500, dev_keys(w), 4000, LONGTERM, U=4, G=50, seed=5)
+    for cuts in ([N], [7000, 13000], [N]):
+        moved = rng.integers(0, nk, 3000).astype(np.uint32)
+        o.localize(moved)
+        s.localize(dev_keys(moved))
+        ho, hs = o.prepare_sample(do, N), s.prepare_sample(ds, N)
+        for c in cuts:
+            ko, vo = o.pull_sample(ho, c)
+            ks, vs = s.pull_sample(hs, c)
+            assert np.array_equal(host_keys(ks), ko)
+            assert np.array_equal(vs.cpu().numpy(), vo)
+    allk = np.arange(nk, dtype=np.uint32)
+    assert np.array_equal(s.owner_of(dev_keys(allk)).cpu().numpy(), np.array([o.owner_of(k) for k in allk]))
