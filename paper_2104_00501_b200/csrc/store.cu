@@ -541,7 +541,12 @@ struct PushPair {
 // updates to those slots are added in shared memory and reach the worker's replica once, when the
 // block ends.  This is what keeps thousands of additions to one hot row from queueing at one L2
 // address.
-template <bool HOT, bool TWO, bool TIER>
+// TIER = 2: nothing is replicated, so there are no slots to key the accumulators on; the block then uses them as a
+// direct-mapped cache of rows: accumulator (key mod tier_rows) is claimed by the first key that asks for it and
+// takes that key's updates until the block ends (other keys that map there go straight to their rows).  Frequent
+// keys show up early and often, so they take most accumulators, and a skewed batch stops queueing at a few L2
+// addresses even when its frequent keys were never marked for replication.
+template <bool HOT, bool TWO, int TIER>
 __global__ void __launch_bounds__(256, 3)
 push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPair A, PushPair B, uint64_t n_items,
                    uint32_t rows_per_item, uint32_t tier_rows)
@@ -551,10 +556,13 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
     const uint32_t L4 = v.L4;
     const uint32_t R = v.R;
     unsigned* touched = reinterpret_cast<unsigned*>(tier_mem + (size_t)tier_rows * L4 * 4);
+    unsigned* tags = touched + (tier_rows + 31) / 32;                  // TIER == 2: key that owns each accumulator
     if (TIER) {
         float4* z = reinterpret_cast<float4*>(tier_mem);
         for (uint32_t e = threadIdx.x; e < tier_rows * L4; e += blockDim.x) z[e] = make_float4(0.f, 0.f, 0.f, 0.f);
         for (uint32_t e = threadIdx.x; e < (tier_rows + 31) / 32; e += blockDim.x) touched[e] = 0u;
+        if (TIER == 2)
+            for (uint32_t e = threadIdx.x; e < tier_rows; e += blockDim.x) tags[e] = NUPS_INVALID_KEY;
         __syncthreads();
     }
     // Windows are visited in an order that interleaves the workers' chunks: the window range is cut
@@ -563,14 +571,14 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
     // hot key; with the tier, a block walks the stretch of its own worker only.
     const uint64_t W = (n + 31) / 32;
     const uint64_t per = (W + R - 1) / R;
-    const uint32_t my_q = TIER ? blockIdx.x % R : 0u;
-    const uint64_t warp = TIER ? ((uint64_t)(blockIdx.x / R) * blockDim.x + threadIdx.x) >> 5
+    const uint32_t my_q = TIER == 1 ? blockIdx.x % R : 0u;
+    const uint64_t warp = TIER == 1 ? ((uint64_t)(blockIdx.x / R) * blockDim.x + threadIdx.x) >> 5
                                : ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint64_t nwarps = TIER ? ((uint64_t)(gridDim.x / R) * blockDim.x) >> 5 : ((uint64_t)gridDim.x * blockDim.x) >> 5;
-    const uint64_t slots = TIER ? per : per * R;
+    const uint64_t nwarps = TIER == 1 ? ((uint64_t)(gridDim.x / R) * blockDim.x) >> 5 : ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint64_t slots = TIER == 1 ? per : per * R;
     auto window_of = [&](uint64_t u) -> uint64_t {
         if (u >= slots) return W;
-        const uint64_t w = TIER ? (uint64_t)my_q * per + u : (u % R) * per + u / R;
+        const uint64_t w = TIER == 1 ? (uint64_t)my_q * per + u : (u % R) * per + u / R;
         return (w < W) ? w : W;
     };
     auto load_key = [&](uint64_t w) -> uint32_t {
@@ -608,7 +616,16 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
                                                       : worker_of_item(i / rows_per_item, n_items, R);
                 dest = ((((unsigned long long)q * v.Hcap + slot) * L4) << 3) | 1ull;
                 hrow = (size_t)q * v.Hcap + slot;
-                if (TIER && slot < tier_rows && q == my_q) tier = (int)slot;
+                if (TIER == 1 && slot < tier_rows && q == my_q) tier = (int)slot;
+            }
+            if (TIER == 2) {
+                const uint32_t at = key % tier_rows;
+                uint32_t owner = tags[at];
+                if (owner == NUPS_INVALID_KEY) {
+                    owner = atomicCAS(&tags[at], NUPS_INVALID_KEY, key);
+                    if (owner == NUPS_INVALID_KEY) owner = key;
+                }
+                if (owner == key) tier = (int)at;
             }
         }
         if (v.count) {
@@ -730,7 +747,7 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
         __syncthreads();
         for (uint32_t sl = threadIdx.x >> 5; sl < tier_rows; sl += blockDim.x >> 5) {
             if (!((touched[sl >> 5] >> (sl & 31)) & 1u)) continue;
-            float* dst = A.slab + ((size_t)my_q * v.Hcap + sl) * L4 * 4;
+            float* dst = TIER == 2 ? A.table + (size_t)tags[sl] * L4 * 4 : A.slab + ((size_t)my_q * v.Hcap + sl) * L4 * 4;
             const float* t = tier_mem + (size_t)sl * L4 * 4;
             for (uint32_t c = lane; c < L4; c += 32)
                 red_add_v4(dst + (size_t)c * 4, make_float4(t[c], t[c + L4], t[c + 2 * L4], t[c + 3 * L4]));
@@ -867,31 +884,39 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
         // shared-memory tier: single-table calls with replicated keys, enough blocks to give every worker some
         uint32_t tier_rows = 0;
         size_t tier_bytes = 0;
-        if (s->H && !two && rows_per_item == 1 && grid >= s->R && n >= 32768) {
+        const bool cache = !s->H && !two && n >= 32768;               // no replicated keys: accumulators as a row cache
+        if ((s->H && !two && rows_per_item == 1 && grid >= s->R && n >= 32768) || cache) {
             const size_t row_bytes = (size_t)s->L * 4;
             size_t budget = 64 * 1024;
-            tier_rows = s->cfg.smem_hot_rows ? s->cfg.smem_hot_rows : (uint32_t)(budget / row_bytes);
-            if (tier_rows > budget / row_bytes) tier_rows = (uint32_t)(budget / row_bytes);
-            if (tier_rows > s->H) tier_rows = (uint32_t)s->H;
-            tier_bytes = tier_rows * row_bytes + ((tier_rows + 31) / 32) * 4;
+            const size_t per_row = row_bytes + (cache ? 4 : 0) + 1;    // sums, owner tag, touched bit (rounded up)
+            tier_rows = s->cfg.smem_hot_rows ? s->cfg.smem_hot_rows : (uint32_t)(budget / per_row);
+            if (tier_rows > budget / per_row) tier_rows = (uint32_t)(budget / per_row);
+            if (cache && tier_rows > 1024) tier_rows = 1024;
+            if (!cache && tier_rows > s->H) tier_rows = (uint32_t)s->H;
+            tier_bytes = tier_rows * row_bytes + ((tier_rows + 31) / 32) * 4 + (cache ? tier_rows * 4 : 0);
             static bool attr_set = false;
             if (tier_rows && !attr_set) {
-                CK(cudaFuncSetAttribute(push_atomic_kernel<true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        (int)(budget + 1024)));
+                CK(cudaFuncSetAttribute(push_atomic_kernel<true, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(budget + 2048)));
+                CK(cudaFuncSetAttribute(push_atomic_kernel<false, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)(budget + 2048)));
                 attr_set = true;
             }
         }
         nups_time_begin(s, st);
-        if (tier_rows) {
+        if (tier_rows && cache) {
+            push_atomic_kernel<false, false, 2><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+                                                                             tier_rows);
+        } else if (tier_rows) {
             grid = grid / s->R * s->R;              // every worker gets the same number of blocks
-            push_atomic_kernel<true, false, true><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
-                                                                                tier_rows);
+            push_atomic_kernel<true, false, 1><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+                                                                             tier_rows);
         } else if (s->H) {
-            if (two) push_atomic_kernel<true, true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
-            else push_atomic_kernel<true, false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+            if (two) push_atomic_kernel<true, true, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+            else push_atomic_kernel<true, false, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
         } else {
-            if (two) push_atomic_kernel<false, true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
-            else push_atomic_kernel<false, false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+            if (two) push_atomic_kernel<false, true, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+            else push_atomic_kernel<false, false, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
         }
         nups_time_end(s, st);
         LAUNCH_CHECK(s);

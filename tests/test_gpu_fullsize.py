@@ -105,7 +105,8 @@ def test_full_size_pull_sample_keys_match_the_oracle(level_name):
     s.close()
 
 
-def test_full_size_ps_pull_is_an_exact_copy_and_push_conserves_every_update():
+@pytest.mark.parametrize("topk", [1000, 0])
+def test_full_size_ps_pull_is_an_exact_copy_and_push_conserves_every_update(topk):
     # the PS sweep's store: 100M keys x 128 floats (51 GB), 1M-key batches ~ Zipf(1.0), top-1000 keys replicated over
     # 8 workers, fast (atomic) mode.  Properties that hold at any size, checked on every key of a batch with torch's
     # own index routines as the textbook definition: a pull returns the stored rows bit for bit, and after the merge
@@ -114,8 +115,9 @@ def test_full_size_ps_pull_is_an_exact_copy_and_push_conserves_every_update():
     NK, L, N = 100_000_000, 128, 1 << 20
     dev = torch.device("cuda")
     s = binding.Store(NK, L, workers=bench.WORKERS, deterministic=False)
-    hot = inputs.zipf_key_of_rank(NK, dev)[:1000]
-    s.set_management(hot.to(torch.int32).contiguous(), binding.REPLICATE)
+    if topk:                                 # without replicated keys the fast push caches frequent rows per block
+        hot = inputs.zipf_key_of_rank(NK, dev)[:topk]
+        s.set_management(hot.to(torch.int32).contiguous(), binding.REPLICATE)
     cdf = inputs.zipf_cdf(NK, 1.0, dev)
     g = torch.Generator(device=dev)
     g.manual_seed(5)
