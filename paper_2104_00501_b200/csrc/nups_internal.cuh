@@ -115,6 +115,7 @@ struct nups_store {
     struct nups_background* bg; // time-based replica synchronisation (background.cu); NULL = never started
     cudaStream_t side;          // nups_run_sgns: a due replica merge runs here, beside the next steps' sample draw
     cudaEvent_t side_fork, side_join;
+    bool push_smem_opted, complex_smem_opted[2][2];   // large dynamic shared memory asked for on this store's device
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };

@@ -1013,16 +1013,15 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     if (per_sm < 1) per_sm = 1;
     uint64_t want = n < (uint64_t)s->sm_count * per_sm ? n : (uint64_t)s->sm_count * per_sm;
     unsigned grid = (unsigned)want;
-    static bool attr_set[2][2] = {{false, false}, {false, false}};
     const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0;
-    if (!attr_set[hi][di]) {
+    if (!s->complex_smem_opted[hi][di]) {
         cudaError_t e;
         if (hi && di) e = cudaFuncSetAttribute(complex_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
         else if (hi) e = cudaFuncSetAttribute(complex_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
         else if (di) e = cudaFuncSetAttribute(complex_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
         else e = cudaFuncSetAttribute(complex_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
         if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
-        attr_set[hi][di] = true;
+        s->complex_smem_opted[hi][di] = true;
     }
     nups_time_begin(s, st);
     DISPATCH_MODE(s, complex_kernel<HOT, DET><<<grid, CPX_THREADS, smem, st>>>(

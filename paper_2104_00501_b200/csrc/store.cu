@@ -894,13 +894,12 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
             if (cache && tier_rows > 1024) tier_rows = 1024;
             if (!cache && tier_rows > s->H) tier_rows = (uint32_t)s->H;
             tier_bytes = tier_rows * row_bytes + ((tier_rows + 31) / 32) * 4 + (cache ? tier_rows * 4 : 0);
-            static bool attr_set = false;
-            if (tier_rows && !attr_set) {
+            if (tier_rows && !s->push_smem_opted) {
                 CK(cudaFuncSetAttribute(push_atomic_kernel<true, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(budget + 2048)));
                 CK(cudaFuncSetAttribute(push_atomic_kernel<false, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(budget + 2048)));
-                attr_set = true;
+                s->push_smem_opted = true;
             }
         }
         nups_time_begin(s, st);
