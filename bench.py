@@ -622,18 +622,21 @@ def run_step_workload(args, device, which):
         nb = 32
         i, j, x = inputs.mf_cells(nb * B, M, N, 0.8, 100, 0.1, 0, device)
         i, j, x = i.to(torch.int32).contiguous(), j.to(torch.int32).contiguous(), x.contiguous()
-        s.count_accesses(torch.cat([i, j]))
+        s.count_accesses(torch.cat([i, j]))                         # the hot set comes from independent draws ...
         hot = s.select_hot(False, 100)
         if hot.numel():
             s.set_management(hot, binding.REPLICATE)
+        if args.mf_order != "random":                                # ... the steps may visit the cells column by column
+            i, j, x = inputs.mf_cells(nb * B, M, N, 0.8, 100, 0.1, 0, device, by_column_of=100 * M)
+            i, j, x = i.to(torch.int32).contiguous(), j.to(torch.int32).contiguous(), x.contiguous()
         state = {"i": 0}
 
         def step():
             a = (state["i"] % nb) * B
             state["i"] += 1
-            s.step_mf(i[a:a + B], j[a:a + B], x[a:a + B], 1e-4, 0.01, loss)
+            s.step_mf(i[a:a + B], j[a:a + B], x[a:a + B], 1e-4, 0.01, loss, by_column=args.mf_order == "column")     # "column-plain": the same cells through nups_step_mf
         per_item, upd, rows_per_item = 4, 2, 2
-        name, cfg = "mf_kernel", f"MF: 10M x 1M, rank 100, batch {B}, L2 0.01"
+        name, cfg = ("mf_runs_kernel" if args.mf_order == "column" else "mf_kernel"), f"MF: 10M x 1M, rank 100, batch {B}, L2 0.01, cells in {args.mf_order} order"
     dt = _time_calls(step, reps)
     s.kernel_timing(True)
     _time_calls(step, reps, warm=0)
@@ -674,6 +677,9 @@ def main():
     ap.add_argument("--ps-keys", type=int, default=100_000_000)
     ap.add_argument("--kge-entities", type=int, default=5_000_000, help="smaller for profiling runs")
     ap.add_argument("--mf-rows", type=int, default=10_000_000, help="smaller for profiling runs")
+    ap.add_argument("--mf-order", default="random", choices=["random", "column", "column-plain"],
+                    help="mf: independent cells, or the first cells of a 1G-cell data set visited column by column "
+                         "(column-plain: those cells through the step call for independent cells)")
     ap.add_argument("--ps-skews", default="0,0.6,1.0,1.4")
     ap.add_argument("--ps-topk", default="0,1000,100000")
     args = ap.parse_args()

@@ -276,6 +276,18 @@ nups_status nups_step_complex(nups_store* store, const uint32_t* d_h, const uint
 nups_status nups_step_mf(nups_store* store, const uint32_t* d_row, const uint32_t* d_col, const float* d_x, uint64_t n,
                          float lr, float l2, float* d_loss_out, void* stream);
 
+/* The same step for cells that arrive column by column (Section 5.1: each worker
+ * visits its cells by column, in random order of columns and of the cells within
+ * a column, to create locality in the column parameter accesses).  In fast mode
+ * a column's row is read once and its updates are summed and added once per
+ * stretch of consecutive cells of that column that one warp works on (all cells
+ * of such a stretch see the column's row from before the stretch, which is the
+ * batch semantics of the deterministic mode).  Any order of cells gives a correct
+ * step; the order only decides how much is saved.  In deterministic mode the
+ * call is nups_step_mf.  Arguments, ownership and errors as nups_step_mf.      */
+nups_status nups_step_mf_by_column(nups_store* store, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
+                                   uint64_t n, float lr, float l2, float* d_loss_out, void* stream);
+
 /* Keys drawn as negatives by the most recent step ([n * K], library-owned
  * device memory, valid until the next step).                                  */
 nups_status nups_last_negatives(nups_store* store, const uint32_t** h_d_keys_out, uint64_t* h_n_out);

@@ -24,7 +24,7 @@ EXPORTS = [
     "nups_create", "nups_destroy", "nups_table_ptr", "nups_table_copy", "nups_init_uniform", "nups_pull", "nups_pull2", "nups_push",
     "nups_push2", "nups_push_noalloc", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
-    "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_run_sgns", "nups_step_complex", "nups_step_mf",
+    "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_run_sgns", "nups_step_complex", "nups_step_mf", "nups_step_mf_by_column",
     "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_get_clip_stats", "nups_strerror", "nups_last_cuda_error",
 ]
 
@@ -87,6 +87,7 @@ def load(build_if_missing: bool = True):
         "nups_run_sgns": [vp, vp, vp, u64, u64, i32, u32, f32, vp, vp],
         "nups_step_complex": [vp, vp, vp, vp, u64, i32, u32, f32, f32, vp, vp],
         "nups_step_mf": [vp, vp, vp, vp, u64, f32, f32, vp, vp],
+        "nups_step_mf_by_column": [vp, vp, vp, vp, u64, f32, f32, vp, vp],
         "nups_last_negatives": [vp, C.POINTER(vp), C.POINTER(u64)],
         "nups_status_check": [vp, vp],
         "nups_get_stats": [vp, C.POINTER(u64), vp],
@@ -307,10 +308,12 @@ class Store:
                                             h.numel(), dist, K, lr, eps, _ptr(loss_out), _stream()),
                   "nups_step_complex")
 
-    def step_mf(self, rows, cols, x, lr, l2, loss_out=None):
-        self._chk(self._l.nups_step_mf(self._s, _ptr(rows, torch.int32), _ptr(cols, torch.int32),
-                                       _ptr(x, torch.float32), rows.numel(), lr, l2, _ptr(loss_out), _stream()),
-                  "nups_step_mf")
+    def step_mf(self, rows, cols, x, lr, l2, loss_out=None, by_column=False):
+        """One matrix-factorization step; by_column: the cells arrive column by column (nups_step_mf_by_column)."""
+        fn = self._l.nups_step_mf_by_column if by_column else self._l.nups_step_mf
+        self._chk(fn(self._s, _ptr(rows, torch.int32), _ptr(cols, torch.int32),
+                     _ptr(x, torch.float32), rows.numel(), lr, l2, _ptr(loss_out), _stream()),
+                  "nups_step_mf_by_column" if by_column else "nups_step_mf")
 
     def last_negatives(self):
         p, n = C.c_void_p(), C.c_uint64()

@@ -223,6 +223,13 @@ __device__ __forceinline__ uint32_t worker_of_item(uint64_t i, uint64_t n, uint3
     return (uint32_t)((i * R) / n);          // calls take fewer than 2^32 items: i * R < 2^40
 }
 
+// First item of worker q's chunk: the smallest i with floor(i * R / n) >= q, i.e. ceil(q * n / R).  A loop whose
+// item index only grows keeps its worker and the next chunk's first item instead of dividing for every item.
+__device__ __forceinline__ uint64_t worker_first_item(uint32_t q, uint64_t n, uint32_t R)
+{
+    return ((uint64_t)q * n + R - 1) / R;
+}
+
 // Sub-handle boundaries of a handle of N samples: b_q = floor(q * N / R).
 __device__ __forceinline__ uint64_t chunk_begin(uint32_t q, uint64_t N, uint32_t R) { return ((uint64_t)q * N) / R; }
 __device__ __forceinline__ uint32_t chunk_of_pos(uint64_t pos, uint64_t N, uint32_t R)

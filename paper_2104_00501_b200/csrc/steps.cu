@@ -1031,8 +1031,201 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     return step_finish(s, n, K + 3, b, d_loss_out, st, !s->cfg.deterministic);
 }
 
-extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
-                                    uint64_t n, float lr, float l2, float* d_loss_out, void* stream)
+// ---------------------------------------------------------------------------------------------
+// matrix factorization over cells that come column by column (Section 5.1: every worker visits its cells
+// by column, to create locality in the accesses to column parameters).  Fast mode only.
+// A warp works on a stretch of consecutive cells.  The keys, cell values and replica slots of 32 cells are
+// loaded by the 32 lanes at once, one window ahead.  The rows of the row keys are fetched MF_RUN_DEPTH cells
+// ahead into a register ring.  The row of the column key stays in registers while the column stays the same
+// (the next column's row is fetched one cell before it is needed), and the column's update is summed in
+// registers and added once when the column changes: a column's row costs one read and one reduction per
+// stretch instead of one per cell.  Within a stretch the cells of a column all see the column's row from
+// before the stretch (the batch semantics of the deterministic mode); rows of row keys are read as they are.
+// ---------------------------------------------------------------------------------------------
+constexpr int MF_RUN_DEPTH = 4;           // divides 32
+constexpr int MF_RUN_BLOCKS = 5;          // resident blocks per multiprocessor the grid is sized for
+
+template <bool HOT, int CH, bool CLIP>
+__global__ void __launch_bounds__(128, MF_RUN_BLOCKS)
+mf_runs_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
+               uint64_t n, float lr, float l2, float* __restrict__ loss_out)
+{
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = v.L4;
+    const float4* val4 = (const float4*)v.val;
+    const float4* slab4 = (const float4*)v.dval;
+    double my_loss = 0.0;
+    const float bound = CLIP ? clip_bound(v) : 0.f;
+    float my_clip = 0.f;
+    unsigned my_clipped = 0;
+    const uint64_t stretch = (n + nwarps - 1) / nwarps;
+    const uint64_t first = warp * stretch < n ? warp * stretch : n;
+    const uint64_t last = first + stretch < n ? first + stretch : n;            // this warp's cells: [first, last)
+
+    // one window = 32 consecutive cells, lane l holds cell l: keys (row key invalid when either key is),
+    // cell value, replica slots
+    struct Window { uint32_t ki, kj; float x; int si, sj; };
+    auto load_window = [&](uint64_t base) {
+        Window w = {NUPS_INVALID_KEY, NUPS_INVALID_KEY, 0.f, -1, -1};
+        const uint64_t i = base + lane;
+        if (i < last) {
+            const uint32_t ki = rowk[i], kj = colk[i];
+            w.x = x[i];
+            if (ki < v.num_keys && kj < v.num_keys) {
+                w.ki = ki; w.kj = kj;
+                if (HOT) { w.si = __ldg(v.slot_of + ki); w.sj = __ldg(v.slot_of + kj); }
+            } else {
+                flag_bad_key(v);
+            }
+        }
+        return w;
+    };
+    Window cur = load_window(first), nxt = load_window(first + 32);
+    // cell t of the current window (t < 32) or of the next one (32 <= t < 64)
+    auto row_key_at = [&](uint32_t t) {
+        const uint32_t a = __shfl_sync(FULL, cur.ki, t & 31), b = __shfl_sync(FULL, nxt.ki, t & 31);
+        return t < 32 ? a : b;
+    };
+    auto col_key_at = [&](uint32_t t) {
+        const uint32_t a = __shfl_sync(FULL, cur.kj, t & 31), b = __shfl_sync(FULL, nxt.kj, t & 31);
+        return t < 32 ? a : b;
+    };
+    auto fetch_row = [&](float4 (&dst)[CH], uint32_t key) {
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            const uint32_t c = lane + 32 * m;
+            dst[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (key != NUPS_INVALID_KEY && c < L4) dst[m] = val4[(uint64_t)key * L4 + c];
+        }
+    };
+
+    float4 ring[MF_RUN_DEPTH][CH];                       // stored rows of the row keys of the next cells
+#pragma unroll
+    for (int u = 0; u < MF_RUN_DEPTH; ++u) fetch_row(ring[u], row_key_at(u));
+    uint32_t h_key = NUPS_INVALID_KEY, h_next_key = NUPS_INVALID_KEY;
+    float4 h[CH], h_next[CH];                            // stored row of the current column, and of the one after it
+    {
+        const uint32_t k0 = col_key_at(0);
+        fetch_row(h_next, k0);
+        h_next_key = k0;
+    }
+    float* held_row = nullptr;                           // column row whose summed update is still in registers
+    float4 held[CH];
+    auto flush_held = [&]() {
+        if (!held_row) return;
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            const uint32_t c = lane + 32 * m;
+            if (c < L4) red_add_v4(held_row + 4 * c, held[m]);
+        }
+        held_row = nullptr;
+    };
+
+    uint32_t q = worker_of_item(first < n ? first : 0, n, v.R);    // worker of the cell at hand, kept up as i grows
+    uint64_t q_end = worker_first_item(q + 1, n, v.R);
+    float window_loss = 0.f;
+    for (uint64_t base = first; base < last; base += 32) {
+        for (uint32_t t0 = 0; t0 < 32; t0 += MF_RUN_DEPTH) {
+            if (base + t0 >= last) break;
+#pragma unroll
+            for (int u = 0; u < MF_RUN_DEPTH; ++u) {
+                const uint32_t t = t0 + u;
+                const uint64_t i = base + t;
+                if (i >= last) break;
+                const uint32_t ki = __shfl_sync(FULL, cur.ki, t), kj = __shfl_sync(FULL, cur.kj, t);
+                const float xv = __shfl_sync(FULL, cur.x, t);
+                const int si = __shfl_sync(FULL, cur.si, t), sj = __shfl_sync(FULL, cur.sj, t);
+                float4 w[CH];
+#pragma unroll
+                for (int m = 0; m < CH; ++m) w[m] = ring[u][m];
+                fetch_row(ring[u], row_key_at(t + MF_RUN_DEPTH));
+                if (ki == NUPS_INVALID_KEY) continue;               // a bad key: flagged when the window was loaded
+                if (kj != h_key) {
+                    if (h_next_key != kj) { fetch_row(h_next, kj); h_next_key = kj; }
+#pragma unroll
+                    for (int m = 0; m < CH; ++m) h[m] = h_next[m];
+                    h_key = kj;
+                }
+                {
+                    const uint32_t kj1 = col_key_at(t + 1);
+                    if (kj1 != NUPS_INVALID_KEY && kj1 != h_key && kj1 != h_next_key) { fetch_row(h_next, kj1); h_next_key = kj1; }
+                }
+                while (i >= q_end) q_end = worker_first_item(++q + 1, n, v.R);
+                const uint64_t pw = si >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)si) * L4 : 0;
+                const uint64_t ph = sj >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)sj) * L4 : 0;
+                float4 hv[CH];
+                float dot = 0.f;
+#pragma unroll
+                for (int m = 0; m < CH; ++m) {
+                    const uint32_t c = lane + 32 * m;
+                    hv[m] = h[m];
+                    if (c < L4) {
+                        if (HOT && si >= 0) w[m] = add4(w[m], slab4[pw + c]);       // the worker's pending replica updates
+                        if (HOT && sj >= 0) hv[m] = add4(hv[m], slab4[ph + c]);
+                    }
+                    dot += w[m].x * hv[m].x + w[m].y * hv[m].y + w[m].z * hv[m].z + w[m].w * hv[m].w;
+                }
+                const float err = xv - warp_sum(dot);
+                float fw = lr, fh = lr;                                 // learning rate times the clipping factor
+                if (CLIP && (si >= 0 || sj >= 0)) {
+                    float nw2 = 0.f, nh2 = 0.f;
+#pragma unroll
+                    for (int m = 0; m < CH; ++m) {
+                        if (lane + 32 * m < L4) {
+                            const float4 a = make_float4(err * hv[m].x - l2 * w[m].x, err * hv[m].y - l2 * w[m].y,
+                                                         err * hv[m].z - l2 * w[m].z, err * hv[m].w - l2 * w[m].w);
+                            const float4 b = make_float4(err * w[m].x - l2 * hv[m].x, err * w[m].y - l2 * hv[m].y,
+                                                         err * w[m].z - l2 * hv[m].z, err * w[m].w - l2 * hv[m].w);
+                            nw2 += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
+                            nh2 += b.x * b.x + b.y * b.y + b.z * b.z + b.w * b.w;
+                        }
+                    }
+                    float applied = 0.f, f;
+                    if (si >= 0) { applied += clip_norm(lr * sqrtf(warp_sum(nw2)), bound, &f); fw = lr * f; }
+                    if (sj >= 0) { applied += clip_norm(lr * sqrtf(warp_sum(nh2)), bound, &f); fh = lr * f; }
+                    my_clip += applied;
+                    my_clipped += (si >= 0 ? 1u : 0u) + (sj >= 0 ? 1u : 0u);
+                }
+                float* ow = si >= 0 ? v.dval + pw * 4 : v.val + (uint64_t)ki * L4 * 4;
+                float* oh = sj >= 0 ? v.dval + ph * 4 : v.val + (uint64_t)kj * L4 * 4;
+                if (held_row != oh) flush_held();
+#pragma unroll
+                for (int m = 0; m < CH; ++m) {
+                    const uint32_t c = lane + 32 * m;
+                    if (c < L4) {
+                        const float4 dw = make_float4(fw * (err * hv[m].x - l2 * w[m].x), fw * (err * hv[m].y - l2 * w[m].y),
+                                                      fw * (err * hv[m].z - l2 * w[m].z), fw * (err * hv[m].w - l2 * w[m].w));
+                        const float4 dh = make_float4(fh * (err * w[m].x - l2 * hv[m].x), fh * (err * w[m].y - l2 * hv[m].y),
+                                                      fh * (err * w[m].z - l2 * hv[m].z), fh * (err * w[m].w - l2 * hv[m].w));
+                        red_add_v4(ow + 4 * c, dw);
+                        held[m] = oh == held_row ? add4(held[m], dh) : dh;
+                    }
+                }
+                held_row = oh;
+                if (lane == 0) {
+                    if (si >= 0) mark_dirty(v, q, si);
+                    if (sj >= 0) mark_dirty(v, q, sj);
+                    if (v.count) { note_access(v, ki, si, 2u); note_access(v, kj, sj, 2u); }
+                    if (v.own) { mark_localize(v, ki, q); mark_localize(v, kj, q); }
+                }
+                window_loss += err * err;
+            }
+        }
+        my_loss += (double)window_loss;
+        window_loss = 0.f;
+        cur = nxt;
+        nxt = load_window(base + 64);
+    }
+    flush_held();
+    loss_finish(v, my_loss, n, loss_out);
+    if (CLIP) clip_finish(v, (double)my_clip, my_clipped);
+}
+
+static nups_status mf_step(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
+                           uint64_t n, float lr, float l2, float* d_loss_out, void* stream, bool cells_by_column)
 {
     if (!s || !d_row || !d_col || !d_x || n == 0 || n * 2 >= (1ull << 32)) return NUPS_EINVAL;
     if (s->L / 4 > 128) return NUPS_EINVAL;
@@ -1044,13 +1237,35 @@ extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const 
     rc = step_buffers(s, n, 2, false, &b);
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
-    unsigned grid = step_grid(s, n, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2));   // resident blocks at that depth's register use
+    const bool by_column = cells_by_column && !s->cfg.deterministic;    // the ordered mode is the same for any order
     nups_time_begin(s, st);
-    DISPATCH_MODE(s, DISPATCH_CLIP(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH, (HOT && CLIP)><<<grid, 128, 0, st>>>(
-        v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out, b.clip_item))));
+    if (by_column) {
+        const unsigned grid = step_grid(s, n, MF_RUN_BLOCKS);
+        DISPATCH_CLIP(s, DISPATCH_CH(v.L4, {
+            if (s->H) mf_runs_kernel<true, CH, CLIP><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, d_loss_out);
+            else mf_runs_kernel<false, CH, false><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, d_loss_out);
+        }));
+    } else {
+        const unsigned grid = step_grid(s, n, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2));   // resident blocks at that depth's register use
+        DISPATCH_MODE(s, DISPATCH_CLIP(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH, (HOT && CLIP)><<<grid, 128, 0, st>>>(
+            v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out, b.clip_item))));
+    }
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return step_finish(s, n, 2, b, d_loss_out, st, !s->cfg.deterministic, true);
+}
+
+extern "C" nups_status nups_step_mf(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
+                                    uint64_t n, float lr, float l2, float* d_loss_out, void* stream)
+{
+    return mf_step(s, d_row, d_col, d_x, n, lr, l2, d_loss_out, stream, false);
+}
+
+extern "C" nups_status nups_step_mf_by_column(nups_store* s, const uint32_t* d_row, const uint32_t* d_col,
+                                              const float* d_x, uint64_t n, float lr, float l2, float* d_loss_out,
+                                              void* stream)
+{
+    return mf_step(s, d_row, d_col, d_x, n, lr, l2, d_loss_out, stream, true);
 }
 
 extern "C" nups_status nups_get_clip_stats(nups_store* s, double* h_sum, uint64_t* h_count, void* stream)

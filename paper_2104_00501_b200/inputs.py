@@ -123,14 +123,30 @@ def kge_triples(num: int, entities: int, relations: int, s_ent: float, s_rel: fl
     return h, r, t
 
 
+def columns_in_visiting_order(num: int, cols: int, s: float, total_cells: int, seed: int, device="cpu") -> torch.Tensor:
+    """Column ranks (0-based) of the first `num` cells of a data set of `total_cells` cells that is visited column by
+    column (Section 5.1, matrix factorization): the columns come in random order, each with all of its cells, and a
+    column of rank r holds max(1, round(total_cells * r^-s / sum_r r^-s)) cells."""
+    g = _gen(seed, device)
+    order = torch.randperm(cols, generator=g, device=device)
+    w = torch.arange(1, cols + 1, device=device, dtype=torch.float64).pow_(-s)
+    cells = torch.round(w / w.sum() * float(total_cells)).clamp_(min=1).to(torch.int64)[order]
+    upto = int(torch.searchsorted(torch.cumsum(cells, 0), torch.tensor([num], device=device)).item()) + 1
+    return torch.repeat_interleave(order[:upto], cells[:upto])[:num]
+
+
 def mf_cells(num: int, rows: int, cols: int, s: float, rank: int, noise: float, seed: int, device="cpu",
-             factor_seed: int = 1234):
+             factor_seed: int = 1234, by_column_of: int = 0):
     """Revealed cells of a rows x cols matrix: indices ~ Zipf(s), value = <true row factor, true column
     factor> + N(0, noise).  True factor entries are N(0, rank^-1/4), made on the fly from a hash of
     (index, component) so that no full factor table is needed.  Row keys [0, rows), column keys
-    [rows, rows + cols)."""
+    [rows, rows + cols).  by_column_of = T > 0: the cells are the first `num` of a T-cell data set in
+    column-by-column visiting order (see columns_in_visiting_order) instead of independent draws."""
     i = zipf_keys(num, rows, s, seed * 2 + 0, device)
-    j = zipf_keys(num, cols, s, seed * 2 + 1, device)
+    if by_column_of:
+        j = rank_to_key(columns_in_visiting_order(num, cols, s, by_column_of, seed * 2 + 1, device), cols, seed=1)
+    else:
+        j = zipf_keys(num, cols, s, seed * 2 + 1, device)
     g = _gen(seed + 77, device)
     sigma = float(rank) ** -0.25
 

@@ -125,6 +125,75 @@ def test_mf_deterministic_parity(L, hot_n):
     assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
 
 
+@pytest.mark.parametrize("L,hot_n,n", [(100, 0, 4096), (100, 25, 4096), (8, 10, 3001), (300, 25, 1500)])
+def test_mf_fast_mode_on_cells_in_column_order(L, hot_n, n):
+    # cells visited column by column (Section 5.1): fast mode sums a column's updates over a stretch of cells before
+    # it adds them.  One step from the same start: every row's total update is the oracle's up to the races between
+    # cells that share a row (second order in the learning rate, which is small here), so a lost or misdirected
+    # sum (a whole stretch of a column) cannot hide in the tolerance
+    M, N, R = 500, 200, 4
+    i, j, x = inputs.mf_cells(n, M, N, 0.8, max(L // 4, 2), 0.1, 0, by_column_of=20 * n)
+    assert len(torch.unique_consecutive(j)) < n // 8               # long runs of one column
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    init = np.random.default_rng(0).normal(0, 0.3, size=(M + N, L)).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, init=init, deterministic=False)
+    if hot_n:
+        o.count_accesses(np.concatenate([i, j]))
+        hot = o.select_hot(True, hot_n)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    lb = loss_buf()
+    lo = o.step_mf(i, j, x, 1e-4, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), 1e-4, 0.01, lb, by_column=True)
+    assert abs(lb.item() - lo) <= 2e-3 * abs(lo)
+    o.sync()
+    s.sync()
+    d_o = o.table(0).astype(np.float64) - init
+    d_s = s.read_table(0).cpu().numpy().astype(np.float64) - init
+    norm = np.linalg.norm(d_o, axis=1)
+    assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.01 * norm + 1e-6)
+    assert norm.max() > 1e-4
+    assert s.status_check() == 0
+
+
+def test_mf_by_column_takes_any_order_bad_keys_and_single_cells():
+    # independent cells (hardly any runs), keys out of range in the middle and at the end, access counting and the
+    # ownership map on: counts are exact, bad cells are skipped and flagged, every row's update is the oracle's
+    M, N, L, R, n = 60, 40, 100, 3, 701
+    i, j, x = inputs.mf_cells(n, M, N, 0.8, 8, 0.1, 1)
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    init = np.random.default_rng(1).normal(0, 0.3, size=(M + N, L)).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, init=init, deterministic=False, count_accesses=True, track_ownership=True)
+    hot = np.array([int(i[0]), int(j[0])], np.uint32)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    lb = loss_buf()
+    lo = o.step_mf(i, j, x, 1e-4, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), 1e-4, 0.01, lb, by_column=True)
+    assert abs(lb.item() - lo) <= 2e-3 * abs(lo)
+    assert s.status_check() == 0
+    one = slice(5, 6)
+    lo = o.step_mf(i[one], j[one], x[one], 1e-4, 0.01)
+    s.step_mf(dev_keys(i[one]), dev_keys(j[one]), dev_f32(x[one]), 1e-4, 0.01, lb, by_column=True)
+    assert abs(lb.item() - lo) <= 1e-4 * abs(lo) + 1e-7
+    o.sync()
+    s.sync()
+    d_o = o.table(0).astype(np.float64) - init
+    d_s = s.read_table(0).cpu().numpy().astype(np.float64) - init
+    norm = np.linalg.norm(d_o, axis=1)
+    assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.01 * norm + 1e-6)
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+    # cells with a key out of range change nothing and raise the flag
+    before = s.read_table(0).clone()
+    bi, bj = i[:40].copy(), j[:40].copy()
+    bi[:] = M + N + 3
+    bj[-1] = 0xFFFFFFF0
+    s.step_mf(dev_keys(bi), dev_keys(bj), dev_f32(x[:40]), 1e-4, 0.01, lb, by_column=True)
+    s.sync()
+    assert s.status_check() == -4
+    assert torch.equal(s.read_table(0), before)
+
+
 def test_fast_mode_reaches_the_oracles_loss_within_one_percent():
     # replicated + asynchronous mode: same number of epochs, final loss within 1 % of the oracle's
     V, L, K, R, batch = 500, 32, 3, 8, 256
