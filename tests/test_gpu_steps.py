@@ -376,22 +376,26 @@ def test_mf_clipping_matches_the_oracle_and_fast_mode_counts_the_same_updates():
     o.set_clipping(0.8)
     o.set_management(hot, REPLICATE)
     stores = {}
-    for det in (True, False):
+    for det, by_column in ((True, False), (False, False), (False, True)):      # ordered, fast, fast by column
         s = binding.Store(M + N, L, workers=R, sync_interval=1, deterministic=det, clip_factor=0.8)
         s.write_table(0, init)
         s.set_management(dev_keys(hot), REPLICATE)
-        stores[det] = s
+        stores[(det, by_column)] = s
     lb = loss_buf()
     for b in range(3):
         sl = slice(b * 500, (b + 1) * 500)
-        lo = o.step_mf(rows[sl], cols[sl], x[sl], 0.05, 0.01)
-        for det, s in stores.items():
-            s.step_mf(dev_keys(rows[sl]), dev_keys(cols[sl]), dev_f32(x[sl]), 0.05, 0.01, lb)
+        order = np.argsort(cols[sl], kind="stable")                          # each step's cells column by column
+        r_b, c_b, x_b = rows[sl][order], cols[sl][order], x[sl][order]
+        lo = o.step_mf(r_b, c_b, x_b, 0.05, 0.01)
+        for (det, by_column), s in stores.items():
+            s.step_mf(dev_keys(r_b), dev_keys(c_b), dev_f32(x_b), 0.05, 0.01, lb, by_column=by_column)
             if det:
                 assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
-    tables_close(o, stores[True])
+            else:
+                assert abs(lb.item() - lo) <= 0.1 * abs(lo)
+    tables_close(o, stores[(True, False)])
     so, co = o.clip_stats()
-    for det, s in stores.items():
+    for (det, by_column), s in stores.items():
         ss, cs = s.clip_stats()
         assert cs == co
         assert ss == pytest.approx(so, rel=1e-5 if det else 0.25)
