@@ -225,3 +225,41 @@ def test_benchmark_sized_mf_batches_match_the_oracle():
     np.testing.assert_allclose(got, o.table(0)[rows], rtol=1e-5, atol=1e-6)
     assert len(hot) > 0 and s.status_check() == 0
     s.close()
+
+
+def test_benchmark_sized_mf_batch_in_column_order_matches_the_oracle():
+    # the by-column kernel in the benchmark's launch configuration (65,536 cells visited column by column, fast mode,
+    # frequent rows and columns replicated): one step from the same start; every key's total update is the oracle's.
+    # The learning rate is tiny so that what a cell sees of the other cells' updates (which the oracle's batch step
+    # never shows it) stays below the tolerance even for rows that hundreds of cells share
+    M, N, L, B, R = 1_000_000, 100_000, 100, 65_536, bench.WORKERS
+    i, j, x = inputs.mf_cells(B, M, N, 0.8, 100, 0.1, 0, by_column_of=100 * M)
+    assert len(torch.unique_consecutive(j)) < B // 100
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    o = Oracle(M + N, L, workers=R, sync_interval=1)
+    s = binding.Store(M + N, L, workers=R, sync_interval=1, deterministic=False)
+    o.init_uniform(0, 5, 0.3)
+    s.init_uniform(0, 5, 0.3)
+    ii, jj, _ = inputs.mf_cells(2 * B, M, N, 0.8, 100, 0.1, 0)
+    o.count_accesses(np.concatenate([inputs.u32(ii), inputs.u32(jj)]))
+    hot = o.select_hot(False, 100)
+    o.set_management(hot, REPLICATE)
+    s.set_management(torch.from_numpy(hot.view(np.int32)).cuda(), binding.REPLICATE)
+    rows = np.unique(np.concatenate([i, j]))
+    start = o.table(0)[rows].astype(np.float64)
+    lb = torch.zeros(1, device="cuda")
+    dk = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).cuda()
+    lr = 2e-6
+    lo = o.step_mf(i, j, x, lr, 0.01)
+    s.step_mf(dk(i), dk(j), torch.from_numpy(x.copy()).cuda(), lr, 0.01, lb, by_column=True)
+    assert abs(lb.item() - lo) <= 2e-3 * abs(lo)
+    got = s.read_table(0)[torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy().astype(np.float64)
+    d_s, d_o = got - start, o.table(0)[rows].astype(np.float64) - start
+    norm = np.linalg.norm(d_o, axis=1)
+    err = np.linalg.norm(d_s - d_o, axis=1)
+    assert np.all(err <= 0.02 * norm + 1e-6)                # every key; the second term is fp32 rounding of the stored rows
+    cells = np.bincount(np.searchsorted(rows, np.concatenate([i, j])), minlength=len(rows))
+    many = cells >= 64
+    assert many.sum() > 50 and np.all(err[many] <= 0.02 * norm[many])
+    assert len(hot) > 0 and s.status_check() == 0
+    s.close()
