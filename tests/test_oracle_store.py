@@ -37,7 +37,7 @@ def test_out_of_range_key_is_skipped_and_flagged():
 
 @pytest.mark.parametrize("R,hot", [(1, []), (4, []), (4, [3, 7, 1]), (8, list(range(10)))])
 def test_conservation_value_is_init_plus_all_pushed_deltas(R, hot):
-    # BASELINE pin: after sync, value = init + sum of pushed deltas, whatever the hot set
+    # pin: after sync, value = init + sum of pushed deltas, whatever the hot set
     nk, L = 10, 6
     rng = np.random.default_rng(1)
     o = Oracle(nk, L, workers=R)
