@@ -143,16 +143,20 @@ def test_mf_fast_mode_on_cells_in_column_order(L, hot_n, n):
         o.set_management(hot, REPLICATE)
         s.set_management(dev_keys(hot), REPLICATE)
     lb = loss_buf()
-    lo = o.step_mf(i, j, x, 1e-4, 0.01)
-    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), 1e-4, 0.01, lb, by_column=True)
+    # a cell may see updates of cells before it, which the oracle's batch step never shows: for a row that c cells
+    # share that changes its update by up to lr * c * |row|^2 (first order), so the learning rate is tiny; the
+    # absolute term is the fp32 rounding of the stored rows
+    lr = 2e-6
+    lo = o.step_mf(i, j, x, lr, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), lr, 0.01, lb, by_column=True)
     assert abs(lb.item() - lo) <= 2e-3 * abs(lo)
     o.sync()
     s.sync()
     d_o = o.table(0).astype(np.float64) - init
     d_s = s.read_table(0).cpu().numpy().astype(np.float64) - init
     norm = np.linalg.norm(d_o, axis=1)
-    assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.01 * norm + 1e-6)
-    assert norm.max() > 1e-4
+    assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.01 * norm + 2e-6)
+    assert norm.max() > 2e-5
     assert s.status_check() == 0
 
 
@@ -168,27 +172,29 @@ def test_mf_by_column_takes_any_order_bad_keys_and_single_cells():
     o.set_management(hot, REPLICATE)
     s.set_management(dev_keys(hot), REPLICATE)
     lb = loss_buf()
-    lo = o.step_mf(i, j, x, 1e-4, 0.01)
-    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), 1e-4, 0.01, lb, by_column=True)
+    lr = 2e-6                                  # tiny, see test_mf_fast_mode_on_cells_in_column_order
+    lo = o.step_mf(i, j, x, lr, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), lr, 0.01, lb, by_column=True)
     assert abs(lb.item() - lo) <= 2e-3 * abs(lo)
     assert s.status_check() == 0
     one = slice(5, 6)
-    lo = o.step_mf(i[one], j[one], x[one], 1e-4, 0.01)
-    s.step_mf(dev_keys(i[one]), dev_keys(j[one]), dev_f32(x[one]), 1e-4, 0.01, lb, by_column=True)
+    lo = o.step_mf(i[one], j[one], x[one], lr, 0.01)
+    s.step_mf(dev_keys(i[one]), dev_keys(j[one]), dev_f32(x[one]), lr, 0.01, lb, by_column=True)
     assert abs(lb.item() - lo) <= 1e-4 * abs(lo) + 1e-7
     o.sync()
     s.sync()
     d_o = o.table(0).astype(np.float64) - init
     d_s = s.read_table(0).cpu().numpy().astype(np.float64) - init
     norm = np.linalg.norm(d_o, axis=1)
-    assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.01 * norm + 1e-6)
+    assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.01 * norm + 2e-6)
+    assert norm.max() > 2e-5
     assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
     # cells with a key out of range change nothing and raise the flag
     before = s.read_table(0).clone()
     bi, bj = i[:40].copy(), j[:40].copy()
     bi[:] = M + N + 3
     bj[-1] = 0xFFFFFFF0
-    s.step_mf(dev_keys(bi), dev_keys(bj), dev_f32(x[:40]), 1e-4, 0.01, lb, by_column=True)
+    s.step_mf(dev_keys(bi), dev_keys(bj), dev_f32(x[:40]), lr, 0.01, lb, by_column=True)
     s.sync()
     assert s.status_check() == -4
     assert torch.equal(s.read_table(0), before)
