@@ -200,6 +200,31 @@ def test_mf_by_column_takes_any_order_bad_keys_and_single_cells():
     assert torch.equal(s.read_table(0), before)
 
 
+def test_mf_by_column_sends_each_cells_update_to_its_own_workers_replica():
+    # no merge after the step: a pull from worker q's part of a call sees the stored row plus q's pending updates
+    # only, so the replicas must hold exactly the updates of the cells that belong to each worker
+    M, N, L, R, n = 80, 30, 100, 5, 2003
+    i, j, x = inputs.mf_cells(n, M, N, 0.8, 8, 0.1, 4, by_column_of=30 * n)
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    init = np.random.default_rng(4).normal(0, 0.3, size=(M + N, L)).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, init=init, deterministic=False, sync_interval=0)
+    o.count_accesses(np.concatenate([i, j]))
+    hot = o.select_hot(True, 12)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    lr = 2e-6
+    o.step_mf(i, j, x, lr, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), lr, 0.01, loss_buf(), by_column=True)
+    keys = np.tile(hot, R).astype(np.uint32)                    # item block q of the pull belongs to worker q
+    want = o.pull(keys).astype(np.float64) - init[keys]
+    got = s.pull(dev_keys(keys)).cpu().numpy().astype(np.float64) - init[keys]
+    norm = np.linalg.norm(want, axis=1)
+    assert np.all(np.linalg.norm(got - want, axis=1) <= 0.01 * norm + 2e-6)
+    per_worker = norm.reshape(R, len(hot))
+    assert (per_worker > 1e-5).sum() >= 2 * R                   # several workers hold updates of several keys ...
+    assert np.ptp(per_worker, axis=0).max() > 1e-5              # ... and not the same ones
+
+
 def test_fast_mode_reaches_the_oracles_loss_within_one_percent():
     # replicated + asynchronous mode: same number of epochs, final loss within 1 % of the oracle's
     V, L, K, R, batch = 500, 32, 3, 8, 256
