@@ -1,17 +1,19 @@
 #!/usr/bin/env python
 """Benchmark of the NuPS sparse access path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload ...]
 
-Workload: skip-gram with negative sampling on a 1M-word vocabulary, dimension 300
-(input and output vectors in one 2M-key store), token stream ~ Zipf(1.0), window 5, 3 negatives per
-pair from unigram^0.75 under pooled reuse (BOUNDED, U = 16, G = 250), batches of 4096 pairs, top 1 %
-of keys replicated, replicas merged every 16 batches, fast (atomic) mode.  One step = one batch through
-the whole path: PrepareSample, PullSample, pulls, dot products, pushes, localize bookkeeping, and the
-periodic merge.  Metric: key accesses per second (2 direct pulls + 3 sampled pulls + 5 pushes per pair).
+Default workload: the parameter-server microbenchmark.  A store of 100M keys x 128 fp32 (51.2 GB), batches of
+1M keys ~ Zipf(1.0), the 1,000 most frequent keys replicated over 8 workers, replicas merged every 16 batches,
+fast (atomic) mode.  One step = one pull of 1M keys + one push of 1M keys (+ the replica merge when it is due) +
+PrepareSample and PullSample (keys and rows) of 1M keys from a Zipf(1.0) target over the whole store under pooled
+reuse (BOUNDED, U = 16, G = 250).  Metric: key accesses per second (every pulled, pushed or sampled key is one).
+The same run adds a `sweep` of the other points of that benchmark (skew 0 / 0.6 / 1.0 / 1.4, top-k 0 / 1k / 100k,
+merge interval 1 / 16 / 256, the four sampling schemes) and one entry for each workload step (skip-gram, ComplEx,
+matrix factorization).
 
-With N > 1 every rank runs an independent replica of the workload on its own GPU (the path has no
-exchange step on one node); the aggregate is total accesses over the slowest rank's time.
+With N > 1 every rank runs an independent replica of the workload on its own GPU (the path has no exchange step
+on one node); the aggregate is total accesses over the slowest rank's time.
 """
 from __future__ import annotations
 
@@ -39,10 +41,43 @@ TOKENS = 100_000_000
 ACCESSES_PER_PAIR = 2 + NEG + (NEG + 2)          # direct pulls + sampled pulls + pushes
 UPDATES_PER_PAIR = NEG + 2
 MAX_DISTINCT_BATCHES = 4096
+WORKLOAD_SGNS = ("SGNS word vectors: vocab 1M, dim 300, 100M-token Zipf(1.0) stream, window 5, 3 negatives unigram^0.75 "
+                 "BOUNDED(U=16,G=250), batch 4096 pairs, top 1% keys replicated, sync every 16 batches, fast (atomic) mode")
+
+# the parameter-server microbenchmark (the default line)
+PS_KEYS, PS_LEN, PS_BATCH = 100_000_000, 128, 1 << 20
+PS_SKEW, PS_TOPK, PS_SYNC, PS_LEVEL = 1.0, 1000, 16, "BOUNDED"
+PS_SKEWS, PS_TOPKS, PS_SYNCS = (0.0, 0.6, 1.0, 1.4), (0, 1000, 100_000), (1, 16, 256)
+PS_LEVELS = ("CONFORM", "BOUNDED", "LONG-TERM", "NON-CONFORM")
+PS_ORACLE_KEYS = 4_000_000                     # the oracle's table is scaled down to fit host memory everywhere
+WORKLOAD_PS = ("PS microbenchmark: 100M keys x 128 fp32, 1M-key batches ~ Zipf(1.0), pull:push 1:1, top-1k keys replicated "
+               "over 8 workers, replicas merged every 16 batches, plus PrepareSample+PullSample of 1M keys from a Zipf(1.0) "
+               "target under BOUNDED(U=16,G=250); one step = one pull + one push + one sample pull, fast (atomic) mode")
 
 # DRAM traffic of one launch of the fused step kernel (16 steps per launch), from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum); valid only for the kernel source it was captured on (sgns_kernel_sha1).
 NCU_TRAFFIC = {"bytes_per_launch": 41620224, "sgns_kernel_sha1": "48f21389a1da332791a366ac05ca6a967def1b94"}
+
+# The same for the kernels of the default line, each from one ncu capture of a 1M-key launch at the line's own
+# configuration (see profiles/): bytes per launch and the hash of the kernel's source text at the time of the capture.
+# A kernel whose source has changed since reports no traffic.
+NCU_TRAFFIC_PS = {
+    "pull": {"bytes_per_launch": None, "sha1": None},
+    "push": {"bytes_per_launch": None, "sha1": None},
+    "sample_rows": {"bytes_per_launch": None, "sha1": None},
+}
+PS_KERNEL_SOURCE = {   # kind -> (kernel name, start and end markers of its source text in store.cu)
+    "pull": ("gather8_kernel", "// The same gather with 256-bit loads and stores", "nups_status nups_gather_internal("),
+    "push": ("push_atomic_kernel", "// push, fast mode: 128-bit reductions", "// push, deterministic mode"),
+    "sample_rows": ("gather8_kernel", "// The same gather with 256-bit loads and stores", "nups_status nups_gather_internal("),
+}
+
+
+def kernel_source_sha1(start_marker, end_marker, name="store.cu"):
+    """Hash of a kernel's source text (the part of the file between two markers)."""
+    src = open(os.path.join(ROOT, "paper_2104_00501_b200", "csrc", name)).read()
+    a = src.index(start_marker)
+    return hashlib.sha1(src[a:src.index(end_marker, a)].encode()).hexdigest()
 
 
 def sgns_kernel_sha1():
@@ -163,7 +198,7 @@ def aggregate_throughput(units_per_rank, seconds, world):
     return units_per_rank * world / seconds
 
 
-def run_ours(args, rank, world, device):
+def run_sgns_line(args, rank, world, device):
     from paper_2104_00501_b200 import binding
     hbm_peak, peak_kind = peaks()
     nb = min(-(-(args.steps + args.warmup) // 64) * 64, MAX_DISTINCT_BATCHES)
@@ -302,9 +337,7 @@ def run_ours(args, rank, world, device):
         "metric": "key accesses/s (pull+push+sample)", "value": value, "unit": "key accesses/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": "SGNS word vectors: vocab 1M, dim 300, 100M-token Zipf(1.0) stream, window 5, "
-                               "3 negatives unigram^0.75 BOUNDED(U=16,G=250), batch 4096 pairs, top 1% keys replicated, "
-                               "sync every 16 batches, fast (atomic) mode",
+        "config": {"workload": WORKLOAD_SGNS,
                    "workers": WORKERS, "l2": "tables (2.4 GB) larger than L2; no explicit flush",
                    "distinct_batches": nb, "replicas": world},
         "updates_per_s": pairs * UPDATES_PER_PAIR / (ms / 1e3),
@@ -330,7 +363,7 @@ def run_ours(args, rank, world, device):
                      "reduction_rate_l2_resident_gbs": red_l2, "reduction_rate_dram_gbs": red_dram},
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(c, o, weights, hot, budget_s=12.0)
+        out["cpu_baseline"] = sgns_cpu_baseline(c, o, weights, hot, budget_s=12.0)
     return out
 
 
@@ -346,7 +379,7 @@ def oracle_setup(weights, hot):
     return o, d
 
 
-def cpu_baseline(c, o_keys, weights, hot, budget_s):
+def sgns_cpu_baseline(c, o_keys, weights, hot, budget_s):
     orc, d = oracle_setup(weights, hot)
     hc, ho = inputs.u32(c), inputs.u32(o_keys)
     nb = len(hc) // BATCH
@@ -362,7 +395,7 @@ def cpu_baseline(c, o_keys, weights, hot, budget_s):
                       f"{dt:.1f} s on one host thread (of {os.cpu_count()} cores)"}
 
 
-def run_reference(args):
+def run_sgns_reference(args):
     dev = "cuda" if torch.cuda.is_available() else "cpu"
     # bounded sample: the pairs of one step are a prefix of a batch, sized after a probe step so that the
     # whole run stays within a few minutes
@@ -397,9 +430,7 @@ def run_reference(args):
         "impl": "reference", "metric": "key accesses/s (pull+push+sample)", "value": value, "unit": "key accesses/s",
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "SGNS word vectors: vocab 1M, dim 300, Zipf(1.0) tokens, window 5, 3 negatives "
-                               "BOUNDED(U=16,G=250), batch 4096 pairs, top 1% keys replicated, sync every 16 batches",
-                   "sample": sample},
+        "config": {"workload": WORKLOAD_SGNS, "sample": sample},
         "cpu_baseline": {"value": value, "unit": "key accesses/s", "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "key accesses/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }

@@ -348,6 +348,12 @@ nups_status nups_get_stats(nups_store* store, uint64_t* h_out, void* stream);
 nups_status nups_kernel_timing(nups_store* store, int enable);
 nups_status nups_kernel_time(nups_store* store, double* h_ms_out, uint64_t* h_launches_out, void* stream);
 
+/* The same, kept apart by kind of kernel: h_ms_out[8] and h_launches_out[8] receive, at index
+ * 0 the row gather of nups_pull*, 1 the scatter-add of nups_push* (fast mode), 2 the fused kernel of
+ * nups_step_*, 3 the row copy of nups_pull_sample, 4 the draw kernel of nups_prepare_sample; the
+ * other entries are zero.  Synchronises the stream and starts afresh, like nups_kernel_time.     */
+nups_status nups_kernel_times(nups_store* store, double* h_ms_out, uint64_t* h_launches_out, void* stream);
+
 /* Measurement aid: the rate at which this GPU applies 128-bit floating-point
  * reductions (red.global.add.v4.f32, the instruction every fast-mode update
  * uses) to distinct, streaming addresses.  Adds zeros to the first `bytes` bytes

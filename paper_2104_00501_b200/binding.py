@@ -25,7 +25,7 @@ EXPORTS = [
     "nups_push2", "nups_push_noalloc", "nups_set_management", "nups_sync", "nups_count_accesses", "nups_get_counts", "nups_select_hot",
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_run_sgns", "nups_step_complex", "nups_step_mf", "nups_step_mf_by_column",
-    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_get_clip_stats", "nups_strerror", "nups_last_cuda_error",
+    "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_kernel_times", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_get_clip_stats", "nups_strerror", "nups_last_cuda_error",
 ]
 
 
@@ -93,6 +93,7 @@ def load(build_if_missing: bool = True):
         "nups_get_stats": [vp, C.POINTER(u64), vp],
         "nups_kernel_timing": [vp, C.c_int],
         "nups_kernel_time": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
+        "nups_kernel_times": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
         "nups_probe_reduction_rate": [vp, u64, u32, C.POINTER(C.c_double), vp],
         "nups_set_sync_period": [vp, u32],
         "nups_get_clip_stats": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
@@ -337,6 +338,14 @@ class Store:
         ms, n = C.c_double(), C.c_uint64()
         self._chk(self._l.nups_kernel_time(self._s, C.byref(ms), C.byref(n), _stream()), "nups_kernel_time")
         return ms.value, n.value
+
+    KERNEL_KINDS = ("pull", "push", "step", "sample_rows", "draw")
+
+    def kernel_times(self):
+        """{kind: (milliseconds, launches)} of the main kernels since the last query, by kind of kernel."""
+        ms, n = (C.c_double * 8)(), (C.c_uint64 * 8)()
+        self._chk(self._l.nups_kernel_times(self._s, ms, n, _stream()), "nups_kernel_times")
+        return {name: (ms[i], n[i]) for i, name in enumerate(self.KERNEL_KINDS)}
 
     def probe_reduction_rate(self, nbytes, reps=10):
         """GB/s of 128-bit floating-point reductions to streaming addresses (the ceiling of fast-mode updates)."""

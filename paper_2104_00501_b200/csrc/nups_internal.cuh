@@ -13,7 +13,8 @@
 #define NUPS_OWNER_DEFAULT 255
 #define NUPS_INVALID_KEY 0xFFFFFFFFu
 #define NUPS_MAX_POOL 1024
-#define NUPS_MAX_TIMED 4096
+#define NUPS_MAX_TIMED 65536
+#define NUPS_TIMED_KINDS 8
 #define NUPS_MAX_STEP_BLOCKS 8192
 #define NUPS_SAMPLE_AHEAD 16
 
@@ -109,13 +110,14 @@ struct nups_store {
     int device, sm_count, max_smem;
     int timing;                // record events around the main kernels?
     cudaEvent_t* ev;           // [2 * NUPS_MAX_TIMED] begin/end pairs
+    unsigned char* ev_kind;    // [NUPS_MAX_TIMED] which kernel the pair brackets (NUPS_TIMED_*)
     uint32_t ev_n;             // pairs recorded since the last query
-    double ev_ms;              // time of pairs folded in when the ring filled up
-    uint64_t ev_launches;
+    double ev_ms[NUPS_TIMED_KINDS];          // time of the pairs folded in so far, by kind
+    uint64_t ev_launches[NUPS_TIMED_KINDS];
     struct nups_background* bg; // time-based replica synchronisation (background.cu); NULL = never started
     cudaStream_t side;          // nups_run_sgns: a due replica merge runs here, beside the next steps' sample draw
     cudaEvent_t side_fork, side_join;
-    bool push_smem_opted, complex_smem_opted[2][2];   // large dynamic shared memory asked for on this store's device
+    bool push_smem_opted, complex_smem_opted[2][2][2];   // large dynamic shared memory asked for on this store's device
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };
@@ -148,7 +150,9 @@ static inline unsigned grid_for(uint64_t work, unsigned per_block, unsigned cap 
 }
 
 View nups_view(const nups_store* s);
-void nups_time_begin(nups_store* s, cudaStream_t st);
+// kinds of kernels that nups_kernel_timing brackets (index into the arrays nups_kernel_times returns)
+enum { NUPS_TIMED_PULL = 0, NUPS_TIMED_PUSH = 1, NUPS_TIMED_STEP = 2, NUPS_TIMED_SAMPLE_ROWS = 3, NUPS_TIMED_DRAW = 4 };
+void nups_time_begin(nups_store* s, cudaStream_t st, int kind);
 void nups_time_end(nups_store* s, cudaStream_t st);
 nups_status nups_scratch(nups_store* s, size_t bytes, char** out);     // grow-only scratch, 256-byte aligned
 nups_status nups_new_epoch(nups_store* s, cudaStream_t st);          // call before taking the view of a call that moves keys

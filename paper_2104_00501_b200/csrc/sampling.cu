@@ -505,6 +505,7 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
     View v = nups_view(s);
     const unsigned long long* off_cur = d.off + (size_t)d.cur * s->R;
     unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
+    nups_time_begin(s, st, NUPS_TIMED_DRAW);
     if (reuse) {
         const ReuseShape sh = reuse_shape(d.U, d.G);
         draw_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R), REUSE_THREADS, sh.smem, st>>>(
@@ -512,6 +513,7 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
     } else {
         draw_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(v, p, off_cur, off_next, hv, N, loc);
     }
+    nups_time_end(s, st);
     LAUNCH_CHECK(s);
     d.cur ^= 1;
     h.used = 1; h.dist = dist; h.N = N; h.cursor = 0;
@@ -803,10 +805,12 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         const uint32_t c8 = s->L / 8;
         const bool fused = d_vals_out && h.cursor == 0 && n == h.N && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) &&
                            ((uintptr_t)d_vals_out & 31) == 0 && (uint64_t)s->R * s->Hcap < 0xFFFFFFFFull;
+        if (fused) nups_time_begin(s, st, NUPS_TIMED_SAMPLE_ROWS);
         if (fused && c8 == 8) lt_place_kernel<8><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
         else if (fused && c8 == 16) lt_place_kernel<16><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
         else if (fused) lt_place_kernel<32><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
         else lt_place_kernel<0><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, nullptr, nullptr, nullptr);
+        if (fused) nups_time_end(s, st);
         LAUNCH_CHECK(s);
         if (fused) {
             h.cursor += n;

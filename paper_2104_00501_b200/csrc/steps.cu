@@ -5,6 +5,7 @@
 // into a row buffer that the ordered push applies afterwards (deterministic mode, all pulls see the
 // values from before the step).
 #include <mutex>
+#include <type_traits>
 #include <vector>
 
 #include "nups_internal.cuh"
@@ -16,11 +17,6 @@ namespace {
 __device__ __forceinline__ float clamp30(float x) { return fminf(30.f, fmaxf(-30.f, x)); }
 __device__ __forceinline__ float sigmoidf_(float x) { return 1.f / (1.f + expf(-x)); }
 __device__ __forceinline__ float softplusf_(float x) { return fmaxf(x, 0.f) + log1pf(expf(-fabsf(x))); }
-
-__device__ __forceinline__ void red_add_v2(float* addr, float2 x)
-{
-    asm volatile("red.global.add.v2.f32 [%0], {%1, %2};" ::"l"(addr), "f"(x.x), "f"(x.y) : "memory");
-}
 
 // lane 0 of the item's warp: access count and replica/in-place statistics for one key
 __device__ __forceinline__ void note_access(const View& v, uint32_t key, int slot, unsigned times)
@@ -301,139 +297,168 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
 
 // ---------------------------------------------------------------------------------------------
 // ComplEx with AdaGrad.  Rows are [re(0..d-1) | im(0..d-1)], d = L/2 (even).  One block of 128 threads
-// works on one triple at a time; thread c owns the two adjacent complex components 2c, 2c+1 (a float2
-// of the real half and the matching float2 of the imaginary half), so d <= 256.  All 2 * (3 + K) rows of
-// the triple (values and accumulators) are brought into shared memory by asynchronous copies at once,
-// each thread its own column; then two passes around one block-wide reduction: pass 1 forms the 1 + K
-// partial scores, the block adds them up, pass 2 forms the gradients and pushes the AdaGrad updates.
+// works on one triple at a time.  All 2 * (3 + K) rows of the triple (values and accumulators) are brought
+// into shared memory as they lie in memory, by asynchronous 16-byte copies that are all in flight at once
+// (thread t moves chunk t of every row and folds the worker's pending replica updates into what it moved).
+// For the arithmetic thread c owns the two adjacent complex components 2c, 2c+1 (a float2 of the real half
+// and the matching float2 of the imaginary half), so d <= 256.  Pass 1 forms the thread's part of the
+// 1 + K scores; they are added up across the block together (one transposed warp reduction for up to 16
+// scores instead of one reduction per score).  Pass 2 forms the gradients and leaves every role's AdaGrad
+// update in the shared-memory rows it no longer needs; after a barrier thread t hands chunk t of every
+// update row to the store with one 128-bit reduction (fast mode) or one 128-bit store into the row buffer
+// of the ordered push (deterministic mode).
+// Deterministic mode computes in double precision between pull and push (scores, gradients, AdaGrad step),
+// rounding once when the update rows are stored; fast mode computes in single precision.
 // ---------------------------------------------------------------------------------------------
-struct C2 { float2 re, im; };
 constexpr int CPX_THREADS = 128;
 constexpr int CPX_MAX_KEYS = 34;          // 3 + K with K <= 30, rounded up
+constexpr int CPX_NS = 16;                // up to this many scores are reduced together
 
-__device__ __forceinline__ C2 c2_zero() { C2 z; z.re = make_float2(0.f, 0.f); z.im = z.re; return z; }
+template <class T> struct CX { T re[2], im[2]; };
 
-__device__ __forceinline__ float c2_score(const C2& h, const C2& r, const C2& t)
+template <class T> __device__ __forceinline__ CX<T> cx_zero() { CX<T> z; z.re[0] = z.re[1] = z.im[0] = z.im[1] = T(0); return z; }
+
+__device__ __forceinline__ float mul_rn(float a, float b) { return __fmul_rn(a, b); }
+__device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(a, b); }
+__device__ __forceinline__ float sub_rn(float a, float b) { return __fsub_rn(a, b); }
+__device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
+
+// the thread's components of a row staged in shared memory
+template <class T>
+__device__ __forceinline__ CX<T> cx_load(const float* row, uint32_t d, uint32_t c)
 {
-    return h.re.x * r.re.x * t.re.x + h.im.x * r.re.x * t.im.x + h.re.x * r.im.x * t.im.x - h.im.x * r.im.x * t.re.x +
-           h.re.y * r.re.y * t.re.y + h.im.y * r.re.y * t.im.y + h.re.y * r.im.y * t.im.y - h.im.y * r.im.y * t.re.y;
+    const float2 a = *reinterpret_cast<const float2*>(row + 2 * c);
+    const float2 b = *reinterpret_cast<const float2*>(row + d + 2 * c);
+    CX<T> x;
+    x.re[0] = (T)a.x; x.re[1] = (T)a.y; x.im[0] = (T)b.x; x.im[1] = (T)b.y;
+    return x;
+}
+__device__ __forceinline__ void cx_store(float* row, uint32_t d, uint32_t c, float r0, float r1, float i0, float i1)
+{
+    *reinterpret_cast<float2*>(row + 2 * c) = make_float2(r0, r1);
+    *reinterpret_cast<float2*>(row + d + 2 * c) = make_float2(i0, i1);
+}
+
+template <class T>
+__device__ __forceinline__ T cx_score(const CX<T>& h, const CX<T>& r, const CX<T>& t)
+{
+    T s = T(0);
+#pragma unroll
+    for (int k = 0; k < 2; ++k)
+        s += h.re[k] * r.re[k] * t.re[k] + h.im[k] * r.re[k] * t.im[k] + h.re[k] * r.im[k] * t.im[k] - h.im[k] * r.im[k] * t.re[k];
+    return s;
 }
 
 // g_h += coef * d(phi)/d(h), likewise for r and t (any of the three may be skipped).  Differences of
 // products are formed without fused multiply-add, so that a gradient that cancels exactly
 // (head == tail) is exactly zero here too.
-__device__ __forceinline__ void c2_grads(const C2& h, const C2& r, const C2& t, float coef, C2* gh, C2* gr, C2* gt)
+template <class T>
+__device__ __forceinline__ void cx_grads(const CX<T>& h, const CX<T>& r, const CX<T>& t, T coef, CX<T>* gh, CX<T>* gr, CX<T>* gt)
 {
-#define NUPS_C1(comp)                                                                                     \
-    {                                                                                                     \
-        const float hr = h.re.comp, hi = h.im.comp, rr = r.re.comp, ri = r.im.comp;                       \
-        const float tr = t.re.comp, ti = t.im.comp;                                                       \
-        if (gh) { gh->re.comp += coef * (rr * tr + ri * ti);                                              \
-                  gh->im.comp += coef * __fsub_rn(__fmul_rn(rr, ti), __fmul_rn(ri, tr)); }                \
-        if (gt) { gt->re.comp += coef * __fsub_rn(__fmul_rn(hr, rr), __fmul_rn(hi, ri));                  \
-                  gt->im.comp += coef * (hi * rr + hr * ri); }                                            \
-        if (gr) { gr->re.comp += coef * (hr * tr + hi * ti);                                              \
-                  gr->im.comp += coef * __fsub_rn(__fmul_rn(hr, ti), __fmul_rn(hi, tr)); }                \
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        const T hr = h.re[k], hi = h.im[k], rr = r.re[k], ri = r.im[k], tr = t.re[k], ti = t.im[k];
+        if (gh) { gh->re[k] += coef * (rr * tr + ri * ti); gh->im[k] += coef * sub_rn(mul_rn(rr, ti), mul_rn(ri, tr)); }
+        if (gt) { gt->re[k] += coef * sub_rn(mul_rn(hr, rr), mul_rn(hi, ri)); gt->im[k] += coef * (hi * rr + hr * ri); }
+        if (gr) { gr->re[k] += coef * (hr * tr + hi * ti); gr->im[k] += coef * sub_rn(mul_rn(hr, ti), mul_rn(hi, tr)); }
     }
-    NUPS_C1(x)
-    NUPS_C1(y)
-#undef NUPS_C1
 }
 
-// step = -lr * g / (sqrt(a + g^2) + eps) with the hardware's reciprocal square root (2 ulp)
+// step = -lr * g / (sqrt(a + g^2) + eps).  Single precision (fast mode): the hardware's reciprocal square
+// root and approximate division (2 ulp each).  Double precision (deterministic mode): IEEE sqrt and division.
 __device__ __forceinline__ float adagrad_step(float g, float g2, float a, float lr, float eps)
 {
     const float y = a + g2;
     const float root = y > 0.f ? y * rsqrtf(y) : 0.f;
     return __fdividef(-lr * g, root + eps);
 }
-
-// AdaGrad update of one key role from the thread's part of its summed gradient:
-// acc += g^2, val -= lr g / (sqrt(acc_pulled + g^2) + eps)
-template <bool DET>
-__device__ __forceinline__ void c2_adagrad_push(const View& v, const C2& g, const C2& a, unsigned long long row,
-                                                unsigned long long pend, uint32_t d2, uint32_t c, float lr, float eps,
-                                                float* uval_row, float* uacc_row)
+__device__ __forceinline__ double adagrad_step(double g, double g2, double a, double lr, double eps)
 {
-    const float2 g2r = make_float2(g.re.x * g.re.x, g.re.y * g.re.y);
-    const float2 g2i = make_float2(g.im.x * g.im.x, g.im.y * g.im.y);
-    const float2 dvr = make_float2(adagrad_step(g.re.x, g2r.x, a.re.x, lr, eps), adagrad_step(g.re.y, g2r.y, a.re.y, lr, eps));
-    const float2 dvi = make_float2(adagrad_step(g.im.x, g2i.x, a.im.x, lr, eps), adagrad_step(g.im.y, g2i.y, a.im.y, lr, eps));
-    if (DET) {
-        float2* ov = (float2*)uval_row;
-        float2* oa = (float2*)uacc_row;
-        ov[c] = dvr; ov[d2 + c] = dvi; oa[c] = g2r; oa[d2 + c] = g2i;
-    } else {
-        float* ov = pend != NO_PEND ? v.dval + pend : v.val + row;
-        float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + row;
-        red_add_v2(ov + 2 * c, dvr); red_add_v2(ov + 2 * (d2 + c), dvi);
-        red_add_v2(oa + 2 * c, g2r); red_add_v2(oa + 2 * (d2 + c), g2i);
-    }
+    return -lr * g / (sqrt(a + g2) + eps);
 }
 
-// the thread's part (re.x, re.y, im.x, im.y) of a parked row, plus the worker's pending replica updates
-__device__ __forceinline__ C2 c2_parked(const float4* park, uint32_t slot_idx, uint32_t tid, const float* slab,
-                                        unsigned long long pend, uint32_t d2)
+// AdaGrad update of one key role from the thread's part of its summed gradient: the update rows
+// (value: -lr g / (sqrt(acc_pulled + g^2) + eps), accumulator: g^2) replace the role's staged rows
+template <class T>
+__device__ __forceinline__ void cx_adagrad(const CX<T>& g, float* val_row, float* acc_row, uint32_t d, uint32_t c, T lr, T eps)
 {
-    const float4 p = park[slot_idx * CPX_THREADS + tid];
-    C2 x;
-    x.re = make_float2(p.x, p.y);
-    x.im = make_float2(p.z, p.w);
-    if (pend != NO_PEND) {
-        const float2* s = (const float2*)(slab + pend);
-        const float2 a = s[tid], b = s[d2 + tid];
-        x.re.x += a.x; x.re.y += a.y; x.im.x += b.x; x.im.y += b.y;
-    }
+    const CX<T> a = cx_load<T>(acc_row, d, c);
+    const T r0 = g.re[0] * g.re[0], r1 = g.re[1] * g.re[1], i0 = g.im[0] * g.im[0], i1 = g.im[1] * g.im[1];
+    cx_store(val_row, d, c, (float)adagrad_step(g.re[0], r0, a.re[0], lr, eps), (float)adagrad_step(g.re[1], r1, a.re[1], lr, eps),
+             (float)adagrad_step(g.im[0], i0, a.im[0], lr, eps), (float)adagrad_step(g.im[1], i1, a.im[1], lr, eps));
+    cx_store(acc_row, d, c, (float)r0, (float)r1, (float)i0, (float)i1);
+}
+
+template <class T>
+__device__ __forceinline__ T warp_sum_t(T x)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
     return x;
 }
 
-__device__ __forceinline__ void cp_async_8(void* smem_dst, const void* gmem_src)
+// Sixteen sums over the warp at once: every lane brings v[0..15]; every lane returns the warp's total of
+// entry (lane >> 1) & 15.  Each step halves what a lane holds: the lane keeps the half its bit selects and
+// hands the other half to its partner (8 + 4 + 2 + 1 shuffles, one more for the last pair of lanes).
+template <class T>
+__device__ __forceinline__ T warp_sum16(T (&v)[CPX_NS], unsigned lane)
 {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
-                 : "memory");
+#pragma unroll
+    for (int half = CPX_NS / 2, bit = 16; half >= 1; half >>= 1, bit >>= 1) {
+        const bool upper = (lane & bit) != 0;
+#pragma unroll
+        for (int k = 0; k < half; ++k) {
+            const T send = upper ? v[k] : v[k + half];
+            const T keep = upper ? v[k + half] : v[k];
+            v[k] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, bit);
+        }
+    }
+    return v[0] + __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
 }
 
-template <bool HOT, bool DET>
+__device__ __forceinline__ float clampT(float x) { return clamp30(x); }
+__device__ __forceinline__ double clampT(double x) { return fmin(30.0, fmax(-30.0, x)); }
+__device__ __forceinline__ float sigmoidT(float x) { return sigmoidf_(x); }
+__device__ __forceinline__ double sigmoidT(double x) { return 1.0 / (1.0 + exp(-x)); }
+__device__ __forceinline__ float softplusT(float x) { return softplusf_(x); }
+__device__ __forceinline__ double softplusT(double x) { return fmax(x, 0.0) + log1p(exp(-fabs(x))); }
+
+template <bool HOT, bool DET, bool RED16>
 __global__ void __launch_bounds__(CPX_THREADS, 4)
 complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restrict__ rk, const uint32_t* __restrict__ tk,
                const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float eps, float* __restrict__ uval,
                float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
                float* __restrict__ loss_out)
 {
-    // park[2 * role][tid] = the thread's part of the role's value row, park[2 * role + 1][tid] = of its
-    // accumulator row; filled by asynchronous copies, all 2 * (3 + K) rows of a triple in flight at once
-    extern __shared__ __align__(16) float4 park[];
+    using T = typename std::conditional<DET, double, float>::type;
+    // rows[2 * role] = the role's value row, rows[2 * role + 1] = its accumulator row, as they lie in memory
+    extern __shared__ __align__(16) float rows[];
     __shared__ unsigned long long s_row[CPX_MAX_KEYS], s_pend[CPX_MAX_KEYS];
-    __shared__ float s_part[CPX_THREADS / 32][32];                 // per-warp partial scores
-    __shared__ int s_ok;
+    __shared__ T s_part[CPX_THREADS / 32][32];                     // per-warp sums of the scores
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t d2 = v.L4, per = K + 3;                         // d/2 component pairs = L/4
+    const uint32_t L4 = v.L4, d2 = v.L4, per = K + 3;              // d/2 component pairs = L/4
     const bool mine = tid < d2;                                    // threads beyond the row width only help reduce
-    const uint64_t L = (uint64_t)v.L4 * 4;
+    const uint32_t L = L4 * 4, d = L / 2;
+    const T lrT = (T)lr, epsT = (T)eps;
     double my_loss = 0.0;
+    s_part[warp][lane] = T(0);
     for (uint64_t i = blockIdx.x; i < n; i += gridDim.x) {
         const uint32_t q = worker_of_item(i, n, v.R);
         // thread j < 3 + K looks up role j: head, relation, tail, negatives
-        if (tid == 0) s_ok = 1;
-        __syncthreads();
         uint32_t key = 0;
-        int slot = -1;
-        if (tid < per) {
-            key = tid == 0 ? hk[i] : tid == 1 ? rk[i] : tid == 2 ? tk[i] : negs[i * K + tid - 3];
-            const bool ok = key < v.num_keys;
-            if (!ok) s_ok = 0;
-            slot = (HOT && ok) ? __ldg(v.slot_of + key) : -1;
-            if (slot < 0) slot = -1;
-            s_row[tid] = (unsigned long long)key * L;
-            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : NO_PEND;
-        }
-        __syncthreads();
-        if (!s_ok) {                                               // a key out of range: the whole item is skipped
+        if (tid < per) key = tid == 0 ? hk[i] : tid == 1 ? rk[i] : tid == 2 ? tk[i] : negs[i * K + tid - 3];
+        // one decision for the whole block (the barrier also ends the previous triple's use of the rows)
+        const int ok = __syncthreads_and(tid >= per || key < v.num_keys);
+        if (!ok) {                                                 // a key out of range: the whole item is skipped
             if (DET && tid < per) ukeys[i * per + tid] = NUPS_INVALID_KEY;
             if (tid == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
             continue;
         }
         if (tid < per) {
+            int slot = HOT ? __ldg(v.slot_of + key) : -1;
+            if (slot < 0) slot = -1;
+            s_row[tid] = (unsigned long long)key * L;
+            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : NO_PEND;
             if (DET) ukeys[i * per + tid] = key;
             if (!DET && slot >= 0) mark_dirty(v, q, slot);
             if (v.count) {
@@ -442,22 +467,20 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             }
             if (v.own && tid < 3) mark_localize(v, key, q);
         }
-        if (mine) {
+        __syncthreads();
+        if (tid < L4) {
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rows) + 16 * tid;
             for (uint32_t role = 0; role < per; ++role) {
-                const float2* a = (const float2*)(v.val + s_row[role]);
-                const float2* b = (const float2*)(v.acc + s_row[role]);
-                float4* pv = park + (2 * role) * CPX_THREADS + tid;
-                float4* pa = park + (2 * role + 1) * CPX_THREADS + tid;
-                cp_async_8(pv, a + tid); cp_async_8((float2*)pv + 1, a + d2 + tid);
-                cp_async_8(pa, b + tid); cp_async_8((float2*)pa + 1, b + d2 + tid);
+                cp_async_16s(dst + (2 * role) * L * 4, v.val + s_row[role] + 4 * tid);
+                cp_async_16s(dst + (2 * role + 1) * L * 4, v.acc + s_row[role] + 4 * tid);
             }
-            asm volatile("cp.async.commit_group;\n cp.async.wait_group 0;" ::: "memory");
+            asm volatile("cp.async.commit_group;" ::: "memory");
         }
         // while this triple is worked on, the rows of the block's next triple start moving towards L2
         {
             const uint64_t nx = i + gridDim.x;
             if (nx < n) {
-                const uint32_t lines_per_row = (uint32_t)((L * 4 + 127) / 128);
+                const uint32_t lines_per_row = (L * 4 + 127) / 128;
                 for (uint32_t e = tid; e < per * lines_per_row; e += CPX_THREADS) {
                     const uint32_t role = e / lines_per_row, line = e % lines_per_row;
                     const uint32_t k = role == 0 ? hk[nx] : role == 1 ? rk[nx] : role == 2 ? tk[nx] : negs[nx * K + role - 3];
@@ -469,62 +492,101 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
                 }
             }
         }
-        C2 h = c2_zero(), r = c2_zero(), t = c2_zero();
-        if (mine) {
-            h = c2_parked(park, 0, tid, v.dval, s_pend[0], d2);
-            r = c2_parked(park, 2, tid, v.dval, s_pend[1], d2);
-            t = c2_parked(park, 4, tid, v.dval, s_pend[2], d2);
-        }
-        // pass 1: partial scores; lane j of each warp ends up holding the warp's sum of score j
-        float part = 0.f;
-        {
-            const float sc = warp_sum(mine ? c2_score(h, r, t) : 0.f);
-            if (lane == 0) part = sc;
-        }
-        for (uint32_t j = 0; j < K; ++j) {
-            float sc = 0.f;
-            if (mine) {
-                const C2 e = c2_parked(park, 2 * (3 + j), tid, v.dval, s_pend[3 + j], d2);
-                sc = (j & 1) == 0 ? c2_score(e, r, t) : c2_score(h, r, e);
+        if (tid < L4) {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            if (HOT) {
+                // the worker's pending replica updates join the chunks this thread staged
+                for (uint32_t role = 0; role < per; ++role) {
+                    const unsigned long long pend = s_pend[role];
+                    if (pend == NO_PEND) continue;
+                    float4* pv = reinterpret_cast<float4*>(rows + (size_t)(2 * role) * L) + tid;
+                    float4* pa = reinterpret_cast<float4*>(rows + (size_t)(2 * role + 1) * L) + tid;
+                    *pv = add4(*pv, *(reinterpret_cast<const float4*>(v.dval + pend) + tid));
+                    *pa = add4(*pa, *(reinterpret_cast<const float4*>(v.dacc + pend) + tid));
+                }
             }
-            sc = warp_sum(sc);
-            if (lane == j + 1) part = sc;
         }
-        s_part[warp][lane] = part;
+        __syncthreads();
+        auto val_row = [&](uint32_t role) { return rows + (size_t)(2 * role) * L; };
+        auto acc_row = [&](uint32_t role) { return rows + (size_t)(2 * role + 1) * L; };
+        CX<T> h = cx_zero<T>(), r = cx_zero<T>(), t = cx_zero<T>();
+        if (mine) { h = cx_load<T>(val_row(0), d, tid); r = cx_load<T>(val_row(1), d, tid); t = cx_load<T>(val_row(2), d, tid); }
+        // pass 1: the thread's part of every score; lane j < 32 of each warp ends up with the warp's sum of score j
+        if (RED16) {
+            T sc[CPX_NS];
+            sc[0] = mine ? cx_score(h, r, t) : T(0);
+#pragma unroll
+            for (int j = 0; j < CPX_NS - 1; ++j) {
+                sc[j + 1] = T(0);
+                if ((uint32_t)j < K && mine) {
+                    const CX<T> e = cx_load<T>(val_row(3 + j), d, tid);
+                    sc[j + 1] = (j & 1) == 0 ? cx_score(e, r, t) : cx_score(h, r, e);
+                }
+            }
+            const T tot = warp_sum16(sc, lane);
+            if ((lane & 1u) == 0) s_part[warp][lane >> 1] = tot;
+        } else {
+            T part = T(0);
+            {
+                const T sc = warp_sum_t(mine ? cx_score(h, r, t) : T(0));
+                if (lane == 0) part = sc;
+            }
+            for (uint32_t j = 0; j < K; ++j) {
+                T sc = T(0);
+                if (mine) {
+                    const CX<T> e = cx_load<T>(val_row(3 + j), d, tid);
+                    sc = (j & 1) == 0 ? cx_score(e, r, t) : cx_score(h, r, e);
+                }
+                sc = warp_sum_t(sc);
+                if (lane == j + 1) part = sc;
+            }
+            s_part[warp][lane] = part;
+        }
         __syncthreads();
         // every thread needs every score: lane j adds the warps' sums of score j, then they are passed around
-        float phi_l = 0.f;
+        T phi_l = T(0);
 #pragma unroll
         for (int w = 0; w < CPX_THREADS / 32; ++w) phi_l += s_part[w][lane];
-        phi_l = clamp30(phi_l);
-        const float coef_l = lane == 0 ? sigmoidf_(phi_l) - 1.f : sigmoidf_(phi_l);
-        float loss_l = lane == 0 ? softplusf_(-phi_l) : (lane <= K ? softplusf_(phi_l) : 0.f);
-        loss_l = warp_sum(loss_l);
-        // pass 2: gradients and updates
-        C2 gh = c2_zero(), gr = c2_zero(), gt = c2_zero();
-        c2_grads(h, r, t, __shfl_sync(0xFFFFFFFFu, coef_l, 0), &gh, &gr, &gt);
+        phi_l = clampT(phi_l);
+        const T coef_l = lane == 0 ? sigmoidT(phi_l) - T(1) : sigmoidT(phi_l);
+        T loss_l = lane == 0 ? softplusT(-phi_l) : (lane <= K ? softplusT(phi_l) : T(0));
+        loss_l = warp_sum_t(loss_l);
+        // pass 2: gradients; each role's update rows replace its staged rows
+        CX<T> gh = cx_zero<T>(), gr = cx_zero<T>(), gt = cx_zero<T>();
+        cx_grads(h, r, t, __shfl_sync(0xFFFFFFFFu, coef_l, 0), &gh, &gr, &gt);
         for (uint32_t j = 0; j < K; ++j) {
-            const float coef = __shfl_sync(0xFFFFFFFFu, coef_l, j + 1);
+            const T coef = __shfl_sync(0xFFFFFFFFu, coef_l, j + 1);
             if (!mine) continue;
-            const C2 e = c2_parked(park, 2 * (3 + j), tid, v.dval, s_pend[3 + j], d2);
-            C2 ge = c2_zero();
-            if ((j & 1) == 0) c2_grads(e, r, t, coef, &ge, &gr, &gt);
-            else c2_grads(h, r, e, coef, &gh, &gr, &ge);
-            const C2 a = c2_parked(park, 2 * (3 + j) + 1, tid, v.dacc, s_pend[3 + j], d2);
-            c2_adagrad_push<DET>(v, ge, a, s_row[3 + j], s_pend[3 + j], d2, tid, lr, eps,
-                                 DET ? uval + (i * per + 3 + j) * L : nullptr, DET ? uacc + (i * per + 3 + j) * L : nullptr);
+            const CX<T> e = cx_load<T>(val_row(3 + j), d, tid);
+            CX<T> ge = cx_zero<T>();
+            if ((j & 1) == 0) cx_grads(e, r, t, coef, &ge, &gr, &gt);
+            else cx_grads(h, r, e, coef, &gh, &gr, &ge);
+            cx_adagrad(ge, val_row(3 + j), acc_row(3 + j), d, tid, lrT, epsT);
         }
         if (mine) {
-            const C2* g3[3] = {&gh, &gr, &gt};
-#pragma unroll
-            for (int role = 0; role < 3; ++role) {
-                const C2 a = c2_parked(park, 2 * role + 1, tid, v.dacc, s_pend[role], d2);
-                c2_adagrad_push<DET>(v, *g3[role], a, s_row[role], s_pend[role], d2, tid, lr, eps,
-                                     DET ? uval + (i * per + role) * L : nullptr, DET ? uacc + (i * per + role) * L : nullptr);
+            cx_adagrad(gh, val_row(0), acc_row(0), d, tid, lrT, epsT);
+            cx_adagrad(gr, val_row(1), acc_row(1), d, tid, lrT, epsT);
+            cx_adagrad(gt, val_row(2), acc_row(2), d, tid, lrT, epsT);
+        }
+        __syncthreads();
+        if (tid < L4) {
+            for (uint32_t role = 0; role < per; ++role) {
+                const float4 dv = reinterpret_cast<const float4*>(val_row(role))[tid];
+                const float4 da = reinterpret_cast<const float4*>(acc_row(role))[tid];
+                if (DET) {
+                    reinterpret_cast<float4*>(uval + (i * per + role) * (uint64_t)L)[tid] = dv;
+                    reinterpret_cast<float4*>(uacc + (i * per + role) * (uint64_t)L)[tid] = da;
+                } else {
+                    const unsigned long long pend = s_pend[role];
+                    float* ov = pend != NO_PEND ? v.dval + pend : v.val + s_row[role];
+                    float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + s_row[role];
+                    red_add_v4(ov + 4 * tid, dv);
+                    red_add_v4(oa + 4 * tid, da);
+                }
             }
         }
         if (tid == 0) {
-            if (DET) loss_item[i] = loss_l;
+            if (DET) loss_item[i] = (float)loss_l;
             my_loss += (double)loss_l;
         }
     }
@@ -864,7 +926,7 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
             if (fit >= 1 && (unsigned)fit < per_sm) per_sm = (unsigned)fit;                                            \
             const uint64_t cap = (uint64_t)s->sm_count * per_sm;                                                       \
             const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);                               \
-            nups_time_begin(s, st);                                                                                    \
+            nups_time_begin(s, st, NUPS_TIMED_STEP);                                                                                    \
             kern<<<grid, 32 * SGNS_WARPS, smem, st>>>(v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
                                                       b.loss_item, d_loss_out, group,                                  \
                                                       loss_acc, b.clip_item);                                          \
@@ -1005,28 +1067,33 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     rc = step_buffers(s, n, K + 3, true, &b);
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
-    // shared memory: one 16-byte column entry per thread for the value and the accumulator row of every role
-    const size_t smem = (size_t)2 * (K + 3) * CPX_THREADS * sizeof(float4);
+    // shared memory: the value and the accumulator row of every role
+    const size_t smem = (size_t)2 * (K + 3) * s->L * sizeof(float);
     if (smem > (size_t)s->max_smem - 4096) return NUPS_EINVAL;
     unsigned per_sm = (unsigned)(((size_t)s->max_smem - 1024) / (smem + 2048));
     if (per_sm > 4) per_sm = 4;
     if (per_sm < 1) per_sm = 1;
     uint64_t want = n < (uint64_t)s->sm_count * per_sm ? n : (uint64_t)s->sm_count * per_sm;
     unsigned grid = (unsigned)want;
-    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0;
-    if (!s->complex_smem_opted[hi][di]) {
-        cudaError_t e;
-        if (hi && di) e = cudaFuncSetAttribute(complex_kernel<true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else if (hi) e = cudaFuncSetAttribute(complex_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else if (di) e = cudaFuncSetAttribute(complex_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        else e = cudaFuncSetAttribute(complex_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);
-        if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
-        s->complex_smem_opted[hi][di] = true;
-    }
-    nups_time_begin(s, st);
-    DISPATCH_MODE(s, complex_kernel<HOT, DET><<<grid, CPX_THREADS, smem, st>>>(
-        v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, b.ukeys, b.loss_item, d_loss_out));
+    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0, ri = K + 1 <= (uint32_t)CPX_NS ? 1 : 0;
+    cudaError_t e = cudaSuccess;
+    nups_time_begin(s, st, NUPS_TIMED_STEP);
+#define NUPS_CPX_GO(RED16_)                                                                                          \
+    DISPATCH_MODE(s, {                                                                                               \
+        auto kern = complex_kernel<HOT, DET, RED16_>;                                                                \
+        if (!s->complex_smem_opted[hi][di][ri]) {                                                                    \
+            e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);         \
+            s->complex_smem_opted[hi][di][ri] = (e == cudaSuccess);                                                  \
+        }                                                                                                            \
+        if (e == cudaSuccess)                                                                                        \
+            kern<<<grid, CPX_THREADS, smem, st>>>(v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc,     \
+                                                  b.ukeys, b.loss_item, d_loss_out);                                 \
+    })
+    if (ri) NUPS_CPX_GO(true);
+    else NUPS_CPX_GO(false);
+#undef NUPS_CPX_GO
     nups_time_end(s, st);
+    if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
     LAUNCH_CHECK(s);
     return step_finish(s, n, K + 3, b, d_loss_out, st, !s->cfg.deterministic);
 }
@@ -1238,7 +1305,7 @@ static nups_status mf_step(nups_store* s, const uint32_t* d_row, const uint32_t*
     if (rc != NUPS_OK) return rc;
     View v = nups_view(s);
     const bool by_column = cells_by_column && !s->cfg.deterministic;    // the ordered mode is the same for any order
-    nups_time_begin(s, st);
+    nups_time_begin(s, st, NUPS_TIMED_STEP);
     if (by_column) {
         const unsigned grid = step_grid(s, n, MF_RUN_BLOCKS);
         DISPATCH_CLIP(s, DISPATCH_CH(v.L4, {

@@ -86,18 +86,20 @@ static void timing_fold(nups_store* s)
 {
     for (uint32_t i = 0; i < s->ev_n; ++i) {
         float ms = 0.f;
+        const int kind = s->ev_kind[i];
         if (cudaEventSynchronize(s->ev[2 * i + 1]) == cudaSuccess &&
             cudaEventElapsedTime(&ms, s->ev[2 * i], s->ev[2 * i + 1]) == cudaSuccess)
-            s->ev_ms += ms;
+            s->ev_ms[kind] += ms;
+        s->ev_launches[kind]++;
     }
-    s->ev_launches += s->ev_n;
     s->ev_n = 0;
     cudaGetLastError();
 }
-void nups_time_begin(nups_store* s, cudaStream_t st)
+void nups_time_begin(nups_store* s, cudaStream_t st, int kind)
 {
     if (!s->timing) return;
     if (s->ev_n == NUPS_MAX_TIMED) timing_fold(s);
+    s->ev_kind[s->ev_n] = (unsigned char)kind;
     cudaEventRecord(s->ev[2 * s->ev_n], st);
 }
 void nups_time_end(nups_store* s, cudaStream_t st)
@@ -106,26 +108,42 @@ void nups_time_end(nups_store* s, cudaStream_t st)
     cudaEventRecord(s->ev[2 * s->ev_n + 1], st);
     s->ev_n++;
 }
+static void timing_clear(nups_store* s)
+{
+    for (int k = 0; k < NUPS_TIMED_KINDS; ++k) { s->ev_ms[k] = 0; s->ev_launches[k] = 0; }
+}
 extern "C" nups_status nups_kernel_timing(nups_store* s, int enable)
 {
     if (!s) return NUPS_EINVAL;
     if (enable && !s->ev) {
         s->ev = (cudaEvent_t*)calloc(2 * NUPS_MAX_TIMED, sizeof(cudaEvent_t));
-        if (!s->ev) return NUPS_ENOMEM;
+        s->ev_kind = (unsigned char*)calloc(NUPS_MAX_TIMED, 1);
+        if (!s->ev || !s->ev_kind) return NUPS_ENOMEM;
         for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) CK(cudaEventCreate(&s->ev[i]));
     }
     if (s->ev) timing_fold(s);
-    s->ev_ms = 0; s->ev_launches = 0;
+    timing_clear(s);
     s->timing = enable ? 1 : 0;
+    return NUPS_OK;
+}
+extern "C" nups_status nups_kernel_times(nups_store* s, double* h_ms_out, uint64_t* h_launches_out, void* stream)
+{
+    if (!s || !h_ms_out || !h_launches_out) return NUPS_EINVAL;
+    CK(cudaStreamSynchronize((cudaStream_t)stream));
+    if (s->ev) timing_fold(s);
+    for (int k = 0; k < NUPS_TIMED_KINDS; ++k) { h_ms_out[k] = s->ev_ms[k]; h_launches_out[k] = s->ev_launches[k]; }
+    timing_clear(s);
     return NUPS_OK;
 }
 extern "C" nups_status nups_kernel_time(nups_store* s, double* h_ms_out, uint64_t* h_launches_out, void* stream)
 {
     if (!s || !h_ms_out || !h_launches_out) return NUPS_EINVAL;
-    CK(cudaStreamSynchronize((cudaStream_t)stream));
-    if (s->ev) timing_fold(s);
-    *h_ms_out = s->ev_ms; *h_launches_out = s->ev_launches;
-    s->ev_ms = 0; s->ev_launches = 0;
+    double ms[NUPS_TIMED_KINDS];
+    uint64_t n[NUPS_TIMED_KINDS];
+    nups_status rc = nups_kernel_times(s, ms, n, stream);
+    if (rc != NUPS_OK) return rc;
+    *h_ms_out = 0; *h_launches_out = 0;
+    for (int k = 0; k < NUPS_TIMED_KINDS; ++k) { *h_ms_out += ms[k]; *h_launches_out += n[k]; }
     return NUPS_OK;
 }
 
@@ -220,6 +238,7 @@ extern "C" nups_status nups_destroy(nups_store* s)
     if (s->ev) {
         for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) cudaEventDestroy(s->ev[i]);
         free(s->ev);
+        free(s->ev_kind);
     }
     cudaGetLastError();
     free(s);
@@ -482,7 +501,7 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
         (uint64_t)s->R * s->Hcap < 0xFFFFFFFFull) {
         const float* table = (const float*)A.table;
         const float* slab = (const float*)A.slab;
-        nups_time_begin(s, st);
+        nups_time_begin(s, st, worker_map == 1 ? NUPS_TIMED_SAMPLE_ROWS : NUPS_TIMED_PULL);
 #define NUPS_G8(C8_)                                                                                                     \
         gather8_kernel<true, C8_><<<grid, 256, 0, st>>>(v, d_keys, n, table, slab, out1, worker_map, map_base, map_total, \
                                                         do_count, d_keys_copy)
@@ -494,7 +513,7 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
         LAUNCH_CHECK(s);
         return NUPS_OK;
     }
-    nups_time_begin(s, st);
+    nups_time_begin(s, st, worker_map == 1 ? NUPS_TIMED_SAMPLE_ROWS : NUPS_TIMED_PULL);
     if (s->H) {
         if (two) gather_kernel<true, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
         else gather_kernel<true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
@@ -902,7 +921,7 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
                 s->push_smem_opted = true;
             }
         }
-        nups_time_begin(s, st);
+        nups_time_begin(s, st, NUPS_TIMED_PUSH);
         if (tier_rows && cache) {
             push_atomic_kernel<false, false, 2><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);

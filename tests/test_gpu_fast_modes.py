@@ -1,0 +1,241 @@
+"""CUDA path vs oracle in fast (atomic, replicated, asynchronous) mode, for the ComplEx and matrix-factorization
+steps: the loss after the same number of epochs within 1 % of the oracle's on a run whose loss really moves, and
+one-step comparisons of every key's total update on batches whose items cannot race."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import CONFORM, REPLICATE
+from paper_2104_00501_b200 import inputs
+from tests.common import ATOL, RTOL, dev_f32, dev_keys, host_keys, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+MF_TWIN_LR = 0.02
+
+
+def loss_buf():
+    return torch.zeros(1, dtype=torch.float32, device="cuda")
+
+
+def test_complex_fast_mode_reaches_the_oracles_loss_within_one_percent():
+    # replicated + asynchronous mode: relations and frequent entities replicated over 8 workers, merged every 4
+    # batches; three epochs; the oracle's loss falls by more than a fifth, the CUDA path ends within 1 % of it,
+    # draws the same negatives and counts the same accesses
+    E, Rl, L, K, R, batch, n = 2000, 20, 64, 10, 8, 256, 4096
+    h, r, t = [inputs.u32(x) for x in inputs.kge_triples(n, E, Rl, 0.9, 1.2, 0)]
+    init = np.random.default_rng(0).normal(0, 0.1, size=(E + Rl, L)).astype(np.float32)
+    o, s = make_pair(E + Rl, L, R=R, init=init, deterministic=False, with_adagrad=True, sync_interval=4,
+                     count_accesses=True)
+    hot = np.concatenate([np.arange(E, E + Rl), np.unique(h)[:30]]).astype(np.uint32)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(0, None, E, CONFORM, seed=9)
+    ds = s.register_distribution(0, None, E, CONFORM, seed=9)
+    lb = loss_buf()
+    lo_hist, ls_hist = [], []
+    nb = n // batch
+    dh, dr, dt = dev_keys(h), dev_keys(r), dev_keys(t)
+    for epoch in range(3):
+        for b in range(nb):
+            sl = slice(b * batch, (b + 1) * batch)
+            lo, negs = o.step_complex(h[sl], r[sl], t[sl], do, K, 0.04, 1e-10, return_negatives=True)
+            s.step_complex(dh[sl], dr[sl], dt[sl], ds, K, 0.04, 1e-10, lb)
+            assert np.array_equal(host_keys(s.last_negatives()), negs)
+            lo_hist.append(lo)
+            ls_hist.append(lb.item())
+    lo, ls = np.mean(lo_hist[-nb:]), np.mean(ls_hist[-nb:])
+    assert lo < 0.8 * np.mean(lo_hist[:4])                              # the run learns something
+    assert abs(ls - lo) <= 0.01 * lo
+    o.sync()
+    s.sync()
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+    # squared gradients only ever grow the accumulators, and by about as much in total
+    acc_s, acc_o = s.read_table(1).cpu().numpy().astype(np.float64), o.table(1).astype(np.float64)
+    assert acc_s.min() >= 0.0 and abs(acc_s.sum() - acc_o.sum()) <= 0.05 * acc_o.sum()
+    assert s.status_check() == 0
+
+
+@pytest.mark.parametrize("L,hot_n,acc0", [(500, 40, 0.1), (64, 0, 0.1), (500, 40, 0.0)])
+def test_complex_fast_mode_one_step_matches_the_oracle_where_items_cannot_race(L, hot_n, acc0):
+    # One batch from the same start.  Every triple has its own head, relation and tail; a triple whose sampled
+    # negatives touch no key of another triple shares no row with anybody, so nothing can race and the fast kernel's
+    # result for its keys must be the oracle's: values within the stated tolerance, accumulators within the rounding
+    # of single-precision gradients.  With accumulators that start at zero the first AdaGrad step is lr long whatever
+    # the gradient's size, so there only components whose squared gradient is not vanishing are compared.
+    E, R, K, n = 100_000, 4, 10, 256
+    rng = np.random.default_rng(3)
+    perm = rng.permutation(E)[:2 * n].astype(np.uint32)
+    h, t = perm[:n], perm[n:]
+    r = (E + np.arange(n)).astype(np.uint32)
+    init = rng.standard_normal(size=(E + n, L), dtype=np.float32) * np.float32(0.1)
+    acc_init = np.float32(acc0) * (1 + rng.random(size=(E + n, L), dtype=np.float32)) if acc0 else None
+    o, s = make_pair(E + n, L, R=R, init=init, acc_init=acc_init, deterministic=False, with_adagrad=True, sync_interval=1)
+    if hot_n:
+        hot = np.concatenate([r[:hot_n], h[:hot_n]]).astype(np.uint32)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(0, None, E, CONFORM, seed=5)
+    ds = s.register_distribution(0, None, E, CONFORM, seed=5)
+    lb = loss_buf()
+    lo, negs = o.step_complex(h, r, t, do, K, 0.1, 1e-10, return_negatives=True)
+    s.step_complex(dev_keys(h), dev_keys(r), dev_keys(t), ds, K, 0.1, 1e-10, lb)
+    assert np.array_equal(host_keys(s.last_negatives()), negs)
+    assert abs(lb.item() - lo) <= 2e-5 * abs(lo)
+    negs = negs.reshape(n, K)
+    uses = np.bincount(np.concatenate([h, t, negs.ravel()]), minlength=E)
+    alone = (uses[negs] == 1).all(axis=1) & (uses[h] == 1) & (uses[t] == 1)    # no key of the triple is anybody else's
+    assert alone.mean() > 0.5
+    keys = np.concatenate([h[alone], r[alone], t[alone], negs[alone].ravel()])
+    idx = torch.from_numpy(keys.astype(np.int64)).cuda()
+    val_s, acc_s = s.read_table(0)[idx].cpu().numpy(), s.read_table(1)[idx].cpu().numpy()
+    val_o, acc_o = o.table(0)[keys], o.table(1)[keys]
+    np.testing.assert_allclose(acc_s, acc_o, rtol=1e-4, atol=1e-9)
+    if acc0:
+        np.testing.assert_allclose(val_s, val_o, rtol=RTOL, atol=ATOL)
+    else:
+        big = acc_o > 1e-8
+        np.testing.assert_allclose(val_s[big], val_o[big], rtol=RTOL, atol=ATOL)
+        assert big.mean() > 0.3
+    assert np.abs(val_o - init[keys]).max() > 1e-3
+    # every squared gradient of the batch arrives: the accumulators' total growth is the oracle's
+    start = acc_init.astype(np.float64).sum() if acc0 else 0.0
+    grow_s = s.read_table(1).sum(dtype=torch.float64).item() - start
+    grow_o = o.table(1).astype(np.float64).sum() - start
+    assert abs(grow_s - grow_o) <= 1e-3 * grow_o
+    assert s.status_check() == 0
+
+
+@pytest.mark.parametrize("deterministic", [True, False])
+def test_complex_skips_a_triple_with_a_key_out_of_range(deterministic):
+    # one triple in the middle of the batch has a head, relation or tail beyond the key space: the item is skipped
+    # as a whole (no update, no loss term), the others are untouched by it, and the status word says so
+    E, Rl, L, K, R, n = 300, 8, 64, 4, 2, 200
+    h, r, t = [inputs.u32(x) for x in inputs.kge_triples(n, E, Rl, 0.9, 1.2, 2)]
+    init = np.random.default_rng(2).normal(0, 0.1, size=(E + Rl, L)).astype(np.float32)
+    acc_init = np.full((E + Rl, L), 0.2, np.float32)
+    mid = n // 2
+    for role, bad in ((0, E + Rl), (1, 0xFFFFFFF0), (2, E + Rl + 77)):
+        hh, rr, tt = h.copy(), r.copy(), t.copy()
+        (hh, rr, tt)[role][mid] = bad
+        o, s = make_pair(E + Rl, L, R=R, init=init, acc_init=acc_init, deterministic=deterministic, with_adagrad=True)
+        hot = np.array([E, E + 1, int(h[0])], np.uint32)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+        do = o.register_distribution(0, None, E, CONFORM, seed=1)
+        ds = s.register_distribution(0, None, E, CONFORM, seed=1)
+        lb = loss_buf()
+        lo = o.step_complex(hh, rr, tt, do, K, 0.05, 1e-10)
+        s.step_complex(dev_keys(hh), dev_keys(rr), dev_keys(tt), ds, K, 0.05, 1e-10, lb)
+        assert abs(lb.item() - lo) <= (1e-5 if deterministic else 1e-3) * abs(lo)
+        assert s.status_check() == -4
+        o.sync()
+        s.sync()
+        got, want = s.read_table(0).cpu().numpy(), o.table(0)
+        if deterministic:
+            np.testing.assert_allclose(got, want, rtol=RTOL, atol=ATOL)
+            np.testing.assert_allclose(s.read_table(1).cpu().numpy(), o.table(1), rtol=RTOL, atol=ATOL)
+        else:
+            # items race on shared rows in fast mode: every key's total update stays near the oracle's, and a key
+            # that the oracle leaves alone (for one, a key that only the skipped item uses) is left alone
+            d_s, d_o = got.astype(np.float64) - init, want.astype(np.float64) - init
+            norm = np.linalg.norm(d_o, axis=1)
+            assert np.all(np.linalg.norm(d_s - d_o, axis=1) <= 0.2 * norm + 1e-5)
+        s.close()
+
+
+def test_mf_fast_mode_reaches_the_oracles_loss_within_one_percent():
+    # plain fast mode (cells in any order, nups_step_mf), frequent keys replicated, merged every 4 batches
+    M, N, L, R, n, batch = 2000, 500, 32, 8, 8192, 512
+    i, j, x = inputs.mf_cells(n, M, N, 0.8, 8, 0.1, 0)
+    i, j, x = inputs.u32(i), inputs.u32(j), x.numpy()
+    init = np.random.default_rng(0).normal(0, 0.3, size=(M + N, L)).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, init=init, deterministic=False, sync_interval=4, count_accesses=True)
+    o.count_accesses(np.concatenate([i, j]))
+    s.count_accesses(dev_keys(np.concatenate([i, j])))
+    hot = o.select_hot(True, 30)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    lb = loss_buf()
+    lo_hist, ls_hist = [], []
+    nb = n // batch
+    di, dj, dx = dev_keys(i), dev_keys(j), dev_f32(x)
+    for epoch in range(4):
+        for b in range(nb):
+            sl = slice(b * batch, (b + 1) * batch)
+            lo_hist.append(o.step_mf(i[sl], j[sl], x[sl], MF_TWIN_LR, 0.01))
+            s.step_mf(di[sl], dj[sl], dx[sl], MF_TWIN_LR, 0.01, lb)
+            ls_hist.append(lb.item())
+    lo, ls = np.mean(lo_hist[-nb:]), np.mean(ls_hist[-nb:])
+    assert lo < 0.9 * np.mean(lo_hist[:4])
+    assert abs(ls - lo) <= 0.01 * lo
+    o.sync()
+    s.sync()
+    assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
+    assert s.status_check() == 0
+
+
+@pytest.mark.parametrize("L,hot_n", [(100, 0), (100, 64), (8, 16)])
+def test_mf_fast_mode_one_step_matches_the_oracle_where_cells_cannot_race(L, hot_n):
+    # cells that share no row key and no column key: nothing races, so the fast kernel (single precision) gives the
+    # oracle's result within the stated tolerance at a normal learning rate
+    M, N, R, n = 5000, 5000, 4, 4000
+    rng = np.random.default_rng(6)
+    i = rng.permutation(M)[:n].astype(np.uint32)
+    j = (M + rng.permutation(N)[:n]).astype(np.uint32)
+    x = rng.normal(0, 1, n).astype(np.float32)
+    init = rng.normal(0, 0.3, size=(M + N, L)).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, init=init, deterministic=False, sync_interval=1)
+    if hot_n:
+        hot = np.concatenate([i[:hot_n], j[hot_n:2 * hot_n]]).astype(np.uint32)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    lb = loss_buf()
+    lo = o.step_mf(i, j, x, 0.01, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), 0.01, 0.01, lb)
+    assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    np.testing.assert_allclose(s.read_table(0).cpu().numpy(), o.table(0), rtol=RTOL, atol=ATOL)
+    assert np.abs(o.table(0) - init).max() > 1e-3
+    assert s.status_check() == 0
+
+
+def _by_column_stretch(n):
+    """Cells per warp of nups_step_mf_by_column for a batch of n cells on the current device (the launch shape the
+    header states: 4 warps per block, 5 resident blocks per multiprocessor, every warp one contiguous stretch)."""
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    blocks = min(-(-n // 4), sms * 5, 8192)
+    warps = blocks * 4
+    return -(-n // warps), warps
+
+
+@pytest.mark.parametrize("L,hot_cols", [(100, 0), (100, 40), (8, 7)])
+def test_mf_by_column_matches_the_oracle_at_a_normal_learning_rate_where_cells_cannot_race(L, hot_cols):
+    # the by-column kernel keeps a column's row in registers over a stretch of cells and adds the column's summed
+    # update once.  Cells built so that the oracle's batch step is exactly what that computes: no two cells share a
+    # row key, every column has 16 cells and they lie inside one warp's stretch.  Learning rate 0.01.
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    per_col = 16
+    n = sms * 5 * 4 * per_col                                 # every warp gets exactly one column's cells
+    stretch, warps = _by_column_stretch(n)
+    assert stretch == per_col and warps * per_col == n
+    M, N, R = n, n // per_col, 4
+    rng = np.random.default_rng(8)
+    i = rng.permutation(M).astype(np.uint32)
+    j = (M + np.repeat(rng.permutation(N), per_col)).astype(np.uint32)
+    x = rng.normal(0, 1, n).astype(np.float32)
+    o, s = make_pair(M + N, L, R=R, deterministic=False, sync_interval=1)
+    o.init_uniform(0, 4, 0.3)
+    s.init_uniform(0, 4, 0.3)
+    if hot_cols:
+        hot = np.unique(j)[::max(1, N // hot_cols)][:hot_cols].astype(np.uint32)
+        o.set_management(hot, REPLICATE)
+        s.set_management(dev_keys(hot), REPLICATE)
+    start = o.table(0).copy()
+    lb = loss_buf()
+    lo = o.step_mf(i, j, x, 0.01, 0.01)
+    s.step_mf(dev_keys(i), dev_keys(j), dev_f32(x), 0.01, 0.01, lb, by_column=True)
+    assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
+    np.testing.assert_allclose(s.read_table(0).cpu().numpy(), o.table(0), rtol=RTOL, atol=ATOL)
+    assert np.abs(o.table(0) - start).max() > 1e-3
+    assert s.status_check() == 0

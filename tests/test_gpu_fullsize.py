@@ -48,24 +48,46 @@ def test_full_size_deterministic_steps_match_the_oracle():
     assert s.status_check() == 0
 
 
-def test_full_size_fast_mode_tracks_the_oracle_loss():
-    # replicated + asynchronous mode as the benchmark runs it: the loss after the same number of
-    # batches stays within 1 % of the oracle's, and the sampled keys are still the oracle's
-    steps = 48
+def test_full_size_fast_mode_applies_the_oracles_updates():
+    # replicated + asynchronous mode as the benchmark runs it (top 1 % of keys replicated over 8 workers, one merge
+    # after 16 batches).  At the benchmark's learning rate the loss hardly moves in so few batches, so the loss says
+    # nothing about the updates; what is compared instead is every touched row's TOTAL update over the 16 batches.
+    # In fast mode a pair may see what other pairs of its batch have already added, which the oracle's batch step
+    # never shows it; that changes a row's update by about the relative change of its partner rows within a batch.
+    # The oracle's rows move by at most 13.5 % over these 16 batches (the most frequent word; 2 % at the 99.9th
+    # percentile), i.e. about 1 % per batch, so 5 % of the update's norm bounds the difference for every row; the
+    # absolute term is 1 % of the smallest single update (8e-6).  A kernel that drops, doubles or misdirects updates
+    # (a role, a replica, a whole launch) lands far outside.
+    steps = bench.SYNC_EVERY
     s, dist, orc, d, c, o = _setup(False, steps)
     hc, ho = inputs.u32(c), inputs.u32(o)
+    start = orc.table().copy()
     lb = torch.zeros(steps, device="cuda")
-    lo = []
+    lo, touched = [], []
     for b in range(steps):
         sl = slice(b * B, (b + 1) * B)
         l, negs = orc.step_sgns(hc[sl], ho[sl], d, K, bench.LR, return_negatives=True)
         lo.append(l)
         s.step_sgns(c[sl], o[sl], dist, K, bench.LR, lb[b:b + 1])
-        if b % 7 == 0:
-            assert np.array_equal(host_keys(s.last_negatives()), negs)
+        assert np.array_equal(host_keys(s.last_negatives()), negs)
+        touched.append(np.concatenate([hc[sl], ho[sl], negs]))
+    assert s.stats()["syncs"] == 1 and orc.stats()["syncs"] == 1          # the merge after the 16th batch has run
+    rows = np.unique(np.concatenate(touched))
+    got = s.read_table()[torch.from_numpy(rows.astype(np.int64)).cuda()].cpu().numpy().astype(np.float64)
+    d_s, d_o = got - start[rows], orc.table()[rows].astype(np.float64) - start[rows]
+    norm = np.linalg.norm(d_o, axis=1)
+    err = np.linalg.norm(d_s - d_o, axis=1)
+    assert np.all(err <= 0.05 * norm + 1e-7), (err / (norm + 1e-30)).max()
+    assert norm.min() > 1e-6 and norm.max() > 1e-4                          # every touched row did move
+    rel = norm / np.linalg.norm(start[rows].astype(np.float64), axis=1)
+    assert rel.max() < 0.2                                                  # ... and by as little as the bound assumes
+    # untouched rows stay bit for bit what they were
+    rng = np.random.default_rng(1)
+    other = np.setdiff1d(rng.integers(0, 2 * V, 20000).astype(np.uint32), rows)
+    same = s.read_table()[torch.from_numpy(other.astype(np.int64)).cuda()].cpu().numpy()
+    assert np.array_equal(same, start[other])
     ls = lb.cpu().numpy()
-    assert abs(ls[-16:].mean() - np.mean(lo[-16:])) <= 0.01 * np.mean(lo[-16:])
-    assert np.all(np.isfinite(ls))
+    assert np.all(np.isfinite(ls)) and abs(ls.mean() - np.mean(lo)) <= 0.01 * np.mean(lo)
     assert s.status_check() == 0
 
 
@@ -159,9 +181,8 @@ def test_benchmark_sized_complex_batches_match_the_oracle():
     # plus accumulator, relations and frequent entities replicated) on a key space the oracle holds in memory: every
     # block works on many triples one after the other, as in the benchmark
     E, Rl, L, B, K, R = 200_000, 1000, 500, 8192, 10, bench.WORKERS
-    # (one batch: AdaGrad's first step of a component is lr long whatever the gradient's size, so a second batch would
-    # start from values that differ wherever a first gradient was within rounding of zero)
-    h, r, t = [inputs.u32(x) for x in inputs.kge_triples(B, E, Rl, 0.9, 1.2, 0)]
+    n_batches = 2
+    h, r, t = [inputs.u32(x) for x in inputs.kge_triples(n_batches * B, E, Rl, 0.9, 1.2, 0)]
     o = Oracle(E + Rl, L, workers=R, with_adagrad=True, sync_interval=1)
     s = binding.Store(E + Rl, L, workers=R, sync_interval=1, deterministic=True, with_adagrad=True)
     o.init_uniform(0, 5, 0.05)
@@ -175,7 +196,7 @@ def test_benchmark_sized_complex_batches_match_the_oracle():
     lb = torch.zeros(1, device="cuda")
     dk = lambda a: torch.from_numpy(np.ascontiguousarray(a).view(np.int32)).cuda()
     touched = []
-    for b in range(1):
+    for b in range(n_batches):
         sl = slice(b * B, (b + 1) * B)
         lo, negs = o.step_complex(h[sl], r[sl], t[sl], do, K, 0.1, 1e-10, return_negatives=True)
         s.step_complex(dk(h[sl]), dk(r[sl]), dk(t[sl]), ds, K, 0.1, 1e-10, lb)
@@ -184,17 +205,11 @@ def test_benchmark_sized_complex_batches_match_the_oracle():
         touched.append(np.concatenate([h[sl], r[sl], t[sl], negs]))
     rows = np.unique(np.concatenate(touched))
     idx = torch.from_numpy(rows.astype(np.int64)).cuda()
-    acc = s.read_table(1)[idx].cpu().numpy()
-    np.testing.assert_allclose(acc, o.table(1)[rows], rtol=1e-4, atol=1e-9)
-    # the first AdaGrad step of a component moves it by lr whatever the gradient's size: compare values where
-    # the oracle's squared gradients are not vanishing
+    # the stated tolerance on every element of every touched row, both tables (deterministic mode computes between
+    # pull and push in double precision, as the oracle does)
+    np.testing.assert_allclose(s.read_table(1)[idx].cpu().numpy(), o.table(1)[rows], rtol=1e-5, atol=1e-6)
+    np.testing.assert_allclose(s.read_table(0)[idx].cpu().numpy(), o.table(0)[rows], rtol=1e-5, atol=1e-6)
     big = o.table(1)[rows] > 1e-8
-    val, ref = s.read_table(0)[idx].cpu().numpy()[big], o.table(0)[rows][big]
-    # ... and a key pushed to by many triples of the batch takes one such step per triple: a handful of components
-    # whose gradient in one of them is within rounding of zero (while others make the sum large) may differ by a
-    # small part of lr; anything else is within tolerance
-    off = ~np.isclose(val, ref, rtol=1e-4, atol=1e-5)
-    assert off.mean() < 1e-5 and (not off.any() or np.abs(val - ref)[off].max() < 0.02)
     assert big.mean() > 0.05 and s.status_check() == 0
     s.close()
 

@@ -90,13 +90,11 @@ def test_complex_deterministic_parity(L, hot_n, K):
         assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
     o.sync()
     s.sync()
-    # the very first AdaGrad step divides by sqrt(g^2): |step| = lr whatever g, so a gradient of
-    # 1e-9 moves a value by 0.1 -- compare where the oracle's gradient is not vanishing
-    tables_close(o, s, 1, rtol=1e-4, atol=1e-9)
-    big = o.table(1) > 1e-8
-    got = s.read_table(0).cpu().numpy()
-    np.testing.assert_allclose(got[big], o.table(0)[big], rtol=1e-4, atol=1e-5)
-    assert big.mean() > 0.05
+    # deterministic mode computes between pull and push in double precision, as the oracle does, so even
+    # AdaGrad's first step (which is lr long whatever the gradient's size) agrees: the stated tolerance, every element
+    tables_close(o, s, 1)
+    tables_close(o, s, 0)
+    assert np.abs(o.table(0) - init).max() > 0.05
     assert np.array_equal(s.counts().cpu().numpy().astype(np.uint64), o.counts())
 
 

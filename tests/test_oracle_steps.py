@@ -304,3 +304,48 @@ def test_clipping_leaves_non_replicated_keys_and_unclipped_runs_alone():
     assert not np.array_equal(base, tight)                   # what was pushed to them; every update got shorter:
     d_base, d_tight = np.abs(base - init).sum(), np.abs(tight - init).sum()
     assert d_tight < d_base
+
+
+def test_scores_beyond_thirty_are_clamped_in_skip_gram():
+    # a positive pair whose score is 50: the clamp makes it 30, so loss = softplus(-30) (9.4e-14, not the
+    # 1.9e-22 of an unclamped 50) and the gradient factor is sigmoid(30) - 1; the centre component that starts
+    # at zero shows the update -lr * g * u exactly
+    V, L, lr = 4, 4, 0.5
+    o = Oracle(2 * V, L, workers=1)
+    o.table()[1] = [5.0, 0.0, 0.0, 0.0]                     # centre v
+    o.table()[V + 2] = [10.0, 1.0, 0.0, 0.0]                # context u: v.u = 50
+    d = o.register_distribution(V, None, 1, CONFORM, seed=0)
+    loss = o.step_sgns(np.array([1], np.uint32), np.array([V + 2], np.uint32), d, 0, lr)
+    g = 1.0 / (1.0 + np.exp(-30.0)) - 1.0
+    assert loss == pytest.approx(softplus(-30.0), rel=1e-5)
+    assert loss > 1e-15                                     # softplus(-50) would be 1.9e-22
+    assert o.table()[1, 1] == pytest.approx(-lr * g * 1.0, rel=1e-5)
+    # a negative sample whose score is 50 (the distribution has one key, so the negative is known): loss term
+    # softplus(30), not 50; a score of -50 for the positive pair: softplus(30) as well
+    o2 = Oracle(2 * V, L, workers=1)
+    o2.table()[1] = [5.0, 0.0, 0.0, 0.0]
+    o2.table()[V] = [10.0, 1.0, 0.0, 0.0]                   # the only key negatives can be
+    o2.table()[V + 3] = [-10.0, 0.0, 0.0, 0.0]              # context: v.u = -50
+    d2 = o2.register_distribution(V, None, 1, CONFORM, seed=0)
+    loss2, negs = o2.step_sgns(np.array([1], np.uint32), np.array([V + 3], np.uint32), d2, 1, lr, return_negatives=True)
+    assert list(negs) == [V]
+    assert loss2 == pytest.approx(2 * softplus(30.0), rel=1e-6)
+    # the gradient factor of the clamped negative is sigmoid(30): u_neg -= lr * sigmoid(30) * v
+    assert o2.table()[V, 0] == pytest.approx(10.0 - lr * (1.0 / (1.0 + np.exp(-30.0))) * 5.0, rel=1e-6)
+
+
+def test_scores_beyond_thirty_are_clamped_in_complex():
+    # d = 1, real parts only: phi = h r t = 50 -> clamped to 30.  With a zero accumulator the first AdaGrad step is
+    # -lr g / (|g| + eps): for g = (sigmoid(30) - 1) * 10 = -9.4e-13 and eps = 1e-10 that is lr * 0.0093, where an
+    # unclamped score of 50 (g = -1.9e-21) would give lr * 1.9e-11
+    o = Oracle(3, 2, workers=1, with_adagrad=True)
+    o.table(0)[:] = np.array([[5.0, 0.0], [1.0, 0.0], [10.0, 0.0]], np.float32)   # h, r, t
+    d = o.register_distribution(0, None, 1, CONFORM, seed=0)
+    lr, eps = 0.1, 1e-10
+    loss = o.step_complex(np.array([0], np.uint32), np.array([1], np.uint32), np.array([2], np.uint32), d, 0, lr, eps)
+    coef = 1.0 / (1.0 + np.exp(-30.0)) - 1.0
+    assert loss == pytest.approx(softplus(-30.0), rel=1e-5)
+    g_r = coef * 5.0 * 10.0                                 # d(phi)/d(r) = h t
+    assert o.table(1)[1, 0] == pytest.approx(g_r ** 2, rel=1e-5)
+    assert o.table(0)[1, 0] - 1.0 == pytest.approx(-lr * g_r / (abs(g_r) + eps), rel=1e-3)
+    assert o.table(0)[1, 0] - 1.0 > 1e-4                    # an unclamped score would move it by 2e-12
