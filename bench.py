@@ -437,92 +437,9 @@ def run_sgns_reference(args):
 
 
 # --------------------------------------------------------------------------------------------
-# pull / push / PullSample microbenchmark (not the default line): 100M keys x 128 floats, batches of
-# 1M keys ~ Zipf(s), top-k replicated; one JSON line per sweep point
+# the parameter-server microbenchmark: 100M keys x 128 floats, batches of 1M keys ~ Zipf(s), top-k
+# replicated, PullSample under the four schemes (stands in for the paper's Sections 5.5-5.7 sweeps)
 # --------------------------------------------------------------------------------------------
-def run_ps_sweep(args, device):
-    from paper_2104_00501_b200 import binding
-    hbm_peak, peak_kind = peaks()
-    NK, L, N = args.ps_keys, 128, 1 << 20
-    row = L * 4
-    reps = max(args.steps, 5)
-    delta = torch.randn(N, L, device=device)
-    out = torch.empty(N, L, device=device)
-    lines = []
-    for skew in [float(x) for x in args.ps_skews.split(",")]:
-        cdf = inputs.zipf_cdf(NK, skew, device) if skew > 0 else None
-        batches = [inputs.zipf_keys(N, NK, skew, 100 + i, device, cdf=cdf).to(torch.int32) for i in range(4)]
-        key_of_rank = None
-        for topk in [int(x) for x in args.ps_topk.split(",")]:
-            s = binding.Store(NK, L, workers=WORKERS, deterministic=False)
-            s.init_uniform(0, 3, 0.1)
-            if topk:
-                if key_of_rank is None:
-                    key_of_rank = inputs.zipf_key_of_rank(NK, device)
-                s.set_management(key_of_rank[:topk].to(torch.int32).contiguous(), binding.REPLICATE)
-            hot_mask = None
-            if topk:
-                hot_mask = torch.zeros(NK, dtype=torch.bool, device=device)
-                hot_mask[key_of_rank[:topk]] = True
-            ucold = []
-            for b in batches:
-                u = torch.unique(b.long())
-                ucold.append(int(u.numel() if hot_mask is None else (~hot_mask[u]).sum()))
-            ucold = float(np.mean(ucold))
-            s.kernel_timing(True)
-            res = {}
-            for op in ("pull", "push"):
-                for i in range(3):
-                    (s.pull(batches[i % 4], out) if op == "pull" else s.push(batches[i % 4], delta))
-                s.kernel_time()
-                for i in range(reps):
-                    (s.pull(batches[i % 4], out) if op == "pull" else s.push(batches[i % 4], delta))
-                    if op == "push" and topk and (i + 1) % 16 == 0:
-                        s.sync()
-                ms, n = s.kernel_time()
-                t = ms / 1e3 / n
-                alg = 4 * N + row * N + (1 if op == "pull" else 2) * row * ucold
-                res[op] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
-                           "frac": alg / t / 1e9 / hbm_peak, "logical_gbs": (4 * N + (2 if op == "pull" else 3) * row * N) / t / 1e9}
-            if topk:
-                # pull again while the replicas hold unmerged updates (the pulls above saw freshly merged replicas,
-                # whose rows need not be read)
-                for i in range(4):
-                    s.push(batches[i % 4], delta)
-                s.kernel_time()
-                for i in range(reps):
-                    s.pull(batches[i % 4], out)
-                ms, n = s.kernel_time()
-                t = ms / 1e3 / n
-                alg = 4 * N + row * N + row * ucold
-                res["pull_with_pending_updates"] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
-                                                    "frac": alg / t / 1e9 / hbm_peak}
-            # replica merge cost: pushes with a merge every `interval` pushes, time per push including its share
-            sync_sweep = {}
-            if topk:
-                s.kernel_timing(False)
-                for interval in (1, 16, 256):
-                    n_push = max(interval, 32)
-                    state = {"i": 0}
-
-                    def push_and_merge():
-                        for _ in range(n_push):
-                            s.push(batches[state["i"] % 4], delta)
-                            state["i"] += 1
-                            if state["i"] % interval == 0:
-                                s.sync()
-                    sync_sweep[str(interval)] = _time_calls(push_and_merge, 2, warm=1) / n_push * 1e6
-            line = {"workload": "ps microbenchmark", "keys": NK, "value_len": L, "batch": N, "zipf_s": skew, "topk": topk,
-                    "distinct_cold_rows": ucold, "peak": hbm_peak, "peak_kind": peak_kind,
-                    "push_us_incl_merge_every": sync_sweep, **res}
-            print(json.dumps(line), flush=True)
-            lines.append(line)
-            s.close()
-            del s
-            torch.cuda.empty_cache()
-    return lines
-
-
 def _time_calls(fn, reps, warm=3):
     """Mean device time of fn() in seconds: CUDA events on the current stream around `reps` calls."""
     for _ in range(warm):
@@ -537,36 +454,464 @@ def _time_calls(fn, reps, warm=3):
     return e0.elapsed_time(e1) / 1e3 / reps
 
 
-def run_sample_sweep(args, device):
-    """PullSample of 1M keys (keys + values) from a Zipf(1.0) target over the whole store, four levels."""
+class PsSetup:
+    """The store of the microbenchmark with its inputs: key batches per skew, update rows, output buffers, the four
+    sampling distributions.  Keys of rank r (0-based, by true frequency) are `hot_keys[r]`; replicating the top k
+    means the first k of them, in that order, so the most frequent key gets hot slot 0."""
+
+    def __init__(self, binding, device, nk, seed=0, levels=PS_LEVELS):
+        self.binding, self.device, self.nk, self.seed = binding, device, nk, seed
+        self.N, self.L, self.row = PS_BATCH, PS_LEN, PS_LEN * 4
+        self.s = binding.Store(nk, PS_LEN, workers=WORKERS, sync_interval=0, deterministic=False, track_ownership=True)
+        self.s.init_uniform(0, 3, 0.1)
+        self.hot_keys = inputs.rank_to_key(torch.arange(min(max(PS_TOPKS), nk), device=device), nk, seed=1).to(torch.int32).contiguous()
+        self.topk = 0
+        g = torch.Generator(device=device)
+        g.manual_seed(17 + seed)
+        self.delta = torch.randn(self.N, self.L, device=device, generator=g)
+        self.out = torch.empty(self.N, self.L, device=device)
+        self.skeys = torch.empty(self.N, dtype=torch.int32, device=device)
+        self.svals = torch.empty(self.N, self.L, device=device)
+        self._batches = {}
+        self.dists = {}
+        if levels:
+            w = inputs.zipf_integer_weights(nk, 1.0, device).to(torch.int32).contiguous()
+            lv = {"CONFORM": binding.CONFORM, "BOUNDED": binding.BOUNDED, "LONG-TERM": binding.LONGTERM,
+                  "NON-CONFORM": binding.NONCONFORM}
+            t0 = time.perf_counter()
+            for name in levels:
+                self.dists[name] = self.s.register_distribution(0, w, nk, lv[name], U=U_REUSE, G=G_POOL, seed=11 + lv[name])
+            torch.cuda.synchronize()
+            self.alias_build_s = (time.perf_counter() - t0) / len(levels)
+            del w
+
+    def batches(self, skew):
+        """Four batches of 1M keys ~ Zipf(skew) over the store's keys (seeded; kept for the skew last asked for)."""
+        if skew not in self._batches:
+            self._batches.clear()
+            cdf = inputs.zipf_cdf(self.nk, skew, self.device) if skew > 0 else None
+            self._batches[skew] = [inputs.zipf_keys(self.N, self.nk, skew, 100 + 10 * self.seed + i, self.device, cdf=cdf)
+                                   .to(torch.int32).contiguous() for i in range(4)]
+            del cdf
+        return self._batches[skew]
+
+    def set_topk(self, k):
+        k = min(k, self.hot_keys.numel())
+        if k < self.topk:
+            self.s.set_management(self.hot_keys[k:self.topk].contiguous(), self.binding.SINGLE)
+        elif k > self.topk:
+            self.s.set_management(self.hot_keys[self.topk:k].contiguous(), self.binding.REPLICATE)
+        self.topk = k
+
+    def distinct_cold(self, keys):
+        """Distinct non-replicated keys of a batch: the rows that have to come from (and go back to) HBM."""
+        u = torch.unique(keys.long())
+        if self.topk:
+            hot = torch.zeros(self.nk, dtype=torch.bool, device=self.device)
+            hot[self.hot_keys[:self.topk].long()] = True
+            u = u[~hot[u]]
+            del hot
+        return int(u.numel())
+
+    def alg_bytes(self, kind, ucold):
+        """Algorithmic bytes of one 1M-key launch: keys + the caller's rows + the distinct cold rows of the table
+        (read once for a pull; read and written once for a push)."""
+        N, row = self.N, self.row
+        if kind == "pull":
+            return 4 * N + row * N + row * ucold
+        if kind == "push":
+            return 4 * N + row * N + 2 * row * ucold
+        if kind == "sample_rows":                    # keys read from the handle and written out, rows written, cold rows read
+            return 8 * N + row * N + row * ucold
+        raise ValueError(kind)
+
+    def sample(self, level):
+        h = self.s.prepare_sample(self.dists[level], self.N)
+        self.s.pull_sample(h, self.N, True, self.skeys, self.svals)
+
+    def close(self):
+        self.s.close()
+        for name in ("delta", "out", "svals", "skeys"):
+            setattr(self, name, None)
+        self._batches.clear()
+        torch.cuda.empty_cache()
+
+
+def ps_point(ps, skew, topk, reps, hbm_peak):
+    """pull and push of 1M keys at one (skew, top-k) point: kernel time by event pairs on the launching stream."""
+    s = ps.s
+    batches = ps.batches(skew)
+    ps.set_topk(topk)
+    N, row = ps.N, ps.row
+    ucold = float(np.mean([ps.distinct_cold(b) for b in batches]))
+    s.kernel_timing(True)
+    res = {}
+    for op in ("pull", "push"):
+        for i in range(3):
+            (s.pull(batches[i % 4], ps.out) if op == "pull" else s.push(batches[i % 4], ps.delta))
+        s.kernel_times()
+        for i in range(reps):
+            (s.pull(batches[i % 4], ps.out) if op == "pull" else s.push(batches[i % 4], ps.delta))
+            if op == "push" and topk and (i + 1) % 16 == 0:
+                s.sync()
+        ms, n = s.kernel_times()[op]
+        t = ms / 1e3 / n
+        alg = ps.alg_bytes(op, ucold)
+        res[op] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9, "frac": alg / t / 1e9 / hbm_peak,
+                   "logical_gbs": (4 * N + (2 if op == "pull" else 3) * row * N) / t / 1e9}
+    if topk:
+        # pull again while the replicas hold unmerged updates (the pulls above saw freshly merged replicas)
+        for i in range(4):
+            s.push(batches[i % 4], ps.delta)
+        s.kernel_times()
+        for i in range(reps):
+            s.pull(batches[i % 4], ps.out)
+        ms, n = s.kernel_times()["pull"]
+        t = ms / 1e3 / n
+        alg = ps.alg_bytes("pull", ucold)
+        res["pull_with_pending_updates"] = {"us": t * 1e6, "keys_per_s": N / t, "algorithmic_gbs": alg / t / 1e9,
+                                            "frac": alg / t / 1e9 / hbm_peak}
+        s.sync()
+    s.kernel_timing(False)
+    return {"zipf_s": skew, "topk": topk, "distinct_cold_rows": ucold, **res}
+
+
+def ps_sync_point(ps, skew, topk, interval):
+    """Pushes of 1M keys with a replica merge every `interval` pushes: device time per push, merges included."""
+    s = ps.s
+    batches = ps.batches(skew)
+    ps.set_topk(topk)
+    n_push = max(interval, 32)
+    state = {"i": 0}
+
+    def push_and_merge():
+        for _ in range(n_push):
+            s.push(batches[state["i"] % 4], ps.delta)
+            state["i"] += 1
+            if state["i"] % interval == 0:
+                s.sync()
+    t = _time_calls(push_and_merge, 2, warm=1) / n_push
+    s.sync()
+    return {"zipf_s": skew, "topk": topk, "merge_every": interval, "push_us_incl_merge": t * 1e6, "keys_per_s": ps.N / t}
+
+
+def ps_sample_point(ps, level, reps, hbm_peak, warm=3):
+    """PrepareSample + PullSample (keys and rows) of 1M keys from the Zipf(1.0) target under one scheme."""
+    N, L = ps.N, ps.L
+    t = _time_calls(lambda: ps.sample(level), max(reps, 1), warm=warm)
+    uniq = int(torch.unique(ps.skeys).numel())
+    draws = N // U_REUSE if level in ("BOUNDED", "LONG-TERM") else N        # pooled reuse draws every pool once
+    alg = 4 * N + L * 4 * N + L * 4 * uniq + 16 * draws                     # keys out, rows out, distinct rows read, alias entries
+    return {"level": level, "us": t * 1e6, "keys_per_s": N / t, "distinct_keys": uniq, "algorithmic_gbs": alg / t / 1e9,
+            "frac": alg / t / 1e9 / hbm_peak}
+
+
+def run_ps_sweep(args, device):
+    """`--workload ps`: one JSON line per (skew, top-k) point."""
     from paper_2104_00501_b200 import binding
     hbm_peak, peak_kind = peaks()
-    NK, L, N = args.ps_keys, 128, 1 << 20
-    s = binding.Store(NK, L, workers=WORKERS, deterministic=False, track_ownership=True)
-    s.init_uniform(0, 3, 0.1)
-    key_of_rank = inputs.zipf_key_of_rank(NK, device)
-    s.set_management(key_of_rank[:1000].to(torch.int32).contiguous(), binding.REPLICATE)
-    w = inputs.zipf_integer_weights(NK, 1.0, device).to(torch.int32).contiguous()
-    t0 = time.perf_counter()
-    dists = {name: s.register_distribution(0, w, NK, lvl, U=U_REUSE, G=G_POOL, seed=11 + lvl)
-             for name, lvl in (("CONFORM", binding.CONFORM), ("BOUNDED", binding.BOUNDED),
-                               ("LONG-TERM", binding.LONGTERM), ("NON-CONFORM", binding.NONCONFORM))}
+    ps = PsSetup(binding, device, args.ps_keys, levels=())
+    for skew in [float(x) for x in args.ps_skews.split(",")]:
+        for topk in [int(x) for x in args.ps_topk.split(",")]:
+            line = {"workload": "ps microbenchmark", "keys": ps.nk, "value_len": ps.L, "batch": ps.N, "peak": hbm_peak,
+                    "peak_kind": peak_kind, **ps_point(ps, skew, topk, max(args.steps, 5), hbm_peak)}
+            if topk:
+                line["push_us_incl_merge_every"] = {str(iv): ps_sync_point(ps, skew, topk, iv)["push_us_incl_merge"]
+                                                    for iv in PS_SYNCS}
+            print(json.dumps(line), flush=True)
+    ps.close()
+
+
+def run_sample_sweep(args, device):
+    """`--workload sample`: PullSample of 1M keys (keys + values) from a Zipf(1.0) target over the whole store."""
+    from paper_2104_00501_b200 import binding
+    hbm_peak, peak_kind = peaks()
+    ps = PsSetup(binding, device, args.ps_keys)
+    ps.set_topk(1000)
+    for level in PS_LEVELS:
+        print(json.dumps({"workload": "PullSample", "keys": ps.nk, "value_len": ps.L, "samples": ps.N, "peak_kind": peak_kind,
+                          "alias_build_s": ps.alias_build_s,
+                          **ps_sample_point(ps, level, args.steps, hbm_peak, warm=min(3, args.warmup))}), flush=True)
+    ps.close()
+
+
+def run_ps_line(args, rank, world, device):
+    """The default line: pull + push + sample pull of 1M keys each per step on the 100M-key store."""
+    from paper_2104_00501_b200 import binding
+    hbm_peak, peak_kind = peaks()
+    K, W = args.steps, args.warmup
+    ps = PsSetup(binding, device, args.ps_keys, seed=rank)
+    s, N, row = ps.s, ps.N, ps.row
+    ps.set_topk(PS_TOPK)
+    batches = ps.batches(PS_SKEW)
+    state = {"pushes": 0}
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def step(i):
+        s.pull(batches[i % 4], ps.out)
+        s.push(batches[(i + 1) % 4], ps.delta)
+        state["pushes"] += 1
+        if state["pushes"] % PS_SYNC == 0:
+            s.sync()
+        ps.sample(PS_LEVEL)
+
+    # warm-up (timed only to size the repetitions: the timed region repeats the K steps until it is a second long)
+    step(0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for i in range(W):
+        step(i)
+    e1.record()
     torch.cuda.synchronize()
-    build_s = (time.perf_counter() - t0) / 4
-    keys = torch.empty(N, dtype=torch.int32, device=device)
-    vals = torch.empty(N, L, device=device)
-    for name, d in dists.items():
-        def once():
-            h = s.prepare_sample(d, N)
-            s.pull_sample(h, N, True, keys, vals)
-        t = _time_calls(once, max(args.steps, 1), warm=min(3, args.warmup))
-        uniq = int(torch.unique(keys).numel())
-        alg = 4 * N + L * 4 * N + L * 4 * uniq + 16 * N
-        print(json.dumps({"workload": "PullSample", "level": name, "keys": NK, "value_len": L, "samples": N,
-                          "us": t * 1e6, "keys_per_s": N / t, "distinct_keys": uniq, "algorithmic_gbs": alg / t / 1e9,
-                          "frac": alg / t / 1e9 / hbm_peak, "peak_kind": peak_kind,
-                          "alias_build_s": build_s}), flush=True)
+    est_ms = e0.elapsed_time(e1) / W
+    reps = int(min(max(5, -(-args.min_timed_ms // (est_ms * K))), max(5, 60000 // (4 * K))))
+    reps = int(max_over_ranks([reps], world, device)[0])
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(reps + 1)]
+    launches0 = s.stats()["launches"]
+    s.kernel_timing(True)
+    barrier()
+    with ClockSampler(torch.cuda.current_device()) as clk:
+        ev[0].record()
+        for r in range(reps):
+            for i in range(K):
+                step(r * K + i)
+            ev[r + 1].record()
+        barrier()
+    rep_ms = [ev[r].elapsed_time(ev[r + 1]) for r in range(reps)]
+    kt = s.kernel_times()
+    s.kernel_timing(False)
+    launches = (s.stats()["launches"] - launches0) / reps
+    assert s.status_check() == 0
+    ms = float(np.median(rep_ms))                               # K steps
+    total_ms = float(sum(rep_ms))
+
+    # roofline of the three main kernels in the launch configuration that was just timed
+    ucold = {"pull": float(np.mean([ps.distinct_cold(b) for b in batches]))}
+    ucold["push"] = ucold["pull"]
+    ucold["sample_rows"] = float(ps.distinct_cold(ps.skeys))
+    kernels = {}
+    for kind in ("pull", "push", "sample_rows"):
+        k_ms, k_n = kt[kind]
+        t = k_ms / 1e3 / max(k_n, 1)
+        alg = ps.alg_bytes(kind, ucold[kind])
+        name, m0, m1 = PS_KERNEL_SOURCE[kind]
+        cap = NCU_TRAFFIC_PS[kind]
+        traffic = cap["bytes_per_launch"] if cap["sha1"] and cap["sha1"] == kernel_source_sha1(m0, m1) else None
+        kernels[kind] = {"kernel": name, "kernel_us": t * 1e6, "launches": int(k_n), "achieved": alg / t / 1e9,
+                         "frac": alg / t / 1e9 / hbm_peak, "algorithmic_bytes_per_launch": alg,
+                         "distinct_cold_rows": ucold[kind], "traffic": traffic,
+                         "share_of_step": (k_ms / max(k_n, 1)) / (total_ms / (reps * K))}
+    draw_ms, draw_n = kt["draw"]
+    dominant = max(kernels, key=lambda k: kernels[k]["kernel_us"])
+    dk = kernels[dominant]
+
+    # end to end through the public API with HOST buffers: every step's keys and update rows start in pinned host memory
+    # and are copied to the device inside the timed region, and every step's results (pulled rows, sampled keys and
+    # rows) are copied back to pinned host memory.  One stream, in call order.
+    e2e_steps = max(3, min(K, 32))
+    hk = [b.cpu().pin_memory() for b in batches]
+    hdelta = ps.delta.cpu().pin_memory()
+    hout = torch.empty((N, ps.L), dtype=torch.float32).pin_memory()
+    hsvals = torch.empty((N, ps.L), dtype=torch.float32).pin_memory()
+    hskeys = torch.empty(N, dtype=torch.int32).pin_memory()
+    dk_pull, dk_push = torch.empty_like(batches[0]), torch.empty_like(batches[0])
+    ddelta = torch.empty_like(ps.delta)
+
+    def e2e_loop(steps, rows_cross):
+        barrier()
+        t0 = time.perf_counter()
+        for i in range(steps):
+            dk_pull.copy_(hk[i % 4], non_blocking=True)
+            s.pull(dk_pull, ps.out)
+            if rows_cross:
+                hout.copy_(ps.out, non_blocking=True)
+            dk_push.copy_(hk[(i + 1) % 4], non_blocking=True)
+            if rows_cross:
+                ddelta.copy_(hdelta, non_blocking=True)
+            s.push(dk_push, ddelta if rows_cross else ps.delta)
+            state["pushes"] += 1
+            if state["pushes"] % PS_SYNC == 0:
+                s.sync()
+            ps.sample(PS_LEVEL)
+            hskeys.copy_(ps.skeys, non_blocking=True)
+            if rows_cross:
+                hsvals.copy_(ps.svals, non_blocking=True)
+        barrier()
+        dt = time.perf_counter() - t0
+        assert int(hskeys[0]) >= 0 and (not rows_cross or np.isfinite(float(hout[0, 0]) + float(hsvals[-1, -1])))
+        return dt
+
+    e2e_loop(1, True)
+    e2e_s = e2e_loop(e2e_steps, True)
+    keys_steps = max(e2e_steps, min(4 * K, 256))
+    keys_s = e2e_loop(keys_steps, False)       # only keys cross the bus: update rows and results stay on the device
+
+    ms, total_ms, e2e_s, keys_s = max_over_ranks([ms, total_ms, e2e_s, keys_s], world, device)
+    acc_step = 3 * N                                            # pulled + pushed + sampled keys
+    out = {
+        "metric": "key accesses/s (pull+push+sample)", "value": aggregate_throughput(K * acc_step, ms / 1e3, world),
+        "unit": "key accesses/s", "n_gpus": world, "steps": K, "warmup": W, "ms_per_step": ms / K,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD_PS, "workers": WORKERS, "keys": ps.nk, "value_len": ps.L, "batch": N,
+                   "l2": "inputs (three 512 MB row buffers, 51 GB table) larger than L2; no explicit flush",
+                   "timed_region": f"median of {reps} back-to-back repetitions of the {K} steps ({total_ms:.0f} ms in all)",
+                   "replicas": world},
+        "updates_per_s": aggregate_throughput(K * N, ms / 1e3, world),
+        "repetitions": reps, "timed_ms_total": total_ms,
+        "clocks": clk.summary(),
+        "e2e": {"value": aggregate_throughput(e2e_steps * acc_step, e2e_s, world), "unit": "key accesses/s",
+                "h2d_bytes_per_step": 4 * N + 4 * N + row * N, "d2h_bytes_per_step": row * N + 4 * N + row * N,
+                "steps": e2e_steps,
+                "note": "keys, update rows, pulled rows, sampled keys and rows all cross the bus: bound by the host link",
+                "keys_only": {"value": aggregate_throughput(keys_steps * acc_step, keys_s, world), "unit": "key accesses/s",
+                              "h2d_bytes_per_step": 8 * N, "d2h_bytes_per_step": 4 * N, "steps": keys_steps,
+                              "note": "update rows and pulled/sampled rows stay on the device (a trainer on the GPU)"}},
+        "gpu_launches": int(round(launches)),
+        "roofline": {"bound": "hbm", "kernel": f"{dk['kernel']} ({dominant})", "achieved": dk["achieved"], "peak": hbm_peak,
+                     "peak_kind": peak_kind, "unit": "GB/s", "frac": dk["frac"], "traffic": dk["traffic"],
+                     "algorithmic_bytes_per_launch": dk["algorithmic_bytes_per_launch"], "kernel_us": dk["kernel_us"],
+                     "kernels": kernels, "draw_kernel_us": draw_ms / max(draw_n, 1) * 1e3},
+    }
+    if rank == 0 and world == 1 and not args.no_sweep:
+        out["sweep"] = ps_sweep(args, ps, hbm_peak, device)
+    ps.close()
+    if rank == 0 and world == 1 and not args.no_sweep:
+        out["sweep"]["steps"] = step_entries(args, device)
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = ps_cpu_baseline(budget_s=12.0)
+    return out
+
+
+def ps_sweep(args, ps, hbm_peak, device):
+    """Every grid point of the microbenchmark: 4 skews x 3 top-k (pull and push), 3 merge intervals, 4 sampling
+    schemes.  Kernel times by event pairs; fractions are algorithmic bytes over the measured copy peak."""
+    reps = max(min(args.steps, 20), 10)
+    sampling = [ps_sample_point(ps, level, reps, hbm_peak) for level in PS_LEVELS]          # at the headline's top-1k
+    merges = [ps_sync_point(ps, PS_SKEW, PS_TOPK, iv) for iv in PS_SYNCS]
+    points = [ps_point(ps, skew, topk, reps, hbm_peak) for skew in PS_SKEWS for topk in PS_TOPKS]
+    return {"pull_push": points, "merge_interval": merges, "pull_sample": sampling, "alias_build_s": ps.alias_build_s,
+            "reps_per_point": reps}
+
+
+def step_entries(args, device):
+    """One entry per workload step (skip-gram, ComplEx, matrix factorization) at the paper-sized configurations."""
+    out = {}
+    try:
+        out["sgns"] = sgns_entry(device, steps=256)
+        out["complex"] = run_step_workload(args, device, "kge", emit=False)
+        out["mf"] = run_step_workload(args, device, "mf", emit=False)
+        mo, args.mf_order = args.mf_order, "column"
+        out["mf_by_column"] = run_step_workload(args, device, "mf", emit=False)
+        args.mf_order = mo
+    finally:
+        torch.cuda.empty_cache()
+    return out
+
+
+def sgns_entry(device, steps):
+    """The skip-gram workload in brief: `steps` steps through nups_run_sgns, 64 per call."""
+    from paper_2104_00501_b200 import binding
+    nb = steps
+    s, dist, hot, c, o, weights = build_store(binding, device, nb, seed=0)
+    losses = torch.zeros(64, dtype=torch.float32, device=device)
+
+    def run():
+        for j in range(0, nb, 64):
+            s.run_sgns(c[j * BATCH:(j + 64) * BATCH], o[j * BATCH:(j + 64) * BATCH], BATCH, dist, NEG, LR, losses)
+    dt = _time_calls(run, 3, warm=1) / nb
+    s.kernel_timing(True)
+    run()
+    k_ms, k_n = s.kernel_times()["step"]
+    s.kernel_timing(False)
     s.close()
+    return {"workload": WORKLOAD_SGNS, "us_per_step": dt * 1e6, "key_accesses_per_s": BATCH * ACCESSES_PER_PAIR / dt,
+            "updates_per_s": BATCH * UPDATES_PER_PAIR / dt, "kernel": "sgns_kernel", "kernel_us_per_launch": k_ms / max(k_n, 1) * 1e3,
+            "steps_per_launch": nb / max(k_n, 1), "final_loss": float(losses.mean())}
+
+
+# --------------------------------------------------------------------------------------------
+# the oracle on the microbenchmark: CPU baseline and reference arm
+# --------------------------------------------------------------------------------------------
+class PsOracle:
+    """The oracle on the same kind of step, with the table scaled down to PS_ORACLE_KEYS keys (a 51 GB table on the
+    host is not something every box has): keys ~ Zipf(1.0) over the smaller key space, the same top-1k replicated."""
+
+    def __init__(self, n_max):
+        import oracle
+        nk = PS_ORACLE_KEYS
+        self.o = oracle.Oracle(nk, PS_LEN, workers=WORKERS)
+        self.o.init_uniform(0, 3, 0.1)
+        hot = inputs.u32(inputs.rank_to_key(torch.arange(PS_TOPK), nk, seed=1))
+        self.o.set_management(hot, oracle.REPLICATE)
+        w = inputs.u32(inputs.zipf_integer_weights(nk, 1.0, "cpu"))
+        self.d = self.o.register_distribution(0, w, nk, oracle.BOUNDED, U=U_REUSE, G=G_POOL, seed=13)
+        cdf = inputs.zipf_cdf(nk, PS_SKEW, "cpu")
+        self.keys = [inputs.u32(inputs.zipf_keys(n_max, nk, PS_SKEW, 100 + i, "cpu", cdf=cdf)) for i in range(2)]
+        self.delta = np.random.default_rng(0).standard_normal((n_max, PS_LEN), dtype=np.float32)
+        self.pushes = 0
+
+    def step(self, i, n):
+        self.o.pull(self.keys[i % 2][:n])
+        self.o.push(self.keys[(i + 1) % 2][:n], self.delta[:n])
+        self.pushes += 1
+        if self.pushes % PS_SYNC == 0:
+            self.o.sync()
+        self.o.pull_sample(self.o.prepare_sample(self.d, n), n, values=True)
+
+    @staticmethod
+    def scaling():
+        return (f"table scaled to {PS_ORACLE_KEYS:,} keys x {PS_LEN} fp32 (2 GB of host memory instead of 51 GB), keys ~ Zipf(1.0) "
+                f"over them, top-1k replicated, same step otherwise")
+
+
+def ps_cpu_baseline(budget_s):
+    n = 65536
+    orc = PsOracle(n)
+    orc.step(0, 4096)
+    t0 = time.perf_counter()
+    done = 0
+    while time.perf_counter() - t0 < budget_s:
+        orc.step(done, n)
+        done += 1
+    dt = time.perf_counter() - t0
+    return {"value": done * 3 * n / dt, "unit": "key accesses/s", "cores": 1, "kind": "oracle",
+            "sample": f"{done} steps of {n} keys per pull, push and sample pull (the workload's steps take {PS_BATCH}), "
+                      f"{PsOracle.scaling()}; {dt:.1f} s on one host thread (of {os.cpu_count()} cores)"}
+
+
+def run_ps_reference(args):
+    """`--impl reference`: the oracle, as it stands, on the default line's workload; every step a bounded sample."""
+    total = args.steps + args.warmup
+    orc = PsOracle(PS_BATCH)
+    probe_n = 16384
+    t0 = time.perf_counter()
+    orc.step(0, probe_n)
+    probe = time.perf_counter() - t0
+    budget = 150.0
+    per_step = int(min(PS_BATCH, max(4096, probe_n * budget / (probe * total) // 4096 * 4096)))
+    for i in range(args.warmup):
+        orc.step(i, per_step)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        orc.step(args.warmup + i, per_step)
+    dt = time.perf_counter() - t0
+    value = args.steps * 3 * per_step / dt
+    sample = (f"{per_step} keys per pull, push and sample pull per step (of the workload's {PS_BATCH}), {PsOracle.scaling()}; "
+              f"single host thread of {os.cpu_count()} cores")
+    return {
+        "impl": "reference", "metric": "key accesses/s (pull+push+sample)", "value": value, "unit": "key accesses/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3 / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD_PS, "workers": WORKERS, "keys": PS_KEYS, "value_len": PS_LEN, "batch": PS_BATCH,
+                   "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "key accesses/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "key accesses/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
 
 
 def run_staleness_sweep(args, device):
@@ -620,7 +965,7 @@ def run_staleness_sweep(args, device):
     store.close()
 
 
-def run_step_workload(args, device, which):
+def run_step_workload(args, device, which, emit=True):
     """ComplEx + AdaGrad (config 3) or matrix factorization (config 4) steps in fast mode."""
     from paper_2104_00501_b200 import binding
     hbm_peak, peak_kind = peaks()
@@ -681,31 +1026,39 @@ def run_step_workload(args, device, which):
     # measures by itself.  floor = both in full overlap, read_then_reduce = one after the other.
     red_dram = s.probe_reduction_rate(2 << 30, 5)
     t_read, t_red = (logical / 2) / (hbm_peak * 1e9), (logical / 2) / (red_dram * 1e9)
-    print(json.dumps({"workload": cfg, "kernel": name, "hot_slots": s.stats()["hot_slots"], "us_per_step": dt * 1e6,
-                      "kernel_us": k_s * 1e6, "key_accesses_per_s": B * per_item / dt, "updates_per_s": B * upd / dt,
-                      "logical_gbs": logical / k_s / 1e9, "logical_frac_of_hbm_peak": logical / k_s / 1e9 / hbm_peak,
-                      "reduction_rate_dram_gbs": red_dram, "floor_us_reads_and_reductions_overlapped": max(t_read, t_red) * 1e6,
-                      "us_read_then_reduce": (t_read + t_red) * 1e6,
-                      "frac_of_overlapped_floor": max(t_read, t_red) / k_s,
-                      "peak_kind": peak_kind, "final_loss": float(loss.item()), "tables": tables}), flush=True)
+    line = {"workload": cfg, "kernel": name, "hot_slots": s.stats()["hot_slots"], "us_per_step": dt * 1e6,
+            "kernel_us": k_s * 1e6, "key_accesses_per_s": B * per_item / dt, "updates_per_s": B * upd / dt,
+            "logical_gbs": logical / k_s / 1e9, "logical_frac_of_hbm_peak": logical / k_s / 1e9 / hbm_peak,
+            "reduction_rate_dram_gbs": red_dram, "floor_us_reads_and_reductions_overlapped": max(t_read, t_red) * 1e6,
+            "us_read_then_reduce": (t_read + t_red) * 1e6,
+            "frac_of_overlapped_floor": max(t_read, t_red) / k_s,
+            "peak_kind": peak_kind, "final_loss": float(loss.item()), "tables": tables}
     s.close()
+    if emit:
+        print(json.dumps(line), flush=True)
+    return line
 
 
 def main():
     global TOKENS, HOT_FRACTION, WORKERS
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=16384)
-    ap.add_argument("--warmup", type=int, default=64)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=8)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="sgns", choices=["sgns", "ps", "sample", "kge", "mf", "staleness"])
+    ap.add_argument("--no-sweep", action="store_true", help="default line only: skip the sweep of the other grid points")
+    ap.add_argument("--min-timed-ms", type=float, default=1000.0,
+                    help="the timed region repeats the K steps until it is at least this long (at least 5 times)")
+    ap.add_argument("--workload", default="psline", choices=["psline", "sgns", "ps", "sample", "kge", "mf", "staleness"],
+                    help="psline (default): the parameter-server microbenchmark line with its sweep; sgns: the skip-gram line; "
+                         "the others print their own lines")
     ap.add_argument("--hot-fraction", type=float, default=HOT_FRACTION, help="share of keys to replicate (default 0.01)")
     ap.add_argument("--workers", type=int, default=WORKERS)
     ap.add_argument("--clip-factor", type=float, default=0.0,
                     help="staleness workload: clip replicated-key updates at this multiple of their mean norm")
     ap.add_argument("--tokens", type=int, default=TOKENS, help="length of the synthetic token stream (profiling runs use less)")
-    ap.add_argument("--ps-keys", type=int, default=100_000_000)
+    ap.add_argument("--ps-keys", type=int, default=PS_KEYS, help="smaller for profiling runs")
     ap.add_argument("--kge-entities", type=int, default=5_000_000, help="smaller for profiling runs")
     ap.add_argument("--mf-rows", type=int, default=10_000_000, help="smaller for profiling runs")
     ap.add_argument("--mf-order", default="random", choices=["random", "column", "column-plain"],
@@ -722,7 +1075,8 @@ def main():
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         if rank == 0:
-            print(json.dumps(run_reference(args)), flush=True)
+            line = run_sgns_reference(args) if args.workload == "sgns" else run_ps_reference(args)
+            print(json.dumps(line), flush=True)
         return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
@@ -742,7 +1096,7 @@ def main():
         return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)
-    out = run_ours(args, rank, world, device)
+    out = run_sgns_line(args, rank, world, device) if args.workload == "sgns" else run_ps_line(args, rank, world, device)
     if rank == 0:
         print(json.dumps(out), flush=True)
     if world > 1:
