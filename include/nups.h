@@ -77,14 +77,25 @@ typedef struct nups_config {
     float    clip_factor;     /* > 0: nups_step_sgns and nups_step_mf clip every update to a   */
                               /*    replicated key at clip_factor times the mean norm of such  */
                               /*    updates so far, see nups_get_clip_stats; 0 = no clipping   */
-    uint32_t reserved[7];
+    uint32_t max_device_mib;  /* > 0: the store never holds more than this many MiB of device memory (tables,   */
+                              /*    maps, replicas, alias tables, handles, scratch); a call that would need    */
+                              /*    more returns NUPS_ENOMEM before it allocates anything and changes nothing  */
+    uint32_t first_epoch;     /* number from which calls that move keys are counted (24 bits, wraps; see        */
+                              /*    track_ownership); only of interest to tests of the wrap-around              */
+    uint32_t merge_mean;      /* 1: a merge adds the MEAN of the pending updates of the workers that touched a  */
+                              /*    replicated key since the last merge instead of their sum (damps the summed  */
+                              /*    duplicate updates of very frequent keys); not with sync_period_us           */
+    uint32_t reserved[4];
 } nups_config;
 
 /* ---- store (Section 3.1: keys, pull, push) -------------------------------- */
 
 /* Allocate a store of num_keys rows of value_len floats, zero-filled, no key
  * replicated.  *h_out receives the store.  NUPS_EINVAL: num_keys == 0 or
- * > 2^32-1, value_len == 0 or not a multiple of 4, workers > 254.             */
+ * > 2^32-1, value_len == 0 or not a multiple of 4, workers > 254.  NUPS_ENOMEM:
+ * the device has not enough memory, or the store's own limit (max_device_mib) is
+ * smaller than what the tables and maps need; that limit is checked before the
+ * device is touched.                                                           */
 nups_status nups_create(uint64_t num_keys, uint32_t value_len, const nups_config* h_cfg, nups_store** h_out);
 
 /* Free everything the store owns.  Synchronises the device.                   */
@@ -159,8 +170,9 @@ nups_status nups_set_management(nups_store* store, const uint32_t* d_keys, uint6
 
 /* sync (Section 3.2: periodic sparse all-reduce of replica updates): for every
  * hot slot touched since the last sync add the workers' pending updates, worker
- * 0 first, to the stored row and clear them.  With no replicated key nothing is
- * launched.                                                                   */
+ * 0 first, to the stored row and clear them (with merge_mean: their sum divided
+ * by the number of workers that touched the slot).  With no replicated key
+ * nothing is launched.                                                        */
 nups_status nups_sync(nups_store* store, void* stream);
 
 /* Add 1 to the access count of every key of the stream (dataset frequency

@@ -59,6 +59,7 @@ def lib():
             "orc_push2": (C.c_int, [C.c_void_p, _u32p, C.c_uint64, _f32p, _f32p]),
             "orc_sync": (C.c_int, [C.c_void_p]),
             "orc_set_clipping": (None, [C.c_void_p, C.c_double]),
+            "orc_set_merge_mean": (None, [C.c_void_p, C.c_int]),
             "orc_clip_stats": (None, [C.c_void_p, C.POINTER(C.c_double), _u64p]),
             "orc_count_accesses": (C.c_int, [C.c_void_p, _u32p, C.c_uint64]),
             "orc_select_hot": (C.c_uint64, [C.c_void_p, C.c_int, C.c_uint64, _u32p]),
@@ -190,6 +191,10 @@ class Oracle:
 
     def sync(self):
         _chk(self._l.orc_sync(self._s), "sync")
+
+    def set_merge_mean(self, on=True):
+        """A sync adds the mean of the pending updates over the workers that pushed to a key, not their sum."""
+        self._l.orc_set_merge_mean(self._s, int(on))
 
     # -- management -------------------------------------------------------
     def count_accesses(self, keys):

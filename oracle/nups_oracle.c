@@ -176,7 +176,8 @@ typedef struct {
     uint32_t* hot_keys;     /* slot -> key                                           */
     uint64_t H, Hcap;
     float *dval, *dacc;     /* [R][Hcap][L] unsynced updates of each worker's replica */
-    uint8_t* dirty;         /* [Hcap] touched since the last sync                    */
+    uint8_t* dirty;         /* [R][Hcap] worker's replica touched since the last sync */
+    int merge_mean;         /* a sync adds the mean over the touching workers        */
     uint64_t* cnt;
     uint8_t* owner;         /* ORC_OWNER_DEFAULT = never moved: owner is key mod R   */
     uint64_t steps, syncs, hot_hits, cold_hits;
@@ -296,7 +297,7 @@ static void push_row(orc_store* s, uint32_t q, uint32_t k, int which, const floa
     if (sl < 0) dst = (which ? s->acc : s->val) + (uint64_t)k * s->L;
     else {
         dst = (which ? s->dacc : s->dval) + ((uint64_t)q * s->Hcap + (uint64_t)sl) * s->L;
-        s->dirty[sl] = 1;
+        s->dirty[(uint64_t)q * s->Hcap + (uint64_t)sl] = 1;
     }
     for (uint32_t e = 0; e < s->L; ++e) dst[e] += d[e];
 }
@@ -347,7 +348,9 @@ int orc_sync(void* p)
     orc_store* s = (orc_store*)p;
     if (s->H == 0) return ORC_OK;              /* nothing replicated: no work at all */
     for (uint64_t sl = 0; sl < s->H; ++sl) {
-        if (!s->dirty[sl]) continue;
+        uint32_t touched = 0;                  /* workers whose replica of the slot was written */
+        for (uint32_t r = 0; r < s->R; ++r) touched += s->dirty[(uint64_t)r * s->Hcap + sl] != 0;
+        if (!touched) continue;
         uint32_t k = s->hot_keys[sl];
         for (int which = 0; which <= (s->with_acc ? 1 : 0); ++which) {
             float* row = (which ? s->acc : s->val) + (uint64_t)k * s->L;
@@ -358,10 +361,13 @@ int orc_sync(void* p)
                     float* d = slab + ((uint64_t)r * s->Hcap + sl) * s->L + e;
                     t += *d; *d = 0.0f;
                 }
+                /* option (not in the paper; it damps the summed duplicate updates of very
+                 * frequent keys): the mean over the workers that pushed, not the sum      */
+                if (s->merge_mean) t = t / (float)touched;
                 row[e] += t;
             }
         }
-        s->dirty[sl] = 0;
+        for (uint32_t r = 0; r < s->R; ++r) s->dirty[(uint64_t)r * s->Hcap + sl] = 0;
     }
     s->syncs++;
     return ORC_OK;
@@ -427,8 +433,8 @@ int orc_set_management(void* p, const uint32_t* keys, uint64_t n, int technique)
             s->dval = (float*)calloc((uint64_t)s->R * cap * s->L, sizeof(float));
             s->dacc = s->with_acc ? (float*)calloc((uint64_t)s->R * cap * s->L, sizeof(float)) : NULL;
             s->hot_keys = (uint32_t*)realloc(s->hot_keys, cap * sizeof(uint32_t));
-            s->dirty = (uint8_t*)realloc(s->dirty, cap);
-            memset(s->dirty, 0, cap);
+            s->dirty = (uint8_t*)realloc(s->dirty, (uint64_t)s->R * cap);
+            memset(s->dirty, 0, (uint64_t)s->R * cap);
             s->Hcap = cap;
         }
         for (uint64_t i = 0; i < n; ++i) {
@@ -709,6 +715,11 @@ static double softplus(double x) { return (x > 0 ? x : 0) + log1p(exp(-fabs(x)))
  * d * (factor * mean / |d|); before any such update has been applied nothing
  * is clipped.  The step's own norms join the statistics when the step ends.   */
 typedef struct { double sum; uint64_t cnt; } clip_step;
+
+void orc_set_merge_mean(void* p, int on)
+{
+    ((orc_store*)p)->merge_mean = on ? 1 : 0;
+}
 
 void orc_set_clipping(void* p, double factor)
 {

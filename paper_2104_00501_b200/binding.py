@@ -32,7 +32,8 @@ EXPORTS = [
 class Config(C.Structure):
     _fields_ = [("workers", C.c_uint32), ("sync_interval", C.c_uint32), ("deterministic", C.c_uint32),
                 ("with_adagrad", C.c_uint32), ("count_accesses", C.c_uint32), ("track_ownership", C.c_uint32),
-                ("smem_hot_rows", C.c_uint32), ("sync_period_us", C.c_uint32), ("clip_factor", C.c_float), ("reserved", C.c_uint32 * 7)]
+                ("smem_hot_rows", C.c_uint32), ("sync_period_us", C.c_uint32), ("clip_factor", C.c_float),
+                ("max_device_mib", C.c_uint32), ("first_epoch", C.c_uint32), ("merge_mean", C.c_uint32), ("reserved", C.c_uint32 * 4)]
 
 
 class NupsError(RuntimeError):
@@ -134,11 +135,13 @@ class Store:
     """One parameter store on the current CUDA device."""
 
     def __init__(self, num_keys, value_len, workers=8, sync_interval=1, deterministic=False, with_adagrad=False,
-                 count_accesses=False, track_ownership=False, smem_hot_rows=0, sync_period_us=0, clip_factor=0.0):
+                 count_accesses=False, track_ownership=False, smem_hot_rows=0, sync_period_us=0, clip_factor=0.0,
+                 max_device_mib=0, first_epoch=0, merge_mean=False):
         self._l = load()
         cfg = Config(workers=workers, sync_interval=sync_interval, deterministic=int(deterministic),
                      with_adagrad=int(with_adagrad), count_accesses=int(count_accesses),
-                     track_ownership=int(track_ownership), smem_hot_rows=smem_hot_rows, sync_period_us=sync_period_us, clip_factor=clip_factor)
+                     track_ownership=int(track_ownership), smem_hot_rows=smem_hot_rows, sync_period_us=sync_period_us,
+                     clip_factor=clip_factor, max_device_mib=max_device_mib, first_epoch=first_epoch, merge_mean=int(merge_mean))
         h = C.c_void_p()
         self._s = None
         self._chk(self._l.nups_create(num_keys, value_len, C.byref(cfg), C.byref(h)), "nups_create")

@@ -54,6 +54,7 @@ struct View {
     uint32_t L4;               // floats per row / 4
     uint32_t R;
     uint32_t count;            // count accesses?
+    uint32_t merge_mean;       // merges add the mean over the workers that touched a slot, not the sum
     uint32_t epoch_tag;        // number of the running call, shifted into the upper 24 bits of an ownership word
     float clip_factor;         // > 0: updates to replicated keys are clipped at this multiple of their mean norm
 };
@@ -99,6 +100,7 @@ struct nups_store {
     double* loss_partial;
     char* scratch;
     size_t scratch_bytes;
+    size_t dev_bytes, dev_cap; // device memory held by the store, and its limit (0 = none)
     uint32_t* negs_buf;        // negatives drawn for the workload steps, possibly several batches ahead
     uint64_t negs_cap;
     uint32_t* last_negs;       // the slice of negs_buf that the most recent step used
@@ -155,6 +157,10 @@ enum { NUPS_TIMED_PULL = 0, NUPS_TIMED_PUSH = 1, NUPS_TIMED_STEP = 2, NUPS_TIMED
 void nups_time_begin(nups_store* s, cudaStream_t st, int kind);
 void nups_time_end(nups_store* s, cudaStream_t st);
 nups_status nups_scratch(nups_store* s, size_t bytes, char** out);     // grow-only scratch, 256-byte aligned
+// Device memory of a store goes through these two so that the store's own limit can refuse a request before the
+// allocator is asked.  nups_dev_alloc leaves *p null on failure.
+nups_status nups_dev_alloc(nups_store* s, void** p, size_t bytes);
+void nups_dev_free(nups_store* s, void* p, size_t bytes);
 nups_status nups_new_epoch(nups_store* s, cudaStream_t st);          // call before taking the view of a call that moves keys
 
 // background.cu

@@ -145,14 +145,15 @@ extern "C" nups_status nups_register_distribution(nups_store* s, uint32_t key_ba
         unsigned long long* inc = (unsigned long long*)sc; sc += align256(n * 8);
         uint32_t* hidx = (uint32_t*)sc; sc += align256(n * 4);
         unsigned long long* d_nL = (unsigned long long*)sc; sc += 256;
-        if (cudaMalloc(&d.table, n * sizeof(AliasEntry)) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        rc = nups_dev_alloc(s, &d.table, n * sizeof(AliasEntry));
+        if (rc != NUPS_OK) return rc;
         unsigned g = grid_for(n, 256);
         alias_classify_kernel<<<g, 256, 0, st>>>(d_weights, n, W, lrank, dex, sex);
         LAUNCH_CHECK(s);
         rc = nups_scan_u64(s, lrank, lrank, n, d_nL, sc, st);
         if (rc == NUPS_OK) rc = nups_scan_u64(s, dex, dex, n, nullptr, sc, st);
         if (rc == NUPS_OK) rc = nups_scan_u64(s, sex, sex, n, nullptr, sc, st);
-        if (rc != NUPS_OK) { cudaFree(d.table); return rc; }
+        if (rc != NUPS_OK) { nups_dev_free(s, d.table, n * sizeof(AliasEntry)); return rc; }
         unsigned long long nL = 0;
         CK(cudaMemcpyAsync(&nL, d_nL, 8, cudaMemcpyDeviceToHost, st));
         CK(cudaStreamSynchronize(st));
@@ -162,7 +163,10 @@ extern "C" nups_status nups_register_distribution(nups_store* s, uint32_t key_ba
         LAUNCH_CHECK(s);
         CK(cudaStreamSynchronize(st));
     }
-    if (cudaMalloc(&d.off, 2 * s->R * 8) != cudaSuccess) { cudaGetLastError(); cudaFree(d.table); return NUPS_ENOMEM; }
+    if (nups_dev_alloc(s, (void**)&d.off, 2 * s->R * 8) != NUPS_OK) {
+        nups_dev_free(s, d.table, d.table ? n * sizeof(AliasEntry) : 0);
+        return NUPS_ENOMEM;
+    }
     CK(cudaMemsetAsync(d.off, 0, 2 * s->R * 8, st));
     CK(cudaStreamSynchronize(st));
     d.used = 1;
@@ -237,16 +241,19 @@ static size_t handle_bytes(uint64_t N, uint32_t R, int level)
     if (level == NUPS_LONGTERM) b += align256(N * 4) + 3 * align256((size_t)R * 16) + 2 * align256((N / 32 + R + 2) * 4);
     return b;
 }
-static HandleView handle_view(char* buf, uint64_t N, uint32_t R)
+static HandleView handle_view(char* buf, uint64_t N, uint32_t R, int level)
 {
     HandleView h;
+    memset(&h, 0, sizeof(h));
     h.keys = (uint32_t*)buf; buf += align256(N * 4);
-    h.post = (uint32_t*)buf; buf += align256(N * 4);
-    h.state = (uint4*)buf; buf += align256((size_t)R * 16);
-    h.prev = (uint4*)buf; buf += align256((size_t)R * 16);
-    h.walk = (uint4*)buf; buf += align256((size_t)R * 16);
-    h.flags = (uint32_t*)buf; buf += align256((N / 32 + R + 2) * 4);
-    h.prefix = (uint32_t*)buf;
+    if (level == NUPS_LONGTERM) {
+        h.post = (uint32_t*)buf; buf += align256(N * 4);
+        h.state = (uint4*)buf; buf += align256((size_t)R * 16);
+        h.prev = (uint4*)buf; buf += align256((size_t)R * 16);
+        h.walk = (uint4*)buf; buf += align256((size_t)R * 16);
+        h.flags = (uint32_t*)buf; buf += align256((N / 32 + R + 2) * 4);
+        h.prefix = (uint32_t*)buf; buf += align256((N / 32 + R + 2) * 4);
+    }
     return h;
 }
 
@@ -488,10 +495,12 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
     if (id < 0) return NUPS_ENOMEM;
     Handle& h = s->handle[id];
     if (h.cap < need) {
-        if (h.buf) CK(cudaFree(h.buf));
-        h.buf = nullptr; h.cap = 0;
         size_t want = need + need / 4;
-        if (cudaMalloc(&h.buf, want) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        if (s->dev_cap && (want > s->dev_cap || s->dev_bytes - h.cap > s->dev_cap - want)) return NUPS_ENOMEM;
+        nups_dev_free(s, h.buf, h.cap);
+        h.buf = nullptr; h.cap = 0;
+        nups_status rc = nups_dev_alloc(s, (void**)&h.buf, want);
+        if (rc != NUPS_OK) return rc;
         h.cap = want;
     }
     const bool reuse = d.level == NUPS_BOUNDED || d.level == NUPS_LONGTERM;
@@ -500,7 +509,7 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
         nups_status rc = nups_new_epoch(s, st);
         if (rc != NUPS_OK) return rc;
     }
-    HandleView hv = handle_view(h.buf, N, s->R);
+    HandleView hv = handle_view(h.buf, N, s->R, d.level);
     DrawParams p = draw_params(d);
     View v = nups_view(s);
     const unsigned long long* off_cur = d.off + (size_t)d.cur * s->R;
@@ -784,7 +793,7 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         if (rc != NUPS_OK) return rc;
     }
     View v = nups_view(s);
-    HandleView hv = handle_view(h.buf, h.N, s->R);
+    HandleView hv = handle_view(h.buf, h.N, s->R, d.level);
     DrawParams p = draw_params(d);
     if (d.level == NUPS_LONGTERM) {
         // sub-handles overlapped by [cursor, cursor + n)
@@ -943,10 +952,12 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
     const uint32_t batches = (plain && !s->cfg.deterministic && !s->cfg.count_accesses && !s->own &&
                               N * NUPS_SAMPLE_AHEAD < (1ull << 28)) ? NUPS_SAMPLE_AHEAD : 1;
     if (N * batches > s->negs_cap) {
-        if (s->negs_buf) CK(cudaFree(s->negs_buf));
-        s->negs_buf = nullptr; s->negs_cap = 0;
         uint64_t want = N * batches + N / 4;
-        if (cudaMalloc(&s->negs_buf, want * 4) != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        if (s->dev_cap && (want * 4 > s->dev_cap || s->dev_bytes - s->negs_cap * 4 > s->dev_cap - want * 4)) return NUPS_ENOMEM;
+        nups_dev_free(s, s->negs_buf, s->negs_cap * 4);
+        s->negs_buf = nullptr; s->negs_cap = 0;
+        rc = nups_dev_alloc(s, (void**)&s->negs_buf, want * 4);
+        if (rc != NUPS_OK) return rc;
         s->negs_cap = want;
     }
     s->last_negs = s->negs_buf;

@@ -296,6 +296,197 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
 }
 
 // ---------------------------------------------------------------------------------------------
+// skip-gram, fast mode with three negatives per pair: rows in registers, runs of one centre word summed.
+// A warp takes a stretch of consecutive pairs of the launch.  Pairs arrive centre by centre (a position of
+// the token stream is paired with every position of its window in turn), so the centre word stays the same
+// over a run of pairs: its row is read once per run and kept in registers, the updates that the run's pairs
+// make to it are summed in registers and added once when the run ends.  All pairs of a run therefore see the
+// centre's row from before the run, which is what the batch semantics of the deterministic mode gives every
+// pair of a step; the rows of context words and negatives are read and updated pair by pair as before.
+// The four other rows of a pair go straight from global memory into registers (lane l owns the 16-byte chunks
+// l, l + 32, ...), the four scores are reduced together (6 shuffles instead of 20), every lane then forms its
+// chunks of the updates.  Keys and replica slots are looked up 32 pairs at a time, one pair per lane.
+// ---------------------------------------------------------------------------------------------
+constexpr int SGNS_RUN_THREADS = 128;
+constexpr int SGNS_RUN_BLOCKS = 4;         // resident blocks per multiprocessor: 128 registers a thread (3 blocks at 158: 103 vs 95 us per launch)
+
+template <bool HOT, int CH>
+__global__ void __launch_bounds__(SGNS_RUN_THREADS, SGNS_RUN_BLOCKS)
+sgns_runs_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restrict__ context,
+                 const uint32_t* __restrict__ negs, uint64_t n, float lr, float* __restrict__ loss_out, uint32_t group,
+                 unsigned long long* __restrict__ loss_acc)
+{
+    constexpr unsigned FULL = 0xFFFFFFFFu;
+    constexpr int K = 3;
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L4 = v.L4;
+    const uint64_t total = n * group;
+    const uint64_t stretch = (total + nwarps - 1) / nwarps;
+    const uint64_t first = warp * stretch < total ? warp * stretch : total;
+    const uint64_t last = first + stretch < total ? first + stretch : total;          // this warp's pairs: [first, last)
+    const float4* val4 = reinterpret_cast<const float4*>(v.val);
+    const float4* slab4 = reinterpret_cast<const float4*>(v.dval);
+
+    // one window = 32 consecutive pairs, lane l holds pair l: keys of the five roles (all invalid when one is) and slots
+    struct Window { uint32_t k[K + 2]; int s[K + 2]; };                              // roles: context, negatives, centre
+    auto load_window = [&](uint64_t base) {
+        Window w;
+#pragma unroll
+        for (int r = 0; r < K + 2; ++r) { w.k[r] = NUPS_INVALID_KEY; w.s[r] = -1; }
+        const uint64_t e = base + lane;
+        if (e < last) {
+            uint32_t k[K + 2];
+            k[0] = context[e];
+#pragma unroll
+            for (int j = 0; j < K; ++j) k[1 + j] = negs[e * K + j];
+            k[K + 1] = center[e];
+            bool ok = true;
+#pragma unroll
+            for (int r = 0; r < K + 2; ++r) ok = ok && k[r] < v.num_keys;
+            if (ok) {
+#pragma unroll
+                for (int r = 0; r < K + 2; ++r) { w.k[r] = k[r]; if (HOT) { const int sl = __ldg(v.slot_of + k[r]); w.s[r] = sl < 0 ? -1 : sl; } }
+            } else {
+                flag_bad_key(v);
+            }
+        }
+        return w;
+    };
+    auto fetch_row = [&](float4 (&dst)[CH], const float4* row) {
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            const uint32_t c = lane + 32 * m;
+            dst[m] = c < L4 ? __ldg(row + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    auto fold_pending = [&](float4 (&dst)[CH], const float4* pend) {
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            const uint32_t c = lane + 32 * m;
+            if (c < L4) dst[m] = add4(dst[m], pend[c]);
+        }
+    };
+
+    Window cur = load_window(first), nxt = load_window(first + 32);
+    float4 a[CH], held[CH];                                 // the run's centre row; the summed updates to it
+    float* held_dst = nullptr;                              // where they go: replica row or stored row
+    auto flush_held = [&]() {
+        if (!held_dst) return;
+#pragma unroll
+        for (int m = 0; m < CH; ++m) {
+            const uint32_t c = lane + 32 * m;
+            if (c < L4) red_add_v4(held_dst + 4 * c, held[m]);
+        }
+        held_dst = nullptr;
+    };
+    // item index within its step, its worker and the worker's last item, kept up as the pairs go by
+    uint32_t step = (uint32_t)((first < total ? first : 0) / n);
+    uint64_t i = (first < total ? first : 0) - (uint64_t)step * n;
+    uint32_t q = worker_of_item(i, n, v.R);
+    uint64_t q_end = worker_first_item(q + 1, n, v.R);
+    float step_loss = 0.f;                                  // this lane's share of the running step's loss
+    double my_loss = 0.0;
+    auto close_step = [&]() {
+        const float sum = warp_sum(step_loss);
+        step_loss = 0.f;
+        if (loss_acc) {
+            if (lane == 0 && sum != 0.f)
+                atomicAdd(loss_acc + (uint32_t)(warp % LOSS_SLOTS) * LOSS_STEPS + step,
+                          (unsigned long long)llrintf(fminf(sum, 4.0e9f / 65536.f) * 65536.f));
+        } else {
+            my_loss += (double)sum;
+        }
+    };
+    for (uint64_t base = first; base < last; base += 32) {
+        const uint32_t in_window = (uint32_t)min((uint64_t)32, last - base);
+        for (uint32_t t = 0; t < in_window; ++t, ++i) {
+            if (i >= n) { close_step(); i -= n; ++step; q = 0; q_end = worker_first_item(1, n, v.R); }
+            while (i >= q_end) q_end = worker_first_item(++q + 1, n, v.R);
+            uint32_t key[K + 2];
+            int slot[K + 2];
+#pragma unroll
+            for (int r = 0; r < K + 2; ++r) {
+                key[r] = __shfl_sync(FULL, cur.k[r], t);
+                slot[r] = HOT ? __shfl_sync(FULL, cur.s[r], t) : -1;
+            }
+            if (key[K + 1] == NUPS_INVALID_KEY) continue;                      // a key out of range: flagged at the lookup
+            // destination rows: the worker's replica row of a replicated key, else the stored row
+            float* dst[K + 2];
+#pragma unroll
+            for (int r = 0; r < K + 2; ++r)
+                dst[r] = slot[r] >= 0 ? v.dval + ((uint64_t)q * v.Hcap + (unsigned)slot[r]) * L4 * 4
+                                      : v.val + (uint64_t)key[r] * L4 * 4;
+            float4 u[K + 1][CH];
+#pragma unroll
+            for (int j = 0; j <= K; ++j) fetch_row(u[j], val4 + (uint64_t)key[j] * L4);
+            if (dst[K + 1] != held_dst) {                                        // a new run: another centre word or worker
+                flush_held();
+                fetch_row(a, val4 + (uint64_t)key[K + 1] * L4);
+                if (HOT && slot[K + 1] >= 0) fold_pending(a, reinterpret_cast<const float4*>(dst[K + 1]));
+#pragma unroll
+                for (int m = 0; m < CH; ++m) held[m] = make_float4(0.f, 0.f, 0.f, 0.f);
+                held_dst = dst[K + 1];
+                if (HOT && slot[K + 1] >= 0 && lane == 0) mark_dirty(v, q, slot[K + 1]);
+            }
+            if (HOT) {
+#pragma unroll
+                for (int j = 0; j <= K; ++j)
+                    if (slot[j] >= 0) fold_pending(u[j], reinterpret_cast<const float4*>(dst[j]));
+            }
+            if (HOT && lane == 0) {
+#pragma unroll
+                for (int j = 0; j <= K; ++j)
+                    if (slot[j] >= 0) mark_dirty(v, q, slot[j]);
+            }
+            // the four scores at once: after the halving steps lane l holds score 2 * bit4(l) + bit3(l)
+            float x[K + 1];
+#pragma unroll
+            for (int j = 0; j <= K; ++j) {
+                float d = 0.f;
+#pragma unroll
+                for (int m = 0; m < CH; ++m) d += a[m].x * u[j][m].x + a[m].y * u[j][m].y + a[m].z * u[j][m].z + a[m].w * u[j][m].w;
+                x[j] = d;
+            }
+            {
+                const bool up16 = (lane & 16) != 0, up8 = (lane & 8) != 0;
+                const float k0 = (up16 ? x[2] : x[0]) + __shfl_xor_sync(FULL, up16 ? x[0] : x[2], 16);
+                const float k1 = (up16 ? x[3] : x[1]) + __shfl_xor_sync(FULL, up16 ? x[1] : x[3], 16);
+                float y = (up8 ? k1 : k0) + __shfl_xor_sync(FULL, up8 ? k0 : k1, 8);
+                y += __shfl_xor_sync(FULL, y, 4);
+                y += __shfl_xor_sync(FULL, y, 2);
+                y += __shfl_xor_sync(FULL, y, 1);
+                const uint32_t mine = ((lane >> 4) & 1u) * 2 + ((lane >> 3) & 1u);      // the score this lane holds
+                y = clamp30(y);
+                const float g_l = sigmoidf_(y) - (mine == 0 ? 1.f : 0.f);
+                if ((lane & 7u) == 0) step_loss += mine == 0 ? softplusf_(-y) : softplusf_(y);
+#pragma unroll
+                for (int j = 0; j <= K; ++j) x[j] = __shfl_sync(FULL, g_l, 16 * (j >> 1) + 8 * (j & 1));   // x[j] = g_j now
+            }
+#pragma unroll
+            for (int m = 0; m < CH; ++m) {
+                const uint32_t c = lane + 32 * m;
+                if (c >= L4) continue;
+                float4 gv = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                for (int j = 0; j <= K; ++j) {
+                    const float sc = -lr * x[j];
+                    red_add_v4(dst[j] + 4 * c, make_float4(sc * a[m].x, sc * a[m].y, sc * a[m].z, sc * a[m].w));
+                    gv.x += x[j] * u[j][m].x; gv.y += x[j] * u[j][m].y; gv.z += x[j] * u[j][m].z; gv.w += x[j] * u[j][m].w;
+                }
+                held[m].x += -lr * gv.x; held[m].y += -lr * gv.y; held[m].z += -lr * gv.z; held[m].w += -lr * gv.w;
+            }
+        }
+        cur = nxt;
+        nxt = load_window(base + 64);
+    }
+    flush_held();
+    close_step();
+    if (!loss_acc) loss_finish(v, my_loss, n, loss_out);
+}
+
+// ---------------------------------------------------------------------------------------------
 // ComplEx with AdaGrad.  Rows are [re(0..d-1) | im(0..d-1)], d = L/2 (even).  One block of 128 threads
 // works on one triple at a time.  All 2 * (3 + K) rows of the triple (values and accumulators) are brought
 // into shared memory as they lie in memory, by asynchronous 16-byte copies that are all in flight at once
@@ -904,6 +1095,30 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
                                unsigned long long* loss_acc, cudaStream_t st)
 {
     View v = nups_view(s);
+    const bool clip_on = s->cfg.clip_factor > 0.f && s->H;
+    if (K == 3 && !s->cfg.deterministic && !s->cfg.count_accesses && !s->own && !clip_on) {
+        // fast mode, nothing to count or move: the kernel that keeps rows in registers and sums runs of one centre word
+        cudaError_t e = cudaSuccess;
+        DISPATCH_CH(v.L4, {
+            auto kern = s->H ? sgns_runs_kernel<true, CH> : sgns_runs_kernel<false, CH>;
+            int fit = 0;
+            e = resident_blocks((const void*)kern, 0, &fit, [&](int* out) {
+                return cudaOccupancyMaxActiveBlocksPerMultiprocessor(out, kern, SGNS_RUN_THREADS, 0); });
+            if (e == cudaSuccess) {
+                if (fit < 1) fit = 1;
+                const uint64_t items = n * group;
+                const uint64_t blocks_needed = (items + SGNS_RUN_THREADS / 32 - 1) / (SGNS_RUN_THREADS / 32);
+                const uint64_t cap = (uint64_t)s->sm_count * (unsigned)fit;
+                const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
+                nups_time_begin(s, st, NUPS_TIMED_STEP);
+                kern<<<grid, SGNS_RUN_THREADS, 0, st>>>(v, d_center, d_context, s->last_negs, n, lr, d_loss_out, group, loss_acc);
+                nups_time_end(s, st);
+            }
+        });
+        if (e != cudaSuccess) return nups_cuda_fail(e, "skip-gram kernel set-up");
+        LAUNCH_CHECK(s);
+        return NUPS_OK;
+    }
     const uint32_t cols = ((v.L4 + 31) / 32) * 32, per = K + 2;    // a warp's staging area: per rows of cols chunks
     const size_t smem = (size_t)per * cols * sizeof(float4) * SGNS_WARPS;
     if (smem > (size_t)s->max_smem - 4096) return NUPS_EINVAL;

@@ -38,18 +38,42 @@ View nups_view(const nups_store* s)
     v.cnt = s->cnt; v.own = s->own; v.epoch_tag = s->epoch << 8; v.st = s->st; v.loss_partial = s->loss_partial;
     v.num_keys = s->num_keys; v.Hcap = s->Hcap; v.H = (uint32_t)s->H; v.L4 = s->L / 4; v.R = s->R;
     v.count = s->cfg.count_accesses;
+    v.merge_mean = s->cfg.merge_mean;
     v.clip_factor = s->cfg.clip_factor;
     return v;
+}
+
+nups_status nups_dev_alloc(nups_store* s, void** p, size_t bytes)
+{
+    *p = nullptr;
+    if (bytes == 0) return NUPS_OK;
+    if (s->dev_cap && (bytes > s->dev_cap || s->dev_bytes > s->dev_cap - bytes)) return NUPS_ENOMEM;   // the store's own limit
+    if (cudaMalloc(p, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        *p = nullptr;
+        return NUPS_ENOMEM;
+    }
+    s->dev_bytes += bytes;
+    return NUPS_OK;
+}
+
+void nups_dev_free(nups_store* s, void* p, size_t bytes)
+{
+    if (!p) return;
+    cudaFree(p);                                   // waits for work that may still use it
+    s->dev_bytes -= bytes < s->dev_bytes ? bytes : s->dev_bytes;
 }
 
 nups_status nups_scratch(nups_store* s, size_t bytes, char** out)
 {
     if (bytes > s->scratch_bytes) {
         size_t want = bytes + bytes / 4 + (1u << 20);
-        if (s->scratch) CK(cudaFree(s->scratch));     // waits for work that may still use it
+        // the limit is judged with the old buffer already handed back; on refusal the old buffer stays
+        if (s->dev_cap && (want > s->dev_cap || s->dev_bytes - s->scratch_bytes > s->dev_cap - want)) return NUPS_ENOMEM;
+        nups_dev_free(s, s->scratch, s->scratch_bytes);
         s->scratch = nullptr; s->scratch_bytes = 0;
-        cudaError_t e = cudaMalloc(&s->scratch, want);
-        if (e != cudaSuccess) { cudaGetLastError(); return NUPS_ENOMEM; }
+        nups_status rc = nups_dev_alloc(s, (void**)&s->scratch, want);
+        if (rc != NUPS_OK) return rc;
         s->scratch_bytes = want;
     }
     *out = s->scratch;
@@ -169,6 +193,15 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     if (c.workers > 254) return NUPS_EINVAL;
     if (c.sync_period_us && c.deterministic) return NUPS_EINVAL;
     if (!(c.clip_factor >= 0.f)) return NUPS_EINVAL;
+    if (c.merge_mean > 1 || (c.merge_mean && c.sync_period_us)) return NUPS_EINVAL;
+    if (c.first_epoch > 0xFFFFFFu) return NUPS_EINVAL;
+    // what the store holds from the start: tables, technique bitmap, slot map, counts, ownership words, status, loss words
+    const size_t table_bytes = (size_t)num_keys * value_len * sizeof(float);
+    const size_t bits_bytes = ((num_keys + 31) / 32) * 4, loss_bytes = 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double);
+    const size_t need = table_bytes * (c.with_adagrad ? 2 : 1) + bits_bytes + num_keys * 4 + num_keys * 8 +
+                        (c.track_ownership ? num_keys * 4 : 0) + sizeof(DevStat) + loss_bytes;
+    const size_t cap = (size_t)c.max_device_mib << 20;
+    if (cap && need > cap) return NUPS_ENOMEM;              // the store's own limit, judged before the device is touched
     int dev = 0, count = 0;
     if (cudaGetDeviceCount(&count) != cudaSuccess || count == 0) {
         snprintf(g_nups_cuda_err, sizeof(g_nups_cuda_err), "no CUDA device");
@@ -179,20 +212,19 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     nups_store* s = (nups_store*)calloc(1, sizeof(nups_store));
     if (!s) return NUPS_ENOMEM;
     s->num_keys = num_keys; s->L = value_len; s->R = c.workers; s->cfg = c; s->device = dev;
+    s->dev_cap = cap;
+    s->epoch = c.first_epoch;
     s->ahead_dist = -1;
     cudaDeviceGetAttribute(&s->sm_count, cudaDevAttrMultiProcessorCount, dev);
     cudaDeviceGetAttribute(&s->max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    size_t table_bytes = (size_t)num_keys * value_len * sizeof(float);
-    bool ok = cudaMalloc(&s->val, table_bytes) == cudaSuccess;
-    if (ok && c.with_adagrad) ok = cudaMalloc(&s->acc, table_bytes) == cudaSuccess;
-    ok = ok && cudaMalloc(&s->hot_bits, ((num_keys + 31) / 32) * 4) == cudaSuccess;
-    ok = ok && cudaMalloc(&s->slot_of, num_keys * 4) == cudaSuccess;
-    ok = ok && cudaMalloc(&s->cnt, num_keys * 8) == cudaSuccess;
-    ok = ok && cudaMalloc(&s->st, sizeof(DevStat)) == cudaSuccess;
-    ok = ok && cudaMalloc(&s->loss_partial, 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double)) == cudaSuccess;
-    if (ok && c.track_ownership) {
-        ok = cudaMalloc(&s->own, num_keys * 4) == cudaSuccess;
-    }
+    bool ok = nups_dev_alloc(s, (void**)&s->val, table_bytes) == NUPS_OK;
+    if (ok && c.with_adagrad) ok = nups_dev_alloc(s, (void**)&s->acc, table_bytes) == NUPS_OK;
+    ok = ok && nups_dev_alloc(s, (void**)&s->hot_bits, bits_bytes) == NUPS_OK;
+    ok = ok && nups_dev_alloc(s, (void**)&s->slot_of, num_keys * 4) == NUPS_OK;
+    ok = ok && nups_dev_alloc(s, (void**)&s->cnt, num_keys * 8) == NUPS_OK;
+    ok = ok && nups_dev_alloc(s, (void**)&s->st, sizeof(DevStat)) == NUPS_OK;
+    ok = ok && nups_dev_alloc(s, (void**)&s->loss_partial, loss_bytes) == NUPS_OK;
+    if (ok && c.track_ownership) ok = nups_dev_alloc(s, (void**)&s->own, num_keys * 4) == NUPS_OK;
     if (!ok) {
         cudaGetLastError();
         nups_destroy(s);
@@ -413,17 +445,18 @@ gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const floa
     const uint64_t L = (uint64_t)v.L4 * 4;
     const uint64_t stride = nwarps * 32;
     uint64_t base = warp * 32;
-    uint32_t key_a = base + lane < n ? __ldg(keys + base + lane) : 0u;
-    uint32_t key_b = base + stride + lane < n ? __ldg(keys + base + stride + lane) : 0u;
+    const uint64_t end = n;
+    uint32_t key_a = base + lane < end ? __ldg(keys + base + lane) : 0u;
+    uint32_t key_b = base + stride + lane < end ? __ldg(keys + base + stride + lane) : 0u;
     uint32_t bits_a = (HOT && key_a < v.num_keys) ? __ldg(v.hot_bits + (key_a >> 5)) : 0u;
-    for (; base < n; base += stride) {
+    for (; base < end; base += stride) {
         const uint64_t i = base + lane;
-        const bool in = i < n;
+        const bool in = i < end;
         const uint32_t key = key_a;
         const uint32_t bits = bits_a;
         key_a = key_b;
         bits_a = (HOT && key_a < v.num_keys) ? __ldg(v.hot_bits + (key_a >> 5)) : 0u;
-        key_b = base + 2 * stride + lane < n ? __ldg(keys + base + 2 * stride + lane) : 0u;
+        key_b = base + 2 * stride + lane < end ? __ldg(keys + base + 2 * stride + lane) : 0u;
         const bool valid = in && key < v.num_keys;
         if (in && !valid) flag_bad_key(v);
         if (keys_copy && in) keys_copy[i] = key;                   // PullSample hands the keys out as well
@@ -445,7 +478,7 @@ gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const floa
                 if (cold_m) atomicAdd(&v.st->cold_hits, (unsigned long long)__popc(cold_m));
             }
         }
-        const int rows = (int)min((uint64_t)32, n - base);
+        const int rows = (int)min((uint64_t)32, end - base);
         for (int r0 = 0; r0 < rows; r0 += UNR * RPI) {
             uint32_t so[UNR], po[UNR];
             F8 a[UNR];
@@ -1013,6 +1046,12 @@ __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
                 }
             }
         }
+        if (v.merge_mean) {                                   // the mean over the workers that touched the slot
+            uint32_t touched = 0;
+            for (uint32_t r = 0; r < v.R; ++r) touched += v.dirty[(size_t)r * v.Hcap + slot] != 0u;
+            const float by = (float)touched;
+            sum = make_float4(__fdiv_rn(sum.x, by), __fdiv_rn(sum.y, by), __fdiv_rn(sum.z, by), __fdiv_rn(sum.w, by));
+        }
         float4* row = table + (uint64_t)key * L4 + c;
         *row = add4(*row, sum);
     }
@@ -1251,12 +1290,21 @@ static nups_status grow_hot(nups_store* s, uint64_t need)
     uint32_t* hk = nullptr;
     uint32_t* dirty = nullptr;
     float *dv = nullptr, *da = nullptr;
-    size_t slab = (size_t)s->R * cap * s->L * sizeof(float);
-    bool ok = cudaMalloc(&hk, cap * 4) == cudaSuccess && cudaMalloc(&dirty, (size_t)s->R * cap * 4) == cudaSuccess &&
-              cudaMalloc(&dv, slab) == cudaSuccess && (!s->acc || cudaMalloc(&da, slab) == cudaSuccess);
+    const size_t slab = (size_t)s->R * cap * s->L * sizeof(float);
+    const size_t slab_old = (size_t)s->R * s->Hcap * s->L * sizeof(float);
+    const size_t want = cap * 4 + (size_t)s->R * cap * 4 + slab * (s->acc ? 2 : 1);
+    const size_t held = s->Hcap * 4 + (size_t)s->R * s->Hcap * 4 + slab_old * (s->acc ? 2 : 1);
+    // old and new replicas exist side by side for a moment; the store's limit is judged on what stays
+    if (s->dev_cap && (want > s->dev_cap || s->dev_bytes - held > s->dev_cap - want)) return NUPS_ENOMEM;
+    const size_t cap_saved = s->dev_cap;
+    s->dev_cap = 0;
+    bool ok = nups_dev_alloc(s, (void**)&hk, cap * 4) == NUPS_OK &&
+              nups_dev_alloc(s, (void**)&dirty, (size_t)s->R * cap * 4) == NUPS_OK &&
+              nups_dev_alloc(s, (void**)&dv, slab) == NUPS_OK && (!s->acc || nups_dev_alloc(s, (void**)&da, slab) == NUPS_OK);
+    s->dev_cap = cap_saved;
     if (!ok) {
-        cudaGetLastError();
-        cudaFree(hk); cudaFree(dirty); cudaFree(dv); cudaFree(da);
+        nups_dev_free(s, hk, cap * 4); nups_dev_free(s, dirty, (size_t)s->R * cap * 4);
+        nups_dev_free(s, dv, slab); nups_dev_free(s, da, slab);
         return NUPS_ENOMEM;
     }
     // pending updates are all zero here (the caller merged them), so fresh zeroed slabs are enough
@@ -1265,7 +1313,8 @@ static nups_status grow_hot(nups_store* s, uint64_t need)
     CK(cudaMemset(dv, 0, slab));
     if (da) CK(cudaMemset(da, 0, slab));
     CK(cudaDeviceSynchronize());
-    cudaFree(s->hot_keys); cudaFree(s->dirty); cudaFree(s->dval); cudaFree(s->dacc);
+    nups_dev_free(s, s->hot_keys, s->Hcap * 4); nups_dev_free(s, s->dirty, (size_t)s->R * s->Hcap * 4);
+    nups_dev_free(s, s->dval, slab_old); nups_dev_free(s, s->dacc, slab_old);
     s->hot_keys = hk; s->dirty = dirty; s->dval = dv; s->dacc = da; s->Hcap = cap;
     return NUPS_OK;
 }

@@ -5,7 +5,7 @@ import torch
 
 from oracle import BOUNDED, CONFORM, LONGTERM, NONCONFORM, REPLICATE
 from paper_2104_00501_b200 import inputs
-from tests.common import dev_keys, host_keys, make_pair
+from tests.common import dev_f32, dev_keys, host_keys, make_pair
 
 pytestmark = pytest.mark.gpu
 
@@ -173,3 +173,34 @@ def test_full_pull_with_values_under_postponing_copies_the_rows_itself(L):
             assert np.array_equal(vs.cpu().numpy(), vo)
     allk = np.arange(nk, dtype=np.uint32)
     assert np.array_equal(s.owner_of(dev_keys(allk)).cpu().numpy(), np.array([o.owner_of(k) for k in allk]))
+
+
+@pytest.mark.parametrize("L,U,G,R", [(128, 16, 250, 8), (64, 4, 100, 3), (256, 16, 250, 8), (512, 3, 250, 2), (1024, 2, 40, 2)])
+def test_pooled_reuse_pull_sample_rows_are_what_each_worker_pulls(L, U, G, R):
+    # The rows that PullSample returns are exactly what the sub-handle's worker pulls at that moment: the stored row
+    # plus that worker's pending replica updates for a replicated key.  Pooled reuse (the same keys come back again and
+    # again), rows of 256 bytes to 4 KB, partial pulls cut inside pools and sub-handles, updates pushed (and left
+    # pending) between the partial pulls.
+    nk = 6000
+    rng = np.random.default_rng(L)
+    init = rng.standard_normal(size=(nk, L), dtype=np.float32)
+    w = inputs.zipf_integer_weights(5000, 1.0).numpy().astype(np.uint32)
+    o, s = make_pair(nk, L, R=R, init=init, deterministic=True, sync_interval=0)
+    hot = (300 + inputs.u32(inputs.zipf_key_of_rank(5000)[:40])).astype(np.uint32)      # the target's most frequent keys
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    do = o.register_distribution(300, w, 5000, BOUNDED, U=U, G=G, seed=21)
+    ds = s.register_distribution(300, dev_keys(w), 5000, BOUNDED, U=U, G=G, seed=21)
+    for N, cuts in ((20000, [20000]), (9001, [1, 130, 4000, 4870]), (U * G * R + 7, [U * G, U * G * (R - 1) + 7])):
+        ho, hs = o.prepare_sample(do, N), s.prepare_sample(ds, N)
+        for c in cuts:
+            # updates that stay pending in the workers' replicas (no merge): every worker sees its own only
+            keys = np.concatenate([hot, rng.integers(0, nk, 200).astype(np.uint32)])
+            delta = rng.standard_normal(size=(len(keys), L), dtype=np.float32)
+            o.push(keys, delta)
+            s.push(dev_keys(keys), dev_f32(delta))
+            ko, vo = o.pull_sample(ho, c)
+            ks, vs = s.pull_sample(hs, c)
+            assert np.array_equal(host_keys(ks), ko)
+            assert np.array_equal(vs.cpu().numpy(), vo)
+    assert s.status_check() == 0

@@ -69,3 +69,19 @@ def test_binding_config_mirrors_the_header_struct():
     assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL
     cfg = binding.Config(workers=255)
     assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL
+
+
+def test_the_stores_own_memory_limit_refuses_before_the_device_is_touched():
+    # 1000 keys x 64 floats need 256,000 bytes of table alone; with a 1 MiB limit a store of 10,000 keys cannot be
+    # created, and that is found out from the sizes alone: NUPS_ENOMEM even on a box without a device
+    lib = binding.load()
+    h = ctypes.c_void_p()
+    cfg = binding.Config(max_device_mib=1)
+    assert lib.nups_create(10_000, 64, ctypes.byref(cfg), ctypes.byref(h)) == binding.ENOMEM
+    assert not h.value
+    cfg = binding.Config(max_device_mib=1, with_adagrad=1)
+    assert lib.nups_create(2_000, 64, ctypes.byref(cfg), ctypes.byref(h)) == binding.ENOMEM      # two tables of 512,000 bytes
+    cfg = binding.Config(merge_mean=1, sync_period_us=50)
+    assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL
+    cfg = binding.Config(first_epoch=1 << 24)
+    assert lib.nups_create(10, 4, ctypes.byref(cfg), ctypes.byref(h)) == binding.EINVAL

@@ -188,3 +188,30 @@ def test_init_uniform_range_mean_and_determinism():
     assert np.array_equal(t, o2.table())
     o2.init_uniform(0, 43, 0.5)
     assert not np.array_equal(t, o2.table())
+
+
+def test_merge_mean_adds_the_mean_over_the_workers_that_pushed():
+    # closed form: a replicated key that two of four workers push to receives (d1 + d2) / 2 at the merge, a key that
+    # one worker pushes to twice receives both updates in full (one worker: mean = sum), a key that is not replicated
+    # is updated in place as always
+    from oracle import Oracle, REPLICATE
+    L, R = 4, 4
+    o = Oracle(8, L, workers=R)
+    o.set_merge_mean(True)
+    o.set_management(np.array([1, 2], np.uint32), REPLICATE)
+    d = np.array([[1.0, 2.0, 4.0, 8.0], [3.0, 2.0, 0.0, -8.0], [0.5, 0.5, 0.5, 0.5], [0.25, 0.0, 0.0, 0.0]], np.float32)
+    # four items, one per worker: workers 0 and 1 push to key 1, workers 2 and 3 to key 5 (not replicated)
+    o.push(np.array([1, 1, 5, 5], np.uint32), d)
+    # eight items, two per worker: worker 0 pushes twice to key 2
+    o.push(np.array([2, 2, 7, 7, 7, 7, 7, 7], np.uint32), np.concatenate([d[:2], np.zeros((6, L), np.float32)]))
+    assert not o.table()[1].any() and not o.table()[2].any()        # still pending in the replicas
+    o.sync()
+    np.testing.assert_array_equal(o.table()[1], (d[0] + d[1]) / 2)
+    np.testing.assert_array_equal(o.table()[2], d[0] + d[1])
+    np.testing.assert_array_equal(o.table()[5], d[2] + d[3])
+    # the flags were cleared: a second merge changes nothing, and a later single push counts one worker
+    o.sync()
+    np.testing.assert_array_equal(o.table()[1], (d[0] + d[1]) / 2)
+    o.push(np.array([1], np.uint32), d[3:4])
+    o.sync()
+    np.testing.assert_array_equal(o.table()[1], (d[0] + d[1]) / 2 + d[3])
