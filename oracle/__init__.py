@@ -15,39 +15,41 @@ import numpy as np
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "nups_oracle.c")
 _LIB = os.path.join(_HERE, "libnups_oracle.so")
+_LIB_F64 = os.path.join(_HERE, "libnups_oracle_f64.so")          # the same source with 8-byte values
 
 SINGLE, REPLICATE = 0, 1
 CONFORM, BOUNDED, LONGTERM, NONCONFORM = 1, 2, 3, 4
 OK, EINVAL, ENOMEM, EKEY, ESTATE = 0, -1, -2, -4, -5
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (strict IEEE: no contraction, no fast-math)."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+def build(force: bool = False, f64: bool = False) -> str:
+    """Compile the oracle with gcc (strict IEEE: no contraction, no fast-math); f64: the build with 8-byte values."""
+    out = _LIB_F64 if f64 else _LIB
+    if force or not os.path.exists(out) or os.path.getmtime(out) < os.path.getmtime(_SRC):
         cmd = ["gcc", "-O2", "-std=gnu11", "-fPIC", "-shared", "-ffp-contract=off", "-fno-fast-math",
-               "-Wall", "-Wextra", "-o", _LIB + ".tmp", _SRC, "-lm"]
+               "-Wall", "-Wextra"] + (["-DORC_REAL=double"] if f64 else []) + ["-o", out + ".tmp", _SRC, "-lm"]
         subprocess.run(cmd, check=True)
-        os.replace(_LIB + ".tmp", _LIB)
-    return _LIB
+        os.replace(out + ".tmp", out)
+    return out
 
 
-_lib = None
+_libs = {}
 
 _u32p = C.POINTER(C.c_uint32)
 _u64p = C.POINTER(C.c_uint64)
-_f32p = C.POINTER(C.c_float)
 
 
-def lib():
-    global _lib
-    if _lib is None:
-        L = C.CDLL(build())
+def lib(f64: bool = False):
+    """The oracle library with 4-byte (default) or 8-byte values; value buffers cross as untyped pointers."""
+    if f64 not in _libs:
+        L = C.CDLL(build(f64=f64))
+        _f32p = C.c_void_p           # `real*` in the C source: float or double, depending on the build
         sig = {
             "orc_philox4x32_10": (None, [_u32p, _u32p, _u32p]),
             "orc_alias_build": (C.c_uint64, [_u32p, C.c_uint64, _u64p, _u32p]),
             "orc_create": (C.c_void_p, [C.c_uint64, C.c_uint32, C.c_uint32, C.c_int, C.c_int, C.c_int, C.c_uint32]),
             "orc_destroy": (None, [C.c_void_p]),
-            "orc_table": (_f32p, [C.c_void_p, C.c_int]),
+            "orc_table": (C.c_void_p, [C.c_void_p, C.c_int]),
             "orc_counts": (_u64p, [C.c_void_p]),
             "orc_status": (C.c_int, [C.c_void_p]),
             "orc_num_hot": (C.c_uint64, [C.c_void_p]),
@@ -75,16 +77,19 @@ def lib():
             "orc_prepare_sample": (C.c_int64, [C.c_void_p, C.c_int, C.c_uint64]),
             "orc_pull_sample": (C.c_int, [C.c_void_p, C.c_int64, C.c_uint64, _u32p, _f32p]),
             "orc_step_sgns": (C.c_int, [C.c_void_p, _u32p, _u32p, C.c_uint64, C.c_int, C.c_uint32, C.c_float,
-                                        _f32p, _u32p]),
+                                        C.POINTER(C.c_float), _u32p]),
             "orc_step_complex": (C.c_int, [C.c_void_p, _u32p, _u32p, _u32p, C.c_uint64, C.c_int, C.c_uint32,
-                                           C.c_float, C.c_float, _f32p, _u32p]),
-            "orc_step_mf": (C.c_int, [C.c_void_p, _u32p, _u32p, _f32p, C.c_uint64, C.c_float, C.c_float, _f32p]),
+                                           C.c_float, C.c_float, C.POINTER(C.c_float), _u32p]),
+            "orc_step_mf": (C.c_int, [C.c_void_p, _u32p, _u32p, C.POINTER(C.c_float), C.c_uint64, C.c_float, C.c_float,
+                                      C.POINTER(C.c_float)]),
         }
         for name, (res, args) in sig.items():
             fn = getattr(L, name)
             fn.restype, fn.argtypes = res, args
-        _lib = L
-    return _lib
+        L.orc_value_bytes.restype, L.orc_value_bytes.argtypes = C.c_int, []
+        assert L.orc_value_bytes() == (8 if f64 else 4)
+        _libs[f64] = L
+    return _libs[f64]
 
 
 def _u32(a):
@@ -94,7 +99,7 @@ def _u32(a):
 
 def _f32(a):
     a = np.ascontiguousarray(a, dtype=np.float32)
-    return a, a.ctypes.data_as(_f32p)
+    return a, a.ctypes.data_as(C.POINTER(C.c_float))
 
 
 def philox4x32_10(ctr, key):
@@ -130,8 +135,10 @@ class Oracle:
     """One store with R logical workers; mirrors the C-ABI calls one to one."""
 
     def __init__(self, num_keys, value_len, workers=8, with_adagrad=False, count_accesses=False,
-                 track_ownership=False, sync_interval=1):
-        self._l = lib()
+                 track_ownership=False, sync_interval=1, value_bytes=4):
+        assert value_bytes in (4, 8)
+        self._l = lib(f64=value_bytes == 8)
+        self.dtype = np.float64 if value_bytes == 8 else np.float32
         self.num_keys, self.L, self.R = int(num_keys), int(value_len), int(workers)
         self.with_adagrad = bool(with_adagrad)
         self._s = self._l.orc_create(self.num_keys, self.L, self.R, int(with_adagrad), int(count_accesses),
@@ -154,7 +161,8 @@ class Oracle:
     def table(self, which=0):
         """Writable numpy view [num_keys, L] of the value (0) or accumulator (1) table."""
         p = self._l.orc_table(self._s, which)
-        return np.ctypeslib.as_array(p, shape=(self.num_keys, self.L))
+        ct = C.c_double if self.dtype == np.float64 else C.c_float
+        return np.ctypeslib.as_array(C.cast(p, C.POINTER(ct)), shape=(self.num_keys, self.L))
 
     def init_uniform(self, which, seed, scale):
         self._l.orc_init_uniform(self._s, which, seed, scale)
@@ -173,18 +181,19 @@ class Oracle:
     # -- direct access ----------------------------------------------------
     def pull(self, keys, with_acc=False):
         k, kp = _u32(keys)
-        out = np.empty((len(k), self.L), np.float32)
-        out2 = np.empty((len(k), self.L), np.float32) if with_acc else None
-        _chk(self._l.orc_pull2(self._s, kp, len(k), out.ctypes.data_as(_f32p),
-                               out2.ctypes.data_as(_f32p) if with_acc else None), "pull")
+        out = np.empty((len(k), self.L), self.dtype)
+        out2 = np.empty((len(k), self.L), self.dtype) if with_acc else None
+        _chk(self._l.orc_pull2(self._s, kp, len(k), out.ctypes.data, out2.ctypes.data if with_acc else None), "pull")
         return (out, out2) if with_acc else out
 
     def push(self, keys, delta, delta_acc=None):
         k, kp = _u32(keys)
-        d, dp = _f32(delta)
+        d = np.ascontiguousarray(delta, dtype=self.dtype)
+        dp = d.ctypes.data
         assert d.shape == (len(k), self.L)
         if delta_acc is not None:
-            a, ap = _f32(delta_acc)
+            a = np.ascontiguousarray(delta_acc, dtype=self.dtype)
+            ap = a.ctypes.data
         else:
             ap = None
         _chk(self._l.orc_push2(self._s, kp, len(k), dp, ap), "push")
@@ -244,9 +253,9 @@ class Oracle:
 
     def pull_sample(self, handle, n, values=True):
         keys = np.zeros(n, np.uint32)
-        vals = np.empty((n, self.L), np.float32) if values else None
+        vals = np.empty((n, self.L), self.dtype) if values else None
         _chk(self._l.orc_pull_sample(self._s, handle, n, keys.ctypes.data_as(_u32p),
-                                     vals.ctypes.data_as(_f32p) if values else None), "pull_sample")
+                                     vals.ctypes.data if values else None), "pull_sample")
         return (keys, vals) if values else keys
 
     # -- workload steps ---------------------------------------------------

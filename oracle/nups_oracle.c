@@ -25,17 +25,19 @@
  * meaning of "local" on a single machine and the step formulas open; the
  * readings taken are written beside each function.
  *
- * Arithmetic: the tables are fp32 and every push is an fp32 add applied in
- * item order; everything a step computes between pull and push (dots, sigmoid,
- * square roots, losses) is done in fp64 and rounded to fp32 once.
+ * Arithmetic: the tables are fp32 (fp64 in the build with -DORC_REAL=double) and
+ * every push is an add in that type applied in item order; everything a step
+ * computes between pull and push (dots, sigmoid, square roots, losses) is done in
+ * fp64 and rounded to the tables' type once.
  *
  * Pins (tests marked "not gpu"): Philox known-answer vectors; exact alias mass
  * invariant and brute-force pmf on tiny tables; chi-square of sampled
  * frequencies; the paper's worked reuse example (Section 4.4); exactly-U reuse
  * inside a U*G window; postponing invariants; conservation
  * value = init + sum of pushed deltas; finite-difference gradients of the three
- * steps; AdaGrad closed form.  Loss trajectories have no external pin beyond
- * those ("parity unpinned" for absolute loss values).
+ * steps; AdaGrad closed form; the +-30 clamp of the scores; the mean-instead-of-sum
+ * merge.  The store and step pins run against both value types.  Loss trajectories
+ * have no external pin beyond those ("parity unpinned" for absolute loss values).
  */
 #include <math.h>
 #include <stdint.h>
@@ -43,6 +45,16 @@
 #include <string.h>
 
 typedef unsigned __int128 u128;
+
+/* Value type of the tables: fp32 (the default build) or fp64 (a second build of this same file with
+ * -DORC_REAL=double; Table 2 of the paper implies 8-byte values for the KGE and MF tasks).  Everything a
+ * step computes between pull and push is double precision in both builds; `real` is what is stored,
+ * pulled, pushed and added.                                                                          */
+#ifndef ORC_REAL
+#define ORC_REAL float
+#endif
+typedef ORC_REAL real;
+int orc_value_bytes(void) { return (int)sizeof(real); }
 
 enum { ORC_OK = 0, ORC_EINVAL = -1, ORC_ENOMEM = -2, ORC_EKEY = -4, ORC_ESTATE = -5 };
 enum { ORC_SINGLE = 0, ORC_REPLICATE = 1 };
@@ -171,11 +183,11 @@ typedef struct {
     uint64_t num_keys;
     uint32_t L, R, sync_interval;
     int with_acc, count_accesses, track_owner;
-    float *val, *acc;
+    real *val, *acc;
     int32_t* slot;          /* key -> hot slot, -1 = single                          */
     uint32_t* hot_keys;     /* slot -> key                                           */
     uint64_t H, Hcap;
-    float *dval, *dacc;     /* [R][Hcap][L] unsynced updates of each worker's replica */
+    real *dval, *dacc;     /* [R][Hcap][L] unsynced updates of each worker's replica */
     uint8_t* dirty;         /* [R][Hcap] worker's replica touched since the last sync */
     int merge_mean;         /* a sync adds the mean over the touching workers        */
     uint64_t* cnt;
@@ -196,8 +208,8 @@ void* orc_create(uint64_t num_keys, uint32_t L, uint32_t R, int with_acc, int co
     orc_store* s = (orc_store*)calloc(1, sizeof(orc_store));
     s->num_keys = num_keys; s->L = L; s->R = R; s->sync_interval = sync_interval;
     s->with_acc = with_acc; s->count_accesses = count_accesses; s->track_owner = track_owner;
-    s->val = (float*)calloc(num_keys * L, sizeof(float));
-    if (with_acc) s->acc = (float*)calloc(num_keys * L, sizeof(float));
+    s->val = (real*)calloc(num_keys * L, sizeof(real));
+    if (with_acc) s->acc = (real*)calloc(num_keys * L, sizeof(real));
     s->slot = (int32_t*)malloc(num_keys * sizeof(int32_t));
     for (uint64_t k = 0; k < num_keys; ++k) s->slot[k] = -1;
     s->cnt = (uint64_t*)calloc(num_keys, sizeof(uint64_t));
@@ -227,7 +239,7 @@ void orc_destroy(void* p)
     free(s->dirty); free(s->cnt); free(s->owner); free(s);
 }
 
-float* orc_table(void* p, int which) { orc_store* s = (orc_store*)p; return which ? s->acc : s->val; }
+real* orc_table(void* p, int which) { orc_store* s = (orc_store*)p; return which ? s->acc : s->val; }
 uint64_t* orc_counts(void* p) { return ((orc_store*)p)->cnt; }
 int orc_status(void* p) { orc_store* s = (orc_store*)p; int r = s->status; s->status = 0; return r; }
 uint64_t orc_num_hot(void* p) { return ((orc_store*)p)->H; }
@@ -245,7 +257,7 @@ void orc_stats(void* p, uint64_t out[4])
 void orc_init_uniform(void* p, int which, uint64_t seed, float scale)
 {
     orc_store* s = (orc_store*)p;
-    float* t = which ? s->acc : s->val;
+    real* t = which ? s->acc : s->val;
     if (!t) return;
     float unit = scale * (1.0f / 8388608.0f);
     uint64_t total = s->num_keys * s->L;
@@ -253,7 +265,7 @@ void orc_init_uniform(void* p, int which, uint64_t seed, float scale)
         uint32_t x[4];
         philox_at(seed, e >> 2, (uint32_t)which, 3, 0, x);
         int32_t v = (int32_t)(x[e & 3] >> 8) - 8388608;
-        t[e] = (float)v * unit;
+        t[e] = (real)((float)v * unit);
     }
 }
 
@@ -274,15 +286,15 @@ static void count_one(orc_store* s, uint32_t k) { if (s->count_accesses) s->cnt[
 
 /* pull (Section 3.1; replicas read through the worker's own copy, Section 3.2):
  * the value at the last sync plus this worker's own unsynced updates.        */
-static void pull_row(orc_store* s, uint32_t q, uint32_t k, int which, float* out)
+static void pull_row(orc_store* s, uint32_t q, uint32_t k, int which, real* out)
 {
-    const float* t = which ? s->acc : s->val;
-    const float* row = t + (uint64_t)k * s->L;
+    const real* t = which ? s->acc : s->val;
+    const real* row = t + (uint64_t)k * s->L;
     int32_t sl = s->slot[k];
     if (sl < 0) {
-        memcpy(out, row, s->L * sizeof(float));
+        memcpy(out, row, s->L * sizeof(real));
     } else {
-        const float* d = (which ? s->dacc : s->dval) + ((uint64_t)q * s->Hcap + (uint64_t)sl) * s->L;
+        const real* d = (which ? s->dacc : s->dval) + ((uint64_t)q * s->Hcap + (uint64_t)sl) * s->L;
         for (uint32_t e = 0; e < s->L; ++e) out[e] = row[e] + d[e];
     }
 }
@@ -290,10 +302,10 @@ static void pull_row(orc_store* s, uint32_t q, uint32_t k, int which, float* out
 /* push (Sections 3.1, 3.1.2): additive.  A replicated key's update stays in
  * the pushing worker's replica until the next sync; any other key is updated
  * in place.                                                                 */
-static void push_row(orc_store* s, uint32_t q, uint32_t k, int which, const float* d)
+static void push_row(orc_store* s, uint32_t q, uint32_t k, int which, const real* d)
 {
     int32_t sl = s->slot[k];
-    float* dst;
+    real* dst;
     if (sl < 0) dst = (which ? s->acc : s->val) + (uint64_t)k * s->L;
     else {
         dst = (which ? s->dacc : s->dval) + ((uint64_t)q * s->Hcap + (uint64_t)sl) * s->L;
@@ -304,15 +316,15 @@ static void push_row(orc_store* s, uint32_t q, uint32_t k, int which, const floa
 
 static void note_hit(orc_store* s, uint32_t k) { if (s->slot[k] >= 0) s->hot_hits++; else s->cold_hits++; }
 
-int orc_pull2(void* p, const uint32_t* keys, uint64_t n, float* out_val, float* out_acc)
+int orc_pull2(void* p, const uint32_t* keys, uint64_t n, real* out_val, real* out_acc)
 {
     orc_store* s = (orc_store*)p;
     if (out_acc && !s->with_acc) return ORC_EINVAL;
     for (uint64_t i = 0; i < n; ++i) {
         uint32_t k = keys[i];
         if (!key_ok(s, k)) {
-            if (out_val) memset(out_val + i * s->L, 0, s->L * sizeof(float));
-            if (out_acc) memset(out_acc + i * s->L, 0, s->L * sizeof(float));
+            if (out_val) memset(out_val + i * s->L, 0, s->L * sizeof(real));
+            if (out_acc) memset(out_acc + i * s->L, 0, s->L * sizeof(real));
             continue;
         }
         uint32_t q = worker_of(s, i, n);
@@ -322,9 +334,9 @@ int orc_pull2(void* p, const uint32_t* keys, uint64_t n, float* out_val, float* 
     }
     return ORC_OK;
 }
-int orc_pull(void* p, const uint32_t* keys, uint64_t n, float* out) { return orc_pull2(p, keys, n, out, NULL); }
+int orc_pull(void* p, const uint32_t* keys, uint64_t n, real* out) { return orc_pull2(p, keys, n, out, NULL); }
 
-int orc_push2(void* p, const uint32_t* keys, uint64_t n, const float* d_val, const float* d_acc)
+int orc_push2(void* p, const uint32_t* keys, uint64_t n, const real* d_val, const real* d_acc)
 {
     orc_store* s = (orc_store*)p;
     if (d_acc && !s->with_acc) return ORC_EINVAL;
@@ -338,7 +350,7 @@ int orc_push2(void* p, const uint32_t* keys, uint64_t n, const float* d_val, con
     }
     return ORC_OK;
 }
-int orc_push(void* p, const uint32_t* keys, uint64_t n, const float* d) { return orc_push2(p, keys, n, d, NULL); }
+int orc_push(void* p, const uint32_t* keys, uint64_t n, const real* d) { return orc_push2(p, keys, n, d, NULL); }
 
 /* sync (Section 3.2: sparse all-reduce, only updated parameters): for every
  * touched hot slot, add the workers' pending updates, worker 0 first, to the
@@ -353,17 +365,17 @@ int orc_sync(void* p)
         if (!touched) continue;
         uint32_t k = s->hot_keys[sl];
         for (int which = 0; which <= (s->with_acc ? 1 : 0); ++which) {
-            float* row = (which ? s->acc : s->val) + (uint64_t)k * s->L;
-            float* slab = which ? s->dacc : s->dval;
+            real* row = (which ? s->acc : s->val) + (uint64_t)k * s->L;
+            real* slab = which ? s->dacc : s->dval;
             for (uint32_t e = 0; e < s->L; ++e) {
-                float t = 0.0f;
+                real t = 0.0f;
                 for (uint32_t r = 0; r < s->R; ++r) {
-                    float* d = slab + ((uint64_t)r * s->Hcap + sl) * s->L + e;
+                    real* d = slab + ((uint64_t)r * s->Hcap + sl) * s->L + e;
                     t += *d; *d = 0.0f;
                 }
                 /* option (not in the paper; it damps the summed duplicate updates of very
                  * frequent keys): the mean over the workers that pushed, not the sum      */
-                if (s->merge_mean) t = t / (float)touched;
+                if (s->merge_mean) t = t / (real)touched;
                 row[e] += t;
             }
         }
@@ -430,8 +442,8 @@ int orc_set_management(void* p, const uint32_t* keys, uint64_t n, int technique)
             /* all pending updates are zero after the sync: a fresh slab is enough */
             uint64_t cap = need;
             free(s->dval); free(s->dacc);
-            s->dval = (float*)calloc((uint64_t)s->R * cap * s->L, sizeof(float));
-            s->dacc = s->with_acc ? (float*)calloc((uint64_t)s->R * cap * s->L, sizeof(float)) : NULL;
+            s->dval = (real*)calloc((uint64_t)s->R * cap * s->L, sizeof(real));
+            s->dacc = s->with_acc ? (real*)calloc((uint64_t)s->R * cap * s->L, sizeof(real)) : NULL;
             s->hot_keys = (uint32_t*)realloc(s->hot_keys, cap * sizeof(uint32_t));
             s->dirty = (uint8_t*)realloc(s->dirty, (uint64_t)s->R * cap);
             memset(s->dirty, 0, (uint64_t)s->R * cap);
@@ -652,7 +664,7 @@ int64_t orc_prepare_sample(void* p, int dist, uint64_t N)
  *   local sampling: start from the iid candidate and take the first local key
  *     at or after it (wrapping inside the distribution's key range), the
  *     candidate itself after ORC_LOCAL_PROBES failures.                     */
-int orc_pull_sample(void* p, int64_t handle, uint64_t n, uint32_t* keys_out, float* vals_out)
+int orc_pull_sample(void* p, int64_t handle, uint64_t n, uint32_t* keys_out, real* vals_out)
 {
     orc_store* s = (orc_store*)p;
     if (handle < 0 || handle >= ORC_MAX_HANDLES || !s->handle[handle].used) return ORC_EINVAL;
@@ -780,11 +792,11 @@ int orc_step_sgns(void* p, const uint32_t* center, const uint32_t* context, uint
         orc_pull_sample(s, h, n * K, nk, NULL);
     }
     if (neg_keys_out) memcpy(neg_keys_out, nk, n * K * sizeof(uint32_t));
-    float* upd = (float*)calloc(n * per * L, sizeof(float));
+    real* upd = (real*)calloc(n * per * L, sizeof(real));
     uint32_t* uk = (uint32_t*)malloc(n * per * sizeof(uint32_t));
     uint8_t* okv = (uint8_t*)calloc(n, 1);
-    float* v = (float*)malloc(L * sizeof(float));
-    float* u = (float*)malloc(L * sizeof(float));
+    real* v = (real*)malloc(L * sizeof(real));
+    real* u = (real*)malloc(L * sizeof(real));
     double* gv = (double*)malloc(L * sizeof(double));
     double* dd = (double*)malloc(L * sizeof(double));
     clip_step clip = {0, 0};
@@ -810,18 +822,18 @@ int orc_step_sgns(void* p, const uint32_t* center, const uint32_t* context, uint
             x = clamp30(x);
             double g = sigmoid(x) - (j == 0 ? 1.0 : 0.0);
             loss += (j == 0) ? softplus(-x) : softplus(x);
-            float* du = upd + (i * per + j) * L;
+            real* du = upd + (i * per + j) * L;
             for (uint32_t e = 0; e < L; ++e) {
                 dd[e] = -(double)lr * g * (double)v[e];
                 gv[e] += g * (double)u[e];
             }
             clip_update(s, kk[j], dd, &clip);
-            for (uint32_t e = 0; e < L; ++e) du[e] = (float)dd[e];
+            for (uint32_t e = 0; e < L; ++e) du[e] = (real)dd[e];
         }
-        float* dv = upd + (i * per + K + 1) * L;
+        real* dv = upd + (i * per + K + 1) * L;
         for (uint32_t e = 0; e < L; ++e) dd[e] = -(double)lr * gv[e];
         clip_update(s, center[i], dd, &clip);
-        for (uint32_t e = 0; e < L; ++e) dv[e] = (float)dd[e];
+        for (uint32_t e = 0; e < L; ++e) dv[e] = (real)dd[e];
     }
     clip_end_of_step(s, &clip);
     loc_queue lq = {0};
@@ -850,7 +862,7 @@ int orc_step_sgns(void* p, const uint32_t* center, const uint32_t* context, uint
  * gradient g per key role (h, r, t, each e_j); with (w, a) the pulled value
  * and accumulator rows: push acc += g^2, val += -lr*g / (sqrt(a + g^2) + eps).
  * Push order within an item: h, r, t, e_0 .. e_{K-1}.                       */
-static void complex_grads(const float* h, const float* r, const float* t, uint32_t d, double coef,
+static void complex_grads(const real* h, const real* r, const real* t, uint32_t d, double coef,
                           double* gh, double* gr, double* gt)
 {
     for (uint32_t i = 0; i < d; ++i) {
@@ -860,7 +872,7 @@ static void complex_grads(const float* h, const float* r, const float* t, uint32
         if (gr) { gr[i] += coef * (hr * tr + hi * ti); gr[d + i] += coef * (hr * ti - hi * tr); }
     }
 }
-static double complex_score(const float* h, const float* r, const float* t, uint32_t d)
+static double complex_score(const real* h, const real* r, const real* t, uint32_t d)
 {
     double phi = 0;
     for (uint32_t i = 0; i < d; ++i) {
@@ -883,12 +895,12 @@ int orc_step_complex(void* p, const uint32_t* hk, const uint32_t* rk, const uint
         orc_pull_sample(s, hd, n * K, nk, NULL);
     }
     if (neg_keys_out) memcpy(neg_keys_out, nk, n * K * sizeof(uint32_t));
-    float* uval = (float*)calloc(n * per * L, sizeof(float));
-    float* uacc = (float*)calloc(n * per * L, sizeof(float));
+    real* uval = (real*)calloc(n * per * L, sizeof(real));
+    real* uacc = (real*)calloc(n * per * L, sizeof(real));
     uint32_t* uk = (uint32_t*)malloc(n * per * sizeof(uint32_t));
     uint8_t* okv = (uint8_t*)calloc(n, 1);
-    float* rows = (float*)malloc(per * L * sizeof(float));     /* pulled values       */
-    float* arow = (float*)malloc(L * sizeof(float));           /* pulled accumulator  */
+    real* rows = (real*)malloc(per * L * sizeof(real));     /* pulled values       */
+    real* arow = (real*)malloc(L * sizeof(real));           /* pulled accumulator  */
     double* g = (double*)malloc(per * L * sizeof(double));
     double loss = 0;
     for (uint64_t i = 0; i < n; ++i) {
@@ -903,12 +915,12 @@ int orc_step_complex(void* p, const uint32_t* hk, const uint32_t* rk, const uint
         for (uint64_t j = 0; j < per; ++j) pull_row(s, q, kk[j], 0, rows + j * L);
         for (int j = 0; j < 3; ++j) { count_one(s, kk[j]); note_hit(s, kk[j]); }
         for (uint64_t e = 0; e < per * L; ++e) g[e] = 0;
-        const float *H = rows, *Rr = rows + L, *T = rows + 2 * L;
+        const real *H = rows, *Rr = rows + L, *T = rows + 2 * L;
         double phi = clamp30(complex_score(H, Rr, T, d));
         loss += softplus(-phi);
         complex_grads(H, Rr, T, d, sigmoid(phi) - 1.0, g, g + L, g + 2 * L);
         for (uint32_t j = 0; j < K; ++j) {
-            const float* E = rows + (3 + j) * L;
+            const real* E = rows + (3 + j) * L;
             double* gE = g + (3 + j) * L;
             if ((j & 1) == 0) {
                 double ph = clamp30(complex_score(E, Rr, T, d));
@@ -922,13 +934,13 @@ int orc_step_complex(void* p, const uint32_t* hk, const uint32_t* rk, const uint
         }
         for (uint64_t j = 0; j < per; ++j) {
             pull_row(s, q, kk[j], 1, arow);
-            float* dv = uval + (i * per + j) * L;
-            float* da = uacc + (i * per + j) * L;
+            real* dv = uval + (i * per + j) * L;
+            real* da = uacc + (i * per + j) * L;
             for (uint32_t e = 0; e < L; ++e) {
                 double ge = g[j * L + e];
                 double g2 = ge * ge;
-                da[e] = (float)g2;
-                dv[e] = (float)(-(double)lr * ge / (sqrt((double)arow[e] + g2) + (double)eps));
+                da[e] = (real)g2;
+                dv[e] = (real)(-(double)lr * ge / (sqrt((double)arow[e] + g2) + (double)eps));
             }
         }
     }
@@ -961,10 +973,10 @@ int orc_step_mf(void* p, const uint32_t* rowk, const uint32_t* colk, const float
 {
     orc_store* s = (orc_store*)p;
     uint32_t L = s->L;
-    float* upd = (float*)calloc(n * 2 * L, sizeof(float));
+    real* upd = (real*)calloc(n * 2 * L, sizeof(real));
     uint8_t* okv = (uint8_t*)calloc(n, 1);
-    float* w = (float*)malloc(L * sizeof(float));
-    float* h = (float*)malloc(L * sizeof(float));
+    real* w = (real*)malloc(L * sizeof(real));
+    real* h = (real*)malloc(L * sizeof(real));
     double* dd = (double*)malloc(L * sizeof(double));
     clip_step clip = {0, 0};
     double loss = 0;
@@ -981,14 +993,14 @@ int orc_step_mf(void* p, const uint32_t* rowk, const uint32_t* colk, const float
         for (uint32_t e = 0; e < L; ++e) dot += (double)w[e] * (double)h[e];
         double err = (double)x[i] - dot;
         loss += err * err;
-        float* dw = upd + (i * 2) * L;
-        float* dh = upd + (i * 2 + 1) * L;
+        real* dw = upd + (i * 2) * L;
+        real* dh = upd + (i * 2 + 1) * L;
         for (uint32_t e = 0; e < L; ++e) dd[e] = (double)lr * (err * (double)h[e] - (double)l2 * (double)w[e]);
         clip_update(s, rowk[i], dd, &clip);
-        for (uint32_t e = 0; e < L; ++e) dw[e] = (float)dd[e];
+        for (uint32_t e = 0; e < L; ++e) dw[e] = (real)dd[e];
         for (uint32_t e = 0; e < L; ++e) dd[e] = (double)lr * (err * (double)w[e] - (double)l2 * (double)h[e]);
         clip_update(s, colk[i], dd, &clip);
-        for (uint32_t e = 0; e < L; ++e) dh[e] = (float)dd[e];
+        for (uint32_t e = 0; e < L; ++e) dh[e] = (real)dd[e];
     }
     clip_end_of_step(s, &clip);
     loc_queue lq = {0};

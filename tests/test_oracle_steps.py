@@ -10,6 +10,20 @@ import pytest
 from oracle import Oracle, CONFORM, REPLICATE
 
 
+@pytest.fixture(params=[4, 8], ids=["fp32", "fp64"], autouse=True)
+def both_value_types(request, monkeypatch):
+    """Every pin of this file runs against both builds of the oracle: 4-byte and 8-byte values."""
+    import oracle
+    init = oracle.Oracle.__init__
+
+    def patched(self, *a, **kw):
+        kw.setdefault("value_bytes", request.param)
+        init(self, *a, **kw)
+    monkeypatch.setattr(oracle.Oracle, "__init__", patched)
+    return request.param
+
+
+
 def softplus(x):
     return np.logaddexp(0.0, x)
 

@@ -8,6 +8,20 @@ import oracle
 from oracle import Oracle, REPLICATE, SINGLE
 
 
+@pytest.fixture(params=[4, 8], ids=["fp32", "fp64"], autouse=True)
+def both_value_types(request, monkeypatch):
+    """Every pin of this file runs against both builds of the oracle: 4-byte and 8-byte values."""
+    import oracle
+    init = oracle.Oracle.__init__
+
+    def patched(self, *a, **kw):
+        kw.setdefault("value_bytes", request.param)
+        init(self, *a, **kw)
+    monkeypatch.setattr(oracle.Oracle, "__init__", patched)
+    return request.param
+
+
+
 def brute_tables(nk, L, seed=0):
     rng = np.random.default_rng(seed)
     return rng.normal(size=(nk, L)).astype(np.float32)
@@ -100,14 +114,16 @@ def test_no_replicated_key_means_no_sync_work():
     assert o.stats()["syncs"] == 0
 
 
-def test_push_applies_duplicates_in_item_order_fp32():
-    # three adds whose fp32 result depends on the order
+def test_push_applies_duplicates_in_item_order(both_value_types):
+    # three adds whose result in the table's precision depends on the order: 2^24 + 1 + 1 in fp32, 2^53 + 1 + 1 in fp64
+    ft, big = (np.float32, 2.0 ** 24) if both_value_types == 4 else (np.float64, 2.0 ** 53)
+    big, small = ft(big), ft(1.0)
     o = Oracle(2, 1, workers=1)
-    big, small = np.float32(2 ** 24), np.float32(1.0)
-    o.push(np.array([0, 0, 0], np.uint32), np.array([[big], [small], [small]], np.float32))
-    assert o.table()[0, 0] == np.float32(np.float32(big + small) + small) == big
+    o.push(np.array([0, 0, 0], np.uint32), np.array([[big], [small], [small]], ft))
+    assert o.table().dtype == ft
+    assert o.table()[0, 0] == ft(ft(big + small) + small) == big
     o2 = Oracle(2, 1, workers=1)
-    o2.push(np.array([0, 0, 0], np.uint32), np.array([[small], [small], [big]], np.float32))
+    o2.push(np.array([0, 0, 0], np.uint32), np.array([[small], [small], [big]], ft))
     assert o2.table()[0, 0] == big + 2
 
 
@@ -215,3 +231,34 @@ def test_merge_mean_adds_the_mean_over_the_workers_that_pushed():
     o.push(np.array([1], np.uint32), d[3:4])
     o.sync()
     np.testing.assert_array_equal(o.table()[1], (d[0] + d[1]) / 2 + d[3])
+
+
+def test_fp64_build_keeps_what_fp32_rounds_away():
+    # conservation in the 8-byte build: value = init + sum of pushed deltas to 1e-15 relative (fp64 additions of a few
+    # dozen terms), and an update of 1e-12 to a value of 1 is kept, which the 4-byte build cannot do
+    nk, L, R = 12, 5, 3
+    rng = np.random.default_rng(7)
+    o = Oracle(nk, L, workers=R, value_bytes=8)
+    init = rng.normal(size=(nk, L))
+    o.table()[:] = init
+    o.set_management(np.array([2, 3, 11], np.uint32), REPLICATE)
+    exact = [[Fraction(float(x)) for x in row] for row in init]
+    for _ in range(4):
+        keys = rng.integers(0, nk, 29).astype(np.uint32)
+        d = rng.normal(size=(29, L)) * 1e-6
+        o.push(keys, d)
+        for i, k in enumerate(keys):
+            for e in range(L):
+                exact[k][e] += Fraction(float(d[i, e]))
+    o.sync()
+    want = np.array([[float(x) for x in row] for row in exact])
+    np.testing.assert_allclose(o.table(), want, rtol=1e-14, atol=0)
+    assert np.abs(o.table() - init).max() > 1e-7
+    one = Oracle(2, 1, workers=1, value_bytes=8)
+    one.table()[:] = 1.0
+    one.push(np.array([0], np.uint32), np.array([[1e-12]]))
+    assert one.table()[0, 0] == 1.0 + 1e-12 and one.table()[1, 0] == 1.0
+    four = Oracle(2, 1, workers=1, value_bytes=4)
+    four.table()[:] = 1.0
+    four.push(np.array([0], np.uint32), np.array([[1e-12]], np.float32))
+    assert four.table()[0, 0] == 1.0
