@@ -830,7 +830,7 @@ def sgns_entry(device, steps):
     s.kernel_timing(False)
     s.close()
     return {"workload": WORKLOAD_SGNS, "us_per_step": dt * 1e6, "key_accesses_per_s": BATCH * ACCESSES_PER_PAIR / dt,
-            "updates_per_s": BATCH * UPDATES_PER_PAIR / dt, "kernel": "sgns_kernel", "kernel_us_per_launch": k_ms / max(k_n, 1) * 1e3,
+            "updates_per_s": BATCH * UPDATES_PER_PAIR / dt, "kernel": "sgns_runs_kernel", "kernel_us_per_launch": k_ms / max(k_n, 1) * 1e3,
             "steps_per_launch": nb / max(k_n, 1), "final_loss": float(losses.mean())}
 
 

@@ -21,8 +21,15 @@
  *   - Keys are uint32 in [0, num_keys).  A key outside the range is never
  *     dereferenced: the access is skipped (a pulled row is zero-filled) and the
  *     device status word is set to NUPS_EKEY; nups_status_check reports it.
- *   - Rows hold `value_len` floats, contiguous; value_len must be a multiple of
- *     4 so that every row starts on a 16-byte boundary.
+ *   - Rows hold `value_len` values, contiguous; a row must be a multiple of 16
+ *     bytes (value_len a multiple of 4 for fp32 values, of 2 for fp64 values).
+ *   - Value type: fp32 unless the store was created with value_bytes = 8.  Then
+ *     both tables, the replicas and every value buffer that crosses this
+ *     interface (the void* arguments of pull, push, table_copy, pull_sample)
+ *     hold doubles; additions are done in double; nups_step_complex and
+ *     nups_step_mf compute in double.  fp32 only: nups_step_sgns / nups_run_sgns,
+ *     nups_step_mf_by_column, clip_factor, sync_period_us,
+ *     nups_probe_reduction_rate (NUPS_ESTATE or NUPS_EINVAL otherwise).
  *   - Item i of a call over n items belongs to logical worker
  *     q(i) = floor(i * workers / n) (contiguous chunks).  Workers stand for the
  *     paper's nodes: each has its own replica of every replicated key and its
@@ -85,14 +92,18 @@ typedef struct nups_config {
     uint32_t merge_mean;      /* 1: a merge adds the MEAN of the pending updates of the workers that touched a  */
                               /*    replicated key since the last merge instead of their sum (damps the summed  */
                               /*    duplicate updates of very frequent keys); not with sync_period_us           */
-    uint32_t reserved[4];
+    uint32_t value_bytes;     /* 0 or 4: fp32 values; 8: fp64 values (Table 2: the knowledge-graph and matrix-  */
+                              /*    factorization tasks use 8-byte values), see "Value type" above              */
+    uint32_t reserved[3];
 } nups_config;
 
 /* ---- store (Section 3.1: keys, pull, push) -------------------------------- */
 
 /* Allocate a store of num_keys rows of value_len floats, zero-filled, no key
  * replicated.  *h_out receives the store.  NUPS_EINVAL: num_keys == 0 or
- * > 2^32-1, value_len == 0 or not a multiple of 4, workers > 254.  NUPS_ENOMEM:
+ * > 2^32-1, value_len == 0 or rows not a multiple of 16 bytes, workers > 254,
+ * value_bytes other than 0, 4, 8, or 8 together with clip_factor or
+ * sync_period_us.  NUPS_ENOMEM:
  * the device has not enough memory, or the store's own limit (max_device_mib) is
  * smaller than what the tables and maps need; that limit is checked before the
  * device is touched.                                                           */
@@ -102,15 +113,15 @@ nups_status nups_create(uint64_t num_keys, uint32_t value_len, const nups_config
 nups_status nups_destroy(nups_store* store);
 
 /* Device pointer of the value (which = 0) or accumulator (which = 1) table,
- * row-major [num_keys][row_stride_floats].  The caller may read or write it in
+ * row-major [num_keys][row_stride_values].  The caller may read or write it in
  * stream order (e.g. to load start values); rows of replicated keys do not
  * include updates that are still pending in replicas.                         */
-nups_status nups_table_ptr(nups_store* store, int which, float** h_ptr, uint64_t* h_row_stride_floats);
+nups_status nups_table_ptr(nups_store* store, int which, void** h_ptr, uint64_t* h_row_stride_values);
 
 /* Copy a whole table between the store and a caller buffer d_buf of
- * num_keys * value_len floats, in stream order: to_store = 1 loads start values
+ * num_keys * value_len values, in stream order: to_store = 1 loads start values
  * into the table, to_store = 0 takes a snapshot of it.                         */
-nups_status nups_table_copy(nups_store* store, int which, float* d_buf, int to_store, void* stream);
+nups_status nups_table_copy(nups_store* store, int which, void* d_buf, int to_store, void* stream);
 
 /* Fill a table with seeded start values: element e gets
  * (int(bits 8..31 of word e mod 4 of Philox4x32-10(counter = (e/4, 0, which, 3),
@@ -121,8 +132,8 @@ nups_status nups_init_uniform(nups_store* store, int which, uint64_t seed, float
  * sees it: the stored row, plus the worker's own pending replica updates when
  * the key is replicated (Section 3.2).  d_out is [n][value_len].
  * nups_pull2 also returns the accumulator rows (either output may be NULL).   */
-nups_status nups_pull(nups_store* store, const uint32_t* d_keys, uint64_t n, float* d_out, void* stream);
-nups_status nups_pull2(nups_store* store, const uint32_t* d_keys, uint64_t n, float* d_out_val, float* d_out_acc,
+nups_status nups_pull(nups_store* store, const uint32_t* d_keys, uint64_t n, void* d_out, void* stream);
+nups_status nups_pull2(nups_store* store, const uint32_t* d_keys, uint64_t n, void* d_out_val, void* d_out_acc,
                        void* stream);
 
 /* push (Section 3.1; replica accumulation Section 3.1.2): add d_delta[i][:] to
@@ -131,9 +142,9 @@ nups_status nups_pull2(nups_store* store, const uint32_t* d_keys, uint64_t n, fl
  * deterministic = 1: per destination row the deltas are added one by one in
  * ascending i.  nups_push2 updates both tables from one call (AdaGrad state
  * lives beside the value, Section 5.1 / Table 2); either delta may be NULL.   */
-nups_status nups_push(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta, void* stream);
-nups_status nups_push2(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta_val,
-                       const float* d_delta_acc, void* stream);
+nups_status nups_push(nups_store* store, const uint32_t* d_keys, uint64_t n, const void* d_delta, void* stream);
+nups_status nups_push2(nups_store* store, const uint32_t* d_keys, uint64_t n, const void* d_delta_val,
+                       const void* d_delta_acc, void* stream);
 
 /* Ordered push for callers that must not allocate device memory while they run:
  * code between the start and end of a latency-critical serving loop, a process
@@ -156,7 +167,7 @@ nups_status nups_push2(nups_store* store, const uint32_t* d_keys, uint64_t n, co
  *     overlaps on the GPU (different streams, no ordering between them) race on
  *     it: order them, or use nups_push for one of them.                        */
 #define NUPS_NOALLOC_MAX_ROWS 65536
-nups_status nups_push_noalloc(nups_store* store, const uint32_t* d_keys, uint64_t n, const float* d_delta,
+nups_status nups_push_noalloc(nups_store* store, const uint32_t* d_keys, uint64_t n, const void* d_delta,
                               void* stream);
 
 /* ---- per-key management (Section 3.2, Section 5.1) ------------------------ */
@@ -243,7 +254,7 @@ nups_status nups_prepare_sample(nups_store* store, int32_t dist, uint64_t N, nup
  *   NON-CONFORM the first key local to the worker at or after an independent
  *               candidate (64 probes, then the candidate itself).             */
 nups_status nups_pull_sample(nups_store* store, nups_handle handle, uint64_t n, uint32_t* d_keys_out,
-                             float* d_vals_out, void* stream);
+                             void* d_vals_out, void* stream);
 
 /* ---- workload steps (Section 5.1) ----------------------------------------- */
 /* One step over a batch of n items: draw the negatives (one handle of n*K

@@ -33,7 +33,8 @@ class Config(C.Structure):
     _fields_ = [("workers", C.c_uint32), ("sync_interval", C.c_uint32), ("deterministic", C.c_uint32),
                 ("with_adagrad", C.c_uint32), ("count_accesses", C.c_uint32), ("track_ownership", C.c_uint32),
                 ("smem_hot_rows", C.c_uint32), ("sync_period_us", C.c_uint32), ("clip_factor", C.c_float),
-                ("max_device_mib", C.c_uint32), ("first_epoch", C.c_uint32), ("merge_mean", C.c_uint32), ("reserved", C.c_uint32 * 4)]
+                ("max_device_mib", C.c_uint32), ("first_epoch", C.c_uint32), ("merge_mean", C.c_uint32), ("value_bytes", C.c_uint32),
+                ("reserved", C.c_uint32 * 3)]
 
 
 class NupsError(RuntimeError):
@@ -136,18 +137,20 @@ class Store:
 
     def __init__(self, num_keys, value_len, workers=8, sync_interval=1, deterministic=False, with_adagrad=False,
                  count_accesses=False, track_ownership=False, smem_hot_rows=0, sync_period_us=0, clip_factor=0.0,
-                 max_device_mib=0, first_epoch=0, merge_mean=False):
+                 max_device_mib=0, first_epoch=0, merge_mean=False, value_bytes=4):
         self._l = load()
         cfg = Config(workers=workers, sync_interval=sync_interval, deterministic=int(deterministic),
                      with_adagrad=int(with_adagrad), count_accesses=int(count_accesses),
                      track_ownership=int(track_ownership), smem_hot_rows=smem_hot_rows, sync_period_us=sync_period_us,
-                     clip_factor=clip_factor, max_device_mib=max_device_mib, first_epoch=first_epoch, merge_mean=int(merge_mean))
+                     clip_factor=clip_factor, max_device_mib=max_device_mib, first_epoch=first_epoch, merge_mean=int(merge_mean),
+                     value_bytes=value_bytes)
         h = C.c_void_p()
         self._s = None
         self._chk(self._l.nups_create(num_keys, value_len, C.byref(cfg), C.byref(h)), "nups_create")
         self._s = h
         self.num_keys, self.L, self.R = int(num_keys), int(value_len), int(workers)
         self.with_adagrad = bool(with_adagrad)
+        self.dtype = torch.float64 if value_bytes == 8 else torch.float32       # what every value buffer holds
         self.device = torch.device("cuda", torch.cuda.current_device())
 
     def _chk(self, code, what):
@@ -178,14 +181,14 @@ class Store:
 
     def write_table(self, which, values):
         """Copy host (or device) values [num_keys, L] into a table."""
-        src = torch.as_tensor(values, dtype=torch.float32).contiguous().cuda()
+        src = torch.as_tensor(values, dtype=self.dtype).contiguous().cuda()
         assert src.shape == (self.num_keys, self.L)
         self._chk(self._l.nups_table_copy(self._s, which, _ptr(src), 1, _stream()), "nups_table_copy")
         torch.cuda.current_stream().synchronize()
 
     def read_table(self, which=0, rows=None):
         """Snapshot of a table (or of the given rows of it) as a new CUDA tensor."""
-        out = torch.empty((self.num_keys, self.L), dtype=torch.float32, device=self.device)
+        out = torch.empty((self.num_keys, self.L), dtype=self.dtype, device=self.device)
         self._chk(self._l.nups_table_copy(self._s, which, _ptr(out), 0, _stream()), "nups_table_copy")
         return out if rows is None else out[rows]
 
@@ -196,10 +199,12 @@ class Store:
     def pull(self, keys, out=None, with_acc=False, out_acc=None):
         n = keys.numel()
         if out is None:
-            out = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+            out = torch.empty((n, self.L), dtype=self.dtype, device=self.device)
+        assert out.dtype == self.dtype
         if with_acc:
             if out_acc is None:
-                out_acc = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+                out_acc = torch.empty((n, self.L), dtype=self.dtype, device=self.device)
+            assert out_acc.dtype == self.dtype
             self._chk(self._l.nups_pull2(self._s, _ptr(keys, torch.int32), n, _ptr(out), _ptr(out_acc), _stream()),
                       "nups_pull2")
             return out, out_acc
@@ -208,11 +213,11 @@ class Store:
 
     def push(self, keys, delta, delta_acc=None):
         n = keys.numel()
-        assert delta is None or (delta.dtype == torch.float32 and delta.numel() == n * self.L)
+        assert delta is None or (delta.dtype == self.dtype and delta.numel() == n * self.L)
         if delta_acc is None:
             self._chk(self._l.nups_push(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _stream()), "nups_push")
         else:
-            assert delta_acc.dtype == torch.float32 and delta_acc.numel() == n * self.L
+            assert delta_acc.dtype == self.dtype and delta_acc.numel() == n * self.L
             self._chk(self._l.nups_push2(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _ptr(delta_acc), _stream()),
                       "nups_push2")
 
@@ -220,7 +225,7 @@ class Store:
         """Ordered push with its sort buffers in the library's fixed device array: for callers that
         may not allocate device memory while they run.  At most NOALLOC_MAX_ROWS rows per call."""
         n = keys.numel()
-        assert delta.dtype == torch.float32 and delta.numel() == n * self.L
+        assert delta.dtype == self.dtype and delta.numel() == n * self.L
         self._chk(self._l.nups_push_noalloc(self._s, _ptr(keys, torch.int32), n, _ptr(delta), _stream()),
                   "nups_push_noalloc")
 
@@ -292,7 +297,8 @@ class Store:
         if keys_out is None:
             keys_out = torch.empty(n, dtype=torch.int32, device=self.device)
         if values and vals_out is None:
-            vals_out = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+            vals_out = torch.empty((n, self.L), dtype=self.dtype, device=self.device)
+        assert not values or vals_out.dtype == self.dtype
         self._chk(self._l.nups_pull_sample(self._s, handle, n, _ptr(keys_out), _ptr(vals_out) if values else None,
                                            _stream()), "nups_pull_sample")
         return (keys_out, vals_out) if values else keys_out

@@ -154,6 +154,7 @@ extern "C" nups_status nups_set_sync_period(nups_store* s, uint32_t period_us)
 {
     if (!s) return NUPS_EINVAL;
     if (period_us && s->cfg.deterministic) return NUPS_ESTATE;     // merges at arbitrary times are not reproducible
+    if (period_us && (s->vb != 4 || s->cfg.merge_mean)) return NUPS_ESTATE;   // the background merge moves fp32 sums only
     if (!s->bg) {
         if (period_us == 0) return NUPS_OK;
         return nups_background_start(s, period_us);

@@ -16,9 +16,10 @@ static __device__ __align__(256) unsigned char g_noalloc_scratch[NUPS_NOALLOC_SC
 #define NUPS_NOALLOC_MAX_DEVICES 64
 static char* g_noalloc_addr[NUPS_NOALLOC_MAX_DEVICES];
 
-extern "C" nups_status nups_push_noalloc(nups_store* s, const uint32_t* d_keys, uint64_t n, const float* d_delta,
+extern "C" nups_status nups_push_noalloc(nups_store* s, const uint32_t* d_keys, uint64_t n, const void* d_delta_,
                                          void* stream)
 {
+    const float* d_delta = (const float*)d_delta_;
     if (!s || (n && (!d_keys || !d_delta))) return NUPS_EINVAL;
     if (!s->cfg.deterministic) return NUPS_ESTATE;
     if (n > NUPS_NOALLOC_MAX_ROWS) {

@@ -55,6 +55,7 @@ struct View {
     uint32_t R;
     uint32_t count;            // count accesses?
     uint32_t merge_mean;       // merges add the mean over the workers that touched a slot, not the sum
+    uint32_t f64;              // values are doubles (rows are still counted in 16-byte chunks, L4)
     uint32_t epoch_tag;        // number of the running call, shifted into the upper 24 bits of an ownership word
     float clip_factor;         // > 0: updates to replicated keys are clipped at this multiple of their mean norm
 };
@@ -84,7 +85,8 @@ struct Handle {
 
 struct nups_store {
     uint64_t num_keys;
-    uint32_t L, R;
+    uint32_t L, R;             // L = row length in 4-byte units (value_len for fp32 values, 2 * value_len for fp64 values)
+    uint32_t value_len, vb;    // values per row; bytes per value (4 or 8)
     nups_config cfg;
     float *val, *acc;
     uint32_t* hot_bits;
@@ -119,7 +121,7 @@ struct nups_store {
     struct nups_background* bg; // time-based replica synchronisation (background.cu); NULL = never started
     cudaStream_t side;          // nups_run_sgns: a due replica merge runs here, beside the next steps' sample draw
     cudaEvent_t side_fork, side_join;
-    bool push_smem_opted, complex_smem_opted[2][2][2];   // large dynamic shared memory asked for on this store's device
+    bool push_smem_opted, complex_smem_opted[2][2][2][2];   // large dynamic shared memory asked for on this store's device
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };
@@ -181,6 +183,7 @@ nups_status nups_sort_pairs(nups_store* s, unsigned long long* k_in, uint32_t* v
                             uint32_t* v_out, uint64_t n, int bits, char* scratch, cudaStream_t st);
 
 // store.cu internals used by steps.cu / sampling.cu
+// (value buffers are passed as float* whatever the value type: storage, counted in 4-byte units)
 nups_status nups_push_internal(nups_store* s, const uint32_t* d_keys, uint64_t n_rows, uint32_t rows_per_item,
                                const float* d_dval, const float* d_dacc, cudaStream_t st);
 size_t nups_push_scratch_bytes(const nups_store* s, uint64_t n_rows);
@@ -364,6 +367,39 @@ __device__ __forceinline__ void st8_stream(float* p, const F8& r)
 }
 
 __device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+
+// A 16-byte chunk of a row holds four floats or two doubles; kernels that only move rows do not care, kernels that add
+// (replica reads, pushes, merges) take the value type as a template argument.
+__device__ __forceinline__ double2 as_d2(float4 a)
+{
+    return make_double2(__hiloint2double(__float_as_int(a.y), __float_as_int(a.x)),
+                        __hiloint2double(__float_as_int(a.w), __float_as_int(a.z)));
+}
+__device__ __forceinline__ float4 as_f4(double2 d)
+{
+    return make_float4(__int_as_float(__double2loint(d.x)), __int_as_float(__double2hiint(d.x)),
+                       __int_as_float(__double2loint(d.y)), __int_as_float(__double2hiint(d.y)));
+}
+template <bool F64>
+__device__ __forceinline__ float4 add_chunk(float4 a, float4 b)
+{
+    if (F64) {
+        const double2 x = as_d2(a), y = as_d2(b);
+        return as_f4(make_double2(x.x + y.x, x.y + y.y));
+    }
+    return add4(a, b);
+}
+template <bool F64>
+__device__ __forceinline__ void red_add_chunk(float* addr, float4 x)
+{
+    if (F64) {
+        const double2 d = as_d2(x);
+        asm volatile("red.global.add.f64 [%0], %1;" ::"l"(addr), "d"(d.x) : "memory");
+        asm volatile("red.global.add.f64 [%0], %1;" ::"l"(addr + 2), "d"(d.y) : "memory");
+    } else {
+        red_add_v4(addr, x);
+    }
+}
 
 __device__ __forceinline__ float warp_sum(float x)
 {

@@ -812,7 +812,7 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         // a full pull of a fresh handle has no entries postponed by earlier calls to emit: the placement pass can copy
         // the rows itself (one table of 64, 128 or 256 floats per row, 32-byte aligned output)
         const uint32_t c8 = s->L / 8;
-        const bool fused = d_vals_out && h.cursor == 0 && n == h.N && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) &&
+        const bool fused = d_vals_out && s->vb == 4 && h.cursor == 0 && n == h.N && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) &&
                            ((uintptr_t)d_vals_out & 31) == 0 && (uint64_t)s->R * s->Hcap < 0xFFFFFFFFull;
         if (fused) nups_time_begin(s, st, NUPS_TIMED_SAMPLE_ROWS);
         if (fused && c8 == 8) lt_place_kernel<8><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
@@ -846,11 +846,11 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
 }
 
 extern "C" nups_status nups_pull_sample(nups_store* s, nups_handle handle, uint64_t n, uint32_t* d_keys_out,
-                                        float* d_vals_out, void* stream)
+                                        void* d_vals_out, void* stream)
 {
     if (!s || handle < 0 || handle >= NUPS_MAX_HANDLES || !s->handle[handle].used) return NUPS_EINVAL;
     if (n && !d_keys_out) return NUPS_EINVAL;
-    return pull_internal(s, (int)handle, n, d_keys_out, d_vals_out, (cudaStream_t)stream);
+    return pull_internal(s, (int)handle, n, d_keys_out, (float*)d_vals_out, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------------------------------------

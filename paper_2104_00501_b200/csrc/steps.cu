@@ -504,6 +504,8 @@ sgns_runs_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __
 constexpr int CPX_THREADS = 128;
 constexpr int CPX_MAX_KEYS = 34;          // 3 + K with K <= 30, rounded up
 constexpr int CPX_NS = 16;                // up to this many scores are reduced together
+// the 16-byte chunks of a row that thread tid moves: one (rows of up to 512 fp32 values), two with 8-byte values
+#define NUPS_CPX_CHUNKS(c) _Pragma("unroll") for (uint32_t c = tid; c < L4 && c < (F64 ? 2u : 1u) * CPX_THREADS; c += CPX_THREADS)
 
 template <class T> struct CX { T re[2], im[2]; };
 
@@ -514,7 +516,9 @@ __device__ __forceinline__ double mul_rn(double a, double b) { return __dmul_rn(
 __device__ __forceinline__ float sub_rn(float a, float b) { return __fsub_rn(a, b); }
 __device__ __forceinline__ double sub_rn(double a, double b) { return __dsub_rn(a, b); }
 
-// the thread's components of a row staged in shared memory
+// the thread's components of a row staged in shared memory (S = the table's value type, T = the type computed in):
+// two adjacent values of the real half and the two matching ones of the imaginary half, each pair one vector access
+// (d is even, so both pairs are aligned to their own size)
 template <class T>
 __device__ __forceinline__ CX<T> cx_load(const float* row, uint32_t d, uint32_t c)
 {
@@ -524,10 +528,24 @@ __device__ __forceinline__ CX<T> cx_load(const float* row, uint32_t d, uint32_t 
     x.re[0] = (T)a.x; x.re[1] = (T)a.y; x.im[0] = (T)b.x; x.im[1] = (T)b.y;
     return x;
 }
+template <class T>
+__device__ __forceinline__ CX<T> cx_load(const double* row, uint32_t d, uint32_t c)
+{
+    const double2 a = *reinterpret_cast<const double2*>(row + 2 * c);
+    const double2 b = *reinterpret_cast<const double2*>(row + d + 2 * c);
+    CX<T> x;
+    x.re[0] = (T)a.x; x.re[1] = (T)a.y; x.im[0] = (T)b.x; x.im[1] = (T)b.y;
+    return x;
+}
 __device__ __forceinline__ void cx_store(float* row, uint32_t d, uint32_t c, float r0, float r1, float i0, float i1)
 {
     *reinterpret_cast<float2*>(row + 2 * c) = make_float2(r0, r1);
     *reinterpret_cast<float2*>(row + d + 2 * c) = make_float2(i0, i1);
+}
+__device__ __forceinline__ void cx_store(double* row, uint32_t d, uint32_t c, double r0, double r1, double i0, double i1)
+{
+    *reinterpret_cast<double2*>(row + 2 * c) = make_double2(r0, r1);
+    *reinterpret_cast<double2*>(row + d + 2 * c) = make_double2(i0, i1);
 }
 
 template <class T>
@@ -570,14 +588,14 @@ __device__ __forceinline__ double adagrad_step(double g, double g2, double a, do
 
 // AdaGrad update of one key role from the thread's part of its summed gradient: the update rows
 // (value: -lr g / (sqrt(acc_pulled + g^2) + eps), accumulator: g^2) replace the role's staged rows
-template <class T>
-__device__ __forceinline__ void cx_adagrad(const CX<T>& g, float* val_row, float* acc_row, uint32_t d, uint32_t c, T lr, T eps)
+template <class T, class S>
+__device__ __forceinline__ void cx_adagrad(const CX<T>& g, S* val_row, S* acc_row, uint32_t d, uint32_t c, T lr, T eps)
 {
     const CX<T> a = cx_load<T>(acc_row, d, c);
     const T r0 = g.re[0] * g.re[0], r1 = g.re[1] * g.re[1], i0 = g.im[0] * g.im[0], i1 = g.im[1] * g.im[1];
-    cx_store(val_row, d, c, (float)adagrad_step(g.re[0], r0, a.re[0], lr, eps), (float)adagrad_step(g.re[1], r1, a.re[1], lr, eps),
-             (float)adagrad_step(g.im[0], i0, a.im[0], lr, eps), (float)adagrad_step(g.im[1], i1, a.im[1], lr, eps));
-    cx_store(acc_row, d, c, (float)r0, (float)r1, (float)i0, (float)i1);
+    cx_store(val_row, d, c, (S)adagrad_step(g.re[0], r0, a.re[0], lr, eps), (S)adagrad_step(g.re[1], r1, a.re[1], lr, eps),
+                (S)adagrad_step(g.im[0], i0, a.im[0], lr, eps), (S)adagrad_step(g.im[1], i1, a.im[1], lr, eps));
+    cx_store(acc_row, d, c, (S)r0, (S)r1, (S)i0, (S)i1);
 }
 
 template <class T>
@@ -614,22 +632,25 @@ __device__ __forceinline__ double sigmoidT(double x) { return 1.0 / (1.0 + exp(-
 __device__ __forceinline__ float softplusT(float x) { return softplusf_(x); }
 __device__ __forceinline__ double softplusT(double x) { return fmax(x, 0.0) + log1p(exp(-fabs(x))); }
 
-template <bool HOT, bool DET, bool RED16>
-__global__ void __launch_bounds__(CPX_THREADS, 4)
+template <bool HOT, bool DET, bool RED16, bool F64>
+__global__ void __launch_bounds__(CPX_THREADS, F64 ? 2 : 4)
 complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restrict__ rk, const uint32_t* __restrict__ tk,
                const uint32_t* __restrict__ negs, uint64_t n, uint32_t K, float lr, float eps, float* __restrict__ uval,
                float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
                float* __restrict__ loss_out)
 {
-    using T = typename std::conditional<DET, double, float>::type;
+    using S = typename std::conditional<F64, double, float>::type;          // what the tables hold
+    using T = typename std::conditional<DET || F64, double, float>::type;   // what the step computes in
     // rows[2 * role] = the role's value row, rows[2 * role + 1] = its accumulator row, as they lie in memory
-    extern __shared__ __align__(16) float rows[];
-    __shared__ unsigned long long s_row[CPX_MAX_KEYS], s_pend[CPX_MAX_KEYS];
+    extern __shared__ __align__(16) unsigned char rows_raw[];
+    S* rows = reinterpret_cast<S*>(rows_raw);
+    __shared__ unsigned long long s_row[CPX_MAX_KEYS], s_pend[CPX_MAX_KEYS];   // offsets in 4-byte units
     __shared__ T s_part[CPX_THREADS / 32][32];                     // per-warp sums of the scores
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const uint32_t L4 = v.L4, d2 = v.L4, per = K + 3;              // d/2 component pairs = L/4
-    const bool mine = tid < d2;                                    // threads beyond the row width only help reduce
-    const uint32_t L = L4 * 4, d = L / 2;
+    const uint32_t L4 = v.L4, per = K + 3;                         // 16-byte chunks of a row
+    const uint32_t L = F64 ? L4 * 2 : L4 * 4, d = L / 2;           // values per row, complex components
+    const uint32_t LU = L4 * 4;                                    // row length in 4-byte units
+    const bool mine = tid < d / 2;                                 // threads beyond the row width only help reduce
     const T lrT = (T)lr, epsT = (T)eps;
     double my_loss = 0.0;
     s_part[warp][lane] = T(0);
@@ -648,8 +669,8 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
         if (tid < per) {
             int slot = HOT ? __ldg(v.slot_of + key) : -1;
             if (slot < 0) slot = -1;
-            s_row[tid] = (unsigned long long)key * L;
-            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * L : NO_PEND;
+            s_row[tid] = (unsigned long long)key * LU;
+            s_pend[tid] = slot >= 0 ? ((unsigned long long)q * v.Hcap + (unsigned)slot) * LU : NO_PEND;
             if (DET) ukeys[i * per + tid] = key;
             if (!DET && slot >= 0) mark_dirty(v, q, slot);
             if (v.count) {
@@ -659,11 +680,13 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             if (v.own && tid < 3) mark_localize(v, key, q);
         }
         __syncthreads();
-        if (tid < L4) {
-            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rows) + 16 * tid;
+        {
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rows);
             for (uint32_t role = 0; role < per; ++role) {
-                cp_async_16s(dst + (2 * role) * L * 4, v.val + s_row[role] + 4 * tid);
-                cp_async_16s(dst + (2 * role + 1) * L * 4, v.acc + s_row[role] + 4 * tid);
+                NUPS_CPX_CHUNKS(c) {
+                    cp_async_16s(dst + ((2 * role) * L4 + c) * 16, v.val + s_row[role] + 4 * c);
+                    cp_async_16s(dst + ((2 * role + 1) * L4 + c) * 16, v.acc + s_row[role] + 4 * c);
+                }
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
         }
@@ -671,29 +694,30 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
         {
             const uint64_t nx = i + gridDim.x;
             if (nx < n) {
-                const uint32_t lines_per_row = (L * 4 + 127) / 128;
+                const uint32_t lines_per_row = (LU * 4 + 127) / 128;
                 for (uint32_t e = tid; e < per * lines_per_row; e += CPX_THREADS) {
                     const uint32_t role = e / lines_per_row, line = e % lines_per_row;
                     const uint32_t k = role == 0 ? hk[nx] : role == 1 ? rk[nx] : role == 2 ? tk[nx] : negs[nx * K + role - 3];
-                    const size_t off = (size_t)k * L + (size_t)line * 32;
-                    if (k < v.num_keys && off + 32 <= (size_t)v.num_keys * L) {       // a whole line inside the table
+                    const size_t off = (size_t)k * LU + (size_t)line * 32;
+                    if (k < v.num_keys && off + 32 <= (size_t)v.num_keys * LU) {      // a whole line inside the table
                         prefetch_l2(v.val + off);
                         prefetch_l2(v.acc + off);
                     }
                 }
             }
         }
-        if (tid < L4) {
-            asm volatile("cp.async.wait_group 0;" ::: "memory");
-            if (HOT) {
-                // the worker's pending replica updates join the chunks this thread staged
-                for (uint32_t role = 0; role < per; ++role) {
-                    const unsigned long long pend = s_pend[role];
-                    if (pend == NO_PEND) continue;
-                    float4* pv = reinterpret_cast<float4*>(rows + (size_t)(2 * role) * L) + tid;
-                    float4* pa = reinterpret_cast<float4*>(rows + (size_t)(2 * role + 1) * L) + tid;
-                    *pv = add4(*pv, *(reinterpret_cast<const float4*>(v.dval + pend) + tid));
-                    *pa = add4(*pa, *(reinterpret_cast<const float4*>(v.dacc + pend) + tid));
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        if (HOT) {
+            // the worker's pending replica updates join the chunks this thread staged
+            float4* staged = reinterpret_cast<float4*>(rows_raw);
+            for (uint32_t role = 0; role < per; ++role) {
+                const unsigned long long pend = s_pend[role];
+                if (pend == NO_PEND) continue;
+                NUPS_CPX_CHUNKS(c) {
+                    float4* pv = staged + (size_t)(2 * role) * L4 + c;
+                    float4* pa = staged + (size_t)(2 * role + 1) * L4 + c;
+                    *pv = add_chunk<F64>(*pv, *(reinterpret_cast<const float4*>(v.dval + pend) + c));
+                    *pa = add_chunk<F64>(*pa, *(reinterpret_cast<const float4*>(v.dacc + pend) + c));
                 }
             }
         }
@@ -760,19 +784,19 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             cx_adagrad(gt, val_row(2), acc_row(2), d, tid, lrT, epsT);
         }
         __syncthreads();
-        if (tid < L4) {
-            for (uint32_t role = 0; role < per; ++role) {
-                const float4 dv = reinterpret_cast<const float4*>(val_row(role))[tid];
-                const float4 da = reinterpret_cast<const float4*>(acc_row(role))[tid];
+        for (uint32_t role = 0; role < per; ++role) {
+            NUPS_CPX_CHUNKS(c) {
+                const float4 dv = reinterpret_cast<const float4*>(val_row(role))[c];
+                const float4 da = reinterpret_cast<const float4*>(acc_row(role))[c];
                 if (DET) {
-                    reinterpret_cast<float4*>(uval + (i * per + role) * (uint64_t)L)[tid] = dv;
-                    reinterpret_cast<float4*>(uacc + (i * per + role) * (uint64_t)L)[tid] = da;
+                    reinterpret_cast<float4*>(uval + (i * per + role) * (uint64_t)LU)[c] = dv;
+                    reinterpret_cast<float4*>(uacc + (i * per + role) * (uint64_t)LU)[c] = da;
                 } else {
                     const unsigned long long pend = s_pend[role];
                     float* ov = pend != NO_PEND ? v.dval + pend : v.val + s_row[role];
                     float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + s_row[role];
-                    red_add_v4(ov + 4 * tid, dv);
-                    red_add_v4(oa + 4 * tid, da);
+                    red_add_chunk<F64>(ov + 4 * c, dv);
+                    red_add_chunk<F64>(oa + 4 * c, da);
                 }
             }
         }
@@ -1160,6 +1184,7 @@ static nups_status sgns_check(nups_store* s, const uint32_t* d_center, const uin
 {
     if (!s || !d_center || !d_context || n == 0 || n * (uint64_t)(K + 2) >= (1ull << 32)) return NUPS_EINVAL;
     if (K > 30) return NUPS_EINVAL;                         // one lane per key of an item
+    if (s->vb != 4) return NUPS_ESTATE;                     // the skip-gram step is single precision only
     if (s->L / 4 > SGNS_MAX_CHUNKS) return NUPS_EINVAL;     // four float4 chunks of a row per lane: at most 512 floats
     return NUPS_OK;
 }
@@ -1272,7 +1297,7 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
                                          void* stream)
 {
     if (!s || !d_h || !d_r || !d_t || n == 0 || n * (uint64_t)(K + 3) >= (1ull << 32)) return NUPS_EINVAL;
-    if (!s->acc || s->L / 4 > CPX_THREADS || K > 30) return NUPS_EINVAL;    // one thread per component pair, one lane per score
+    if (!s->acc || s->value_len / 4 > CPX_THREADS || (s->value_len & 3) || K > 30) return NUPS_EINVAL;    // one thread per component pair, one lane per score
     cudaStream_t st = (cudaStream_t)stream;
     nups_status rc = nups_draw_negatives(s, dist, n * K, st);
     if (rc != NUPS_OK) return rc;
@@ -1290,22 +1315,23 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
     if (per_sm < 1) per_sm = 1;
     uint64_t want = n < (uint64_t)s->sm_count * per_sm ? n : (uint64_t)s->sm_count * per_sm;
     unsigned grid = (unsigned)want;
-    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0, ri = K + 1 <= (uint32_t)CPX_NS ? 1 : 0;
+    const int hi = s->H ? 1 : 0, di = s->cfg.deterministic ? 1 : 0, ri = K + 1 <= (uint32_t)CPX_NS ? 1 : 0, fi = s->vb == 8 ? 1 : 0;
+    if (fi && grid > (unsigned)s->sm_count * 2) grid = (unsigned)s->sm_count * 2;      // the 8-byte variant: two blocks per multiprocessor
     cudaError_t e = cudaSuccess;
     nups_time_begin(s, st, NUPS_TIMED_STEP);
-#define NUPS_CPX_GO(RED16_)                                                                                          \
+#define NUPS_CPX_GO(RED16_, F64_)                                                                                    \
     DISPATCH_MODE(s, {                                                                                               \
-        auto kern = complex_kernel<HOT, DET, RED16_>;                                                                \
-        if (!s->complex_smem_opted[hi][di][ri]) {                                                                    \
+        auto kern = complex_kernel<HOT, DET, RED16_, F64_>;                                                          \
+        if (!s->complex_smem_opted[hi][di][ri][fi]) {                                                                \
             e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, s->max_smem - 4096);         \
-            s->complex_smem_opted[hi][di][ri] = (e == cudaSuccess);                                                  \
+            s->complex_smem_opted[hi][di][ri][fi] = (e == cudaSuccess);                                              \
         }                                                                                                            \
         if (e == cudaSuccess)                                                                                        \
             kern<<<grid, CPX_THREADS, smem, st>>>(v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc,     \
                                                   b.ukeys, b.loss_item, d_loss_out);                                 \
     })
-    if (ri) NUPS_CPX_GO(true);
-    else NUPS_CPX_GO(false);
+    if (fi) { if (ri) NUPS_CPX_GO(true, true); else NUPS_CPX_GO(false, true); }
+    else { if (ri) NUPS_CPX_GO(true, false); else NUPS_CPX_GO(false, false); }
 #undef NUPS_CPX_GO
     nups_time_end(s, st);
     if (e != cudaSuccess) return nups_cuda_fail(e, "cudaFuncSetAttribute");
@@ -1506,11 +1532,84 @@ mf_runs_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __rest
     if (CLIP) clip_finish(v, (double)my_clip, my_clipped);
 }
 
+// ---------------------------------------------------------------------------------------------
+// matrix factorization on 8-byte values: one warp per cell, lanes stride over the row's values, everything
+// in double precision.  (Plain: the single-precision kernels above are the tuned ones.)
+// ---------------------------------------------------------------------------------------------
+namespace {
+template <bool HOT, bool DET>
+__global__ void __launch_bounds__(128)
+mf_f64_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
+              uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
+              float* __restrict__ loss_item, float* __restrict__ loss_out)
+{
+    const unsigned lane = threadIdx.x & 31;
+    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
+    const uint32_t L = v.L4 * 2;                               // values per row
+    const double* val = reinterpret_cast<const double*>(v.val);
+    const double* slab = reinterpret_cast<const double*>(v.dval);
+    double* uout = reinterpret_cast<double*>(upd);
+    const double lrd = (double)lr, l2d = (double)l2;
+    double my_loss = 0.0;
+    for (uint64_t i = warp; i < n; i += nwarps) {
+        const uint32_t ki = rowk[i], kj = colk[i];
+        const bool ok = ki < v.num_keys && kj < v.num_keys;
+        if (DET && lane == 0) {
+            ukeys[2 * i] = ok ? ki : NUPS_INVALID_KEY;
+            ukeys[2 * i + 1] = ok ? kj : NUPS_INVALID_KEY;
+        }
+        if (!ok) {
+            if (lane == 0) { flag_bad_key(v); if (DET) loss_item[i] = 0.f; }
+            continue;
+        }
+        const uint32_t q = worker_of_item(i, n, v.R);
+        const int si = HOT ? __ldg(v.slot_of + ki) : -1, sj = HOT ? __ldg(v.slot_of + kj) : -1;
+        const double* wrow = val + (uint64_t)ki * L;
+        const double* hrow = val + (uint64_t)kj * L;
+        const double* wpend = si >= 0 ? slab + ((uint64_t)q * v.Hcap + (unsigned)si) * L : nullptr;
+        const double* hpend = sj >= 0 ? slab + ((uint64_t)q * v.Hcap + (unsigned)sj) * L : nullptr;
+        double dot = 0.0;
+        for (uint32_t e = lane; e < L; e += 32) {
+            const double w = wrow[e] + (wpend ? wpend[e] : 0.0), h = hrow[e] + (hpend ? hpend[e] : 0.0);
+            dot += w * h;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xFFFFFFFFu, dot, o);
+        const double err = (double)x[i] - dot;
+        double* ow = DET ? uout + (2 * i) * (uint64_t)L : reinterpret_cast<double*>(si >= 0 ? v.dval : v.val) +
+                                                              (si >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)si) * L : (uint64_t)ki * L);
+        double* oh = DET ? uout + (2 * i + 1) * (uint64_t)L : reinterpret_cast<double*>(sj >= 0 ? v.dval : v.val) +
+                                                                  (sj >= 0 ? ((uint64_t)q * v.Hcap + (unsigned)sj) * L : (uint64_t)kj * L);
+        for (uint32_t e = lane; e < L; e += 32) {
+            const double w = wrow[e] + (wpend ? wpend[e] : 0.0), h = hrow[e] + (hpend ? hpend[e] : 0.0);
+            const double dw = lrd * (err * h - l2d * w), dh = lrd * (err * w - l2d * h);
+            if (DET) { ow[e] = dw; oh[e] = dh; }
+            else { atomicAdd(ow + e, dw); atomicAdd(oh + e, dh); }
+        }
+        if (lane == 0) {
+            if (!DET) {
+                if (si >= 0) mark_dirty(v, q, si);
+                if (sj >= 0) mark_dirty(v, q, sj);
+            }
+            if (v.count) {
+                note_access(v, ki, si, DET ? 1u : 2u);
+                note_access(v, kj, sj, DET ? 1u : 2u);
+            }
+            if (v.own) { mark_localize(v, ki, q); mark_localize(v, kj, q); }
+            if (DET) loss_item[i] = (float)(err * err);
+        }
+        my_loss += err * err;
+    }
+    if (!DET) loss_finish(v, my_loss, n, loss_out);
+}
+}  // namespace
+
 static nups_status mf_step(nups_store* s, const uint32_t* d_row, const uint32_t* d_col, const float* d_x,
                            uint64_t n, float lr, float l2, float* d_loss_out, void* stream, bool cells_by_column)
 {
     if (!s || !d_row || !d_col || !d_x || n == 0 || n * 2 >= (1ull << 32)) return NUPS_EINVAL;
-    if (s->L / 4 > 128) return NUPS_EINVAL;
+    if (s->vb == 4 && s->L / 4 > 128) return NUPS_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
     s->last_negs_n = 0;
     nups_status rc = nups_new_epoch(s, st);
@@ -1521,7 +1620,11 @@ static nups_status mf_step(nups_store* s, const uint32_t* d_row, const uint32_t*
     View v = nups_view(s);
     const bool by_column = cells_by_column && !s->cfg.deterministic;    // the ordered mode is the same for any order
     nups_time_begin(s, st, NUPS_TIMED_STEP);
-    if (by_column) {
+    if (s->vb == 8) {
+        const unsigned grid = step_grid(s, n, 8);
+        DISPATCH_MODE(s, mf_f64_kernel<HOT, DET><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys,
+                                                                      b.loss_item, d_loss_out));
+    } else if (by_column) {
         const unsigned grid = step_grid(s, n, MF_RUN_BLOCKS);
         DISPATCH_CLIP(s, DISPATCH_CH(v.L4, {
             if (s->H) mf_runs_kernel<true, CH, CLIP><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, d_loss_out);

@@ -39,6 +39,7 @@ View nups_view(const nups_store* s)
     v.num_keys = s->num_keys; v.Hcap = s->Hcap; v.H = (uint32_t)s->H; v.L4 = s->L / 4; v.R = s->R;
     v.count = s->cfg.count_accesses;
     v.merge_mean = s->cfg.merge_mean;
+    v.f64 = s->vb == 8;
     v.clip_factor = s->cfg.clip_factor;
     return v;
 }
@@ -185,10 +186,16 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
 {
     if (!out) return NUPS_EINVAL;
     *out = nullptr;
-    if (num_keys == 0 || num_keys > 0xFFFFFFFFull || value_len == 0 || (value_len & 3)) return NUPS_EINVAL;
+    if (num_keys == 0 || num_keys > 0xFFFFFFFFull || value_len == 0) return NUPS_EINVAL;
     nups_config c;
     memset(&c, 0, sizeof(c));
     if (cfg) c = *cfg;
+    if (c.value_bytes == 0) c.value_bytes = 4;
+    if (c.value_bytes != 4 && c.value_bytes != 8) return NUPS_EINVAL;
+    if (((uint64_t)value_len * c.value_bytes) & 15) return NUPS_EINVAL;       // rows are multiples of 16 bytes
+    if (c.value_bytes == 8 && (c.clip_factor > 0.f || c.sync_period_us)) return NUPS_EINVAL;
+    if ((uint64_t)value_len * (c.value_bytes / 4) > 0xFFFFFFFFull) return NUPS_EINVAL;
+    const uint32_t units = value_len * (c.value_bytes / 4);                     // row length in 4-byte units
     if (c.workers == 0) c.workers = 8;
     if (c.workers > 254) return NUPS_EINVAL;
     if (c.sync_period_us && c.deterministic) return NUPS_EINVAL;
@@ -196,7 +203,7 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     if (c.merge_mean > 1 || (c.merge_mean && c.sync_period_us)) return NUPS_EINVAL;
     if (c.first_epoch > 0xFFFFFFu) return NUPS_EINVAL;
     // what the store holds from the start: tables, technique bitmap, slot map, counts, ownership words, status, loss words
-    const size_t table_bytes = (size_t)num_keys * value_len * sizeof(float);
+    const size_t table_bytes = (size_t)num_keys * units * sizeof(float);
     const size_t bits_bytes = ((num_keys + 31) / 32) * 4, loss_bytes = 4 * NUPS_MAX_STEP_BLOCKS * sizeof(double);
     const size_t need = table_bytes * (c.with_adagrad ? 2 : 1) + bits_bytes + num_keys * 4 + num_keys * 8 +
                         (c.track_ownership ? num_keys * 4 : 0) + sizeof(DevStat) + loss_bytes;
@@ -211,7 +218,8 @@ extern "C" nups_status nups_create(uint64_t num_keys, uint32_t value_len, const 
     CK(cudaGetDevice(&dev));
     nups_store* s = (nups_store*)calloc(1, sizeof(nups_store));
     if (!s) return NUPS_ENOMEM;
-    s->num_keys = num_keys; s->L = value_len; s->R = c.workers; s->cfg = c; s->device = dev;
+    s->num_keys = num_keys; s->L = units; s->value_len = value_len; s->vb = c.value_bytes; s->R = c.workers; s->cfg = c;
+    s->device = dev;
     s->dev_cap = cap;
     s->epoch = c.first_epoch;
     s->ahead_dist = -1;
@@ -277,19 +285,19 @@ extern "C" nups_status nups_destroy(nups_store* s)
     return NUPS_OK;
 }
 
-extern "C" nups_status nups_table_ptr(nups_store* s, int which, float** ptr, uint64_t* stride)
+extern "C" nups_status nups_table_ptr(nups_store* s, int which, void** ptr, uint64_t* stride)
 {
     if (!s || !ptr || (which != 0 && which != 1)) return NUPS_EINVAL;
     if (which == 1 && !s->acc) return NUPS_EINVAL;
     *ptr = which ? s->acc : s->val;
-    if (stride) *stride = s->L;
+    if (stride) *stride = s->value_len;
     return NUPS_OK;
 }
 
-extern "C" nups_status nups_table_copy(nups_store* s, int which, float* d_buf, int to_store, void* stream)
+extern "C" nups_status nups_table_copy(nups_store* s, int which, void* d_buf, int to_store, void* stream)
 {
     if (!s || !d_buf || (which != 0 && which != 1) || (which == 1 && !s->acc)) return NUPS_EINVAL;
-    float* t = which ? s->acc : s->val;
+    void* t = which ? s->acc : s->val;
     size_t bytes = (size_t)s->num_keys * s->L * sizeof(float);
     CK(cudaMemcpyAsync(to_store ? t : d_buf, to_store ? d_buf : t, bytes, cudaMemcpyDeviceToDevice,
                        (cudaStream_t)stream));
@@ -312,14 +320,32 @@ __global__ void init_uniform_kernel(float4* t, uint64_t total4, uint64_t seed, u
     }
 }
 
+// the same values (each exactly representable in fp32) into a table of doubles
+__global__ void init_uniform_f64_kernel(double* t, uint64_t total4, uint64_t seed, uint32_t which, float unit)
+{
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (; i < total4; i += stride) {
+        uint32_t x[4];
+        philox_at(seed, i, which, 3, 0, x);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) t[4 * i + k] = (double)__fmul_rn((float)((int)(x[k] >> 8) - 8388608), unit);
+    }
+}
+
 extern "C" nups_status nups_init_uniform(nups_store* s, int which, uint64_t seed, float scale, void* stream)
 {
     if (!s || (which != 0 && which != 1) || (which == 1 && !s->acc)) return NUPS_EINVAL;
     cudaStream_t st = (cudaStream_t)stream;
-    uint64_t total4 = s->num_keys * (s->L / 4);
+    const uint64_t values = s->num_keys * (uint64_t)s->value_len;
+    if (values & 3) return NUPS_EINVAL;                       // the generator makes four values at a time
+    const uint64_t total4 = values / 4;
     float unit = scale * (1.0f / 8388608.0f);
-    init_uniform_kernel<<<grid_for(total4, 256, (unsigned)s->sm_count * 16), 256, 0, st>>>(
-        (float4*)(which ? s->acc : s->val), total4, seed, (uint32_t)which, unit);
+    const unsigned grid = grid_for(total4, 256, (unsigned)s->sm_count * 16);
+    if (s->vb == 8)
+        init_uniform_f64_kernel<<<grid, 256, 0, st>>>((double*)(which ? s->acc : s->val), total4, seed, (uint32_t)which, unit);
+    else
+        init_uniform_kernel<<<grid, 256, 0, st>>>((float4*)(which ? s->acc : s->val), total4, seed, (uint32_t)which, unit);
     LAUNCH_CHECK(s);
     return NUPS_OK;
 }
@@ -339,7 +365,7 @@ struct TablePair {
     float4* out;           // [n][L]
 };
 
-template <bool HOT, bool TWO>
+template <bool HOT, bool TWO, bool F64>
 __global__ void __launch_bounds__(256, 4)
 gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A, TablePair B, int map,
               uint64_t map_base, uint64_t map_total, int do_count, uint32_t* __restrict__ keys_copy)
@@ -407,8 +433,8 @@ gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A
                         else a[u] = __ldg(A.table + so[u] + c);
                         if (TWO) b[u] = __ldg(B.table + so[u] + c);
                         if (HOT && po[u] != NO_ROW) {
-                            a[u] = add4(a[u], A.slab[po[u] + c]);
-                            if (TWO) b[u] = add4(b[u], B.slab[po[u] + c]);
+                            a[u] = add_chunk<F64>(a[u], A.slab[po[u] + c]);
+                            if (TWO) b[u] = add_chunk<F64>(b[u], B.slab[po[u] + c]);
                         }
                     }
                 }
@@ -530,7 +556,7 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
     // 187 vs 180 us, so those calls keep the 128-bit kernel.)
     const uint32_t c8 = s->L / 8;
     float* out1 = two ? nullptr : A.out ? (float*)A.out : nullptr;
-    if (s->H && !two && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) && ((uintptr_t)out1 & 31) == 0 &&
+    if (s->H && s->vb == 4 && !two && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) && ((uintptr_t)out1 & 31) == 0 &&
         (uint64_t)s->R * s->Hcap < 0xFFFFFFFFull) {
         const float* table = (const float*)A.table;
         const float* slab = (const float*)A.slab;
@@ -547,28 +573,35 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
         return NUPS_OK;
     }
     nups_time_begin(s, st, worker_map == 1 ? NUPS_TIMED_SAMPLE_ROWS : NUPS_TIMED_PULL);
-    if (s->H) {
-        if (two) gather_kernel<true, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
-        else gather_kernel<true, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
+#define NUPS_GATHER(HOT_, TWO_, F64_)                                                                                  \
+    gather_kernel<HOT_, TWO_, F64_><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, \
+                                                          d_keys_copy)
+    if (s->vb == 8) {                        // only replica reads add; rows without a replica are copied whatever they hold
+        if (s->H) { if (two) NUPS_GATHER(true, true, true); else NUPS_GATHER(true, false, true); }
+        else { if (two) NUPS_GATHER(false, true, false); else NUPS_GATHER(false, false, false); }
+    } else if (s->H) {
+        if (two) NUPS_GATHER(true, true, false); else NUPS_GATHER(true, false, false);
     } else {
-        if (two) gather_kernel<false, true><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
-        else gather_kernel<false, false><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, d_keys_copy);
+        if (two) NUPS_GATHER(false, true, false); else NUPS_GATHER(false, false, false);
     }
+#undef NUPS_GATHER
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
     return NUPS_OK;
 }
 
-extern "C" nups_status nups_pull2(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out_val,
-                                  float* d_out_acc, void* stream)
+extern "C" nups_status nups_pull2(nups_store* s, const uint32_t* d_keys, uint64_t n, void* d_out_val_, void* d_out_acc_,
+                                  void* stream)
 {
+    float* d_out_val = (float*)d_out_val_;
+    float* d_out_acc = (float*)d_out_acc_;
     if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
     if (d_out_acc && !s->acc) return NUPS_EINVAL;
     if (n && !d_out_val && !d_out_acc) return NUPS_EINVAL;
     return nups_gather_internal(s, d_keys, n, d_out_val, d_out_acc, 0, 0, n, 1, (cudaStream_t)stream, nullptr);
 }
 
-extern "C" nups_status nups_pull(nups_store* s, const uint32_t* d_keys, uint64_t n, float* d_out, void* stream)
+extern "C" nups_status nups_pull(nups_store* s, const uint32_t* d_keys, uint64_t n, void* d_out, void* stream)
 {
     if (n && !d_out) return NUPS_EINVAL;
     return nups_pull2(s, d_keys, n, d_out, nullptr, stream);
@@ -598,7 +631,7 @@ struct PushPair {
 // takes that key's updates until the block ends (other keys that map there go straight to their rows).  Frequent
 // keys show up early and often, so they take most accumulators, and a skewed batch stops queueing at a few L2
 // addresses even when its frequent keys were never marked for replication.
-template <bool HOT, bool TWO, int TIER>
+template <bool HOT, bool TWO, int TIER, bool F64>
 __global__ void __launch_bounds__(256, 3)
 push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPair A, PushPair B, uint64_t n_items,
                    uint32_t rows_per_item, uint32_t tier_rows)
@@ -733,8 +766,8 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
                         } else {
                             const bool h = HOT && (de[u4] & 1ull);
                             const uint64_t off = (de[u4] >> 3) * 4 + (uint64_t)c * 4;
-                            red_add_v4((h ? A.slab : A.table) + off, a[u4]);
-                            if (TWO) red_add_v4((h ? B.slab : B.table) + off, b[u4]);
+                            red_add_chunk<F64>((h ? A.slab : A.table) + off, a[u4]);
+                            if (TWO) red_add_chunk<F64>((h ? B.slab : B.table) + off, b[u4]);
                         }
                     }
                 }
@@ -776,8 +809,8 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
 #pragma unroll
                     for (int u4 = 0; u4 < PUSH_UNROLL; ++u4) {
                         if (m[u4] >= 0) {
-                            a = add4(a, x[u4]);
-                            if (TWO) b = add4(b, y[u4]);
+                            a = add_chunk<F64>(a, x[u4]);
+                            if (TWO) b = add_chunk<F64>(b, y[u4]);
                         }
                     }
                 }
@@ -786,8 +819,8 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
                     atomicAdd(t, a.x); atomicAdd(t + L4, a.y); atomicAdd(t + 2 * L4, a.z); atomicAdd(t + 3 * L4, a.w);
                 } else {
                     const uint64_t off = (de >> 3) * 4 + (uint64_t)c * 4;
-                    red_add_v4((h ? A.slab : A.table) + off, a);
-                    if (TWO) red_add_v4((h ? B.slab : B.table) + off, b);
+                    red_add_chunk<F64>((h ? A.slab : A.table) + off, a);
+                    if (TWO) red_add_chunk<F64>((h ? B.slab : B.table) + off, b);
                 }
             }
             if (TIER && tr >= 0 && lane == 0 && !((touched[tr >> 5] >> (tr & 31)) & 1u))
@@ -846,6 +879,7 @@ __global__ void push_dest_kernel(View v, const uint32_t* __restrict__ keys, uint
     }
 }
 
+template <bool F64>
 __global__ void __launch_bounds__(256)
 push_ordered_kernel(View v, const unsigned long long* __restrict__ dest, const uint32_t* __restrict__ idx, uint64_t n,
                     unsigned long long invalid_dest, const float4* __restrict__ dv, const float4* __restrict__ da)
@@ -880,17 +914,17 @@ push_ordered_kernel(View v, const unsigned long long* __restrict__ dest, const u
             uint64_t o2 = (uint64_t)idx[p + 2] * L4 + c, o3 = (uint64_t)idx[p + 3] * L4 + c;
             if (dv) {
                 float4 x0 = dv[o0], x1 = dv[o1], x2 = dv[o2], x3 = dv[o3];
-                a = add4(add4(add4(add4(a, x0), x1), x2), x3);
+                a = add_chunk<F64>(add_chunk<F64>(add_chunk<F64>(add_chunk<F64>(a, x0), x1), x2), x3);
             }
             if (da) {
                 float4 y0 = da[o0], y1 = da[o1], y2 = da[o2], y3 = da[o3];
-                b = add4(add4(add4(add4(b, y0), y1), y2), y3);
+                b = add_chunk<F64>(add_chunk<F64>(add_chunk<F64>(add_chunk<F64>(b, y0), y1), y2), y3);
             }
         }
         for (; p < end; ++p) {
             uint64_t o = (uint64_t)idx[p] * L4 + c;
-            if (dv) a = add4(a, dv[o]);
-            if (da) b = add4(b, da[o]);
+            if (dv) a = add_chunk<F64>(a, dv[o]);
+            if (da) b = add_chunk<F64>(b, da[o]);
         }
         if (dv) tv[c] = a;
         if (da) ta[c] = b;
@@ -936,8 +970,8 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
         // shared-memory tier: single-table calls with replicated keys, enough blocks to give every worker some
         uint32_t tier_rows = 0;
         size_t tier_bytes = 0;
-        const bool cache = !s->H && !two && n >= 32768;               // no replicated keys: accumulators as a row cache
-        if ((s->H && !two && rows_per_item == 1 && grid >= s->R && n >= 32768) || cache) {
+        const bool cache = !s->H && !two && n >= 32768 && s->vb == 4;  // no replicated keys: accumulators as a row cache
+        if ((s->H && !two && rows_per_item == 1 && grid >= s->R && n >= 32768 && s->vb == 4) || cache) {
             const size_t row_bytes = (size_t)s->L * 4;
             size_t budget = 64 * 1024;
             const size_t per_row = row_bytes + (cache ? 4 : 0) + 1;    // sums, owner tag, touched bit (rounded up)
@@ -947,27 +981,33 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
             if (!cache && tier_rows > s->H) tier_rows = (uint32_t)s->H;
             tier_bytes = tier_rows * row_bytes + ((tier_rows + 31) / 32) * 4 + (cache ? tier_rows * 4 : 0);
             if (tier_rows && !s->push_smem_opted) {
-                CK(cudaFuncSetAttribute(push_atomic_kernel<true, false, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                CK(cudaFuncSetAttribute(push_atomic_kernel<true, false, 1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(budget + 2048)));
-                CK(cudaFuncSetAttribute(push_atomic_kernel<false, false, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                CK(cudaFuncSetAttribute(push_atomic_kernel<false, false, 2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)(budget + 2048)));
                 s->push_smem_opted = true;
             }
         }
         nups_time_begin(s, st, NUPS_TIMED_PUSH);
         if (tier_rows && cache) {
-            push_atomic_kernel<false, false, 2><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+            push_atomic_kernel<false, false, 2, false><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);
         } else if (tier_rows) {
             grid = grid / s->R * s->R;              // every worker gets the same number of blocks
-            push_atomic_kernel<true, false, 1><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+            push_atomic_kernel<true, false, 1, false><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);
-        } else if (s->H) {
-            if (two) push_atomic_kernel<true, true, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
-            else push_atomic_kernel<true, false, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
         } else {
-            if (two) push_atomic_kernel<false, true, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
-            else push_atomic_kernel<false, false, 0><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0);
+#define NUPS_PUSH0(HOT_, TWO_, F64_) \
+    push_atomic_kernel<HOT_, TWO_, 0, F64_><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0)
+            if (s->vb == 8) {
+                if (s->H) { if (two) NUPS_PUSH0(true, true, true); else NUPS_PUSH0(true, false, true); }
+                else { if (two) NUPS_PUSH0(false, true, true); else NUPS_PUSH0(false, false, true); }
+            } else if (s->H) {
+                if (two) NUPS_PUSH0(true, true, false); else NUPS_PUSH0(true, false, false);
+            } else {
+                if (two) NUPS_PUSH0(false, true, false); else NUPS_PUSH0(false, false, false);
+            }
+#undef NUPS_PUSH0
         }
         nups_time_end(s, st);
         LAUNCH_CHECK(s);
@@ -987,22 +1027,28 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
     LAUNCH_CHECK(s);
     rc = nups_sort_pairs(s, k0, v0, k1, v1, n, bits, sc, st);
     if (rc != NUPS_OK) return rc;
-    push_ordered_kernel<<<grid_for(n * 32, 256), 256, 0, st>>>(v, k1, v1, n, invalid_dest, (const float4*)d_dval,
-                                                               (const float4*)d_dacc);
+    if (s->vb == 8)
+        push_ordered_kernel<true><<<grid_for(n * 32, 256), 256, 0, st>>>(v, k1, v1, n, invalid_dest, (const float4*)d_dval,
+                                                                         (const float4*)d_dacc);
+    else
+        push_ordered_kernel<false><<<grid_for(n * 32, 256), 256, 0, st>>>(v, k1, v1, n, invalid_dest, (const float4*)d_dval,
+                                                                          (const float4*)d_dacc);
     LAUNCH_CHECK(s);
     return NUPS_OK;
 }
 
-extern "C" nups_status nups_push2(nups_store* s, const uint32_t* d_keys, uint64_t n, const float* d_dval,
-                                  const float* d_dacc, void* stream)
+extern "C" nups_status nups_push2(nups_store* s, const uint32_t* d_keys, uint64_t n, const void* d_dval_,
+                                  const void* d_dacc_, void* stream)
 {
+    const float* d_dval = (const float*)d_dval_;
+    const float* d_dacc = (const float*)d_dacc_;
     if (!s || (n && !d_keys) || n >= (1ull << 32)) return NUPS_EINVAL;
     if (d_dacc && !s->acc) return NUPS_EINVAL;
     if (n && !d_dval && !d_dacc) return NUPS_EINVAL;
     return nups_push_internal(s, d_keys, n, 1, d_dval, d_dacc, (cudaStream_t)stream);
 }
 
-extern "C" nups_status nups_push(nups_store* s, const uint32_t* d_keys, uint64_t n, const float* d_delta, void* stream)
+extern "C" nups_status nups_push(nups_store* s, const uint32_t* d_keys, uint64_t n, const void* d_delta, void* stream)
 {
     if (n && !d_delta) return NUPS_EINVAL;
     return nups_push2(s, d_keys, n, d_delta, nullptr, stream);
@@ -1012,6 +1058,7 @@ extern "C" nups_status nups_push(nups_store* s, const uint32_t* d_keys, uint64_t
 // sync: merge the workers' pending updates of every touched hot slot into the stored row,
 // worker 0 first, and clear them.
 // ---------------------------------------------------------------------------------------------
+template <bool F64>
 __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
 {
     const uint32_t L4 = v.L4;
@@ -1041,7 +1088,7 @@ __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 if (d[u]) {
-                    sum = add4(sum, x[u]);
+                    sum = add_chunk<F64>(sum, x[u]);
                     slab[((uint64_t)(r0 + u) * v.Hcap + slot) * L4 + c] = zero;
                 }
             }
@@ -1049,11 +1096,16 @@ __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
         if (v.merge_mean) {                                   // the mean over the workers that touched the slot
             uint32_t touched = 0;
             for (uint32_t r = 0; r < v.R; ++r) touched += v.dirty[(size_t)r * v.Hcap + slot] != 0u;
-            const float by = (float)touched;
-            sum = make_float4(__fdiv_rn(sum.x, by), __fdiv_rn(sum.y, by), __fdiv_rn(sum.z, by), __fdiv_rn(sum.w, by));
+            if (F64) {
+                const double2 d = as_d2(sum);
+                sum = as_f4(make_double2(__ddiv_rn(d.x, (double)touched), __ddiv_rn(d.y, (double)touched)));
+            } else {
+                const float by = (float)touched;
+                sum = make_float4(__fdiv_rn(sum.x, by), __fdiv_rn(sum.y, by), __fdiv_rn(sum.z, by), __fdiv_rn(sum.w, by));
+            }
         }
         float4* row = table + (uint64_t)key * L4 + c;
-        *row = add4(*row, sum);
+        *row = add_chunk<F64>(*row, sum);
     }
 }
 
@@ -1062,7 +1114,8 @@ nups_status nups_sync_internal(nups_store* s, cudaStream_t st)
     if (s->H == 0) return NUPS_OK;        // nothing replicated: no work at all
     View v = nups_view(s);
     nups_background_begin(s, st);
-    sync_kernel<<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
+    if (s->vb == 8) sync_kernel<true><<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
+    else sync_kernel<false><<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) e = cudaMemsetAsync(s->dirty, 0, (size_t)s->R * s->Hcap * sizeof(uint32_t), st);
     nups_background_end(s, st);
@@ -1451,6 +1504,7 @@ red_probe_kernel(float* base, uint64_t n4)
 extern "C" nups_status nups_probe_reduction_rate(nups_store* s, uint64_t bytes, uint32_t reps, double* h_gbs_out, void* stream)
 {
     if (!s || !h_gbs_out || reps == 0) return NUPS_EINVAL;
+    if (s->vb != 4) return NUPS_ESTATE;                       // the probe adds single-precision zeros
     cudaStream_t st = (cudaStream_t)stream;
     const uint64_t table_bytes = (uint64_t)s->num_keys * s->L * sizeof(float);
     if (bytes > table_bytes) bytes = table_bytes;
