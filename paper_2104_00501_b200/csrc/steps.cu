@@ -680,7 +680,16 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             if (v.own && tid < 3) mark_localize(v, key, q);
         }
         __syncthreads();
-        {
+        if constexpr (!F64) {                                      // at most one chunk per thread
+            if (tid < L4) {
+                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rows) + 16 * tid;
+                for (uint32_t role = 0; role < per; ++role) {
+                    cp_async_16s(dst + (2 * role) * LU * 4, v.val + s_row[role] + 4 * tid);
+                    cp_async_16s(dst + (2 * role + 1) * LU * 4, v.acc + s_row[role] + 4 * tid);
+                }
+                asm volatile("cp.async.commit_group;" ::: "memory");
+            }
+        } else {
             const uint32_t dst = (uint32_t)__cvta_generic_to_shared(rows);
             for (uint32_t role = 0; role < per; ++role) {
                 NUPS_CPX_CHUNKS(c) {
@@ -706,18 +715,34 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
                 }
             }
         }
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        if (HOT) {
-            // the worker's pending replica updates join the chunks this thread staged
-            float4* staged = reinterpret_cast<float4*>(rows_raw);
-            for (uint32_t role = 0; role < per; ++role) {
-                const unsigned long long pend = s_pend[role];
-                if (pend == NO_PEND) continue;
-                NUPS_CPX_CHUNKS(c) {
-                    float4* pv = staged + (size_t)(2 * role) * L4 + c;
-                    float4* pa = staged + (size_t)(2 * role + 1) * L4 + c;
-                    *pv = add_chunk<F64>(*pv, *(reinterpret_cast<const float4*>(v.dval + pend) + c));
-                    *pa = add_chunk<F64>(*pa, *(reinterpret_cast<const float4*>(v.dacc + pend) + c));
+        if constexpr (!F64) {
+            if (tid < L4) {
+                asm volatile("cp.async.wait_group 0;" ::: "memory");
+                if (HOT) {
+                    // the worker's pending replica updates join the chunks this thread staged
+                    for (uint32_t role = 0; role < per; ++role) {
+                        const unsigned long long pend = s_pend[role];
+                        if (pend == NO_PEND) continue;
+                        float4* pv = reinterpret_cast<float4*>(rows + (size_t)(2 * role) * L) + tid;
+                        float4* pa = reinterpret_cast<float4*>(rows + (size_t)(2 * role + 1) * L) + tid;
+                        *pv = add4(*pv, *(reinterpret_cast<const float4*>(v.dval + pend) + tid));
+                        *pa = add4(*pa, *(reinterpret_cast<const float4*>(v.dacc + pend) + tid));
+                    }
+                }
+            }
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+            if (HOT) {
+                float4* staged = reinterpret_cast<float4*>(rows_raw);
+                for (uint32_t role = 0; role < per; ++role) {
+                    const unsigned long long pend = s_pend[role];
+                    if (pend == NO_PEND) continue;
+                    NUPS_CPX_CHUNKS(c) {
+                        float4* pv = staged + (size_t)(2 * role) * L4 + c;
+                        float4* pa = staged + (size_t)(2 * role + 1) * L4 + c;
+                        *pv = add_chunk<true>(*pv, *(reinterpret_cast<const float4*>(v.dval + pend) + c));
+                        *pa = add_chunk<true>(*pa, *(reinterpret_cast<const float4*>(v.dacc + pend) + c));
+                    }
                 }
             }
         }
@@ -784,19 +809,38 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
             cx_adagrad(gt, val_row(2), acc_row(2), d, tid, lrT, epsT);
         }
         __syncthreads();
-        for (uint32_t role = 0; role < per; ++role) {
-            NUPS_CPX_CHUNKS(c) {
-                const float4 dv = reinterpret_cast<const float4*>(val_row(role))[c];
-                const float4 da = reinterpret_cast<const float4*>(acc_row(role))[c];
-                if (DET) {
-                    reinterpret_cast<float4*>(uval + (i * per + role) * (uint64_t)LU)[c] = dv;
-                    reinterpret_cast<float4*>(uacc + (i * per + role) * (uint64_t)LU)[c] = da;
-                } else {
-                    const unsigned long long pend = s_pend[role];
-                    float* ov = pend != NO_PEND ? v.dval + pend : v.val + s_row[role];
-                    float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + s_row[role];
-                    red_add_chunk<F64>(ov + 4 * c, dv);
-                    red_add_chunk<F64>(oa + 4 * c, da);
+        if constexpr (!F64) {
+            if (tid < L4) {
+                for (uint32_t role = 0; role < per; ++role) {
+                    const float4 dv = reinterpret_cast<const float4*>(val_row(role))[tid];
+                    const float4 da = reinterpret_cast<const float4*>(acc_row(role))[tid];
+                    if (DET) {
+                        reinterpret_cast<float4*>(uval + (i * per + role) * (uint64_t)LU)[tid] = dv;
+                        reinterpret_cast<float4*>(uacc + (i * per + role) * (uint64_t)LU)[tid] = da;
+                    } else {
+                        const unsigned long long pend = s_pend[role];
+                        float* ov = pend != NO_PEND ? v.dval + pend : v.val + s_row[role];
+                        float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + s_row[role];
+                        red_add_v4(ov + 4 * tid, dv);
+                        red_add_v4(oa + 4 * tid, da);
+                    }
+                }
+            }
+        } else {
+            for (uint32_t role = 0; role < per; ++role) {
+                NUPS_CPX_CHUNKS(c) {
+                    const float4 dv = reinterpret_cast<const float4*>(val_row(role))[c];
+                    const float4 da = reinterpret_cast<const float4*>(acc_row(role))[c];
+                    if (DET) {
+                        reinterpret_cast<float4*>(uval + (i * per + role) * (uint64_t)LU)[c] = dv;
+                        reinterpret_cast<float4*>(uacc + (i * per + role) * (uint64_t)LU)[c] = da;
+                    } else {
+                        const unsigned long long pend = s_pend[role];
+                        float* ov = pend != NO_PEND ? v.dval + pend : v.val + s_row[role];
+                        float* oa = pend != NO_PEND ? v.dacc + pend : v.acc + s_row[role];
+                        red_add_chunk<true>(ov + 4 * c, dv);
+                        red_add_chunk<true>(oa + 4 * c, da);
+                    }
                 }
             }
         }
