@@ -58,13 +58,16 @@ WORKLOAD_PS = ("PS microbenchmark: 100M keys x 128 fp32, 1M-key batches ~ Zipf(1
 # (dram__bytes_read.sum + dram__bytes_write.sum); valid only for the kernel source it was captured on (sgns_kernel_sha1).
 NCU_TRAFFIC = {"bytes_per_launch": 41620224, "sgns_kernel_sha1": "48f21389a1da332791a366ac05ca6a967def1b94"}
 
-# The same for the kernels of the default line, each from one ncu capture of a 1M-key launch at the line's own
-# configuration (see profiles/): bytes per launch and the hash of the kernel's source text at the time of the capture.
-# A kernel whose source has changed since reports no traffic.
+# The same for the kernels of the default line.  A 100M-key launch is too large to capture under ncu, so each figure comes
+# from one capture of the same command with --ps-keys 4000000 (2 GB table, the same 1M-key batches, kernels and launch shapes;
+# see profiles/ps_line_kernels_dram_traffic.md): DRAM bytes of that launch, its algorithmic bytes, and the hash of the
+# kernel's source text at the time.  The traffic reported for the timed launch is scaled by the algorithmic bytes, which is
+# what the capture shows the traffic follows.  A kernel whose source has changed since reports no traffic.
 NCU_TRAFFIC_PS = {
-    "pull": {"bytes_per_launch": None, "sha1": None},
-    "push": {"bytes_per_launch": None, "sha1": None},
-    "sample_rows": {"bytes_per_launch": None, "sha1": None},
+    "pull": {"dram_bytes": 216868608 + 481223168, "algorithmic_bytes": 694418688, "sha1": "b5c5269d9508cff997a885e6dfe9a9a4db40087a"},
+    "push": {"dram_bytes": 712465664 + 126748160, "algorithmic_bytes": 847772160, "sha1": "9b4554f0f9febfe25eb8b01cdb087d578b1a276e"},
+    "sample_rows": {"dram_bytes": 27684864 + 478492928, "algorithmic_bytes": 562094080,
+                    "sha1": "b5c5269d9508cff997a885e6dfe9a9a4db40087a"},
 }
 PS_KERNEL_SOURCE = {   # kind -> (kernel name, start and end markers of its source text in store.cu)
     "pull": ("gather8_kernel", "// The same gather with 256-bit loads and stores", "nups_status nups_gather_internal("),
@@ -701,7 +704,7 @@ def run_ps_line(args, rank, world, device):
         alg = ps.alg_bytes(kind, ucold[kind])
         name, m0, m1 = PS_KERNEL_SOURCE[kind]
         cap = NCU_TRAFFIC_PS[kind]
-        traffic = cap["bytes_per_launch"] if cap["sha1"] and cap["sha1"] == kernel_source_sha1(m0, m1) else None
+        traffic = (cap["dram_bytes"] * alg / cap["algorithmic_bytes"] if cap["sha1"] == kernel_source_sha1(m0, m1) else None)
         kernels[kind] = {"kernel": name, "kernel_us": t * 1e6, "launches": int(k_n), "achieved": alg / t / 1e9,
                          "frac": alg / t / 1e9 / hbm_peak, "algorithmic_bytes_per_launch": alg,
                          "distinct_cold_rows": ucold[kind], "traffic": traffic,
@@ -774,6 +777,7 @@ def run_ps_line(args, rank, world, device):
         "gpu_launches": int(round(launches)),
         "roofline": {"bound": "hbm", "kernel": f"{dk['kernel']} ({dominant})", "achieved": dk["achieved"], "peak": hbm_peak,
                      "peak_kind": peak_kind, "unit": "GB/s", "frac": dk["frac"], "traffic": dk["traffic"],
+                     "traffic_note": "ncu DRAM bytes of a 1M-key launch on a 4M-key table, scaled by the algorithmic bytes",
                      "algorithmic_bytes_per_launch": dk["algorithmic_bytes_per_launch"], "kernel_us": dk["kernel_us"],
                      "kernels": kernels, "draw_kernel_us": draw_ms / max(draw_n, 1) * 1e3},
     }
