@@ -54,9 +54,9 @@ WORKLOAD_PS = ("PS microbenchmark: 100M keys x 128 fp32, 1M-key batches ~ Zipf(1
                "over 8 workers, replicas merged every 16 batches, plus PrepareSample+PullSample of 1M keys from a Zipf(1.0) "
                "target under BOUNDED(U=16,G=250); one step = one pull + one push + one sample pull, fast (atomic) mode")
 
-# DRAM traffic of one launch of the fused step kernel (16 steps per launch), from an ncu capture
+# DRAM traffic of one launch of the fused step kernel (sgns_runs_kernel, 16 steps per launch, 10M-token stream), from an ncu capture
 # (dram__bytes_read.sum + dram__bytes_write.sum); valid only for the kernel source it was captured on (sgns_kernel_sha1).
-NCU_TRAFFIC = {"bytes_per_launch": 41620224, "sgns_kernel_sha1": "48f21389a1da332791a366ac05ca6a967def1b94"}
+NCU_TRAFFIC = {"bytes_per_launch": 38886656 + 4509952, "sgns_kernel_sha1": "a667c3d0875db94740ac74690bf25a99019ad7aa"}
 
 # The same for the kernels of the default line.  A 100M-key launch is too large to capture under ncu, so each figure comes
 # from one capture of the same command with --ps-keys 4000000 (2 GB table, the same 1M-key batches, kernels and launch shapes;
@@ -64,10 +64,10 @@ NCU_TRAFFIC = {"bytes_per_launch": 41620224, "sgns_kernel_sha1": "48f21389a1da33
 # kernel's source text at the time.  The traffic reported for the timed launch is scaled by the algorithmic bytes, which is
 # what the capture shows the traffic follows.  A kernel whose source has changed since reports no traffic.
 NCU_TRAFFIC_PS = {
-    "pull": {"dram_bytes": 216868608 + 481223168, "algorithmic_bytes": 694418688, "sha1": "b5c5269d9508cff997a885e6dfe9a9a4db40087a"},
-    "push": {"dram_bytes": 712465664 + 126748160, "algorithmic_bytes": 847772160, "sha1": "9b4554f0f9febfe25eb8b01cdb087d578b1a276e"},
-    "sample_rows": {"dram_bytes": 27684864 + 478492928, "algorithmic_bytes": 562094080,
-                    "sha1": "b5c5269d9508cff997a885e6dfe9a9a4db40087a"},
+    "pull": {"dram_bytes": 216834048 + 481267712, "algorithmic_bytes": 694418688, "sha1": "d6be6ab4363bba8db6eba30551f6fe4750727ba0"},
+    "push": {"dram_bytes": 712477440 + 126427904, "algorithmic_bytes": 847772160, "sha1": "029989f9f74886ae15aab066044712e5cb64b40a"},
+    "sample_rows": {"dram_bytes": 27761408 + 478582016, "algorithmic_bytes": 562094080,
+                    "sha1": "d6be6ab4363bba8db6eba30551f6fe4750727ba0"},
 }
 PS_KERNEL_SOURCE = {   # kind -> (kernel name, start and end markers of its source text in store.cu)
     "pull": ("gather8_kernel", "// The same gather with 256-bit loads and stores", "nups_status nups_gather_internal("),
@@ -353,7 +353,7 @@ def run_sgns_line(args, rank, world, device):
                 "one_call_per_step": {"value": step_calls * BATCH * world * ACCESSES_PER_PAIR / per_step_s,
                                       "unit": "key accesses/s", "steps": step_calls}},
         "gpu_launches": int(launches),
-        "roofline": {"bound": "hbm", "kernel": "sgns_kernel (fused step)", "achieved": alg_bytes / k_s / 1e9,
+        "roofline": {"bound": "hbm", "kernel": "sgns_runs_kernel (fused step, 16 steps per launch)", "achieved": alg_bytes / k_s / 1e9,
                      "peak": hbm_peak, "peak_kind": peak_kind, "unit": "GB/s",
                      "frac": alg_bytes / k_s / 1e9 / hbm_peak, "traffic": traffic,
                      "algorithmic_bytes_per_launch": alg_bytes, "logical_bytes_per_launch": logical_bytes,

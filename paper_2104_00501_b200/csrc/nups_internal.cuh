@@ -165,6 +165,38 @@ nups_status nups_dev_alloc(nups_store* s, void** p, size_t bytes);
 void nups_dev_free(nups_store* s, void* p, size_t bytes);
 nups_status nups_new_epoch(nups_store* s, cudaStream_t st);          // call before taking the view of a call that moves keys
 
+// Programmatic dependent launch.  A kernel started through nups_launch_dependent may become resident while the kernel
+// before it on the stream is still draining its last blocks, which hides the launch latency between the back-to-back
+// kernels of a training loop.  Such a kernel calls grid_dependency_wait() before its first access to global memory: the
+// wait returns once every earlier kernel of the stream has finished and its writes are visible, so the order of the
+// stream's work is what it is with a plain launch.  The call is a no-op in a kernel that was launched the plain way.
+// It also lets the NEXT kernel of the stream become resident early; that one can only start once every block of this
+// kernel has been scheduled, so the blocks waiting there never take a place that this kernel still needs.
+#ifdef __CUDACC__
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;");
+}
+
+template <class... KArgs, class... Args>
+static inline cudaError_t nups_launch_dependent(void (*kernel)(KArgs...), dim3 grid, unsigned block, size_t smem,
+                                                cudaStream_t st, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#endif
+
 // background.cu
 nups_status nups_background_start(nups_store* s, uint32_t period_us);
 void nups_background_stop(nups_store* s);

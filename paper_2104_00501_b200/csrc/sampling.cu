@@ -335,6 +335,7 @@ __device__ __forceinline__ uint32_t first_local_warp(const View& v, const DrawPa
 __global__ void draw_iid_kernel(View v, DrawParams p, const unsigned long long* __restrict__ off_cur,
                                 unsigned long long* __restrict__ off_next, HandleView h, uint64_t N, int localize)
 {
+    grid_dependency_wait();
     const uint32_t R = v.R;
     if (blockIdx.x == 0)
         for (uint32_t w = threadIdx.x; w < R; w += blockDim.x)
@@ -460,6 +461,7 @@ __global__ void draw_reuse_kernel(View v, DrawParams p, const unsigned long long
                                   unsigned long long* __restrict__ off_next, HandleView h, uint64_t N, int localize,
                                   int longterm, uint32_t T)
 {
+    grid_dependency_wait();
     const uint32_t q = blockIdx.y, R = v.R;
     const unsigned long long b0 = chunk_begin(q, N, R), size = chunk_begin(q + 1, N, R) - b0;
     const unsigned long long s0 = off_cur[q];
@@ -517,10 +519,10 @@ static nups_status prepare_internal(nups_store* s, int32_t dist, uint64_t N, int
     nups_time_begin(s, st, NUPS_TIMED_DRAW);
     if (reuse) {
         const ReuseShape sh = reuse_shape(d.U, d.G);
-        draw_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R), REUSE_THREADS, sh.smem, st>>>(
-            v, p, off_cur, off_next, hv, N, loc, d.level == NUPS_LONGTERM, sh.T);
+        nups_launch_dependent(draw_reuse_kernel, dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R), REUSE_THREADS,
+                              sh.smem, st, v, p, off_cur, off_next, hv, N, loc, d.level == NUPS_LONGTERM, sh.T);
     } else {
-        draw_iid_kernel<<<grid_for(N, 256), 256, 0, st>>>(v, p, off_cur, off_next, hv, N, loc);
+        nups_launch_dependent(draw_iid_kernel, grid_for(N, 256), 256, 0, st, v, p, off_cur, off_next, hv, N, loc);
     }
     nups_time_end(s, st);
     LAUNCH_CHECK(s);
@@ -561,6 +563,7 @@ __device__ __forceinline__ void count_sample(const View& v, uint32_t key, bool e
 __global__ void emit_kernel(View v, DrawParams p, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, int local_only,
                             uint32_t* __restrict__ out)
 {
+    grid_dependency_wait();
     uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     bool in = o < n;
     uint32_t k = 0;
@@ -603,6 +606,7 @@ __device__ __forceinline__ LtChunk lt_chunk(uint32_t q, uint64_t N, uint32_t R, 
 
 __global__ void lt_flags_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first)
 {
+    grid_dependency_wait();
     const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
     if (!c.active) return;
     const unsigned lane = threadIdx.x & 31;
@@ -622,6 +626,7 @@ __global__ void __launch_bounds__(LT_THREADS)
 lt_scan_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, uint32_t q_first,
                uint32_t* __restrict__ out)
 {
+    grid_dependency_wait();
     __shared__ unsigned sh_tl, sh_old;
     __shared__ unsigned warp_tot[LT_THREADS / 32];
     __shared__ unsigned long long sh_stop;       // walk position right after the last entry that must be emitted
@@ -710,6 +715,7 @@ lt_place_kernel(View v, HandleView h, uint64_t N, uint64_t cursor, uint64_t n, u
                 uint32_t* __restrict__ out, const float* __restrict__ table, const float* slab,
                 float* __restrict__ out_vals)
 {
+    grid_dependency_wait();
     const LtChunk c = lt_chunk(q_first + blockIdx.y, N, v.R, cursor, n);
     if (!c.active) return;
     const unsigned lane = threadIdx.x & 31;
@@ -805,9 +811,9 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         }
         const uint64_t max_size = (h.N + s->R - 1) / s->R;
         const dim3 by_word(grid_for(max_size / 32 + 2, 8), ql - qf + 1);
-        lt_flags_kernel<<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf);
+        nups_launch_dependent(lt_flags_kernel, by_word, 256, 0, st, v, hv, h.N, h.cursor, n, qf);
         LAUNCH_CHECK(s);
-        lt_scan_kernel<<<ql - qf + 1, LT_THREADS, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out);
+        nups_launch_dependent(lt_scan_kernel, ql - qf + 1, LT_THREADS, 0, st, v, hv, h.N, h.cursor, n, qf, d_keys_out);
         LAUNCH_CHECK(s);
         // a full pull of a fresh handle has no entries postponed by earlier calls to emit: the placement pass can copy
         // the rows itself (one table of 64, 128 or 256 floats per row, 32-byte aligned output)
@@ -815,10 +821,10 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         const bool fused = d_vals_out && s->vb == 4 && h.cursor == 0 && n == h.N && s->L % 8 == 0 && (c8 == 8 || c8 == 16 || c8 == 32) &&
                            ((uintptr_t)d_vals_out & 31) == 0 && (uint64_t)s->R * s->Hcap < 0xFFFFFFFFull;
         if (fused) nups_time_begin(s, st, NUPS_TIMED_SAMPLE_ROWS);
-        if (fused && c8 == 8) lt_place_kernel<8><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
-        else if (fused && c8 == 16) lt_place_kernel<16><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
-        else if (fused) lt_place_kernel<32><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
-        else lt_place_kernel<0><<<by_word, 256, 0, st>>>(v, hv, h.N, h.cursor, n, qf, d_keys_out, nullptr, nullptr, nullptr);
+        if (fused && c8 == 8) nups_launch_dependent(lt_place_kernel<8>, by_word, 256, 0, st, v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
+        else if (fused && c8 == 16) nups_launch_dependent(lt_place_kernel<16>, by_word, 256, 0, st, v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
+        else if (fused) nups_launch_dependent(lt_place_kernel<32>, by_word, 256, 0, st, v, hv, h.N, h.cursor, n, qf, d_keys_out, s->val, s->dval, d_vals_out);
+        else nups_launch_dependent(lt_place_kernel<0>, by_word, 256, 0, st, v, hv, h.N, h.cursor, n, qf, d_keys_out, nullptr, nullptr, nullptr);
         if (fused) nups_time_end(s, st);
         LAUNCH_CHECK(s);
         if (fused) {
@@ -833,7 +839,7 @@ static nups_status pull_internal(nups_store* s, int id, uint64_t n, uint32_t* d_
         if (h.cursor == h.N) h.used = 0;
         return nups_gather_internal(s, hv.keys + (h.cursor - n), n, d_vals_out, nullptr, 1, h.cursor - n, h.N, 0, st, d_keys_out);
     } else {
-        emit_kernel<<<grid_for(n, 256), 256, 0, st>>>(v, p, hv, h.N, h.cursor, n, d.level == NUPS_NONCONFORM, d_keys_out);
+        nups_launch_dependent(emit_kernel, grid_for(n, 256), 256, 0, st, v, p, hv, h.N, h.cursor, n, d.level == NUPS_NONCONFORM, d_keys_out);
         LAUNCH_CHECK(s);
     }
     if (d_vals_out) {
@@ -864,6 +870,7 @@ __global__ void draw_direct_iid_kernel(View v, DrawParams p, const unsigned long
                                        unsigned long long* __restrict__ off_next, uint64_t N, uint32_t batches,
                                        int local_only, int localize, uint32_t* __restrict__ out)
 {
+    grid_dependency_wait();
     const uint64_t o = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t bt = blockIdx.y;
     const bool in = o < N;
@@ -890,6 +897,7 @@ __global__ void draw_direct_reuse_kernel(View v, DrawParams p, const unsigned lo
                                          unsigned long long* __restrict__ off_next, uint64_t N, uint32_t batches,
                                          int localize, uint32_t* __restrict__ out, uint32_t T)
 {
+    grid_dependency_wait();
     const uint32_t q = blockIdx.y, R = v.R;
     if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0)
         for (uint32_t w = threadIdx.x; w < R; w += blockDim.x)
@@ -982,10 +990,10 @@ nups_status nups_draw_negatives(nups_store* s, int32_t dist, uint64_t N, cudaStr
     unsigned long long* off_next = d.off + (size_t)(d.cur ^ 1) * s->R;
     if (d.level == NUPS_BOUNDED) {
         const ReuseShape sh = reuse_shape(d.U, d.G);
-        draw_direct_reuse_kernel<<<dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R, batches), REUSE_THREADS, sh.smem,
-                                   st>>>(v, p, off_cur, off_next, N, batches, localize, s->negs_buf, sh.T);
+        nups_launch_dependent(draw_direct_reuse_kernel, dim3(reuse_pools((N + s->R - 1) / s->R, d.U, d.G), s->R, batches),
+                              REUSE_THREADS, sh.smem, st, v, p, off_cur, off_next, N, batches, localize, s->negs_buf, sh.T);
     } else {
-        draw_direct_iid_kernel<<<dim3(grid_for(N, 256), batches), 256, 0, st>>>(v, p, off_cur, off_next, N, batches,
+        nups_launch_dependent(draw_direct_iid_kernel, dim3(grid_for(N, 256), batches), 256, 0, st, v, p, off_cur, off_next, N, batches,
                                                                               d.level == NUPS_NONCONFORM, localize,
                                                                               s->negs_buf);
     }

@@ -109,6 +109,7 @@ sgns_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __restr
             float* __restrict__ loss_out, uint32_t group,
             unsigned long long* __restrict__ loss_acc, float2* __restrict__ clip_item)
 {
+    grid_dependency_wait();
     extern __shared__ __align__(16) float4 park_all[];
     __shared__ const float4* s_src[SGNS_WARPS][32];                // the role's stored row
     __shared__ float* s_dst[SGNS_WARPS][32];                       // where its update goes: replica row or stored row
@@ -323,6 +324,7 @@ sgns_runs_kernel(View v, const uint32_t* __restrict__ center, const uint32_t* __
                  const uint32_t* __restrict__ negs, uint64_t n, float lr, float* __restrict__ loss_out, uint32_t group,
                  unsigned long long* __restrict__ loss_acc)
 {
+    grid_dependency_wait();
     constexpr unsigned FULL = 0xFFFFFFFFu;
     constexpr int K = 3;
     const unsigned lane = threadIdx.x & 31;
@@ -646,6 +648,7 @@ complex_kernel(View v, const uint32_t* __restrict__ hk, const uint32_t* __restri
                float* __restrict__ uacc, uint32_t* __restrict__ ukeys, float* __restrict__ loss_item,
                float* __restrict__ loss_out)
 {
+    grid_dependency_wait();
     using S = typename std::conditional<F64, double, float>::type;          // what the tables hold
     using T = typename std::conditional<DET || F64, double, float>::type;   // what the step computes in
     // rows[2 * role] = the role's value row, rows[2 * role + 1] = its accumulator row, as they lie in memory
@@ -876,6 +879,7 @@ mf_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict_
           uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
           float* __restrict__ loss_item, float* __restrict__ loss_out, float2* __restrict__ clip_item)
 {
+    grid_dependency_wait();
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -1186,7 +1190,7 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
                 const uint64_t cap = (uint64_t)s->sm_count * (unsigned)fit;
                 const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);
                 nups_time_begin(s, st, NUPS_TIMED_STEP);
-                kern<<<grid, SGNS_RUN_THREADS, 0, st>>>(v, d_center, d_context, s->last_negs, n, lr, d_loss_out, group, loss_acc);
+                nups_launch_dependent(kern, grid, SGNS_RUN_THREADS, 0, st, v, d_center, d_context, s->last_negs, n, lr, d_loss_out, group, loss_acc);
                 nups_time_end(s, st);
             }
         });
@@ -1217,7 +1221,7 @@ static nups_status sgns_launch(nups_store* s, const uint32_t* d_center, const ui
             const uint64_t cap = (uint64_t)s->sm_count * per_sm;                                                       \
             const unsigned grid = (unsigned)(blocks_needed < cap ? blocks_needed : cap);                               \
             nups_time_begin(s, st, NUPS_TIMED_STEP);                                                                                    \
-            kern<<<grid, 32 * SGNS_WARPS, smem, st>>>(v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
+            nups_launch_dependent(kern, grid, 32 * SGNS_WARPS, smem, st, v, d_center, d_context, s->last_negs, n, K, lr, b.uval, b.ukeys, \
                                                       b.loss_item, d_loss_out, group,                                  \
                                                       loss_acc, b.clip_item);                                          \
             nups_time_end(s, st);                                                                                      \
@@ -1261,6 +1265,7 @@ extern "C" nups_status nups_step_sgns(nups_store* s, const uint32_t* d_center, c
 // per-step losses of a grouped launch: fixed-point sums -> means, and the sums are cleared for the next group
 __global__ void loss_group_kernel(unsigned long long* acc, uint32_t group, uint64_t n, float* loss_out)
 {
+    grid_dependency_wait();
     const uint32_t g = threadIdx.x;
     if (g >= group) return;
     unsigned long long sum = 0;
@@ -1318,7 +1323,7 @@ extern "C" nups_status nups_run_sgns(nups_store* s, const uint32_t* d_center, co
         if (group > 1) s->ahead_next += (uint32_t)(group - 1);            // those batches are handed out now
         rc = sgns_launch(s, d_center + t * batch, d_context + t * batch, batch, K, lr, b, nullptr, (uint32_t)group, acc, st);
         if (rc != NUPS_OK) return rc;
-        loss_group_kernel<<<1, LOSS_STEPS, 0, st>>>(acc, (uint32_t)group, batch, d_loss_out ? d_loss_out + t : nullptr);
+        nups_launch_dependent(loss_group_kernel, 1, LOSS_STEPS, 0, st, acc, (uint32_t)group, batch, d_loss_out ? d_loss_out + t : nullptr);
         LAUNCH_CHECK(s);
         if (s->cfg.clip_factor > 0.f && s->H) {
             clip_fold_kernel<<<1, 256, 0, st>>>(s->st, nullptr, 0);      // the launch's clipping statistics join the rest
@@ -1378,7 +1383,7 @@ extern "C" nups_status nups_step_complex(nups_store* s, const uint32_t* d_h, con
             s->complex_smem_opted[hi][di][ri][fi] = (e == cudaSuccess);                                              \
         }                                                                                                            \
         if (e == cudaSuccess)                                                                                        \
-            kern<<<grid, CPX_THREADS, smem, st>>>(v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc,     \
+            nups_launch_dependent(kern, grid, CPX_THREADS, smem, st, v, d_h, d_r, d_t, s->last_negs, n, K, lr, eps, b.uval, b.uacc, \
                                                   b.ukeys, b.loss_item, d_loss_out);                                 \
     })
     if (fi) { if (ri) NUPS_CPX_GO(true, true); else NUPS_CPX_GO(false, true); }
@@ -1409,6 +1414,7 @@ __global__ void __launch_bounds__(128, MF_RUN_BLOCKS)
 mf_runs_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restrict__ colk, const float* __restrict__ x,
                uint64_t n, float lr, float l2, float* __restrict__ loss_out)
 {
+    grid_dependency_wait();
     constexpr unsigned FULL = 0xFFFFFFFFu;
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -1594,6 +1600,7 @@ mf_f64_kernel(View v, const uint32_t* __restrict__ rowk, const uint32_t* __restr
               uint64_t n, float lr, float l2, float* __restrict__ upd, uint32_t* __restrict__ ukeys,
               float* __restrict__ loss_item, float* __restrict__ loss_out)
 {
+    grid_dependency_wait();
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -1673,17 +1680,17 @@ static nups_status mf_step(nups_store* s, const uint32_t* d_row, const uint32_t*
     nups_time_begin(s, st, NUPS_TIMED_STEP);
     if (s->vb == 8) {
         const unsigned grid = step_grid(s, n, 8);
-        DISPATCH_MODE(s, mf_f64_kernel<HOT, DET><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys,
+        DISPATCH_MODE(s, nups_launch_dependent(mf_f64_kernel<HOT, DET>, grid, 128, 0, st, v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys,
                                                                       b.loss_item, d_loss_out));
     } else if (by_column) {
         const unsigned grid = step_grid(s, n, MF_RUN_BLOCKS);
         DISPATCH_CLIP(s, DISPATCH_CH(v.L4, {
-            if (s->H) mf_runs_kernel<true, CH, CLIP><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, d_loss_out);
-            else mf_runs_kernel<false, CH, false><<<grid, 128, 0, st>>>(v, d_row, d_col, d_x, n, lr, l2, d_loss_out);
+            if (s->H) nups_launch_dependent(mf_runs_kernel<true, CH, CLIP>, grid, 128, 0, st, v, d_row, d_col, d_x, n, lr, l2, d_loss_out);
+            else nups_launch_dependent(mf_runs_kernel<false, CH, false>, grid, 128, 0, st, v, d_row, d_col, d_x, n, lr, l2, d_loss_out);
         }));
     } else {
         const unsigned grid = step_grid(s, n, MF_DEPTH <= 2 ? 6 : (MF_DEPTH <= 4 ? 4 : 2));   // resident blocks at that depth's register use
-        DISPATCH_MODE(s, DISPATCH_CLIP(s, DISPATCH_CH(v.L4, mf_kernel<HOT, DET, CH, (HOT && CLIP)><<<grid, 128, 0, st>>>(
+        DISPATCH_MODE(s, DISPATCH_CLIP(s, DISPATCH_CH(v.L4, nups_launch_dependent(mf_kernel<HOT, DET, CH, (HOT && CLIP)>, grid, 128, 0, st,
             v, d_row, d_col, d_x, n, lr, l2, b.uval, b.ukeys, b.loss_item, d_loss_out, b.clip_item))));
     }
     nups_time_end(s, st);

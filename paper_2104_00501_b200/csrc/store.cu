@@ -370,6 +370,7 @@ __global__ void __launch_bounds__(256, 4)
 gather_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, TablePair A, TablePair B, int map,
               uint64_t map_base, uint64_t map_total, int do_count, uint32_t* __restrict__ keys_copy)
 {
+    grid_dependency_wait();
     const unsigned lane = threadIdx.x & 31;
     const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint64_t nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
@@ -462,6 +463,7 @@ gather8_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, const floa
                const float* slab, float* __restrict__ out, int map, uint64_t map_base, uint64_t map_total, int do_count,
                uint32_t* __restrict__ keys_copy)
 {
+    grid_dependency_wait();
     constexpr int RPI = 32 / C8;                       // rows per warp instruction
     constexpr int UNR = 2;                             // instructions in flight
     const unsigned lane = threadIdx.x & 31;
@@ -562,7 +564,7 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
         const float* slab = (const float*)A.slab;
         nups_time_begin(s, st, worker_map == 1 ? NUPS_TIMED_SAMPLE_ROWS : NUPS_TIMED_PULL);
 #define NUPS_G8(C8_)                                                                                                     \
-        gather8_kernel<true, C8_><<<grid, 256, 0, st>>>(v, d_keys, n, table, slab, out1, worker_map, map_base, map_total, \
+        nups_launch_dependent(gather8_kernel<true, C8_>, grid, 256, 0, st, v, d_keys, n, table, slab, out1, worker_map, map_base, map_total, \
                                                         do_count, d_keys_copy)
         if (c8 == 8) NUPS_G8(8);
         else if (c8 == 16) NUPS_G8(16);
@@ -574,7 +576,7 @@ nups_status nups_gather_internal(nups_store* s, const uint32_t* d_keys, uint64_t
     }
     nups_time_begin(s, st, worker_map == 1 ? NUPS_TIMED_SAMPLE_ROWS : NUPS_TIMED_PULL);
 #define NUPS_GATHER(HOT_, TWO_, F64_)                                                                                  \
-    gather_kernel<HOT_, TWO_, F64_><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, \
+    nups_launch_dependent(gather_kernel<HOT_, TWO_, F64_>, grid, 256, 0, st, v, d_keys, n, A, B, worker_map, map_base, map_total, do_count, \
                                                           d_keys_copy)
     if (s->vb == 8) {                        // only replica reads add; rows without a replica are copied whatever they hold
         if (s->H) { if (two) NUPS_GATHER(true, true, true); else NUPS_GATHER(true, false, true); }
@@ -636,6 +638,7 @@ __global__ void __launch_bounds__(256, 3)
 push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPair A, PushPair B, uint64_t n_items,
                    uint32_t rows_per_item, uint32_t tier_rows)
 {
+    grid_dependency_wait();
     extern __shared__ __align__(16) float tier_mem[];                  // TIER: [tier_rows][L] sums, then touched bits
     const unsigned lane = threadIdx.x & 31;
     const uint32_t L4 = v.L4;
@@ -990,15 +993,15 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
         }
         nups_time_begin(s, st, NUPS_TIMED_PUSH);
         if (tier_rows && cache) {
-            push_atomic_kernel<false, false, 2, false><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+            nups_launch_dependent(push_atomic_kernel<false, false, 2, false>, grid, 256, tier_bytes, st, v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);
         } else if (tier_rows) {
             grid = grid / s->R * s->R;              // every worker gets the same number of blocks
-            push_atomic_kernel<true, false, 1, false><<<grid, 256, tier_bytes, st>>>(v, d_keys, n, A, B, n_items, rows_per_item,
+            nups_launch_dependent(push_atomic_kernel<true, false, 1, false>, grid, 256, tier_bytes, st, v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);
         } else {
 #define NUPS_PUSH0(HOT_, TWO_, F64_) \
-    push_atomic_kernel<HOT_, TWO_, 0, F64_><<<grid, 256, 0, st>>>(v, d_keys, n, A, B, n_items, rows_per_item, 0)
+    nups_launch_dependent(push_atomic_kernel<HOT_, TWO_, 0, F64_>, grid, 256, 0, st, v, d_keys, n, A, B, n_items, rows_per_item, 0)
             if (s->vb == 8) {
                 if (s->H) { if (two) NUPS_PUSH0(true, true, true); else NUPS_PUSH0(true, false, true); }
                 else { if (two) NUPS_PUSH0(false, true, true); else NUPS_PUSH0(false, false, true); }
@@ -1061,6 +1064,7 @@ extern "C" nups_status nups_push(nups_store* s, const uint32_t* d_keys, uint64_t
 template <bool F64>
 __global__ void sync_kernel(View v, const uint32_t* __restrict__ hot_keys)
 {
+    grid_dependency_wait();
     const uint32_t L4 = v.L4;
     uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     uint64_t total = (uint64_t)v.H * L4;
@@ -1114,8 +1118,8 @@ nups_status nups_sync_internal(nups_store* s, cudaStream_t st)
     if (s->H == 0) return NUPS_OK;        // nothing replicated: no work at all
     View v = nups_view(s);
     nups_background_begin(s, st);
-    if (s->vb == 8) sync_kernel<true><<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
-    else sync_kernel<false><<<grid_for(s->H * (s->L / 4), 256), 256, 0, st>>>(v, s->hot_keys);
+    if (s->vb == 8) nups_launch_dependent(sync_kernel<true>, grid_for(s->H * (s->L / 4), 256), 256, 0, st, v, s->hot_keys);
+    else nups_launch_dependent(sync_kernel<false>, grid_for(s->H * (s->L / 4), 256), 256, 0, st, v, s->hot_keys);
     cudaError_t e = cudaGetLastError();
     if (e == cudaSuccess) e = cudaMemsetAsync(s->dirty, 0, (size_t)s->R * s->Hcap * sizeof(uint32_t), st);
     nups_background_end(s, st);
