@@ -64,9 +64,9 @@ NCU_TRAFFIC = {"bytes_per_launch": 38886656 + 4509952, "sgns_kernel_sha1": "a667
 # kernel's source text at the time.  The traffic reported for the timed launch is scaled by the algorithmic bytes, which is
 # what the capture shows the traffic follows.  A kernel whose source has changed since reports no traffic.
 NCU_TRAFFIC_PS = {
-    "pull": {"dram_bytes": 216834048 + 481267712, "algorithmic_bytes": 694418688, "sha1": "d6be6ab4363bba8db6eba30551f6fe4750727ba0"},
-    "push": {"dram_bytes": 712477440 + 126427904, "algorithmic_bytes": 847772160, "sha1": "029989f9f74886ae15aab066044712e5cb64b40a"},
-    "sample_rows": {"dram_bytes": 27761408 + 478582016, "algorithmic_bytes": 562094080,
+    "pull": {"dram_bytes": 216757504 + 481016320, "algorithmic_bytes": 694418688, "sha1": "d6be6ab4363bba8db6eba30551f6fe4750727ba0"},
+    "push": {"dram_bytes": 712619776 + 126636032, "algorithmic_bytes": 847772160, "sha1": "0a8c080becb64f3aaf867fbcd3f9c9bc21bc1399"},
+    "sample_rows": {"dram_bytes": 27681024 + 478645504, "algorithmic_bytes": 562094080,
                     "sha1": "d6be6ab4363bba8db6eba30551f6fe4750727ba0"},
 }
 PS_KERNEL_SOURCE = {   # kind -> (kernel name, start and end markers of its source text in store.cu)

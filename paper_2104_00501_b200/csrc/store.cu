@@ -615,7 +615,12 @@ extern "C" nups_status nups_pull(nups_store* s, const uint32_t* d_keys, uint64_t
 // a hot destination receives one reduction per window instead of one per row.
 // TWO = a second table gets its own deltas from the same call.
 // ---------------------------------------------------------------------------------------------
-constexpr int PUSH_UNROLL = 4;
+// Two rows in flight per warp and four resident blocks of 256 threads per multiprocessor (64 registers a thread): measured
+// against four rows and three blocks (80 registers), the extra warps are worth more than the deeper unrolling at every skew
+// (1M keys x 128 floats: 275 vs 279 us at s = 0, 195 vs 199 us at s = 1.0 with 1,000 replicated keys, 138 vs 152 us at s = 1.4).
+constexpr int PUSH_UNROLL = 2;
+constexpr int PUSH_THREADS = 256;
+constexpr int PUSH_BLOCKS = 4;            // one table; calls that update two tables at once keep three (80 registers)
 
 struct PushPair {
     const float4* delta;   // [n][L] updates
@@ -634,7 +639,7 @@ struct PushPair {
 // keys show up early and often, so they take most accumulators, and a skewed batch stops queueing at a few L2
 // addresses even when its frequent keys were never marked for replication.
 template <bool HOT, bool TWO, int TIER, bool F64>
-__global__ void __launch_bounds__(256, 3)
+__global__ void __launch_bounds__(PUSH_THREADS, TWO ? PUSH_BLOCKS - 1 : PUSH_BLOCKS)
 push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPair A, PushPair B, uint64_t n_items,
                    uint32_t rows_per_item, uint32_t tier_rows)
 {
@@ -736,7 +741,7 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
         unsigned singles = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) == 1);
         unsigned multis = __ballot_sync(0xFFFFFFFFu, leader && __popc(grp) > 1);
 
-        // rows that are alone in their window: four at a time
+        // rows that are alone in their window: PUSH_UNROLL at a time
         while (singles) {
             int src[PUSH_UNROLL], tr[PUSH_UNROLL];
             unsigned long long de[PUSH_UNROLL];
@@ -782,7 +787,7 @@ push_atomic_kernel(View v, const uint32_t* __restrict__ keys, uint64_t n, PushPa
                         atomicOr(&touched[tr[u4] >> 5], 1u << (tr[u4] & 31));
             }
         }
-        // destinations hit more than once in the window: sum the members (loads four at a time), one reduction
+        // destinations hit more than once in the window: sum the members (loads PUSH_UNROLL at a time), one reduction
         while (multis) {
             const int ld = __ffs(multis) - 1;
             multis &= multis - 1;
@@ -965,10 +970,10 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
     View v = nups_view(s);
     uint64_t n_items = n / rows_per_item;
     if (!s->cfg.deterministic) {
-        unsigned grid = grid_for(n, 32 * 8, (unsigned)s->sm_count * 3);  // 3 resident blocks per SM, grid-stride
+        const bool two = d_dval && d_dacc;
+        unsigned grid = grid_for(n, PUSH_THREADS, (unsigned)s->sm_count * (two ? PUSH_BLOCKS - 1 : PUSH_BLOCKS));  // resident at once, grid-stride
         PushPair V = {(const float4*)d_dval, s->val, s->dval};
         PushPair C = {(const float4*)d_dacc, s->acc, s->dacc};
-        const bool two = d_dval && d_dacc;
         PushPair A = d_dval ? V : C, B = C;
         // shared-memory tier: single-table calls with replicated keys, enough blocks to give every worker some
         uint32_t tier_rows = 0;
@@ -976,7 +981,7 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
         const bool cache = !s->H && !two && n >= 32768 && s->vb == 4;  // no replicated keys: accumulators as a row cache
         if ((s->H && !two && rows_per_item == 1 && grid >= s->R && n >= 32768 && s->vb == 4) || cache) {
             const size_t row_bytes = (size_t)s->L * 4;
-            size_t budget = 64 * 1024;
+            size_t budget = (size_t)(192 / PUSH_BLOCKS) * 1024;                 // the blocks of a multiprocessor share 192 KB
             const size_t per_row = row_bytes + (cache ? 4 : 0) + 1;    // sums, owner tag, touched bit (rounded up)
             tier_rows = s->cfg.smem_hot_rows ? s->cfg.smem_hot_rows : (uint32_t)(budget / per_row);
             if (tier_rows > budget / per_row) tier_rows = (uint32_t)(budget / per_row);
@@ -993,15 +998,15 @@ nups_status nups_push_with_scratch(nups_store* s, const uint32_t* d_keys, uint64
         }
         nups_time_begin(s, st, NUPS_TIMED_PUSH);
         if (tier_rows && cache) {
-            nups_launch_dependent(push_atomic_kernel<false, false, 2, false>, grid, 256, tier_bytes, st, v, d_keys, n, A, B, n_items, rows_per_item,
+            nups_launch_dependent(push_atomic_kernel<false, false, 2, false>, grid, PUSH_THREADS, tier_bytes, st, v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);
         } else if (tier_rows) {
             grid = grid / s->R * s->R;              // every worker gets the same number of blocks
-            nups_launch_dependent(push_atomic_kernel<true, false, 1, false>, grid, 256, tier_bytes, st, v, d_keys, n, A, B, n_items, rows_per_item,
+            nups_launch_dependent(push_atomic_kernel<true, false, 1, false>, grid, PUSH_THREADS, tier_bytes, st, v, d_keys, n, A, B, n_items, rows_per_item,
                                                                              tier_rows);
         } else {
 #define NUPS_PUSH0(HOT_, TWO_, F64_) \
-    nups_launch_dependent(push_atomic_kernel<HOT_, TWO_, 0, F64_>, grid, 256, 0, st, v, d_keys, n, A, B, n_items, rows_per_item, 0)
+    nups_launch_dependent(push_atomic_kernel<HOT_, TWO_, 0, F64_>, grid, PUSH_THREADS, 0, st, v, d_keys, n, A, B, n_items, rows_per_item, 0)
             if (s->vb == 8) {
                 if (s->H) { if (two) NUPS_PUSH0(true, true, true); else NUPS_PUSH0(true, false, true); }
                 else { if (two) NUPS_PUSH0(false, true, true); else NUPS_PUSH0(false, false, true); }
