@@ -170,3 +170,40 @@ def test_scores_beyond_thirty_are_clamped_like_the_oracles():
     assert abs(lb.item() - lo) <= 1e-5 * abs(lo)
     tables_close(oc, sc, 0)
     tables_close(oc, sc, 1)
+
+
+@pytest.mark.parametrize("deterministic", [True, False])
+def test_calls_see_what_the_streams_earlier_kernels_wrote(deterministic):
+    """The kernels may become resident before the stream's previous kernel has ended (they are launched as programmatic
+    dependents) but wait before they read: keys and update rows written by the caller's kernels just before a call, with
+    no synchronization in between, are the ones the call uses, and a call's results are there for the caller's next kernel."""
+    nk, L, n = 4000, 32, 3000
+    init = inputs.normal_init(nk, L, 0.1, 5)
+    o, s = make_pair(nk, L, R=4, init=init, deterministic=deterministic)
+    hot = np.arange(0, 64, dtype=np.uint32)
+    o.set_management(hot, REPLICATE)
+    s.set_management(dev_keys(hot), REPLICATE)
+    rng = np.random.default_rng(7)
+    k0 = rng.integers(0, nk, n).astype(np.uint32)
+    d0 = rng.standard_normal((n, L)).astype(np.float32)
+    keys = dev_keys(k0)
+    delta = dev_f32(d0)
+    out = torch.empty((n, L), device="cuda")
+    total = torch.zeros((), device="cuda", dtype=torch.float64)
+    want_total = 0.0
+    for it in range(12):
+        keys.copy_((keys.long() * 7 + it) % nk)              # the caller's kernels write keys and rows ...
+        delta.mul_(-0.5).add_(float(it))
+        s.push(keys, delta)                                  # ... which the very next launches read
+        s.pull(keys, out)
+        total += out.double().sum()                          # and the caller's next kernel reads the result
+        k0 = ((k0.astype(np.int64) * 7 + it) % nk).astype(np.uint32)
+        d0 = (d0 * np.float32(-0.5) + np.float32(it)).astype(np.float32)
+        o.push(k0, d0)
+        want_total += float(o.pull(k0).astype(np.float64).sum())
+    if deterministic:
+        tables_equal(o, s)
+        assert abs(total.item() - want_total) <= 1e-9 * max(1.0, abs(want_total))
+    else:                                                    # additions in another order: rounding only
+        tables_close(o, s, rtol=1e-4, atol=1e-4)
+        assert abs(total.item() - want_total) <= 1e-5 * max(1.0, abs(want_total))
