@@ -947,6 +947,47 @@ def run_ps_reference(args):
     }
 
 
+def run_shard_sweep(args, device):
+    """The partitioned table on ONE GPU: 8 shards (every shard its own allocation, wired by address) standing in for 8
+    ranks, 1M-key Zipf batches pulled and pushed through one rank's table.  All shards are local HBM here, so this
+    measures the kernels' addressing, not NVLink: on several GPUs (N - 1) / N of the rows cross the links."""
+    from paper_2104_00501_b200 import binding, sharded
+    hbm_peak, peak_kind = peaks()
+    nk, n_shards, L, N = args.ps_keys, 8, PS_LEN, PS_BATCH
+    tables = [binding.ShardTable(nk, L, n_shards, j) for j in range(n_shards)]
+    sharded.connect_local(tables)
+    t = tables[0]
+    g = torch.Generator(device=device)
+    g.manual_seed(17)
+    delta = torch.randn(N, L, device=device, generator=g)
+    out = torch.empty(N, L, device=device)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for skew in [float(x) for x in args.ps_skews.split(",")]:
+        cdf = inputs.zipf_cdf(nk, skew, device) if skew > 0 else None
+        batches = [inputs.zipf_keys(N, nk, skew, 100 + i, device, cdf=cdf).to(torch.int32).contiguous() for i in range(4)]
+        del cdf
+        ucold = float(np.mean([torch.unique(b.long()).numel() for b in batches]))
+        line = {"workload": "partitioned table, 8 shards on one GPU: %d keys x %d fp32, 1M-key batches ~ Zipf(%.1f)" % (nk, L, skew),
+                "zipf_s": skew, "distinct_rows": ucold, "peak_kind": peak_kind}
+        for kind, call in (("pull", lambda b: t.pull(b, out)), ("push", lambda b: t.push(b, delta))):
+            for b in batches:
+                call(b)
+            torch.cuda.synchronize()
+            reps = 20
+            e0.record()
+            for r in range(reps):
+                call(batches[r % 4])
+            e1.record()
+            torch.cuda.synchronize()
+            us = e0.elapsed_time(e1) * 1e3 / reps
+            alg = 4 * N + L * 4 * N + (1 if kind == "pull" else 2) * L * 4 * ucold
+            line[kind] = {"us": us, "keys_per_s": N / us * 1e6, "algorithmic_gbs": alg / us / 1e3, "frac": alg / us / 1e3 / hbm_peak}
+        assert t.status_check() == 0
+        print(json.dumps(line), flush=True)
+    for x in tables:
+        x.close()
+
+
 def run_staleness_sweep(args, device):
     """The SGNS workload with replicas merged by step count (every 16 batches) or by time: throughput and loss after
     the same number of steps from the same start values.  The periods span the paper's staleness experiment (125, 25
@@ -1083,7 +1124,7 @@ def main():
     ap.add_argument("--no-sweep", action="store_true", help="default line only: skip the sweep of the other grid points")
     ap.add_argument("--min-timed-ms", type=float, default=1000.0,
                     help="the timed region repeats the K steps until it is at least this long (at least 5 times)")
-    ap.add_argument("--workload", default="psline", choices=["psline", "sgns", "ps", "sample", "kge", "mf", "staleness"],
+    ap.add_argument("--workload", default="psline", choices=["psline", "sgns", "ps", "sample", "kge", "mf", "staleness", "shard"],
                     help="psline (default): the parameter-server microbenchmark line with its sweep; sgns: the skip-gram line; "
                          "the others print their own lines")
     ap.add_argument("--hot-fraction", type=float, default=HOT_FRACTION, help="share of keys to replicate (default 0.01)")
@@ -1126,6 +1167,9 @@ def main():
         return
     if args.workload == "staleness":
         run_staleness_sweep(args, device)
+        return
+    if args.workload == "shard":
+        run_shard_sweep(args, device)
         return
     if world > 1:
         torch.distributed.init_process_group("nccl", device_id=device)

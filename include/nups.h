@@ -385,6 +385,56 @@ nups_status nups_kernel_times(nups_store* store, double* h_ms_out, uint64_t* h_l
  * in fast mode.  Synchronises the stream.                                      */
 nups_status nups_probe_reduction_rate(nups_store* store, uint64_t bytes, uint32_t reps, double* h_gbs_out, void* stream);
 
+/* ---------------------------------------------------------------------------
+ * A value table partitioned over several GPUs (Section 3.1: the servers of a
+ * parameter server hold disjoint parts of the parameters, classically by key
+ * range; Section 3.2: a worker reaches a parameter held elsewhere through that
+ * node).  Among GPUs of one NVLink domain the owner's memory is addressable, so
+ * the access is made by the calling GPU's own kernel: pull loads the row from
+ * the owner's memory, push adds to it there with floating-point reductions.
+ * No message, no exchange of keys, no work on the owner.
+ *
+ * Shard j holds the fp32 rows of keys [j * kps, (j + 1) * kps), kps =
+ * ceil(num_keys / n_shards).  Every process creates one object for its own
+ * shard (my_shard), which allocates and zero-fills that shard on the current
+ * device, and attaches the first-row address of every other shard:
+ *   - a pointer valid in this process (a shard of another object of the same
+ *     process; for another device the caller has enabled peer access), or
+ *   - the handle another process exported for its shard (CUDA IPC; peer access
+ *     is enabled by the mapping).
+ * Handles are plain bytes: ship them with whatever the processes use to talk
+ * (torch.distributed, a file).  An attached shard must outlive the attachment.
+ * Values are fp32; keys out of range are skipped as in the store (a pulled row
+ * is zero-filled, nups_shard_status_check reports NUPS_EKEY).  Not replicated:
+ * keys hot enough to be replicated belong in a per-GPU nups_store.
+ * Ordering: calls are stream-ordered on the calling GPU only.  Updates pushed
+ * by another GPU are seen by a pull that is ordered after them by the caller's
+ * own means (an event, a barrier between processes); additions to one row from
+ * several GPUs at once all arrive, in no defined order.
+ * nups_shard_pull / nups_shard_push return NUPS_ESTATE until every shard is
+ * attached.  Errors of the CUDA runtime: NUPS_ECUDA, text from
+ * nups_shard_last_error.                                                      */
+typedef struct nups_shard_table nups_shard_table;
+#define NUPS_MAX_SHARDS 16
+#define NUPS_SHARD_HANDLE_BYTES 64
+nups_status nups_shard_table_create(uint64_t num_keys, uint32_t value_len, uint32_t n_shards, uint32_t my_shard,
+                                    nups_shard_table** out);
+void nups_shard_table_destroy(nups_shard_table* table);
+/* device address and size in bytes of this process's shard (for same-process attachment and for filling it) */
+nups_status nups_shard_table_local(nups_shard_table* table, void** h_ptr_out, uint64_t* h_bytes_out);
+/* whole-shard copy between the local shard and a device buffer of kps * value_len floats (to_table != 0: into the shard) */
+nups_status nups_shard_table_copy(nups_shard_table* table, void* d_rows, int to_table, void* stream);
+/* handle of the local shard for another process: NUPS_SHARD_HANDLE_BYTES bytes written to h_handle_out */
+nups_status nups_shard_table_export(nups_shard_table* table, unsigned char* h_handle_out);
+nups_status nups_shard_table_attach(nups_shard_table* table, uint32_t shard, void* d_first_row);
+nups_status nups_shard_table_attach_ipc(nups_shard_table* table, uint32_t shard, const unsigned char* h_handle);
+/* d_out / d_delta: [n][value_len] fp32, 16-byte aligned, on the calling GPU */
+nups_status nups_shard_pull(nups_shard_table* table, const uint32_t* d_keys, uint64_t n, void* d_out, void* stream);
+nups_status nups_shard_push(nups_shard_table* table, const uint32_t* d_keys, uint64_t n, const void* d_delta, void* stream);
+/* synchronises the stream; NUPS_EKEY once after a key out of range was seen */
+nups_status nups_shard_status_check(nups_shard_table* table, void* stream);
+const char* nups_shard_last_error(const nups_shard_table* table);
+
 const char* nups_strerror(nups_status status);
 const char* nups_last_cuda_error(void);
 

@@ -26,6 +26,9 @@ EXPORTS = [
     "nups_get_hot", "nups_localize", "nups_get_owner", "nups_register_distribution", "nups_get_alias_table",
     "nups_prepare_sample", "nups_pull_sample", "nups_step_sgns", "nups_run_sgns", "nups_step_complex", "nups_step_mf", "nups_step_mf_by_column",
     "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_kernel_times", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_get_clip_stats", "nups_strerror", "nups_last_cuda_error",
+    "nups_shard_table_create", "nups_shard_table_destroy", "nups_shard_table_local", "nups_shard_table_copy", "nups_shard_table_export",
+    "nups_shard_table_attach", "nups_shard_table_attach_ipc", "nups_shard_pull", "nups_shard_push", "nups_shard_status_check",
+    "nups_shard_last_error",
 ]
 
 
@@ -99,12 +102,23 @@ def load(build_if_missing: bool = True):
         "nups_probe_reduction_rate": [vp, u64, u32, C.POINTER(C.c_double), vp],
         "nups_set_sync_period": [vp, u32],
         "nups_get_clip_stats": [vp, C.POINTER(C.c_double), C.POINTER(u64), vp],
+        "nups_shard_table_create": [u64, u32, u32, u32, C.POINTER(vp)],
+        "nups_shard_table_local": [vp, C.POINTER(vp), C.POINTER(u64)],
+        "nups_shard_table_copy": [vp, vp, C.c_int, vp],
+        "nups_shard_table_export": [vp, C.c_char_p],
+        "nups_shard_table_attach": [vp, u32, vp],
+        "nups_shard_table_attach_ipc": [vp, u32, C.c_char_p],
+        "nups_shard_pull": [vp, vp, u64, vp, vp],
+        "nups_shard_push": [vp, vp, u64, vp, vp],
+        "nups_shard_status_check": [vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
         fn.restype, fn.argtypes = C.c_int32, args
     L.nups_strerror.restype, L.nups_strerror.argtypes = C.c_char_p, [C.c_int32]
     L.nups_last_cuda_error.restype, L.nups_last_cuda_error.argtypes = C.c_char_p, []
+    L.nups_shard_last_error.restype, L.nups_shard_last_error.argtypes = C.c_char_p, [vp]
+    L.nups_shard_table_destroy.restype, L.nups_shard_table_destroy.argtypes = None, [vp]
     _lib = L
     return L
 
@@ -378,3 +392,85 @@ class Store:
     def set_sync_period(self, period_us):
         """Background merging of the replicas every `period_us` microseconds; 0 stops it."""
         self._chk(self._l.nups_set_sync_period(self._s, period_us), "nups_set_sync_period")
+
+
+MAX_SHARDS = 16
+SHARD_HANDLE_BYTES = 64
+
+
+class ShardTable:
+    """This process's part of a value table partitioned over several GPUs by key range; every shard is reached through
+    peer memory by the calling GPU's own kernels (marshalling only: see `nups_shard_*` in include/nups.h)."""
+
+    def __init__(self, num_keys, value_len, n_shards, my_shard):
+        self._l = load()
+        self.num_keys, self.L, self.n_shards, self.my_shard = num_keys, value_len, n_shards, my_shard
+        self.keys_per_shard = -(-num_keys // n_shards)
+        self.device = torch.device("cuda", torch.cuda.current_device())
+        h = C.c_void_p()
+        self._t = None
+        self._chk(self._l.nups_shard_table_create(num_keys, value_len, n_shards, my_shard, C.byref(h)), "nups_shard_table_create")
+        self._t = h
+
+    def _chk(self, rc, what):
+        if rc != 0:
+            detail = self._l.nups_strerror(rc).decode()
+            if self._t is not None and rc == ECUDA:
+                detail += ": " + self._l.nups_shard_last_error(self._t).decode()
+            raise NupsError(rc, what, detail)
+
+    def close(self):
+        if self._t is not None:
+            self._l.nups_shard_table_destroy(self._t)
+            self._t = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def local_address(self):
+        p, n = C.c_void_p(), C.c_uint64()
+        self._chk(self._l.nups_shard_table_local(self._t, C.byref(p), C.byref(n)), "nups_shard_table_local")
+        return p.value, n.value
+
+    def write_local(self, rows):
+        """Fill the local shard from [keys_per_shard, value_len] fp32 values (host or device)."""
+        t = torch.as_tensor(rows, dtype=torch.float32).to(self.device).contiguous()
+        assert t.numel() == self.keys_per_shard * self.L
+        self._chk(self._l.nups_shard_table_copy(self._t, _ptr(t), 1, _stream()), "nups_shard_table_copy")
+        torch.cuda.current_stream().synchronize()
+
+    def read_local(self):
+        out = torch.empty((self.keys_per_shard, self.L), dtype=torch.float32, device=self.device)
+        self._chk(self._l.nups_shard_table_copy(self._t, _ptr(out), 0, _stream()), "nups_shard_table_copy")
+        torch.cuda.current_stream().synchronize()
+        return out
+
+    def export_handle(self) -> bytes:
+        buf = C.create_string_buffer(SHARD_HANDLE_BYTES)
+        self._chk(self._l.nups_shard_table_export(self._t, buf), "nups_shard_table_export")
+        return buf.raw
+
+    def attach(self, shard, address):
+        self._chk(self._l.nups_shard_table_attach(self._t, shard, C.c_void_p(address)), "nups_shard_table_attach")
+
+    def attach_handle(self, shard, handle: bytes):
+        assert len(handle) == SHARD_HANDLE_BYTES
+        self._chk(self._l.nups_shard_table_attach_ipc(self._t, shard, handle), "nups_shard_table_attach_ipc")
+
+    def pull(self, keys, out=None):
+        n = keys.numel()
+        if out is None:
+            out = torch.empty((n, self.L), dtype=torch.float32, device=self.device)
+        self._chk(self._l.nups_shard_pull(self._t, _ptr(keys, torch.int32), n, _ptr(out, torch.float32), _stream()), "nups_shard_pull")
+        return out
+
+    def push(self, keys, delta):
+        n = keys.numel()
+        assert delta.dtype == torch.float32 and delta.numel() == n * self.L
+        self._chk(self._l.nups_shard_push(self._t, _ptr(keys, torch.int32), n, _ptr(delta), _stream()), "nups_shard_push")
+
+    def status_check(self):
+        return self._l.nups_shard_status_check(self._t, _stream())

@@ -10,7 +10,7 @@ from concurrent.futures import ThreadPoolExecutor
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libnups.so")
-SOURCES = ["store.cu", "primitives.cu", "sampling.cu", "steps.cu", "noalloc.cu", "background.cu"]
+SOURCES = ["store.cu", "primitives.cu", "sampling.cu", "steps.cu", "noalloc.cu", "background.cu", "shard.cu"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]
 
