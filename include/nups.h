@@ -365,7 +365,11 @@ nups_status nups_get_stats(nups_store* store, uint64_t* h_out, void* stream);
 /* Timing aid for benchmarks.  While enabled, the library records a pair of CUDA
  * events on the call's stream around the main kernel of nups_pull*, nups_push*
  * (fast mode) and nups_step_* (the row gather, the scatter-add, the fused step
- * kernel).  nups_kernel_time synchronises the stream, adds up the elapsed
+ * kernel).  nups_kernel_timing only switches the recording on or off (no
+ * synchronisation; pairs already recorded stay until they are queried), so a
+ * caller can time some repetitions of a loop and leave the others undisturbed:
+ * an event between two kernels keeps the second from starting while the first
+ * drains.  nups_kernel_time synchronises the stream, adds up the elapsed
  * times of all pairs recorded since the last query, returns the sum in
  * milliseconds and the number of launches, and starts afresh.                 */
 nups_status nups_kernel_timing(nups_store* store, int enable);

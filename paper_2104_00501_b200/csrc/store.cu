@@ -146,9 +146,7 @@ extern "C" nups_status nups_kernel_timing(nups_store* s, int enable)
         if (!s->ev || !s->ev_kind) return NUPS_ENOMEM;
         for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) CK(cudaEventCreate(&s->ev[i]));
     }
-    if (s->ev) timing_fold(s);
-    timing_clear(s);
-    s->timing = enable ? 1 : 0;
+    s->timing = enable ? 1 : 0;       // what was recorded stays until it is queried: switching costs no synchronisation
     return NUPS_OK;
 }
 extern "C" nups_status nups_kernel_times(nups_store* s, double* h_ms_out, uint64_t* h_launches_out, void* stream)
