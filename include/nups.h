@@ -439,6 +439,27 @@ nups_status nups_shard_push(nups_shard_table* table, const uint32_t* d_keys, uin
 nups_status nups_shard_status_check(nups_shard_table* table, void* stream);
 const char* nups_shard_last_error(const nups_shard_table* table);
 
+/* Merging a whole store across GPUs (Section 3.2: replicas are synchronised by
+ * an all-reduce of the updates they have accumulated).  Use: every GPU holds a
+ * nups_store of the same keys (the keys replicated across GPUs: a small store)
+ * and pulls and pushes it on its own.  `which` = 0 value table, 1 accumulator.
+ *   nups_merge_mark    all GPUs hold the same table now (after the same
+ *                      initialisation): remember it as the agreed state.
+ *                      Allocates num_keys rows (NUPS_ENOMEM under the limit).
+ *   nups_merge_export  merges the store's own replicas (nups_sync), then writes
+ *                      own = table - agreed into d_own_out ([num_keys][value_len],
+ *                      the store's value type).  NUPS_ESTATE before a mark.
+ *   (the caller sums the exported buffers over all GPUs into d_total: one
+ *    all-reduce with NCCL or any other transport; d_own must keep its content)
+ *   nups_merge_apply   table += d_total - d_own (by reductions, so pushes may
+ *                      run beside it), agreed += d_total.
+ * Afterwards every GPU's table is the agreed state plus what that GPU added
+ * since its export; nothing pushed between export and apply is lost.  With one
+ * GPU (d_total = d_own) the table is unchanged.                               */
+nups_status nups_merge_mark(nups_store* store, int which, void* stream);
+nups_status nups_merge_export(nups_store* store, int which, void* d_own_out, void* stream);
+nups_status nups_merge_apply(nups_store* store, int which, const void* d_total, const void* d_own, void* stream);
+
 const char* nups_strerror(nups_status status);
 const char* nups_last_cuda_error(void);
 

@@ -28,7 +28,7 @@ EXPORTS = [
     "nups_last_negatives", "nups_status_check", "nups_get_stats", "nups_kernel_timing", "nups_kernel_time", "nups_kernel_times", "nups_probe_reduction_rate", "nups_set_sync_period", "nups_get_clip_stats", "nups_strerror", "nups_last_cuda_error",
     "nups_shard_table_create", "nups_shard_table_destroy", "nups_shard_table_local", "nups_shard_table_copy", "nups_shard_table_export",
     "nups_shard_table_attach", "nups_shard_table_attach_ipc", "nups_shard_pull", "nups_shard_push", "nups_shard_status_check",
-    "nups_shard_last_error",
+    "nups_shard_last_error", "nups_merge_mark", "nups_merge_export", "nups_merge_apply",
 ]
 
 
@@ -111,6 +111,9 @@ def load(build_if_missing: bool = True):
         "nups_shard_pull": [vp, vp, u64, vp, vp],
         "nups_shard_push": [vp, vp, u64, vp, vp],
         "nups_shard_status_check": [vp, vp],
+        "nups_merge_mark": [vp, C.c_int, vp],
+        "nups_merge_export": [vp, C.c_int, vp, vp],
+        "nups_merge_apply": [vp, C.c_int, vp, vp, vp],
     }
     for name, args in sig.items():
         fn = getattr(L, name)
@@ -388,6 +391,22 @@ class Store:
         sm, cnt = C.c_double(0), C.c_uint64(0)
         self._chk(self._l.nups_get_clip_stats(self._s, C.byref(sm), C.byref(cnt), _stream()), "nups_get_clip_stats")
         return sm.value, cnt.value
+
+    def merge_mark(self, which=0):
+        """All GPUs hold the same table now: the agreed state that merges across GPUs start from."""
+        self._chk(self._l.nups_merge_mark(self._s, which, _stream()), "nups_merge_mark")
+
+    def merge_export(self, which=0, out=None):
+        """This GPU's additions since the agreed state, [num_keys, value_len] (its own replicas merged first)."""
+        if out is None:
+            out = torch.empty((self.num_keys, self.L), dtype=self.dtype, device=self.device)
+        self._chk(self._l.nups_merge_export(self._s, which, _ptr(out), _stream()), "nups_merge_export")
+        return out
+
+    def merge_apply(self, total, own, which=0):
+        """Take over the other GPUs' additions: `total` = sum of every GPU's export, `own` = this GPU's."""
+        assert total.dtype == self.dtype and own.dtype == self.dtype and total.numel() == own.numel() == self.num_keys * self.L
+        self._chk(self._l.nups_merge_apply(self._s, which, _ptr(total), _ptr(own), _stream()), "nups_merge_apply")
 
     def set_sync_period(self, period_us):
         """Background merging of the replicas every `period_us` microseconds; 0 stops it."""

@@ -122,6 +122,7 @@ struct nups_store {
     cudaStream_t side;          // nups_run_sgns: a due replica merge runs here, beside the next steps' sample draw
     cudaEvent_t side_fork, side_join;
     bool push_smem_opted, complex_smem_opted[2][2][2][2];   // large dynamic shared memory asked for on this store's device
+    float* merge_snap[2];       // merging across GPUs (shard.cu): each table as all GPUs last agreed on it; NULL = never marked
     Dist dist[NUPS_MAX_DISTS];
     Handle handle[NUPS_MAX_HANDLES];
 };

@@ -335,3 +335,86 @@ extern "C" nups_status nups_shard_status_check(nups_shard_table* t, void* stream
     }
     return NUPS_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// Merging a replicated store across GPUs (Section 3.2: replicas are synchronised by an all-reduce of their accumulated
+// updates).  Every GPU keeps a whole nups_store of the keys that are replicated across GPUs (a small one: the hot keys)
+// and updates it on its own.  `snap` is the table as all GPUs last agreed on it.  A merge is three steps: every GPU
+// exports own = table - snap (after merging its own workers' replicas into the table); the caller adds the exported
+// buffers up over all GPUs (one all-reduce); every GPU applies table += total - own and snap += total.  Afterwards all
+// tables are the agreed values plus whatever each GPU added since its export, which the next merge carries over:
+// nothing that arrives between export and apply is lost, and the additions to the table are reductions, so pushes may
+// run beside them.
+// ---------------------------------------------------------------------------------------------
+template <class T>
+__global__ void merge_export_kernel(const T* __restrict__ table, const T* __restrict__ snap, T* __restrict__ own, uint64_t n)
+{
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x)
+        own[i] = table[i] - snap[i];
+}
+
+template <class T>
+__global__ void merge_apply_kernel(T* table, T* __restrict__ snap, const T* __restrict__ total, const T* __restrict__ own,
+                                   uint64_t n)
+{
+    for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (uint64_t)gridDim.x * blockDim.x) {
+        const T t = total[i], others = t - own[i];
+        if (others != T(0)) atomicAdd(table + i, others);
+        snap[i] += t;
+    }
+}
+
+static bool merge_args_ok(const nups_store* s, int which)
+{
+    return s && (which == 0 || which == 1) && (which == 0 || s->acc);
+}
+
+extern "C" nups_status nups_merge_mark(nups_store* s, int which, void* stream)
+{
+    if (!merge_args_ok(s, which)) return NUPS_EINVAL;
+    const size_t bytes = (size_t)s->num_keys * s->L * sizeof(float);
+    if (!s->merge_snap[which]) {
+        nups_status rc = nups_dev_alloc(s, (void**)&s->merge_snap[which], bytes);
+        if (rc != NUPS_OK) return rc;
+    }
+    nups_status rc = nups_sync_internal(s, (cudaStream_t)stream);           // the workers' replicas belong to the table
+    if (rc != NUPS_OK) return rc;
+    CK(cudaMemcpyAsync(s->merge_snap[which], which ? s->acc : s->val, bytes, cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_merge_export(nups_store* s, int which, void* d_own_out, void* stream)
+{
+    if (!merge_args_ok(s, which) || !d_own_out) return NUPS_EINVAL;
+    if (!s->merge_snap[which]) return NUPS_ESTATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    nups_status rc = nups_sync_internal(s, st);
+    if (rc != NUPS_OK) return rc;
+    const uint64_t words = (uint64_t)s->num_keys * s->L;
+    const void* table = which ? s->acc : s->val;
+    if (s->vb == 8)
+        merge_export_kernel<double><<<grid_for(words / 2, 256, (unsigned)s->sm_count * 8), 256, 0, st>>>(
+            (const double*)table, (const double*)s->merge_snap[which], (double*)d_own_out, words / 2);
+    else
+        merge_export_kernel<float><<<grid_for(words, 256, (unsigned)s->sm_count * 8), 256, 0, st>>>(
+            (const float*)table, s->merge_snap[which], (float*)d_own_out, words);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}
+
+extern "C" nups_status nups_merge_apply(nups_store* s, int which, const void* d_total, const void* d_own, void* stream)
+{
+    if (!merge_args_ok(s, which) || !d_total || !d_own) return NUPS_EINVAL;
+    if (!s->merge_snap[which]) return NUPS_ESTATE;
+    cudaStream_t st = (cudaStream_t)stream;
+    const uint64_t words = (uint64_t)s->num_keys * s->L;
+    void* table = which ? s->acc : s->val;
+    if (s->vb == 8)
+        merge_apply_kernel<double><<<grid_for(words / 2, 256, (unsigned)s->sm_count * 8), 256, 0, st>>>(
+            (double*)table, (double*)s->merge_snap[which], (const double*)d_total, (const double*)d_own, words / 2);
+    else
+        merge_apply_kernel<float><<<grid_for(words, 256, (unsigned)s->sm_count * 8), 256, 0, st>>>(
+            (float*)table, s->merge_snap[which], (const float*)d_total, (const float*)d_own, words);
+    LAUNCH_CHECK(s);
+    return NUPS_OK;
+}

@@ -273,6 +273,7 @@ extern "C" nups_status nups_destroy(nups_store* s)
     cudaFree(s->val); cudaFree(s->acc); cudaFree(s->hot_bits); cudaFree(s->slot_of); cudaFree(s->hot_keys);
     cudaFree(s->dval); cudaFree(s->dacc); cudaFree(s->dirty); cudaFree(s->cnt); cudaFree(s->own);
     cudaFree(s->st); cudaFree(s->loss_partial); cudaFree(s->scratch); cudaFree(s->negs_buf);
+    cudaFree(s->merge_snap[0]); cudaFree(s->merge_snap[1]);
     if (s->ev) {
         for (int i = 0; i < 2 * NUPS_MAX_TIMED; ++i) cudaEventDestroy(s->ev[i]);
         free(s->ev);

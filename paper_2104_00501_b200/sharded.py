@@ -53,3 +53,19 @@ def connect_process_group(table, group=None) -> None:
         if k != rank:
             table.attach_handle(k, h)
     dist.barrier(group)
+
+
+def merge_across_ranks(store, group=None, which=0) -> None:
+    """Merge a store that every rank holds a copy of (the keys replicated across GPUs; Section 3.2's replica
+    synchronisation): every rank exports what it added since the ranks last agreed, one all-reduce sums the exports, every
+    rank takes over the others' part.  The sum is NCCL's on GPUs; under any other backend (two test processes on one GPU,
+    which NCCL does not serve) the buffer goes through host memory."""
+    own = store.merge_export(which)
+    total = own.clone()
+    if dist.get_backend(group) == "nccl":
+        dist.all_reduce(total, group=group)
+    else:
+        host = total.cpu()
+        dist.all_reduce(host, group=group)
+        total.copy_(host)
+    store.merge_apply(total, own, which)

@@ -120,6 +120,66 @@ def test_keys_out_of_range_unattached_shards_and_empty_calls():
         assert e.value.code == binding.EINVAL
 
 
+def test_stores_of_two_ranks_merge_to_the_oracles_single_store():
+    """Two stores (two GPUs' copies of the keys replicated across GPUs), each with its own workers' replicas, updated
+    apart and merged: both end up as the oracle's one store that took all the updates.  Values are small integers, so
+    that sums are exact in any order; the sum of the two exports stands for the all-reduce."""
+    from oracle import REPLICATE
+    nk, L, n = 300, 16, 4000
+    rng = np.random.default_rng(21)
+    init = rng.integers(-9, 10, (nk, L)).astype(np.float32)
+    o = Oracle(nk, L, workers=4)
+    o.table(0)[:] = init
+    stores = [binding.Store(nk, L, workers=4, deterministic=False) for _ in range(2)]
+    hot = np.arange(0, 40, dtype=np.uint32)
+    o.set_management(hot, REPLICATE)
+    for s in stores:
+        s.write_table(0, init)
+        s.set_management(dev_keys(hot), REPLICATE)
+        with pytest.raises(binding.NupsError) as e:
+            s.merge_export()
+        assert e.value.code == binding.ESTATE                      # nothing agreed on yet
+        s.merge_mark()
+    for rnd in range(3):
+        late = []
+        for s in stores:
+            k = (rng.zipf(1.2, n) % nk).astype(np.uint32)
+            d = rng.integers(-2, 3, (n, L)).astype(np.float32)
+            s.push(dev_keys(k), dev_f32(d))
+            o.push(k, d)
+        owns = [s.merge_export() for s in stores]
+        total = owns[0] + owns[1]
+        for s in stores:                                           # updates that arrive between export and apply
+            k = rng.integers(0, nk, 50).astype(np.uint32)
+            d = rng.integers(-2, 3, (50, L)).astype(np.float32)
+            s.push(dev_keys(k), dev_f32(d))
+            late.append((k, d))
+        for s, own in zip(stores, owns):
+            s.merge_apply(total, own)
+        o.sync()
+        if rnd < 2:
+            # the late updates are still each store's own: the next round carries them over
+            for k, d in late:
+                o.push(k, d)
+            continue
+        # last round: merge once more so that the late updates are shared too
+        for k, d in late:
+            o.push(k, d)
+        owns = [s.merge_export() for s in stores]
+        total = owns[0] + owns[1]
+        for s, own in zip(stores, owns):
+            s.merge_apply(total, own)
+        o.sync()
+    for s in stores:
+        s.sync()
+        assert np.array_equal(s.read_table(0).cpu().numpy(), o.table(0))
+    # one rank alone: total = own leaves the table as it is
+    before = stores[0].read_table(0).clone()
+    own = stores[0].merge_export()
+    stores[0].merge_apply(own.clone(), own)
+    assert torch.equal(stores[0].read_table(0), before)
+
+
 def _process(rank, world, port, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     sys.path.insert(0, ROOT)
@@ -152,6 +212,24 @@ def _process(rank, world, port, out):
     ok = bool(np.array_equal(got, o.pull(every))) and t.status_check() == B.OK
     dist.barrier()                                                 # nobody unmaps while the other still reads
     t.close()
+    # a store that both processes hold (the keys replicated across GPUs), updated apart, merged over the process group
+    hk, hL = 64, 8
+    hinit = np.random.default_rng(1).integers(-5, 6, (hk, hL)).astype(np.float32)
+    ho = O(hk, hL, workers=1)
+    ho.table(0)[:] = hinit
+    hs = B.Store(hk, hL, workers=2, deterministic=False)
+    hs.write_table(0, hinit)
+    hs.merge_mark()
+    for rnd in range(2):
+        for r in range(world):
+            kk = np.random.default_rng(100 + 10 * rnd + r).integers(0, hk, 500).astype(np.uint32)
+            dd = np.random.default_rng(200 + 10 * rnd + r).integers(-2, 3, (500, hL)).astype(np.float32)
+            if r == rank:
+                hs.push(torch.from_numpy(kk.view(np.int32)).cuda(), torch.from_numpy(dd).cuda())
+            ho.push(kk, dd)
+        S.merge_across_ranks(hs)
+    ok = ok and bool(np.array_equal(hs.read_table(0).cpu().numpy(), ho.table(0)))
+    hs.close()
     out.put((rank, ok))
     dist.destroy_process_group()
 

@@ -59,6 +59,24 @@ class FileShards:
             m.flush()
 
 
+class HostStore:
+    """Stand-in for the merge calls of `binding.Store`: the same three-step protocol in numpy (the arithmetic of the
+    real calls is checked against the oracle on the GPU; here it is the exchange between ranks that is under test)."""
+
+    def __init__(self, init):
+        import torch
+        self.torch = torch
+        self.table = init.copy()
+        self.snap = init.copy()
+
+    def merge_export(self, which=0):
+        return self.torch.from_numpy(self.table - self.snap)
+
+    def merge_apply(self, total, own, which=0):
+        self.table += (total - own).numpy()
+        self.snap += total.numpy()
+
+
 def _rank(rank, world, port, folder, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     sys.path.insert(0, ROOT)
@@ -93,6 +111,20 @@ def _rank(rank, world, port, folder, out):
         every = np.arange(num_keys, dtype=np.uint32)
         ok = ok and np.array_equal(t.pull(every), o.pull(every))
         dist.barrier()
+    # a store that every rank holds, updated apart and merged over the group: every rank ends up with the oracle's table
+    hinit = np.random.default_rng(2).integers(-5, 6, (20, L)).astype(np.float32)
+    ho = Oracle(20, L, workers=1)
+    ho.table(0)[:] = hinit
+    hs = HostStore(hinit)
+    for rnd in range(3):
+        for r in range(world):
+            kk = np.random.default_rng(60 + 10 * rnd + r).integers(0, 20, 30).astype(np.uint32)
+            dd = np.random.default_rng(70 + 10 * rnd + r).integers(-3, 4, (30, L)).astype(np.float32)
+            if r == rank:
+                np.add.at(hs.table, kk, dd)
+            ho.push(kk, dd)
+        sharded.merge_across_ranks(hs)
+        ok = ok and np.array_equal(hs.table, ho.table(0)) and np.array_equal(hs.snap, ho.table(0))
     right = [t.attached[k] == os.path.join(folder, f"s{k}").encode().ljust(64, b"\0") for k in sorted(t.attached)]
     out.put((rank, sorted(t.attached), right, refused, bool(ok)))
     dist.destroy_process_group()
