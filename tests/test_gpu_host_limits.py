@@ -47,6 +47,11 @@ def test_every_allocating_call_respects_the_stores_limit_and_leaves_the_store_us
     _enomem(lambda: s.step_sgns(c, c, d, 3, 0.1))
     s.step_sgns(c[:100].contiguous(), c[:100].contiguous(), d, 3, 0.1)
     assert s.status_check() == 0
+    # the agreed copy of the table that merging across GPUs keeps (another 3.2 MB) does not fit either
+    _enomem(lambda: s.merge_mark())
+    with pytest.raises(binding.NupsError) as e:
+        s.merge_export()
+    assert e.value.code == binding.ESTATE
     s.close()
     # without a limit the same calls succeed
     s = binding.Store(nk, L, workers=R, deterministic=True, track_ownership=True)
